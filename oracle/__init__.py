@@ -1,0 +1,287 @@
+"""CPU checker for the lazy-message-passing hot path (test infrastructure).
+
+Thin ctypes wrappers over `retexo_oracle.c` plus the K-round training loop of
+Section 3.1 written out in Python (`lmp_train`).  Only the tests, the smoke
+check and the benchmark's CPU-baseline leg use this package; the CUDA library
+neither imports nor links it.
+
+Parity status: pinned by tests/test_oracle_*.py.  Agreement with the paper's
+printed accuracy / timing tables needs the public datasets: parity unpinned.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "retexo_oracle.c")
+_LIB = os.path.join(_HERE, "libretexo_oracle.so")
+_lib = None
+
+GCN, SAGE_MEAN, GAT = 0, 1, 2
+SGD, ADAM = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the checker with gcc (-O2, OpenMP)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.oracle_theta_size.restype = C.c_int64
+        _lib.oracle_bf16_round.restype = C.c_float
+        _lib.oracle_bf16_round.argtypes = [C.c_float]
+    return _lib
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _f32(a):
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise RuntimeError("%s failed with oracle status %d" % (what, rc))
+
+
+def n_threads() -> int:
+    return int(os.environ.get("OMP_NUM_THREADS", os.cpu_count() or 1))
+
+
+def bf16_round(a: np.ndarray) -> np.ndarray:
+    """Round fp32 values to the nearest bf16 (ties to even), returned as fp32."""
+    a = _f32(a)
+    f = lib().oracle_bf16_round
+    return np.array([f(float(v)) for v in a.ravel()], dtype=np.float32).reshape(a.shape)
+
+
+# ---------------------------------------------------------------- aggregation
+def aggregate(aggr: int, rowptr: np.ndarray, colidx: np.ndarray, q: np.ndarray,
+              rows: Optional[np.ndarray] = None, gat: Optional[Dict] = None,
+              return_alpha: bool = False):
+    """AGGR (+ COMBINE) of Eq. 1 for all nodes, or for the listed `rows`.
+
+    GCN -> [n, d]; SAGE_MEAN -> [n, 2d] (self | mean); GAT -> [n, heads*dh]
+    (q is the projected input; gat = dict(heads, head_dim, a_src, a_dst,
+    negative_slope, add_self_loop))."""
+    n = rowptr.shape[0] - 1
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+    colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+    q = _f32(q)
+    dim = q.shape[1]
+    rows_a = None if rows is None else np.ascontiguousarray(rows, dtype=np.int64)
+    cnt = n if rows is None else rows_a.shape[0]
+    L = lib()
+    if aggr == GCN:
+        out = np.zeros((cnt, dim), dtype=np.float32)
+        rc = L.oracle_aggregate_gcn(C.c_int64(n), _p(rowptr), _p(colidx), _p(q), C.c_int64(q.shape[1]),
+                                    C.c_int32(dim), _p(out), C.c_int64(dim), _p(rows_a), C.c_int64(cnt))
+        _check(rc, "oracle_aggregate_gcn")
+        return out
+    if aggr == SAGE_MEAN:
+        out = np.zeros((cnt, 2 * dim), dtype=np.float32)
+        rc = L.oracle_aggregate_sage_mean(C.c_int64(n), _p(rowptr), _p(colidx), _p(q), C.c_int64(q.shape[1]),
+                                          C.c_int32(dim), _p(out), C.c_int64(2 * dim), _p(rows_a),
+                                          C.c_int64(cnt))
+        _check(rc, "oracle_aggregate_sage_mean")
+        return out
+    if aggr == GAT:
+        heads, dh = int(gat["heads"]), int(gat["head_dim"])
+        assert heads * dh == dim
+        a_src, a_dst = _f32(gat["a_src"]), _f32(gat["a_dst"])
+        out = np.zeros((cnt, dim), dtype=np.float32)
+        ae = aself = None
+        if return_alpha:
+            ae = np.zeros((colidx.shape[0], heads), dtype=np.float64)
+            aself = np.zeros((n, heads), dtype=np.float64)
+        rc = L.oracle_aggregate_gat(C.c_int64(n), _p(rowptr), _p(colidx), _p(q), C.c_int64(q.shape[1]),
+                                    C.c_int32(heads), C.c_int32(dh), _p(a_src), _p(a_dst),
+                                    C.c_double(float(gat.get("negative_slope", 0.2))),
+                                    C.c_int32(int(gat.get("add_self_loop", 1))),
+                                    _p(out), C.c_int64(dim), _p(rows_a), C.c_int64(cnt), _p(ae), _p(aself))
+        _check(rc, "oracle_aggregate_gat")
+        return (out, ae, aself) if return_alpha else out
+    raise ValueError("unknown aggregator")
+
+
+# ---------------------------------------------------------------- per-node model
+class Mlp:
+    """State of one round's per-node model in double precision."""
+
+    def __init__(self, d_in: int, hidden: int, n_classes: int, w1, b1, w2=None, b2=None,
+                 optimizer: int = ADAM, lr: float = 0.003, beta1: float = 0.9, beta2: float = 0.999,
+                 eps: float = 1e-8, round_bf16: bool = True):
+        self.d_in, self.hidden, self.n_classes = int(d_in), int(hidden), int(n_classes)
+        parts = [np.asarray(w1, dtype=np.float64).ravel(), np.asarray(b1, dtype=np.float64).ravel()]
+        if hidden > 0:
+            parts += [np.asarray(w2, dtype=np.float64).ravel(), np.asarray(b2, dtype=np.float64).ravel()]
+        self.theta = np.ascontiguousarray(np.concatenate(parts))
+        assert self.theta.shape[0] == lib().oracle_theta_size(C.c_int32(d_in), C.c_int32(hidden),
+                                                              C.c_int32(n_classes))
+        self.m = np.zeros_like(self.theta)
+        self.v = np.zeros_like(self.theta)
+        self.optimizer, self.lr, self.beta1, self.beta2, self.eps = optimizer, lr, beta1, beta2, eps
+        self.step = 0
+        self.round_bf16 = bool(round_bf16)
+
+    def copy(self) -> "Mlp":
+        o = Mlp.__new__(Mlp)
+        o.__dict__.update(self.__dict__)
+        o.theta, o.m, o.v = self.theta.copy(), self.m.copy(), self.v.copy()
+        return o
+
+    def unpack(self, theta: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+        t = self.theta if theta is None else theta
+        out1 = self.hidden if self.hidden > 0 else self.n_classes
+        o = 0
+        d = {"w1": t[o:o + self.d_in * out1].reshape(self.d_in, out1)}
+        o += self.d_in * out1
+        d["b1"] = t[o:o + out1]
+        o += out1
+        if self.hidden > 0:
+            d["w2"] = t[o:o + self.hidden * self.n_classes].reshape(self.hidden, self.n_classes)
+            o += self.hidden * self.n_classes
+            d["b2"] = t[o:o + self.n_classes]
+        return d
+
+    def train_step(self, x: np.ndarray, y: np.ndarray, row_idx: Optional[np.ndarray] = None,
+                   return_grad: bool = False):
+        """One full-batch step on rows x[row_idx] (all rows of x if None) with
+        labels y (one per batch row).  Returns the loss before the update."""
+        x = _f32(x)
+        y = np.ascontiguousarray(y, dtype=np.int32)
+        ri = None if row_idx is None else np.ascontiguousarray(row_idx, dtype=np.int32)
+        n_rows = x.shape[0] if ri is None else ri.shape[0]
+        assert y.shape[0] == n_rows
+        loss = C.c_double(0.0)
+        grad = np.zeros_like(self.theta) if return_grad else None
+        self.step += 1
+        rc = lib().oracle_mlp_train_step(
+            C.c_int32(self.d_in), C.c_int32(self.hidden), C.c_int32(self.n_classes),
+            _p(self.theta), _p(self.m), _p(self.v), C.c_int32(self.optimizer),
+            C.c_double(self.lr), C.c_double(self.beta1), C.c_double(self.beta2), C.c_double(self.eps),
+            C.c_int64(self.step), C.c_int32(int(self.round_bf16)),
+            _p(x), C.c_int64(x.shape[1]), _p(ri), C.c_int64(n_rows), _p(y), C.byref(loss), _p(grad))
+        _check(rc, "oracle_mlp_train_step")
+        return (loss.value, grad) if return_grad else loss.value
+
+    def embed(self, x: np.ndarray, row_idx: Optional[np.ndarray] = None, y: Optional[np.ndarray] = None,
+              want_hidden: bool = False, want_logits: bool = True):
+        """Forward over rows; returns dict(hidden, logits, pred, correct)."""
+        x = _f32(x)
+        ri = None if row_idx is None else np.ascontiguousarray(row_idx, dtype=np.int32)
+        n_rows = x.shape[0] if ri is None else ri.shape[0]
+        hid = np.zeros((n_rows, self.hidden), dtype=np.float32) if (want_hidden and self.hidden > 0) else None
+        lg = np.zeros((n_rows, self.n_classes), dtype=np.float32) if want_logits else None
+        pred = np.zeros(n_rows, dtype=np.int32)
+        yy = None if y is None else np.ascontiguousarray(y, dtype=np.int32)
+        correct = C.c_uint64(0)
+        rc = lib().oracle_embed(
+            C.c_int32(self.d_in), C.c_int32(self.hidden), C.c_int32(self.n_classes), _p(self.theta),
+            C.c_int32(int(self.round_bf16)), _p(x), C.c_int64(x.shape[1]), _p(ri), C.c_int64(n_rows),
+            _p(hid), C.c_int64(self.hidden), _p(lg), C.c_int64(self.n_classes), _p(pred), _p(yy),
+            C.byref(correct))
+        _check(rc, "oracle_embed")
+        return dict(hidden=hid, logits=lg, pred=pred, correct=int(correct.value))
+
+
+# ---------------------------------------------------------------- counting
+def cross_partition(rowptr: np.ndarray, colidx: np.ndarray, part: np.ndarray, n_parts: int,
+                    dims: Sequence[int], elem_bytes: int = 4) -> Dict:
+    n = rowptr.shape[0] - 1
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+    colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+    part = np.ascontiguousarray(part, dtype=np.int32)
+    dims_a = np.ascontiguousarray(dims, dtype=np.int32)
+    K = dims_a.shape[0]
+    ce, bp, bt = C.c_uint64(0), C.c_uint64(0), C.c_uint64(0)
+    bpr = np.zeros(K, dtype=np.uint64)
+    send = np.zeros(n_parts, dtype=np.uint64)
+    recv = np.zeros(n_parts, dtype=np.uint64)
+    rc = lib().oracle_cross_partition(C.c_int64(n), _p(rowptr), _p(colidx), _p(part), C.c_int32(n_parts),
+                                      C.c_int32(K), _p(dims_a), C.c_int32(elem_bytes),
+                                      C.byref(ce), C.byref(bp), _p(bpr), C.byref(bt), _p(send), _p(recv))
+    _check(rc, "oracle_cross_partition")
+    return dict(cross_edges=int(ce.value), boundary_pairs=int(bp.value), bytes_per_round=bpr,
+                bytes_total=int(bt.value), send_per_part=send, recv_per_part=recv,
+                dv_lazy_lt=2 * int(bt.value))
+
+
+# ---------------------------------------------------------------- the K-round loop
+def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
+              rowptr, colidx, features, labels, train_idx, val_idx, test_idx,
+              weights: List[Dict[str, np.ndarray]], gat: Optional[Dict] = None,
+              optimizer: int = ADAM, round_bf16: bool = True, eval_every: int = 1,
+              part=None, n_parts: int = 0) -> Dict:
+    """Lazy message passing (Section 3.1): for each layer m = 1..K, one
+    message-passing round builds the layer's inputs, the layer (with a
+    temporary classifier unless it is the last) is trained alone for R
+    iterations, the iterate with the best validation accuracy (earliest on
+    ties) is kept, and its representations feed the next round."""
+    labels = np.ascontiguousarray(labels, dtype=np.int32)
+    q = _f32(features)
+    y_tr, y_va, y_te = labels[train_idx], labels[val_idx], labels[test_idx]
+    report = dict(rounds=[], n_aggregations=0, n_steps=0)
+    if part is not None:
+        dims = []
+        d = q.shape[1]
+        for m in range(K):
+            dims.append(d)
+            d = hidden
+        report["counts"] = cross_partition(rowptr, colidx, part, n_parts, dims, 4)
+    for m in range(1, K + 1):
+        w = weights[m - 1]
+        if aggr == GAT:
+            proj = Mlp(q.shape[1], 0, w["w_att"].shape[1], w["w_att"], np.zeros(w["w_att"].shape[1]),
+                       round_bf16=round_bf16)
+            p = proj.embed(q)["logits"]          # P = Q W_att (no bias, no activation)
+            g = dict(gat)
+            g["a_src"], g["a_dst"] = w["a_src"], w["a_dst"]
+            x = aggregate(GAT, rowptr, colidx, p, gat=g)
+        else:
+            x = aggregate(aggr, rowptr, colidx, q)
+        report["n_aggregations"] += 1
+        hid = hidden if m < K else 0
+        model = Mlp(x.shape[1], hid, n_classes, w["w1"], w["b1"], w.get("w2"), w.get("b2"),
+                    optimizer=optimizer, lr=lr, round_bf16=round_bf16)
+        best, best_correct, best_iter = None, -1, -1
+        losses, val_hist = [], []
+        for r in range(1, R + 1):
+            losses.append(model.train_step(x, y_tr, row_idx=train_idx))
+            report["n_steps"] += 1
+            if r % eval_every == 0 or r == R:
+                c = model.embed(x, row_idx=val_idx, y=y_va, want_logits=False)["correct"]
+                val_hist.append(c)
+                if c > best_correct:
+                    best, best_correct, best_iter = model.copy(), c, r
+        last_test = model.embed(x, row_idx=test_idx, y=y_te, want_logits=False)["correct"]
+        best_test = best.embed(x, row_idx=test_idx, y=y_te, want_logits=False)["correct"]
+        rd = dict(round=m, losses=np.asarray(losses), val_correct=np.asarray(val_hist),
+                  best_iter=best_iter, best_val_correct=best_correct,
+                  test_correct_best=best_test, test_correct_last=last_test, model=best, x=x)
+        if m < K:
+            q = best.embed(x, want_hidden=True, want_logits=False)["hidden"]
+            rd["q_out"] = q
+        else:
+            fin = best.embed(x, want_logits=True)
+            rd["logits"], rd["pred"] = fin["logits"], fin["pred"]
+        report["rounds"].append(rd)
+    report["test_acc"] = report["rounds"][-1]["test_correct_best"] / max(1, len(test_idx))
+    report["test_acc_last"] = report["rounds"][-1]["test_correct_last"] / max(1, len(test_idx))
+    report["val_acc"] = report["rounds"][-1]["best_val_correct"] / max(1, len(val_idx))
+    return report

@@ -1,0 +1,524 @@
+/*
+ * CPU checker for the on-device hot path of lazy message passing
+ * ("Scalable Neural Network Training over Distributed Graphs", Retexo).
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE.  It is a plain, slow restatement of the
+ * paper's definitions, used only by the tests, by the smoke check and as the
+ * timed CPU baseline.  The CUDA library never calls it and shares no source,
+ * header, table or helper with it.
+ *
+ * Conventions
+ *   - graph: symmetric CSR (both directions of every undirected edge stored),
+ *     no self loops, no duplicate entries (Section 2.1: "the graphs are
+ *     undirected"); rowptr is int64, colidx int32.
+ *   - features / representations are fp32 in memory; every sum is carried in
+ *     double and rounded to fp32 once at the end.
+ *   - counts are exact uint64.
+ *   - OpenMP is used only over independent output rows (or over fixed chunks
+ *     that are combined in index order), so no result depends on the number
+ *     of threads.
+ *
+ * Parity status: every function here is pinned by tests/test_oracle_*.py
+ * (dense brute force, closed forms, invariants, library special cases).  What
+ * cannot be pinned is agreement with the paper's printed accuracy and timing
+ * tables, which need the public datasets: parity unpinned for those.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_OK 0
+#define ORACLE_BAD_ARG 1
+#define ORACLE_NO_MEM 2
+
+/* ------------------------------------------------------------------ */
+/* bf16 operand rounding (round to nearest, ties to even, of the top   */
+/* 16 bits of an IEEE-754 binary32; NaN stays NaN)                      */
+/* ------------------------------------------------------------------ */
+static float bf16_round(float x)
+{
+    uint32_t u;
+    memcpy(&u, &x, 4);
+    if ((u & 0x7f800000u) == 0x7f800000u) {       /* inf / nan: truncate, keep nan */
+        if (u & 0x007fffffu) u |= 0x00400000u;
+        u &= 0xffff0000u;
+    } else {
+        uint32_t lsb = (u >> 16) & 1u;
+        u += 0x7fffu + lsb;
+        u &= 0xffff0000u;
+    }
+    memcpy(&x, &u, 4);
+    return x;
+}
+
+float oracle_bf16_round(float x) { return bf16_round(x); }
+
+static double opnd(double x, int round_bf16)
+{
+    return round_bf16 ? (double)bf16_round((float)x) : x;
+}
+
+/* ================================================================== */
+/* Aggregation, Eq. 1:  AGGR over u in N(v) of Q^{m-1}_u               */
+/* `rows` selects destination nodes (NULL = all); output row i belongs */
+/* to node rows[i].                                                    */
+/* ================================================================== */
+
+/* GCN: Z = D^-1/2 (A + I) D^-1/2 Q with D = degree + 1 (the self loop is
+ * implicit).  Section 2.2 names the GCN aggregator; the symmetric
+ * normalisation is that of the cited GCN layer.  Isolated node: Z_v = Q_v. */
+int oracle_aggregate_gcn(int64_t n, const int64_t *rowptr, const int32_t *colidx,
+                         const float *q, int64_t ldq, int32_t dim,
+                         float *out, int64_t ldout,
+                         const int64_t *rows, int64_t n_rows)
+{
+    if (n < 0 || dim < 0 || ldq < dim || ldout < dim) return ORACLE_BAD_ARG;
+    int64_t cnt = rows ? n_rows : n;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t i = 0; i < cnt; ++i) {
+        int64_t v = rows ? rows[i] : i;
+        double *acc = (double *)calloc((size_t)(dim > 0 ? dim : 1), sizeof(double));
+        if (!acc) { failed = 1; continue; }
+        double nv = 1.0 / sqrt((double)(rowptr[v + 1] - rowptr[v]) + 1.0);
+        for (int32_t j = 0; j < dim; ++j) acc[j] = nv * (double)q[v * ldq + j];
+        for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+            int64_t u = colidx[e];
+            double nu = 1.0 / sqrt((double)(rowptr[u + 1] - rowptr[u]) + 1.0);
+            for (int32_t j = 0; j < dim; ++j) acc[j] += nu * (double)q[u * ldq + j];
+        }
+        for (int32_t j = 0; j < dim; ++j) out[i * ldout + j] = (float)(nv * acc[j]);
+        free(acc);
+    }
+    return failed ? ORACLE_NO_MEM : ORACLE_OK;
+}
+
+/* GraphSAGE mean with COMBINE = concatenation (Section 2.2): columns [0,dim)
+ * are the node's own row, columns [dim,2dim) the mean over N(v) (v itself
+ * excluded); a node without neighbours gets a zero mean. */
+int oracle_aggregate_sage_mean(int64_t n, const int64_t *rowptr, const int32_t *colidx,
+                               const float *q, int64_t ldq, int32_t dim,
+                               float *out, int64_t ldout,
+                               const int64_t *rows, int64_t n_rows)
+{
+    if (n < 0 || dim < 0 || ldq < dim || ldout < 2 * (int64_t)dim) return ORACLE_BAD_ARG;
+    int64_t cnt = rows ? n_rows : n;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t i = 0; i < cnt; ++i) {
+        int64_t v = rows ? rows[i] : i;
+        double *acc = (double *)calloc((size_t)(dim > 0 ? dim : 1), sizeof(double));
+        if (!acc) { failed = 1; continue; }
+        int64_t deg = rowptr[v + 1] - rowptr[v];
+        for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+            int64_t u = colidx[e];
+            for (int32_t j = 0; j < dim; ++j) acc[j] += (double)q[u * ldq + j];
+        }
+        for (int32_t j = 0; j < dim; ++j) {
+            out[i * ldout + j] = q[v * ldq + j];
+            out[i * ldout + dim + j] = deg > 0 ? (float)(acc[j] / (double)deg) : 0.0f;
+        }
+        free(acc);
+    }
+    return failed ? ORACLE_NO_MEM : ORACLE_OK;
+}
+
+/* GAT (cited in Section 2.2; formula of the cited layer).  p holds the
+ * already projected rows, heads*head_dim wide, head k in columns
+ * [k*head_dim, (k+1)*head_dim).  For destination v and head k:
+ *   s_u = <a_src[k], p_u^k>,  t_v = <a_dst[k], p_v^k>
+ *   e_uv = LeakyReLU_slope(s_u + t_v)  for u in N(v) (and u = v if
+ *                                      add_self_loop)
+ *   alpha_uv = softmax over those u of e_uv
+ *   Z_v^k = sum_u alpha_uv p_u^k
+ * A node whose softmax set is empty gets zeros.
+ * alpha_edge [n_edges x heads] and alpha_self [n x heads] (both optional,
+ * only with rows == NULL) receive the attention weights. */
+int oracle_aggregate_gat(int64_t n, const int64_t *rowptr, const int32_t *colidx,
+                         const float *p, int64_t ldp, int32_t heads, int32_t head_dim,
+                         const float *a_src, const float *a_dst, double slope,
+                         int32_t add_self_loop,
+                         float *out, int64_t ldout,
+                         const int64_t *rows, int64_t n_rows,
+                         double *alpha_edge, double *alpha_self)
+{
+    int32_t dim = heads * head_dim;
+    if (n < 0 || heads <= 0 || head_dim <= 0 || ldp < dim || ldout < dim) return ORACLE_BAD_ARG;
+    if (rows && (alpha_edge || alpha_self)) return ORACLE_BAD_ARG;
+    double *s = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1) * heads);
+    double *t = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1) * heads);
+    if (!s || !t) { free(s); free(t); return ORACLE_NO_MEM; }
+#pragma omp parallel for
+    for (int64_t u = 0; u < n; ++u)
+        for (int32_t k = 0; k < heads; ++k) {
+            double ss = 0.0, tt = 0.0;
+            for (int32_t j = 0; j < head_dim; ++j) {
+                double x = (double)p[u * ldp + k * head_dim + j];
+                ss += (double)a_src[k * head_dim + j] * x;
+                tt += (double)a_dst[k * head_dim + j] * x;
+            }
+            s[u * heads + k] = ss;
+            t[u * heads + k] = tt;
+        }
+    int64_t cnt = rows ? n_rows : n;
+    int failed = 0;
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t i = 0; i < cnt; ++i) {
+        int64_t v = rows ? rows[i] : i;
+        int64_t deg = rowptr[v + 1] - rowptr[v];
+        int64_t m = deg + (add_self_loop ? 1 : 0);
+        double *e = (double *)malloc(sizeof(double) * (size_t)(m > 0 ? m : 1));
+        double *acc = (double *)malloc(sizeof(double) * (size_t)head_dim);
+        if (!e || !acc) { free(e); free(acc); failed = 1; continue; }
+        for (int32_t k = 0; k < heads; ++k) {
+            for (int64_t a = 0; a < m; ++a) {
+                int64_t u = a < deg ? (int64_t)colidx[rowptr[v] + a] : v;
+                double z = s[u * heads + k] + t[v * heads + k];
+                e[a] = z > 0.0 ? z : slope * z;
+            }
+            double mx = -INFINITY, den = 0.0;
+            for (int64_t a = 0; a < m; ++a) if (e[a] > mx) mx = e[a];
+            for (int64_t a = 0; a < m; ++a) { e[a] = exp(e[a] - mx); den += e[a]; }
+            for (int32_t j = 0; j < head_dim; ++j) acc[j] = 0.0;
+            for (int64_t a = 0; a < m; ++a) {
+                int64_t u = a < deg ? (int64_t)colidx[rowptr[v] + a] : v;
+                double alpha = e[a] / den;
+                if (a < deg) { if (alpha_edge) alpha_edge[(rowptr[v] + a) * heads + k] = alpha; }
+                else if (alpha_self) alpha_self[v * heads + k] = alpha;
+                for (int32_t j = 0; j < head_dim; ++j)
+                    acc[j] += alpha * (double)p[u * ldp + k * head_dim + j];
+            }
+            for (int32_t j = 0; j < head_dim; ++j)
+                out[i * ldout + k * head_dim + j] = m > 0 ? (float)acc[j] : 0.0f;
+        }
+        free(e);
+        free(acc);
+    }
+    free(s);
+    free(t);
+    return failed ? ORACLE_NO_MEM : ORACLE_OK;
+}
+
+/* ================================================================== */
+/* Per-node model of one round (Section 3.1): f_theta = Linear+ReLU,   */
+/* temporary classifier C_theta = Linear; last round: one Linear.      */
+/* theta is one flat double array:                                     */
+/*   hidden > 0 : [ W1 (d_in x hidden) | b1 (hidden) |                 */
+/*                  W2 (hidden x n_classes) | b2 (n_classes) ]         */
+/*   hidden == 0: [ W1 (d_in x n_classes) | b1 (n_classes) ]           */
+/* matrices row-major [in x out].                                       */
+/* round_bf16 != 0: both operands of every matrix product are rounded  */
+/* to bf16 first ("bf16 inputs, wider accumulate"); sums, biases,      */
+/* softmax and the optimiser stay in double.                           */
+/* ================================================================== */
+
+int64_t oracle_theta_size(int32_t d_in, int32_t hidden, int32_t n_classes)
+{
+    if (hidden > 0)
+        return (int64_t)d_in * hidden + hidden + (int64_t)hidden * n_classes + n_classes;
+    return (int64_t)d_in * n_classes + n_classes;
+}
+
+/* forward for one input row; a1 = pre-activation (hidden wide, may be NULL
+ * when hidden == 0), logits = n_classes wide */
+static void forward_row(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
+                        int round_bf16, const float *xrow, const double *w1r, const double *w2r,
+                        double *a1, double *logits)
+{
+    if (hidden > 0) {
+        const double *b1 = theta + (int64_t)d_in * hidden;
+        const double *b2 = b1 + hidden + (int64_t)hidden * n_classes;
+        for (int32_t j = 0; j < hidden; ++j) a1[j] = 0.0;
+        for (int32_t k = 0; k < d_in; ++k) {
+            double xv = opnd((double)xrow[k], round_bf16);
+            if (xv == 0.0) continue;
+            const double *wrow = w1r + (int64_t)k * hidden;
+            for (int32_t j = 0; j < hidden; ++j) a1[j] += xv * wrow[j];
+        }
+        for (int32_t j = 0; j < hidden; ++j) a1[j] += b1[j];
+        for (int32_t c = 0; c < n_classes; ++c) logits[c] = 0.0;
+        for (int32_t j = 0; j < hidden; ++j) {
+            double h = a1[j] > 0.0 ? a1[j] : 0.0;
+            h = opnd(h, round_bf16);
+            if (h == 0.0) continue;
+            const double *wrow = w2r + (int64_t)j * n_classes;
+            for (int32_t c = 0; c < n_classes; ++c) logits[c] += h * wrow[c];
+        }
+        for (int32_t c = 0; c < n_classes; ++c) logits[c] += b2[c];
+    } else {
+        const double *b1 = theta + (int64_t)d_in * n_classes;
+        for (int32_t c = 0; c < n_classes; ++c) logits[c] = 0.0;
+        for (int32_t k = 0; k < d_in; ++k) {
+            double xv = opnd((double)xrow[k], round_bf16);
+            if (xv == 0.0) continue;
+            const double *wrow = w1r + (int64_t)k * n_classes;
+            for (int32_t c = 0; c < n_classes; ++c) logits[c] += xv * wrow[c];
+        }
+        for (int32_t c = 0; c < n_classes; ++c) logits[c] += b1[c];
+    }
+}
+
+/* copies of the weight matrices with the operand rounding applied */
+static int rounded_weights(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
+                           int round_bf16, double **w1r, double **w2r)
+{
+    int32_t out1 = hidden > 0 ? hidden : n_classes;
+    int64_t n1 = (int64_t)d_in * out1;
+    *w1r = (double *)malloc(sizeof(double) * (size_t)(n1 > 0 ? n1 : 1));
+    *w2r = NULL;
+    if (!*w1r) return ORACLE_NO_MEM;
+    for (int64_t i = 0; i < n1; ++i) (*w1r)[i] = opnd(theta[i], round_bf16);
+    if (hidden > 0) {
+        int64_t n2 = (int64_t)hidden * n_classes;
+        const double *w2 = theta + n1 + hidden;
+        *w2r = (double *)malloc(sizeof(double) * (size_t)(n2 > 0 ? n2 : 1));
+        if (!*w2r) { free(*w1r); return ORACLE_NO_MEM; }
+        for (int64_t i = 0; i < n2; ++i) (*w2r)[i] = opnd(w2[i], round_bf16);
+    }
+    return ORACLE_OK;
+}
+
+#define GRAD_CHUNKS 64
+
+/* One full-batch training step (Section 2.3: forward, loss, backward, update;
+ * one worker, so the gradient average at the master is the identity).
+ *   loss = mean_i CE(softmax(logits_i), y_i)
+ * Batch row i is x[row_idx ? row_idx[i] : i]; y[i] is its label.
+ * optimizer: 0 = SGD (theta -= lr g), 1 = Adam (bias-corrected, eps outside
+ * the root, no weight decay); `step` is the 1-based count of this update.
+ * grad_out (optional) receives the gradient, laid out like theta. */
+int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
+                          double *theta, double *adam_m, double *adam_v,
+                          int32_t optimizer, double lr, double beta1, double beta2, double eps,
+                          int64_t step, int32_t round_bf16,
+                          const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                          const int32_t *y, double *loss_out, double *grad_out)
+{
+    if (d_in <= 0 || n_classes <= 0 || hidden < 0 || n_rows <= 0 || ldx < d_in) return ORACLE_BAD_ARG;
+    if (optimizer == 1 && (!adam_m || !adam_v || step < 1)) return ORACLE_BAD_ARG;
+    int64_t nt = oracle_theta_size(d_in, hidden, n_classes);
+    int32_t out1 = hidden > 0 ? hidden : n_classes;
+    double *w1r, *w2r;
+    if (rounded_weights(d_in, hidden, n_classes, theta, round_bf16, &w1r, &w2r)) return ORACLE_NO_MEM;
+
+    /* per-row results of the forward/backward through the row-local part */
+    double *d1 = (double *)malloc(sizeof(double) * (size_t)n_rows * out1);       /* grad wrt first linear output */
+    double *hd = hidden > 0 ? (double *)malloc(sizeof(double) * (size_t)n_rows * hidden) : NULL;
+    double *dl = hidden > 0 ? (double *)malloc(sizeof(double) * (size_t)n_rows * n_classes) : NULL;
+    double *row_loss = (double *)malloc(sizeof(double) * (size_t)n_rows);
+    double *grad = (double *)calloc((size_t)nt, sizeof(double));
+    int bad_label = 0;
+    if (!d1 || (hidden > 0 && (!hd || !dl)) || !row_loss || !grad) {
+        free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad);
+        return ORACLE_NO_MEM;
+    }
+
+#pragma omp parallel
+    {
+        double *a1 = (double *)malloc(sizeof(double) * (size_t)(hidden > 0 ? hidden : 1));
+        double *lg = (double *)malloc(sizeof(double) * (size_t)n_classes);
+#pragma omp for schedule(static)
+        for (int64_t i = 0; i < n_rows; ++i) {
+            int64_t r = row_idx ? row_idx[i] : i;
+            forward_row(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg);
+            int32_t yi = y[i];
+            if (yi < 0 || yi >= n_classes) { bad_label = 1; yi = 0; }
+            double mx = lg[0];
+            for (int32_t c = 1; c < n_classes; ++c) if (lg[c] > mx) mx = lg[c];
+            double den = 0.0;
+            for (int32_t c = 0; c < n_classes; ++c) den += exp(lg[c] - mx);
+            row_loss[i] = (mx + log(den)) - lg[yi];
+            double *g = hidden > 0 ? dl + i * n_classes : d1 + i * out1;
+            for (int32_t c = 0; c < n_classes; ++c)
+                g[c] = (exp(lg[c] - mx) / den - (c == yi ? 1.0 : 0.0)) / (double)n_rows;
+            if (hidden > 0) {
+                for (int32_t j = 0; j < hidden; ++j) {
+                    double h = a1[j] > 0.0 ? a1[j] : 0.0;
+                    hd[i * hidden + j] = h;
+                    double acc = 0.0;
+                    if (a1[j] > 0.0) {
+                        const double *wrow = w2r + (int64_t)j * n_classes;
+                        for (int32_t c = 0; c < n_classes; ++c) acc += opnd(g[c], round_bf16) * wrow[c];
+                    }
+                    d1[i * hidden + j] = acc;
+                }
+            }
+        }
+        free(a1);
+        free(lg);
+    }
+
+    double loss = 0.0;
+    for (int64_t i = 0; i < n_rows; ++i) loss += row_loss[i];
+    loss /= (double)n_rows;
+
+    /* weight gradients: sums over batch rows, taken in fixed chunks of rows
+     * that are then added in chunk order */
+    double *part = (double *)calloc((size_t)GRAD_CHUNKS * (size_t)nt, sizeof(double));
+    if (!part) {
+        free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad);
+        return ORACLE_NO_MEM;
+    }
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int ch = 0; ch < GRAD_CHUNKS; ++ch) {
+        int64_t lo = n_rows * ch / GRAD_CHUNKS, hi = n_rows * (ch + 1) / GRAD_CHUNKS;
+        double *g = part + (int64_t)ch * nt;
+        double *gw1 = g, *gb1 = g + (int64_t)d_in * out1;
+        double *gw2 = gb1 + out1, *gb2 = gw2 + (int64_t)hidden * n_classes;
+        for (int64_t i = lo; i < hi; ++i) {
+            int64_t r = row_idx ? row_idx[i] : i;
+            const float *xrow = x + r * ldx;
+            const double *d1row = d1 + i * out1;
+            /* dW1 = X^T d1,  db1 = sum d1 */
+            for (int32_t k = 0; k < d_in; ++k) {
+                double xv = opnd((double)xrow[k], round_bf16);
+                if (xv == 0.0) continue;
+                double *grow = gw1 + (int64_t)k * out1;
+                for (int32_t j = 0; j < out1; ++j) grow[j] += xv * opnd(d1row[j], round_bf16);
+            }
+            for (int32_t j = 0; j < out1; ++j) gb1[j] += d1row[j];
+            if (hidden > 0) {
+                /* dW2 = Hd^T dL,  db2 = sum dL */
+                const double *dlrow = dl + i * n_classes;
+                for (int32_t j = 0; j < hidden; ++j) {
+                    double h = opnd(hd[i * hidden + j], round_bf16);
+                    if (h == 0.0) continue;
+                    double *grow = gw2 + (int64_t)j * n_classes;
+                    for (int32_t c = 0; c < n_classes; ++c) grow[c] += h * opnd(dlrow[c], round_bf16);
+                }
+                for (int32_t c = 0; c < n_classes; ++c) gb2[c] += dlrow[c];
+            }
+        }
+    }
+    for (int ch = 0; ch < GRAD_CHUNKS; ++ch)
+        for (int64_t p = 0; p < nt; ++p) grad[p] += part[(int64_t)ch * nt + p];
+    free(part);
+
+    /* update */
+    if (optimizer == 0) {
+        for (int64_t p = 0; p < nt; ++p) theta[p] -= lr * grad[p];
+    } else {
+        double c1 = 1.0 - pow(beta1, (double)step), c2 = 1.0 - pow(beta2, (double)step);
+        for (int64_t p = 0; p < nt; ++p) {
+            adam_m[p] = beta1 * adam_m[p] + (1.0 - beta1) * grad[p];
+            adam_v[p] = beta2 * adam_v[p] + (1.0 - beta2) * grad[p] * grad[p];
+            double mh = adam_m[p] / c1, vh = adam_v[p] / c2;
+            theta[p] -= lr * mh / (sqrt(vh) + eps);
+        }
+    }
+    if (loss_out) *loss_out = loss;
+    if (grad_out) memcpy(grad_out, grad, sizeof(double) * (size_t)nt);
+    free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad);
+    return bad_label ? ORACLE_BAD_ARG : ORACLE_OK;
+}
+
+/* Forward of the trained per-node model over a set of rows.
+ *   hidden > 0: hidden_out = ReLU(x W1 + b1)  — the representation Q^m that
+ *               the next round aggregates, the classifier being dropped
+ *               (Section 3.1) — and/or logits = hidden W2 + b2;
+ *   hidden == 0: logits = x W1 + b1 (hidden_out must be NULL).
+ * pred = argmax of the fp32-rounded logits, lowest index on ties;
+ * correct = number of rows with pred == y[i] (y optional). */
+int oracle_embed(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
+                 int32_t round_bf16,
+                 const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                 float *hidden_out, int64_t ld_hidden,
+                 float *logits_out, int64_t ld_logits,
+                 int32_t *pred_out, const int32_t *y, uint64_t *correct_out)
+{
+    if (d_in <= 0 || n_classes <= 0 || hidden < 0 || n_rows < 0 || ldx < d_in) return ORACLE_BAD_ARG;
+    if (hidden == 0 && hidden_out) return ORACLE_BAD_ARG;
+    double *w1r, *w2r;
+    if (rounded_weights(d_in, hidden, n_classes, theta, round_bf16, &w1r, &w2r)) return ORACLE_NO_MEM;
+    uint64_t correct = 0;
+#pragma omp parallel reduction(+ : correct)
+    {
+        double *a1 = (double *)malloc(sizeof(double) * (size_t)(hidden > 0 ? hidden : 1));
+        double *lg = (double *)malloc(sizeof(double) * (size_t)n_classes);
+#pragma omp for schedule(static)
+        for (int64_t i = 0; i < n_rows; ++i) {
+            int64_t r = row_idx ? row_idx[i] : i;
+            forward_row(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg);
+            if (hidden_out)
+                for (int32_t j = 0; j < hidden; ++j)
+                    hidden_out[i * ld_hidden + j] = (float)(a1[j] > 0.0 ? a1[j] : 0.0);
+            if (logits_out)
+                for (int32_t c = 0; c < n_classes; ++c) logits_out[i * ld_logits + c] = (float)lg[c];
+            int32_t best = 0;
+            for (int32_t c = 1; c < n_classes; ++c)
+                if ((float)lg[c] > (float)lg[best]) best = c;
+            if (pred_out) pred_out[i] = best;
+            if (y && best == y[i]) correct += 1;
+        }
+        free(a1);
+        free(lg);
+    }
+    if (correct_out) *correct_out = correct;
+    free(w1r);
+    free(w2r);
+    return ORACLE_OK;
+}
+
+/* ================================================================== */
+/* Messages and bytes that cross a given node partition in one lazy    */
+/* message-passing round (Section 2.1 boundary nodes; Appendix A.1).   */
+/*   cross_edges    = #{CSR entries (u,v): part[u] != part[v]}         */
+/*   boundary_pairs = #{distinct (u, part[v]) over those entries}      */
+/*                  = sum over workers i of B_i (its boundary nodes)   */
+/*   send_per_part[p] = pairs whose node u lives in p                  */
+/*   recv_per_part[p] = pairs whose destination partition is p  (=B_p) */
+/*   bytes_per_round[m] = boundary_pairs * dims[m] * elem_bytes        */
+/*   bytes_total = sum_m bytes_per_round[m]; the appendix' DV^lazy_lt  */
+/*   counts every message at sender and receiver, i.e. 2 * bytes_total */
+/* ================================================================== */
+static int cmp_i32(const void *a, const void *b)
+{
+    int32_t x = *(const int32_t *)a, y = *(const int32_t *)b;
+    return (x > y) - (x < y);
+}
+
+int oracle_cross_partition(int64_t n, const int64_t *rowptr, const int32_t *colidx,
+                           const int32_t *part, int32_t n_parts,
+                           int32_t K, const int32_t *dims, int32_t elem_bytes,
+                           uint64_t *cross_edges, uint64_t *boundary_pairs,
+                           uint64_t *bytes_per_round, uint64_t *bytes_total,
+                           uint64_t *send_per_part, uint64_t *recv_per_part)
+{
+    if (n < 0 || n_parts <= 0 || K < 0 || elem_bytes <= 0) return ORACLE_BAD_ARG;
+    for (int64_t v = 0; v < n; ++v)
+        if (part[v] < 0 || part[v] >= n_parts) return ORACLE_BAD_ARG;
+    uint64_t ce = 0, bp = 0;
+    if (send_per_part) memset(send_per_part, 0, sizeof(uint64_t) * (size_t)n_parts);
+    if (recv_per_part) memset(recv_per_part, 0, sizeof(uint64_t) * (size_t)n_parts);
+    for (int64_t u = 0; u < n; ++u) {
+        int64_t deg = rowptr[u + 1] - rowptr[u];
+        if (deg == 0) continue;
+        int32_t *dst = (int32_t *)malloc(sizeof(int32_t) * (size_t)deg);
+        if (!dst) return ORACLE_NO_MEM;
+        int64_t m = 0;
+        for (int64_t e = rowptr[u]; e < rowptr[u + 1]; ++e) {
+            int64_t v = colidx[e];
+            if (part[v] != part[u]) dst[m++] = part[v];
+        }
+        ce += (uint64_t)m;
+        qsort(dst, (size_t)m, sizeof(int32_t), cmp_i32);
+        for (int64_t a = 0; a < m; ++a) {
+            if (a > 0 && dst[a] == dst[a - 1]) continue;
+            bp += 1;
+            if (send_per_part) send_per_part[part[u]] += 1;
+            if (recv_per_part) recv_per_part[dst[a]] += 1;
+        }
+        free(dst);
+    }
+    uint64_t tot = 0;
+    for (int32_t m = 0; m < K; ++m) {
+        uint64_t b = bp * (uint64_t)dims[m] * (uint64_t)elem_bytes;
+        if (bytes_per_round) bytes_per_round[m] = b;
+        tot += b;
+    }
+    if (cross_edges) *cross_edges = ce;
+    if (boundary_pairs) *boundary_pairs = bp;
+    if (bytes_total) *bytes_total = tot;
+    return ORACLE_OK;
+}

@@ -1,0 +1,443 @@
+"""Seeded synthetic workloads shaped like the paper's benchmark graphs.
+
+This module only *draws inputs*: graphs (symmetric CSR, no self loops, no
+duplicate entries, columns sorted within a row), node features, labels,
+train/val/test index sets, a partition id per node and the initial weights of
+every round's per-node model.  It holds none of the method's arithmetic (no
+aggregation, no MLP, no counting) and depends on numpy alone, so the CPU
+checker and the CUDA library can both be fed from it without sharing code.
+
+The shapes follow the dataset-statistics table of the paper's Appendix B
+(Cora-, PubMed-, Facebook-page-, Reddit- and ogbn-products-sized graphs); the
+records themselves are random draws, not the public datasets.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional
+
+import numpy as np
+
+GCN, SAGE_MEAN, GAT = 0, 1, 2
+AGGR_NAMES = {GCN: "gcn", SAGE_MEAN: "sage_mean", GAT: "gat"}
+
+
+@dataclass
+class Workload:
+    name: str
+    aggr: int                 # GCN / SAGE_MEAN / GAT
+    K: int                    # rounds = GNN layers
+    R: int                    # training iterations per round
+    hidden: int
+    n_classes: int
+    lr: float
+    n_nodes: int
+    rowptr: np.ndarray        # int64 [n_nodes + 1]
+    colidx: np.ndarray        # int32 [n_edges], both directions stored
+    features: np.ndarray      # float32 [n_nodes, d0]
+    labels: np.ndarray        # int32 [n_nodes]
+    train_idx: np.ndarray     # int32, sorted
+    val_idx: np.ndarray
+    test_idx: np.ndarray
+    part: np.ndarray          # int32 [n_nodes]
+    n_parts: int
+    heads: int = 0            # GAT only
+    head_dim: int = 0
+    negative_slope: float = 0.2
+    seed: int = 0
+    meta: Dict[str, float] = field(default_factory=dict)
+
+    @property
+    def n_edges(self) -> int:
+        return int(self.colidx.shape[0])
+
+    @property
+    def d0(self) -> int:
+        return int(self.features.shape[1])
+
+    def round_dims(self) -> List[Dict[str, int]]:
+        """Per round m = 1..K: width that is aggregated, MLP input width,
+        hidden width (0 in the last round) — the shapes of Eq. 1 with the
+        temporary classifier of Section 3.1."""
+        out = []
+        d_prev = self.d0
+        for m in range(1, self.K + 1):
+            if self.aggr == GAT:
+                agg_in = self.heads * self.head_dim      # projected width
+                d_in = agg_in
+            elif self.aggr == SAGE_MEAN:
+                agg_in = d_prev
+                d_in = 2 * d_prev
+            else:
+                agg_in = d_prev
+                d_in = d_prev
+            hid = self.hidden if m < self.K else 0
+            out.append(dict(round=m, rep_dim=d_prev, agg_dim=agg_in, d_in=d_in, hidden=hid))
+            d_prev = self.hidden
+        return out
+
+
+# --------------------------------------------------------------------------
+# graph helpers
+# --------------------------------------------------------------------------
+
+def csr_from_undirected(n: int, a: np.ndarray, b: np.ndarray):
+    """Symmetric CSR from distinct undirected pairs (a[i] != b[i])."""
+    a = a.astype(np.int64, copy=False)
+    b = b.astype(np.int64, copy=False)
+    key = np.concatenate([a * n + b, b * n + a])
+    key.sort(kind="stable")
+    rows = key // n
+    cols = (key - rows * n).astype(np.int32)
+    counts = np.bincount(rows, minlength=n)
+    rowptr = np.zeros(n + 1, dtype=np.int64)
+    np.cumsum(counts, out=rowptr[1:])
+    return rowptr, cols
+
+
+def _dedup_pairs(n: int, u: np.ndarray, v: np.ndarray):
+    keep = u != v
+    u, v = u[keep], v[keep]
+    lo = np.minimum(u, v).astype(np.int64)
+    hi = np.maximum(u, v).astype(np.int64)
+    return lo * n + hi            # caller uniques
+
+
+def _sample_by_weight(rng, cum: np.ndarray, lo: np.ndarray, hi: np.ndarray):
+    """Draw indices i with probability proportional to the weights whose
+    cumulative sum is `cum`, restricted to the mass interval [lo, hi)."""
+    r = lo + rng.random(lo.shape[0]) * (hi - lo)
+    idx = np.searchsorted(cum, r, side="right")
+    return np.minimum(idx, cum.shape[0] - 1)
+
+
+def _power_law_weights(n: int, exponent: float, max_over_mean: Optional[float]):
+    """w_i = (i + i0)^(-1/(exponent-1)); i0 is solved by bisection so that
+    max(w)/mean(w) equals `max_over_mean` (None: i0 = 1)."""
+    a = 1.0 / (exponent - 1.0)
+    i = np.arange(n, dtype=np.float64)
+
+    def ratio(i0):
+        w = (i + i0) ** (-a)
+        return w[0] / w.mean()
+
+    if max_over_mean is None:
+        i0 = 1.0
+    else:
+        lo_, hi_ = 1e-3, float(n) * 10
+        if ratio(lo_) < max_over_mean:
+            i0 = lo_
+        else:
+            for _ in range(100):
+                mid = np.sqrt(lo_ * hi_)
+                if ratio(mid) > max_over_mean:
+                    lo_ = mid
+                else:
+                    hi_ = mid
+            i0 = np.sqrt(lo_ * hi_)
+    return (i + i0) ** (-a)
+
+
+def random_graph(rng, n: int, n_und: int, labels: np.ndarray, weights: Optional[np.ndarray],
+                 frac_within: Optional[float], keep_cross: Optional[float]):
+    """Draw exactly `n_und` distinct undirected edges (fewer only if the graph
+    saturates).
+
+    weights      : endpoint propensities (None = uniform), Chung-Lu style.
+    frac_within  : if set, this share of candidate edges takes its second
+                   endpoint from the first endpoint's label block
+                   (degree-corrected SBM); the rest from anywhere.
+    keep_cross   : if set, a candidate whose endpoints differ in label is kept
+                   with this probability (homophily by rejection).
+    The propensities are dealt to node ids in a seeded random order, so node
+    id says nothing about degree.
+    """
+    if weights is None:
+        weights = np.ones(n, dtype=np.float64)
+    else:
+        weights = weights[rng.permutation(n)]
+    n_blocks = int(labels.max()) + 1
+    order = np.argsort(labels, kind="stable")          # nodes grouped by block
+    w_sorted = weights[order]
+    cum = np.cumsum(w_sorted)
+    total = cum[-1]
+    blk_sorted = labels[order]
+    starts = np.searchsorted(blk_sorted, np.arange(n_blocks), side="left")
+    ends = np.searchsorted(blk_sorted, np.arange(n_blocks), side="right")
+    cum0 = np.concatenate([[0.0], cum])
+    blk_lo = cum0[starts]
+    blk_hi = cum0[ends]
+
+    have = np.empty(0, dtype=np.int64)
+    need = n_und
+    for _ in range(64):
+        if need <= 0:
+            break
+        m = int(need * 1.15) + 1024
+        zeros = np.zeros(m)
+        iu = _sample_by_weight(rng, cum, zeros, zeros + total)
+        if frac_within is not None:
+            within = rng.random(m) < frac_within
+            b = blk_sorted[iu]
+            lo = np.where(within, blk_lo[b], 0.0)
+            hi = np.where(within, blk_hi[b], total)
+            iv = _sample_by_weight(rng, cum, lo, hi)
+        else:
+            iv = _sample_by_weight(rng, cum, zeros, zeros + total)
+        if keep_cross is not None:
+            cross = blk_sorted[iu] != blk_sorted[iv]
+            keep = (~cross) | (rng.random(m) < keep_cross)
+            iu, iv = iu[keep], iv[keep]
+        keys = _dedup_pairs(n, order[iu], order[iv])
+        have = np.unique(np.concatenate([have, keys]))
+        if have.shape[0] >= n_und:
+            break
+        need = n_und - have.shape[0]
+    if have.shape[0] > n_und:
+        sel = rng.permutation(have.shape[0])[:n_und]
+        sel.sort()
+        have = have[sel]
+    a = have // n
+    b = have - a * n
+    return csr_from_undirected(n, a, b)
+
+
+# --------------------------------------------------------------------------
+# features / labels / splits
+# --------------------------------------------------------------------------
+
+def _zipf_labels(rng, n, n_classes):
+    p = 1.0 / np.arange(1, n_classes + 1)
+    p /= p.sum()
+    return rng.choice(n_classes, size=n, p=p).astype(np.int32)
+
+
+def _gaussian_features(rng, labels, dim, shift):
+    n_classes = int(labels.max()) + 1
+    u = rng.standard_normal((n_classes, dim))
+    u /= np.linalg.norm(u, axis=1, keepdims=True)
+    f = rng.standard_normal((labels.shape[0], dim), dtype=np.float32)
+    f += (shift * u[labels]).astype(np.float32)
+    return f
+
+
+def _bag_of_words(rng, labels, dim, ones_per_row, class_words, class_share):
+    """Binary rows: `ones_per_row` draws, `class_share` of them from the
+    label's own word set, the rest uniform; duplicates collapse."""
+    n = labels.shape[0]
+    n_classes = int(labels.max()) + 1
+    sets = np.stack([rng.choice(dim, size=class_words, replace=False) for _ in range(n_classes)])
+    f = np.zeros((n, dim), dtype=np.float32)
+    from_class = rng.random((n, ones_per_row)) < class_share
+    pick_c = sets[labels[:, None], rng.integers(0, class_words, size=(n, ones_per_row))]
+    pick_u = rng.integers(0, dim, size=(n, ones_per_row))
+    cols = np.where(from_class, pick_c, pick_u)
+    f[np.arange(n)[:, None], cols] = 1.0
+    return f
+
+
+def _tfidf_like(rng, labels, dim, nnz_per_row, class_words, class_share):
+    """Non-negative sparse rows, support biased to the label's word set,
+    magnitudes |N(0,1)|, rows L2-normalised."""
+    n = labels.shape[0]
+    n_classes = int(labels.max()) + 1
+    sets = np.stack([rng.choice(dim, size=class_words, replace=False) for _ in range(n_classes)])
+    from_class = rng.random((n, nnz_per_row)) < class_share
+    pick_c = sets[labels[:, None], rng.integers(0, class_words, size=(n, nnz_per_row))]
+    pick_u = rng.integers(0, dim, size=(n, nnz_per_row))
+    cols = np.where(from_class, pick_c, pick_u)
+    f = np.zeros((n, dim), dtype=np.float32)
+    f[np.arange(n)[:, None], cols] = np.abs(rng.standard_normal((n, nnz_per_row))).astype(np.float32)
+    nrm = np.linalg.norm(f, axis=1, keepdims=True)
+    nrm[nrm == 0] = 1.0
+    return (f / nrm).astype(np.float32)
+
+
+def _split_per_class(rng, labels, per_class, n_val, n_test):
+    n_classes = int(labels.max()) + 1
+    train = []
+    for c in range(n_classes):
+        members = np.flatnonzero(labels == c)
+        train.append(rng.permutation(members)[:per_class])
+    train = np.concatenate(train)
+    rest = np.setdiff1d(np.arange(labels.shape[0]), train)
+    rest = rng.permutation(rest)
+    val, test = rest[:n_val], rest[n_val:n_val + n_test]
+    return (np.sort(train).astype(np.int32), np.sort(val).astype(np.int32),
+            np.sort(test).astype(np.int32))
+
+
+def _split_fraction(rng, n, f_train, f_val):
+    p = rng.permutation(n)
+    a = int(round(f_train * n))
+    b = a + int(round(f_val * n))
+    return (np.sort(p[:a]).astype(np.int32), np.sort(p[a:b]).astype(np.int32),
+            np.sort(p[b:]).astype(np.int32))
+
+
+# --------------------------------------------------------------------------
+# the five configurations
+# --------------------------------------------------------------------------
+
+def _scaled(x: int, scale: float, floor: int) -> int:
+    return max(floor, int(round(x * scale)))
+
+
+def make_config(index: int, seed: int = 0, scale: float = 1.0) -> Workload:
+    """Build configuration `index` (1..5).  `scale` < 1 shrinks node and edge
+    counts proportionally (feature widths, class counts and degree shape are
+    kept) so that CPU-side tests can run a small copy of the large graphs."""
+    ss = np.random.SeedSequence([seed, index])
+    s_graph, s_feat, s_lab, s_split, s_part = [np.random.default_rng(s) for s in ss.spawn(5)]
+
+    if index == 1:
+        n = _scaled(2708, scale, 70)
+        n_und = _scaled(5278, scale, 100)
+        labels = (np.arange(n) * 7 // n).astype(np.int32)
+        labels = labels[s_lab.permutation(n)]
+        rowptr, colidx = random_graph(s_graph, n, n_und, labels, None, 0.8, None)
+        feats = _bag_of_words(s_feat, labels, 1433, 19, 200, 0.4)
+        tr, va, te = _split_per_class(s_split, labels, 20 if scale == 1.0 else 5,
+                                      _scaled(500, scale, 20), _scaled(1000, scale, 20))
+        part = np.arange(n, dtype=np.int32)
+        return Workload("cfg1_gcn_cora_like", GCN, 3, 100, 64, 7, 0.003, n, rowptr, colidx, feats,
+                        labels, tr, va, te, part, n, seed=seed)
+
+    if index == 2:
+        n = _scaled(19717, scale, 100)
+        n_und = _scaled(44324, scale, 200)
+        labels = s_lab.integers(0, 3, size=n).astype(np.int32)
+        w = _power_law_weights(n, 2.5, None)
+        rowptr, colidx = random_graph(s_graph, n, n_und, labels, w, None, 0.25)
+        feats = _tfidf_like(s_feat, labels, 500, 50, 120, 0.35)
+        tr, va, te = _split_per_class(s_split, labels, 20, _scaled(500, scale, 20), _scaled(1000, scale, 20))
+        part = s_part.integers(0, 100, size=n).astype(np.int32)
+        return Workload("cfg2_sage_pubmed_like", SAGE_MEAN, 3, 100, 128, 3, 0.003, n, rowptr, colidx,
+                        feats, labels, tr, va, te, part, 100, seed=seed)
+
+    if index == 3:
+        n = _scaled(22470, scale, 100)
+        n_und = _scaled(171002, scale, 400)
+        labels = s_lab.integers(0, 4, size=n).astype(np.int32)
+        mean_deg = 2.0 * n_und / n
+        w = _power_law_weights(n, 2.5, min(700.0, n / 4) / mean_deg)
+        rowptr, colidx = random_graph(s_graph, n, n_und, labels, w, None, 0.25)
+        feats = _gaussian_features(s_feat, labels, 128, 0.5 * np.sqrt(8.0))
+        tr, va, te = _split_fraction(s_split, n, 0.50, 0.25)
+        part = np.arange(n, dtype=np.int32)
+        return Workload("cfg3_gat_fbpage_like", GAT, 2, 100, 64, 4, 0.003, n, rowptr, colidx, feats,
+                        labels, tr, va, te, part, n, heads=4, head_dim=16, seed=seed)
+
+    if index == 4:
+        n = _scaled(232965, scale, 400)
+        n_und = min(_scaled(57_300_000, scale, 2000), n * (n - 1) // 8)
+        labels = s_lab.integers(0, 41, size=n).astype(np.int32)
+        mean_deg = 2.0 * n_und / n
+        w = _power_law_weights(n, 2.5, min(20000.0, n / 6) / mean_deg)
+        rowptr, colidx = random_graph(s_graph, n, n_und, labels, w, 0.7, None)
+        feats = _gaussian_features(s_feat, labels, 602, 0.5 * np.sqrt(8.0))
+        tr, va, te = _split_fraction(s_split, n, 0.66, 0.10)
+        part = s_part.integers(0, 1000, size=n).astype(np.int32)
+        return Workload("cfg4_sage_reddit_like", SAGE_MEAN, 3, 200, 256, 41, 0.01, n, rowptr, colidx,
+                        feats, labels, tr, va, te, part, 1000, seed=seed)
+
+    if index == 5:
+        n = _scaled(2_449_029, scale, 1000)
+        n_und = _scaled(61_900_000, scale, 5000)
+        labels = _zipf_labels(s_lab, n, 47)
+        w = _power_law_weights(n, 2.5, None)
+        rowptr, colidx = random_graph(s_graph, n, n_und, labels, w, 0.6, None)
+        feats = _gaussian_features(s_feat, labels, 100, 0.5 * np.sqrt(8.0))
+        tr, va, te = _split_fraction(s_split, n, 0.08, 0.02)
+        part = np.arange(n, dtype=np.int32)
+        return Workload("cfg5_gcn_products_like", GCN, 3, 200, 256, 47, 0.003, n, rowptr, colidx,
+                        feats, labels, tr, va, te, part, n, seed=seed)
+
+    raise ValueError("config index must be 1..5")
+
+
+# --------------------------------------------------------------------------
+# initial weights (inputs to both the checker and the CUDA path)
+# --------------------------------------------------------------------------
+
+def glorot(rng, fan_in: int, fan_out: int) -> np.ndarray:
+    lim = np.sqrt(6.0 / (fan_in + fan_out))
+    return rng.uniform(-lim, lim, size=(fan_in, fan_out)).astype(np.float32)
+
+
+def initial_weights(wl: Workload, seed: Optional[int] = None) -> List[Dict[str, np.ndarray]]:
+    """Glorot-uniform draws for each round's per-node model, row-major
+    [in x out]; for GAT also the frozen projection and attention vectors."""
+    ss = np.random.SeedSequence([wl.seed if seed is None else seed, 7919])
+    rngs = [np.random.default_rng(s) for s in ss.spawn(wl.K)]
+    out = []
+    for rd, rng in zip(wl.round_dims(), rngs):
+        w: Dict[str, np.ndarray] = {}
+        if wl.aggr == GAT:
+            hd = wl.heads * wl.head_dim
+            w["w_att"] = glorot(rng, rd["rep_dim"], hd)
+            w["a_src"] = glorot(rng, wl.head_dim, wl.heads).T.copy()   # [heads, head_dim]
+            w["a_dst"] = glorot(rng, wl.head_dim, wl.heads).T.copy()
+        if rd["hidden"] > 0:
+            w["w1"] = glorot(rng, rd["d_in"], rd["hidden"])
+            w["b1"] = np.zeros(rd["hidden"], dtype=np.float32)
+            w["w2"] = glorot(rng, rd["hidden"], wl.n_classes)
+            w["b2"] = np.zeros(wl.n_classes, dtype=np.float32)
+        else:
+            w["w1"] = glorot(rng, rd["d_in"], wl.n_classes)
+            w["b1"] = np.zeros(wl.n_classes, dtype=np.float32)
+        out.append(w)
+    return out
+
+
+# --------------------------------------------------------------------------
+# small hand-sized graphs for edge-case tests
+# --------------------------------------------------------------------------
+
+def csr_from_edge_list(n: int, edges) -> tuple:
+    e = np.asarray(list(edges), dtype=np.int64).reshape(-1, 2)
+    if e.shape[0] == 0:
+        return np.zeros(n + 1, dtype=np.int64), np.zeros(0, dtype=np.int32)
+    lo = np.minimum(e[:, 0], e[:, 1])
+    hi = np.maximum(e[:, 0], e[:, 1])
+    keep = lo != hi
+    keys = np.unique(lo[keep] * n + hi[keep])
+    return csr_from_undirected(n, keys // n, keys % n)
+
+
+def ring_graph(n: int):
+    return csr_from_edge_list(n, [(i, (i + 1) % n) for i in range(n)])
+
+
+def complete_graph(n: int):
+    return csr_from_edge_list(n, [(i, j) for i in range(n) for j in range(i + 1, n)])
+
+
+def star_graph(n_leaves: int):
+    return csr_from_edge_list(n_leaves + 1, [(0, i) for i in range(1, n_leaves + 1)])
+
+
+def degree_ladder_graph(degrees, seed: int = 0):
+    """A graph with one hub per entry of `degrees`, each hub attached to that
+    many private leaves, plus one isolated node at the end.  Used to cross
+    every degree bin of the aggregation kernels (0, 1, 2, 33, 1025, ...)."""
+    edges = []
+    nxt = len(degrees)
+    for h, d in enumerate(degrees):
+        for _ in range(d):
+            edges.append((h, nxt))
+            nxt += 1
+    n = nxt + 1
+    rng = np.random.default_rng(seed)
+    perm = rng.permutation(n)
+    e = np.asarray(edges, dtype=np.int64).reshape(-1, 2)
+    rowptr, colidx = csr_from_edge_list(n, perm[e] if e.size else [])
+    return n, rowptr, colidx, perm
+
+
+def random_small_graph(n: int, n_und: int, seed: int = 0):
+    rng = np.random.default_rng(seed)
+    labels = np.zeros(n, dtype=np.int32)
+    n_und = min(n_und, n * (n - 1) // 2)
+    rowptr, colidx = random_graph(rng, n, n_und, labels, None, None, None)
+    return rowptr, colidx

@@ -1,0 +1,60 @@
+"""The K-round lazy-message-passing loop of the CPU checker (Section 3.1)."""
+import numpy as np
+
+import oracle
+from paper_2302_13053_b200 import workloads as wl
+
+
+def run(w, R, **kw):
+    gat = dict(heads=w.heads, head_dim=w.head_dim, negative_slope=w.negative_slope,
+               add_self_loop=1) if w.aggr == wl.GAT else None
+    return oracle.lmp_train(w.aggr, w.K, R, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features,
+                            w.labels, w.train_idx, w.val_idx, w.test_idx, wl.initial_weights(w), gat=gat,
+                            part=w.part, n_parts=w.n_parts, **kw)
+
+
+def test_loop_issues_k_aggregations_and_k_times_r_steps():
+    for idx, scale in ((1, 0.2), (2, 0.05), (3, 0.05)):
+        w = wl.make_config(idx, scale=scale)
+        rep = run(w, 4)
+        assert rep["n_aggregations"] == w.K          # one message-passing round per layer
+        assert rep["n_steps"] == w.K * 4
+        dims = [r["x"].shape[1] for r in rep["rounds"]]
+        assert dims == [d["d_in"] for d in w.round_dims()]
+        assert rep["rounds"][-1]["logits"].shape == (w.n_nodes, w.n_classes)
+        for r in rep["rounds"][:-1]:
+            assert r["q_out"].shape == (w.n_nodes, w.hidden) and (r["q_out"] >= 0).all()
+
+
+def test_best_validation_iterate_is_the_earliest_maximum():
+    w = wl.make_config(1, scale=0.3)
+    rep = run(w, 12)
+    for r in rep["rounds"]:
+        assert r["best_iter"] == int(np.argmax(r["val_correct"])) + 1
+        assert r["best_val_correct"] == r["val_correct"].max()
+
+
+def test_more_rounds_help_when_features_are_weak_and_homophily_is_strong():
+    """Qualitative claim of Sections 3.1 / 4.2: a further hop adds signal."""
+    rng = np.random.default_rng(0)
+    n, o = 600, 3
+    labels = rng.integers(0, o, n).astype(np.int32)
+    rowptr, colidx = wl.random_graph(rng, n, 2400, labels, None, 0.9, None)
+    feats = (0.35 * np.eye(o)[labels] + rng.standard_normal((n, o))).astype(np.float32)
+    tr, va, te = wl._split_fraction(rng, n, 0.3, 0.2)
+    acc = {}
+    for K in (1, 3):
+        ws = []
+        d = o
+        for m in range(K):
+            hid = 16 if m < K - 1 else 0
+            r2 = np.random.default_rng(m)
+            w = dict(w1=wl.glorot(r2, d, hid or o), b1=np.zeros(hid or o, dtype=np.float32))
+            if hid:
+                w["w2"], w["b2"] = wl.glorot(r2, hid, o), np.zeros(o, dtype=np.float32)
+            ws.append(w)
+            d = hid
+        rep = oracle.lmp_train(oracle.GCN, K, 60, 16, o, 0.02, rowptr, colidx, feats, labels, tr, va, te, ws,
+                               round_bf16=False)
+        acc[K] = rep["test_acc"]
+    assert acc[3] > acc[1] + 0.05, acc
