@@ -1,0 +1,295 @@
+/*
+ * retexo.h — C ABI of the on-device hot path of lazy message passing (LMP),
+ * the layer-by-layer GNN training order of "Scalable Neural Network Training
+ * over Distributed Graphs" (Retexo).
+ *
+ * One LMP round m = 1..K (Section 3.1) is, on the device:
+ *   1. one full-graph neighbour aggregation of the previous representations
+ *      Q^{m-1} (Eq. 1: AGGR + COMBINE)                   -> retexo_aggregate
+ *   2. R full-batch training iterations of the per-node model
+ *      (f_theta = Linear+ReLU, temporary classifier C_theta = Linear; the last
+ *      round is a single Linear)                          -> retexo_mlp_train_step
+ *   3. emission of Q^m = ReLU(X W1 + b1) with the classifier dropped, or of
+ *      logits / predictions / accuracy                    -> retexo_embed
+ * and, once per graph + partition, the number of boundary-node messages and
+ * bytes one round sends across the partition (Section 2.1, Appendix A.1)
+ *                                                         -> retexo_cross_partition_bytes
+ * retexo_lmp_train runs the whole K-round loop on the device.
+ *
+ * General rules
+ *   - Plain C, no exceptions.  Every function returns a retexo_status
+ *     (RETEXO_OK = 0); retexo_status_string names it.
+ *   - Unless a parameter says "host", every array pointer is a DEVICE pointer
+ *     owned by the caller.  The library never allocates or frees device
+ *     memory: scratch comes from the caller's `workspace` (size from the
+ *     matching *_workspace_size query, 256-byte aligned).
+ *   - Work is enqueued on the caller's stream (`stream` is a cudaStream_t
+ *     passed as void*, NULL = default stream) without synchronising, except
+ *     where stated.  Scalar results go to caller-provided device memory.
+ *   - Arguments are validated on the host first; a call that returns an error
+ *     other than RETEXO_ERR_CUDA has launched nothing.  Inputs are never
+ *     modified.  There is no CPU fallback: without a CUDA device every
+ *     compute call fails with RETEXO_ERR_CUDA.
+ *   - Results are deterministic: no floating-point atomics are used, so the
+ *     same inputs give the same bits on every call.
+ *   - Graphs are symmetric CSR (both directions of each undirected edge
+ *     stored; Section 2.1: graphs are undirected), without self loops or
+ *     duplicate entries, column indices ascending inside a row.
+ */
+#ifndef RETEXO_H
+#define RETEXO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum retexo_status {
+    RETEXO_OK = 0,
+    RETEXO_ERR_INVALID_ARG = 1,   /* null pointer, negative size, bad enum, ld too small */
+    RETEXO_ERR_BAD_GRAPH = 2,     /* reported by retexo_validate_csr */
+    RETEXO_ERR_ALIGNMENT = 3,     /* a pointer / leading dimension breaks a stated alignment rule */
+    RETEXO_ERR_WORKSPACE = 4,     /* workspace NULL, misaligned or too small */
+    RETEXO_ERR_UNSUPPORTED = 5,   /* shape outside what the kernels cover (stated per call) */
+    RETEXO_ERR_CUDA = 6,          /* a CUDA runtime call or launch failed / no device */
+    RETEXO_ERR_TIMEOUT = 7        /* a bounded device-side wait gave up (status word set) */
+} retexo_status;
+
+const char* retexo_status_string(int status);
+/* Library version, major*10000 + minor*100 + patch. */
+int retexo_version(void);
+
+/* ------------------------------------------------------------------ graph */
+typedef struct retexo_csr {
+    int64_t n_nodes;
+    int64_t n_edges;          /* = rowptr[n_nodes]; directed count = 2 |E_undirected| */
+    const int64_t* rowptr;    /* device, [n_nodes + 1] */
+    const int32_t* colidx;    /* device, [n_edges] */
+} retexo_csr;
+
+/* Checks rowptr[0] == 0, rowptr monotone, rowptr[n] == n_edges, 0 <= colidx < n,
+ * no self loop, strictly ascending columns inside a row.  Writes to
+ * status_out (device, int64[2]): [0] = number of violations found,
+ * [1] = index (row or edge) of one of them (-1 if none).  Host reads it after
+ * synchronising.  Needs no workspace. */
+int retexo_validate_csr(const retexo_csr* g, int64_t* status_out, void* stream);
+
+/* ------------------------------------------------------------ aggregation */
+typedef enum retexo_aggr { RETEXO_GCN = 0, RETEXO_SAGE_MEAN = 1, RETEXO_GAT = 2 } retexo_aggr;
+
+typedef struct retexo_gat_params {
+    int32_t heads, head_dim;        /* dim must equal heads * head_dim; heads <= 8 */
+    const float* a_src;             /* device, [heads x head_dim], applied to the neighbour u */
+    const float* a_dst;             /* device, [heads x head_dim], applied to the destination v */
+    float negative_slope;           /* LeakyReLU slope of the edge score */
+    int32_t add_self_loop;          /* 1: v attends over N(v) and itself */
+} retexo_gat_params;
+
+size_t retexo_aggregate_workspace_size(int64_t n_nodes, int64_t n_edges, int32_t type, int32_t dim,
+                                       int32_t heads);
+
+/* One message-passing round over the whole graph: the AGGR (+ COMBINE) of
+ * Eq. 1 applied to q = Q^{m-1} (fp32, row-major, row stride ldq >= dim).
+ *   RETEXO_GCN       out[v] = n_v ( n_v q[v] + sum_{u in N(v)} n_u q[u] ),
+ *                    n_x = (deg x + 1)^-1/2  (symmetric normalisation with an
+ *                    implicit self loop); out is [n x dim].
+ *   RETEXO_SAGE_MEAN mean[v] = (1/deg v) sum_{u in N(v)} q[u], zeros if
+ *                    deg v = 0.  concat_self = 1: out is [n x 2 dim] with
+ *                    q[v] in columns [0,dim) and the mean in [dim, 2 dim)
+ *                    (COMBINE = concatenation); concat_self = 0: out is
+ *                    [n x dim], the mean only.
+ *   RETEXO_GAT       q holds already projected rows, head k in columns
+ *                    [k*head_dim, (k+1)*head_dim).  Per head:
+ *                    e_uv = LeakyReLU(<a_src,q_u> + <a_dst,q_v>),
+ *                    alpha = softmax over u in N(v) (+ v), out[v] = sum alpha q[u];
+ *                    scores, softmax and weighted sum happen in one pass.
+ *                    Rows with an empty softmax set give zeros.  dim <= 256.
+ * out      fp32 [n x ldout], may be NULL if out_bf16 is given.
+ * out_bf16 optional bf16 (round-to-nearest-even) copy of the same matrix,
+ *          row stride ldout_bf16 elements; NULL if not wanted.
+ * Sums are taken in CSR order per row in fp32; rows of at least 2048 entries
+ * are split over the warps of one block and combined in a fixed order.
+ * 128-bit loads are used when q is 16-byte aligned, ldq % 4 == 0 and
+ * ldq >= round_up(dim, 4); 64-bit loads under the analogous rule; otherwise
+ * scalar loads.  Nothing is an error for being unaligned.
+ * dim <= 4096.  Errors: INVALID_ARG, WORKSPACE, UNSUPPORTED. */
+int retexo_aggregate(const retexo_csr* g, int32_t type,
+                     const float* q, int64_t ldq, int32_t dim,
+                     const retexo_gat_params* gat,
+                     float* out, int64_t ldout, int32_t concat_self,
+                     void* out_bf16, int64_t ldout_bf16,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+/* --------------------------------------------------------- per-node model */
+typedef enum retexo_optimizer { RETEXO_SGD = 0, RETEXO_ADAM = 1 } retexo_optimizer;
+
+/* The trainable part of round m (Section 3.1).  theta is one flat fp32
+ * device array, matrices row-major [in x out]:
+ *   hidden > 0 : [ W1 (d_in x hidden) | b1 (hidden) | W2 (hidden x n_classes) | b2 (n_classes) ]
+ *   hidden == 0: [ W1 (d_in x n_classes) | b1 (n_classes) ]       (last round)
+ * adam_m / adam_v have the same length (NULL for SGD).  `step` counts the
+ * updates already applied; retexo_mlp_train_step increments it.
+ * Every matrix product takes both operands rounded to bf16 and accumulates in
+ * fp32; biases, softmax, loss and the optimiser are fp32. */
+typedef struct retexo_mlp {
+    int32_t d_in, hidden, n_classes;
+    float* theta;
+    float* adam_m;
+    float* adam_v;
+    int32_t optimizer;              /* retexo_optimizer */
+    float lr, beta1, beta2, eps;    /* Adam: bias-corrected, eps outside the root, no weight decay */
+    int64_t step;
+} retexo_mlp;
+
+int64_t retexo_theta_size(int32_t d_in, int32_t hidden, int32_t n_classes);
+
+/* Gathers rows of a matrix into a dense bf16 batch: dst[i] = bf16(src[idx ? idx[i] : i]).
+ * src is fp32 (src_is_bf16 = 0) or bf16 (1), row stride ld_src elements;
+ * dst is bf16 [n_rows x ld_dst], ld_dst >= dim; columns [dim, ld_dst) are
+ * zero-filled.  dst_t (optional) receives the transpose, bf16 [dim x ld_t],
+ * ld_t >= n_rows, columns [n_rows, ld_t) zero-filled.  Needs no workspace. */
+int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld_src, int32_t dim,
+                     const int32_t* idx, int64_t n_rows,
+                     void* dst, int64_t ld_dst, void* dst_t, int64_t ld_t, void* stream);
+
+size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes,
+                                            int64_t n_rows);
+
+/* One full-batch training iteration (Section 2.3: forward, loss, backward,
+ * update; with a single worker the gradient average is the identity):
+ *   hidden > 0 : Hd = ReLU(X W1 + b1), L = Hd W2 + b2
+ *   hidden == 0: L = X W1 + b1
+ *   loss = mean_i CE(softmax(L_i), y_i), gradients by back-propagation,
+ *   then one SGD / Adam update of theta in place.
+ * x     bf16 [n_rows x ldx]: the batch, one training node per row
+ *       (retexo_pack_rows builds it once per round); ldx % 8 == 0 and x
+ *       16-byte aligned.
+ * x_t   optional bf16 [d_in x ld_xt] transpose of x (ld_xt % 8 == 0), lets the
+ *       weight-gradient product stream both operands along the batch; NULL
+ *       is allowed.
+ * y     int32 [n_rows] labels in [0, n_classes).
+ * loss_out  device float, the loss before the update (may be NULL).
+ * grad_out  optional device fp32 array shaped like theta: the gradient.
+ * Increments model->step (host struct).  n_classes <= 64, hidden <= 512.
+ * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED. */
+int retexo_mlp_train_step(retexo_mlp* model,
+                          const void* x, int64_t ldx, const void* x_t, int64_t ld_xt,
+                          const int32_t* y, int64_t n_rows,
+                          float* loss_out, float* grad_out,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+size_t retexo_embed_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows);
+
+/* Forward of the per-node model over rows x[row_idx ? row_idx[i] : i]
+ * (x bf16, row stride ldx, 16-byte aligned, ldx % 8 == 0):
+ *   hidden_out / hidden_out_bf16 : ReLU(x W1 + b1), i.e. the representation
+ *       Q^m handed to the next round once the classifier is dropped
+ *       (requires hidden > 0); fp32 [n_rows x ld_hidden] and/or bf16
+ *       [n_rows x ld_hidden_bf16];
+ *   logits_out : fp32 [n_rows x ld_logits];
+ *   pred_out   : int32 [n_rows], argmax of the fp32 logits, lowest class on ties;
+ *   correct_out: uint64, number of rows with pred == y[i] (y: int32 [n_rows]).
+ * Every output pointer may be NULL.  With hidden > 0 and only hidden outputs
+ * requested the classifier is not evaluated. */
+int retexo_embed(const retexo_mlp* model,
+                 const void* x, int64_t ldx, const int32_t* row_idx, int64_t n_rows,
+                 float* hidden_out, int64_t ld_hidden,
+                 void* hidden_out_bf16, int64_t ld_hidden_bf16,
+                 float* logits_out, int64_t ld_logits,
+                 int32_t* pred_out, const int32_t* y, uint64_t* correct_out,
+                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------ cross-partition traffic */
+size_t retexo_cross_partition_workspace_size(int64_t n_nodes, int64_t n_edges, int32_t n_parts);
+
+/* Messages and bytes one LMP round sends across a given node partition.
+ * A message is one (node u, destination partition p) pair with p != part[u]
+ * and some neighbour of u living in p: u is a boundary node of worker p
+ * (Section 2.1) and its representation crosses once per round (Appendix A.1).
+ *   cross_edges     = #{CSR entries (u,v) : part[u] != part[v]}
+ *   boundary_pairs  = number of distinct such pairs = sum over workers of B_i
+ *   bytes_per_round[m] = boundary_pairs * dims[m] * elem_bytes, m = 0..K-1,
+ *                        dims[m] = width of the representation sent in round m+1
+ *   bytes_total     = sum over rounds; the appendix' DV^lazy_lt counts each
+ *                     message at sender and receiver, i.e. 2 * bytes_total
+ *   send_per_part[p] = pairs whose node lives in p; recv_per_part[p] = pairs
+ *                     destined to p (= B_p).  Optional, uint64 [n_parts].
+ * part: int32 [n_nodes] with values in [0, n_parts) (a value outside that range
+ * sets every scalar output to UINT64_MAX); dims: HOST int32 [K].
+ * All outputs are device uint64, exact.  Errors: INVALID_ARG, WORKSPACE. */
+int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* part, int32_t n_parts,
+                                 int32_t K, const int32_t* dims, int32_t elem_bytes,
+                                 uint64_t* cross_edges, uint64_t* boundary_pairs,
+                                 uint64_t* bytes_per_round, uint64_t* bytes_total,
+                                 uint64_t* send_per_part, uint64_t* recv_per_part,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+
+/* -------------------------------------------------- the K-round LMP loop */
+typedef struct retexo_lmp_config {
+    int32_t aggr;                   /* retexo_aggr */
+    int32_t K;                      /* rounds = GNN layers, 1..8 */
+    int32_t R;                      /* training iterations per round */
+    int32_t d0;                     /* feature width */
+    int32_t hidden;                 /* width of Q^1..Q^{K-1} */
+    int32_t n_classes;
+    int32_t optimizer;
+    float lr, beta1, beta2, eps;
+    int32_t eval_every;             /* validate every this many iterations (and at the last) */
+    int32_t gat_heads, gat_head_dim;
+    float gat_negative_slope;
+    int32_t memory_is_host;         /* 0: every input array below is on the device;
+                                       1: every input array is in HOST memory and is copied to the
+                                          device inside the call; results are also written to host */
+} retexo_lmp_config;
+
+typedef struct retexo_lmp_inputs {
+    retexo_csr graph;
+    const float* features; int64_t ld_features;       /* fp32 [n x ld] */
+    const int32_t* labels;                            /* [n] */
+    const int32_t* train_idx; int64_t n_train;
+    const int32_t* val_idx;   int64_t n_val;
+    const int32_t* test_idx;  int64_t n_test;
+    const int32_t* part; int32_t n_parts;             /* may be NULL: skip the count */
+    const float* const* theta0;    /* HOST array of K pointers to the initial theta of each round
+                                      (pointees: device or host memory, like the other inputs) */
+    const float* const* gat_w;     /* GAT only: HOST array of K pointers, each to
+                                      [rep_dim x heads*head_dim | a_src | a_dst] fp32 (frozen) */
+} retexo_lmp_inputs;
+
+typedef struct retexo_lmp_outputs {
+    float* loss_history;            /* [K*R] loss of every iteration */
+    uint64_t* val_correct;          /* [K*R] validation hits per iteration (UINT64_MAX where not evaluated) */
+    uint64_t* best_val_correct;     /* [K] */
+    int32_t* best_iter;             /* [K] 1-based iteration whose model was kept */
+    uint64_t* test_correct;         /* [K] test hits of the kept model of each round */
+    uint64_t* test_correct_last;    /* [K] test hits of the last iterate */
+    uint64_t* counts;               /* [4 + K]: cross_edges, boundary_pairs, bytes_total, 2*bytes_total,
+                                       then bytes_per_round; untouched if part == NULL */
+    float* final_logits; int64_t ld_logits;   /* [n x ld] logits of the last round's kept model; may be NULL */
+    int32_t* final_pred;            /* [n]; may be NULL */
+    float* const* theta_best;       /* HOST array of K pointers receiving each round's kept theta; may be NULL */
+} retexo_lmp_outputs;
+
+size_t retexo_lmp_workspace_size(const retexo_lmp_config* cfg, int64_t n_nodes, int64_t n_edges,
+                                 int64_t n_train, int64_t n_val, int64_t n_test, int32_t n_parts);
+
+/* Lazy message passing (Section 3.1), entirely on the device: for m = 1..K
+ * { aggregate Q^{m-1} once; train the round's per-node model for R iterations
+ *   from theta0[m]; every eval_every iterations measure validation accuracy
+ *   and keep the iterate with the most hits (earliest on ties); emit Q^m from
+ *   the kept model (last round: logits, predictions, test accuracy) }.
+ * GAT: the round's projection and attention vectors (gat_w[m]) are fixed
+ * draws, P = Q^{m-1} W_att is computed once, then aggregated.
+ * With memory_is_host = 0 the call only enqueues work (outputs are device
+ * memory); with 1 it copies inputs in, runs, copies outputs to the host
+ * arrays and synchronises the stream before returning. */
+int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_inputs* in,
+                     const retexo_lmp_outputs* out,
+                     void* workspace, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RETEXO_H */

@@ -1,0 +1,481 @@
+// Full-graph neighbour aggregation of one message-passing round (Eq. 1):
+// GCN symmetric-normalised sum, GraphSAGE mean (+ self concat), and the fused
+// GAT edge-score / segment-softmax / weighted-sum pass, over a CSR graph.
+//
+// The work is a gather-reduce bound by the memory system, not a dense
+// contraction: rows are streamed with the widest aligned vector loads, one
+// warp per destination row (a whole block for rows of >= kHeavyDegree
+// entries), several neighbour rows in flight per lane, sums in registers.
+#include "common.cuh"
+
+namespace retexo {
+
+constexpr int kHeavyDegree = 2048;     // rows at least this long get a whole block
+constexpr int kAggThreads = 256;
+constexpr int kAggWarps = kAggThreads / kWarp;
+constexpr int kUnroll = 4;             // neighbour rows in flight per lane and column chunk
+
+// ---------------------------------------------------------------- pre-pass
+// coef[v]: GCN (deg+1)^-1/2, SAGE 1/deg (0 for isolated nodes).  Also lists
+// the heavy rows (order irrelevant: each row's result does not depend on it).
+__global__ void prep_rows_kernel(int64_t n, const int64_t* __restrict__ rowptr, int mode,
+                                 float* __restrict__ coef, int32_t* __restrict__ heavy_list,
+                                 int32_t* __restrict__ heavy_count) {
+    int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (v >= n) return;
+    int64_t deg = rowptr[v + 1] - rowptr[v];
+    float c;
+    if (mode == RETEXO_GCN) c = 1.0f / sqrtf((float)deg + 1.0f);
+    else c = deg > 0 ? 1.0f / (float)deg : 0.0f;
+    coef[v] = c;
+    if (deg >= kHeavyDegree) {
+        int32_t slot = atomicAdd(heavy_count, 1);
+        heavy_list[slot] = (int32_t)v;
+    }
+}
+
+// ---------------------------------------------------------------- vectors
+template <int VEC> struct VecT;
+template <> struct VecT<4> { using type = float4; };
+template <> struct VecT<2> { using type = float2; };
+template <> struct VecT<1> { using type = float; };
+
+template <int VEC>
+__device__ __forceinline__ void vec_zero(typename VecT<VEC>::type& a);
+template <> __device__ __forceinline__ void vec_zero<4>(float4& a) { a = make_float4(0.f, 0.f, 0.f, 0.f); }
+template <> __device__ __forceinline__ void vec_zero<2>(float2& a) { a = make_float2(0.f, 0.f); }
+template <> __device__ __forceinline__ void vec_zero<1>(float& a) { a = 0.f; }
+
+__device__ __forceinline__ void vec_fma(float4& a, float w, const float4& x) {
+    a.x = fmaf(w, x.x, a.x); a.y = fmaf(w, x.y, a.y); a.z = fmaf(w, x.z, a.z); a.w = fmaf(w, x.w, a.w);
+}
+__device__ __forceinline__ void vec_fma(float2& a, float w, const float2& x) {
+    a.x = fmaf(w, x.x, a.x); a.y = fmaf(w, x.y, a.y);
+}
+__device__ __forceinline__ void vec_fma(float& a, float w, const float& x) { a = fmaf(w, x, a); }
+__device__ __forceinline__ void vec_add(float4& a, const float4& x) { a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w; }
+__device__ __forceinline__ void vec_add(float2& a, const float2& x) { a.x += x.x; a.y += x.y; }
+__device__ __forceinline__ void vec_add(float& a, const float& x) { a += x; }
+
+template <int VEC>
+__device__ __forceinline__ float vec_get(const typename VecT<VEC>::type& a, int i);
+template <> __device__ __forceinline__ float vec_get<4>(const float4& a, int i) {
+    return i == 0 ? a.x : i == 1 ? a.y : i == 2 ? a.z : a.w;
+}
+template <> __device__ __forceinline__ float vec_get<2>(const float2& a, int i) { return i == 0 ? a.x : a.y; }
+template <> __device__ __forceinline__ float vec_get<1>(const float& a, int) { return a; }
+
+struct AggArgs {
+    int64_t n;
+    const int64_t* rowptr;
+    const int32_t* colidx;
+    const float* q;
+    int64_t ldq;
+    int32_t dim;
+    const float* coef;
+    float* out;             // may be null
+    int64_t ldout;
+    __nv_bfloat16* out16;   // may be null
+    int64_t ldout16;
+    int32_t concat_self;    // SAGE
+    const int32_t* heavy_list;
+    const int32_t* heavy_count;
+};
+
+// Adds the neighbour rows of CSR entries [beg, end) into acc, in order, for the
+// column vectors this lane owns in pass `pass`.  GCN weighs each row by coef[u].
+template <int VEC, int CH, bool GCN>
+__device__ __forceinline__ void accumulate_range(const AggArgs& a, int64_t beg, int64_t end, int lane,
+                                                 int vec0, int nvec,
+                                                 typename VecT<VEC>::type (&acc)[CH]) {
+    using V = typename VecT<VEC>::type;
+    const int64_t ldv = a.ldq / VEC;
+    const V* __restrict__ qv = reinterpret_cast<const V*>(a.q);
+    for (int64_t e0 = beg; e0 < end; e0 += kWarp) {
+        const int cnt = (int)min((int64_t)kWarp, end - e0);
+        int my_u = 0;
+        float my_w = 0.f;
+        if (lane < cnt) {
+            my_u = __ldg(a.colidx + e0 + lane);
+            if (GCN) my_w = __ldg(a.coef + my_u);
+        }
+        int j = 0;
+        for (; j + kUnroll <= cnt; j += kUnroll) {
+            V x[kUnroll][CH];
+            float w[kUnroll];
+#pragma unroll
+            for (int t = 0; t < kUnroll; ++t) {
+                const int u = __shfl_sync(0xffffffffu, my_u, j + t);
+                if (GCN) w[t] = __shfl_sync(0xffffffffu, my_w, j + t);
+                const V* row = qv + (int64_t)u * ldv;
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    const int vi = vec0 + c * kWarp + lane;
+                    if (vi < nvec) x[t][c] = __ldg(row + vi);
+                    else vec_zero<VEC>(x[t][c]);
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < kUnroll; ++t)
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    if (GCN) vec_fma(acc[c], w[t], x[t][c]);
+                    else vec_add(acc[c], x[t][c]);
+                }
+        }
+        for (; j < cnt; ++j) {
+            const int u = __shfl_sync(0xffffffffu, my_u, j);
+            float w = 0.f;
+            if (GCN) w = __shfl_sync(0xffffffffu, my_w, j);
+            const V* row = qv + (int64_t)u * ldv;
+#pragma unroll
+            for (int c = 0; c < CH; ++c) {
+                const int vi = vec0 + c * kWarp + lane;
+                if (vi < nvec) {
+                    V x = __ldg(row + vi);
+                    if (GCN) vec_fma(acc[c], w, x);
+                    else vec_add(acc[c], x);
+                }
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void store_elem(const AggArgs& a, int64_t v, int col, float val) {
+    if (a.out) a.out[v * a.ldout + col] = val;
+    if (a.out16) a.out16[v * a.ldout16 + col] = f32_to_bf16(val);
+}
+
+// Finishes row v for the column vectors of this lane: GCN adds the self term
+// and scales, SAGE divides by the degree and (optionally) copies the self row.
+template <int VEC, int CH, bool GCN>
+__device__ __forceinline__ void finish_row(const AggArgs& a, int64_t v, int lane, int vec0, int nvec,
+                                           typename VecT<VEC>::type (&acc)[CH]) {
+    using V = typename VecT<VEC>::type;
+    const V* __restrict__ self = reinterpret_cast<const V*>(a.q) + v * (a.ldq / VEC);
+    const float cv = a.coef[v];
+    const int64_t deg = a.rowptr[v + 1] - a.rowptr[v];
+#pragma unroll
+    for (int c = 0; c < CH; ++c) {
+        const int vi = vec0 + c * kWarp + lane;
+        if (vi >= nvec) continue;
+        const V s = self[vi];
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) {
+            const int col = vi * VEC + i;
+            if (col >= a.dim) continue;
+            const float sv = vec_get<VEC>(s, i);
+            const float av = vec_get<VEC>(acc[c], i);
+            if (GCN) {
+                store_elem(a, v, col, cv * fmaf(cv, sv, av));
+            } else {
+                const float mean = deg > 0 ? av / (float)deg : 0.0f;
+                if (a.concat_self) {
+                    store_elem(a, v, col, sv);
+                    store_elem(a, v, a.dim + col, mean);
+                } else {
+                    store_elem(a, v, col, mean);
+                }
+            }
+        }
+    }
+}
+
+// One warp per destination row; heavy rows are skipped here.
+template <int VEC, int CH, bool GCN>
+__global__ void __launch_bounds__(kAggThreads) agg_warp_rows_kernel(AggArgs a) {
+    using V = typename VecT<VEC>::type;
+    const int lane = threadIdx.x & 31;
+    const int64_t v = blockIdx.x * (int64_t)kAggWarps + (threadIdx.x >> 5);
+    if (v >= a.n) return;
+    const int64_t beg = a.rowptr[v], end = a.rowptr[v + 1];
+    if (end - beg >= kHeavyDegree) return;
+    const int nvec = (a.dim + VEC - 1) / VEC;
+    for (int vec0 = 0; vec0 < nvec; vec0 += CH * kWarp) {
+        V acc[CH];
+#pragma unroll
+        for (int c = 0; c < CH; ++c) vec_zero<VEC>(acc[c]);
+        accumulate_range<VEC, CH, GCN>(a, beg, end, lane, vec0, nvec, acc);
+        finish_row<VEC, CH, GCN>(a, v, lane, vec0, nvec, acc);
+    }
+}
+
+// One block per heavy row: warp w sums the w-th contiguous slice of the row's
+// entries; the slices are then added in warp order (fixed, so deterministic).
+template <int VEC, int CH, bool GCN>
+__global__ void __launch_bounds__(kAggThreads) agg_block_rows_kernel(AggArgs a) {
+    using V = typename VecT<VEC>::type;
+    __shared__ V part[kAggWarps][CH * kWarp];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n_heavy = *a.heavy_count;
+    const int nvec = (a.dim + VEC - 1) / VEC;
+    for (int h = blockIdx.x; h < n_heavy; h += gridDim.x) {
+        const int64_t v = a.heavy_list[h];
+        const int64_t beg = a.rowptr[v], end = a.rowptr[v + 1];
+        const int64_t len = end - beg;
+        // slice boundaries on multiples of 32 entries
+        const int64_t chunks = (len + kWarp - 1) / kWarp;
+        const int64_t c0 = chunks * warp / kAggWarps, c1 = chunks * (warp + 1) / kAggWarps;
+        const int64_t sbeg = beg + c0 * kWarp, send = min(end, beg + c1 * kWarp);
+        for (int vec0 = 0; vec0 < nvec; vec0 += CH * kWarp) {
+            V acc[CH];
+#pragma unroll
+            for (int c = 0; c < CH; ++c) vec_zero<VEC>(acc[c]);
+            accumulate_range<VEC, CH, GCN>(a, sbeg, send, lane, vec0, nvec, acc);
+#pragma unroll
+            for (int c = 0; c < CH; ++c) part[warp][c * kWarp + lane] = acc[c];
+            __syncthreads();
+            if (warp == 0) {
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    V s = part[0][c * kWarp + lane];
+                    for (int w = 1; w < kAggWarps; ++w) vec_add(s, part[w][c * kWarp + lane]);
+                    acc[c] = s;
+                }
+                finish_row<VEC, CH, GCN>(a, v, lane, vec0, nvec, acc);
+            }
+            __syncthreads();
+        }
+    }
+}
+
+template <int VEC, int CH, bool GCN>
+static int launch_agg(const AggArgs& a, int n_sm, cudaStream_t st) {
+    if (a.n > 0) {
+        const int64_t blocks = (a.n + kAggWarps - 1) / kAggWarps;
+        agg_warp_rows_kernel<VEC, CH, GCN><<<(unsigned)blocks, kAggThreads, 0, st>>>(a);
+        agg_block_rows_kernel<VEC, CH, GCN><<<n_sm * 2, kAggThreads, 0, st>>>(a);
+    }
+    return launch_status();
+}
+
+template <int VEC, bool GCN>
+static int dispatch_ch(const AggArgs& a, int n_sm, cudaStream_t st) {
+    const int nvec = (a.dim + VEC - 1) / VEC;
+    const int need = (nvec + kWarp - 1) / kWarp;      // column chunks for one pass
+    if (need <= 1) return launch_agg<VEC, 1, GCN>(a, n_sm, st);
+    if (need <= 2) return launch_agg<VEC, 2, GCN>(a, n_sm, st);
+    if (need <= 3) return launch_agg<VEC, 3, GCN>(a, n_sm, st);
+    if (need <= 4) return launch_agg<VEC, 4, GCN>(a, n_sm, st);
+    if (need <= 5) return launch_agg<VEC, 5, GCN>(a, n_sm, st);
+    return launch_agg<VEC, 6, GCN>(a, n_sm, st);      // wider rows: several passes of 6 chunks
+}
+
+// ---------------------------------------------------------------- GAT
+constexpr int kGatMaxHeads = 8;
+
+struct GatArgs {
+    int64_t n;
+    const int64_t* rowptr;
+    const int32_t* colidx;
+    const float* p;
+    int64_t ldp;
+    int32_t heads, head_dim, dim;
+    const float* a_src;
+    const float* a_dst;
+    float slope;
+    int32_t self_loop;
+    float* s;               // [n x heads] scratch
+    float* t;
+    float* out;
+    int64_t ldout;
+    __nv_bfloat16* out16;
+    int64_t ldout16;
+};
+
+// s_u = <a_src, p_u>, t_u = <a_dst, p_u> per head; one warp per node.
+__global__ void __launch_bounds__(kAggThreads) gat_scores_kernel(GatArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int64_t u = blockIdx.x * (int64_t)kAggWarps + (threadIdx.x >> 5);
+    if (u >= a.n) return;
+    const float* row = a.p + u * a.ldp;
+    for (int h = 0; h < a.heads; ++h) {
+        float ss = 0.f, tt = 0.f;
+        for (int j = lane; j < a.head_dim; j += kWarp) {
+            const float x = row[h * a.head_dim + j];
+            ss = fmaf(a.a_src[h * a.head_dim + j], x, ss);
+            tt = fmaf(a.a_dst[h * a.head_dim + j], x, tt);
+        }
+        ss = warp_sum(ss);
+        tt = warp_sum(tt);
+        if (lane == 0) {
+            a.s[u * a.heads + h] = ss;
+            a.t[u * a.heads + h] = tt;
+        }
+    }
+}
+
+// One warp per destination v.  Entries are taken 32 at a time: lane j scores
+// entry j for every head, the chunk maximum and the rescale of the running
+// softmax state are warp reductions (one exp per entry and head in total),
+// then all lanes add the weighted neighbour rows for the columns they own.
+template <int NC>
+__global__ void __launch_bounds__(kAggThreads) gat_rows_kernel(GatArgs a) {
+    __shared__ float p_s[kAggWarps][kWarp][kGatMaxHeads];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t v = blockIdx.x * (int64_t)kAggWarps + warp;
+    if (v >= a.n) return;
+    const int64_t beg = a.rowptr[v];
+    const int64_t deg = a.rowptr[v + 1] - beg;
+    const int64_t total = deg + (a.self_loop ? 1 : 0);
+
+    float m[kGatMaxHeads], l[kGatMaxHeads], tv[kGatMaxHeads];
+#pragma unroll
+    for (int h = 0; h < kGatMaxHeads; ++h) {
+        m[h] = -INFINITY;
+        l[h] = 0.f;
+        tv[h] = h < a.heads ? a.t[v * a.heads + h] : 0.f;
+    }
+    float acc[NC];
+    int head_of[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        acc[c] = 0.f;
+        const int col = c * kWarp + lane;
+        head_of[c] = col < a.dim ? col / a.head_dim : 0;
+    }
+
+    for (int64_t e0 = 0; e0 < total; e0 += kWarp) {
+        const int cnt = (int)min((int64_t)kWarp, total - e0);
+        int my_u = 0;
+        float e[kGatMaxHeads];
+        const bool valid = lane < cnt;
+        if (valid) my_u = (e0 + lane < deg) ? __ldg(a.colidx + beg + e0 + lane) : (int)v;
+#pragma unroll
+        for (int h = 0; h < kGatMaxHeads; ++h) {
+            e[h] = -INFINITY;
+            if (valid && h < a.heads) {
+                const float z = a.s[(int64_t)my_u * a.heads + h] + tv[h];
+                e[h] = z > 0.f ? z : a.slope * z;
+            }
+        }
+        float scale[kGatMaxHeads];
+#pragma unroll
+        for (int h = 0; h < kGatMaxHeads; ++h) {
+            scale[h] = 1.f;
+            if (h < a.heads) {
+                const float mn = fmaxf(m[h], warp_max(e[h]));     // finite: cnt >= 1
+                scale[h] = expf(m[h] - mn);                       // exp(-inf) = 0 on the first chunk
+                const float pj = valid ? expf(e[h] - mn) : 0.f;
+                l[h] = l[h] * scale[h] + warp_sum(pj);
+                m[h] = mn;
+                p_s[warp][lane][h] = pj;
+            }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            float sc = 1.f;
+#pragma unroll
+            for (int h = 0; h < kGatMaxHeads; ++h) if (h == head_of[c]) sc = scale[h];
+            acc[c] *= sc;
+        }
+        for (int j = 0; j < cnt; ++j) {
+            const int u = __shfl_sync(0xffffffffu, my_u, j);
+            const float* row = a.p + (int64_t)u * a.ldp;
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                const int col = c * kWarp + lane;
+                if (col < a.dim) acc[c] = fmaf(p_s[warp][j][head_of[c]], __ldg(row + col), acc[c]);
+            }
+        }
+        __syncwarp();
+    }
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int col = c * kWarp + lane;
+        if (col >= a.dim) continue;
+        float den = 1.f;
+#pragma unroll
+        for (int h = 0; h < kGatMaxHeads; ++h) if (h == head_of[c]) den = l[h];
+        const float val = total > 0 ? acc[c] / den : 0.f;
+        if (a.out) a.out[v * a.ldout + col] = val;
+        if (a.out16) a.out16[v * a.ldout16 + col] = f32_to_bf16(val);
+    }
+}
+
+}  // namespace retexo
+
+using namespace retexo;
+
+extern "C" size_t retexo_aggregate_workspace_size(int64_t n_nodes, int64_t n_edges, int32_t type,
+                                                  int32_t dim, int32_t heads) {
+    (void)n_edges; (void)dim;
+    Sizer s;
+    if (n_nodes < 0) return 0;
+    if (type == RETEXO_GAT) {
+        s.take<float>((size_t)n_nodes * (size_t)(heads > 0 ? heads : 1));
+        s.take<float>((size_t)n_nodes * (size_t)(heads > 0 ? heads : 1));
+    } else {
+        s.take<float>((size_t)n_nodes);        // coef
+        s.take<int32_t>((size_t)n_nodes);      // heavy row list
+        s.take<int32_t>(64);                   // heavy row count
+    }
+    return s.off + kAlign;
+}
+
+extern "C" int retexo_aggregate(const retexo_csr* g, int32_t type, const float* q, int64_t ldq, int32_t dim,
+                                const retexo_gat_params* gat, float* out, int64_t ldout,
+                                int32_t concat_self, void* out_bf16, int64_t ldout_bf16,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+    if (!g || g->n_nodes < 0 || g->n_edges < 0 || g->n_nodes > INT32_MAX) return RETEXO_ERR_INVALID_ARG;
+    if (type != RETEXO_GCN && type != RETEXO_SAGE_MEAN && type != RETEXO_GAT) return RETEXO_ERR_INVALID_ARG;
+    if (dim <= 0 || ldq < dim || (!out && !out_bf16)) return RETEXO_ERR_INVALID_ARG;
+    if (g->n_nodes > 0 && (!g->rowptr || !q || (g->n_edges > 0 && !g->colidx))) return RETEXO_ERR_INVALID_ARG;
+    const int64_t width = (type == RETEXO_SAGE_MEAN && concat_self) ? 2 * (int64_t)dim : dim;
+    if (out && ldout < width) return RETEXO_ERR_INVALID_ARG;
+    if (out_bf16 && ldout_bf16 < width) return RETEXO_ERR_INVALID_ARG;
+    if (dim > 4096) return RETEXO_ERR_UNSUPPORTED;
+    if (type == RETEXO_GAT) {
+        if (!gat || gat->heads <= 0 || gat->head_dim <= 0 || !gat->a_src || !gat->a_dst) return RETEXO_ERR_INVALID_ARG;
+        if ((int64_t)gat->heads * gat->head_dim != dim) return RETEXO_ERR_INVALID_ARG;
+        if (gat->heads > kGatMaxHeads || dim > 256) return RETEXO_ERR_UNSUPPORTED;
+    }
+    const size_t need = retexo_aggregate_workspace_size(g->n_nodes, g->n_edges, type, dim, gat ? gat->heads : 0);
+    if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
+    if (g->n_nodes == 0) return RETEXO_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return RETEXO_ERR_CUDA;
+    Arena ws(workspace, workspace_bytes);
+    const int64_t n = g->n_nodes;
+
+    if (type == RETEXO_GAT) {
+        GatArgs a;
+        a.n = n; a.rowptr = g->rowptr; a.colidx = g->colidx; a.p = q; a.ldp = ldq;
+        a.heads = gat->heads; a.head_dim = gat->head_dim; a.dim = dim;
+        a.a_src = gat->a_src; a.a_dst = gat->a_dst; a.slope = gat->negative_slope;
+        a.self_loop = gat->add_self_loop ? 1 : 0;
+        a.s = ws.take<float>((size_t)n * gat->heads);
+        a.t = ws.take<float>((size_t)n * gat->heads);
+        a.out = out; a.ldout = ldout;
+        a.out16 = static_cast<__nv_bfloat16*>(out_bf16); a.ldout16 = ldout_bf16;
+        const unsigned blocks = (unsigned)((n + kAggWarps - 1) / kAggWarps);
+        gat_scores_kernel<<<blocks, kAggThreads, 0, st>>>(a);
+        const int nc = (dim + kWarp - 1) / kWarp;
+        if (nc <= 1) gat_rows_kernel<1><<<blocks, kAggThreads, 0, st>>>(a);
+        else if (nc <= 2) gat_rows_kernel<2><<<blocks, kAggThreads, 0, st>>>(a);
+        else if (nc <= 4) gat_rows_kernel<4><<<blocks, kAggThreads, 0, st>>>(a);
+        else gat_rows_kernel<8><<<blocks, kAggThreads, 0, st>>>(a);
+        return launch_status();
+    }
+
+    AggArgs a;
+    a.n = n; a.rowptr = g->rowptr; a.colidx = g->colidx; a.q = q; a.ldq = ldq; a.dim = dim;
+    float* coef = ws.take<float>((size_t)n);
+    int32_t* heavy_list = ws.take<int32_t>((size_t)n);
+    int32_t* heavy_count = ws.take<int32_t>(64);
+    a.coef = coef; a.heavy_list = heavy_list; a.heavy_count = heavy_count;
+    a.out = out; a.ldout = ldout;
+    a.out16 = static_cast<__nv_bfloat16*>(out_bf16); a.ldout16 = ldout_bf16;
+    a.concat_self = concat_self ? 1 : 0;
+    RETEXO_CUDA_TRY(cudaMemsetAsync(heavy_count, 0, sizeof(int32_t), st));
+    prep_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(n, g->rowptr, type, coef, heavy_list, heavy_count);
+
+    const bool gcn = type == RETEXO_GCN;
+    const bool v4 = aligned_to(q, 16) && ldq % 4 == 0 && ldq >= (dim + 3) / 4 * 4;
+    const bool v2 = aligned_to(q, 8) && ldq % 2 == 0 && ldq >= (dim + 1) / 2 * 2;
+    if (v4) return gcn ? dispatch_ch<4, true>(a, n_sm, st) : dispatch_ch<4, false>(a, n_sm, st);
+    if (v2) return gcn ? dispatch_ch<2, true>(a, n_sm, st) : dispatch_ch<2, false>(a, n_sm, st);
+    return gcn ? dispatch_ch<1, true>(a, n_sm, st) : dispatch_ch<1, false>(a, n_sm, st);
+}

@@ -1,0 +1,373 @@
+// Exact count of the boundary-node messages (and bytes) one lazy
+// message-passing round sends across a node partition (Section 2.1,
+// Appendix A.1), plus the CSR validator.  Integer work only; all tallies use
+// integer atomics, whose result does not depend on the order they land in.
+#include "common.cuh"
+
+namespace retexo {
+
+constexpr int kCntThreads = 256;
+constexpr int kCntWarps = kCntThreads / kWarp;
+constexpr int kBitmapParts = 8192;                  // per-warp shared bitmap covers this many partitions
+constexpr int kBitmapWords = kBitmapParts / 32;
+constexpr int kHashSlots = 2048;                    // per-warp shared hash set
+constexpr int kHashMaxDeg = 1024;                   // rows up to this length use it
+constexpr int kHashWarps = 4;
+constexpr int kBigRowBlocks = 64;                   // blocks (and global bitmaps) of the long-row pass
+
+struct CountArgs {
+    int64_t n;
+    const int64_t* rowptr;
+    const int32_t* colidx;
+    const int32_t* part;
+    int32_t n_parts;
+    unsigned long long* cross_edges;      // accumulators (zeroed before launch)
+    unsigned long long* pairs;
+    unsigned long long* send;             // may be null
+    unsigned long long* recv;             // may be null
+    int32_t* big_list;                    // rows deferred to the long-row pass
+    int32_t* big_count;
+    uint32_t* big_bitmaps;                // kBigRowBlocks x words_per_bitmap, all zero between rows
+    int64_t words_per_bitmap;
+    unsigned long long* bad_part;         // set to 1 if a partition id is out of range
+};
+
+// Partition id of node x; an id outside [0, n_parts) raises the flag and is
+// replaced by 0 so that every table access stays in bounds.
+__device__ __forceinline__ int32_t part_of(const CountArgs& a, int64_t x) {
+    const int32_t p = __ldg(a.part + x);
+    if ((uint32_t)p >= (uint32_t)a.n_parts) {
+        *a.bad_part = 1ull;
+        return 0;
+    }
+    return p;
+}
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// Partition count <= kBitmapParts: one warp per row, the set of destination
+// partitions already seen is a bitmap in shared memory.
+__global__ void __launch_bounds__(kCntThreads) count_bitmap_kernel(CountArgs a) {
+    __shared__ uint32_t bm[kCntWarps][kBitmapWords];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = lane; i < kBitmapWords; i += kWarp) bm[warp][i] = 0u;
+    __syncwarp();
+    unsigned long long my_cross = 0, my_pairs = 0;
+    const int64_t stride = (int64_t)gridDim.x * kCntWarps;
+    for (int64_t u = blockIdx.x * (int64_t)kCntWarps + warp; u < a.n; u += stride) {
+        const int64_t beg = a.rowptr[u], end = a.rowptr[u + 1];
+        if (beg == end) continue;
+        const int32_t pu = part_of(a, u);
+        unsigned row_new = 0;
+        for (int64_t e0 = beg; e0 < end; e0 += kWarp) {
+            const int64_t e = e0 + lane;
+            const bool valid = e < end;
+            int32_t pv = pu;
+            if (valid) pv = part_of(a, __ldg(a.colidx + e));
+            const bool cross = pv != pu;
+            bool is_new = false;
+            if (cross) {
+                const uint32_t bit = 1u << (pv & 31);
+                const uint32_t old = atomicOr(&bm[warp][pv >> 5], bit);
+                is_new = !(old & bit);
+                if (is_new && a.recv) atomicAdd(a.recv + pv, 1ull);
+            }
+            my_cross += cross ? 1ull : 0ull;
+            row_new += __popc(__ballot_sync(0xffffffffu, is_new));
+        }
+        __syncwarp();
+        // clear the touched words again
+        if (end - beg >= kBitmapWords) {
+            for (int i = lane; i < kBitmapWords; i += kWarp) bm[warp][i] = 0u;
+        } else {
+            for (int64_t e = beg + lane; e < end; e += kWarp) {
+                const int32_t pv = part_of(a, __ldg(a.colidx + e));
+                bm[warp][pv >> 5] = 0u;
+            }
+        }
+        __syncwarp();
+        if (lane == 0) {
+            my_pairs += row_new;
+            if (a.send && row_new) atomicAdd(a.send + pu, (unsigned long long)row_new);
+        }
+    }
+    my_cross = warp_sum_u64(my_cross);
+    if (lane == 0) {
+        if (my_cross) atomicAdd(a.cross_edges, my_cross);
+        if (my_pairs) atomicAdd(a.pairs, my_pairs);
+    }
+}
+
+__device__ __forceinline__ uint32_t hash32(uint32_t x) {
+    x ^= x >> 16; x *= 0x7feb352du; x ^= x >> 15; x *= 0x846ca68bu; x ^= x >> 16;
+    return x;
+}
+
+// Any partition count: one warp per row.
+//  1. If the destination partitions come in non-decreasing order along the row
+//     (true for node-level and for range partitions, the columns being
+//     sorted), equal ones are adjacent and a compare with the previous entry
+//     finds the distinct ones.
+//  2. Otherwise rows of up to kHashMaxDeg entries use a hash set in shared
+//     memory; longer ones are listed for the long-row pass.
+__global__ void __launch_bounds__(kHashWarps * kWarp) count_general_kernel(CountArgs a) {
+    __shared__ int32_t tab[kHashWarps][kHashSlots];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = lane; i < kHashSlots; i += kWarp) tab[warp][i] = -1;
+    __syncwarp();
+    unsigned long long my_cross = 0, my_pairs = 0;
+    const int64_t stride = (int64_t)gridDim.x * kHashWarps;
+    for (int64_t u = blockIdx.x * (int64_t)kHashWarps + warp; u < a.n; u += stride) {
+        const int64_t beg = a.rowptr[u], end = a.rowptr[u + 1];
+        if (beg == end) continue;
+        const int32_t pu = part_of(a, u);
+        // pass 1: order check + adjacent-distinct count
+        bool mono = true;
+        unsigned n_cross = 0, n_new = 0;
+        int32_t carry = -1;
+        for (int64_t e0 = beg; e0 < end; e0 += kWarp) {
+            const int64_t e = e0 + lane;
+            const bool valid = e < end;
+            const int32_t pv = valid ? part_of(a, __ldg(a.colidx + e)) : INT32_MAX;
+            int32_t prev = __shfl_up_sync(0xffffffffu, pv, 1);
+            if (lane == 0) prev = carry;
+            mono = mono && __all_sync(0xffffffffu, pv >= prev);
+            const bool cross = valid && pv != pu;
+            n_cross += __popc(__ballot_sync(0xffffffffu, cross));
+            n_new += __popc(__ballot_sync(0xffffffffu, cross && pv != prev));
+            carry = __shfl_sync(0xffffffffu, pv, kWarp - 1);
+        }
+        if (lane == 0) my_cross += n_cross;
+        if (n_cross == 0) continue;
+        if (mono) {
+            if (a.recv) {
+                carry = -1;
+                for (int64_t e0 = beg; e0 < end; e0 += kWarp) {
+                    const int64_t e = e0 + lane;
+                    const bool valid = e < end;
+                    const int32_t pv = valid ? part_of(a, __ldg(a.colidx + e)) : INT32_MAX;
+                    int32_t prev = __shfl_up_sync(0xffffffffu, pv, 1);
+                    if (lane == 0) prev = carry;
+                    if (valid && pv != pu && pv != prev) atomicAdd(a.recv + pv, 1ull);
+                    carry = __shfl_sync(0xffffffffu, pv, kWarp - 1);
+                }
+            }
+        } else if (end - beg <= kHashMaxDeg) {
+            n_new = 0;
+            for (int64_t e0 = beg; e0 < end; e0 += kWarp) {
+                const int64_t e = e0 + lane;
+                bool is_new = false;
+                if (e < end) {
+                    const int32_t pv = part_of(a, __ldg(a.colidx + e));
+                    if (pv != pu) {
+                        uint32_t h = hash32((uint32_t)pv) & (kHashSlots - 1);
+                        for (int probe = 0; probe < kHashSlots; ++probe) {      // table is never full
+                            const int32_t old = atomicCAS(&tab[warp][h], -1, pv);
+                            if (old == -1) { is_new = true; break; }
+                            if (old == pv) break;
+                            h = (h + 1) & (kHashSlots - 1);
+                        }
+                        if (is_new && a.recv) atomicAdd(a.recv + pv, 1ull);
+                    }
+                }
+                n_new += __popc(__ballot_sync(0xffffffffu, is_new));
+            }
+            __syncwarp();
+            for (int i = lane; i < kHashSlots; i += kWarp) tab[warp][i] = -1;
+            __syncwarp();
+        } else {
+            if (lane == 0) {
+                const int32_t slot = atomicAdd(a.big_count, 1);
+                a.big_list[slot] = (int32_t)u;
+            }
+            continue;      // pairs of this row are counted by the long-row pass
+        }
+        if (lane == 0) {
+            my_pairs += n_new;
+            if (a.send && n_new) atomicAdd(a.send + pu, (unsigned long long)n_new);
+        }
+    }
+    if (lane == 0) {
+        if (my_cross) atomicAdd(a.cross_edges, my_cross);
+        if (my_pairs) atomicAdd(a.pairs, my_pairs);
+    }
+}
+
+// Long unordered rows with many partitions: one block per row, the seen-set is
+// a bitmap in global memory owned by the block (all zero on entry and exit).
+__global__ void __launch_bounds__(kCntThreads) count_big_rows_kernel(CountArgs a) {
+    __shared__ unsigned int block_new;
+    uint32_t* bm = a.big_bitmaps + (int64_t)blockIdx.x * a.words_per_bitmap;
+    const int n_big = *a.big_count;
+    for (int r = blockIdx.x; r < n_big; r += gridDim.x) {
+        const int64_t u = a.big_list[r];
+        const int64_t beg = a.rowptr[u], end = a.rowptr[u + 1];
+        const int32_t pu = part_of(a, u);
+        if (threadIdx.x == 0) block_new = 0;
+        __syncthreads();
+        unsigned mine = 0;
+        for (int64_t e = beg + threadIdx.x; e < end; e += kCntThreads) {
+            const int32_t pv = part_of(a, __ldg(a.colidx + e));
+            if (pv == pu) continue;
+            const uint32_t bit = 1u << (pv & 31);
+            const uint32_t old = atomicOr(bm + (pv >> 5), bit);
+            if (!(old & bit)) {
+                ++mine;
+                if (a.recv) atomicAdd(a.recv + pv, 1ull);
+            }
+        }
+        if (mine) atomicAdd(&block_new, mine);
+        __syncthreads();
+        for (int64_t e = beg + threadIdx.x; e < end; e += kCntThreads) {
+            const int32_t pv = part_of(a, __ldg(a.colidx + e));
+            bm[pv >> 5] = 0u;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0 && block_new) {
+            atomicAdd(a.pairs, (unsigned long long)block_new);
+            if (a.send) atomicAdd(a.send + pu, (unsigned long long)block_new);
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void count_finalize_kernel(const unsigned long long* cross_acc, const unsigned long long* pairs_acc,
+                                      const unsigned long long* bad_part, int32_t K, const int32_t* dims, int32_t elem_bytes,
+                                      uint64_t* cross_edges, uint64_t* boundary_pairs,
+                                      uint64_t* bytes_per_round, uint64_t* bytes_total) {
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    if (*bad_part) {          // a partition id was out of range: poison the results
+        if (cross_edges) *cross_edges = UINT64_MAX;
+        if (boundary_pairs) *boundary_pairs = UINT64_MAX;
+        for (int m = 0; m < K; ++m) if (bytes_per_round) bytes_per_round[m] = UINT64_MAX;
+        if (bytes_total) *bytes_total = UINT64_MAX;
+        return;
+    }
+    const uint64_t bp = *pairs_acc;
+    if (cross_edges) *cross_edges = *cross_acc;
+    if (boundary_pairs) *boundary_pairs = bp;
+    uint64_t tot = 0;
+    for (int m = 0; m < K; ++m) {
+        const uint64_t b = bp * (uint64_t)dims[m] * (uint64_t)elem_bytes;
+        if (bytes_per_round) bytes_per_round[m] = b;
+        tot += b;
+    }
+    if (bytes_total) *bytes_total = tot;
+}
+
+// ---------------------------------------------------------------- validator
+__global__ void validate_csr_kernel(int64_t n, int64_t n_edges, const int64_t* rowptr, const int32_t* colidx,
+                                    unsigned long long* bad, long long* where) {
+    const int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (v > n) return;
+    bool wrong = false;
+    if (v == 0 && rowptr[0] != 0) wrong = true;
+    if (v == n) {
+        if (rowptr[n] != n_edges) wrong = true;
+    } else {
+        const int64_t beg = rowptr[v], end = rowptr[v + 1];
+        if (beg > end || beg < 0 || end > n_edges) wrong = true;
+        else {
+            int64_t prev = -1;
+            for (int64_t e = beg; e < end; ++e) {
+                const int64_t c = colidx[e];
+                if (c < 0 || c >= n || c == v || c <= prev) { wrong = true; break; }
+                prev = c;
+            }
+        }
+    }
+    if (wrong) {
+        atomicAdd(bad, 1ull);
+        atomicMax(where, (long long)v);
+    }
+}
+
+}  // namespace retexo
+
+using namespace retexo;
+
+extern "C" int retexo_validate_csr(const retexo_csr* g, int64_t* status_out, void* stream) {
+    if (!g || !status_out || g->n_nodes < 0 || g->n_edges < 0) return RETEXO_ERR_INVALID_ARG;
+    if (!g->rowptr || (g->n_edges > 0 && !g->colidx)) return RETEXO_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const long long init[2] = {0, -1};
+    RETEXO_CUDA_TRY(cudaMemcpyAsync(status_out, init, sizeof(init), cudaMemcpyHostToDevice, st));
+    const int64_t threads = g->n_nodes + 1;
+    validate_csr_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(
+        g->n_nodes, g->n_edges, g->rowptr, g->colidx,
+        reinterpret_cast<unsigned long long*>(status_out), reinterpret_cast<long long*>(status_out + 1));
+    return launch_status();
+}
+
+extern "C" size_t retexo_cross_partition_workspace_size(int64_t n_nodes, int64_t n_edges, int32_t n_parts) {
+    (void)n_edges;
+    if (n_nodes < 0 || n_parts <= 0) return 0;
+    Sizer s;
+    s.take<unsigned long long>(32);                       // accumulators
+    s.take<int32_t>(64);                                  // dims copy
+    if (n_parts > kBitmapParts) {
+        s.take<int32_t>((size_t)n_nodes);                 // long-row list
+        s.take<int32_t>(64);
+        s.take<uint32_t>((size_t)kBigRowBlocks * (size_t)((n_parts + 31) / 32));
+    }
+    return s.off + kAlign;
+}
+
+extern "C" int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* part, int32_t n_parts,
+                                            int32_t K, const int32_t* dims, int32_t elem_bytes,
+                                            uint64_t* cross_edges, uint64_t* boundary_pairs,
+                                            uint64_t* bytes_per_round, uint64_t* bytes_total,
+                                            uint64_t* send_per_part, uint64_t* recv_per_part,
+                                            void* workspace, size_t workspace_bytes, void* stream) {
+    if (!g || g->n_nodes < 0 || g->n_edges < 0 || g->n_nodes > INT32_MAX) return RETEXO_ERR_INVALID_ARG;
+    if (n_parts <= 0 || K < 0 || K > 64 || elem_bytes <= 0 || (K > 0 && !dims)) return RETEXO_ERR_INVALID_ARG;
+    if (g->n_nodes > 0 && (!g->rowptr || !part || (g->n_edges > 0 && !g->colidx))) return RETEXO_ERR_INVALID_ARG;
+    for (int m = 0; m < K; ++m) if (dims[m] < 0) return RETEXO_ERR_INVALID_ARG;
+    const size_t need = retexo_cross_partition_workspace_size(g->n_nodes, g->n_edges, n_parts);
+    if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return RETEXO_ERR_CUDA;
+
+    Arena ws(workspace, workspace_bytes);
+    unsigned long long* acc = ws.take<unsigned long long>(32);
+    int32_t* dims_dev = ws.take<int32_t>(64);
+    CountArgs a;
+    a.n = g->n_nodes; a.rowptr = g->rowptr; a.colidx = g->colidx; a.part = part; a.n_parts = n_parts;
+    a.cross_edges = acc; a.pairs = acc + 1; a.bad_part = acc + 2;
+    a.send = reinterpret_cast<unsigned long long*>(send_per_part);
+    a.recv = reinterpret_cast<unsigned long long*>(recv_per_part);
+    a.big_list = nullptr; a.big_count = nullptr; a.big_bitmaps = nullptr; a.words_per_bitmap = 0;
+
+    RETEXO_CUDA_TRY(cudaMemsetAsync(acc, 0, 32 * sizeof(unsigned long long), st));
+    if (K > 0) RETEXO_CUDA_TRY(cudaMemcpyAsync(dims_dev, dims, sizeof(int32_t) * K, cudaMemcpyHostToDevice, st));
+    if (send_per_part) RETEXO_CUDA_TRY(cudaMemsetAsync(send_per_part, 0, sizeof(uint64_t) * (size_t)n_parts, st));
+    if (recv_per_part) RETEXO_CUDA_TRY(cudaMemsetAsync(recv_per_part, 0, sizeof(uint64_t) * (size_t)n_parts, st));
+
+    if (a.n > 0) {
+        if (n_parts <= kBitmapParts) {
+            const int64_t want = (a.n + kCntWarps - 1) / kCntWarps;
+            const unsigned blocks = (unsigned)(want < (int64_t)n_sm * 8 ? want : (int64_t)n_sm * 8);
+            count_bitmap_kernel<<<blocks, kCntThreads, 0, st>>>(a);
+        } else {
+            a.big_list = ws.take<int32_t>((size_t)a.n);
+            a.big_count = ws.take<int32_t>(64);
+            a.words_per_bitmap = (n_parts + 31) / 32;
+            a.big_bitmaps = ws.take<uint32_t>((size_t)kBigRowBlocks * (size_t)a.words_per_bitmap);
+            RETEXO_CUDA_TRY(cudaMemsetAsync(a.big_count, 0, sizeof(int32_t), st));
+            RETEXO_CUDA_TRY(cudaMemsetAsync(a.big_bitmaps, 0,
+                                            sizeof(uint32_t) * (size_t)kBigRowBlocks * (size_t)a.words_per_bitmap, st));
+            const int64_t want = (a.n + kHashWarps - 1) / kHashWarps;
+            const unsigned blocks = (unsigned)(want < (int64_t)n_sm * 16 ? want : (int64_t)n_sm * 16);
+            count_general_kernel<<<blocks, kHashWarps * kWarp, 0, st>>>(a);
+            count_big_rows_kernel<<<kBigRowBlocks, kCntThreads, 0, st>>>(a);
+        }
+    }
+    count_finalize_kernel<<<1, 32, 0, st>>>(acc, acc + 1, acc + 2, K, dims_dev, elem_bytes, cross_edges, boundary_pairs,
+                                            bytes_per_round, bytes_total);
+    return launch_status();
+}

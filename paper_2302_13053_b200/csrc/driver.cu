@@ -1,0 +1,397 @@
+// The K-round lazy-message-passing loop (Section 3.1) run from one host call:
+// per round one aggregation, R training iterations with validation and
+// best-iterate tracking on the device (no host round trips inside the loop),
+// then the emission of the next representations.
+#include <vector>
+
+#include "common.cuh"
+#include "mlp_plan.h"
+
+using namespace retexo;
+
+namespace retexo {
+
+typedef __nv_bfloat16 bf16;
+
+static inline int64_t round_up(int64_t x, int64_t a) { return (x + a - 1) / a * a; }
+
+__global__ void gather_i32_kernel(const int32_t* __restrict__ src, const int32_t* __restrict__ idx, int64_t n,
+                                  int32_t* __restrict__ dst) {
+    const int64_t i = blockIdx.x * 256ll + threadIdx.x;
+    if (i < n) dst[i] = src[idx[i]];
+}
+
+// Keeps the iterate with the most validation hits, earliest on ties.  Every
+// thread takes the same decision from (cur, best); the bookkeeping kernel that
+// follows then updates best.
+__global__ void snapshot_if_better_kernel(const unsigned long long* cur, const unsigned long long* best,
+                                          const int32_t* have_best, const float* theta, float* theta_best,
+                                          int64_t nt) {
+    if (*have_best && *cur <= *best) return;
+    const int64_t p = blockIdx.x * 256ll + threadIdx.x;
+    if (p < nt) theta_best[p] = theta[p];
+}
+__global__ void record_validation_kernel(const unsigned long long* cur, unsigned long long* best, int32_t* have_best,
+                                         int32_t iter, int32_t* best_iter, unsigned long long* history_slot) {
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    *history_slot = *cur;
+    if (!*have_best || *cur > *best) {
+        *best = *cur;
+        *best_iter = iter;
+        *have_best = 1;
+    }
+}
+__global__ void fill_u64_kernel(unsigned long long* p, int64_t n, unsigned long long v) {
+    const int64_t i = blockIdx.x * 256ll + threadIdx.x;
+    if (i < n) p[i] = v;
+}
+__global__ void pack_counts_kernel(const uint64_t* cross, const uint64_t* pairs, const uint64_t* total,
+                                   const uint64_t* per_round, int K, uint64_t* out) {
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    out[0] = *cross; out[1] = *pairs; out[2] = *total;
+    out[3] = *total == UINT64_MAX ? UINT64_MAX : 2 * *total;
+    for (int m = 0; m < K; ++m) out[4 + m] = per_round[m];
+}
+
+struct RoundDims { int32_t rep_dim, agg_dim, d_in, hidden; };
+
+static RoundDims round_dims(const retexo_lmp_config& c, int m /*1-based*/) {
+    RoundDims r;
+    r.rep_dim = m == 1 ? c.d0 : c.hidden;
+    if (c.aggr == RETEXO_GAT) { r.agg_dim = c.gat_heads * c.gat_head_dim; r.d_in = r.agg_dim; }
+    else if (c.aggr == RETEXO_SAGE_MEAN) { r.agg_dim = r.rep_dim; r.d_in = 2 * r.rep_dim; }
+    else { r.agg_dim = r.rep_dim; r.d_in = r.rep_dim; }
+    r.hidden = m < c.K ? c.hidden : 0;
+    return r;
+}
+
+struct LmpBuffers {
+    // staged inputs (host mode only)
+    int64_t* rowptr; int32_t* colidx; float* features; int32_t* labels;
+    int32_t *train_idx, *val_idx, *test_idx, *part;
+    // representations
+    float* q[2];
+    bf16* x16; bf16* q16; float* proj; bf16* watt16; float* gat_vec; float* gat_stage;
+    bf16 *xtr16, *xval16;
+    int32_t *y_tr, *y_val, *y_test;
+    float *theta, *adam_m, *adam_v, *theta_best;
+    unsigned long long *cur_correct, *best_correct, *scratch_u64;
+    int32_t *have_best, *best_iter_cur;
+    // device copies of the outputs
+    float* loss_history; unsigned long long* val_history;
+    unsigned long long *best_val, *test_best, *test_last; int32_t* best_iter;
+    uint64_t* counts; uint64_t* count_raw;
+    float* final_logits; int32_t* final_pred;
+    void *ws_step, *ws_embed, *ws_agg, *ws_count;
+    size_t ws_step_bytes, ws_embed_bytes, ws_agg_bytes, ws_count_bytes;
+};
+
+template <typename Taker>
+static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t n_tr, int64_t n_val, int64_t n_te,
+                       int32_t n_parts, Taker& t, LmpBuffers* b) {
+    LmpBuffers l{};
+    const bool host = c.memory_is_host != 0;
+    int32_t max_din = 0, max_rep = 0;
+    int64_t max_nt = 0;
+    size_t step_b = 0, embed_b = 0, agg_b = 0;
+    for (int m = 1; m <= c.K; ++m) {
+        const RoundDims r = round_dims(c, m);
+        if (r.d_in > max_din) max_din = r.d_in;
+        if (r.rep_dim > max_rep) max_rep = r.rep_dim;
+        const int64_t nt = retexo_theta_size(r.d_in, r.hidden, c.n_classes);
+        if (nt > max_nt) max_nt = nt;
+        size_t s = retexo_mlp_train_step_workspace_size(r.d_in, r.hidden, c.n_classes, n_tr);
+        if (s > step_b) step_b = s;
+        s = retexo_embed_workspace_size(r.d_in, r.hidden, c.n_classes, n);
+        if (s > embed_b) embed_b = s;
+        s = retexo_aggregate_workspace_size(n, e, c.aggr, r.agg_dim, c.gat_heads);
+        if (s > agg_b) agg_b = s;
+    }
+    const int64_t ld16 = round_up(max_din, 8);
+    if (host) {
+        l.rowptr = t.template take<int64_t>((size_t)n + 1);
+        l.colidx = t.template take<int32_t>((size_t)e);
+        l.features = t.template take<float>((size_t)n * round_up(c.d0, 32));
+        l.labels = t.template take<int32_t>((size_t)n);
+        l.train_idx = t.template take<int32_t>((size_t)n_tr);
+        l.val_idx = t.template take<int32_t>((size_t)n_val);
+        l.test_idx = t.template take<int32_t>((size_t)n_te);
+        l.part = t.template take<int32_t>(n_parts > 0 ? (size_t)n : 1);
+    }
+    const size_t qsz = c.K > 1 ? (size_t)n * round_up(c.hidden, 32) : 1;
+    l.q[0] = t.template take<float>(qsz);
+    l.q[1] = t.template take<float>(c.K > 2 ? qsz : 1);
+    l.x16 = t.template take<bf16>((size_t)n * ld16);
+    if (c.aggr == RETEXO_GAT) {
+        const int32_t hd = c.gat_heads * c.gat_head_dim;
+        l.q16 = t.template take<bf16>((size_t)n * round_up(max_rep, 8));
+        l.proj = t.template take<float>((size_t)n * round_up(hd, 32));
+        l.watt16 = t.template take<bf16>((size_t)max_rep * hd);
+        l.gat_vec = t.template take<float>((size_t)2 * hd);
+        l.gat_stage = t.template take<float>((size_t)max_rep * hd + 2 * hd);
+    }
+    l.xtr16 = t.template take<bf16>((size_t)n_tr * ld16);
+    l.xval16 = t.template take<bf16>((size_t)(n_val > 0 ? n_val : 1) * ld16);
+    l.y_tr = t.template take<int32_t>((size_t)n_tr);
+    l.y_val = t.template take<int32_t>((size_t)(n_val > 0 ? n_val : 1));
+    l.y_test = t.template take<int32_t>((size_t)(n_te > 0 ? n_te : 1));
+    l.theta = t.template take<float>((size_t)max_nt);
+    l.adam_m = t.template take<float>((size_t)max_nt);
+    l.adam_v = t.template take<float>((size_t)max_nt);
+    l.theta_best = t.template take<float>((size_t)max_nt);
+    l.cur_correct = t.template take<unsigned long long>(4);
+    l.best_correct = t.template take<unsigned long long>(4);
+    l.scratch_u64 = t.template take<unsigned long long>(4);
+    l.have_best = t.template take<int32_t>(4);
+    l.best_iter_cur = t.template take<int32_t>(4);
+    l.loss_history = t.template take<float>((size_t)c.K * c.R);
+    l.val_history = t.template take<unsigned long long>((size_t)c.K * c.R);
+    l.best_val = t.template take<unsigned long long>((size_t)c.K);
+    l.test_best = t.template take<unsigned long long>((size_t)c.K);
+    l.test_last = t.template take<unsigned long long>((size_t)c.K);
+    l.best_iter = t.template take<int32_t>((size_t)c.K);
+    l.counts = t.template take<uint64_t>((size_t)4 + c.K);
+    l.count_raw = t.template take<uint64_t>((size_t)4 + c.K);
+    if (host) {
+        l.final_logits = t.template take<float>((size_t)n * c.n_classes);
+        l.final_pred = t.template take<int32_t>((size_t)n);
+    }
+    l.ws_step_bytes = step_b; l.ws_embed_bytes = embed_b; l.ws_agg_bytes = agg_b;
+    l.ws_count_bytes = n_parts > 0 ? retexo_cross_partition_workspace_size(n, e, n_parts) : 0;
+    l.ws_step = t.template take<char>(step_b);
+    l.ws_embed = t.template take<char>(embed_b);
+    l.ws_agg = t.template take<char>(agg_b);
+    l.ws_count = t.template take<char>(l.ws_count_bytes ? l.ws_count_bytes : 1);
+    if (b) *b = l;
+}
+
+struct NullTaker2 {
+    Sizer s;
+    template <typename T> T* take(size_t count) { s.take<T>(count); return nullptr; }
+};
+
+static int check_cfg(const retexo_lmp_config* c) {
+    if (!c) return RETEXO_ERR_INVALID_ARG;
+    if (c->K < 1 || c->K > 8 || c->R < 1 || c->d0 <= 0 || c->n_classes <= 0) return RETEXO_ERR_INVALID_ARG;
+    if (c->K > 1 && c->hidden <= 0) return RETEXO_ERR_INVALID_ARG;
+    if (c->aggr != RETEXO_GCN && c->aggr != RETEXO_SAGE_MEAN && c->aggr != RETEXO_GAT) return RETEXO_ERR_INVALID_ARG;
+    if (c->aggr == RETEXO_GAT && (c->gat_heads <= 0 || c->gat_head_dim <= 0)) return RETEXO_ERR_INVALID_ARG;
+    if (c->eval_every < 1) return RETEXO_ERR_INVALID_ARG;
+    if (c->n_classes > 64 || c->hidden > 512) return RETEXO_ERR_UNSUPPORTED;
+    return RETEXO_OK;
+}
+
+}  // namespace retexo
+
+extern "C" size_t retexo_lmp_workspace_size(const retexo_lmp_config* cfg, int64_t n_nodes, int64_t n_edges,
+                                            int64_t n_train, int64_t n_val, int64_t n_test, int32_t n_parts) {
+    if (check_cfg(cfg) != RETEXO_OK || n_nodes <= 0 || n_edges < 0 || n_train <= 0 || n_val < 0 || n_test < 0) return 0;
+    NullTaker2 t;
+    lmp_layout(*cfg, n_nodes, n_edges, n_train, n_val, n_test, n_parts, t, nullptr);
+    return t.s.off + kAlign;
+}
+
+extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_inputs* in,
+                                const retexo_lmp_outputs* out, void* workspace, size_t workspace_bytes,
+                                void* stream) {
+    RETEXO_TRY(check_cfg(cfg));
+    if (!in || !out) return RETEXO_ERR_INVALID_ARG;
+    const retexo_lmp_config& c = *cfg;
+    const int64_t n = in->graph.n_nodes, e = in->graph.n_edges;
+    if (n <= 0 || e < 0 || n > INT32_MAX || !in->graph.rowptr || (e > 0 && !in->graph.colidx)) return RETEXO_ERR_INVALID_ARG;
+    if (!in->features || in->ld_features < c.d0 || !in->labels) return RETEXO_ERR_INVALID_ARG;
+    if (!in->train_idx || in->n_train <= 0 || in->n_val < 0 || in->n_test < 0) return RETEXO_ERR_INVALID_ARG;
+    if ((in->n_val > 0 && !in->val_idx) || (in->n_test > 0 && !in->test_idx)) return RETEXO_ERR_INVALID_ARG;
+    if (!in->theta0 || (c.aggr == RETEXO_GAT && !in->gat_w)) return RETEXO_ERR_INVALID_ARG;
+    for (int m = 0; m < c.K; ++m) {
+        if (!in->theta0[m]) return RETEXO_ERR_INVALID_ARG;
+        if (c.aggr == RETEXO_GAT && !in->gat_w[m]) return RETEXO_ERR_INVALID_ARG;
+    }
+    if (in->part && in->n_parts <= 0) return RETEXO_ERR_INVALID_ARG;
+    if (out->final_logits && out->ld_logits < c.n_classes) return RETEXO_ERR_INVALID_ARG;
+    const int32_t n_parts = in->part ? in->n_parts : 0;
+    const size_t need = retexo_lmp_workspace_size(cfg, n, e, in->n_train, in->n_val, in->n_test, n_parts);
+    if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool host = c.memory_is_host != 0;
+    const cudaMemcpyKind in_kind = host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+    const cudaMemcpyKind out_kind = host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice;
+
+    Arena ws(workspace, workspace_bytes);
+    LmpBuffers b{};
+    lmp_layout(c, n, e, in->n_train, in->n_val, in->n_test, n_parts, ws, &b);
+    const int64_t n_tr = in->n_train, n_val = in->n_val, n_te = in->n_test;
+
+    // ---- inputs
+    retexo_csr g = in->graph;
+    const float* feat = in->features;
+    int64_t ld_feat = in->ld_features;
+    const int32_t *labels = in->labels, *train_idx = in->train_idx, *val_idx = in->val_idx, *test_idx = in->test_idx;
+    const int32_t* part = in->part;
+    if (host) {
+        RETEXO_CUDA_TRY(cudaMemcpyAsync(b.rowptr, g.rowptr, sizeof(int64_t) * (size_t)(n + 1), in_kind, st));
+        if (e > 0) RETEXO_CUDA_TRY(cudaMemcpyAsync(b.colidx, g.colidx, sizeof(int32_t) * (size_t)e, in_kind, st));
+        const int64_t ldp = round_up(c.d0, 32);
+        if (ldp != c.d0) RETEXO_CUDA_TRY(cudaMemsetAsync(b.features, 0, sizeof(float) * (size_t)n * ldp, st));
+        RETEXO_CUDA_TRY(cudaMemcpy2DAsync(b.features, sizeof(float) * ldp, feat, sizeof(float) * ld_feat,
+                                          sizeof(float) * c.d0, (size_t)n, in_kind, st));
+        RETEXO_CUDA_TRY(cudaMemcpyAsync(b.labels, labels, sizeof(int32_t) * (size_t)n, in_kind, st));
+        RETEXO_CUDA_TRY(cudaMemcpyAsync(b.train_idx, train_idx, sizeof(int32_t) * (size_t)n_tr, in_kind, st));
+        if (n_val) RETEXO_CUDA_TRY(cudaMemcpyAsync(b.val_idx, val_idx, sizeof(int32_t) * (size_t)n_val, in_kind, st));
+        if (n_te) RETEXO_CUDA_TRY(cudaMemcpyAsync(b.test_idx, test_idx, sizeof(int32_t) * (size_t)n_te, in_kind, st));
+        if (part) RETEXO_CUDA_TRY(cudaMemcpyAsync(b.part, part, sizeof(int32_t) * (size_t)n, in_kind, st));
+        g.rowptr = b.rowptr; g.colidx = b.colidx; feat = b.features; ld_feat = ldp;
+        labels = b.labels; train_idx = b.train_idx; val_idx = b.val_idx; test_idx = b.test_idx;
+        if (part) part = b.part;
+    }
+    gather_i32_kernel<<<(unsigned)((n_tr + 255) / 256), 256, 0, st>>>(labels, train_idx, n_tr, b.y_tr);
+    if (n_val) gather_i32_kernel<<<(unsigned)((n_val + 255) / 256), 256, 0, st>>>(labels, val_idx, n_val, b.y_val);
+    if (n_te) gather_i32_kernel<<<(unsigned)((n_te + 255) / 256), 256, 0, st>>>(labels, test_idx, n_te, b.y_test);
+    fill_u64_kernel<<<(unsigned)(((int64_t)c.K * c.R + 255) / 256), 256, 0, st>>>(b.val_history, (int64_t)c.K * c.R,
+                                                                                  ~0ull);
+
+    // ---- messages and bytes across the partition, all rounds
+    if (part) {
+        int32_t dims[8];
+        for (int m = 1; m <= c.K; ++m) dims[m - 1] = round_dims(c, m).rep_dim;
+        RETEXO_TRY(retexo_cross_partition_bytes(&g, part, n_parts, c.K, dims, 4, b.count_raw, b.count_raw + 1,
+                                                b.count_raw + 4, b.count_raw + 2, nullptr, nullptr, b.ws_count,
+                                                b.ws_count_bytes, st));
+        pack_counts_kernel<<<1, 32, 0, st>>>(b.count_raw, b.count_raw + 1, b.count_raw + 2, b.count_raw + 4, c.K,
+                                             b.counts);
+    }
+
+    {   // padding columns of the bf16 inputs are never read as data, but keep them defined
+        int32_t max_din = 0;
+        for (int m = 1; m <= c.K; ++m) if (round_dims(c, m).d_in > max_din) max_din = round_dims(c, m).d_in;
+        RETEXO_CUDA_TRY(cudaMemsetAsync(b.x16, 0, sizeof(bf16) * (size_t)n * (size_t)round_up(max_din, 8), st));
+    }
+    const float* q = feat;
+    int64_t ldq = ld_feat;
+    for (int m = 1; m <= c.K; ++m) {
+        const RoundDims r = round_dims(c, m);
+        const int64_t ld16 = round_up(r.d_in, 8);
+        const int64_t nt = retexo_theta_size(r.d_in, r.hidden, c.n_classes);
+
+        // ---- one message-passing round: X = COMBINE(Q, AGGR(Q)), emitted in bf16 for the model
+        if (c.aggr == RETEXO_GAT) {
+            const int32_t hd = r.agg_dim;
+            const int64_t ldq16 = round_up(r.rep_dim, 8), ldp = round_up(hd, 32);
+            const size_t wcount = (size_t)r.rep_dim * hd + 2 * (size_t)hd;
+            RETEXO_CUDA_TRY(cudaMemcpyAsync(b.gat_stage, in->gat_w[m - 1], sizeof(float) * wcount,
+                                            cudaMemcpyDefault, st));
+            RETEXO_TRY(convert_f32_to_bf16_launch(b.gat_stage, b.watt16, (int64_t)r.rep_dim * hd, st));
+            RETEXO_CUDA_TRY(cudaMemcpyAsync(b.gat_vec, b.gat_stage + (size_t)r.rep_dim * hd, sizeof(float) * 2 * hd,
+                                            cudaMemcpyDeviceToDevice, st));
+            RETEXO_TRY(retexo_pack_rows(q, 0, ldq, r.rep_dim, nullptr, n, b.q16, ldq16, nullptr, 0, st));
+            // P = Q W_att: the projection as a bias-free single linear layer
+            RETEXO_TRY(project_rows_launch(b.q16, ldq16, b.watt16, hd, n, hd, r.rep_dim, b.proj, ldp, st));
+            retexo_gat_params gp;
+            gp.heads = c.gat_heads; gp.head_dim = c.gat_head_dim; gp.a_src = b.gat_vec; gp.a_dst = b.gat_vec + hd;
+            gp.negative_slope = c.gat_negative_slope; gp.add_self_loop = 1;
+            RETEXO_TRY(retexo_aggregate(&g, RETEXO_GAT, b.proj, ldp, hd, &gp, nullptr, 0, 0, b.x16, ld16, b.ws_agg,
+                                        b.ws_agg_bytes, st));
+        } else {
+            RETEXO_TRY(retexo_aggregate(&g, c.aggr, q, ldq, r.agg_dim, nullptr, nullptr, 0, 1, b.x16, ld16, b.ws_agg,
+                                        b.ws_agg_bytes, st));
+        }
+
+        // ---- the round's batches and model state
+        RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld16, nullptr, 0, st));
+        if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, b.xval16, ld16, nullptr, 0, st));
+        RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta, in->theta0[m - 1], sizeof(float) * (size_t)nt, cudaMemcpyDefault, st));
+        RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta_best, b.theta, sizeof(float) * (size_t)nt, cudaMemcpyDeviceToDevice, st));
+        RETEXO_CUDA_TRY(cudaMemsetAsync(b.adam_m, 0, sizeof(float) * (size_t)nt, st));
+        RETEXO_CUDA_TRY(cudaMemsetAsync(b.adam_v, 0, sizeof(float) * (size_t)nt, st));
+        RETEXO_CUDA_TRY(cudaMemsetAsync(b.best_correct, 0, sizeof(unsigned long long), st));
+        RETEXO_CUDA_TRY(cudaMemsetAsync(b.have_best, 0, sizeof(int32_t), st));
+        RETEXO_CUDA_TRY(cudaMemsetAsync(b.best_iter_cur, 0, sizeof(int32_t), st));
+
+        retexo_mlp model{};
+        model.d_in = r.d_in; model.hidden = r.hidden; model.n_classes = c.n_classes;
+        model.theta = b.theta; model.adam_m = b.adam_m; model.adam_v = b.adam_v;
+        model.optimizer = c.optimizer; model.lr = c.lr; model.beta1 = c.beta1; model.beta2 = c.beta2;
+        model.eps = c.eps; model.step = 0;
+        retexo_mlp best = model;
+        best.theta = b.theta_best;
+
+        // ---- R training iterations; validation and best-iterate tracking stay on the device
+        for (int it = 1; it <= c.R; ++it) {
+            float* loss_slot = b.loss_history + (size_t)(m - 1) * c.R + (it - 1);
+            RETEXO_TRY(retexo_mlp_train_step(&model, b.xtr16, ld16, nullptr, 0, b.y_tr, n_tr, loss_slot, nullptr,
+                                             b.ws_step, b.ws_step_bytes, st));
+            if (n_val && (it % c.eval_every == 0 || it == c.R)) {
+                RETEXO_TRY(retexo_embed(&model, b.xval16, ld16, nullptr, n_val, nullptr, 0, nullptr, 0, nullptr, 0,
+                                        nullptr, b.y_val, reinterpret_cast<uint64_t*>(b.cur_correct), b.ws_embed,
+                                        b.ws_embed_bytes, st));
+                snapshot_if_better_kernel<<<(unsigned)((nt + 255) / 256), 256, 0, st>>>(
+                    b.cur_correct, b.best_correct, b.have_best, b.theta, b.theta_best, nt);
+                record_validation_kernel<<<1, 32, 0, st>>>(b.cur_correct, b.best_correct, b.have_best, it,
+                                                           b.best_iter_cur,
+                                                           b.val_history + (size_t)(m - 1) * c.R + (it - 1));
+            }
+        }
+        if (!n_val) {   // nothing to select on: keep the last iterate
+            RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta_best, b.theta, sizeof(float) * (size_t)nt, cudaMemcpyDeviceToDevice, st));
+            const int32_t last = c.R;
+            RETEXO_CUDA_TRY(cudaMemcpyAsync(b.best_iter_cur, &last, sizeof(int32_t), cudaMemcpyHostToDevice, st));
+        }
+        RETEXO_CUDA_TRY(cudaMemcpyAsync(b.best_val + (m - 1), b.best_correct, sizeof(unsigned long long),
+                                        cudaMemcpyDeviceToDevice, st));
+        RETEXO_CUDA_TRY(cudaMemcpyAsync(b.best_iter + (m - 1), b.best_iter_cur, sizeof(int32_t),
+                                        cudaMemcpyDeviceToDevice, st));
+
+        // ---- test accuracy of the kept and of the last iterate
+        if (n_te) {
+            RETEXO_TRY(retexo_embed(&best, b.x16, ld16, test_idx, n_te, nullptr, 0, nullptr, 0, nullptr, 0, nullptr,
+                                    b.y_test, reinterpret_cast<uint64_t*>(b.test_best + (m - 1)), b.ws_embed,
+                                    b.ws_embed_bytes, st));
+            RETEXO_TRY(retexo_embed(&model, b.x16, ld16, test_idx, n_te, nullptr, 0, nullptr, 0, nullptr, 0, nullptr,
+                                    b.y_test, reinterpret_cast<uint64_t*>(b.test_last + (m - 1)), b.ws_embed,
+                                    b.ws_embed_bytes, st));
+        } else {
+            RETEXO_CUDA_TRY(cudaMemsetAsync(b.test_best + (m - 1), 0, sizeof(unsigned long long), st));
+            RETEXO_CUDA_TRY(cudaMemsetAsync(b.test_last + (m - 1), 0, sizeof(unsigned long long), st));
+        }
+        if (out->theta_best && out->theta_best[m - 1])
+            RETEXO_CUDA_TRY(cudaMemcpyAsync(out->theta_best[m - 1], b.theta_best, sizeof(float) * (size_t)nt,
+                                            cudaMemcpyDefault, st));
+
+        // ---- emit Q^m (classifier dropped) or the final logits
+        if (m < c.K) {
+            float* qn = b.q[(m - 1) & 1];
+            const int64_t ldn = round_up(c.hidden, 32);
+            RETEXO_TRY(retexo_embed(&best, b.x16, ld16, nullptr, n, qn, ldn, nullptr, 0, nullptr, 0, nullptr, nullptr,
+                                    nullptr, b.ws_embed, b.ws_embed_bytes, st));
+            q = qn;
+            ldq = ldn;
+        } else if (out->final_logits || out->final_pred) {
+            float* lg = host ? b.final_logits : out->final_logits;
+            const int64_t ldl = host ? c.n_classes : out->ld_logits;
+            int32_t* pr = host ? b.final_pred : out->final_pred;
+            RETEXO_TRY(retexo_embed(&best, b.x16, ld16, nullptr, n, nullptr, 0, nullptr, 0,
+                                    out->final_logits ? lg : nullptr, ldl, out->final_pred ? pr : nullptr, nullptr,
+                                    nullptr, b.ws_embed, b.ws_embed_bytes, st));
+        }
+    }
+
+    // ---- results
+    const size_t kr = (size_t)c.K * c.R;
+    if (out->loss_history) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->loss_history, b.loss_history, sizeof(float) * kr, out_kind, st));
+    if (out->val_correct) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->val_correct, b.val_history, sizeof(uint64_t) * kr, out_kind, st));
+    if (out->best_val_correct) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->best_val_correct, b.best_val, sizeof(uint64_t) * c.K, out_kind, st));
+    if (out->best_iter) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->best_iter, b.best_iter, sizeof(int32_t) * c.K, out_kind, st));
+    if (out->test_correct) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->test_correct, b.test_best, sizeof(uint64_t) * c.K, out_kind, st));
+    if (out->test_correct_last) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->test_correct_last, b.test_last, sizeof(uint64_t) * c.K, out_kind, st));
+    if (out->counts && part) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->counts, b.counts, sizeof(uint64_t) * (4 + c.K), out_kind, st));
+    if (host) {
+        if (out->final_logits)
+            RETEXO_CUDA_TRY(cudaMemcpy2DAsync(out->final_logits, sizeof(float) * out->ld_logits, b.final_logits,
+                                              sizeof(float) * c.n_classes, sizeof(float) * c.n_classes, (size_t)n,
+                                              out_kind, st));
+        if (out->final_pred)
+            RETEXO_CUDA_TRY(cudaMemcpyAsync(out->final_pred, b.final_pred, sizeof(int32_t) * (size_t)n, out_kind, st));
+        RETEXO_CUDA_TRY(cudaStreamSynchronize(st));
+    }
+    return launch_status();
+}

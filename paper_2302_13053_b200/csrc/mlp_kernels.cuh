@@ -1,0 +1,305 @@
+// Kernels of the per-node model (Section 3.1): batch packing, a general
+// CUDA-core bf16 GEMM with fused epilogues (used for the skinny products and
+// as the path for shapes the tensor-core kernel does not take), softmax
+// cross-entropy with its gradient, arg-max/accuracy, and the fused
+// gradient-reduce + optimiser update.
+#pragma once
+#include "common.cuh"
+
+namespace retexo {
+
+typedef __nv_bfloat16 bf16;
+
+// ---------------------------------------------------------------- packing
+// dst[i][c] = bf16(src[idx ? idx[i] : i][c]); dst_t[c][i] likewise.  Padding
+// columns of both outputs are written as zero.
+template <bool SRC_BF16>
+__global__ void __launch_bounds__(256) pack_rows_kernel(const void* __restrict__ src, int64_t ld_src, int32_t dim,
+                                                        const int32_t* __restrict__ idx, int64_t n_rows,
+                                                        bf16* __restrict__ dst, int64_t ld_dst,
+                                                        bf16* __restrict__ dst_t, int64_t ld_t) {
+    __shared__ float tile[32][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;     // 32 x 8
+    const int64_t r0 = blockIdx.x * 32ll;
+    const int64_t c0 = blockIdx.y * 32ll;
+    for (int i = ty; i < 32; i += 8) {
+        const int64_t r = r0 + i, c = c0 + tx;
+        float v = 0.f;
+        if (r < n_rows && c < dim) {
+            const int64_t sr = idx ? idx[r] : r;
+            v = SRC_BF16 ? bf16_to_f32(static_cast<const bf16*>(src)[sr * ld_src + c])
+                         : static_cast<const float*>(src)[sr * ld_src + c];
+        }
+        tile[i][tx] = v;
+        if (dst && r < n_rows && c < ld_dst) dst[r * ld_dst + c] = f32_to_bf16(v);
+    }
+    if (!dst_t) return;
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) {
+        const int64_t c = c0 + i, r = r0 + tx;
+        if (c < dim && r < ld_t) dst_t[c * ld_t + r] = f32_to_bf16(tile[tx][i]);
+    }
+}
+
+// ---------------------------------------------------------------- GEMM
+constexpr int kBM = 64, kBN = 64, kBK = 32, kGemmThreads = 256;
+
+enum EpiMode { EPI_PARTIAL = 0, EPI_BIAS = 1, EPI_MASK = 2 };
+
+struct GemmArgs {
+    int64_t M, N, K;
+    const bf16* A; int64_t lda;            // A_T = false: [M x K]; true: stored [K x M]
+    const int32_t* a_row_idx;              // optional row gather for A (A_T = false only)
+    const bf16* B; int64_t ldb;            // B_T = false: [K x N]; true: stored [N x K]
+    int64_t k_chunk;                       // K range per blockIdx.z (multiple of kBK)
+    int mode;
+    int relu;                              // EPI_BIAS
+    const float* bias;                     // EPI_BIAS, [N] (may be null)
+    float* out_f32; int64_t ld_f32;        // EPI_BIAS (may be null)
+    bf16* out_bf16; int64_t ld_bf16;       // EPI_BIAS / EPI_MASK (may be null)
+    const bf16* mask; int64_t ld_mask;     // EPI_MASK: keep acc where mask > 0
+    float* colsum;                         // EPI_MASK: [gridDim.y x N] column sums of the kept values
+    float* partial;                        // EPI_PARTIAL: [gridDim.z x M x N]
+};
+
+template <bool A_T, bool B_T>
+__global__ void __launch_bounds__(kGemmThreads) gemm_bf16_kernel(GemmArgs g) {
+    __shared__ __align__(16) float As[kBK][kBM + 4];
+    __shared__ __align__(16) float Bs[kBK][kBN + 4];
+    __shared__ float cs[16][kBN];
+    const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
+    const int64_t m0 = blockIdx.y * (int64_t)kBM, n0 = blockIdx.x * (int64_t)kBN;
+    const int64_t kbeg = blockIdx.z * g.k_chunk;
+    const int64_t kend = min(g.K, kbeg + g.k_chunk);
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int64_t k0 = kbeg; k0 < kend; k0 += kBK) {
+#pragma unroll
+        for (int i = 0; i < (kBM * kBK) / kGemmThreads; ++i) {
+            const int e = t + i * kGemmThreads;
+            int m, k;
+            if (A_T) { k = e / kBM; m = e % kBM; } else { m = e / kBK; k = e % kBK; }
+            const int64_t gm = m0 + m, gk = k0 + k;
+            float v = 0.f;
+            if (gm < g.M && gk < kend) {
+                if (A_T) v = bf16_to_f32(g.A[gk * g.lda + gm]);
+                else {
+                    const int64_t r = g.a_row_idx ? g.a_row_idx[gm] : gm;
+                    v = bf16_to_f32(g.A[r * g.lda + gk]);
+                }
+            }
+            As[k][m] = v;
+        }
+#pragma unroll
+        for (int i = 0; i < (kBN * kBK) / kGemmThreads; ++i) {
+            const int e = t + i * kGemmThreads;
+            int n, k;
+            if (B_T) { n = e / kBK; k = e % kBK; } else { k = e / kBN; n = e % kBN; }
+            const int64_t gn = n0 + n, gk = k0 + k;
+            float v = 0.f;
+            if (gn < g.N && gk < kend) v = bf16_to_f32(B_T ? g.B[gn * g.ldb + gk] : g.B[gk * g.ldb + gn]);
+            Bs[k][n] = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kBK; ++k) {
+            const float4 a = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
+            const float4 b = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
+            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+
+    if (g.mode == EPI_PARTIAL) {
+        float* p = g.partial + (int64_t)blockIdx.z * g.M * g.N;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int64_t m = m0 + ty * 4 + i;
+            if (m >= g.M) continue;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int64_t n = n0 + tx * 4 + j;
+                if (n < g.N) p[m * g.N + n] = acc[i][j];
+            }
+        }
+        return;
+    }
+    if (g.mode == EPI_BIAS) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int64_t m = m0 + ty * 4 + i;
+            if (m >= g.M) continue;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int64_t n = n0 + tx * 4 + j;
+                if (n >= g.N) continue;
+                float v = acc[i][j] + (g.bias ? g.bias[n] : 0.f);
+                if (g.relu) v = fmaxf(v, 0.f);
+                if (g.out_f32) g.out_f32[m * g.ld_f32 + n] = v;
+                if (g.out_bf16) g.out_bf16[m * g.ld_bf16 + n] = f32_to_bf16(v);
+            }
+        }
+        return;
+    }
+    // EPI_MASK
+    float col[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int64_t m = m0 + ty * 4 + i;
+        if (m >= g.M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int64_t n = n0 + tx * 4 + j;
+            if (n >= g.N) continue;
+            const float v = bf16_to_f32(g.mask[m * g.ld_mask + n]) > 0.f ? acc[i][j] : 0.f;
+            g.out_bf16[m * g.ld_bf16 + n] = f32_to_bf16(v);
+            col[j] += v;
+        }
+    }
+    if (g.colsum) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) cs[ty][tx * 4 + j] = col[j];
+        __syncthreads();
+        if (t < kBN && n0 + t < g.N) {
+            float s = 0.f;
+            for (int r = 0; r < 16; ++r) s += cs[r][t];
+            g.colsum[(int64_t)blockIdx.y * g.N + n0 + t] = s;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- softmax CE
+// One warp per row (n_classes <= 64).  Writes dL = (softmax - onehot)/n_rows as
+// bf16 (row stride ld_dl, padding columns zero), and per-block partial sums of
+// the loss and of the columns of the unrounded dL.
+constexpr int kSmThreads = 256;
+__global__ void __launch_bounds__(kSmThreads) softmax_ce_kernel(const float* __restrict__ logits, int64_t ld_logits,
+                                                                const int32_t* __restrict__ y, int64_t n_rows,
+                                                                int32_t n_classes, bf16* __restrict__ dl, int64_t ld_dl,
+                                                                float* __restrict__ loss_partial,
+                                                                float* __restrict__ colsum_partial) {
+    __shared__ float s_loss[kSmThreads / kWarp];
+    __shared__ float s_col[kSmThreads / kWarp][64];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float inv_n = 1.0f / (float)n_rows;
+    float my_loss = 0.f, c0 = 0.f, c1 = 0.f;
+    const int64_t stride = (int64_t)gridDim.x * (kSmThreads / kWarp);
+    for (int64_t r = blockIdx.x * (int64_t)(kSmThreads / kWarp) + warp; r < n_rows; r += stride) {
+        const float* row = logits + r * ld_logits;
+        const float l0 = lane < n_classes ? row[lane] : -INFINITY;
+        const float l1 = lane + 32 < n_classes ? row[lane + 32] : -INFINITY;
+        const float mx = warp_max(fmaxf(l0, l1));
+        const float e0 = lane < n_classes ? expf(l0 - mx) : 0.f;
+        const float e1 = lane + 32 < n_classes ? expf(l1 - mx) : 0.f;
+        const float den = warp_sum(e0 + e1);
+        const int32_t yi = y[r];
+        const float ly = __shfl_sync(0xffffffffu, (yi & 32) ? l1 : l0, yi & 31);
+        my_loss += (mx + logf(den)) - ly;
+        const float g0 = (e0 / den - (lane == yi ? 1.f : 0.f)) * inv_n;
+        const float g1 = (e1 / den - (lane + 32 == yi ? 1.f : 0.f)) * inv_n;
+        if (lane < ld_dl) dl[r * ld_dl + lane] = f32_to_bf16(lane < n_classes ? g0 : 0.f);
+        if (lane + 32 < ld_dl) dl[r * ld_dl + lane + 32] = f32_to_bf16(lane + 32 < n_classes ? g1 : 0.f);
+        if (lane < n_classes) c0 += g0;
+        if (lane + 32 < n_classes) c1 += g1;
+    }
+    if (lane == 0) s_loss[warp] = my_loss;
+    s_col[warp][lane] = c0;
+    s_col[warp][lane + 32] = c1;
+    __syncthreads();
+    if (threadIdx.x < 64) {
+        float s = 0.f;
+        for (int w = 0; w < kSmThreads / kWarp; ++w) s += s_col[w][threadIdx.x];
+        if (threadIdx.x < n_classes) colsum_partial[(int64_t)blockIdx.x * n_classes + threadIdx.x] = s;
+    }
+    if (threadIdx.x == 0) {
+        float s = 0.f;
+        for (int w = 0; w < kSmThreads / kWarp; ++w) s += s_loss[w];
+        loss_partial[blockIdx.x] = s;
+    }
+}
+
+// ---------------------------------------------------------------- arg-max / accuracy
+__global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ logits, int64_t ld, int64_t n_rows,
+                                                     int32_t n_classes, int32_t* __restrict__ pred,
+                                                     const int32_t* __restrict__ y,
+                                                     unsigned long long* __restrict__ correct) {
+    const int64_t r = blockIdx.x * 256ll + threadIdx.x;
+    int hit = 0;
+    if (r < n_rows) {
+        const float* row = logits + r * ld;
+        int best = 0;
+        float bv = row[0];
+        for (int c = 1; c < n_classes; ++c) {
+            const float v = row[c];
+            if (v > bv) { bv = v; best = c; }       // strict: lowest index wins ties
+        }
+        if (pred) pred[r] = best;
+        if (y && best == y[r]) hit = 1;
+    }
+    if (correct) {
+        const unsigned b = __ballot_sync(0xffffffffu, hit);
+        if ((threadIdx.x & 31) == 0 && b) atomicAdd(correct, (unsigned long long)__popc(b));
+    }
+}
+
+// ---------------------------------------------------------------- optimiser
+struct GradSeg {
+    int64_t size;              // parameters in this segment
+    const float* partial;      // [count x size], summed in index order
+    int64_t count;
+};
+struct UpdateArgs {
+    GradSeg seg[4];
+    int n_seg;
+    float* theta;
+    float* m;
+    float* v;
+    float* grad_out;           // may be null
+    int optimizer;
+    float lr, beta1, beta2, eps, corr1, corr2;     // corr = 1 - beta^step
+    const float* loss_partial; int64_t n_loss; float inv_rows; float* loss_out;
+};
+
+__global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
+    const int64_t p = blockIdx.x * 256ll + threadIdx.x;
+    if (p == 0 && u.loss_out) {
+        float s = 0.f;
+        for (int64_t i = 0; i < u.n_loss; ++i) s += u.loss_partial[i];
+        *u.loss_out = s * u.inv_rows;
+    }
+    int64_t off = 0;
+    for (int s = 0; s < u.n_seg; ++s) {
+        if (p < off + u.seg[s].size) {
+            const int64_t q = p - off;
+            float g = 0.f;
+            for (int64_t z = 0; z < u.seg[s].count; ++z) g += u.seg[s].partial[z * u.seg[s].size + q];
+            if (u.grad_out) u.grad_out[p] = g;
+            if (u.optimizer == RETEXO_SGD) {
+                u.theta[p] -= u.lr * g;
+            } else {
+                const float m = u.beta1 * u.m[p] + (1.f - u.beta1) * g;
+                const float v = u.beta2 * u.v[p] + (1.f - u.beta2) * g * g;
+                u.m[p] = m;
+                u.v[p] = v;
+                u.theta[p] -= u.lr * (m / u.corr1) / (sqrtf(v / u.corr2) + u.eps);
+            }
+            return;
+        }
+        off += u.seg[s].size;
+    }
+}
+
+__global__ void __launch_bounds__(256) f32_to_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int64_t n) {
+    const int64_t i = blockIdx.x * 256ll + threadIdx.x;
+    if (i < n) dst[i] = f32_to_bf16(src[i]);
+}
+
+}  // namespace retexo

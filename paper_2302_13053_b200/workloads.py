@@ -4,7 +4,7 @@ This module only *draws inputs*: graphs (symmetric CSR, no self loops, no
 duplicate entries, columns sorted within a row), node features, labels,
 train/val/test index sets, a partition id per node and the initial weights of
 every round's per-node model.  It holds none of the method's arithmetic (no
-aggregation, no MLP, no counting) and depends on numpy alone, so the CPU
+aggregation, no MLP, no counting) and depends only on numpy and scipy.sparse, so the CPU
 checker and the CUDA library can both be fed from it without sharing code.
 
 The shapes follow the dataset-statistics table of the paper's Appendix B
@@ -81,32 +81,38 @@ class Workload:
 # graph helpers
 # --------------------------------------------------------------------------
 
+def csr_from_upper(n: int, upper):
+    """Symmetric CSR (int64 rowptr, int32 sorted colidx) from a scipy CSR
+    matrix holding each undirected edge once as (min, max), columns sorted."""
+    lower = upper.T.tocsr()                      # counting sort: rows b, columns a ascending
+    up_ptr = upper.indptr.astype(np.int64)
+    lo_ptr = lower.indptr.astype(np.int64)
+    rowptr = up_ptr + lo_ptr
+    colidx = np.empty(int(rowptr[-1]), dtype=np.int32)
+    # row v = [neighbours a < v (from lower)] ++ [neighbours b > v (from upper)]
+    lo_rows = np.repeat(np.arange(n, dtype=np.int64), np.diff(lo_ptr))
+    colidx[rowptr[lo_rows] + (np.arange(lo_rows.shape[0], dtype=np.int64) - lo_ptr[lo_rows])] = lower.indices
+    del lo_rows
+    up_rows = np.repeat(np.arange(n, dtype=np.int64), np.diff(up_ptr))
+    colidx[rowptr[up_rows] + np.diff(lo_ptr)[up_rows] +
+           (np.arange(up_rows.shape[0], dtype=np.int64) - up_ptr[up_rows])] = upper.indices
+    return rowptr, colidx
+
+
 def csr_from_undirected(n: int, a: np.ndarray, b: np.ndarray):
     """Symmetric CSR from distinct undirected pairs (a[i] != b[i])."""
-    a = a.astype(np.int64, copy=False)
-    b = b.astype(np.int64, copy=False)
-    key = np.concatenate([a * n + b, b * n + a])
-    key.sort(kind="stable")
-    rows = key // n
-    cols = (key - rows * n).astype(np.int32)
-    counts = np.bincount(rows, minlength=n)
-    rowptr = np.zeros(n + 1, dtype=np.int64)
-    np.cumsum(counts, out=rowptr[1:])
-    return rowptr, cols
+    import scipy.sparse as sp
+    lo = np.minimum(a, b).astype(np.int32)
+    hi = np.maximum(a, b).astype(np.int32)
+    upper = sp.coo_matrix((np.ones(lo.shape[0], dtype=np.int8), (lo, hi)), shape=(n, n)).tocsr()
+    upper.sort_indices()
+    return csr_from_upper(n, upper)
 
 
-def _dedup_pairs(n: int, u: np.ndarray, v: np.ndarray):
-    keep = u != v
-    u, v = u[keep], v[keep]
-    lo = np.minimum(u, v).astype(np.int64)
-    hi = np.maximum(u, v).astype(np.int64)
-    return lo * n + hi            # caller uniques
-
-
-def _sample_by_weight(rng, cum: np.ndarray, lo: np.ndarray, hi: np.ndarray):
-    """Draw indices i with probability proportional to the weights whose
+def _sample_by_weight(rng, cum: np.ndarray, lo, hi, m: int):
+    """Draw m indices with probability proportional to the weights whose
     cumulative sum is `cum`, restricted to the mass interval [lo, hi)."""
-    r = lo + rng.random(lo.shape[0]) * (hi - lo)
+    r = lo + rng.random(m) * (hi - lo)
     idx = np.searchsorted(cum, r, side="right")
     return np.minimum(idx, cum.shape[0] - 1)
 
@@ -138,6 +144,9 @@ def _power_law_weights(n: int, exponent: float, max_over_mean: Optional[float]):
     return (i + i0) ** (-a)
 
 
+_DRAW_CHUNKS = 16      # fixed, so that the draw does not depend on the core count
+
+
 def random_graph(rng, n: int, n_und: int, labels: np.ndarray, weights: Optional[np.ndarray],
                  frac_within: Optional[float], keep_cross: Optional[float]):
     """Draw exactly `n_und` distinct undirected edges (fewer only if the graph
@@ -152,54 +161,69 @@ def random_graph(rng, n: int, n_und: int, labels: np.ndarray, weights: Optional[
     The propensities are dealt to node ids in a seeded random order, so node
     id says nothing about degree.
     """
+    import scipy.sparse as sp
+    from concurrent.futures import ThreadPoolExecutor
+
     if weights is None:
         weights = np.ones(n, dtype=np.float64)
     else:
         weights = weights[rng.permutation(n)]
     n_blocks = int(labels.max()) + 1
-    order = np.argsort(labels, kind="stable")          # nodes grouped by block
-    w_sorted = weights[order]
-    cum = np.cumsum(w_sorted)
+    order = np.argsort(labels, kind="stable").astype(np.int32)      # nodes grouped by block
+    cum = np.cumsum(weights[order])
     total = cum[-1]
     blk_sorted = labels[order]
     starts = np.searchsorted(blk_sorted, np.arange(n_blocks), side="left")
     ends = np.searchsorted(blk_sorted, np.arange(n_blocks), side="right")
     cum0 = np.concatenate([[0.0], cum])
-    blk_lo = cum0[starts]
-    blk_hi = cum0[ends]
+    blk_lo, blk_hi = cum0[starts], cum0[ends]
 
-    have = np.empty(0, dtype=np.int64)
-    need = n_und
-    for _ in range(64):
-        if need <= 0:
-            break
-        m = int(need * 1.15) + 1024
-        zeros = np.zeros(m)
-        iu = _sample_by_weight(rng, cum, zeros, zeros + total)
+    def draw(args):
+        seed, m = args
+        r = np.random.default_rng(seed)
+        iu = _sample_by_weight(r, cum, 0.0, total, m)
         if frac_within is not None:
-            within = rng.random(m) < frac_within
+            within = r.random(m) < frac_within
             b = blk_sorted[iu]
-            lo = np.where(within, blk_lo[b], 0.0)
-            hi = np.where(within, blk_hi[b], total)
-            iv = _sample_by_weight(rng, cum, lo, hi)
+            iv = _sample_by_weight(r, cum, np.where(within, blk_lo[b], 0.0), np.where(within, blk_hi[b], total), m)
         else:
-            iv = _sample_by_weight(rng, cum, zeros, zeros + total)
+            iv = _sample_by_weight(r, cum, 0.0, total, m)
+        keep = iu != iv
         if keep_cross is not None:
-            cross = blk_sorted[iu] != blk_sorted[iv]
-            keep = (~cross) | (rng.random(m) < keep_cross)
-            iu, iv = iu[keep], iv[keep]
-        keys = _dedup_pairs(n, order[iu], order[iv])
-        have = np.unique(np.concatenate([have, keys]))
-        if have.shape[0] >= n_und:
+            keep &= (blk_sorted[iu] == blk_sorted[iv]) | (r.random(m) < keep_cross)
+        u, v = order[iu[keep]], order[iv[keep]]
+        return np.minimum(u, v), np.maximum(u, v)
+
+    upper = sp.csr_matrix((n, n), dtype=np.int8)
+    yield_rate = 1.0
+    for attempt in range(64):
+        need = n_und - upper.nnz
+        if need <= 0 or upper.nnz >= n * (n - 1) // 2:
             break
-        need = n_und - have.shape[0]
-    if have.shape[0] > n_und:
-        sel = rng.permutation(have.shape[0])[:n_und]
-        sel.sort()
-        have = have[sel]
-    a = have // n
-    b = have - a * n
-    return csr_from_undirected(n, a, b)
+        m = int(need * (1.08 if attempt == 0 else 1.3) / max(yield_rate, 1e-3)) + 1024
+        per = (m + _DRAW_CHUNKS - 1) // _DRAW_CHUNKS
+        seeds = rng.bit_generator.seed_seq.spawn(_DRAW_CHUNKS)
+        with ThreadPoolExecutor(max_workers=min(_DRAW_CHUNKS, 16)) as ex:
+            parts = list(ex.map(draw, [(sd, per) for sd in seeds]))
+        lo = np.concatenate([p[0] for p in parts])
+        hi = np.concatenate([p[1] for p in parts])
+        del parts
+        add = sp.coo_matrix((np.ones(lo.shape[0], dtype=np.int8), (lo, hi)), shape=(n, n)).tocsr()
+        before = upper.nnz
+        upper = upper + add if upper.nnz else add
+        upper.sum_duplicates()
+        upper.data[:] = 1
+        yield_rate = max((upper.nnz - before) / float(per * _DRAW_CHUNKS), 1e-3)
+    if upper.nnz > n_und:                      # thin out to the exact count
+        excess = upper.nnz - n_und
+        drop = np.unique(rng.integers(0, upper.nnz, size=int(excess * 1.3) + 64))
+        while drop.shape[0] < excess:
+            drop = np.unique(np.concatenate([drop, rng.integers(0, upper.nnz, size=excess)]))
+        drop = rng.permutation(drop)[:excess]
+        upper.data[drop] = 0
+        upper.eliminate_zeros()
+    upper.sort_indices()
+    return csr_from_upper(n, upper)
 
 
 # --------------------------------------------------------------------------

@@ -1,0 +1,121 @@
+"""CUDA per-node model (retexo_pack_rows, retexo_mlp_train_step, retexo_embed)
+against the CPU checker.
+
+Both sides round the operands of every matrix product to bf16 and accumulate
+wider (GPU fp32, checker double), so against the checker run with the same
+operand rounding the logits agree far inside the stated 2e-2 relative
+tolerance; the unrounded checker is compared at 2e-2 as well."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import assert_logits_close, dev
+
+pytestmark = pytest.mark.gpu
+
+
+def B():
+    from paper_2302_13053_b200 import binding
+    return binding
+
+
+def make_pair(d_in, hidden, n_classes, seed, opt=oracle.ADAM, lr=0.01):
+    rng = np.random.default_rng(seed)
+    out1 = hidden if hidden > 0 else n_classes
+    w1 = (rng.standard_normal((d_in, out1)) / np.sqrt(d_in)).astype(np.float32)
+    b1 = (rng.standard_normal(out1) * 0.1).astype(np.float32)
+    w2 = (rng.standard_normal((hidden, n_classes)) / np.sqrt(max(hidden, 1))).astype(np.float32) if hidden else None
+    b2 = (rng.standard_normal(n_classes) * 0.1).astype(np.float32) if hidden else None
+    ref = oracle.Mlp(d_in, hidden, n_classes, w1, b1, w2, b2, optimizer=opt, lr=lr, round_bf16=True)
+    gpu = B().Mlp(d_in, hidden, n_classes, w1, b1, w2, b2, optimizer=opt, lr=lr)
+    return ref, gpu
+
+
+def test_pack_rows_gathers_rounds_and_transposes():
+    rng = np.random.default_rng(0)
+    src = rng.standard_normal((70, 37)).astype(np.float32)
+    idx = rng.integers(0, 70, 45).astype(np.int32)
+    want = torch.from_numpy(src[idx]).to(torch.bfloat16)
+    for source in (dev(src), dev(src).to(torch.bfloat16)):
+        dst, dst_t = B().retexo_pack_rows(source, dev(idx), transpose=True)
+        assert dst.shape == (45, 40) and dst_t.shape == (37, 48)
+        ref = want if source.dtype == torch.float32 else want
+        assert torch.equal(dst[:, :37].cpu(), ref)
+        assert torch.equal(dst_t[:, :45].cpu(), ref.T)
+        assert dst[:, 37:].abs().sum() == 0 and dst_t[:, 45:].abs().sum() == 0
+    dst, _ = B().retexo_pack_rows(dev(src), None, dim=20)
+    assert torch.equal(dst[:, :20].cpu(), torch.from_numpy(src[:, :20]).to(torch.bfloat16))
+
+
+@pytest.mark.parametrize("d_in,hidden,n_classes,n", [(5, 0, 3, 17), (64, 64, 7, 140), (33, 20, 4, 65),
+                                                     (1433, 64, 7, 140), (100, 256, 47, 300), (1204, 256, 41, 513),
+                                                     (256, 0, 3, 60), (70, 512, 64, 129)])
+@pytest.mark.parametrize("opt", [oracle.SGD, oracle.ADAM])
+def test_train_steps_track_the_checker(d_in, hidden, n_classes, n, opt):
+    rng = np.random.default_rng(d_in + hidden)
+    x = rng.standard_normal((n, d_in)).astype(np.float32)
+    y = rng.integers(0, n_classes, n).astype(np.int32)
+    ref, gpu = make_pair(d_in, hidden, n_classes, 1, opt=opt, lr=0.02)
+    x16, x_t = B().retexo_pack_rows(dev(x), None, transpose=True)
+    yd = dev(y)
+    for it in range(4):
+        rl, rg = ref.train_step(x, y, return_grad=True)
+        gl, gg = B().retexo_mlp_train_step(gpu, x16, yd, x_t=x_t, return_grad=True)
+        assert abs(gl.item() - rl) <= 2e-4 * max(1.0, abs(rl)), (it, gl.item(), rl)
+        gg = gg.cpu().numpy().astype(np.float64)
+        scale = np.abs(rg).max()
+        assert np.abs(gg - rg).max() <= 2e-3 * scale + 1e-7, (it, np.abs(gg - rg).max(), scale)
+        assert gpu.step == ref.step == it + 1
+    # weights after 4 updates (fp32 state on the GPU, double in the checker)
+    gt = gpu.theta.cpu().numpy().astype(np.float64)
+    assert np.abs(gt - ref.theta).max() <= 5e-3 * max(1.0, np.abs(ref.theta).max())
+
+
+def test_zero_weights_give_log_of_class_count():
+    n, d, h, o = 50, 12, 8, 5
+    x = np.random.default_rng(3).standard_normal((n, d)).astype(np.float32)
+    y = np.random.default_rng(4).integers(0, o, n).astype(np.int32)
+    gpu = B().Mlp(d, h, o, np.zeros((d, h)), np.zeros(h), np.zeros((h, o)), np.zeros(o), optimizer=oracle.SGD, lr=0.1)
+    x16, _ = B().retexo_pack_rows(dev(x))
+    loss = B().retexo_mlp_train_step(gpu, x16, dev(y))
+    assert abs(loss.item() - np.log(o)) < 1e-6
+
+
+@pytest.mark.parametrize("d_in,hidden,n_classes,n", [(64, 64, 7, 500), (1000, 128, 3, 300), (33, 0, 5, 200),
+                                                     (602, 256, 41, 257)])
+def test_embed_matches_checker_and_stated_tolerance(d_in, hidden, n_classes, n):
+    rng = np.random.default_rng(7)
+    x = rng.standard_normal((n, d_in)).astype(np.float32)
+    ref, gpu = make_pair(d_in, hidden, n_classes, 2)
+    y = rng.integers(0, n_classes, n).astype(np.int32)
+    x16, _ = B().retexo_pack_rows(dev(x))
+    out = B().retexo_embed(gpu, x16, y=dev(y), want_hidden=hidden > 0, want_hidden_bf16=hidden > 0,
+                           want_logits=True, want_pred=True)
+    r = ref.embed(x, y=y, want_hidden=hidden > 0)
+    lg = out["logits"].cpu().numpy()
+    assert_logits_close(lg, r["logits"], rel=2e-3, what="vs bf16-operand checker")
+    exact = oracle.Mlp(d_in, hidden, n_classes, **{k: v for k, v in ref.unpack().items()}, round_bf16=False)
+    assert_logits_close(lg, exact.embed(x)["logits"], rel=2e-2, what="vs unrounded checker")
+    if hidden > 0:
+        h = out["hidden"].cpu().numpy()
+        assert_logits_close(h, r["hidden"], rel=2e-3, what="hidden")
+        assert torch.equal(out["hidden_bf16"][:, :hidden].cpu(), out["hidden"].to(torch.bfloat16).cpu())
+    # predictions: exact wherever the reference margin is clear of the tolerance
+    srt = np.sort(r["logits"], axis=1)
+    clear = (srt[:, -1] - srt[:, -2]) > 4e-3 * np.abs(r["logits"]).max(axis=1)
+    pred = out["pred"].cpu().numpy()
+    np.testing.assert_array_equal(pred[clear], r["pred"][clear])
+    np.testing.assert_array_equal(pred, lg.argmax(1))            # argmax of its own logits, lowest index on ties
+    assert out["correct"] == int((pred == y).sum())
+    # row gather
+    idx = rng.integers(0, n, 77).astype(np.int32)
+    sub = B().retexo_embed(gpu, x16, row_idx=dev(idx), want_logits=True)
+    np.testing.assert_array_equal(sub["logits"].cpu().numpy(), lg[idx])
+
+
+def test_argmax_tie_rule_lowest_index():
+    gpu = B().Mlp(8, 0, 4, np.zeros((8, 4)), np.array([1.0, 3.0, 3.0, 3.0]))
+    x16, _ = B().retexo_pack_rows(dev(np.ones((5, 8), dtype=np.float32)))
+    out = B().retexo_embed(gpu, x16, want_pred=True)
+    assert out["pred"].cpu().tolist() == [1] * 5
