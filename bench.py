@@ -1,0 +1,429 @@
+#!/usr/bin/env python
+"""Benchmark of the lazy-message-passing hot path on B200.
+
+One "step" is one pass of the whole hot path over one synthetic workload: the
+cross-partition count, then for each of the K rounds one full-graph
+aggregation, R training iterations of the round's per-node model (with
+validation every iteration and best-iterate tracking) and the emission of the
+next representations — i.e. one end-to-end K-round training run.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1..5] [--impl reference]
+
+Prints one JSON line.  `value` = edges aggregated per second of whole-job time
+(K rounds x directed edges / step time, summed over replicas); `ms_per_step`
+is the end-to-end K-round train time.  With --gpus N > 1 (under torchrun) every
+rank runs an independent replica: the path is specified for one GPU, without
+sharding or collectives.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "edges aggregated/s"
+UNIT = "edges/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_burst=p["bf16_tflops"], bf16_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_burst=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def build_workload(index: int, scale: float):
+    from paper_2302_13053_b200 import workloads as wl
+    t = time.time()
+    w = wl.make_config(index, scale=scale)
+    ws = wl.initial_weights(w)
+    return w, ws, time.time() - t
+
+
+def make_problem(w, ws, host: bool, R: int):
+    from paper_2302_13053_b200 import binding as B
+    return B.LmpProblem(w.aggr, w.K, R, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
+                        w.train_idx, w.val_idx, w.test_idx, ws, part=w.part, n_parts=w.n_parts, heads=w.heads,
+                        head_dim=w.head_dim, negative_slope=w.negative_slope, host=host)
+
+
+def launches_per_step(w, R: int) -> int:
+    """Kernels the library launches in one K-round run (memsets and copies not counted)."""
+    from paper_2302_13053_b200 import workloads as wl
+    total = 3 + 1                                    # label gathers, history fill
+    n_parts = w.n_parts
+    total += (2 if n_parts <= 8192 else 3) + 1       # count kernels + finalize + pack
+    for rd in w.round_dims():
+        h = rd["hidden"]
+        if w.aggr == wl.GAT:
+            total += 1 + 1 + 1 + 2                   # weight convert, pack, projection, scores + rows
+        else:
+            total += 3                               # prep, warp rows, block rows
+        total += 2                                   # train / val batches
+        step = 8 if h > 0 else 5
+        ev = (4 if h > 0 else 3) + 2
+        total += R * (step + ev)
+        total += 2 * (4 if h > 0 else 3)             # test accuracy, kept and last iterate
+        total += 2 if h > 0 else 3                   # emission of Q^m / final logits
+    return total
+
+
+def time_calls(fn, reps: int, warm: int = 3):
+    import torch
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+    for a, b in evs:
+        a.record()
+        fn()
+        b.record()
+    torch.cuda.synchronize()
+    ts = [a.elapsed_time(b) for a, b in evs]
+    return statistics.mean(ts), min(ts)
+
+
+def phase_breakdown(w, ws, R: int, peaks):
+    """Times each entry point alone, at the shapes and launch configuration the
+    K-round run uses, and derives the roofline figures per kernel."""
+    import torch
+    from paper_2302_13053_b200 import binding as B
+    from paper_2302_13053_b200 import workloads as wl
+    dev = "cuda"
+    rp = torch.from_numpy(w.rowptr).to(dev)
+    ci = torch.from_numpy(w.colidx).to(dev)
+    n, e = w.n_nodes, w.n_edges
+    tr = torch.from_numpy(w.train_idx).to(dev)
+    va = torch.from_numpy(w.val_idx).to(dev)
+    y = torch.from_numpy(w.labels).to(dev)
+    y_tr, y_va = y[tr.long()].contiguous(), y[va.long()].contiguous()
+    phases = []
+    q = None
+    for rd, wt in zip(w.round_dims(), ws):
+        m = rd["round"]
+        d = rd["agg_dim"]
+        ld = (rd["rep_dim"] + 31) // 32 * 32
+        if m == 1:
+            q = torch.zeros((n, ld), dtype=torch.float32, device=dev)
+            q[:, :w.d0] = torch.from_numpy(w.features).to(dev)
+        else:
+            q = torch.rand((n, ld), dtype=torch.float32, device=dev)
+        width = rd["d_in"]
+        x16 = torch.empty((n, (width + 7) // 8 * 8), dtype=torch.bfloat16, device=dev)
+        if w.aggr == wl.GAT:
+            hd = w.heads * w.head_dim
+            p = torch.randn((n, (hd + 31) // 32 * 32), dtype=torch.float32, device=dev)
+            gat = dict(heads=w.heads, head_dim=w.head_dim, a_src=torch.from_numpy(wt["a_src"]),
+                       a_dst=torch.from_numpy(wt["a_dst"]), negative_slope=w.negative_slope, add_self_loop=1)
+            fn = lambda: B.retexo_aggregate(w.aggr, rp, ci, p, dim=hd, gat=gat, want_f32=False, out_bf16=x16)
+            alg = e * (4 * hd + 4 * w.heads + 4) + 8 * (n + 1) + n * hd * 2
+        else:
+            fn = lambda: B.retexo_aggregate(w.aggr, rp, ci, q, dim=d, want_f32=False, out_bf16=x16)
+            alg = e * (4 * d + 4) + 8 * (n + 1) + n * width * 2
+        mean_ms, best_ms = time_calls(fn, 5)
+        phases.append(dict(kernel="aggregate", round=m, calls_per_step=1, ms=mean_ms, best_ms=best_ms, bound="hbm",
+                           algorithmic_bytes=alg, achieved=alg / mean_ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s",
+                           edges_per_s=e / mean_ms * 1e3))
+        # the round's model at its training / validation / full shapes
+        model = B.Mlp(rd["d_in"], rd["hidden"], w.n_classes, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
+        xtr, xtr_t = B.retexo_pack_rows(x16, tr, dim=width, transpose=True)
+        xva, _ = B.retexo_pack_rows(x16, va, dim=width)
+        H, O = rd["hidden"], w.n_classes
+        n_tr, n_va = tr.numel(), va.numel()
+        if H > 0:
+            flops_step = 2.0 * n_tr * (2 * width * H + 3 * H * O)
+            flops_fwd = lambda rows: 2.0 * rows * (width * H + H * O)
+        else:
+            flops_step = 2.0 * n_tr * 2 * width * O
+            flops_fwd = lambda rows: 2.0 * rows * width * O
+        import ctypes as C
+        need = B.lib().retexo_mlp_train_step_workspace_size(C.c_int32(width), C.c_int32(H), C.c_int32(O),
+                                                            C.c_int64(n_tr))
+        ws_step = torch.empty(int(need), dtype=torch.uint8, device=dev)
+        mean_ms, best_ms = time_calls(lambda: B.retexo_mlp_train_step(model, xtr, y_tr, x_t=xtr_t, workspace=ws_step), 10)
+        phases.append(dict(kernel="mlp_train_step", round=m, calls_per_step=R, ms=mean_ms, best_ms=best_ms,
+                           bound="tensor", flops=flops_step, achieved=flops_step / mean_ms / 1e9,
+                           peak=peaks["bf16_sustained"], unit="TFLOP/s"))
+        mean_ms, best_ms = time_calls(lambda: B.retexo_embed(model, xva, y=y_va), 10)
+        phases.append(dict(kernel="embed_validation", round=m, calls_per_step=R, ms=mean_ms, best_ms=best_ms,
+                           bound="tensor", flops=flops_fwd(n_va), achieved=flops_fwd(n_va) / mean_ms / 1e9,
+                           peak=peaks["bf16_sustained"], unit="TFLOP/s"))
+        if H > 0:
+            mean_ms, best_ms = time_calls(lambda: B.retexo_embed(model, x16, want_hidden=True), 3, warm=1)
+            fl = 2.0 * n * width * H
+        else:
+            mean_ms, best_ms = time_calls(lambda: B.retexo_embed(model, x16, want_logits=True, want_pred=True), 3, warm=1)
+            fl = 2.0 * n * width * O
+        phases.append(dict(kernel="embed_all_rows", round=m, calls_per_step=1, ms=mean_ms, best_ms=best_ms,
+                           bound="tensor", flops=fl, achieved=fl / mean_ms / 1e9, peak=peaks["bf16_sustained"],
+                           unit="TFLOP/s"))
+        del model, xtr, xtr_t, xva, ws_step
+    part = torch.from_numpy(w.part).to(dev)
+    dims = [rd["rep_dim"] for rd in w.round_dims()]
+    mean_ms, best_ms = time_calls(lambda: B.retexo_cross_partition_bytes(rp, ci, part, w.n_parts, dims, 4,
+                                                                         per_part=False), 5)
+    alg = 8 * e + 8 * (n + 1) + 4 * n
+    phases.append(dict(kernel="cross_partition_count", round=0, calls_per_step=1, ms=mean_ms, best_ms=best_ms,
+                       bound="hbm", algorithmic_bytes=alg, achieved=alg / mean_ms / 1e6, peak=peaks["hbm_gbs"],
+                       unit="GB/s"))
+    for p in phases:
+        p["frac"] = p["achieved"] / p["peak"]
+    return phases
+
+
+def oracle_sample(w, ws, R: int, budget_rows: int = 1536, budget_train: int = 2048):
+    """Times the CPU checker on a bounded sample of the workload and
+    extrapolates to one full step (K rounds)."""
+    import oracle
+    rng = np.random.default_rng(0)
+    n, e = w.n_nodes, w.n_edges
+    deg = np.diff(w.rowptr)
+    rows = np.sort(rng.choice(n, size=min(n, budget_rows), replace=False))
+    sample_edges = int(deg[rows].sum())
+    total = 0.0
+    detail = []
+    for rd, wt in zip(w.round_dims(), ws):
+        d = rd["rep_dim"]
+        q = w.features if rd["round"] == 1 else rng.standard_normal((n, d)).astype(np.float32)
+        t = time.time()
+        if w.aggr == 2:
+            hd = w.heads * w.head_dim
+            p = rng.standard_normal((n, hd)).astype(np.float32)
+            oracle.aggregate(2, w.rowptr, w.colidx, p, rows=rows,
+                             gat=dict(heads=w.heads, head_dim=w.head_dim, a_src=wt["a_src"], a_dst=wt["a_dst"]))
+        else:
+            oracle.aggregate(w.aggr, w.rowptr, w.colidx, q, rows=rows)
+        t_agg = (time.time() - t) * (e / max(1, sample_edges))
+        n_tr = len(w.train_idx)
+        sub = min(n_tr, budget_train)
+        x = rng.standard_normal((sub, rd["d_in"])).astype(np.float32)
+        y = w.labels[w.train_idx[:sub]]
+        m = oracle.Mlp(rd["d_in"], rd["hidden"], w.n_classes, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
+        t = time.time()
+        m.train_step(x, y)
+        t_step = (time.time() - t) * (n_tr / sub)
+        t = time.time()
+        m.embed(x, y=y, want_logits=False)
+        t_fwd_row = (time.time() - t) / sub
+        t_round = t_agg + R * (t_step + t_fwd_row * len(w.val_idx)) + t_fwd_row * (n + 2 * len(w.test_idx))
+        detail.append(dict(round=rd["round"], aggregate_s=t_agg, train_step_s=t_step, round_s=t_round))
+        total += t_round
+    return total, detail, "aggregation of %d sampled rows (%d edges) and one train step + forward on %d train rows per round, scaled to the full graph and R=%d" % (len(rows), sample_edges, min(len(w.train_idx), budget_train), R)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    w, ws, _ = build_workload(args.config, args.scale)
+    R = args.iters or w.R
+    times = []
+    sample = ""
+    for _ in range(args.warmup):
+        oracle_sample(w, ws, R, budget_rows=256, budget_train=256)
+    for _ in range(args.steps):
+        t, detail, sample = oracle_sample(w, ws, R)
+        times.append(t)
+    step_s = statistics.mean(times)
+    value = w.K * w.n_edges / step_s
+    line = dict(impl="reference", metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=step_s * 1e3, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=w.name, n_nodes=w.n_nodes, n_edges=w.n_edges, K=w.K, R=R,
+                            note="CPU checker timed on a bounded sample per step and extrapolated"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=oracle.n_threads(), kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=4, help="workload 1..5 (default 4: the Reddit-shaped SAGE run)")
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (profiling captures only)")
+    ap.add_argument("--iters", type=int, default=0, help="override R, the iterations per round")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-breakdown", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2302_13053_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl")
+    peaks = load_peaks()
+
+    w, ws, gen_s = build_workload(args.config, args.scale)
+    R = args.iters or w.R
+    prob = make_problem(w, ws, host=False, R=R)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        B.retexo_lmp_train(prob)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(args.steps):
+        B.retexo_lmp_train(prob)
+    stop.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = start.elapsed_time(stop)
+    if world > 1:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    edges_per_step = w.K * w.n_edges
+    value = world * edges_per_step / (ms_per_step * 1e-3)
+    res = prob.results()
+
+    # ---- end to end through the host-buffer entry point: H2D of all inputs and D2H of results inside
+    e2e = None
+    if not args.no_e2e:
+        del prob
+        torch.cuda.empty_cache()
+        hprob = make_problem(w, ws, host=True, R=R)
+        for _ in range(2):
+            B.retexo_lmp_train(hprob)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            B.retexo_lmp_train(hprob)          # synchronises the stream before returning
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        e2e = dict(value=world * edges_per_step * args.steps / dt, unit=UNIT, ms_per_step=dt / args.steps * 1e3,
+                   h2d_bytes_per_step=int(hprob.h2d_bytes), d2h_bytes_per_step=int(hprob.d2h_bytes))
+        del hprob
+        torch.cuda.empty_cache()
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+                ms_per_step=ms_per_step, higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16",
+                data="synthetic",
+                config=dict(workload=w.name, n_nodes=w.n_nodes, n_edges=w.n_edges, d0=w.d0, K=w.K, R=R,
+                            hidden=w.hidden, n_classes=w.n_classes, n_train=len(w.train_idx),
+                            aggregation_dtype="fp32 in, fp32 accumulate", mlp_dtype="bf16 operands, fp32 accumulate",
+                            l2="inputs larger than L2, no flush" if w.n_nodes * w.d0 * 4 > 126e6 else
+                               "working set fits L2: reported warm",
+                            parallelism="replicas only" if world > 1 else "single GPU",
+                            generation_s=round(gen_s, 1)),
+                clocks=clocks, e2e=e2e, gpu_launches=launches_per_step(w, R) * args.steps,
+                end_to_end_train_time_ms=ms_per_step,
+                accuracy=dict(test=res["test_acc"], test_last_iterate=res["test_acc_last"]),
+                counts=dict(cross_edges=res["counts"]["cross_edges"], boundary_pairs=res["counts"]["boundary_pairs"],
+                            bytes_total=res["counts"]["bytes_total"]))
+
+    if not args.no_breakdown:
+        phases = phase_breakdown(w, ws, R, peaks)
+        for p in phases:
+            p["share_of_step"] = p["ms"] * p["calls_per_step"] / ms_per_step
+        dom = max(phases, key=lambda p: p["share_of_step"])
+        line["roofline"] = dict(kernel="%s round %d" % (dom["kernel"], dom["round"]), bound=dom["bound"],
+                                achieved=dom["achieved"], peak=dom["peak"], unit=dom["unit"], frac=dom["frac"],
+                                traffic=None, peak_source=peaks["source"], share_of_step=dom["share_of_step"])
+        line["phases"] = [dict(kernel=p["kernel"], round=p["round"], ms=round(p["ms"], 4), calls=p["calls_per_step"],
+                               share=round(p["share_of_step"], 4), bound=p["bound"], achieved=round(p["achieved"], 2),
+                               unit=p["unit"], frac=round(p["frac"], 4),
+                               **({"edges_per_s": p["edges_per_s"]} if "edges_per_s" in p else {}))
+                          for p in phases]
+    if not args.no_cpu_baseline:
+        import oracle
+        t, detail, sample = oracle_sample(w, ws, R)
+        line["cpu_baseline"] = dict(value=edges_per_step / t, unit=UNIT, cores=oracle.n_threads(), kind="oracle",
+                                    sample=sample, est_step_s=t)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -180,6 +180,16 @@ class Mlp:
         _check(rc, "oracle_mlp_train_step")
         return (loss.value, grad) if return_grad else loss.value
 
+    def apply_update(self, grad: np.ndarray) -> None:
+        """The optimiser update alone, with a gradient given by the caller."""
+        g = np.ascontiguousarray(grad, dtype=np.float64)
+        assert g.shape == self.theta.shape
+        self.step += 1
+        rc = lib().oracle_apply_update(C.c_int64(self.theta.shape[0]), _p(self.theta), _p(self.m), _p(self.v), _p(g),
+                                       C.c_int32(self.optimizer), C.c_double(self.lr), C.c_double(self.beta1),
+                                       C.c_double(self.beta2), C.c_double(self.eps), C.c_int64(self.step))
+        _check(rc, "oracle_apply_update")
+
     def embed(self, x: np.ndarray, row_idx: Optional[np.ndarray] = None, y: Optional[np.ndarray] = None,
               want_hidden: bool = False, want_logits: bool = True):
         """Forward over rows; returns dict(hidden, logits, pred, correct)."""
@@ -227,12 +237,18 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
               rowptr, colidx, features, labels, train_idx, val_idx, test_idx,
               weights: List[Dict[str, np.ndarray]], gat: Optional[Dict] = None,
               optimizer: int = ADAM, round_bf16: bool = True, eval_every: int = 1,
-              part=None, n_parts: int = 0) -> Dict:
+              part=None, n_parts: int = 0, forced_best_iter: Optional[Sequence[int]] = None) -> Dict:
     """Lazy message passing (Section 3.1): for each layer m = 1..K, one
     message-passing round builds the layer's inputs, the layer (with a
     temporary classifier unless it is the last) is trained alone for R
     iterations, the iterate with the best validation accuracy (earliest on
-    ties) is kept, and its representations feed the next round."""
+    ties) is kept, and its representations feed the next round.
+
+    forced_best_iter (a test hook): keep the given 1-based iterate in each
+    round instead of the checker's own choice.  The choice is an arg-max over
+    floating-point results, so two correct implementations may pick different
+    iterates on a flat validation curve; fixing it lets everything downstream
+    of the choice be compared."""
     labels = np.ascontiguousarray(labels, dtype=np.int32)
     q = _f32(features)
     y_tr, y_va, y_te = labels[train_idx], labels[val_idx], labels[test_idx]
@@ -267,7 +283,10 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
             if r % eval_every == 0 or r == R:
                 c = model.embed(x, row_idx=val_idx, y=y_va, want_logits=False)["correct"]
                 val_hist.append(c)
-                if c > best_correct:
+                if forced_best_iter is not None:
+                    if r == forced_best_iter[m - 1]:
+                        best, best_correct, best_iter = model.copy(), c, r
+                elif c > best_correct:
                     best, best_correct, best_iter = model.copy(), c, r
         last_test = model.embed(x, row_idx=test_idx, y=y_te, want_logits=False)["correct"]
         best_test = best.embed(x, row_idx=test_idx, y=y_te, want_logits=False)["correct"]

@@ -279,6 +279,27 @@ static int rounded_weights(int32_t d_in, int32_t hidden, int32_t n_classes, cons
     return ORACLE_OK;
 }
 
+/* The optimiser update alone: SGD (theta -= lr g) or Adam (bias-corrected,
+ * eps outside the root, no weight decay); `step` is the 1-based count of this
+ * update.  Also callable on its own, e.g. with a gradient computed elsewhere. */
+int oracle_apply_update(int64_t nt, double *theta, double *adam_m, double *adam_v, const double *grad,
+                        int32_t optimizer, double lr, double beta1, double beta2, double eps, int64_t step)
+{
+    if (optimizer == 0) {
+        for (int64_t p = 0; p < nt; ++p) theta[p] -= lr * grad[p];
+        return ORACLE_OK;
+    }
+    if (!adam_m || !adam_v || step < 1) return ORACLE_BAD_ARG;
+    double c1 = 1.0 - pow(beta1, (double)step), c2 = 1.0 - pow(beta2, (double)step);
+    for (int64_t p = 0; p < nt; ++p) {
+        adam_m[p] = beta1 * adam_m[p] + (1.0 - beta1) * grad[p];
+        adam_v[p] = beta2 * adam_v[p] + (1.0 - beta2) * grad[p] * grad[p];
+        double mh = adam_m[p] / c1, vh = adam_v[p] / c2;
+        theta[p] -= lr * mh / (sqrt(vh) + eps);
+    }
+    return ORACLE_OK;
+}
+
 #define GRAD_CHUNKS 64
 
 /* One full-batch training step (Section 2.3: forward, loss, backward, update;
@@ -395,18 +416,7 @@ int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
         for (int64_t p = 0; p < nt; ++p) grad[p] += part[(int64_t)ch * nt + p];
     free(part);
 
-    /* update */
-    if (optimizer == 0) {
-        for (int64_t p = 0; p < nt; ++p) theta[p] -= lr * grad[p];
-    } else {
-        double c1 = 1.0 - pow(beta1, (double)step), c2 = 1.0 - pow(beta2, (double)step);
-        for (int64_t p = 0; p < nt; ++p) {
-            adam_m[p] = beta1 * adam_m[p] + (1.0 - beta1) * grad[p];
-            adam_v[p] = beta2 * adam_v[p] + (1.0 - beta2) * grad[p] * grad[p];
-            double mh = adam_m[p] / c1, vh = adam_v[p] / c2;
-            theta[p] -= lr * mh / (sqrt(vh) + eps);
-        }
-    }
+    oracle_apply_update(nt, theta, adam_m, adam_v, grad, optimizer, lr, beta1, beta2, eps, step);
     if (loss_out) *loss_out = loss;
     if (grad_out) memcpy(grad_out, grad, sizeof(double) * (size_t)nt);
     free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad);

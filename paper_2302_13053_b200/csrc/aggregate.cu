@@ -420,8 +420,10 @@ extern "C" int retexo_aggregate(const retexo_csr* g, int32_t type, const float* 
                                 void* workspace, size_t workspace_bytes, void* stream) {
     if (!g || g->n_nodes < 0 || g->n_edges < 0 || g->n_nodes > INT32_MAX) return RETEXO_ERR_INVALID_ARG;
     if (type != RETEXO_GCN && type != RETEXO_SAGE_MEAN && type != RETEXO_GAT) return RETEXO_ERR_INVALID_ARG;
-    if (dim <= 0 || ldq < dim || (!out && !out_bf16)) return RETEXO_ERR_INVALID_ARG;
-    if (g->n_nodes > 0 && (!g->rowptr || !q || (g->n_edges > 0 && !g->colidx))) return RETEXO_ERR_INVALID_ARG;
+    if (dim <= 0 || ldq < dim) return RETEXO_ERR_INVALID_ARG;
+    if (g->n_nodes == 0) return RETEXO_OK;                      // nothing to aggregate
+    if (!out && !out_bf16) return RETEXO_ERR_INVALID_ARG;
+    if (!g->rowptr || !q || (g->n_edges > 0 && !g->colidx)) return RETEXO_ERR_INVALID_ARG;
     const int64_t width = (type == RETEXO_SAGE_MEAN && concat_self) ? 2 * (int64_t)dim : dim;
     if (out && ldout < width) return RETEXO_ERR_INVALID_ARG;
     if (out_bf16 && ldout_bf16 < width) return RETEXO_ERR_INVALID_ARG;
@@ -433,7 +435,6 @@ extern "C" int retexo_aggregate(const retexo_csr* g, int32_t type, const float* 
     }
     const size_t need = retexo_aggregate_workspace_size(g->n_nodes, g->n_edges, type, dim, gat ? gat->heads : 0);
     if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
-    if (g->n_nodes == 0) return RETEXO_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int n_sm = sm_count();
     if (n_sm <= 0) return RETEXO_ERR_CUDA;

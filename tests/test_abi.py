@@ -55,6 +55,9 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
     g = _Csr(-1, 0, None, None)
     assert lib.retexo_aggregate(C.byref(g), 0, None, C.c_int64(4), 4, None, None, C.c_int64(4), 1, None,
                                 C.c_int64(0), None, C.c_size_t(0), None) == INVALID
+    g = _Csr(0, 0, None, None)       # an empty graph is a valid no-op
+    assert lib.retexo_aggregate(C.byref(g), 0, None, C.c_int64(4), 4, None, None, C.c_int64(4), 1, None,
+                                C.c_int64(0), None, C.c_size_t(0), None) == 0
     g = _Csr(4, 0, 1, None)          # null feature pointer, no outputs
     assert lib.retexo_aggregate(C.byref(g), 0, None, C.c_int64(4), 4, None, None, C.c_int64(4), 1, None,
                                 C.c_int64(0), None, C.c_size_t(0), None) == INVALID

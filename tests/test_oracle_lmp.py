@@ -58,3 +58,13 @@ def test_more_rounds_help_when_features_are_weak_and_homophily_is_strong():
                                round_bf16=False)
         acc[K] = rep["test_acc"]
     assert acc[3] > acc[1] + 0.05, acc
+
+
+def test_forced_iterate_hook_keeps_the_named_iterate():
+    w = wl.make_config(1, scale=0.3)
+    free = run(w, 8)
+    same = run(w, 8, forced_best_iter=[r["best_iter"] for r in free["rounds"]])
+    np.testing.assert_array_equal(free["rounds"][-1]["logits"], same["rounds"][-1]["logits"])
+    other = run(w, 8, forced_best_iter=[8, 8, 8])
+    assert [r["best_iter"] for r in other["rounds"]] == [8, 8, 8]
+    assert other["rounds"][0]["test_correct_best"] == other["rounds"][0]["test_correct_last"]

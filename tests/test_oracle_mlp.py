@@ -199,3 +199,19 @@ def test_embed_hidden_logits_prediction_and_tie_rule():
     # exact ties -> lowest class index
     tie = oracle.Mlp(2, 0, 4, np.zeros((2, 4)), np.array([1.0, 3.0, 3.0, 3.0]), round_bf16=False)
     assert list(tie.embed(np.ones((3, 2), dtype=np.float32))["pred"]) == [1, 1, 1]
+
+
+def test_apply_update_alone_equals_the_update_inside_a_step():
+    rng = np.random.default_rng(13)
+    x = rng.standard_normal((20, 6)).astype(np.float32)
+    y = rng.integers(0, 3, 20).astype(np.int32)
+    for opt in (oracle.SGD, oracle.ADAM):
+        a = make(6, 4, 3, 14, optimizer=opt, lr=0.05, round_bf16=False)
+        b = a.copy()
+        for _ in range(3):
+            probe = a.copy()
+            _, g = probe.train_step(x, y, return_grad=True)
+            a.train_step(x, y)
+            b.apply_update(g)
+            np.testing.assert_array_equal(a.theta, b.theta)
+            assert a.step == b.step
