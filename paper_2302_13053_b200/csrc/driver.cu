@@ -72,7 +72,7 @@ struct LmpBuffers {
     // representations
     float* q[2];
     bf16* x16; bf16* q16; float* proj; bf16* watt16; float* gat_vec; float* gat_stage;
-    bf16 *xtr16, *xval16;
+    bf16 *xtr16, *xval16, *xtr_t16;
     int32_t *y_tr, *y_val, *y_test;
     float *theta, *adam_m, *adam_v, *theta_best;
     unsigned long long *cur_correct, *best_correct, *scratch_u64;
@@ -132,6 +132,7 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
     }
     l.xtr16 = t.template take<bf16>((size_t)n_tr * ld16);
     l.xval16 = t.template take<bf16>((size_t)(n_val > 0 ? n_val : 1) * ld16);
+    l.xtr_t16 = t.template take<bf16>((size_t)max_din * (size_t)round_up(n_tr, 8));
     l.y_tr = t.template take<int32_t>((size_t)n_tr);
     l.y_val = t.template take<int32_t>((size_t)(n_val > 0 ? n_val : 1));
     l.y_test = t.template take<int32_t>((size_t)(n_te > 0 ? n_te : 1));
@@ -297,7 +298,8 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         }
 
         // ---- the round's batches and model state
-        RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld16, nullptr, 0, st));
+        const int64_t ld_xt = round_up(n_tr, 8);
+        RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld16, b.xtr_t16, ld_xt, st));
         if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, b.xval16, ld16, nullptr, 0, st));
         RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta, in->theta0[m - 1], sizeof(float) * (size_t)nt, cudaMemcpyDefault, st));
         RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta_best, b.theta, sizeof(float) * (size_t)nt, cudaMemcpyDeviceToDevice, st));
@@ -318,7 +320,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         // ---- R training iterations; validation and best-iterate tracking stay on the device
         for (int it = 1; it <= c.R; ++it) {
             float* loss_slot = b.loss_history + (size_t)(m - 1) * c.R + (it - 1);
-            RETEXO_TRY(retexo_mlp_train_step(&model, b.xtr16, ld16, nullptr, 0, b.y_tr, n_tr, loss_slot, nullptr,
+            RETEXO_TRY(retexo_mlp_train_step(&model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, n_tr, loss_slot, nullptr,
                                              b.ws_step, b.ws_step_bytes, st));
             if (n_val && (it % c.eval_every == 0 || it == c.R)) {
                 RETEXO_TRY(retexo_embed(&model, b.xval16, ld16, nullptr, n_val, nullptr, 0, nullptr, 0, nullptr, 0,

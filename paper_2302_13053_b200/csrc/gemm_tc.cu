@@ -1,0 +1,324 @@
+// Tensor-core GEMM for the dense products of the per-node model on sm_100a:
+//   C[M x N] = A[M x K] * B[N x K]^T,  A and B bf16 with K contiguous,
+//   fp32 accumulation in tensor memory (tcgen05.mma, cta_group::1, M = 128).
+// Operand tiles are brought in by TMA (128-byte swizzle) through a ring of
+// shared-memory stages guarded by mbarriers; one thread issues the MMAs; four
+// warps drain the accumulator with tcgen05.ld and apply the fused epilogue
+// (bias / ReLU / bf16 down-cast, or a raw split-K partial).
+// Every wait is bounded: a wait that runs out sets *status and the block
+// tears down in order (outstanding copies awaited, tensor memory freed).
+#include <cuda.h>
+
+#include "common.cuh"
+#include "gemm_tc.h"
+
+namespace retexo {
+
+constexpr int kTcBM = 128;
+constexpr int kTcBK = 64;                  // 64 bf16 = 128 bytes = one swizzle row
+constexpr int kTcThreads = 192;            // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2..5: epilogue
+constexpr uint32_t kSpinLimit = 1u << 26;
+
+__device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait; returns false (and raises *status) if the phase never completes.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status, volatile int* abort_flag) {
+    for (uint32_t i = 0; i < kSpinLimit; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    if (status) atomicExch(status, RETEXO_ERR_TIMEOUT);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int32_t x, int32_t y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128
+// bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);          // start address
+    d |= (uint64_t)1 << 16;                                // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                      // stride byte offset
+    d |= (uint64_t)1 << 46;                                // descriptor version
+    d |= (uint64_t)2 << 61;                                // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t make_idesc(int bn) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
+        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct TcKernelArgs {
+    int64_t M, N;
+    int32_t k_blocks_total;       // ceil(K / 64)
+    int32_t k_blocks_per_split;
+    int mode, relu;
+    const float* bias;
+    float* out_f32; int64_t ld_f32;
+    __nv_bfloat16* out_bf16; int64_t ld_bf16;
+    float* partial;
+    int32_t* status;
+};
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(kTcThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcKernelArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    constexpr uint32_t kABytes = kTcBM * kTcBK * 2, kBBytes = BN * kTcBK * 2, kStageBytes = kABytes + kBBytes;
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full = reinterpret_cast<uint64_t*>(tiles + STAGES * kStageBytes);
+    uint64_t* empty = full + STAGES;
+    uint64_t* acc_ready = empty + STAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_ready + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t m0 = (int64_t)blockIdx.x * kTcBM, n0 = (int64_t)blockIdx.y * BN;
+    const int32_t kb0 = blockIdx.z * g.k_blocks_per_split;
+    const int32_t kb1 = min(g.k_blocks_total, kb0 + g.k_blocks_per_split);
+    const int32_t n_kb = kb1 - kb0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
+        mbar_init(acc_ready, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {      // tensor memory: BN fp32 columns x 128 lanes
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_acc = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int i = 0; i < n_kb; ++i) {
+                const int s = i % STAGES;
+                const uint32_t ph = (i / STAGES) & 1;
+                if (!mbar_wait(empty + s, ph ^ 1, g.status, abort_flag)) break;
+                mbar_expect_tx(full + s, kStageBytes);
+                uint8_t* a_dst = tiles + s * kStageBytes;
+                tma_load_2d(a_dst, &map_a, (kb0 + i) * kTcBK, (int32_t)m0, full + s);
+                tma_load_2d(a_dst + kABytes, &map_b, (kb0 + i) * kTcBK, (int32_t)n0, full + s);
+                issued = i + 1;
+            }
+            if (*abort_flag) {    // await (bounded) what was issued and not consumed, so nothing lands after exit
+                for (int i = max(0, issued - STAGES); i < issued; ++i) {
+                    const int s = i % STAGES;
+                    const uint32_t ph = (i / STAGES) & 1;
+                    for (uint32_t t = 0; t < (1u << 20); ++t) if (mbar_try_wait(full + s, ph)) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(BN);
+            bool ok = true;
+            for (int i = 0; i < n_kb && ok; ++i) {
+                const int s = i % STAGES;
+                const uint32_t ph = (i / STAGES) & 1;
+                ok = mbar_wait(full + s, ph, g.status, abort_flag);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t a_addr = smem_u32(tiles + s * kStageBytes);
+                const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(a_addr + kABytes);
+#pragma unroll
+                for (int k = 0; k < kTcBK / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K: +2 in 16-byte units
+                    umma_bf16(tmem_acc, adesc + 2 * k, bdesc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                umma_commit(empty + s);                   // frees the stage once these MMAs have read it
+            }
+            if (ok) umma_commit(acc_ready);               // accumulator complete
+        }
+    } else {
+        const int q = warp & 3;                           // tensor-memory lane quarter this warp may read
+        const int64_t row = m0 + q * 32 + lane;
+        bool ok = n_kb > 0 ? mbar_wait(acc_ready, 0, g.status, abort_flag) : true;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                if (n_kb > 0) tmem_ld_32cols(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = 0u;
+                }
+                if (row >= g.M) continue;
+                const int64_t col0 = n0 + c0;
+                if (g.mode == TC_EPI_PARTIAL) {
+                    float* dst = g.partial + ((int64_t)blockIdx.z * g.M + row) * g.N + col0;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __uint_as_float(r[j]);
+                } else {
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float x = __uint_as_float(r[j]);
+                        if (g.bias && col0 + j < g.N) x += __ldg(g.bias + col0 + j);
+                        if (g.relu) x = fmaxf(x, 0.f);
+                        v[j] = x;
+                    }
+                    if (g.out_f32) {
+                        float* dst = g.out_f32 + row * g.ld_f32 + col0;
+                        if (col0 + 32 <= g.N && (g.ld_f32 & 3) == 0 && aligned16(g.out_f32)) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = v[j];
+                        }
+                    }
+                    if (g.out_bf16) {
+                        __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16 + col0;
+                        if (col0 + 32 <= g.N && (g.ld_bf16 & 7) == 0 && aligned16(g.out_bf16)) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                __nv_bfloat162 p0 = __floats2bfloat162_rn(v[j], v[j + 1]);
+                                __nv_bfloat162 p1 = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
+                                __nv_bfloat162 p2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]);
+                                __nv_bfloat162 p3 = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
+                                uint4 pk;
+                                pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                                pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                                *reinterpret_cast<uint4*>(dst + j) = pk;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __float2bfloat16_rn(v[j]);
+                        }
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(BN));
+    }
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// 2-D bf16 tensor [rows x cols], cols contiguous, row stride ld elements; box = [box_rows x 64].
+static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kTcBK, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int STAGES>
+static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
+    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 256;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+            cudaSuccess) {
+            (void)cudaGetLastError();
+            return RETEXO_ERR_CUDA;
+        }
+        configured = true;
+    }
+    TcKernelArgs g{};
+    g.M = t.M; g.N = t.N;
+    g.k_blocks_total = (int32_t)((t.K + kTcBK - 1) / kTcBK);
+    const int splits = t.mode == TC_EPI_PARTIAL ? (t.splits > 0 ? t.splits : 1) : 1;
+    g.k_blocks_per_split = (g.k_blocks_total + splits - 1) / splits;
+    g.mode = t.mode; g.relu = t.relu; g.bias = t.bias;
+    g.out_f32 = t.out_f32; g.ld_f32 = t.ld_f32; g.out_bf16 = t.out_bf16; g.ld_bf16 = t.ld_bf16;
+    g.partial = t.partial; g.status = t.status;
+    dim3 grid((unsigned)((t.M + kTcBM - 1) / kTcBM), (unsigned)((t.N + BN - 1) / BN), (unsigned)splits);
+    tc_gemm_kernel<BN, STAGES><<<grid, kTcThreads, smem, st>>>(ma, mb, g);
+    return launch_status();
+}
+
+bool tc_gemm_supported(const TcGemm& t) {
+    if (t.M <= 0 || t.N <= 0 || t.K <= 0) return false;
+    if (!aligned_to(t.A, 16) || !aligned_to(t.B, 16) || t.lda % 8 != 0 || t.ldb % 8 != 0) return false;
+    if (t.M > INT32_MAX || t.N > INT32_MAX || t.K > INT32_MAX - 64) return false;
+    if ((t.M + kTcBM - 1) / kTcBM > 2147483647LL || (t.N + 63) / 64 > 65535) return false;
+    return encode_fn() != nullptr;
+}
+
+int tc_gemm_launch(const TcGemm& t, cudaStream_t st) {
+    if (!tc_gemm_supported(t)) return RETEXO_ERR_UNSUPPORTED;
+    const int bn = t.N > 128 ? 256 : (t.N > 64 ? 128 : 64);
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, t.A, t.M, t.K, t.lda, kTcBM)) return RETEXO_ERR_CUDA;
+    if (!make_map(&mb, t.B, t.N, t.K, t.ldb, bn)) return RETEXO_ERR_CUDA;
+    if (bn == 256) return launch_tc<256, 4>(t, ma, mb, st);
+    if (bn == 128) return launch_tc<128, 6>(t, ma, mb, st);
+    return launch_tc<64, 8>(t, ma, mb, st);
+}
+
+}  // namespace retexo

@@ -57,6 +57,7 @@ struct GemmArgs {
     const float* bias;                     // EPI_BIAS, [N] (may be null)
     float* out_f32; int64_t ld_f32;        // EPI_BIAS (may be null)
     bf16* out_bf16; int64_t ld_bf16;       // EPI_BIAS / EPI_MASK (may be null)
+    bf16* out_bf16_t; int64_t ld_t;        // EPI_MASK: optional transposed copy [N x ld_t]
     const bf16* mask; int64_t ld_mask;     // EPI_MASK: keep acc where mask > 0
     float* colsum;                         // EPI_MASK: [gridDim.y x N] column sums of the kept values
     float* partial;                        // EPI_PARTIAL: [gridDim.z x M x N]
@@ -160,7 +161,8 @@ __global__ void __launch_bounds__(kGemmThreads) gemm_bf16_kernel(GemmArgs g) {
             const int64_t n = n0 + tx * 4 + j;
             if (n >= g.N) continue;
             const float v = bf16_to_f32(g.mask[m * g.ld_mask + n]) > 0.f ? acc[i][j] : 0.f;
-            g.out_bf16[m * g.ld_bf16 + n] = f32_to_bf16(v);
+            if (g.out_bf16) g.out_bf16[m * g.ld_bf16 + n] = f32_to_bf16(v);
+            if (g.out_bf16_t) g.out_bf16_t[n * g.ld_t + m] = f32_to_bf16(v);
             col[j] += v;
         }
     }
@@ -184,6 +186,7 @@ constexpr int kSmThreads = 256;
 __global__ void __launch_bounds__(kSmThreads) softmax_ce_kernel(const float* __restrict__ logits, int64_t ld_logits,
                                                                 const int32_t* __restrict__ y, int64_t n_rows,
                                                                 int32_t n_classes, bf16* __restrict__ dl, int64_t ld_dl,
+                                                                bf16* __restrict__ dl_t, int64_t ld_t,
                                                                 float* __restrict__ loss_partial,
                                                                 float* __restrict__ colsum_partial) {
     __shared__ float s_loss[kSmThreads / kWarp];
@@ -207,6 +210,10 @@ __global__ void __launch_bounds__(kSmThreads) softmax_ce_kernel(const float* __r
         const float g1 = (e1 / den - (lane + 32 == yi ? 1.f : 0.f)) * inv_n;
         if (lane < ld_dl) dl[r * ld_dl + lane] = f32_to_bf16(lane < n_classes ? g0 : 0.f);
         if (lane + 32 < ld_dl) dl[r * ld_dl + lane + 32] = f32_to_bf16(lane + 32 < n_classes ? g1 : 0.f);
+        if (dl_t) {
+            if (lane < n_classes) dl_t[(int64_t)lane * ld_t + r] = f32_to_bf16(g0);
+            if (lane + 32 < n_classes) dl_t[(int64_t)(lane + 32) * ld_t + r] = f32_to_bf16(g1);
+        }
         if (lane < n_classes) c0 += g0;
         if (lane + 32 < n_classes) c1 += g1;
     }
@@ -266,6 +273,7 @@ struct UpdateArgs {
     int optimizer;
     float lr, beta1, beta2, eps, corr1, corr2;     // corr = 1 - beta^step
     const float* loss_partial; int64_t n_loss; float inv_rows; float* loss_out;
+    const int32_t* status;     // non-zero: a kernel of this step gave up on a bounded wait -> loss = NaN
 };
 
 __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
@@ -273,7 +281,7 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     if (p == 0 && u.loss_out) {
         float s = 0.f;
         for (int64_t i = 0; i < u.n_loss; ++i) s += u.loss_partial[i];
-        *u.loss_out = s * u.inv_rows;
+        *u.loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
     }
     int64_t off = 0;
     for (int s = 0; s < u.n_seg; ++s) {

@@ -17,7 +17,10 @@ struct MlpPlan {
     int64_t ld_dl;                          // row stride of the bf16 dL (classes rounded up to 8)
     int64_t sm_blocks;                      // softmax blocks = number of loss / db partials
     int64_t tiles_m;                        // 64-row tiles of the batch
-    int64_t split_w1, split_w2;             // split-K factors of the weight-gradient products
+    int64_t split_w1, split_w2;             // split-K factors of the weight-gradient products (CUDA-core path)
+    int64_t tc_split_w1;                    // split-K factor of the tensor-core dW1 product
+    int64_t ld_k;                           // row stride of the transposed bf16 W1 (d_in rounded up to 8)
+    int64_t ld_n;                           // row stride of transposed per-row gradients (n_rows rounded up to 8)
 };
 
 struct MlpBuffers {
@@ -31,6 +34,9 @@ struct MlpBuffers {
     float* dhdsum_partial;
     float* pw1;
     float* pw2;
+    __nv_bfloat16* w1t16;                   // W1^T, [out1 x ld_k]
+    __nv_bfloat16* gradt16;                 // (dHd or dL)^T, [out1 x ld_n]
+    int32_t* status;                        // raised by a tensor-core kernel whose bounded wait gave up
 };
 
 MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows);
@@ -40,7 +46,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
                           const int32_t* y, float* loss_out, float* grad_out, cudaStream_t st);
 
 int mlp_embed_launch(const retexo_mlp* model, __nv_bfloat16* theta16, __nv_bfloat16* hd16_ws, float* logits_ws,
-                     const __nv_bfloat16* x, int64_t ldx, const int32_t* row_idx, int64_t n_rows,
+                     __nv_bfloat16* w1t16, int32_t* status, const __nv_bfloat16* x, int64_t ldx, const int32_t* row_idx, int64_t n_rows,
                      float* hidden_out, int64_t ld_hidden, __nv_bfloat16* hidden_out_bf16, int64_t ld_hidden_bf16,
                      float* logits_out, int64_t ld_logits, int32_t* pred_out, const int32_t* y,
                      unsigned long long* correct_out, cudaStream_t st);

@@ -107,12 +107,14 @@ def test_embed_matches_checker_and_stated_tolerance(d_in, hidden, n_classes, n):
                            want_logits=True, want_pred=True)
     r = ref.embed(x, y=y, want_hidden=hidden > 0)
     lg = out["logits"].cpu().numpy()
-    assert_logits_close(lg, r["logits"], rel=2e-3, what="vs bf16-operand checker")
+    # 5e-3: one hidden unit whose fp32 and fp64 pre-activations straddle a bf16 rounding boundary
+    # differs by a bf16 ulp (2^-8 relative) and moves a logit by up to |w2| x that
+    assert_logits_close(lg, r["logits"], rel=5e-3, what="vs bf16-operand checker")
     exact = oracle.Mlp(d_in, hidden, n_classes, **{k: v for k, v in ref.unpack().items()}, round_bf16=False)
     assert_logits_close(lg, exact.embed(x)["logits"], rel=2e-2, what="vs unrounded checker")
     if hidden > 0:
         h = out["hidden"].cpu().numpy()
-        assert_logits_close(h, r["hidden"], rel=2e-3, what="hidden")
+        assert_logits_close(h, r["hidden"], rel=1e-3, what="hidden")
         assert torch.equal(out["hidden_bf16"][:, :hidden].cpu(), out["hidden"].to(torch.bfloat16).cpu())
     # predictions: exact wherever the reference margin is clear of the tolerance
     srt = np.sort(r["logits"], axis=1)
@@ -124,7 +126,9 @@ def test_embed_matches_checker_and_stated_tolerance(d_in, hidden, n_classes, n):
     # row gather
     idx = rng.integers(0, n, 77).astype(np.int32)
     sub = B().retexo_embed(gpu, x16, row_idx=dev(idx), want_logits=True)
-    np.testing.assert_array_equal(sub["logits"].cpu().numpy(), lg[idx])
+    # (gathered rows take the CUDA-core product, dense ones the tensor cores: same values up to
+    # summation order and the bf16 rounding of the hidden layer that follows it)
+    assert_logits_close(sub["logits"].cpu().numpy(), lg[idx], rel=5e-3, what="row gather")
 
 
 def test_argmax_tie_rule_lowest_index():
