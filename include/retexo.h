@@ -226,6 +226,35 @@ int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* part, int32
                                  uint64_t* send_per_part, uint64_t* recv_per_part,
                                  void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same count for callers that cannot allocate device memory at all: code
+ * running inside a framework that owns the allocator, a plug-in loaded into a
+ * process whose memory budget is fixed up front, a latency-critical loop where
+ * cudaMalloc's implicit synchronisation is not acceptable.  (The paper has no
+ * counterpart of this call; it is a convenience of this library.)
+ * It needs no workspace argument: its scratch is a fixed 4 MiB array inside
+ * the library image (retexo_cross_partition_static_scratch_bytes), which every
+ * GPU that loads the library holds until the process exits.  The call itself
+ * calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - Limit: a problem whose scratch need
+ *     (retexo_cross_partition_workspace_size) exceeds that array is rejected
+ *     with RETEXO_ERR_UNSUPPORTED and nothing is launched.  Up to 8192
+ *     partitions the need is about 1 KiB whatever the graph's size; beyond
+ *     that it grows as 4 n_nodes + 8 n_parts bytes (+ 1 KiB).
+ *   - The first call on a device looks the array's device address up
+ *     (one-time set-up, per device, with that device current); make that first
+ *     call before any stream capture.
+ *   - All calls on a device share the one array: two calls whose kernels may
+ *     overlap on the GPU (different streams, no ordering) race and give wrong
+ *     counts.  Calls ordered on one stream are fine; each call clears the
+ *     counters it uses.
+ * Arguments, outputs and errors otherwise as retexo_cross_partition_bytes. */
+size_t retexo_cross_partition_static_scratch_bytes(void);
+int retexo_cross_partition_bytes_static(const retexo_csr* g, const int32_t* part, int32_t n_parts,
+                                        int32_t K, const int32_t* dims, int32_t elem_bytes,
+                                        uint64_t* cross_edges, uint64_t* boundary_pairs,
+                                        uint64_t* bytes_per_round, uint64_t* bytes_total,
+                                        uint64_t* send_per_part, uint64_t* recv_per_part, void* stream);
+
 /* -------------------------------------------------- the K-round LMP loop */
 typedef struct retexo_lmp_config {
     int32_t aggr;                   /* retexo_aggr */

@@ -67,7 +67,9 @@ class _LmpOutputs(C.Structure):
 EXPORTS = ["retexo_status_string", "retexo_version", "retexo_validate_csr", "retexo_aggregate_workspace_size",
            "retexo_aggregate", "retexo_theta_size", "retexo_pack_rows", "retexo_mlp_train_step_workspace_size",
            "retexo_mlp_train_step", "retexo_embed_workspace_size", "retexo_embed",
-           "retexo_cross_partition_workspace_size", "retexo_cross_partition_bytes", "retexo_lmp_workspace_size",
+           "retexo_cross_partition_workspace_size", "retexo_cross_partition_bytes",
+           "retexo_cross_partition_static_scratch_bytes", "retexo_cross_partition_bytes_static",
+           "retexo_lmp_workspace_size",
            "retexo_lmp_train"]
 
 
@@ -83,7 +85,7 @@ def lib():
         L.retexo_status_string.argtypes = [C.c_int]
         for name in ("retexo_aggregate_workspace_size", "retexo_mlp_train_step_workspace_size",
                      "retexo_embed_workspace_size", "retexo_cross_partition_workspace_size",
-                     "retexo_lmp_workspace_size"):
+                     "retexo_lmp_workspace_size", "retexo_cross_partition_static_scratch_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.retexo_theta_size.restype = C.c_int64
         _lib = L
@@ -296,6 +298,24 @@ def retexo_cross_partition_bytes(rowptr: torch.Tensor, colidx: torch.Tensor, par
                 bytes_per_round=s[3:3 + K].copy(), dv_lazy_lt=2 * int(s[2]),
                 send_per_part=None if send is None else send.cpu().numpy().view(np.uint64),
                 recv_per_part=None if recv is None else recv.cpu().numpy().view(np.uint64))
+
+
+def retexo_cross_partition_bytes_static(rowptr: torch.Tensor, colidx: torch.Tensor, part: torch.Tensor, n_parts: int,
+                                        dims: Sequence[int], out: torch.Tensor, elem_bytes: int = 4) -> None:
+    """The count through the entry point that allocates nothing.  This wrapper allocates nothing
+    either: `out` is a caller-provided int64 device tensor of 3 + len(dims) elements that receives
+    cross_edges, boundary_pairs, bytes_total and then the bytes of each round (read them as
+    uint64 after synchronising)."""
+    assert part.dtype == torch.int32 and out.dtype == torch.int64 and out.numel() >= 3 + len(dims)
+    K = len(dims)
+    g = _csr(rowptr, colidx)
+    dims_a = (C.c_int32 * max(K, 1))(*[int(d) for d in dims])
+    base = out.data_ptr()
+    rc = lib().retexo_cross_partition_bytes_static(C.byref(g), _ptr(part), C.c_int32(n_parts), C.c_int32(K), dims_a,
+                                                   C.c_int32(elem_bytes), C.c_void_p(base), C.c_void_p(base + 8),
+                                                   C.c_void_p(base + 24), C.c_void_p(base + 16), None, None,
+                                                   _stream())
+    _check(rc, "retexo_cross_partition_bytes_static")
 
 
 def pack_theta(w: Dict[str, np.ndarray]) -> np.ndarray:

@@ -2,6 +2,8 @@
 // message-passing round sends across a node partition (Section 2.1,
 // Appendix A.1), plus the CSR validator.  Integer work only; all tallies use
 // integer atomics, whose result does not depend on the order they land in.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace retexo {
@@ -370,4 +372,54 @@ extern "C" int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* 
     count_finalize_kernel<<<1, 32, 0, st>>>(acc, acc + 1, acc + 2, K, dims_dev, elem_bytes, cross_edges, boundary_pairs,
                                             bytes_per_round, bytes_total);
     return launch_status();
+}
+
+// ---------------------------------------------------------------- no-allocation variant
+namespace retexo {
+
+// Scratch of the allocation-free entry point.  It lives in the library image, so
+// every GPU that loads the library holds these 4 MiB until the process exits.
+constexpr size_t kStaticScratchBytes = size_t(4) << 20;
+static __device__ __align__(256) unsigned char g_static_count_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+static std::mutex g_static_scratch_mutex;
+static void* g_static_scratch_addr[kMaxDevices] = {};
+
+// In host code the array's name is only a handle for the runtime, not a device
+// address: the address is looked up once per device, with that device current.
+static int static_scratch_address(void** out) {
+    int dev = 0;
+    RETEXO_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return RETEXO_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_addr[dev]) {
+        void* ptr = nullptr;
+        RETEXO_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_static_count_scratch));
+        g_static_scratch_addr[dev] = ptr;
+    }
+    *out = g_static_scratch_addr[dev];
+    return RETEXO_OK;
+}
+
+}  // namespace retexo
+
+extern "C" size_t retexo_cross_partition_static_scratch_bytes(void) { return kStaticScratchBytes; }
+
+extern "C" int retexo_cross_partition_bytes_static(const retexo_csr* g, const int32_t* part, int32_t n_parts,
+                                                   int32_t K, const int32_t* dims, int32_t elem_bytes,
+                                                   uint64_t* cross_edges, uint64_t* boundary_pairs,
+                                                   uint64_t* bytes_per_round, uint64_t* bytes_total,
+                                                   uint64_t* send_per_part, uint64_t* recv_per_part, void* stream) {
+    if (!g || g->n_nodes < 0 || g->n_edges < 0 || n_parts <= 0) return RETEXO_ERR_INVALID_ARG;
+    const size_t need = retexo_cross_partition_workspace_size(g->n_nodes, g->n_edges, n_parts);
+    if (need == 0) return RETEXO_ERR_INVALID_ARG;
+    if (need > kStaticScratchBytes) return RETEXO_ERR_UNSUPPORTED;     // beyond the built-in scratch
+    void* scratch = nullptr;
+    RETEXO_TRY(static_scratch_address(&scratch));
+    // The counters and lists inside the scratch are cleared by the call below before use, so
+    // what an earlier call left there does not matter.
+    return retexo_cross_partition_bytes(g, part, n_parts, K, dims, elem_bytes, cross_edges, boundary_pairs,
+                                        bytes_per_round, bytes_total, send_per_part, recv_per_part, scratch,
+                                        kStaticScratchBytes, stream);
 }
