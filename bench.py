@@ -183,7 +183,7 @@ def phase_breakdown(w, ws, R: int, peaks):
                            edges_per_s=e / mean_ms * 1e3))
         # the round's model at its training / validation / full shapes
         model = B.Mlp(rd["d_in"], rd["hidden"], w.n_classes, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
-        xtr, xtr_t = B.retexo_pack_rows(x16, tr, dim=width, transpose=True)
+        xtr, xtr_t = B.retexo_pack_rows(x16, tr, dim=width, transpose=True, ones_row=True)
         xva, _ = B.retexo_pack_rows(x16, va, dim=width)
         H, O = rd["hidden"], w.n_classes
         n_tr, n_va = tr.numel(), va.numel()

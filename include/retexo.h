@@ -132,7 +132,10 @@ typedef enum retexo_optimizer { RETEXO_SGD = 0, RETEXO_ADAM = 1 } retexo_optimiz
  * adam_m / adam_v have the same length (NULL for SGD).  `step` counts the
  * updates already applied; retexo_mlp_train_step increments it.
  * Every matrix product takes both operands rounded to bf16 and accumulates in
- * fp32; biases, softmax, loss and the optimiser are fp32. */
+ * fp32 on the tensor cores (a bias gradient is the product of the all-ones
+ * vector with the layer's output gradient and follows the same rule); biases,
+ * softmax, loss and the optimiser are fp32.  A device-side wait that runs out
+ * (it never should) makes the reported loss NaN. */
 typedef struct retexo_mlp {
     int32_t d_in, hidden, n_classes;
     float* theta;
@@ -149,10 +152,13 @@ int64_t retexo_theta_size(int32_t d_in, int32_t hidden, int32_t n_classes);
  * src is fp32 (src_is_bf16 = 0) or bf16 (1), row stride ld_src elements;
  * dst is bf16 [n_rows x ld_dst], ld_dst >= dim; columns [dim, ld_dst) are
  * zero-filled.  dst_t (optional) receives the transpose, bf16 [dim x ld_t],
- * ld_t >= n_rows, columns [n_rows, ld_t) zero-filled.  Needs no workspace. */
+ * ld_t >= n_rows, columns [n_rows, ld_t) zero-filled; with ones_row = 1 it has
+ * one more row (index dim) that holds 1 for every batch row: the form
+ * retexo_mlp_train_step takes as x_t.  dst may be NULL if only the transpose
+ * is wanted.  Needs no workspace. */
 int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld_src, int32_t dim,
                      const int32_t* idx, int64_t n_rows,
-                     void* dst, int64_t ld_dst, void* dst_t, int64_t ld_t, void* stream);
+                     void* dst, int64_t ld_dst, void* dst_t, int64_t ld_t, int32_t ones_row, void* stream);
 
 size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes,
                                             int64_t n_rows);
@@ -166,9 +172,12 @@ size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_
  * x     bf16 [n_rows x ldx]: the batch, one training node per row
  *       (retexo_pack_rows builds it once per round); ldx % 8 == 0 and x
  *       16-byte aligned.
- * x_t   optional bf16 [d_in x ld_xt] transpose of x (ld_xt % 8 == 0), lets the
- *       weight-gradient product stream both operands along the batch; NULL
- *       is allowed.
+ * x_t   optional bf16 [(d_in + 1) x ld_xt]: the transpose of x with one more
+ *       row of ones (retexo_pack_rows with ones_row = 1; ld_xt % 8 == 0,
+ *       16-byte aligned).  The weight-gradient product streams it along the
+ *       batch; the row of ones makes the bias gradient one more output row.
+ *       NULL is allowed: the call then builds it in the workspace, at the
+ *       price of one more pass over x per call.
  * y     int32 [n_rows] labels in [0, n_classes).
  * loss_out  device float, the loss before the update (may be NULL).
  * grad_out  optional device fp32 array shaped like theta: the gradient.

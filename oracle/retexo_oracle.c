@@ -210,7 +210,9 @@ int oracle_aggregate_gat(int64_t n, const int64_t *rowptr, const int32_t *colidx
 /* matrices row-major [in x out].                                       */
 /* round_bf16 != 0: both operands of every matrix product are rounded  */
 /* to bf16 first ("bf16 inputs, wider accumulate"); sums, biases,      */
-/* softmax and the optimiser stay in double.                           */
+/* softmax and the optimiser stay in double.  A bias gradient is the   */
+/* product of the all-ones vector with the layer's output gradient, so */
+/* it sums the rounded gradient like any other product.                */
 /* ================================================================== */
 
 int64_t oracle_theta_size(int32_t d_in, int32_t hidden, int32_t n_classes)
@@ -391,16 +393,16 @@ int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
             int64_t r = row_idx ? row_idx[i] : i;
             const float *xrow = x + r * ldx;
             const double *d1row = d1 + i * out1;
-            /* dW1 = X^T d1,  db1 = sum d1 */
+            /* dW1 = X^T d1,  db1 = 1^T d1 */
             for (int32_t k = 0; k < d_in; ++k) {
                 double xv = opnd((double)xrow[k], round_bf16);
                 if (xv == 0.0) continue;
                 double *grow = gw1 + (int64_t)k * out1;
                 for (int32_t j = 0; j < out1; ++j) grow[j] += xv * opnd(d1row[j], round_bf16);
             }
-            for (int32_t j = 0; j < out1; ++j) gb1[j] += d1row[j];
+            for (int32_t j = 0; j < out1; ++j) gb1[j] += opnd(d1row[j], round_bf16);
             if (hidden > 0) {
-                /* dW2 = Hd^T dL,  db2 = sum dL */
+                /* dW2 = Hd^T dL,  db2 = 1^T dL */
                 const double *dlrow = dl + i * n_classes;
                 for (int32_t j = 0; j < hidden; ++j) {
                     double h = opnd(hd[i * hidden + j], round_bf16);
@@ -408,7 +410,7 @@ int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
                     double *grow = gw2 + (int64_t)j * n_classes;
                     for (int32_t c = 0; c < n_classes; ++c) grow[c] += h * opnd(dlrow[c], round_bf16);
                 }
-                for (int32_t c = 0; c < n_classes; ++c) gb2[c] += dlrow[c];
+                for (int32_t c = 0; c < n_classes; ++c) gb2[c] += opnd(dlrow[c], round_bf16);
             }
         }
     }

@@ -170,9 +170,9 @@ def retexo_aggregate(aggr: int, rowptr: torch.Tensor, colidx: torch.Tensor, q: t
 
 
 def retexo_pack_rows(src: torch.Tensor, idx: Optional[torch.Tensor] = None, dim: Optional[int] = None,
-                     transpose: bool = False):
+                     transpose: bool = False, ones_row: bool = False):
     """bf16 batch of the rows src[idx] (all rows if idx is None).  Returns
-    (dst [n_rows, round_up(dim, 8)], dst_t [dim, round_up(n_rows, 8)] or None)."""
+    (dst [n_rows, round_up(dim, 8)], dst_t [dim (+1 with ones_row), round_up(n_rows, 8)] or None)."""
     assert src.dtype in (torch.float32, torch.bfloat16) and src.stride(1) == 1
     dim = int(src.shape[1] if dim is None else dim)
     n_rows = int(src.shape[0] if idx is None else idx.numel())
@@ -183,12 +183,13 @@ def retexo_pack_rows(src: torch.Tensor, idx: Optional[torch.Tensor] = None, dim:
     ld_t = 0
     if transpose:
         ld_t = (n_rows + 7) // 8 * 8
-        dst_t = torch.empty((dim, ld_t), dtype=torch.bfloat16, device=dev)
+        dst_t = torch.empty((dim + (1 if ones_row else 0), ld_t), dtype=torch.bfloat16, device=dev)
     if idx is not None:
         assert idx.dtype == torch.int32
     rc = lib().retexo_pack_rows(_ptr(src), C.c_int32(1 if src.dtype == torch.bfloat16 else 0),
                                 C.c_int64(src.stride(0)), C.c_int32(dim), _ptr(idx), C.c_int64(n_rows),
-                                _ptr(dst), C.c_int64(ld), _ptr(dst_t), C.c_int64(ld_t), _stream())
+                                _ptr(dst), C.c_int64(ld), _ptr(dst_t), C.c_int64(ld_t),
+                                C.c_int32(1 if (ones_row and transpose) else 0), _stream())
     _check(rc, "retexo_pack_rows")
     return dst, dst_t
 

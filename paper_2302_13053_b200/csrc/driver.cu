@@ -132,7 +132,7 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
     }
     l.xtr16 = t.template take<bf16>((size_t)n_tr * ld16);
     l.xval16 = t.template take<bf16>((size_t)(n_val > 0 ? n_val : 1) * ld16);
-    l.xtr_t16 = t.template take<bf16>((size_t)max_din * (size_t)round_up(n_tr, 8));
+    l.xtr_t16 = t.template take<bf16>((size_t)(max_din + 1) * (size_t)round_up(n_tr, 8));
     l.y_tr = t.template take<int32_t>((size_t)n_tr);
     l.y_val = t.template take<int32_t>((size_t)(n_val > 0 ? n_val : 1));
     l.y_test = t.template take<int32_t>((size_t)(n_te > 0 ? n_te : 1));
@@ -284,7 +284,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
             RETEXO_TRY(convert_f32_to_bf16_launch(b.gat_stage, b.watt16, (int64_t)r.rep_dim * hd, st));
             RETEXO_CUDA_TRY(cudaMemcpyAsync(b.gat_vec, b.gat_stage + (size_t)r.rep_dim * hd, sizeof(float) * 2 * hd,
                                             cudaMemcpyDeviceToDevice, st));
-            RETEXO_TRY(retexo_pack_rows(q, 0, ldq, r.rep_dim, nullptr, n, b.q16, ldq16, nullptr, 0, st));
+            RETEXO_TRY(retexo_pack_rows(q, 0, ldq, r.rep_dim, nullptr, n, b.q16, ldq16, nullptr, 0, 0, st));
             // P = Q W_att: the projection as a bias-free single linear layer
             RETEXO_TRY(project_rows_launch(b.q16, ldq16, b.watt16, hd, n, hd, r.rep_dim, b.proj, ldp, st));
             retexo_gat_params gp;
@@ -299,8 +299,8 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
 
         // ---- the round's batches and model state
         const int64_t ld_xt = round_up(n_tr, 8);
-        RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld16, b.xtr_t16, ld_xt, st));
-        if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, b.xval16, ld16, nullptr, 0, st));
+        RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld16, b.xtr_t16, ld_xt, 1, st));
+        if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, b.xval16, ld16, nullptr, 0, 0, st));
         RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta, in->theta0[m - 1], sizeof(float) * (size_t)nt, cudaMemcpyDefault, st));
         RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta_best, b.theta, sizeof(float) * (size_t)nt, cudaMemcpyDeviceToDevice, st));
         RETEXO_CUDA_TRY(cudaMemsetAsync(b.adam_m, 0, sizeof(float) * (size_t)nt, st));

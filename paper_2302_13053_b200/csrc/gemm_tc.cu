@@ -99,6 +99,8 @@ struct TcKernelArgs {
     const float* bias;
     float* out_f32; int64_t ld_f32;
     __nv_bfloat16* out_bf16; int64_t ld_bf16;
+    __nv_bfloat16* out_bf16_t; int64_t ld_t; int ones_row_t;
+    const __nv_bfloat16* mask; int64_t ld_mask;
     float* partial;
     int32_t* status;
 };
@@ -196,6 +198,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     float* dst = g.partial + ((int64_t)blockIdx.z * g.M + row) * g.N + col0;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __uint_as_float(r[j]);
+                } else if (g.mode == TC_EPI_MASK_T) {
+                    const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (col0 + j >= g.N) continue;
+                        const float keep = __bfloat162float(mrow[j]) > 0.f ? __uint_as_float(r[j]) : 0.f;
+                        g.out_bf16_t[(col0 + j) * g.ld_t + row] = __float2bfloat16_rn(keep);
+                    }
                 } else {
                     float v[32];
 #pragma unroll
@@ -215,6 +225,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                             for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = v[j];
                         }
+                    }
+                    if (g.out_bf16_t) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < g.N) g.out_bf16_t[(col0 + j) * g.ld_t + row] = __float2bfloat16_rn(v[j]);
+                        if (g.ones_row_t && col0 == 0) g.out_bf16_t[g.N * g.ld_t + row] = __float2bfloat16_rn(1.0f);
                     }
                     if (g.out_bf16) {
                         __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16 + col0;
@@ -296,6 +312,8 @@ static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& 
     g.k_blocks_per_split = (g.k_blocks_total + splits - 1) / splits;
     g.mode = t.mode; g.relu = t.relu; g.bias = t.bias;
     g.out_f32 = t.out_f32; g.ld_f32 = t.ld_f32; g.out_bf16 = t.out_bf16; g.ld_bf16 = t.ld_bf16;
+    g.out_bf16_t = t.out_bf16_t; g.ld_t = t.ld_t; g.ones_row_t = t.ones_row_t;
+    g.mask = t.mask; g.ld_mask = t.ld_mask;
     g.partial = t.partial; g.status = t.status;
     dim3 grid((unsigned)((t.M + kTcBM - 1) / kTcBM), (unsigned)((t.N + BN - 1) / BN), (unsigned)splits);
     tc_gemm_kernel<BN, STAGES><<<grid, kTcThreads, smem, st>>>(ma, mb, g);
@@ -304,6 +322,8 @@ static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& 
 
 bool tc_gemm_supported(const TcGemm& t) {
     if (t.M <= 0 || t.N <= 0 || t.K <= 0) return false;
+    if (t.mode == TC_EPI_MASK_T && (!t.mask || !t.out_bf16_t)) return false;
+    if (t.mode == TC_EPI_PARTIAL && !t.partial) return false;
     if (!aligned_to(t.A, 16) || !aligned_to(t.B, 16) || t.lda % 8 != 0 || t.ldb % 8 != 0) return false;
     if (t.M > INT32_MAX || t.N > INT32_MAX || t.K > INT32_MAX - 64) return false;
     if ((t.M + kTcBM - 1) / kTcBM > 2147483647LL || (t.N + 63) / 64 > 65535) return false;

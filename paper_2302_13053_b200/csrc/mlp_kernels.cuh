@@ -12,12 +12,14 @@ typedef __nv_bfloat16 bf16;
 
 // ---------------------------------------------------------------- packing
 // dst[i][c] = bf16(src[idx ? idx[i] : i][c]); dst_t[c][i] likewise.  Padding
-// columns of both outputs are written as zero.
+// columns of both outputs are written as zero.  With ones_row, dst_t gets one
+// more row (index dim) holding 1 for every batch row: the all-ones row that
+// makes the bias gradient one more output row of the weight-gradient product.
 template <bool SRC_BF16>
 __global__ void __launch_bounds__(256) pack_rows_kernel(const void* __restrict__ src, int64_t ld_src, int32_t dim,
                                                         const int32_t* __restrict__ idx, int64_t n_rows,
                                                         bf16* __restrict__ dst, int64_t ld_dst,
-                                                        bf16* __restrict__ dst_t, int64_t ld_t) {
+                                                        bf16* __restrict__ dst_t, int64_t ld_t, int ones_row) {
     __shared__ float tile[32][33];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;     // 32 x 8
     const int64_t r0 = blockIdx.x * 32ll;
@@ -39,70 +41,60 @@ __global__ void __launch_bounds__(256) pack_rows_kernel(const void* __restrict__
         const int64_t c = c0 + i, r = r0 + tx;
         if (c < dim && r < ld_t) dst_t[c * ld_t + r] = f32_to_bf16(tile[tx][i]);
     }
+    if (ones_row && blockIdx.y == 0 && ty == 0) {
+        const int64_t r = r0 + tx;
+        if (r < ld_t) dst_t[(int64_t)dim * ld_t + r] = f32_to_bf16(r < n_rows ? 1.0f : 0.0f);
+    }
 }
 
 // ---------------------------------------------------------------- GEMM
 constexpr int kBM = 64, kBN = 64, kBK = 32, kGemmThreads = 256;
 
-enum EpiMode { EPI_PARTIAL = 0, EPI_BIAS = 1, EPI_MASK = 2 };
-
 struct GemmArgs {
     int64_t M, N, K;
-    const bf16* A; int64_t lda;            // A_T = false: [M x K]; true: stored [K x M]
-    const int32_t* a_row_idx;              // optional row gather for A (A_T = false only)
-    const bf16* B; int64_t ldb;            // B_T = false: [K x N]; true: stored [N x K]
-    int64_t k_chunk;                       // K range per blockIdx.z (multiple of kBK)
-    int mode;
-    int relu;                              // EPI_BIAS
-    const float* bias;                     // EPI_BIAS, [N] (may be null)
-    float* out_f32; int64_t ld_f32;        // EPI_BIAS (may be null)
-    bf16* out_bf16; int64_t ld_bf16;       // EPI_BIAS / EPI_MASK (may be null)
-    bf16* out_bf16_t; int64_t ld_t;        // EPI_MASK: optional transposed copy [N x ld_t]
-    const bf16* mask; int64_t ld_mask;     // EPI_MASK: keep acc where mask > 0
-    float* colsum;                         // EPI_MASK: [gridDim.y x N] column sums of the kept values
-    float* partial;                        // EPI_PARTIAL: [gridDim.z x M x N]
+    const bf16* A; int64_t lda;            // [M x K], row-major
+    const int32_t* a_row_idx;              // optional row gather for A
+    const bf16* B; int64_t ldb;            // [K x N], row-major
+    int relu;
+    const float* bias;                     // [N] (may be null)
+    float* out_f32; int64_t ld_f32;        // (may be null)
+    bf16* out_bf16; int64_t ld_bf16;       // (may be null)
 };
 
-template <bool A_T, bool B_T>
+// out = A B (+ bias) (ReLU), bf16 operands, fp32 accumulation on the CUDA cores.
+// Takes what the tensor-core kernel cannot: gathered rows and operands that
+// break the TMA alignment rules.
 __global__ void __launch_bounds__(kGemmThreads) gemm_bf16_kernel(GemmArgs g) {
     __shared__ __align__(16) float As[kBK][kBM + 4];
     __shared__ __align__(16) float Bs[kBK][kBN + 4];
-    __shared__ float cs[16][kBN];
     const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
     const int64_t m0 = blockIdx.y * (int64_t)kBM, n0 = blockIdx.x * (int64_t)kBN;
-    const int64_t kbeg = blockIdx.z * g.k_chunk;
-    const int64_t kend = min(g.K, kbeg + g.k_chunk);
     float acc[4][4];
 #pragma unroll
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
-    for (int64_t k0 = kbeg; k0 < kend; k0 += kBK) {
+    for (int64_t k0 = 0; k0 < g.K; k0 += kBK) {
 #pragma unroll
         for (int i = 0; i < (kBM * kBK) / kGemmThreads; ++i) {
             const int e = t + i * kGemmThreads;
-            int m, k;
-            if (A_T) { k = e / kBM; m = e % kBM; } else { m = e / kBK; k = e % kBK; }
+            const int m = e / kBK, k = e % kBK;
             const int64_t gm = m0 + m, gk = k0 + k;
             float v = 0.f;
-            if (gm < g.M && gk < kend) {
-                if (A_T) v = bf16_to_f32(g.A[gk * g.lda + gm]);
-                else {
-                    const int64_t r = g.a_row_idx ? g.a_row_idx[gm] : gm;
-                    v = bf16_to_f32(g.A[r * g.lda + gk]);
-                }
+            if (gm < g.M && gk < g.K) {
+                const int64_t r = g.a_row_idx ? g.a_row_idx[gm] : gm;
+                v = bf16_to_f32(g.A[r * g.lda + gk]);
             }
             As[k][m] = v;
         }
 #pragma unroll
         for (int i = 0; i < (kBN * kBK) / kGemmThreads; ++i) {
             const int e = t + i * kGemmThreads;
-            int n, k;
-            if (B_T) { n = e / kBK; k = e % kBK; } else { k = e / kBN; n = e % kBN; }
+            const int k = e / kBN, n = e % kBN;
             const int64_t gn = n0 + n, gk = k0 + k;
             float v = 0.f;
-            if (gn < g.N && gk < kend) v = bf16_to_f32(B_T ? g.B[gn * g.ldb + gk] : g.B[gk * g.ldb + gn]);
+            if (gn < g.N && gk < g.K) v = bf16_to_f32(g.B[gk * g.ldb + gn]);
             Bs[k][n] = v;
         }
         __syncthreads();
@@ -118,40 +110,6 @@ __global__ void __launch_bounds__(kGemmThreads) gemm_bf16_kernel(GemmArgs g) {
         }
         __syncthreads();
     }
-
-    if (g.mode == EPI_PARTIAL) {
-        float* p = g.partial + (int64_t)blockIdx.z * g.M * g.N;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int64_t m = m0 + ty * 4 + i;
-            if (m >= g.M) continue;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int64_t n = n0 + tx * 4 + j;
-                if (n < g.N) p[m * g.N + n] = acc[i][j];
-            }
-        }
-        return;
-    }
-    if (g.mode == EPI_BIAS) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int64_t m = m0 + ty * 4 + i;
-            if (m >= g.M) continue;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const int64_t n = n0 + tx * 4 + j;
-                if (n >= g.N) continue;
-                float v = acc[i][j] + (g.bias ? g.bias[n] : 0.f);
-                if (g.relu) v = fmaxf(v, 0.f);
-                if (g.out_f32) g.out_f32[m * g.ld_f32 + n] = v;
-                if (g.out_bf16) g.out_bf16[m * g.ld_bf16 + n] = f32_to_bf16(v);
-            }
-        }
-        return;
-    }
-    // EPI_MASK
-    float col[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int64_t m = m0 + ty * 4 + i;
@@ -160,40 +118,28 @@ __global__ void __launch_bounds__(kGemmThreads) gemm_bf16_kernel(GemmArgs g) {
         for (int j = 0; j < 4; ++j) {
             const int64_t n = n0 + tx * 4 + j;
             if (n >= g.N) continue;
-            const float v = bf16_to_f32(g.mask[m * g.ld_mask + n]) > 0.f ? acc[i][j] : 0.f;
+            float v = acc[i][j] + (g.bias ? g.bias[n] : 0.f);
+            if (g.relu) v = fmaxf(v, 0.f);
+            if (g.out_f32) g.out_f32[m * g.ld_f32 + n] = v;
             if (g.out_bf16) g.out_bf16[m * g.ld_bf16 + n] = f32_to_bf16(v);
-            if (g.out_bf16_t) g.out_bf16_t[n * g.ld_t + m] = f32_to_bf16(v);
-            col[j] += v;
-        }
-    }
-    if (g.colsum) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) cs[ty][tx * 4 + j] = col[j];
-        __syncthreads();
-        if (t < kBN && n0 + t < g.N) {
-            float s = 0.f;
-            for (int r = 0; r < 16; ++r) s += cs[r][t];
-            g.colsum[(int64_t)blockIdx.y * g.N + n0 + t] = s;
         }
     }
 }
 
 // ---------------------------------------------------------------- softmax CE
 // One warp per row (n_classes <= 64).  Writes dL = (softmax - onehot)/n_rows as
-// bf16 (row stride ld_dl, padding columns zero), and per-block partial sums of
-// the loss and of the columns of the unrounded dL.
+// bf16, row-major (row stride ld_dl, padding columns zero) and transposed
+// (dl_t [n_classes x ld_t]), and per-block partial sums of the loss.
 constexpr int kSmThreads = 256;
 __global__ void __launch_bounds__(kSmThreads) softmax_ce_kernel(const float* __restrict__ logits, int64_t ld_logits,
                                                                 const int32_t* __restrict__ y, int64_t n_rows,
                                                                 int32_t n_classes, bf16* __restrict__ dl, int64_t ld_dl,
                                                                 bf16* __restrict__ dl_t, int64_t ld_t,
-                                                                float* __restrict__ loss_partial,
-                                                                float* __restrict__ colsum_partial) {
+                                                                float* __restrict__ loss_partial) {
     __shared__ float s_loss[kSmThreads / kWarp];
-    __shared__ float s_col[kSmThreads / kWarp][64];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const float inv_n = 1.0f / (float)n_rows;
-    float my_loss = 0.f, c0 = 0.f, c1 = 0.f;
+    float my_loss = 0.f;
     const int64_t stride = (int64_t)gridDim.x * (kSmThreads / kWarp);
     for (int64_t r = blockIdx.x * (int64_t)(kSmThreads / kWarp) + warp; r < n_rows; r += stride) {
         const float* row = logits + r * ld_logits;
@@ -208,24 +154,17 @@ __global__ void __launch_bounds__(kSmThreads) softmax_ce_kernel(const float* __r
         my_loss += (mx + logf(den)) - ly;
         const float g0 = (e0 / den - (lane == yi ? 1.f : 0.f)) * inv_n;
         const float g1 = (e1 / den - (lane + 32 == yi ? 1.f : 0.f)) * inv_n;
-        if (lane < ld_dl) dl[r * ld_dl + lane] = f32_to_bf16(lane < n_classes ? g0 : 0.f);
-        if (lane + 32 < ld_dl) dl[r * ld_dl + lane + 32] = f32_to_bf16(lane + 32 < n_classes ? g1 : 0.f);
+        if (dl) {
+            if (lane < ld_dl) dl[r * ld_dl + lane] = f32_to_bf16(lane < n_classes ? g0 : 0.f);
+            if (lane + 32 < ld_dl) dl[r * ld_dl + lane + 32] = f32_to_bf16(lane + 32 < n_classes ? g1 : 0.f);
+        }
         if (dl_t) {
             if (lane < n_classes) dl_t[(int64_t)lane * ld_t + r] = f32_to_bf16(g0);
             if (lane + 32 < n_classes) dl_t[(int64_t)(lane + 32) * ld_t + r] = f32_to_bf16(g1);
         }
-        if (lane < n_classes) c0 += g0;
-        if (lane + 32 < n_classes) c1 += g1;
     }
     if (lane == 0) s_loss[warp] = my_loss;
-    s_col[warp][lane] = c0;
-    s_col[warp][lane + 32] = c1;
     __syncthreads();
-    if (threadIdx.x < 64) {
-        float s = 0.f;
-        for (int w = 0; w < kSmThreads / kWarp; ++w) s += s_col[w][threadIdx.x];
-        if (threadIdx.x < n_classes) colsum_partial[(int64_t)blockIdx.x * n_classes + threadIdx.x] = s;
-    }
     if (threadIdx.x == 0) {
         float s = 0.f;
         for (int w = 0; w < kSmThreads / kWarp; ++w) s += s_loss[w];
@@ -264,7 +203,7 @@ struct GradSeg {
     int64_t count;
 };
 struct UpdateArgs {
-    GradSeg seg[4];
+    GradSeg seg[2];
     int n_seg;
     float* theta;
     float* m;

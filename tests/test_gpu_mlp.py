@@ -46,6 +46,11 @@ def test_pack_rows_gathers_rounds_and_transposes():
         assert dst[:, 37:].abs().sum() == 0 and dst_t[:, 45:].abs().sum() == 0
     dst, _ = B().retexo_pack_rows(dev(src), None, dim=20)
     assert torch.equal(dst[:, :20].cpu(), torch.from_numpy(src[:, :20]).to(torch.bfloat16))
+    # the row of ones that carries the bias gradient through the weight-gradient product
+    _, dst_t = B().retexo_pack_rows(dev(src), dev(idx), transpose=True, ones_row=True)
+    assert dst_t.shape == (38, 48)
+    assert torch.equal(dst_t[:37, :45].cpu(), want.T)
+    assert torch.equal(dst_t[37].float().cpu(), torch.cat([torch.ones(45), torch.zeros(3)]))
 
 
 @pytest.mark.parametrize("d_in,hidden,n_classes,n", [(5, 0, 3, 17), (64, 64, 7, 140), (33, 20, 4, 65),
@@ -59,7 +64,7 @@ def test_train_steps_track_the_checker(d_in, hidden, n_classes, n, opt):
     # Adam's first steps move every weight by about lr whatever the gradient's size, so weights whose
     # gradient is at rounding level take a different step in fp32 and fp64: keep that step small.
     ref, gpu = make_pair(d_in, hidden, n_classes, 1, opt=opt, lr=0.02 if opt == oracle.SGD else 1e-3)
-    x16, x_t = B().retexo_pack_rows(dev(x), None, transpose=True)
+    x16, x_t = B().retexo_pack_rows(dev(x), None, transpose=True, ones_row=True)
     yd = dev(y)
     for it in range(4):
         # Every iteration starts from the GPU's own state, so that each step is compared on its
@@ -91,7 +96,7 @@ def test_zero_weights_give_log_of_class_count():
     y = np.random.default_rng(4).integers(0, o, n).astype(np.int32)
     gpu = B().Mlp(d, h, o, np.zeros((d, h)), np.zeros(h), np.zeros((h, o)), np.zeros(o), optimizer=oracle.SGD, lr=0.1)
     x16, _ = B().retexo_pack_rows(dev(x))
-    loss = B().retexo_mlp_train_step(gpu, x16, dev(y))
+    loss = B().retexo_mlp_train_step(gpu, x16, dev(y))      # no x_t given: the call builds it itself
     assert abs(loss.item() - np.log(o)) < 1e-6
 
 

@@ -173,9 +173,9 @@ def test_operand_rounding_happens_exactly_at_the_matrix_products():
     g = m.unpack(grad)
     assert abs(loss - loss_ref) < 1e-12
     np.testing.assert_allclose(g["w2"], dw2.numpy(), atol=1e-13)
-    np.testing.assert_allclose(g["b2"], dl.sum(0).numpy(), atol=1e-13)
+    np.testing.assert_allclose(g["b2"], r(dl.numpy()).sum(0).numpy(), atol=1e-13)     # 1^T dL is a product too
     np.testing.assert_allclose(g["w1"], dw1.numpy(), atol=1e-13)
-    np.testing.assert_allclose(g["b1"], dhd.sum(0).numpy(), atol=1e-13)
+    np.testing.assert_allclose(g["b1"], r(dhd.numpy()).sum(0).numpy(), atol=1e-13)
 
 
 def test_embed_hidden_logits_prediction_and_tie_rule():
