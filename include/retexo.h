@@ -109,8 +109,8 @@ size_t retexo_aggregate_workspace_size(int64_t n_nodes, int64_t n_edges, int32_t
  * out      fp32 [n x ldout], may be NULL if out_bf16 is given.
  * out_bf16 optional bf16 (round-to-nearest-even) copy of the same matrix,
  *          row stride ldout_bf16 elements; NULL if not wanted.
- * Sums are taken in CSR order per row in fp32; rows of at least 2048 entries
- * are split over the warps of one block and combined in a fixed order.
+ * Sums are taken in CSR order per row in fp32; rows of at least 4096 entries
+ * are cut into segments of 2048 entries whose sums are added in segment order.
  * 128-bit loads are used when q is 16-byte aligned, ldq % 4 == 0 and
  * ldq >= round_up(dim, 4); 64-bit loads under the analogous rule; otherwise
  * scalar loads.  Nothing is an error for being unaligned.

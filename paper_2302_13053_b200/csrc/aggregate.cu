@@ -3,24 +3,35 @@
 // GAT edge-score / segment-softmax / weighted-sum pass, over a CSR graph.
 //
 // The work is a gather-reduce bound by the memory system, not a dense
-// contraction: rows are streamed with the widest aligned vector loads, one
-// warp per destination row (a whole block for rows of >= kHeavyDegree
-// entries), several neighbour rows in flight per lane, sums in registers.
+// contraction: neighbour rows are streamed with the widest aligned vector
+// loads, several rows in flight per lane, sums kept in registers.  Work is
+// handed out warp by warp from one counter (a persistent grid), so a power-law
+// degree distribution does not leave SMs idle: rows of kHeavyDegree entries or
+// more are cut into segments of kSegLen entries that are handed out first,
+// each segment's partial sum goes to scratch, and a second kernel adds a row's
+// segments in order.  Nothing depends on which warp ran what, so results are
+// the same bits on every call.
 #include "common.cuh"
 
 namespace retexo {
 
-constexpr int kHeavyDegree = 2048;     // rows at least this long get a whole block
+constexpr int kHeavyDegree = 4096;     // rows at least this long are cut into segments
+constexpr int kSegLen = 2048;          // entries per segment
 constexpr int kAggThreads = 256;
 constexpr int kAggWarps = kAggThreads / kWarp;
 constexpr int kUnroll = 4;             // neighbour rows in flight per lane and column chunk
 
+// Upper bound on the number of segments of a graph with n_edges entries.
+static inline int64_t max_segments(int64_t n_edges) { return n_edges / kSegLen + n_edges / kHeavyDegree + 1; }
+
 // ---------------------------------------------------------------- pre-pass
 // coef[v]: GCN (deg+1)^-1/2, SAGE 1/deg (0 for isolated nodes).  Also lists
-// the heavy rows (order irrelevant: each row's result does not depend on it).
+// the heavy rows and their segments (list order is arbitrary; no result
+// depends on it).
 __global__ void prep_rows_kernel(int64_t n, const int64_t* __restrict__ rowptr, int mode,
                                  float* __restrict__ coef, int32_t* __restrict__ heavy_list,
-                                 int32_t* __restrict__ heavy_count) {
+                                 int32_t* __restrict__ heavy_seg_base, int32_t* __restrict__ seg_slot,
+                                 int32_t* __restrict__ counters /* [0] heavy rows, [1] segments, [2] work */) {
     int64_t v = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (v >= n) return;
     int64_t deg = rowptr[v + 1] - rowptr[v];
@@ -29,8 +40,12 @@ __global__ void prep_rows_kernel(int64_t n, const int64_t* __restrict__ rowptr, 
     else c = deg > 0 ? 1.0f / (float)deg : 0.0f;
     coef[v] = c;
     if (deg >= kHeavyDegree) {
-        int32_t slot = atomicAdd(heavy_count, 1);
+        const int32_t slot = atomicAdd(counters + 0, 1);
+        const int32_t nseg = (int32_t)((deg + kSegLen - 1) / kSegLen);
+        const int32_t base = atomicAdd(counters + 1, nseg);
         heavy_list[slot] = (int32_t)v;
+        heavy_seg_base[slot] = base;
+        for (int32_t i = 0; i < nseg; ++i) seg_slot[base + i] = slot;
     }
 }
 
@@ -78,8 +93,12 @@ struct AggArgs {
     __nv_bfloat16* out16;   // may be null
     int64_t ldout16;
     int32_t concat_self;    // SAGE
-    const int32_t* heavy_list;
-    const int32_t* heavy_count;
+    const int32_t* heavy_list;       // [heavy rows] node id
+    const int32_t* heavy_seg_base;   // [heavy rows] first segment of the row
+    const int32_t* seg_slot;         // [segments] index into heavy_list
+    int32_t* counters;               // [0] heavy rows, [1] segments, [2] next work item
+    float* seg_partial;              // [segments x round_up(dim, 4)] raw sums
+    int64_t ld_partial;
 };
 
 // Adds the neighbour rows of CSR entries [beg, end) into acc, in order, for the
@@ -181,71 +200,104 @@ __device__ __forceinline__ void finish_row(const AggArgs& a, int64_t v, int lane
     }
 }
 
-// One warp per destination row; heavy rows are skipped here.
+// Persistent kernel: each warp draws work items from one counter.  Items
+// [0, n_seg) are segments of heavy rows (their raw sums go to scratch), items
+// [n_seg, n_seg + n) are whole rows (heavy ones are skipped: their segments
+// cover them).
 template <int VEC, int CH, bool GCN>
-__global__ void __launch_bounds__(kAggThreads) agg_warp_rows_kernel(AggArgs a) {
+__global__ void __launch_bounds__(kAggThreads) agg_rows_kernel(AggArgs a) {
     using V = typename VecT<VEC>::type;
     const int lane = threadIdx.x & 31;
-    const int64_t v = blockIdx.x * (int64_t)kAggWarps + (threadIdx.x >> 5);
-    if (v >= a.n) return;
-    const int64_t beg = a.rowptr[v], end = a.rowptr[v + 1];
-    if (end - beg >= kHeavyDegree) return;
     const int nvec = (a.dim + VEC - 1) / VEC;
-    for (int vec0 = 0; vec0 < nvec; vec0 += CH * kWarp) {
-        V acc[CH];
+    const int64_t n_seg = a.counters[1];
+    const int64_t total = n_seg + a.n;
+    for (;;) {
+        int64_t item = 0;
+        if (lane == 0) item = atomicAdd(reinterpret_cast<unsigned int*>(a.counters + 2), 1u);
+        item = __shfl_sync(0xffffffffu, item, 0);
+        if (item >= total) break;
+        if (item < n_seg) {
+            const int32_t slot = a.seg_slot[item];
+            const int64_t v = a.heavy_list[slot];
+            const int64_t i = item - a.heavy_seg_base[slot];
+            const int64_t beg = a.rowptr[v] + i * kSegLen;
+            const int64_t end = min(a.rowptr[v + 1], beg + kSegLen);
+            for (int vec0 = 0; vec0 < nvec; vec0 += CH * kWarp) {
+                V acc[CH];
 #pragma unroll
-        for (int c = 0; c < CH; ++c) vec_zero<VEC>(acc[c]);
-        accumulate_range<VEC, CH, GCN>(a, beg, end, lane, vec0, nvec, acc);
-        finish_row<VEC, CH, GCN>(a, v, lane, vec0, nvec, acc);
+                for (int c = 0; c < CH; ++c) vec_zero<VEC>(acc[c]);
+                accumulate_range<VEC, CH, GCN>(a, beg, end, lane, vec0, nvec, acc);
+                float* dst = a.seg_partial + item * a.ld_partial;
+#pragma unroll
+                for (int c = 0; c < CH; ++c) {
+                    const int vi = vec0 + c * kWarp + lane;
+                    if (vi >= nvec) continue;
+#pragma unroll
+                    for (int k = 0; k < VEC; ++k) dst[vi * VEC + k] = vec_get<VEC>(acc[c], k);
+                }
+            }
+        } else {
+            const int64_t v = item - n_seg;
+            const int64_t beg = a.rowptr[v], end = a.rowptr[v + 1];
+            if (end - beg >= kHeavyDegree) continue;
+            for (int vec0 = 0; vec0 < nvec; vec0 += CH * kWarp) {
+                V acc[CH];
+#pragma unroll
+                for (int c = 0; c < CH; ++c) vec_zero<VEC>(acc[c]);
+                accumulate_range<VEC, CH, GCN>(a, beg, end, lane, vec0, nvec, acc);
+                finish_row<VEC, CH, GCN>(a, v, lane, vec0, nvec, acc);
+            }
+        }
     }
 }
 
-// One block per heavy row: warp w sums the w-th contiguous slice of the row's
-// entries; the slices are then added in warp order (fixed, so deterministic).
+// One warp per heavy row: adds the row's segment sums in segment order and
+// finishes the row.
 template <int VEC, int CH, bool GCN>
-__global__ void __launch_bounds__(kAggThreads) agg_block_rows_kernel(AggArgs a) {
+__global__ void __launch_bounds__(kAggThreads) agg_combine_kernel(AggArgs a) {
     using V = typename VecT<VEC>::type;
-    __shared__ V part[kAggWarps][CH * kWarp];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int n_heavy = *a.heavy_count;
+    const int lane = threadIdx.x & 31;
     const int nvec = (a.dim + VEC - 1) / VEC;
-    for (int h = blockIdx.x; h < n_heavy; h += gridDim.x) {
+    const int n_heavy = a.counters[0];
+    for (int h = blockIdx.x * kAggWarps + (threadIdx.x >> 5); h < n_heavy; h += gridDim.x * kAggWarps) {
         const int64_t v = a.heavy_list[h];
-        const int64_t beg = a.rowptr[v], end = a.rowptr[v + 1];
-        const int64_t len = end - beg;
-        // slice boundaries on multiples of 32 entries
-        const int64_t chunks = (len + kWarp - 1) / kWarp;
-        const int64_t c0 = chunks * warp / kAggWarps, c1 = chunks * (warp + 1) / kAggWarps;
-        const int64_t sbeg = beg + c0 * kWarp, send = min(end, beg + c1 * kWarp);
+        const int64_t deg = a.rowptr[v + 1] - a.rowptr[v];
+        const int nseg = (int)((deg + kSegLen - 1) / kSegLen);
+        const float* src = a.seg_partial + (int64_t)a.heavy_seg_base[h] * a.ld_partial;
         for (int vec0 = 0; vec0 < nvec; vec0 += CH * kWarp) {
             V acc[CH];
 #pragma unroll
             for (int c = 0; c < CH; ++c) vec_zero<VEC>(acc[c]);
-            accumulate_range<VEC, CH, GCN>(a, sbeg, send, lane, vec0, nvec, acc);
-#pragma unroll
-            for (int c = 0; c < CH; ++c) part[warp][c * kWarp + lane] = acc[c];
-            __syncthreads();
-            if (warp == 0) {
+            for (int i = 0; i < nseg; ++i) {
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
-                    V s = part[0][c * kWarp + lane];
-                    for (int w = 1; w < kAggWarps; ++w) vec_add(s, part[w][c * kWarp + lane]);
-                    acc[c] = s;
+                    const int vi = vec0 + c * kWarp + lane;
+                    if (vi >= nvec) continue;
+                    float t[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                    for (int k = 0; k < VEC; ++k) t[k] = src[(int64_t)i * a.ld_partial + vi * VEC + k];
+                    V x;
+                    if constexpr (VEC == 4) x = make_float4(t[0], t[1], t[2], t[3]);
+                    else if constexpr (VEC == 2) x = make_float2(t[0], t[1]);
+                    else x = t[0];
+                    vec_add(acc[c], x);
                 }
-                finish_row<VEC, CH, GCN>(a, v, lane, vec0, nvec, acc);
             }
-            __syncthreads();
+            finish_row<VEC, CH, GCN>(a, v, lane, vec0, nvec, acc);
         }
     }
 }
 
 template <int VEC, int CH, bool GCN>
 static int launch_agg(const AggArgs& a, int n_sm, cudaStream_t st) {
-    if (a.n > 0) {
-        const int64_t blocks = (a.n + kAggWarps - 1) / kAggWarps;
-        agg_warp_rows_kernel<VEC, CH, GCN><<<(unsigned)blocks, kAggThreads, 0, st>>>(a);
-        agg_block_rows_kernel<VEC, CH, GCN><<<n_sm * 2, kAggThreads, 0, st>>>(a);
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, agg_rows_kernel<VEC, CH, GCN>, kAggThreads, 0) !=
+            cudaSuccess || per_sm < 1) {
+        (void)cudaGetLastError();
+        per_sm = 1;
     }
+    agg_rows_kernel<VEC, CH, GCN><<<n_sm * per_sm, kAggThreads, 0, st>>>(a);
+    agg_combine_kernel<VEC, CH, GCN><<<n_sm, kAggThreads, 0, st>>>(a);
     return launch_status();
 }
 
@@ -400,16 +452,18 @@ using namespace retexo;
 
 extern "C" size_t retexo_aggregate_workspace_size(int64_t n_nodes, int64_t n_edges, int32_t type,
                                                   int32_t dim, int32_t heads) {
-    (void)n_edges; (void)dim;
     Sizer s;
     if (n_nodes < 0) return 0;
     if (type == RETEXO_GAT) {
         s.take<float>((size_t)n_nodes * (size_t)(heads > 0 ? heads : 1));
         s.take<float>((size_t)n_nodes * (size_t)(heads > 0 ? heads : 1));
     } else {
-        s.take<float>((size_t)n_nodes);        // coef
-        s.take<int32_t>((size_t)n_nodes);      // heavy row list
-        s.take<int32_t>(64);                   // heavy row count
+        s.take<float>((size_t)n_nodes);                                   // coef
+        s.take<int32_t>((size_t)(n_edges / kHeavyDegree + 1));            // heavy rows
+        s.take<int32_t>((size_t)(n_edges / kHeavyDegree + 1));            // their first segment
+        s.take<int32_t>((size_t)max_segments(n_edges));                   // segment -> heavy row
+        s.take<int32_t>(64);                                              // counters
+        s.take<float>((size_t)max_segments(n_edges) * (size_t)((dim + 3) / 4 * 4));   // segment sums
     }
     return s.off + kAlign;
 }
@@ -464,14 +518,21 @@ extern "C" int retexo_aggregate(const retexo_csr* g, int32_t type, const float* 
     AggArgs a;
     a.n = n; a.rowptr = g->rowptr; a.colidx = g->colidx; a.q = q; a.ldq = ldq; a.dim = dim;
     float* coef = ws.take<float>((size_t)n);
-    int32_t* heavy_list = ws.take<int32_t>((size_t)n);
-    int32_t* heavy_count = ws.take<int32_t>(64);
-    a.coef = coef; a.heavy_list = heavy_list; a.heavy_count = heavy_count;
+    const int64_t e = g->n_edges;
+    int32_t* heavy_list = ws.take<int32_t>((size_t)(e / kHeavyDegree + 1));
+    int32_t* heavy_seg_base = ws.take<int32_t>((size_t)(e / kHeavyDegree + 1));
+    int32_t* seg_slot = ws.take<int32_t>((size_t)max_segments(e));
+    int32_t* counters = ws.take<int32_t>(64);
+    a.ld_partial = (dim + 3) / 4 * 4;
+    a.seg_partial = ws.take<float>((size_t)max_segments(e) * (size_t)a.ld_partial);
+    a.coef = coef; a.heavy_list = heavy_list; a.heavy_seg_base = heavy_seg_base; a.seg_slot = seg_slot;
+    a.counters = counters;
     a.out = out; a.ldout = ldout;
     a.out16 = static_cast<__nv_bfloat16*>(out_bf16); a.ldout16 = ldout_bf16;
     a.concat_self = concat_self ? 1 : 0;
-    RETEXO_CUDA_TRY(cudaMemsetAsync(heavy_count, 0, sizeof(int32_t), st));
-    prep_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(n, g->rowptr, type, coef, heavy_list, heavy_count);
+    RETEXO_CUDA_TRY(cudaMemsetAsync(counters, 0, 64 * sizeof(int32_t), st));
+    prep_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(n, g->rowptr, type, coef, heavy_list,
+                                                                  heavy_seg_base, seg_slot, counters);
 
     const bool gcn = type == RETEXO_GCN;
     const bool v4 = aligned_to(q, 16) && ldq % 4 == 0 && ldq >= (dim + 3) / 4 * 4;

@@ -108,10 +108,10 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
         if (s > agg_b) agg_b = s;
     }
     const int64_t ld16 = round_up(max_din, 8);
+    l.features = t.template take<float>((size_t)n * round_up(c.d0, 32));   // 128-byte-row copy of the features
     if (host) {
         l.rowptr = t.template take<int64_t>((size_t)n + 1);
         l.colidx = t.template take<int32_t>((size_t)e);
-        l.features = t.template take<float>((size_t)n * round_up(c.d0, 32));
         l.labels = t.template take<int32_t>((size_t)n);
         l.train_idx = t.template take<int32_t>((size_t)n_tr);
         l.val_idx = t.template take<int32_t>((size_t)n_val);
@@ -244,6 +244,15 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         g.rowptr = b.rowptr; g.colidx = b.colidx; feat = b.features; ld_feat = ldp;
         labels = b.labels; train_idx = b.train_idx; val_idx = b.val_idx; test_idx = b.test_idx;
         if (part) part = b.part;
+    } else if (ld_feat % 4 != 0 || !aligned_to(feat, 16)) {
+        // rows that do not start on 16-byte boundaries would force narrow loads on the dominant
+        // gather of round 1: re-lay them once with rows of whole 128-byte lines
+        const int64_t ldp = round_up(c.d0, 32);
+        if (ldp != c.d0) RETEXO_CUDA_TRY(cudaMemsetAsync(b.features, 0, sizeof(float) * (size_t)n * ldp, st));
+        RETEXO_CUDA_TRY(cudaMemcpy2DAsync(b.features, sizeof(float) * ldp, feat, sizeof(float) * ld_feat,
+                                          sizeof(float) * c.d0, (size_t)n, cudaMemcpyDeviceToDevice, st));
+        feat = b.features;
+        ld_feat = ldp;
     }
     gather_i32_kernel<<<(unsigned)((n_tr + 255) / 256), 256, 0, st>>>(labels, train_idx, n_tr, b.y_tr);
     if (n_val) gather_i32_kernel<<<(unsigned)((n_val + 255) / 256), 256, 0, st>>>(labels, val_idx, n_val, b.y_val);

@@ -102,8 +102,42 @@ struct TcKernelArgs {
     __nv_bfloat16* out_bf16_t; int64_t ld_t; int ones_row_t;
     const __nv_bfloat16* mask; int64_t ld_mask;
     float* partial;
+    const int32_t* y; float inv_rows; float* loss_partial;
+    int32_t* pred; unsigned long long* correct;
     int32_t* status;
 };
+
+constexpr int kStagePitch = 80;                       // bytes per column in the transpose staging (64 + 16 pad)
+constexpr int kStageBytesPerWarp = 32 * kStagePitch;
+
+// Writes a warp's 32 x 32 block (lane = row, v[j] = column col0 + j) into the transposed output
+// out_t[col][row].  Full, aligned blocks go through shared memory so that every column leaves
+// as one 64-byte run; ragged ones fall back to guarded element stores.
+__device__ __forceinline__ void store_block_transposed(__nv_bfloat16* out_t, int64_t ld_t, int64_t col0, int64_t n_cols,
+                                                       int64_t row0, int64_t M, const float (&v)[32], uint8_t* stage,
+                                                       int lane) {
+    const bool fast = row0 + 32 <= M && (ld_t & 7) == 0 && aligned16(out_t);
+    if (fast) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            *reinterpret_cast<__nv_bfloat16*>(stage + j * kStagePitch + lane * 2) = __float2bfloat16_rn(v[j]);
+        __syncwarp();
+        if (col0 + lane < n_cols) {
+            __nv_bfloat16* dst = out_t + (col0 + lane) * ld_t + row0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                *reinterpret_cast<uint4*>(dst + 8 * i) = *reinterpret_cast<const uint4*>(stage + lane * kStagePitch + 16 * i);
+        }
+        __syncwarp();
+    } else {
+        const int64_t row = row0 + lane;
+        if (row < M) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (col0 + j < n_cols) out_t[(col0 + j) * ld_t + row] = __float2bfloat16_rn(v[j]);
+        }
+    }
+}
 
 template <int BN, int STAGES>
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -116,6 +150,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint64_t* acc_ready = empty + STAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_ready + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    float* warp_loss = reinterpret_cast<float*>(tmem_slot + 2);                  // [4]
+    uint8_t* stage_base = reinterpret_cast<uint8_t*>(                           // 4 x kStageBytesPerWarp, 16-byte aligned
+        (reinterpret_cast<uintptr_t>(tmem_slot) + 64 + 15) & ~uintptr_t(15));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t m0 = (int64_t)blockIdx.x * kTcBM, n0 = (int64_t)blockIdx.y * BN;
@@ -180,10 +217,96 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         const int q = warp & 3;                           // tensor-memory lane quarter this warp may read
-        const int64_t row = m0 + q * 32 + lane;
+        const int64_t row0 = m0 + q * 32;
+        const int64_t row = row0 + lane;
+        uint8_t* stage = stage_base + q * kStageBytesPerWarp;
         bool ok = n_kb > 0 ? mbar_wait(acc_ready, 0, g.status, abort_flag) : true;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok) {
+        if (BN == 64 && (g.mode == TC_EPI_SOFTMAX_CE || g.mode == TC_EPI_ARGMAX)) {
+            // the thread owns the whole row of logits
+            float v[64];
+            if (ok) {
+#pragma unroll
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t r[32];
+                    if (n_kb > 0) tmem_ld_32cols(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                    else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = 0u;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int c = c0 + j;
+                        v[c] = c < g.N ? __uint_as_float(r[j]) + (g.bias ? __ldg(g.bias + c) : 0.f) : -INFINITY;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int c = 0; c < 64; ++c) v[c] = 0.f;
+            }
+            const bool live = ok && row < g.M;
+            const int32_t yi = (live && g.y) ? g.y[row] : -1;
+            if (g.mode == TC_EPI_ARGMAX) {
+                int best = 0;
+                float bv = v[0];
+#pragma unroll
+                for (int c = 1; c < 64; ++c) if (v[c] > bv) { bv = v[c]; best = c; }   // strict: lowest index wins ties
+                if (live) {
+                    if (g.pred) g.pred[row] = best;
+                    if (g.out_f32) {
+#pragma unroll
+                        for (int c = 0; c < 64; ++c) if (c < g.N) g.out_f32[row * g.ld_f32 + c] = v[c];
+                    }
+                }
+                if (g.correct) {
+                    const unsigned hits = __ballot_sync(0xffffffffu, live && best == yi);
+                    if (lane == 0 && hits) atomicAdd(g.correct, (unsigned long long)__popc(hits));
+                }
+            } else {
+                float mx = v[0];
+#pragma unroll
+                for (int c = 1; c < 64; ++c) mx = fmaxf(mx, v[c]);
+                float den = 0.f, ly = 0.f;
+#pragma unroll
+                for (int c = 0; c < 64; ++c) {
+                    ly = c == yi ? v[c] : ly;
+                    v[c] = c < g.N ? expf(v[c] - mx) : 0.f;
+                    den += v[c];
+                }
+                float loss = live ? (mx + logf(den)) - ly : 0.f;
+                const float scale = g.inv_rows / den;
+#pragma unroll
+                for (int c = 0; c < 64; ++c) v[c] = c < g.N ? (v[c] * scale - (c == yi ? g.inv_rows : 0.f)) : 0.f;
+                if (live && g.out_bf16) {       // dL row-major, ld_bf16 <= 64 and a multiple of 8
+                    __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16;
+#pragma unroll
+                    for (int c = 0; c < 64; c += 8) {
+                        if (c >= g.ld_bf16) break;
+                        __nv_bfloat162 p0 = __floats2bfloat162_rn(v[c], v[c + 1]), p1 = __floats2bfloat162_rn(v[c + 2], v[c + 3]);
+                        __nv_bfloat162 p2 = __floats2bfloat162_rn(v[c + 4], v[c + 5]), p3 = __floats2bfloat162_rn(v[c + 6], v[c + 7]);
+                        uint4 pk;
+                        pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                        pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                        *reinterpret_cast<uint4*>(dst + c) = pk;
+                    }
+                }
+                if (ok && g.out_bf16_t) {
+#pragma unroll
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        if (c0 >= g.N) break;
+                        float blk[32];
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) blk[j] = v[c0 + j];
+                        store_block_transposed(g.out_bf16_t, g.ld_t, c0, g.N, row0, g.M, blk, stage, lane);
+                    }
+                }
+                loss = warp_sum(loss);
+                if (lane == 0) warp_loss[q] = loss;
+                asm volatile("bar.sync 1, 128;" ::: "memory");      // the four epilogue warps only
+                if (q == 0 && lane == 0 && g.loss_partial)
+                    g.loss_partial[blockIdx.x] = ((warp_loss[0] + warp_loss[1]) + warp_loss[2]) + warp_loss[3];
+            }
+        } else if (ok) {
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
@@ -192,20 +315,43 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int j = 0; j < 32; ++j) r[j] = 0u;
                 }
-                if (row >= g.M) continue;
                 const int64_t col0 = n0 + c0;
+                if (col0 >= g.N) continue;
                 if (g.mode == TC_EPI_PARTIAL) {
+                    if (row >= g.M) continue;
                     float* dst = g.partial + ((int64_t)blockIdx.z * g.M + row) * g.N + col0;
+                    if (col0 + 32 <= g.N && (g.N & 3) == 0 && aligned16(g.partial)) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __uint_as_float(r[j]);
-                } else if (g.mode == TC_EPI_MASK_T) {
-                    const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
+                        for (int j = 0; j < 32; j += 4)
+                            *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                                              __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                    } else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        if (col0 + j >= g.N) continue;
-                        const float keep = __bfloat162float(mrow[j]) > 0.f ? __uint_as_float(r[j]) : 0.f;
-                        g.out_bf16_t[(col0 + j) * g.ld_t + row] = __float2bfloat16_rn(keep);
+                        for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __uint_as_float(r[j]);
                     }
+                } else if (g.mode == TC_EPI_MASK_T) {
+                    float v[32];
+                    if (row < g.M) {
+                        const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
+                        if (col0 + 32 <= g.N && (g.ld_mask & 7) == 0 && aligned16(g.mask)) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                const uint4 pk = *reinterpret_cast<const uint4*>(mrow + j);
+                                const __nv_bfloat16* mv = reinterpret_cast<const __nv_bfloat16*>(&pk);
+#pragma unroll
+                                for (int k = 0; k < 8; ++k)
+                                    v[j + k] = __bfloat162float(mv[k]) > 0.f ? __uint_as_float(r[j + k]) : 0.f;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                v[j] = (col0 + j < g.N && __bfloat162float(mrow[j]) > 0.f) ? __uint_as_float(r[j]) : 0.f;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                    }
+                    store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane);
                 } else {
                     float v[32];
 #pragma unroll
@@ -215,6 +361,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         if (g.relu) x = fmaxf(x, 0.f);
                         v[j] = x;
                     }
+                    if (g.out_bf16_t) {
+                        store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane);
+                        if (g.ones_row_t && col0 == 0 && row < g.M) g.out_bf16_t[g.N * g.ld_t + row] = __float2bfloat16_rn(1.0f);
+                    }
+                    if (row >= g.M) continue;
                     if (g.out_f32) {
                         float* dst = g.out_f32 + row * g.ld_f32 + col0;
                         if (col0 + 32 <= g.N && (g.ld_f32 & 3) == 0 && aligned16(g.out_f32)) {
@@ -225,12 +376,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                             for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = v[j];
                         }
-                    }
-                    if (g.out_bf16_t) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (col0 + j < g.N) g.out_bf16_t[(col0 + j) * g.ld_t + row] = __float2bfloat16_rn(v[j]);
-                        if (g.ones_row_t && col0 == 0) g.out_bf16_t[g.N * g.ld_t + row] = __float2bfloat16_rn(1.0f);
                     }
                     if (g.out_bf16) {
                         __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16 + col0;
@@ -295,7 +440,7 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t c
 
 template <int BN, int STAGES>
 static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
-    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 256;
+    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 512 + 4 * kStageBytesPerWarp;
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
@@ -315,6 +460,7 @@ static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& 
     g.out_bf16_t = t.out_bf16_t; g.ld_t = t.ld_t; g.ones_row_t = t.ones_row_t;
     g.mask = t.mask; g.ld_mask = t.ld_mask;
     g.partial = t.partial; g.status = t.status;
+    g.y = t.y; g.inv_rows = t.inv_rows; g.loss_partial = t.loss_partial; g.pred = t.pred; g.correct = t.correct;
     dim3 grid((unsigned)((t.M + kTcBM - 1) / kTcBM), (unsigned)((t.N + BN - 1) / BN), (unsigned)splits);
     tc_gemm_kernel<BN, STAGES><<<grid, kTcThreads, smem, st>>>(ma, mb, g);
     return launch_status();
@@ -324,6 +470,8 @@ bool tc_gemm_supported(const TcGemm& t) {
     if (t.M <= 0 || t.N <= 0 || t.K <= 0) return false;
     if (t.mode == TC_EPI_MASK_T && (!t.mask || !t.out_bf16_t)) return false;
     if (t.mode == TC_EPI_PARTIAL && !t.partial) return false;
+    if ((t.mode == TC_EPI_SOFTMAX_CE || t.mode == TC_EPI_ARGMAX) && t.N > 64) return false;
+    if (t.mode == TC_EPI_SOFTMAX_CE && (!t.y || (t.out_bf16 && (t.ld_bf16 % 8 != 0 || t.ld_bf16 > 64)))) return false;
     if (!aligned_to(t.A, 16) || !aligned_to(t.B, 16) || t.lda % 8 != 0 || t.ldb % 8 != 0) return false;
     if (t.M > INT32_MAX || t.N > INT32_MAX || t.K > INT32_MAX - 64) return false;
     if ((t.M + kTcBM - 1) / kTcBM > 2147483647LL || (t.N + 63) / 64 > 65535) return false;

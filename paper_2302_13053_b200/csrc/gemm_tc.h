@@ -6,7 +6,7 @@
 
 namespace retexo {
 
-enum TcEpilogue { TC_EPI_BIAS = 0, TC_EPI_PARTIAL = 1, TC_EPI_MASK_T = 2 };
+enum TcEpilogue { TC_EPI_BIAS = 0, TC_EPI_PARTIAL = 1, TC_EPI_MASK_T = 2, TC_EPI_SOFTMAX_CE = 3, TC_EPI_ARGMAX = 4 };
 
 // C[M x N] = A[M x K] * B[N x K]^T with A and B bf16, K contiguous (row strides
 // lda / ldb elements, multiples of 8; bases 16-byte aligned).
@@ -21,6 +21,13 @@ enum TcEpilogue { TC_EPI_BIAS = 0, TC_EPI_PARTIAL = 1, TC_EPI_MASK_T = 2 };
 //   TC_EPI_MASK_T : out_bf16_t[n][m] = acc[m][n] where mask[m][n] > 0 (bf16, row stride
 //                   ld_mask), else 0: the ReLU gate applied to a back-propagated gradient,
 //                   stored transposed.
+//   TC_EPI_SOFTMAX_CE (N <= 64): logits = acc + bias; per row the softmax cross-entropy against
+//                   label y[m] and its gradient dL = (softmax - onehot) * inv_rows, written as bf16
+//                   row-major (out_bf16, ld_bf16 a multiple of 8, padding columns zero) and
+//                   transposed (out_bf16_t [N x ld_t]); loss_partial[blockIdx.x] = sum of the
+//                   block's row losses.  The logits never leave the SM.
+//   TC_EPI_ARGMAX (N <= 64): logits = acc + bias; pred[m] = arg-max (lowest index on ties),
+//                   *correct += number of rows with pred == y[m]; optional fp32 logits (out_f32).
 // status: device word that receives RETEXO_ERR_TIMEOUT if a bounded wait gives up.
 struct TcGemm {
     const __nv_bfloat16* A; int64_t lda;
@@ -33,6 +40,8 @@ struct TcGemm {
     __nv_bfloat16* out_bf16_t; int64_t ld_t; int ones_row_t;
     const __nv_bfloat16* mask; int64_t ld_mask;
     float* partial;
+    const int32_t* y; float inv_rows; float* loss_partial;      // TC_EPI_SOFTMAX_CE / TC_EPI_ARGMAX
+    int32_t* pred; unsigned long long* correct;                  // TC_EPI_ARGMAX (both optional)
     int32_t* status;
 };
 

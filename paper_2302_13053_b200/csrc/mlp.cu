@@ -62,8 +62,7 @@ MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_row
     p.ld_h = round_up8(hidden > 0 ? hidden : 1);
     p.ld_k = round_up8(d_in);
     p.ld_n = round_up8(n_rows);
-    p.sm_blocks = (n_rows + 7) / 8 < kTargetBlocks ? (n_rows + 7) / 8 : kTargetBlocks;
-    if (p.sm_blocks < 1) p.sm_blocks = 1;
+    p.sm_blocks = (n_rows + 127) / 128;          // one loss partial per 128-row tile of the head product
     p.split_w1 = tc_split((int64_t)d_in + 1, p.out1, n_rows);
     p.split_w2 = hidden > 0 ? tc_split((int64_t)hidden + 1, n_classes, n_rows) : 0;
     return p;
@@ -203,22 +202,22 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         ld_xt = p.ld_n;
     }
 
-    // ---- forward
+    // ---- forward; the class-dimension product ends in the loss: softmax, cross-entropy and dL
+    //      are computed in its epilogue, where one thread holds a whole row of logits
     TcGemm fwd = tc_base(x, ldx, b.w1t16, p.ld_k, n, out1, d_in, b.status);
     fwd.bias = b1;
+    TcGemm head = fwd;
     if (H > 0) {
         fwd.relu = 1; fwd.out_bf16 = b.hd16; fwd.ld_bf16 = p.ld_h;
         fwd.out_bf16_t = b.hdt16; fwd.ld_t = p.ld_n; fwd.ones_row_t = 1;
         RETEXO_TRY(tc_gemm_launch(fwd, st));
-        TcGemm lg = tc_base(b.hd16, p.ld_h, b.w2t16, p.ld_h, n, O, H, b.status);
-        lg.bias = b2; lg.out_f32 = b.logits; lg.ld_f32 = O;
-        RETEXO_TRY(tc_gemm_launch(lg, st));
-    } else {
-        fwd.out_f32 = b.logits; fwd.ld_f32 = O;
-        RETEXO_TRY(tc_gemm_launch(fwd, st));
+        head = tc_base(b.hd16, p.ld_h, b.w2t16, p.ld_h, n, O, H, b.status);
+        head.bias = b2;
     }
-    softmax_ce_kernel<<<(unsigned)p.sm_blocks, kSmThreads, 0, st>>>(b.logits, O, y, n, O, H > 0 ? b.dl16 : nullptr,
-                                                                    p.ld_dl, b.dlt16, p.ld_n, b.loss_partial);
+    head.mode = TC_EPI_SOFTMAX_CE; head.y = y; head.inv_rows = 1.0f / (float)n; head.loss_partial = b.loss_partial;
+    head.out_bf16 = H > 0 ? b.dl16 : nullptr; head.ld_bf16 = p.ld_dl;
+    head.out_bf16_t = b.dlt16; head.ld_t = p.ld_n;
+    RETEXO_TRY(tc_gemm_launch(head, st));
     // ---- backward
     const bf16* grad1_t = b.dlt16;      // gradient at the first layer's output, transposed
     if (H > 0) {
@@ -349,13 +348,16 @@ extern "C" int retexo_embed(const retexo_mlp* model, const void* x, int64_t ldx,
                                             hidden_out_bf16, ld_hidden_bf16, nullptr, 0, 0, st));
             if (want_logits) {
                 TcGemm l2 = tc_base(h16, ld16, b.w2t16, p.ld_h, n_rows, O, H, b.status);
-                l2.bias = b2; l2.out_f32 = lg; l2.ld_f32 = ld_lg;
+                l2.bias = b2; l2.mode = TC_EPI_ARGMAX; l2.out_f32 = logits_out; l2.ld_f32 = ld_logits;
+                l2.pred = pred_out; l2.y = y; l2.correct = correct;
                 RETEXO_TRY(tc_gemm_launch(l2, st));
             }
         } else if (want_logits) {
-            fwd.out_f32 = lg; fwd.ld_f32 = ld_lg;
+            fwd.mode = TC_EPI_ARGMAX; fwd.out_f32 = logits_out; fwd.ld_f32 = ld_logits;
+            fwd.pred = pred_out; fwd.y = y; fwd.correct = correct;
             RETEXO_TRY(tc_gemm_launch(fwd, st));
         }
+        return launch_status();
     }
     if (pred_out || correct)
         argmax_kernel<<<(unsigned)((n_rows + 255) / 256), 256, 0, st>>>(lg, ld_lg, n_rows, O, pred_out, y, correct);

@@ -31,7 +31,7 @@ def run_gpu(aggr, rowptr, colidx, q, ld=None, dim=None, **kw):
     return out.cpu().numpy(), out16.float().cpu().numpy()
 
 
-LADDER = [0, 1, 2, 31, 32, 33, 63, 64, 65, 1025, 2047, 2048, 2049, 5000]
+LADDER = [0, 1, 2, 31, 32, 33, 63, 64, 65, 1025, 2047, 2048, 2049, 4095, 4096, 4097, 9000]   # 4096: rows cut into segments
 
 
 @pytest.mark.parametrize("aggr", [oracle.GCN, oracle.SAGE_MEAN])
