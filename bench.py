@@ -117,11 +117,11 @@ def launches_per_step(w, R: int) -> int:
         else:
             total += 3                               # prep, warp rows, block rows
         total += 2                                   # train / val batches
-        step = 8 if h > 0 else 5
-        ev = (4 if h > 0 else 3) + 2
+        step = 8 if h > 0 else 4                     # weight shadows, products, reduce + update
+        ev = (4 if h > 0 else 2) + 2                 # validation forward + snapshot / bookkeeping
         total += R * (step + ev)
         total += 2 * (4 if h > 0 else 3)             # test accuracy, kept and last iterate
-        total += 2 if h > 0 else 3                   # emission of Q^m / final logits
+        total += 3 if h > 0 else 2                   # emission of Q^m / final logits
     return total
 
 

@@ -65,21 +65,30 @@ __global__ void __launch_bounds__(kCntThreads) count_bitmap_kernel(CountArgs a) 
         if (beg == end) continue;
         const int32_t pu = part_of(a, u);
         unsigned row_new = 0;
-        for (int64_t e0 = beg; e0 < end; e0 += kWarp) {
-            const int64_t e = e0 + lane;
-            const bool valid = e < end;
-            int32_t pv = pu;
-            if (valid) pv = part_of(a, __ldg(a.colidx + e));
-            const bool cross = pv != pu;
-            bool is_new = false;
-            if (cross) {
-                const uint32_t bit = 1u << (pv & 31);
-                const uint32_t old = atomicOr(&bm[warp][pv >> 5], bit);
-                is_new = !(old & bit);
-                if (is_new && a.recv) atomicAdd(a.recv + pv, 1ull);
+        // four chunks of 32 entries per trip: the index loads, then the partition-id gathers, are
+        // issued together, so a trip costs two memory latencies instead of eight
+        for (int64_t e0 = beg; e0 < end; e0 += 4 * kWarp) {
+            int32_t nb[4], pv[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int64_t e = e0 + t * kWarp + lane;
+                nb[t] = e < end ? __ldg(a.colidx + e) : -1;
             }
-            my_cross += cross ? 1ull : 0ull;
-            row_new += __popc(__ballot_sync(0xffffffffu, is_new));
+#pragma unroll
+            for (int t = 0; t < 4; ++t) pv[t] = nb[t] >= 0 ? part_of(a, nb[t]) : pu;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const bool cross = pv[t] != pu;
+                bool is_new = false;
+                if (cross) {
+                    const uint32_t bit = 1u << (pv[t] & 31);
+                    const uint32_t old = atomicOr(&bm[warp][pv[t] >> 5], bit);
+                    is_new = !(old & bit);
+                    if (is_new && a.recv) atomicAdd(a.recv + pv[t], 1ull);
+                }
+                my_cross += cross ? 1ull : 0ull;
+                row_new += __popc(__ballot_sync(0xffffffffu, is_new));
+            }
         }
         __syncwarp();
         // clear the touched words again
