@@ -140,7 +140,7 @@ __device__ __forceinline__ void store_block_transposed(__nv_bfloat16* out_t, int
 }
 
 template <int BN, int STAGES>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 2)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcKernelArgs g) {
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t kABytes = kTcBM * kTcBK * 2, kBBytes = BN * kTcBK * 2, kStageBytes = kABytes + kBBytes;
@@ -484,9 +484,9 @@ int tc_gemm_launch(const TcGemm& t, cudaStream_t st) {
     CUtensorMap ma, mb;
     if (!make_map(&ma, t.A, t.M, t.K, t.lda, kTcBM)) return RETEXO_ERR_CUDA;
     if (!make_map(&mb, t.B, t.N, t.K, t.ldb, bn)) return RETEXO_ERR_CUDA;
-    if (bn == 256) return launch_tc<256, 4>(t, ma, mb, st);
-    if (bn == 128) return launch_tc<128, 6>(t, ma, mb, st);
-    return launch_tc<64, 8>(t, ma, mb, st);
+    if (bn == 256) return launch_tc<256, 2>(t, ma, mb, st);
+    if (bn == 128) return launch_tc<128, 3>(t, ma, mb, st);
+    return launch_tc<64, 4>(t, ma, mb, st);
 }
 
 }  // namespace retexo
