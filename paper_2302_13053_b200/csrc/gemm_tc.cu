@@ -95,6 +95,7 @@ struct TcKernelArgs {
     int64_t M, N;
     int32_t k_blocks_total;       // ceil(K / 64)
     int32_t k_blocks_per_split;
+    int32_t splits;
     int mode, relu;
     const float* bias;
     float* out_f32; int64_t ld_f32;
@@ -107,8 +108,24 @@ struct TcKernelArgs {
     int32_t* status;
 };
 
-constexpr int kStagePitch = 80;                       // bytes per column in the transpose staging (64 + 16 pad)
-constexpr int kStageBytesPerWarp = 32 * kStagePitch;
+// Per-warp staging of one 32 x 32 bf16 block: 32 lines of 64 bytes.  A line is one output row
+// (row-major store) or one output column (transposed store).  The four 16-byte pieces of a line
+// are XOR-swizzled with the line index so that both the fill (one thread per row) and the drain
+// (eight lines of 64 contiguous bytes per instruction) are free of bank conflicts.
+constexpr int kStageBytesPerWarp = 32 * 64;
+__device__ __forceinline__ int stage_piece(int line, int piece) { return piece ^ ((line >> 1) & 3); }
+
+// Drains the staged block: line L goes to dst + L * stride (elements), 64 contiguous bytes each.
+__device__ __forceinline__ void drain_stage(const uint8_t* stage, __nv_bfloat16* dst, int64_t stride, int64_t n_lines,
+                                            int lane) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int line = (lane >> 2) + 8 * i, piece = lane & 3;
+        if (line < n_lines)
+            *reinterpret_cast<uint4*>(dst + line * stride + piece * 8) =
+                *reinterpret_cast<const uint4*>(stage + line * 64 + stage_piece(line, piece) * 16);
+    }
+}
 
 // Writes a warp's 32 x 32 block (lane = row, v[j] = column col0 + j) into the transposed output
 // out_t[col][row].  Full, aligned blocks go through shared memory so that every column leaves
@@ -119,15 +136,12 @@ __device__ __forceinline__ void store_block_transposed(__nv_bfloat16* out_t, int
     const bool fast = row0 + 32 <= M && (ld_t & 7) == 0 && aligned16(out_t);
     if (fast) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-            *reinterpret_cast<__nv_bfloat16*>(stage + j * kStagePitch + lane * 2) = __float2bfloat16_rn(v[j]);
+        for (int j = 0; j < 32; ++j)      // line j = column col0 + j; this lane's row is element `lane` of the line
+            *reinterpret_cast<__nv_bfloat16*>(stage + j * 64 + stage_piece(j, lane >> 3) * 16 + (lane & 7) * 2) =
+                __float2bfloat16_rn(v[j]);
         __syncwarp();
-        if (col0 + lane < n_cols) {
-            __nv_bfloat16* dst = out_t + (col0 + lane) * ld_t + row0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-                *reinterpret_cast<uint4*>(dst + 8 * i) = *reinterpret_cast<const uint4*>(stage + lane * kStagePitch + 16 * i);
-        }
+        const int64_t n_lines = n_cols - col0 < 32 ? n_cols - col0 : 32;
+        drain_stage(stage, out_t + col0 * ld_t + row0, ld_t, n_lines, lane);
         __syncwarp();
     } else {
         const int64_t row = row0 + lane;
@@ -139,35 +153,57 @@ __device__ __forceinline__ void store_block_transposed(__nv_bfloat16* out_t, int
     }
 }
 
+// Row-major counterpart: out[row][col0 .. col0+32).  The caller guarantees a full, aligned
+// block of columns; rows beyond M are dropped.
+__device__ __forceinline__ void store_block_rows(__nv_bfloat16* out, int64_t ld, int64_t col0, int64_t row0, int64_t M,
+                                                 const float (&v)[32], uint8_t* stage, int lane) {
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {         // line = this lane's row; four 16-byte pieces of 8 columns
+        __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * p], v[8 * p + 1]), b = __floats2bfloat162_rn(v[8 * p + 2], v[8 * p + 3]);
+        __nv_bfloat162 c = __floats2bfloat162_rn(v[8 * p + 4], v[8 * p + 5]), d = __floats2bfloat162_rn(v[8 * p + 6], v[8 * p + 7]);
+        uint4 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&a); pk.y = *reinterpret_cast<uint32_t*>(&b);
+        pk.z = *reinterpret_cast<uint32_t*>(&c); pk.w = *reinterpret_cast<uint32_t*>(&d);
+        *reinterpret_cast<uint4*>(stage + lane * 64 + stage_piece(lane, p) * 16) = pk;
+    }
+    __syncwarp();
+    const int64_t n_lines = M - row0 < 32 ? M - row0 : 32;
+    drain_stage(stage, out + row0 * ld + col0, ld, n_lines, lane);
+    __syncwarp();
+}
+
 template <int BN, int STAGES>
-__global__ void __launch_bounds__(kTcThreads, 2)
+__global__ void __launch_bounds__(kTcThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcKernelArgs g) {
+    // Persistent: the block walks over output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...  The
+    // stage ring runs on across tiles and the accumulator is double-buffered in tensor memory, so
+    // the loads and MMAs of the next tile overlap the epilogue of the current one.
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t kABytes = kTcBM * kTcBK * 2, kBBytes = BN * kTcBK * 2, kStageBytes = kABytes + kBBytes;
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(tiles + STAGES * kStageBytes);
     uint64_t* empty = full + STAGES;
-    uint64_t* acc_ready = empty + STAGES;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_ready + 1);
+    uint64_t* acc_full = empty + STAGES;          // [2] accumulator b holds a finished tile
+    uint64_t* acc_empty = acc_full + 2;           // [2] accumulator b has been drained
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* warp_loss = reinterpret_cast<float*>(tmem_slot + 2);                  // [4]
     uint8_t* stage_base = reinterpret_cast<uint8_t*>(                           // 4 x kStageBytesPerWarp, 16-byte aligned
         (reinterpret_cast<uintptr_t>(tmem_slot) + 64 + 15) & ~uintptr_t(15));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t m0 = (int64_t)blockIdx.x * kTcBM, n0 = (int64_t)blockIdx.y * BN;
-    const int32_t kb0 = blockIdx.z * g.k_blocks_per_split;
-    const int32_t kb1 = min(g.k_blocks_total, kb0 + g.k_blocks_per_split);
-    const int32_t n_kb = kb1 - kb0;
+    const int64_t n_m = (g.M + kTcBM - 1) / kTcBM, n_n = (g.N + BN - 1) / BN;
+    const int64_t per_split = n_m * n_n;
+    const int64_t n_tiles = per_split * g.splits;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
-        mbar_init(acc_ready, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, 4); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {      // tensor memory: BN fp32 columns x 128 lanes
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(BN));
+    if (warp == 1) {      // tensor memory: two accumulators of BN fp32 columns x 128 lanes
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * BN));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -177,234 +213,260 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (warp == 0) {
         if (lane == 0) {
-            int issued = 0;
-            for (int i = 0; i < n_kb; ++i) {
-                const int s = i % STAGES;
-                const uint32_t ph = (i / STAGES) & 1;
-                if (!mbar_wait(empty + s, ph ^ 1, g.status, abort_flag)) break;
-                mbar_expect_tx(full + s, kStageBytes);
-                uint8_t* a_dst = tiles + s * kStageBytes;
-                tma_load_2d(a_dst, &map_a, (kb0 + i) * kTcBK, (int32_t)m0, full + s);
-                tma_load_2d(a_dst + kABytes, &map_b, (kb0 + i) * kTcBK, (int32_t)n0, full + s);
-                issued = i + 1;
+            int64_t it = 0;                       // k-blocks issued so far, over all tiles
+            bool ok = true;
+            for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+                const int64_t z = t / per_split, rem = t % per_split;
+                const int32_t m0 = (int32_t)((rem % n_m) * kTcBM), n0 = (int32_t)((rem / n_m) * BN);
+                const int32_t kb0 = (int32_t)z * g.k_blocks_per_split;
+                const int32_t kb1 = min(g.k_blocks_total, kb0 + g.k_blocks_per_split);
+                for (int32_t kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int s = (int)(it % STAGES);
+                    const uint32_t ph = (uint32_t)(it / STAGES) & 1;
+                    if (!mbar_wait(empty + s, ph ^ 1, g.status, abort_flag)) { ok = false; break; }
+                    mbar_expect_tx(full + s, kStageBytes);
+                    uint8_t* a_dst = tiles + s * kStageBytes;
+                    tma_load_2d(a_dst, &map_a, kb * kTcBK, m0, full + s);
+                    tma_load_2d(a_dst + kABytes, &map_b, kb * kTcBK, n0, full + s);
+                }
             }
             if (*abort_flag) {    // await (bounded) what was issued and not consumed, so nothing lands after exit
-                for (int i = max(0, issued - STAGES); i < issued; ++i) {
-                    const int s = i % STAGES;
-                    const uint32_t ph = (i / STAGES) & 1;
-                    for (uint32_t t = 0; t < (1u << 20); ++t) if (mbar_try_wait(full + s, ph)) break;
+                for (int64_t i = it > STAGES ? it - STAGES : 0; i < it; ++i) {
+                    const int s = (int)(i % STAGES);
+                    const uint32_t ph = (uint32_t)(i / STAGES) & 1;
+                    for (uint32_t w = 0; w < (1u << 20); ++w) if (mbar_try_wait(full + s, ph)) break;
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc(BN);
+            int64_t it = 0, lt = 0;               // k-blocks consumed, tiles done by this block
             bool ok = true;
-            for (int i = 0; i < n_kb && ok; ++i) {
-                const int s = i % STAGES;
-                const uint32_t ph = (i / STAGES) & 1;
-                ok = mbar_wait(full + s, ph, g.status, abort_flag);
+            for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++lt) {
+                const int64_t z = t / per_split;
+                const int32_t kb0 = (int32_t)z * g.k_blocks_per_split;
+                const int32_t kb1 = min(g.k_blocks_total, kb0 + g.k_blocks_per_split);
+                const int b = (int)(lt & 1);
+                const uint32_t pb = (uint32_t)(lt >> 1) & 1;
+                ok = mbar_wait(acc_empty + b, pb ^ 1, g.status, abort_flag);      // drained by the epilogue
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t a_addr = smem_u32(tiles + s * kStageBytes);
-                const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(a_addr + kABytes);
+                const uint32_t acc_addr = tmem_acc + (uint32_t)(b * BN);
+                for (int32_t kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int s = (int)(it % STAGES);
+                    const uint32_t ph = (uint32_t)(it / STAGES) & 1;
+                    ok = mbar_wait(full + s, ph, g.status, abort_flag);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t a_addr = smem_u32(tiles + s * kStageBytes);
+                    const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(a_addr + kABytes);
 #pragma unroll
-                for (int k = 0; k < kTcBK / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K: +2 in 16-byte units
-                    umma_bf16(tmem_acc, adesc + 2 * k, bdesc + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
-                umma_commit(empty + s);                   // frees the stage once these MMAs have read it
+                    for (int k = 0; k < kTcBK / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K: +2 in 16-byte units
+                        umma_bf16(acc_addr, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                    umma_commit(empty + s);                   // frees the stage once these MMAs have read it
+                }
+                if (ok) umma_commit(acc_full + b);            // accumulator complete (at once for an empty K range)
             }
-            if (ok) umma_commit(acc_ready);               // accumulator complete
         }
     } else {
         const int q = warp & 3;                           // tensor-memory lane quarter this warp may read
-        const int64_t row0 = m0 + q * 32;
-        const int64_t row = row0 + lane;
         uint8_t* stage = stage_base + q * kStageBytesPerWarp;
-        bool ok = n_kb > 0 ? mbar_wait(acc_ready, 0, g.status, abort_flag) : true;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (BN == 64 && (g.mode == TC_EPI_SOFTMAX_CE || g.mode == TC_EPI_ARGMAX)) {
-            // the thread owns the whole row of logits
-            float v[64];
-            if (ok) {
+        int64_t lt = 0;
+        for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++lt) {
+            const int64_t z = t / per_split, rem = t % per_split;
+            const int64_t mt = rem % n_m;
+            const int64_t m0 = mt * kTcBM, n0 = (rem / n_m) * BN;
+            const int32_t kb0 = (int32_t)z * g.k_blocks_per_split;
+            const int32_t n_kb = min(g.k_blocks_total, kb0 + g.k_blocks_per_split) - kb0;
+            const int b = (int)(lt & 1);
+            const uint32_t pb = (uint32_t)(lt >> 1) & 1;
+            const uint32_t acc_addr = tmem_acc + (uint32_t)(b * BN);
+            const int64_t row0 = m0 + q * 32;
+            const int64_t row = row0 + lane;
+            const bool ok = mbar_wait(acc_full + b, pb, g.status, abort_flag);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            if (!ok) break;
+            if (BN == 64 && (g.mode == TC_EPI_SOFTMAX_CE || g.mode == TC_EPI_ARGMAX)) {
+                // the thread owns the whole row of logits
+                float v[64];
+                if (ok) {
 #pragma unroll
-                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    for (int c0 = 0; c0 < 64; c0 += 32) {
+                        uint32_t r[32];
+                        if (n_kb > 0) tmem_ld_32cols(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                        else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) r[j] = 0u;
+                        }
+                        const float bias_lane = (g.bias && c0 + lane < g.N) ? __ldg(g.bias + c0 + lane) : 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int c = c0 + j;
+                            v[c] = c < g.N ? __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j) : -INFINITY;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) v[c] = 0.f;
+                }
+                const bool live = ok && row < g.M;
+                const int32_t yi = (live && g.y) ? g.y[row] : -1;
+                if (g.mode == TC_EPI_ARGMAX) {
+                    int best = 0;
+                    float bv = v[0];
+#pragma unroll
+                    for (int c = 1; c < 64; ++c) if (v[c] > bv) { bv = v[c]; best = c; }   // strict: lowest index wins ties
+                    if (live) {
+                        if (g.pred) g.pred[row] = best;
+                        if (g.out_f32) {
+#pragma unroll
+                            for (int c = 0; c < 64; ++c) if (c < g.N) g.out_f32[row * g.ld_f32 + c] = v[c];
+                        }
+                    }
+                    if (g.correct) {
+                        const unsigned hits = __ballot_sync(0xffffffffu, live && best == yi);
+                        if (lane == 0 && hits) atomicAdd(g.correct, (unsigned long long)__popc(hits));
+                    }
+                } else {
+                    float mx = v[0];
+#pragma unroll
+                    for (int c = 1; c < 64; ++c) mx = fmaxf(mx, v[c]);
+                    float den = 0.f, ly = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) {
+                        ly = c == yi ? v[c] : ly;
+                        v[c] = c < g.N ? expf(v[c] - mx) : 0.f;
+                        den += v[c];
+                    }
+                    float loss = live ? (mx + logf(den)) - ly : 0.f;
+                    const float scale = g.inv_rows / den;
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) v[c] = c < g.N ? (v[c] * scale - (c == yi ? g.inv_rows : 0.f)) : 0.f;
+                    if (live && g.out_bf16) {       // dL row-major, ld_bf16 <= 64 and a multiple of 8
+                        __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16;
+#pragma unroll
+                        for (int c = 0; c < 64; c += 8) {
+                            if (c >= g.ld_bf16) break;
+                            __nv_bfloat162 p0 = __floats2bfloat162_rn(v[c], v[c + 1]), p1 = __floats2bfloat162_rn(v[c + 2], v[c + 3]);
+                            __nv_bfloat162 p2 = __floats2bfloat162_rn(v[c + 4], v[c + 5]), p3 = __floats2bfloat162_rn(v[c + 6], v[c + 7]);
+                            uint4 pk;
+                            pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                            pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                            *reinterpret_cast<uint4*>(dst + c) = pk;
+                        }
+                    }
+                    if (ok && g.out_bf16_t) {
+#pragma unroll
+                        for (int c0 = 0; c0 < 64; c0 += 32) {
+                            if (c0 >= g.N) break;
+                            float blk[32];
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) blk[j] = v[c0 + j];
+                            store_block_transposed(g.out_bf16_t, g.ld_t, c0, g.N, row0, g.M, blk, stage, lane);
+                        }
+                    }
+                    loss = warp_sum(loss);
+                    if (lane == 0) warp_loss[q] = loss;
+                    asm volatile("bar.sync 1, 128;" ::: "memory");      // the four epilogue warps only
+                    if (q == 0 && lane == 0 && g.loss_partial)
+                        g.loss_partial[mt] = ((warp_loss[0] + warp_loss[1]) + warp_loss[2]) + warp_loss[3];
+                    asm volatile("bar.sync 1, 128;" ::: "memory");      // warp_loss is reused by the next tile
+                }
+            } else if (ok) {
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
                     uint32_t r[32];
-                    if (n_kb > 0) tmem_ld_32cols(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                    if (n_kb > 0) tmem_ld_32cols(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
                     else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j) r[j] = 0u;
                     }
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int c = c0 + j;
-                        v[c] = c < g.N ? __uint_as_float(r[j]) + (g.bias ? __ldg(g.bias + c) : 0.f) : -INFINITY;
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int c = 0; c < 64; ++c) v[c] = 0.f;
-            }
-            const bool live = ok && row < g.M;
-            const int32_t yi = (live && g.y) ? g.y[row] : -1;
-            if (g.mode == TC_EPI_ARGMAX) {
-                int best = 0;
-                float bv = v[0];
-#pragma unroll
-                for (int c = 1; c < 64; ++c) if (v[c] > bv) { bv = v[c]; best = c; }   // strict: lowest index wins ties
-                if (live) {
-                    if (g.pred) g.pred[row] = best;
-                    if (g.out_f32) {
-#pragma unroll
-                        for (int c = 0; c < 64; ++c) if (c < g.N) g.out_f32[row * g.ld_f32 + c] = v[c];
-                    }
-                }
-                if (g.correct) {
-                    const unsigned hits = __ballot_sync(0xffffffffu, live && best == yi);
-                    if (lane == 0 && hits) atomicAdd(g.correct, (unsigned long long)__popc(hits));
-                }
-            } else {
-                float mx = v[0];
-#pragma unroll
-                for (int c = 1; c < 64; ++c) mx = fmaxf(mx, v[c]);
-                float den = 0.f, ly = 0.f;
-#pragma unroll
-                for (int c = 0; c < 64; ++c) {
-                    ly = c == yi ? v[c] : ly;
-                    v[c] = c < g.N ? expf(v[c] - mx) : 0.f;
-                    den += v[c];
-                }
-                float loss = live ? (mx + logf(den)) - ly : 0.f;
-                const float scale = g.inv_rows / den;
-#pragma unroll
-                for (int c = 0; c < 64; ++c) v[c] = c < g.N ? (v[c] * scale - (c == yi ? g.inv_rows : 0.f)) : 0.f;
-                if (live && g.out_bf16) {       // dL row-major, ld_bf16 <= 64 and a multiple of 8
-                    __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16;
-#pragma unroll
-                    for (int c = 0; c < 64; c += 8) {
-                        if (c >= g.ld_bf16) break;
-                        __nv_bfloat162 p0 = __floats2bfloat162_rn(v[c], v[c + 1]), p1 = __floats2bfloat162_rn(v[c + 2], v[c + 3]);
-                        __nv_bfloat162 p2 = __floats2bfloat162_rn(v[c + 4], v[c + 5]), p3 = __floats2bfloat162_rn(v[c + 6], v[c + 7]);
-                        uint4 pk;
-                        pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-                        pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-                        *reinterpret_cast<uint4*>(dst + c) = pk;
-                    }
-                }
-                if (ok && g.out_bf16_t) {
-#pragma unroll
-                    for (int c0 = 0; c0 < 64; c0 += 32) {
-                        if (c0 >= g.N) break;
-                        float blk[32];
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) blk[j] = v[c0 + j];
-                        store_block_transposed(g.out_bf16_t, g.ld_t, c0, g.N, row0, g.M, blk, stage, lane);
-                    }
-                }
-                loss = warp_sum(loss);
-                if (lane == 0) warp_loss[q] = loss;
-                asm volatile("bar.sync 1, 128;" ::: "memory");      // the four epilogue warps only
-                if (q == 0 && lane == 0 && g.loss_partial)
-                    g.loss_partial[blockIdx.x] = ((warp_loss[0] + warp_loss[1]) + warp_loss[2]) + warp_loss[3];
-            }
-        } else if (ok) {
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                uint32_t r[32];
-                if (n_kb > 0) tmem_ld_32cols(tmem_acc + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-                else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = 0u;
-                }
-                const int64_t col0 = n0 + c0;
-                if (col0 >= g.N) continue;
-                if (g.mode == TC_EPI_PARTIAL) {
-                    if (row >= g.M) continue;
-                    float* dst = g.partial + ((int64_t)blockIdx.z * g.M + row) * g.N + col0;
-                    if (col0 + 32 <= g.N && (g.N & 3) == 0 && aligned16(g.partial)) {
-#pragma unroll
-                        for (int j = 0; j < 32; j += 4)
-                            *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
-                                                                              __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __uint_as_float(r[j]);
-                    }
-                } else if (g.mode == TC_EPI_MASK_T) {
-                    float v[32];
-                    if (row < g.M) {
-                        const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
-                        if (col0 + 32 <= g.N && (g.ld_mask & 7) == 0 && aligned16(g.mask)) {
-#pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
-                                const uint4 pk = *reinterpret_cast<const uint4*>(mrow + j);
-                                const __nv_bfloat16* mv = reinterpret_cast<const __nv_bfloat16*>(&pk);
-#pragma unroll
-                                for (int k = 0; k < 8; ++k)
-                                    v[j + k] = __bfloat162float(mv[k]) > 0.f ? __uint_as_float(r[j + k]) : 0.f;
-                            }
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                v[j] = (col0 + j < g.N && __bfloat162float(mrow[j]) > 0.f) ? __uint_as_float(r[j]) : 0.f;
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) v[j] = 0.f;
-                    }
-                    store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane);
-                } else {
-                    float v[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float x = __uint_as_float(r[j]);
-                        if (g.bias && col0 + j < g.N) x += __ldg(g.bias + col0 + j);
-                        if (g.relu) x = fmaxf(x, 0.f);
-                        v[j] = x;
-                    }
-                    if (g.out_bf16_t) {
-                        store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane);
-                        if (g.ones_row_t && col0 == 0 && row < g.M) g.out_bf16_t[g.N * g.ld_t + row] = __float2bfloat16_rn(1.0f);
-                    }
-                    if (row >= g.M) continue;
-                    if (g.out_f32) {
-                        float* dst = g.out_f32 + row * g.ld_f32 + col0;
-                        if (col0 + 32 <= g.N && (g.ld_f32 & 3) == 0 && aligned16(g.out_f32)) {
+                    const int64_t col0 = n0 + c0;
+                    if (col0 >= g.N) continue;
+                    if (g.mode == TC_EPI_PARTIAL) {
+                        if (row >= g.M) continue;
+                        float* dst = g.partial + ((int64_t)z * g.M + row) * g.N + col0;
+                        if (col0 + 32 <= g.N && (g.N & 3) == 0 && aligned16(g.partial)) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 4)
-                                *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                                *reinterpret_cast<float4*>(dst + j) = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]),
+                                                                                  __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
                         } else {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = v[j];
+                            for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __uint_as_float(r[j]);
                         }
-                    }
-                    if (g.out_bf16) {
-                        __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16 + col0;
-                        if (col0 + 32 <= g.N && (g.ld_bf16 & 7) == 0 && aligned16(g.out_bf16)) {
+                    } else if (g.mode == TC_EPI_MASK_T) {
+                        float v[32];
+                        if (row < g.M) {
+                            const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
+                            if (col0 + 32 <= g.N && (g.ld_mask & 7) == 0 && aligned16(g.mask)) {
 #pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
-                                __nv_bfloat162 p0 = __floats2bfloat162_rn(v[j], v[j + 1]);
-                                __nv_bfloat162 p1 = __floats2bfloat162_rn(v[j + 2], v[j + 3]);
-                                __nv_bfloat162 p2 = __floats2bfloat162_rn(v[j + 4], v[j + 5]);
-                                __nv_bfloat162 p3 = __floats2bfloat162_rn(v[j + 6], v[j + 7]);
-                                uint4 pk;
-                                pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-                                pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-                                *reinterpret_cast<uint4*>(dst + j) = pk;
+                                for (int j = 0; j < 32; j += 8) {
+                                    const uint4 pk = *reinterpret_cast<const uint4*>(mrow + j);
+                                    const __nv_bfloat16* mv = reinterpret_cast<const __nv_bfloat16*>(&pk);
+#pragma unroll
+                                    for (int k = 0; k < 8; ++k)
+                                        v[j + k] = __bfloat162float(mv[k]) > 0.f ? __uint_as_float(r[j + k]) : 0.f;
+                                }
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    v[j] = (col0 + j < g.N && __bfloat162float(mrow[j]) > 0.f) ? __uint_as_float(r[j]) : 0.f;
                             }
                         } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                        }
+                        store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane);
+                    } else {
+                        float v[32];
+                        // one coalesced bias load per chunk, handed round by shuffles (32 same-address loads per
+                        // thread cost more than the rest of the epilogue together)
+                        const float bias_lane = (g.bias && col0 + lane < g.N) ? __ldg(g.bias + col0 + lane) : 0.f;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            float x = __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j);
+                            if (g.relu) x = fmaxf(x, 0.f);
+                            v[j] = x;
+                        }
+                        if (g.out_bf16_t) {
+                            store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane);
+                            if (g.ones_row_t && col0 == 0 && row < g.M) g.out_bf16_t[g.N * g.ld_t + row] = __float2bfloat16_rn(1.0f);
+                        }
+                        const bool rows_fast = g.out_bf16 && col0 + 32 <= g.N && (g.ld_bf16 & 7) == 0 && aligned16(g.out_bf16);
+                        if (rows_fast) store_block_rows(g.out_bf16, g.ld_bf16, col0, row0, g.M, v, stage, lane);
+                        if (row >= g.M) continue;
+                        if (g.out_f32) {
+                            float* dst = g.out_f32 + row * g.ld_f32 + col0;
+                            if (col0 + 32 <= g.N && (g.ld_f32 & 3) == 0 && aligned16(g.out_f32)) {
+#pragma unroll
+                                for (int j = 0; j < 32; j += 4)
+                                    *reinterpret_cast<float4*>(dst + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = v[j];
+                            }
+                        }
+                        if (g.out_bf16 && !rows_fast) {
+                            __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16 + col0;
 #pragma unroll
                             for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __float2bfloat16_rn(v[j]);
                         }
                     }
                 }
             }
+            // hand the accumulator back to the MMA thread
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(acc_empty + b)) : "memory");
         }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(BN));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(2 * BN));
     }
 }
 
@@ -455,13 +517,17 @@ static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& 
     g.k_blocks_total = (int32_t)((t.K + kTcBK - 1) / kTcBK);
     const int splits = t.mode == TC_EPI_PARTIAL ? (t.splits > 0 ? t.splits : 1) : 1;
     g.k_blocks_per_split = (g.k_blocks_total + splits - 1) / splits;
+    g.splits = splits;
     g.mode = t.mode; g.relu = t.relu; g.bias = t.bias;
     g.out_f32 = t.out_f32; g.ld_f32 = t.ld_f32; g.out_bf16 = t.out_bf16; g.ld_bf16 = t.ld_bf16;
     g.out_bf16_t = t.out_bf16_t; g.ld_t = t.ld_t; g.ones_row_t = t.ones_row_t;
     g.mask = t.mask; g.ld_mask = t.ld_mask;
     g.partial = t.partial; g.status = t.status;
     g.y = t.y; g.inv_rows = t.inv_rows; g.loss_partial = t.loss_partial; g.pred = t.pred; g.correct = t.correct;
-    dim3 grid((unsigned)((t.M + kTcBM - 1) / kTcBM), (unsigned)((t.N + BN - 1) / BN), (unsigned)splits);
+    const int64_t n_tiles = ((t.M + kTcBM - 1) / kTcBM) * ((t.N + BN - 1) / BN) * splits;
+    const int n_sm = sm_count();
+    if (n_sm <= 0) return RETEXO_ERR_CUDA;
+    const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);      // one persistent block per SM
     tc_gemm_kernel<BN, STAGES><<<grid, kTcThreads, smem, st>>>(ma, mb, g);
     return launch_status();
 }
@@ -484,9 +550,9 @@ int tc_gemm_launch(const TcGemm& t, cudaStream_t st) {
     CUtensorMap ma, mb;
     if (!make_map(&ma, t.A, t.M, t.K, t.lda, kTcBM)) return RETEXO_ERR_CUDA;
     if (!make_map(&mb, t.B, t.N, t.K, t.ldb, bn)) return RETEXO_ERR_CUDA;
-    if (bn == 256) return launch_tc<256, 2>(t, ma, mb, st);
-    if (bn == 128) return launch_tc<128, 3>(t, ma, mb, st);
-    return launch_tc<64, 4>(t, ma, mb, st);
+    if (bn == 256) return launch_tc<256, 4>(t, ma, mb, st);
+    if (bn == 128) return launch_tc<128, 6>(t, ma, mb, st);
+    return launch_tc<64, 8>(t, ma, mb, st);
 }
 
 }  // namespace retexo
