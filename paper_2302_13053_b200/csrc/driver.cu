@@ -327,14 +327,19 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         best.theta = b.theta_best;
 
         // ---- R training iterations; validation and best-iterate tracking stay on the device
+        const MlpPlan plan = make_plan(r.d_in, r.hidden, c.n_classes, n_tr);
+        MlpBuffers sb{};
+        mlp_step_buffers(plan, b.ws_step, b.ws_step_bytes, &sb);
+        bf16* val_hd = reinterpret_cast<bf16*>(b.ws_embed);      // [n_val x ld_h] scratch of the validation forward
         for (int it = 1; it <= c.R; ++it) {
             float* loss_slot = b.loss_history + (size_t)(m - 1) * c.R + (it - 1);
-            RETEXO_TRY(retexo_mlp_train_step(&model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, n_tr, loss_slot, nullptr,
-                                             b.ws_step, b.ws_step_bytes, st));
+            // the update of iteration it-1 left bf16 copies of the current weights behind
+            RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, loss_slot,
+                                             nullptr, it > 1, st));
+            model.step += 1;
             if (n_val && (it % c.eval_every == 0 || it == c.R)) {
-                RETEXO_TRY(retexo_embed(&model, b.xval16, ld16, nullptr, n_val, nullptr, 0, nullptr, 0, nullptr, 0,
-                                        nullptr, b.y_val, reinterpret_cast<uint64_t*>(b.cur_correct), b.ws_embed,
-                                        b.ws_embed_bytes, st));
+                RETEXO_TRY(mlp_count_hits_launch(plan, sb, &model, b.xval16, ld16, n_val, val_hd, b.y_val,
+                                                 b.cur_correct, st));
                 snapshot_if_better_kernel<<<(unsigned)((nt + 255) / 256), 256, 0, st>>>(
                     b.cur_correct, b.best_correct, b.have_best, b.theta, b.theta_best, nt);
                 record_validation_kernel<<<1, 32, 0, st>>>(b.cur_correct, b.best_correct, b.have_best, it,

@@ -90,6 +90,11 @@ static void layout(const MlpPlan& p, Taker& t, MlpBuffers* out) {
     if (out) *out = b;
 }
 
+void mlp_step_buffers(const MlpPlan& p, void* workspace, size_t bytes, MlpBuffers* out) {
+    Arena ws(workspace, bytes);
+    layout(p, ws, out);
+}
+
 struct NullTaker {
     Sizer s;
     template <typename T> T* take(size_t count) { s.take<T>(count); return nullptr; }
@@ -177,7 +182,7 @@ extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t l
     MlpBuffers b{};
     layout(p, ws, &b);
     RETEXO_TRY(mlp_train_step_launch(p, b, model, static_cast<const bf16*>(x), ldx,
-                                     static_cast<const bf16*>(x_t), ld_xt, y, loss_out, grad_out, st));
+                                     static_cast<const bf16*>(x_t), ld_xt, y, loss_out, grad_out, false, st));
     model->step += 1;
     return RETEXO_OK;
 }
@@ -188,14 +193,14 @@ namespace retexo {
 // already applied.
 int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
                           const bf16* x, int64_t ldx, const bf16* x_t, int64_t ld_xt, const int32_t* y,
-                          float* loss_out, float* grad_out, cudaStream_t st) {
+                          float* loss_out, float* grad_out, bool shadows_ready, cudaStream_t st) {
     const int64_t n = p.n_rows;
     const int32_t d_in = p.d_in, H = p.hidden, O = p.n_classes, out1 = p.out1;
     const float* theta = model->theta;
     const float* b1 = theta + (int64_t)d_in * out1;
     const float* b2 = b1 + out1 + (int64_t)H * O;
     RETEXO_CUDA_TRY(cudaMemsetAsync(b.status, 0, sizeof(int32_t), st));
-    RETEXO_TRY(build_weight_shadows(p, b, theta, st));
+    if (!shadows_ready) RETEXO_TRY(build_weight_shadows(p, b, theta, st));
     if (!x_t) {      // no transposed batch from the caller: build [X^T ; 1] here (one more pass over X per call)
         RETEXO_TRY(retexo_pack_rows(x, 1, ldx, d_in, nullptr, n, nullptr, 0, b.xt16, p.ld_n, 1, st));
         x_t = b.xt16;
@@ -246,8 +251,31 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     u.corr2 = (float)(1.0 - pow((double)model->beta2, t));
     u.loss_partial = b.loss_partial; u.n_loss = p.sm_blocks; u.inv_rows = 1.0f / (float)n; u.loss_out = loss_out;
     u.status = b.status;
+    u.w1t16 = b.w1t16; u.ld_k = p.ld_k; u.w2t16 = H > 0 ? b.w2t16 : nullptr; u.ld_h = p.ld_h;
+    u.w2p16 = H > 0 ? b.w2p16 : nullptr; u.ld_dl = p.ld_dl;
+    u.d_in = d_in; u.out1 = out1; u.hidden = H; u.n_classes = O;
     reduce_update_kernel<<<(unsigned)((p.nt + 255) / 256), 256, 0, st>>>(u);
     return launch_status();
+}
+
+int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model, const bf16* x, int64_t ldx,
+                          int64_t n_rows, bf16* hd_ws, const int32_t* y, unsigned long long* correct, cudaStream_t st) {
+    const int32_t d_in = p.d_in, H = p.hidden, O = p.n_classes, out1 = p.out1;
+    const float* b1 = model->theta + (int64_t)d_in * out1;
+    const float* b2 = b1 + out1 + (int64_t)H * O;
+    RETEXO_CUDA_TRY(cudaMemsetAsync(correct, 0, sizeof(unsigned long long), st));
+    if (n_rows == 0) return RETEXO_OK;
+    TcGemm fwd = tc_base(x, ldx, b.w1t16, p.ld_k, n_rows, out1, d_in, b.status);
+    fwd.bias = b1;
+    if (H > 0) {
+        fwd.relu = 1; fwd.out_bf16 = hd_ws; fwd.ld_bf16 = p.ld_h;
+        RETEXO_TRY(tc_gemm_launch(fwd, st));
+        TcGemm l2 = tc_base(hd_ws, p.ld_h, b.w2t16, p.ld_h, n_rows, O, H, b.status);
+        l2.bias = b2; l2.mode = TC_EPI_ARGMAX; l2.y = y; l2.correct = correct;
+        return tc_gemm_launch(l2, st);
+    }
+    fwd.mode = TC_EPI_ARGMAX; fwd.y = y; fwd.correct = correct;
+    return tc_gemm_launch(fwd, st);
 }
 
 }  // namespace retexo

@@ -203,7 +203,7 @@ struct GradSeg {
     int64_t count;
 };
 struct UpdateArgs {
-    GradSeg seg[2];
+    GradSeg seg[2];            // [W1 | b1] and (hidden > 0) [W2 | b2], each laid out like theta
     int n_seg;
     float* theta;
     float* m;
@@ -213,34 +213,61 @@ struct UpdateArgs {
     float lr, beta1, beta2, eps, corr1, corr2;     // corr = 1 - beta^step
     const float* loss_partial; int64_t n_loss; float inv_rows; float* loss_out;
     const int32_t* status;     // non-zero: a kernel of this step gave up on a bounded wait -> loss = NaN
+    // bf16 copies of the updated weights in the orientations the next products read (optional)
+    bf16* w1t16; int64_t ld_k;       // W1^T [out1 x ld_k]
+    bf16* w2t16; int64_t ld_h;       // W2^T [n_classes x ld_h]
+    bf16* w2p16; int64_t ld_dl;      // W2   [hidden x ld_dl]
+    int32_t d_in, out1, hidden, n_classes;
 };
 
+// Sums each parameter's split-K partials in index order, applies the optimiser, and refreshes
+// the bf16 weight copies.  Block 0 also reduces the loss (fixed order: per-lane strided sums,
+// then a shuffle tree).
 __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     const int64_t p = blockIdx.x * 256ll + threadIdx.x;
-    if (p == 0 && u.loss_out) {
+    if (blockIdx.x == 0 && threadIdx.x < 32 && u.loss_out) {
         float s = 0.f;
-        for (int64_t i = 0; i < u.n_loss; ++i) s += u.loss_partial[i];
-        *u.loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
+        for (int64_t i = threadIdx.x; i < u.n_loss; i += 32) s += u.loss_partial[i];
+        s = warp_sum(s);
+        if (threadIdx.x == 0) *u.loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
     }
-    int64_t off = 0;
-    for (int s = 0; s < u.n_seg; ++s) {
-        if (p < off + u.seg[s].size) {
-            const int64_t q = p - off;
-            float g = 0.f;
-            for (int64_t z = 0; z < u.seg[s].count; ++z) g += u.seg[s].partial[z * u.seg[s].size + q];
-            if (u.grad_out) u.grad_out[p] = g;
-            if (u.optimizer == RETEXO_SGD) {
-                u.theta[p] -= u.lr * g;
-            } else {
-                const float m = u.beta1 * u.m[p] + (1.f - u.beta1) * g;
-                const float v = u.beta2 * u.v[p] + (1.f - u.beta2) * g * g;
-                u.m[p] = m;
-                u.v[p] = v;
-                u.theta[p] -= u.lr * (m / u.corr1) / (sqrtf(v / u.corr2) + u.eps);
-            }
-            return;
+    const int64_t size0 = u.seg[0].size;
+    const int sidx = p < size0 ? 0 : 1;
+    if (sidx >= u.n_seg) return;
+    const int64_t q = sidx == 0 ? p : p - size0;
+    const int64_t size = sidx == 0 ? size0 : u.seg[1].size;
+    if (q >= size) return;
+    const float* part = sidx == 0 ? u.seg[0].partial : u.seg[1].partial;
+    const int64_t count = sidx == 0 ? u.seg[0].count : u.seg[1].count;
+    float g = 0.f;
+    int64_t z = 0;
+    for (; z + 4 <= count; z += 4) {          // loads issued together, added in index order
+        const float a = part[z * size + q], b = part[(z + 1) * size + q];
+        const float c = part[(z + 2) * size + q], d = part[(z + 3) * size + q];
+        g += a; g += b; g += c; g += d;
+    }
+    for (; z < count; ++z) g += part[z * size + q];
+    if (u.grad_out) u.grad_out[p] = g;
+    float t;
+    if (u.optimizer == RETEXO_SGD) {
+        t = u.theta[p] - u.lr * g;
+    } else {
+        const float m = u.beta1 * u.m[p] + (1.f - u.beta1) * g;
+        const float v = u.beta2 * u.v[p] + (1.f - u.beta2) * g * g;
+        u.m[p] = m;
+        u.v[p] = v;
+        t = u.theta[p] - u.lr * (m / u.corr1) / (sqrtf(v / u.corr2) + u.eps);
+    }
+    u.theta[p] = t;
+    if (sidx == 0) {
+        if (u.w1t16 && q < (int64_t)u.d_in * u.out1) {
+            const int64_t k = q / u.out1, j = q % u.out1;
+            u.w1t16[j * u.ld_k + k] = f32_to_bf16(t);
         }
-        off += u.seg[s].size;
+    } else if (q < (int64_t)u.hidden * u.n_classes) {
+        const int64_t jh = q / u.n_classes, c = q % u.n_classes;
+        if (u.w2t16) u.w2t16[c * u.ld_h + jh] = f32_to_bf16(t);
+        if (u.w2p16) u.w2p16[jh * u.ld_dl + c] = f32_to_bf16(t);
     }
 }
 

@@ -42,9 +42,21 @@ struct MlpBuffers {
 
 MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows);
 
+// Lays the step's scratch buffers out over a workspace of retexo_mlp_train_step_workspace_size bytes.
+void mlp_step_buffers(const MlpPlan& p, void* workspace, size_t bytes, MlpBuffers* out);
+
+// One training iteration.  shadows_ready: the bf16 weight copies in `b` already hold the
+// current theta (the previous iteration's update refreshed them), so they are not rebuilt.
+// On return they hold the updated theta.
 int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
                           const __nv_bfloat16* x, int64_t ldx, const __nv_bfloat16* x_t, int64_t ld_xt,
-                          const int32_t* y, float* loss_out, float* grad_out, cudaStream_t st);
+                          const int32_t* y, float* loss_out, float* grad_out, bool shadows_ready, cudaStream_t st);
+
+// Forward + arg-max + hit count over a dense batch with the weight copies in `b` (which must
+// hold model->theta): what validation needs after every iteration.  hd_ws: bf16 [n_rows x p.ld_h].
+int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
+                          const __nv_bfloat16* x, int64_t ldx, int64_t n_rows, __nv_bfloat16* hd_ws,
+                          const int32_t* y, unsigned long long* correct, cudaStream_t st);
 
 // out[M x N] (fp32, row stride ld_out) = A[M x K] (bf16) * B[K x N] (bf16), no bias.
 int project_rows_launch(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb, int64_t M, int64_t N,
