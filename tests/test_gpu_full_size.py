@@ -1,0 +1,123 @@
+"""Parity at the full sizes of the two large configurations, in the launch configuration the
+benchmark times (128-byte feature rows, bf16 model input written by the aggregation kernel,
+transposed train batch with its row of ones): outputs the CPU checker can compute one by one
+are sampled (destination rows incl. the longest ones; one whole training iteration), counts
+are compared exactly."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2302_13053_b200 import workloads as wl
+from gpu_util import assert_rows_close, dev
+
+pytestmark = pytest.mark.gpu
+
+_cache = {}
+
+
+def config(idx):
+    if idx not in _cache:
+        _cache.clear()                      # one large graph in host memory at a time
+        _cache[idx] = wl.make_config(idx)
+    return _cache[idx]
+
+
+def sampled_rows(w, k=256):
+    deg = np.diff(w.rowptr)
+    rng = np.random.default_rng(1)
+    rows = np.concatenate([np.argsort(deg)[-24:], np.argsort(deg)[:8], rng.choice(w.n_nodes, k, replace=False)])
+    return np.unique(rows)
+
+
+@pytest.mark.parametrize("idx", [4, 5])
+def test_round_one_aggregation_on_sampled_rows(idx):
+    from paper_2302_13053_b200 import binding as B
+    w = config(idx)
+    n, d = w.n_nodes, w.d0
+    ld = (d + 31) // 32 * 32
+    q = torch.zeros((n, ld), dtype=torch.float32, device="cuda")
+    q[:, :d] = dev(w.features)
+    rp, ci = dev(w.rowptr), dev(w.colidx)
+    assert B.retexo_validate_csr(rp, ci) == (0, -1)
+    out, out16 = B.retexo_aggregate(w.aggr, rp, ci, q, dim=d, want_f32=True, want_bf16=True)
+    torch.cuda.synchronize()
+    rows = sampled_rows(w)
+    ref = oracle.aggregate(w.aggr, w.rowptr, w.colidx, w.features, rows=rows)
+    got = out[torch.from_numpy(rows).cuda()].cpu().numpy()
+    assert_rows_close(got, ref, what=w.name)
+    width = ref.shape[1]
+    assert torch.equal(out16[:, :width], out.to(torch.bfloat16))          # the bf16 copy is the same result rounded once
+    # linearity of the aggregation as a whole-matrix property: A(2q) == 2 A(q) bit for bit
+    out2, _ = B.retexo_aggregate(w.aggr, rp, ci, q * 2, dim=d)
+    assert torch.equal(out2, out * 2)
+
+
+@pytest.mark.parametrize("idx", [4, 5])
+def test_cross_partition_counts_exact(idx):
+    from paper_2302_13053_b200 import binding as B
+    w = config(idx)
+    dims = [r["rep_dim"] for r in w.round_dims()]
+    ref = oracle.cross_partition(w.rowptr, w.colidx, w.part, w.n_parts, dims, 4)
+    got = B.retexo_cross_partition_bytes(dev(w.rowptr), dev(w.colidx), dev(w.part), w.n_parts, dims, 4)
+    for k in ("cross_edges", "boundary_pairs", "bytes_total", "dv_lazy_lt"):
+        assert got[k] == ref[k], k
+    np.testing.assert_array_equal(got["bytes_per_round"], ref["bytes_per_round"])
+    np.testing.assert_array_equal(got["send_per_part"], ref["send_per_part"])
+    np.testing.assert_array_equal(got["recv_per_part"], ref["recv_per_part"])
+    if w.n_parts == w.n_nodes:
+        assert got["boundary_pairs"] == w.n_edges           # node-level partition: every edge is a message
+
+
+def test_one_training_iteration_of_the_reddit_shaped_round_one():
+    from paper_2302_13053_b200 import binding as B
+    w = config(4)
+    n, d = w.n_nodes, w.d0
+    ld = (d + 31) // 32 * 32
+    q = torch.zeros((n, ld), dtype=torch.float32, device="cuda")
+    q[:, :d] = dev(w.features)
+    _, x16 = B.retexo_aggregate(w.aggr, dev(w.rowptr), dev(w.colidx), q, dim=d, want_f32=False, want_bf16=True)
+    tr = dev(w.train_idx)
+    xtr, xtr_t = B.retexo_pack_rows(x16, tr, dim=2 * d, transpose=True, ones_row=True)
+    y = w.labels[w.train_idx]
+    wt = wl.initial_weights(w)[0]
+    gpu = B.Mlp(2 * d, w.hidden, w.n_classes, wt["w1"], wt["b1"], wt["w2"], wt["b2"], lr=w.lr)
+    ref = oracle.Mlp(2 * d, w.hidden, w.n_classes, wt["w1"], wt["b1"], wt["w2"], wt["b2"], lr=w.lr, round_bf16=True)
+    x_host = xtr[:, :2 * d].float().cpu().numpy()           # the checker sees the very batch the GPU trains on
+    given = ref.copy()
+    rl, rg = ref.train_step(x_host, y, return_grad=True)
+    gl, gg = B.retexo_mlp_train_step(gpu, xtr, dev(y), x_t=xtr_t, return_grad=True)
+    assert abs(gl.item() - rl) <= 2e-4 * max(1.0, abs(rl)), (gl.item(), rl)
+    gg = gg.cpu().numpy().astype(np.float64)
+    err, scale = np.abs(gg - rg), np.abs(rg).max()
+    assert err.max() <= 5e-3 * scale + 1e-7, (err.max(), scale)
+    assert np.median(err) <= 2e-5 * scale
+    given.apply_update(gg)
+    assert np.abs(gpu.theta.cpu().numpy() - given.theta).max() <= 2e-6 * max(1.0, np.abs(given.theta).max())
+
+
+def test_whole_run_properties_on_the_products_shaped_graph():
+    """At a size the checker cannot train on in reasonable time: the K-round run must be repeatable
+    bit for bit, count every edge as a message, reduce the loss in every round, and beat chance."""
+    from paper_2302_13053_b200 import binding as B
+    w = config(5)
+    ws = wl.initial_weights(w)
+    res = []
+    for _ in range(2):
+        prob = B.LmpProblem(w.aggr, w.K, 30, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
+                            w.train_idx, w.val_idx, w.test_idx, ws, part=w.part, n_parts=w.n_parts)
+        B.retexo_lmp_train(prob)
+        torch.cuda.synchronize()
+        res.append(prob.results())
+        del prob
+        torch.cuda.empty_cache()
+    a, b = res
+    np.testing.assert_array_equal(a["loss_history"], b["loss_history"])
+    np.testing.assert_array_equal(a["final_logits"], b["final_logits"])
+    assert a["counts"]["boundary_pairs"] == w.n_edges == a["counts"]["cross_edges"]
+    assert np.isfinite(a["loss_history"]).all()
+    assert (a["loss_history"][:, -1] < a["loss_history"][:, 0]).all()
+    assert a["test_acc"] > 3.0 / w.n_classes
+    for m in range(w.K):
+        v = a["val_correct"][m].astype(np.int64)
+        assert a["best_iter"][m] == int(np.argmax(v)) + 1
