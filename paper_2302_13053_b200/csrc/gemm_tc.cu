@@ -78,7 +78,9 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint6
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-__device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&r)[32]) {
+// Starts the load of 32 accumulator columns (this warp's 32 lanes) into r; the values may be
+// used only after tmem_ld_wait(r).
+__device__ __forceinline__ void tmem_ld_issue(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -88,7 +90,17 @@ __device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&r)[32]
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+// Waits for the loads in flight.  The registers are passed through as in/out operands so that
+// no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
 }
 
 struct TcKernelArgs {
@@ -291,20 +303,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 // the thread owns the whole row of logits
                 float v[64];
                 if (ok) {
+                    uint32_t ra[32], rb[32];
+                    if (n_kb > 0) {       // both halves of the row in flight together
+                        tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16), ra);
+                        tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + 32u, rb);
+                        tmem_ld_wait(ra);
+                        tmem_ld_wait(rb);
+                    } else {
 #pragma unroll
-                    for (int c0 = 0; c0 < 64; c0 += 32) {
-                        uint32_t r[32];
-                        if (n_kb > 0) tmem_ld_32cols(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-                        else {
+                        for (int j = 0; j < 32; ++j) { ra[j] = 0u; rb[j] = 0u; }
+                    }
+                    const float bias_a = (g.bias && lane < g.N) ? __ldg(g.bias + lane) : 0.f;
+                    const float bias_b = (g.bias && 32 + lane < g.N) ? __ldg(g.bias + 32 + lane) : 0.f;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) r[j] = 0u;
-                        }
-                        const float bias_lane = (g.bias && c0 + lane < g.N) ? __ldg(g.bias + c0 + lane) : 0.f;
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const int c = c0 + j;
-                            v[c] = c < g.N ? __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j) : -INFINITY;
-                        }
+                    for (int j = 0; j < 32; ++j) {
+                        v[j] = j < g.N ? __uint_as_float(ra[j]) + __shfl_sync(0xffffffffu, bias_a, j) : -INFINITY;
+                        v[32 + j] = 32 + j < g.N ? __uint_as_float(rb[j]) + __shfl_sync(0xffffffffu, bias_b, j) : -INFINITY;
                     }
                 } else {
 #pragma unroll
@@ -374,14 +388,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     asm volatile("bar.sync 1, 128;" ::: "memory");      // warp_loss is reused by the next tile
                 }
             } else if (ok) {
+                // the load of chunk c + 1 is in flight while chunk c is processed
+                uint32_t nxt[32];
+                if (n_kb > 0) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16), nxt);
+                else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) nxt[j] = 0u;
+                }
 #pragma unroll 1
                 for (int c0 = 0; c0 < BN; c0 += 32) {
                     uint32_t r[32];
-                    if (n_kb > 0) tmem_ld_32cols(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
-                    else {
+                    if (n_kb > 0) tmem_ld_wait(nxt);
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) r[j] = 0u;
-                    }
+                    for (int j = 0; j < 32; ++j) r[j] = nxt[j];
+                    if (n_kb > 0 && c0 + 32 < BN) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)(c0 + 32), nxt);
                     const int64_t col0 = n0 + c0;
                     if (col0 >= g.N) continue;
                     if (g.mode == TC_EPI_PARTIAL) {
