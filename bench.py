@@ -34,6 +34,12 @@ import numpy as np
 METRIC = "edges aggregated/s"
 UNIT = "edges/s"
 
+# DRAM bytes (read + write) per launch of the aggregation kernel, from the one-pass ncu capture
+# summarised in profiles/agg_rows_kernel_cfg4.txt.  Valid for that kernel and workload only:
+# set an entry to None when agg_rows_kernel or the workload changes.
+AGG_DRAM_TRAFFIC = {("cfg4_sage_reddit_like", 1): 193.76e9, ("cfg4_sage_reddit_like", 2): 55.57e9,
+                    ("cfg4_sage_reddit_like", 3): 55.59e9}
+
 
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -180,7 +186,7 @@ def phase_breakdown(w, ws, R: int, peaks):
         mean_ms, best_ms = time_calls(fn, 5)
         phases.append(dict(kernel="aggregate", round=m, calls_per_step=1, ms=mean_ms, best_ms=best_ms, bound="hbm",
                            algorithmic_bytes=alg, achieved=alg / mean_ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s",
-                           edges_per_s=e / mean_ms * 1e3))
+                           edges_per_s=e / mean_ms * 1e3, traffic=AGG_DRAM_TRAFFIC.get((w.name, m))))
         # the round's model at its training / validation / full shapes
         model = B.Mlp(rd["d_in"], rd["hidden"], w.n_classes, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
         xtr, xtr_t = B.retexo_pack_rows(x16, tr, dim=width, transpose=True, ones_row=True)
@@ -409,7 +415,16 @@ def main():
         dom = max(phases, key=lambda p: p["share_of_step"])
         line["roofline"] = dict(kernel="%s round %d" % (dom["kernel"], dom["round"]), bound=dom["bound"],
                                 achieved=dom["achieved"], peak=dom["peak"], unit=dom["unit"], frac=dom["frac"],
-                                traffic=None, peak_source=peaks["source"], share_of_step=dom["share_of_step"])
+                                traffic=dom.get("traffic"), peak_source=peaks["source"],
+                                share_of_step=dom["share_of_step"],
+                                note="tensor-core products of one training iteration (tc_gemm_kernel launches)"
+                                if dom["bound"] == "tensor" else "CSR gather-reduce (agg_rows_kernel)")
+        # the memory-bound side of the path, against the measured HBM copy bandwidth
+        line["roofline_aggregation"] = [
+            dict(round=p["round"], bound="hbm", achieved=p["achieved"], peak=p["peak"], unit="GB/s", frac=p["frac"],
+                 traffic=p.get("traffic"), ms=p["ms"], edges_per_s=p["edges_per_s"],
+                 dram_gbs=(p["traffic"] / p["ms"] / 1e6) if p.get("traffic") else None)
+            for p in phases if p["kernel"] == "aggregate"]
         line["phases"] = [dict(kernel=p["kernel"], round=p["round"], ms=round(p["ms"], 4), calls=p["calls_per_step"],
                                share=round(p["share_of_step"], 4), bound=p["bound"], achieved=round(p["achieved"], 2),
                                unit=p["unit"], frac=round(p["frac"], 4),

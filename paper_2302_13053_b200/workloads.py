@@ -371,7 +371,7 @@ def make_config(index: int, seed: int = 0, scale: float = 1.0) -> Workload:
         labels = _zipf_labels(s_lab, n, 47)
         w = _power_law_weights(n, 2.5, None)
         rowptr, colidx = random_graph(s_graph, n, n_und, labels, w, 0.6, None)
-        feats = _gaussian_features(s_feat, labels, 100, 0.5 * np.sqrt(8.0))
+        feats = _gaussian_features(s_feat, labels, 100, 0.5)
         tr, va, te = _split_fraction(s_split, n, 0.08, 0.02)
         part = np.arange(n, dtype=np.int32)
         return Workload("cfg5_gcn_products_like", GCN, 3, 200, 256, 47, 0.003, n, rowptr, colidx,
