@@ -16,7 +16,8 @@ namespace retexo {
 
 constexpr int kTcBM = 128;
 constexpr int kTcBK = 64;                  // 64 bf16 = 128 bytes = one swizzle row
-constexpr int kTcThreads = 192;            // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2..5: epilogue
+constexpr int kTcThreads = 320;            // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2..9: epilogue
+constexpr int kEpiWarps = 8;               // two per tensor-memory lane quarter, each taking half of the columns
 constexpr uint32_t kSpinLimit = 1u << 26;
 
 __device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
@@ -200,7 +201,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* warp_loss = reinterpret_cast<float*>(tmem_slot + 2);                  // [4]
-    uint8_t* stage_base = reinterpret_cast<uint8_t*>(                           // 4 x kStageBytesPerWarp, 16-byte aligned
+    uint8_t* stage_base = reinterpret_cast<uint8_t*>(                           // kEpiWarps x kStageBytesPerWarp, 16-byte aligned
         (reinterpret_cast<uintptr_t>(tmem_slot) + 64 + 15) & ~uintptr_t(15));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -210,7 +211,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, 4); }
+        // a thread that owns a whole row of logits needs all the columns: those epilogues use four warps
+        const bool row_owner = BN == 64 && (g.mode == TC_EPI_SOFTMAX_CE || g.mode == TC_EPI_ARGMAX);
+        for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, row_owner ? 4 : kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -283,9 +286,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         const int q = warp & 3;                           // tensor-memory lane quarter this warp may read
-        uint8_t* stage = stage_base + q * kStageBytesPerWarp;
+        const int half = (warp - 2) >> 2;                 // which half of the tile's columns this warp drains
+        uint8_t* stage = stage_base + (warp - 2) * kStageBytesPerWarp;
+        const bool row_owner = BN == 64 && (g.mode == TC_EPI_SOFTMAX_CE || g.mode == TC_EPI_ARGMAX);
         int64_t lt = 0;
-        for (int64_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++lt) {
+        for (int64_t t = blockIdx.x; t < n_tiles && !(row_owner && half == 1); t += gridDim.x, ++lt) {
             const int64_t z = t / per_split, rem = t % per_split;
             const int64_t mt = rem % n_m;
             const int64_t m0 = mt * kTcBM, n0 = (rem / n_m) * BN;
@@ -390,18 +395,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             } else if (ok) {
                 // the load of chunk c + 1 is in flight while chunk c is processed
                 uint32_t nxt[32];
-                if (n_kb > 0) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16), nxt);
+                constexpr int kHalfCols = BN / 2;
+                const int c_begin = half * kHalfCols, c_end = c_begin + kHalfCols;
+                if (n_kb > 0) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)c_begin, nxt);
                 else {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) nxt[j] = 0u;
                 }
 #pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 32) {
+                for (int c0 = c_begin; c0 < c_end; c0 += 32) {
                     uint32_t r[32];
                     if (n_kb > 0) tmem_ld_wait(nxt);
 #pragma unroll
                     for (int j = 0; j < 32; ++j) r[j] = nxt[j];
-                    if (n_kb > 0 && c0 + 32 < BN) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)(c0 + 32), nxt);
+                    if (n_kb > 0 && c0 + 32 < c_end) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)(c0 + 32), nxt);
                     const int64_t col0 = n0 + c0;
                     if (col0 >= g.N) continue;
                     if (g.mode == TC_EPI_PARTIAL) {
@@ -522,7 +529,7 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t c
 
 template <int BN, int STAGES>
 static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
-    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 512 + 4 * kStageBytesPerWarp;
+    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 512 + kEpiWarps * kStageBytesPerWarp;
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
