@@ -124,8 +124,8 @@ def launches_per_step(w, R: int) -> int:
             total += 3                               # prep, warp rows, block rows
         total += 2                                   # train / val batches
         step = 6 if h > 0 else 3                     # products, reduce + update (+ weight copies once)
-        ev = (2 if h > 0 else 1) + 2                 # validation forward + snapshot / bookkeeping
-        total += R * (step + ev) + (2 if h > 0 else 1)
+        total += R * (step + 1) + (2 if h > 0 else 1)     # + bookkeeping of the validation count that rides along
+        total += (2 if h > 0 else 1) + 1             # stand-alone validation of the last iterate + snapshot
         total += 2 * (4 if h > 0 else 3)             # test accuracy, kept and last iterate
         total += 3 if h > 0 else 2                   # emission of Q^m / final logits
     return total

@@ -100,7 +100,7 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
         if (r.rep_dim > max_rep) max_rep = r.rep_dim;
         const int64_t nt = retexo_theta_size(r.d_in, r.hidden, c.n_classes);
         if (nt > max_nt) max_nt = nt;
-        size_t s = retexo_mlp_train_step_workspace_size(r.d_in, r.hidden, c.n_classes, n_tr);
+        size_t s = mlp_step_workspace_size(make_plan(r.d_in, r.hidden, c.n_classes, n_tr, n_val));
         if (s > step_b) step_b = s;
         s = retexo_embed_workspace_size(r.d_in, r.hidden, c.n_classes, n);
         if (s > embed_b) embed_b = s;
@@ -130,8 +130,8 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
         l.gat_vec = t.template take<float>((size_t)2 * hd);
         l.gat_stage = t.template take<float>((size_t)max_rep * hd + 2 * hd);
     }
-    l.xtr16 = t.template take<bf16>((size_t)n_tr * ld16);
-    l.xval16 = t.template take<bf16>((size_t)(n_val > 0 ? n_val : 1) * ld16);
+    l.xtr16 = t.template take<bf16>((size_t)(n_tr + n_val) * ld16);     // training rows, then validation rows
+    l.xval16 = nullptr;
     l.xtr_t16 = t.template take<bf16>((size_t)(max_din + 1) * (size_t)round_up(n_tr, 8));
     l.y_tr = t.template take<int32_t>((size_t)n_tr);
     l.y_val = t.template take<int32_t>((size_t)(n_val > 0 ? n_val : 1));
@@ -309,7 +309,8 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         // ---- the round's batches and model state
         const int64_t ld_xt = round_up(n_tr, 8);
         RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld16, b.xtr_t16, ld_xt, 1, st));
-        if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, b.xval16, ld16, nullptr, 0, 0, st));
+        bf16* xval16 = b.xtr16 + (size_t)n_tr * ld16;
+        if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, xval16, ld16, nullptr, 0, 0, st));
         RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta, in->theta0[m - 1], sizeof(float) * (size_t)nt, cudaMemcpyDefault, st));
         RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta_best, b.theta, sizeof(float) * (size_t)nt, cudaMemcpyDeviceToDevice, st));
         RETEXO_CUDA_TRY(cudaMemsetAsync(b.adam_m, 0, sizeof(float) * (size_t)nt, st));
@@ -327,18 +328,28 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         best.theta = b.theta_best;
 
         // ---- R training iterations; validation and best-iterate tracking stay on the device
-        const MlpPlan plan = make_plan(r.d_in, r.hidden, c.n_classes, n_tr);
+        const MlpPlan plan = make_plan(r.d_in, r.hidden, c.n_classes, n_tr, n_val);
         MlpBuffers sb{};
         mlp_step_buffers(plan, b.ws_step, b.ws_step_bytes, &sb);
-        bf16* val_hd = reinterpret_cast<bf16*>(b.ws_embed);      // [n_val x ld_h] scratch of the validation forward
+        bf16* val_hd = reinterpret_cast<bf16*>(b.ws_embed);      // [n_val x ld_h] scratch of a stand-alone validation forward
+        const EvalTail tail{b.y_val, b.cur_correct, b.best_correct, b.have_best, b.theta_best};
+        int pending_it = 0;       // iteration whose weights still await their validation count
         for (int it = 1; it <= c.R; ++it) {
             float* loss_slot = b.loss_history + (size_t)(m - 1) * c.R + (it - 1);
-            // the update of iteration it-1 left bf16 copies of the current weights behind
+            // The weights of iteration it-1 are validated inside this iteration's forward pass (the
+            // validation rows ride along; the update kernel keeps them if they are the best so far).
+            // The update of iteration it-1 also left bf16 copies of the current weights behind.
             RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, loss_slot,
-                                             nullptr, it > 1, st));
+                                             nullptr, it > 1, pending_it ? &tail : nullptr, st));
             model.step += 1;
-            if (n_val && (it % c.eval_every == 0 || it == c.R)) {
-                RETEXO_TRY(mlp_count_hits_launch(plan, sb, &model, b.xval16, ld16, n_val, val_hd, b.y_val,
+            if (pending_it)
+                record_validation_kernel<<<1, 32, 0, st>>>(b.cur_correct, b.best_correct, b.have_best, pending_it,
+                                                           b.best_iter_cur,
+                                                           b.val_history + (size_t)(m - 1) * c.R + (pending_it - 1));
+            const bool want = n_val && (it % c.eval_every == 0 || it == c.R);
+            pending_it = (want && it < c.R) ? it : 0;
+            if (want && it == c.R) {      // the last iterate has no next iteration to ride on
+                RETEXO_TRY(mlp_count_hits_launch(plan, sb, &model, xval16, ld16, n_val, val_hd, b.y_val,
                                                  b.cur_correct, st));
                 snapshot_if_better_kernel<<<(unsigned)((nt + 255) / 256), 256, 0, st>>>(
                     b.cur_correct, b.best_correct, b.have_best, b.theta, b.theta_best, nt);

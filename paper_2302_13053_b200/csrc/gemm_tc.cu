@@ -118,6 +118,7 @@ struct TcKernelArgs {
     float* partial;
     const int32_t* y; float inv_rows; float* loss_partial;
     int32_t* pred; unsigned long long* correct;
+    int64_t n_train; const int32_t* y_eval;       // SOFTMAX_CE: rows >= n_train are evaluated, not trained on
     int32_t* status;
 };
 
@@ -329,8 +330,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int c = 0; c < 64; ++c) v[c] = 0.f;
                 }
-                const bool live = ok && row < g.M;
+                const bool is_eval = g.mode == TC_EPI_SOFTMAX_CE && row >= g.n_train;
+                const bool live = ok && row < g.M && !is_eval;
                 const int32_t yi = (live && g.y) ? g.y[row] : -1;
+                if (g.mode == TC_EPI_SOFTMAX_CE && m0 + kTcBM > g.n_train && g.n_train < g.M) {
+                    // this tile holds evaluation rows: arg-max (lowest index on ties) and hit count
+                    int best = 0;
+                    float bv = v[0];
+#pragma unroll
+                    for (int c = 1; c < 64; ++c) if (v[c] > bv) { bv = v[c]; best = c; }
+                    const bool hit = ok && is_eval && row < g.M && best == g.y_eval[row - g.n_train];
+                    const unsigned hits = __ballot_sync(0xffffffffu, hit);
+                    if (lane == 0 && hits) atomicAdd(g.correct, (unsigned long long)__popc(hits));
+                }
                 if (g.mode == TC_EPI_ARGMAX) {
                     int best = 0;
                     float bv = v[0];
@@ -382,7 +394,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             float blk[32];
 #pragma unroll
                             for (int j = 0; j < 32; ++j) blk[j] = v[c0 + j];
-                            store_block_transposed(g.out_bf16_t, g.ld_t, c0, g.N, row0, g.M, blk, stage, lane);
+                            store_block_transposed(g.out_bf16_t, g.ld_t, c0, g.N, row0, g.n_train, blk, stage, lane);
                         }
                     }
                     loss = warp_sum(loss);
@@ -551,6 +563,8 @@ static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& 
     g.mask = t.mask; g.ld_mask = t.ld_mask;
     g.partial = t.partial; g.status = t.status;
     g.y = t.y; g.inv_rows = t.inv_rows; g.loss_partial = t.loss_partial; g.pred = t.pred; g.correct = t.correct;
+    g.n_train = (t.mode == TC_EPI_SOFTMAX_CE && t.eval_from > 0 && t.eval_from < t.M) ? t.eval_from : t.M;
+    g.y_eval = t.y_eval;
     const int64_t n_tiles = ((t.M + kTcBM - 1) / kTcBM) * ((t.N + BN - 1) / BN) * splits;
     const int n_sm = sm_count();
     if (n_sm <= 0) return RETEXO_ERR_CUDA;

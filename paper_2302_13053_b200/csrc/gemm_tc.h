@@ -41,6 +41,9 @@ struct TcGemm {
     const __nv_bfloat16* mask; int64_t ld_mask;
     float* partial;
     const int32_t* y; float inv_rows; float* loss_partial;      // TC_EPI_SOFTMAX_CE / TC_EPI_ARGMAX
+    // TC_EPI_SOFTMAX_CE only: rows [eval_from, M) are not trained on but only evaluated: their arg-max is
+    // compared with y_eval[row - eval_from] and the hits are added to *correct (0 = no such rows)
+    int64_t eval_from; const int32_t* y_eval;
     int32_t* pred; unsigned long long* correct;                  // TC_EPI_ARGMAX (both optional)
     int32_t* status;
 };

@@ -53,16 +53,16 @@ static int64_t tc_split(int64_t M, int64_t N, int64_t K) {
     return s;
 }
 
-MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows) {
+MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval) {
     MlpPlan p{};
-    p.d_in = d_in; p.hidden = hidden; p.n_classes = n_classes; p.n_rows = n_rows;
+    p.d_in = d_in; p.hidden = hidden; p.n_classes = n_classes; p.n_rows = n_rows; p.n_eval = n_eval;
     p.out1 = hidden > 0 ? hidden : n_classes;
     p.nt = retexo_theta_size(d_in, hidden, n_classes);
     p.ld_dl = round_up8(n_classes);
     p.ld_h = round_up8(hidden > 0 ? hidden : 1);
     p.ld_k = round_up8(d_in);
-    p.ld_n = round_up8(n_rows);
-    p.sm_blocks = (n_rows + 127) / 128;          // one loss partial per 128-row tile of the head product
+    p.ld_n = round_up8(n_rows + n_eval);
+    p.sm_blocks = (n_rows + n_eval + 127) / 128;          // one loss partial per 128-row tile of the head product
     p.split_w1 = tc_split((int64_t)d_in + 1, p.out1, n_rows);
     p.split_w2 = hidden > 0 ? tc_split((int64_t)hidden + 1, n_classes, n_rows) : 0;
     return p;
@@ -72,12 +72,13 @@ template <typename Taker>
 static void layout(const MlpPlan& p, Taker& t, MlpBuffers* out) {
     MlpBuffers b{};
     const size_t n = (size_t)p.n_rows;
+    const size_t n_all = (size_t)(p.n_rows + p.n_eval);
     const bool h = p.hidden > 0;
     b.w1t16 = t.template take<bf16>((size_t)p.out1 * p.ld_k);
     b.w2t16 = t.template take<bf16>(h ? (size_t)p.n_classes * p.ld_h : 1);
     b.w2p16 = t.template take<bf16>(h ? (size_t)p.hidden * p.ld_dl : 1);
     b.xt16 = t.template take<bf16>((size_t)(p.d_in + 1) * p.ld_n);
-    b.hd16 = t.template take<bf16>(h ? n * p.ld_h : 1);
+    b.hd16 = t.template take<bf16>(h ? n_all * p.ld_h : 1);
     b.hdt16 = t.template take<bf16>(h ? (size_t)(p.hidden + 1) * p.ld_n : 1);
     b.logits = t.template take<float>(n * p.n_classes);
     b.dl16 = t.template take<bf16>(n * p.ld_dl);
@@ -99,6 +100,12 @@ struct NullTaker {
     Sizer s;
     template <typename T> T* take(size_t count) { s.take<T>(count); return nullptr; }
 };
+
+size_t mlp_step_workspace_size(const MlpPlan& p) {
+    NullTaker t;
+    layout(p, t, nullptr);
+    return t.s.off + kAlign;
+}
 
 static int check_model(const retexo_mlp* m) {
     if (!m || m->d_in <= 0 || m->hidden < 0 || m->n_classes <= 0 || !m->theta) return RETEXO_ERR_INVALID_ARG;
@@ -157,10 +164,7 @@ extern "C" int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld
 extern "C" size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes,
                                                        int64_t n_rows) {
     if (d_in <= 0 || hidden < 0 || n_classes <= 0 || n_rows <= 0) return 0;
-    MlpPlan p = make_plan(d_in, hidden, n_classes, n_rows);
-    NullTaker t;
-    layout(p, t, nullptr);
-    return t.s.off + kAlign;
+    return mlp_step_workspace_size(make_plan(d_in, hidden, n_classes, n_rows));
 }
 
 extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t ldx, const void* x_t, int64_t ld_xt,
@@ -182,7 +186,7 @@ extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t l
     MlpBuffers b{};
     layout(p, ws, &b);
     RETEXO_TRY(mlp_train_step_launch(p, b, model, static_cast<const bf16*>(x), ldx,
-                                     static_cast<const bf16*>(x_t), ld_xt, y, loss_out, grad_out, false, st));
+                                     static_cast<const bf16*>(x_t), ld_xt, y, loss_out, grad_out, false, nullptr, st));
     model->step += 1;
     return RETEXO_OK;
 }
@@ -193,8 +197,10 @@ namespace retexo {
 // already applied.
 int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
                           const bf16* x, int64_t ldx, const bf16* x_t, int64_t ld_xt, const int32_t* y,
-                          float* loss_out, float* grad_out, bool shadows_ready, cudaStream_t st) {
+                          float* loss_out, float* grad_out, bool shadows_ready, const EvalTail* tail,
+                          cudaStream_t st) {
     const int64_t n = p.n_rows;
+    const int64_t n_all = n + (tail ? p.n_eval : 0);          // evaluation rows ride along in the forward pass
     const int32_t d_in = p.d_in, H = p.hidden, O = p.n_classes, out1 = p.out1;
     const float* theta = model->theta;
     const float* b1 = theta + (int64_t)d_in * out1;
@@ -209,19 +215,21 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
 
     // ---- forward; the class-dimension product ends in the loss: softmax, cross-entropy and dL
     //      are computed in its epilogue, where one thread holds a whole row of logits
-    TcGemm fwd = tc_base(x, ldx, b.w1t16, p.ld_k, n, out1, d_in, b.status);
+    if (tail) RETEXO_CUDA_TRY(cudaMemsetAsync(tail->correct, 0, sizeof(unsigned long long), st));
+    TcGemm fwd = tc_base(x, ldx, b.w1t16, p.ld_k, n_all, out1, d_in, b.status);
     fwd.bias = b1;
     TcGemm head = fwd;
     if (H > 0) {
         fwd.relu = 1; fwd.out_bf16 = b.hd16; fwd.ld_bf16 = p.ld_h;
         fwd.out_bf16_t = b.hdt16; fwd.ld_t = p.ld_n; fwd.ones_row_t = 1;
         RETEXO_TRY(tc_gemm_launch(fwd, st));
-        head = tc_base(b.hd16, p.ld_h, b.w2t16, p.ld_h, n, O, H, b.status);
+        head = tc_base(b.hd16, p.ld_h, b.w2t16, p.ld_h, n_all, O, H, b.status);
         head.bias = b2;
     }
     head.mode = TC_EPI_SOFTMAX_CE; head.y = y; head.inv_rows = 1.0f / (float)n; head.loss_partial = b.loss_partial;
     head.out_bf16 = H > 0 ? b.dl16 : nullptr; head.ld_bf16 = p.ld_dl;
     head.out_bf16_t = b.dlt16; head.ld_t = p.ld_n;
+    if (tail) { head.eval_from = n; head.y_eval = tail->y_eval; head.correct = tail->correct; }
     RETEXO_TRY(tc_gemm_launch(head, st));
     // ---- backward
     const bf16* grad1_t = b.dlt16;      // gradient at the first layer's output, transposed
@@ -254,6 +262,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     u.w1t16 = b.w1t16; u.ld_k = p.ld_k; u.w2t16 = H > 0 ? b.w2t16 : nullptr; u.ld_h = p.ld_h;
     u.w2p16 = H > 0 ? b.w2p16 : nullptr; u.ld_dl = p.ld_dl;
     u.d_in = d_in; u.out1 = out1; u.hidden = H; u.n_classes = O;
+    if (tail) { u.snap_cur = tail->correct; u.snap_best = tail->best; u.snap_have = tail->have_best; u.theta_best = tail->theta_best; }
     reduce_update_kernel<<<(unsigned)((p.nt + 255) / 256), 256, 0, st>>>(u);
     return launch_status();
 }

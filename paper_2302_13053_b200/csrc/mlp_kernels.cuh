@@ -218,6 +218,9 @@ struct UpdateArgs {
     bf16* w2t16; int64_t ld_h;       // W2^T [n_classes x ld_h]
     bf16* w2p16; int64_t ld_dl;      // W2   [hidden x ld_dl]
     int32_t d_in, out1, hidden, n_classes;
+    // keep-the-best snapshot of theta as it is before this update (optional, see EvalTail)
+    const unsigned long long* snap_cur; const unsigned long long* snap_best; const int32_t* snap_have;
+    float* theta_best;
 };
 
 // Sums each parameter's split-K partials in index order, applies the optimiser, and refreshes
@@ -248,6 +251,7 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     }
     for (; z < count; ++z) g += part[z * size + q];
     if (u.grad_out) u.grad_out[p] = g;
+    if (u.theta_best && (!*u.snap_have || *u.snap_cur > *u.snap_best)) u.theta_best[p] = u.theta[p];
     float t;
     if (u.optimizer == RETEXO_SGD) {
         t = u.theta[p] - u.lr * g;

@@ -14,11 +14,12 @@ constexpr int64_t kSmCountTarget = 148;     // one tensor-core block per SM
 
 struct MlpPlan {
     int32_t d_in, hidden, n_classes, out1;  // out1 = width of the first linear layer's output
-    int64_t n_rows, nt;                     // nt = parameters in theta
+    int64_t n_rows, nt;                     // training rows; nt = parameters in theta
+    int64_t n_eval;                         // rows after the training rows that are only evaluated (validation)
     int64_t ld_dl;                          // row stride of bf16 dL and of the padded W2 (classes rounded up to 8)
     int64_t ld_h;                           // row stride of bf16 Hd and of W2^T (hidden rounded up to 8)
     int64_t ld_k;                           // row stride of W1^T (d_in rounded up to 8)
-    int64_t ld_n;                           // row stride of everything stored transposed (n_rows rounded up to 8)
+    int64_t ld_n;                           // row stride of everything stored transposed (all rows, rounded up to 8)
     int64_t sm_blocks;                      // softmax blocks = number of loss partials
     int64_t split_w1, split_w2;             // split-K factors of the two weight-gradient products
 };
@@ -40,7 +41,20 @@ struct MlpBuffers {
     int32_t* status;                        // raised by a tensor-core kernel whose bounded wait gave up
 };
 
-MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows);
+MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval = 0);
+size_t mlp_step_workspace_size(const MlpPlan& p);
+
+// Validation folded into a training iteration: the batch holds p.n_eval more rows after the
+// training rows; the forward pass covers them too, the loss epilogue counts their hits into
+// *correct (weights as they are before this iteration's update), and the update kernel first
+// copies theta to theta_best if that count beats *best (or nothing was kept yet).
+struct EvalTail {
+    const int32_t* y_eval;
+    unsigned long long* correct;
+    const unsigned long long* best;
+    const int32_t* have_best;
+    float* theta_best;
+};
 
 // Lays the step's scratch buffers out over a workspace of retexo_mlp_train_step_workspace_size bytes.
 void mlp_step_buffers(const MlpPlan& p, void* workspace, size_t bytes, MlpBuffers* out);
@@ -50,7 +64,8 @@ void mlp_step_buffers(const MlpPlan& p, void* workspace, size_t bytes, MlpBuffer
 // On return they hold the updated theta.
 int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
                           const __nv_bfloat16* x, int64_t ldx, const __nv_bfloat16* x_t, int64_t ld_xt,
-                          const int32_t* y, float* loss_out, float* grad_out, bool shadows_ready, cudaStream_t st);
+                          const int32_t* y, float* loss_out, float* grad_out, bool shadows_ready,
+                          const EvalTail* tail, cudaStream_t st);
 
 // Forward + arg-max + hit count over a dense batch with the weight copies in `b` (which must
 // hold model->theta): what validation needs after every iteration.  hd_ws: bf16 [n_rows x p.ld_h].
