@@ -205,6 +205,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint8_t* stage_base = reinterpret_cast<uint8_t*>(                           // kEpiWarps x kStageBytesPerWarp, 16-byte aligned
         (reinterpret_cast<uintptr_t>(tmem_slot) + 64 + 15) & ~uintptr_t(15));
 
+    float (*xch)[2][128] = reinterpret_cast<float (*)[2][128]>(stage_base + kEpiWarps * kStageBytesPerWarp);   // [4][2][128]
+
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t n_m = (g.M + kTcBM - 1) / kTcBM, n_n = (g.N + BN - 1) / BN;
     const int64_t per_split = n_m * n_n;
@@ -212,8 +214,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
-        // a thread that owns a whole row of logits needs all the columns: those epilogues use four warps
-        const bool row_owner = BN == 64 && (g.mode == TC_EPI_SOFTMAX_CE || g.mode == TC_EPI_ARGMAX);
+        // the arg-max epilogue lets one thread own a whole row of logits: it uses four of the eight warps
+        const bool row_owner = BN == 64 && g.mode == TC_EPI_ARGMAX;
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, row_owner ? 4 : kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -289,7 +291,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int q = warp & 3;                           // tensor-memory lane quarter this warp may read
         const int half = (warp - 2) >> 2;                 // which half of the tile's columns this warp drains
         uint8_t* stage = stage_base + (warp - 2) * kStageBytesPerWarp;
-        const bool row_owner = BN == 64 && (g.mode == TC_EPI_SOFTMAX_CE || g.mode == TC_EPI_ARGMAX);
+        const bool row_owner = BN == 64 && g.mode == TC_EPI_ARGMAX;
         int64_t lt = 0;
         for (int64_t t = blockIdx.x; t < n_tiles && !(row_owner && half == 1); t += gridDim.x, ++lt) {
             const int64_t z = t / per_split, rem = t % per_split;
@@ -305,7 +307,85 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool ok = mbar_wait(acc_full + b, pb, g.status, abort_flag);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (!ok) break;
-            if (BN == 64 && (g.mode == TC_EPI_SOFTMAX_CE || g.mode == TC_EPI_ARGMAX)) {
+            if (BN == 64 && g.mode == TC_EPI_SOFTMAX_CE) {
+                // Two threads share a row of logits: warp q takes columns [0, 32), warp q + 4 columns
+                // [32, 64); row maximum, sum and the label's logit are exchanged through shared memory.
+                const int cb = half * 32;
+                const int slot = q * 32 + lane;                          // this row's slot in the exchange arrays
+                float v[32];
+                {
+                    uint32_t r[32];
+                    if (n_kb > 0) { tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)cb, r); tmem_ld_wait(r); }
+                    else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = 0u;
+                    }
+                    const float bias_lane = (g.bias && cb + lane < g.N) ? __ldg(g.bias + cb + lane) : 0.f;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        v[j] = cb + j < g.N ? __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j) : -INFINITY;
+                }
+                const bool is_eval = row >= g.n_train;
+                const bool live = row < g.M && !is_eval;
+                const int32_t yi = (live && g.y) ? g.y[row] : -1;
+                float mx = v[0];
+                int best = 0;
+#pragma unroll
+                for (int j = 1; j < 32; ++j) if (v[j] > mx) { mx = v[j]; best = j; }      // strict: lowest index on ties
+                xch[0][half][slot] = mx;
+                xch[1][half][slot] = __int_as_float(cb + best);
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                const float m0v = xch[0][0][slot], m1v = xch[0][1][slot];
+                if (g.n_train < g.M && m0 + kTcBM > g.n_train && half == 0) {
+                    // evaluation rows in this tile: arg-max over both halves (the lower half wins ties)
+                    const int arg = m1v > m0v ? __float_as_int(xch[1][1][slot]) : __float_as_int(xch[1][0][slot]);
+                    const bool hit = is_eval && row < g.M && arg == g.y_eval[row - g.n_train];
+                    const unsigned hits = __ballot_sync(0xffffffffu, hit);
+                    if (lane == 0 && hits) atomicAdd(g.correct, (unsigned long long)__popc(hits));
+                }
+                mx = fmaxf(m0v, m1v);
+                float den = 0.f, ly = 0.f;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    ly = cb + j == yi ? v[j] : ly;
+                    v[j] = cb + j < g.N ? __expf(v[j] - mx) : 0.f;
+                    den += v[j];
+                }
+                xch[2][half][slot] = den;
+                xch[3][half][slot] = ly;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                den = xch[2][0][slot] + xch[2][1][slot];
+                ly = xch[3][0][slot] + xch[3][1][slot];
+                const float scale = g.inv_rows / den;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) v[j] = cb + j < g.N ? (v[j] * scale - (cb + j == yi ? g.inv_rows : 0.f)) : 0.f;
+                if (live && g.out_bf16) {       // dL row-major: this thread's columns, 16 bytes at a time
+                    __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16 + cb;
+#pragma unroll
+                    for (int c = 0; c < 32; c += 8) {
+                        if (cb + c >= g.ld_bf16) break;
+                        __nv_bfloat162 p0 = __floats2bfloat162_rn(v[c], v[c + 1]), p1 = __floats2bfloat162_rn(v[c + 2], v[c + 3]);
+                        __nv_bfloat162 p2 = __floats2bfloat162_rn(v[c + 4], v[c + 5]), p3 = __floats2bfloat162_rn(v[c + 6], v[c + 7]);
+                        uint4 pk;
+                        pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
+                        pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
+                        *reinterpret_cast<uint4*>(dst + c) = pk;
+                    }
+                }
+                if (g.out_bf16_t && cb < g.N)
+                    store_block_transposed(g.out_bf16_t, g.ld_t, cb, g.N, row0, g.n_train, v, stage, lane);
+                if (half == 0) {
+                    float loss = live ? (mx + __logf(den)) - ly : 0.f;
+                    loss = warp_sum(loss);
+                    if (lane == 0) warp_loss[q] = loss;
+                }
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                if (warp == 2 && lane == 0 && g.loss_partial)
+                    g.loss_partial[mt] = ((warp_loss[0] + warp_loss[1]) + warp_loss[2]) + warp_loss[3];
+                // (the exchange arrays and warp_loss are next written after the following tile's first
+                //  barrier-protected phase: every warp passes two more barriers before reusing them)
+            } else if (BN == 64 && g.mode == TC_EPI_ARGMAX) {
+
                 // the thread owns the whole row of logits
                 float v[64];
                 if (ok) {
@@ -541,7 +621,7 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t c
 
 template <int BN, int STAGES>
 static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
-    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 512 + kEpiWarps * kStageBytesPerWarp;
+    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 512 + kEpiWarps * kStageBytesPerWarp + 4 * 2 * 128 * 4;
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
