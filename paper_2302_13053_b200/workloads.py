@@ -358,7 +358,7 @@ def make_config(index: int, seed: int = 0, scale: float = 1.0) -> Workload:
         labels = s_lab.integers(0, 41, size=n).astype(np.int32)
         mean_deg = 2.0 * n_und / n
         w = _power_law_weights(n, 2.5, min(20000.0, n / 6) / mean_deg)
-        rowptr, colidx = random_graph(s_graph, n, n_und, labels, w, 0.5, None)
+        rowptr, colidx = random_graph(s_graph, n, n_und, labels, w, 0.56, None)
         feats = _gaussian_features(s_feat, labels, 602, 0.05)
         tr, va, te = _split_fraction(s_split, n, 0.66, 0.10)
         part = s_part.integers(0, 1000, size=n).astype(np.int32)
