@@ -248,7 +248,7 @@ int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* part, int32
  *     (retexo_cross_partition_workspace_size) exceeds that array is rejected
  *     with RETEXO_ERR_UNSUPPORTED and nothing is launched.  Up to 8192
  *     partitions the need is about 1 KiB whatever the graph's size; beyond
- *     that it grows as 4 n_nodes + 8 n_parts bytes (+ 1 KiB).
+ *     that it grows as 4 n_nodes + 18.5 n_parts bytes (+ 1 KiB).
  *   - The first call on a device looks the array's device address up
  *     (one-time set-up, per device, with that device current); make that first
  *     call before any stream capture.

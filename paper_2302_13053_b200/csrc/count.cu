@@ -12,10 +12,12 @@ constexpr int kCntThreads = 256;
 constexpr int kCntWarps = kCntThreads / kWarp;
 constexpr int kBitmapParts = 8192;                  // per-warp shared bitmap covers this many partitions
 constexpr int kBitmapWords = kBitmapParts / 32;
-constexpr int kHashSlots = 2048;                    // per-warp shared hash set
-constexpr int kHashMaxDeg = 1024;                   // rows up to this length use it
+constexpr int kHashSlots = 1024;                    // per-warp shared hash set
+constexpr int kHashMaxDeg = 512;                    // rows up to this length use it
 constexpr int kHashWarps = 4;
-constexpr int kBigRowBlocks = 64;                   // blocks (and global bitmaps) of the long-row pass
+constexpr int kBigRowBlocks = 148;                  // blocks (and global bitmaps) of the long-row pass
+constexpr int kBlockRowDeg = 4096;                  // rows longer than this go to the long-row pass at once
+constexpr int32_t kCrossCounted = INT32_MIN;        // list flag: the row's cross edges are already tallied
 
 struct CountArgs {
     int64_t n;
@@ -136,21 +138,38 @@ __global__ void __launch_bounds__(kHashWarps * kWarp) count_general_kernel(Count
         const int64_t beg = a.rowptr[u], end = a.rowptr[u + 1];
         if (beg == end) continue;
         const int32_t pu = part_of(a, u);
-        // pass 1: order check + adjacent-distinct count
+        if (end - beg > kBlockRowDeg) {     // a whole block takes this row (a single warp would be a long tail)
+            if (lane == 0) {
+                const int32_t slot = atomicAdd(a.big_count, 1);
+                a.big_list[slot] = (int32_t)u;
+            }
+            continue;
+        }
+        // pass 1: order check + adjacent-distinct count, four chunks of 32 entries per trip
         bool mono = true;
         unsigned n_cross = 0, n_new = 0;
         int32_t carry = -1;
-        for (int64_t e0 = beg; e0 < end; e0 += kWarp) {
-            const int64_t e = e0 + lane;
-            const bool valid = e < end;
-            const int32_t pv = valid ? part_of(a, __ldg(a.colidx + e)) : INT32_MAX;
-            int32_t prev = __shfl_up_sync(0xffffffffu, pv, 1);
-            if (lane == 0) prev = carry;
-            mono = mono && __all_sync(0xffffffffu, pv >= prev);
-            const bool cross = valid && pv != pu;
-            n_cross += __popc(__ballot_sync(0xffffffffu, cross));
-            n_new += __popc(__ballot_sync(0xffffffffu, cross && pv != prev));
-            carry = __shfl_sync(0xffffffffu, pv, kWarp - 1);
+        for (int64_t e0 = beg; e0 < end; e0 += 4 * kWarp) {
+            int32_t nb[4], pvs[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int64_t e = e0 + t * kWarp + lane;
+                nb[t] = e < end ? __ldg(a.colidx + e) : -1;
+            }
+#pragma unroll
+            for (int t = 0; t < 4; ++t) pvs[t] = nb[t] >= 0 ? part_of(a, nb[t]) : INT32_MAX;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int32_t pv = pvs[t];
+                const bool valid = nb[t] >= 0;
+                int32_t prev = __shfl_up_sync(0xffffffffu, pv, 1);
+                if (lane == 0) prev = carry;
+                mono = mono && __all_sync(0xffffffffu, pv >= prev);
+                const bool cross = valid && pv != pu;
+                n_cross += __popc(__ballot_sync(0xffffffffu, cross));
+                n_new += __popc(__ballot_sync(0xffffffffu, cross && pv != prev));
+                carry = __shfl_sync(0xffffffffu, pv, kWarp - 1);
+            }
         }
         if (lane == 0) my_cross += n_cross;
         if (n_cross == 0) continue;
@@ -193,7 +212,7 @@ __global__ void __launch_bounds__(kHashWarps * kWarp) count_general_kernel(Count
         } else {
             if (lane == 0) {
                 const int32_t slot = atomicAdd(a.big_count, 1);
-                a.big_list[slot] = (int32_t)u;
+                a.big_list[slot] = (int32_t)u | kCrossCounted;
             }
             continue;      // pairs of this row are counted by the long-row pass
         }
@@ -211,15 +230,62 @@ __global__ void __launch_bounds__(kHashWarps * kWarp) count_general_kernel(Count
 // Long unordered rows with many partitions: one block per row, the seen-set is
 // a bitmap in global memory owned by the block (all zero on entry and exit).
 __global__ void __launch_bounds__(kCntThreads) count_big_rows_kernel(CountArgs a) {
-    __shared__ unsigned int block_new;
+    __shared__ unsigned int block_new, block_cross;
     uint32_t* bm = a.big_bitmaps + (int64_t)blockIdx.x * a.words_per_bitmap;
     const int n_big = *a.big_count;
     for (int r = blockIdx.x; r < n_big; r += gridDim.x) {
-        const int64_t u = a.big_list[r];
+        const int32_t entry = a.big_list[r];
+        const bool cross_counted = (entry & kCrossCounted) != 0;      // a warp already found it unordered
+        const int64_t u = entry & INT32_MAX;
         const int64_t beg = a.rowptr[u], end = a.rowptr[u + 1];
         const int32_t pu = part_of(a, u);
-        if (threadIdx.x == 0) block_new = 0;
+        if (threadIdx.x == 0) { block_new = 0; block_cross = 0; }
         __syncthreads();
+        if (!cross_counted) {
+            // ordered rows (node-level or range partitions): compare every entry with its predecessor
+            bool mono = true;
+            unsigned n_cross = 0, n_adj = 0;
+            for (int64_t e0 = beg + threadIdx.x; e0 < end; e0 += 4 * kCntThreads) {
+                int32_t nb[4], pb[4], pv[4], pp[4];
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int64_t e = e0 + (int64_t)t * kCntThreads;
+                    nb[t] = e < end ? __ldg(a.colidx + e) : -1;
+                    pb[t] = (e < end && e > beg) ? __ldg(a.colidx + e - 1) : -1;
+                }
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    pv[t] = nb[t] >= 0 ? part_of(a, nb[t]) : INT32_MAX;
+                    pp[t] = pb[t] >= 0 ? part_of(a, pb[t]) : -1;
+                }
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    if (nb[t] < 0) continue;
+                    mono = mono && pv[t] >= pp[t];
+                    if (pv[t] != pu) { ++n_cross; if (pv[t] != pp[t]) ++n_adj; }
+                }
+            }
+            if (n_cross) atomicAdd(&block_cross, n_cross);
+            const int all_mono = __syncthreads_and(mono ? 1 : 0);
+            if (threadIdx.x == 0 && block_cross) atomicAdd(a.cross_edges, (unsigned long long)block_cross);
+            if (all_mono) {
+                if (n_adj) atomicAdd(&block_new, n_adj);
+                if (a.recv) {
+                    for (int64_t e = beg + threadIdx.x; e < end; e += kCntThreads) {
+                        const int32_t pv = part_of(a, __ldg(a.colidx + e));
+                        const int32_t pp = e > beg ? part_of(a, __ldg(a.colidx + e - 1)) : -1;
+                        if (pv != pu && pv != pp) atomicAdd(a.recv + pv, 1ull);
+                    }
+                }
+                __syncthreads();
+                if (threadIdx.x == 0 && block_new) {
+                    atomicAdd(a.pairs, (unsigned long long)block_new);
+                    if (a.send) atomicAdd(a.send + pu, (unsigned long long)block_new);
+                }
+                __syncthreads();
+                continue;
+            }
+        }
         unsigned mine = 0;
         for (int64_t e = beg + threadIdx.x; e < end; e += kCntThreads) {
             const int32_t pv = part_of(a, __ldg(a.colidx + e));
@@ -373,7 +439,7 @@ extern "C" int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* 
             RETEXO_CUDA_TRY(cudaMemsetAsync(a.big_bitmaps, 0,
                                             sizeof(uint32_t) * (size_t)kBigRowBlocks * (size_t)a.words_per_bitmap, st));
             const int64_t want = (a.n + kHashWarps - 1) / kHashWarps;
-            const unsigned blocks = (unsigned)(want < (int64_t)n_sm * 16 ? want : (int64_t)n_sm * 16);
+            const unsigned blocks = (unsigned)(want < (int64_t)n_sm * 32 ? want : (int64_t)n_sm * 32);
             count_general_kernel<<<blocks, kHashWarps * kWarp, 0, st>>>(a);
             count_big_rows_kernel<<<kBigRowBlocks, kCntThreads, 0, st>>>(a);
         }

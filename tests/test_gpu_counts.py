@@ -45,7 +45,7 @@ def test_node_level_partition_and_single_partition():
 
 def test_every_dedup_path_of_the_many_partition_kernel():
     """Node-level ids scrambled (rows not ordered -> hash set), a long scrambled
-    row (> 1024 entries -> global bitmap), range partitions (ordered rows)."""
+    row (> 512 entries -> global bitmap), range partitions (ordered rows)."""
     n, rowptr, colidx, _ = wl.degree_ladder_graph([3, 40, 900, 1500, 6000], seed=4)
     rng = np.random.default_rng(4)
     n_parts = 20000
