@@ -95,6 +95,23 @@ class ClockSampler:
                     reasons=sorted(reasons), samples=len(sm))
 
 
+def max_over_ranks(value: float, world: int, device: str = "cuda") -> float:
+    """The slowest rank's time: what a multi-replica step takes."""
+    if world <= 1:
+        return value
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(edges_per_step: int, world: int, ms_per_step: float) -> float:
+    """Replicas only: every rank aggregates its own copy of the graph, so the job's throughput is
+    world x the per-replica edges over the slowest replica's step time."""
+    return world * edges_per_step / (ms_per_step * 1e-3)
+
+
 def build_workload(index: int, scale: float):
     from paper_2302_13053_b200 import workloads as wl
     t = time.time()
@@ -354,14 +371,10 @@ def main():
     stop.record()
     barrier()
     clocks = sampler.stop()
-    ms = start.elapsed_time(stop)
-    if world > 1:
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(start.elapsed_time(stop), world)
     ms_per_step = ms / args.steps
     edges_per_step = w.K * w.n_edges
-    value = world * edges_per_step / (ms_per_step * 1e-3)
+    value = whole_job_value(edges_per_step, world, ms_per_step)
     res = prob.results()
 
     # ---- end to end through the host-buffer entry point: H2D of all inputs and D2H of results inside
@@ -377,11 +390,7 @@ def main():
         for _ in range(args.steps):
             B.retexo_lmp_train(hprob)          # synchronises the stream before returning
         torch.cuda.synchronize()
-        dt = time.perf_counter() - t0
-        if world > 1:
-            t = torch.tensor([dt], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dt = float(t.item())
+        dt = max_over_ranks(time.perf_counter() - t0, world)
         e2e = dict(value=world * edges_per_step * args.steps / dt, unit=UNIT, ms_per_step=dt / args.steps * 1e3,
                    h2d_bytes_per_step=int(hprob.h2d_bytes), d2h_bytes_per_step=int(hprob.d2h_bytes))
         del hprob

@@ -385,8 +385,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 // (the exchange arrays and warp_loss are next written after the following tile's first
                 //  barrier-protected phase: every warp passes two more barriers before reusing them)
             } else if (BN == 64 && g.mode == TC_EPI_ARGMAX) {
-
-                // the thread owns the whole row of logits
+                // one thread owns the whole row of logits (four of the eight warps take part)
                 float v[64];
                 if (ok) {
                     uint32_t ra[32], rb[32];
@@ -410,79 +409,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                     for (int c = 0; c < 64; ++c) v[c] = 0.f;
                 }
-                const bool is_eval = g.mode == TC_EPI_SOFTMAX_CE && row >= g.n_train;
-                const bool live = ok && row < g.M && !is_eval;
+                const bool live = ok && row < g.M;
                 const int32_t yi = (live && g.y) ? g.y[row] : -1;
-                if (g.mode == TC_EPI_SOFTMAX_CE && m0 + kTcBM > g.n_train && g.n_train < g.M) {
-                    // this tile holds evaluation rows: arg-max (lowest index on ties) and hit count
-                    int best = 0;
-                    float bv = v[0];
+                int best = 0;
+                float bv = v[0];
 #pragma unroll
-                    for (int c = 1; c < 64; ++c) if (v[c] > bv) { bv = v[c]; best = c; }
-                    const bool hit = ok && is_eval && row < g.M && best == g.y_eval[row - g.n_train];
-                    const unsigned hits = __ballot_sync(0xffffffffu, hit);
-                    if (lane == 0 && hits) atomicAdd(g.correct, (unsigned long long)__popc(hits));
+                for (int c = 1; c < 64; ++c) if (v[c] > bv) { bv = v[c]; best = c; }   // strict: lowest index wins ties
+                if (live) {
+                    if (g.pred) g.pred[row] = best;
+                    if (g.out_f32) {
+#pragma unroll
+                        for (int c = 0; c < 64; ++c) if (c < g.N) g.out_f32[row * g.ld_f32 + c] = v[c];
+                    }
                 }
-                if (g.mode == TC_EPI_ARGMAX) {
-                    int best = 0;
-                    float bv = v[0];
-#pragma unroll
-                    for (int c = 1; c < 64; ++c) if (v[c] > bv) { bv = v[c]; best = c; }   // strict: lowest index wins ties
-                    if (live) {
-                        if (g.pred) g.pred[row] = best;
-                        if (g.out_f32) {
-#pragma unroll
-                            for (int c = 0; c < 64; ++c) if (c < g.N) g.out_f32[row * g.ld_f32 + c] = v[c];
-                        }
-                    }
-                    if (g.correct) {
-                        const unsigned hits = __ballot_sync(0xffffffffu, live && best == yi);
-                        if (lane == 0 && hits) atomicAdd(g.correct, (unsigned long long)__popc(hits));
-                    }
-                } else {
-                    float mx = v[0];
-#pragma unroll
-                    for (int c = 1; c < 64; ++c) mx = fmaxf(mx, v[c]);
-                    float den = 0.f, ly = 0.f;
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) {
-                        ly = c == yi ? v[c] : ly;
-                        v[c] = c < g.N ? expf(v[c] - mx) : 0.f;
-                        den += v[c];
-                    }
-                    float loss = live ? (mx + logf(den)) - ly : 0.f;
-                    const float scale = g.inv_rows / den;
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) v[c] = c < g.N ? (v[c] * scale - (c == yi ? g.inv_rows : 0.f)) : 0.f;
-                    if (live && g.out_bf16) {       // dL row-major, ld_bf16 <= 64 and a multiple of 8
-                        __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16;
-#pragma unroll
-                        for (int c = 0; c < 64; c += 8) {
-                            if (c >= g.ld_bf16) break;
-                            __nv_bfloat162 p0 = __floats2bfloat162_rn(v[c], v[c + 1]), p1 = __floats2bfloat162_rn(v[c + 2], v[c + 3]);
-                            __nv_bfloat162 p2 = __floats2bfloat162_rn(v[c + 4], v[c + 5]), p3 = __floats2bfloat162_rn(v[c + 6], v[c + 7]);
-                            uint4 pk;
-                            pk.x = *reinterpret_cast<uint32_t*>(&p0); pk.y = *reinterpret_cast<uint32_t*>(&p1);
-                            pk.z = *reinterpret_cast<uint32_t*>(&p2); pk.w = *reinterpret_cast<uint32_t*>(&p3);
-                            *reinterpret_cast<uint4*>(dst + c) = pk;
-                        }
-                    }
-                    if (ok && g.out_bf16_t) {
-#pragma unroll
-                        for (int c0 = 0; c0 < 64; c0 += 32) {
-                            if (c0 >= g.N) break;
-                            float blk[32];
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) blk[j] = v[c0 + j];
-                            store_block_transposed(g.out_bf16_t, g.ld_t, c0, g.N, row0, g.n_train, blk, stage, lane);
-                        }
-                    }
-                    loss = warp_sum(loss);
-                    if (lane == 0) warp_loss[q] = loss;
-                    asm volatile("bar.sync 1, 128;" ::: "memory");      // the four epilogue warps only
-                    if (q == 0 && lane == 0 && g.loss_partial)
-                        g.loss_partial[mt] = ((warp_loss[0] + warp_loss[1]) + warp_loss[2]) + warp_loss[3];
-                    asm volatile("bar.sync 1, 128;" ::: "memory");      // warp_loss is reused by the next tile
+                if (g.correct) {
+                    const unsigned hits = __ballot_sync(0xffffffffu, live && best == yi);
+                    if (lane == 0 && hits) atomicAdd(g.correct, (unsigned long long)__popc(hits));
                 }
             } else if (ok) {
                 // the load of chunk c + 1 is in flight while chunk c is processed
