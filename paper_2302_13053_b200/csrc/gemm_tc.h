@@ -6,7 +6,8 @@
 
 namespace retexo {
 
-enum TcEpilogue { TC_EPI_BIAS = 0, TC_EPI_PARTIAL = 1, TC_EPI_MASK_T = 2, TC_EPI_SOFTMAX_CE = 3, TC_EPI_ARGMAX = 4 };
+enum TcEpilogue { TC_EPI_BIAS = 0, TC_EPI_PARTIAL = 1, TC_EPI_MASK_T = 2, TC_EPI_SOFTMAX_CE = 3, TC_EPI_ARGMAX = 4,
+                  TC_EPI_MASK = 5 };
 
 // C[M x N] = A[M x K] * B[N x K]^T with A and B bf16, K contiguous (row strides
 // lda / ldb elements, multiples of 8; bases 16-byte aligned).
@@ -21,6 +22,7 @@ enum TcEpilogue { TC_EPI_BIAS = 0, TC_EPI_PARTIAL = 1, TC_EPI_MASK_T = 2, TC_EPI
 //   TC_EPI_MASK_T : out_bf16_t[n][m] = acc[m][n] where mask[m][n] > 0 (bf16, row stride
 //                   ld_mask), else 0: the ReLU gate applied to a back-propagated gradient,
 //                   stored transposed.
+//   TC_EPI_MASK   : out_bf16[m][n] = acc[m][n] where mask[m][n] > 0, else 0 (same gate, everything row-major).
 //   TC_EPI_SOFTMAX_CE (N <= 64): logits = acc + bias; per row the softmax cross-entropy against
 //                   label y[m] and its gradient dL = (softmax - onehot) * inv_rows, written as bf16
 //                   row-major (out_bf16, ld_bf16 a multiple of 8, padding columns zero) and

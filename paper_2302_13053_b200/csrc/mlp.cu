@@ -6,7 +6,7 @@
 // hence the transposed copies kept next to the row-major ones:
 //   forward   Hd  = ReLU(X W1 + b1)           A = X        B = W1^T
 //             L   = Hd W2 + b2                A = Hd       B = W2^T
-//   backward  dHd = (dL W2^T) .* [Hd > 0]     A = dL       B = W2 (rows padded)   -> stored as dHd^T
+//   backward  dHd^T = (W2 dL^T) .* [Hd^T > 0] A = W2 (rows padded)   B = dL
 //             [dW2 ; db2] = [Hd^T ; 1] dL     A = [Hd^T;1] B = dL^T               split over the batch
 //             [dW1 ; db1] = [X^T ; 1] dHd     A = [X^T;1]  B = dHd^T              split over the batch
 // The all-ones row turns each bias gradient into one more output row, so the
@@ -234,8 +234,10 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     // ---- backward
     const bf16* grad1_t = b.dlt16;      // gradient at the first layer's output, transposed
     if (H > 0) {
-        TcGemm bk = tc_base(b.dl16, p.ld_dl, b.w2p16, p.ld_dl, n, H, O, b.status);
-        bk.mode = TC_EPI_MASK_T; bk.mask = b.hd16; bk.ld_mask = p.ld_h; bk.out_bf16_t = b.dhdt16; bk.ld_t = p.ld_n;
+        // dHd^T = W2 dL^T, gated by Hd^T > 0: computed directly in the transposed orientation the weight
+        // gradient reads, so mask and output are both row-major for the epilogue
+        TcGemm bk = tc_base(b.w2p16, p.ld_dl, b.dl16, p.ld_dl, H, n, O, b.status);
+        bk.mode = TC_EPI_MASK; bk.mask = b.hdt16; bk.ld_mask = p.ld_n; bk.out_bf16 = b.dhdt16; bk.ld_bf16 = p.ld_n;
         RETEXO_TRY(tc_gemm_launch(bk, st));
         TcGemm g2 = tc_base(b.hdt16, p.ld_n, b.dlt16, p.ld_n, (int64_t)H + 1, O, n, b.status);
         g2.mode = TC_EPI_PARTIAL; g2.splits = (int)p.split_w2; g2.partial = b.pw2;
