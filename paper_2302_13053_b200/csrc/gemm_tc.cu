@@ -457,7 +457,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                             for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __uint_as_float(r[j]);
                         }
-                    } else if (g.mode == TC_EPI_MASK_T) {
+                    } else if (g.mode == TC_EPI_MASK_T || g.mode == TC_EPI_MASK) {
                         float v[32];
                         if (row < g.M) {
                             const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
@@ -479,7 +479,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] = 0.f;
                         }
-                        store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane);
+                        if (g.mode == TC_EPI_MASK_T) {
+                            store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane);
+                        } else if (col0 + 32 <= g.N && (g.ld_bf16 & 7) == 0 && aligned16(g.out_bf16)) {
+                            store_block_rows(g.out_bf16, g.ld_bf16, col0, row0, g.M, v, stage, lane);
+                        } else if (row < g.M) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + j < g.N) g.out_bf16[row * g.ld_bf16 + col0 + j] = __float2bfloat16_rn(v[j]);
+                        }
                     } else {
                         float v[32];
                         // one coalesced bias load per chunk, handed round by shuffles (32 same-address loads per
@@ -598,6 +606,7 @@ static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& 
 bool tc_gemm_supported(const TcGemm& t) {
     if (t.M <= 0 || t.N <= 0 || t.K <= 0) return false;
     if (t.mode == TC_EPI_MASK_T && (!t.mask || !t.out_bf16_t)) return false;
+    if (t.mode == TC_EPI_MASK && (!t.mask || !t.out_bf16)) return false;
     if (t.mode == TC_EPI_PARTIAL && !t.partial) return false;
     if ((t.mode == TC_EPI_SOFTMAX_CE || t.mode == TC_EPI_ARGMAX) && t.N > 64) return false;
     if (t.mode == TC_EPI_SOFTMAX_CE && (!t.y || (t.out_bf16 && (t.ld_bf16 % 8 != 0 || t.ld_bf16 > 64)))) return false;
