@@ -22,7 +22,7 @@ _SRC = os.path.join(_HERE, "retexo_oracle.c")
 _LIB = os.path.join(_HERE, "libretexo_oracle.so")
 _lib = None
 
-GCN, SAGE_MEAN, GAT = 0, 1, 2
+GCN, SAGE_MEAN, GAT, SAGE_MAX = 0, 1, 2, 3
 SGD, ADAM = 0, 1
 
 
@@ -76,7 +76,7 @@ def aggregate(aggr: int, rowptr: np.ndarray, colidx: np.ndarray, q: np.ndarray,
               return_alpha: bool = False):
     """AGGR (+ COMBINE) of Eq. 1 for all nodes, or for the listed `rows`.
 
-    GCN -> [n, d]; SAGE_MEAN -> [n, 2d] (self | mean); GAT -> [n, heads*dh]
+    GCN -> [n, d]; SAGE_MEAN / SAGE_MAX -> [n, 2d] (self | mean or max); GAT -> [n, heads*dh]
     (q is the projected input; gat = dict(heads, head_dim, a_src, a_dst,
     negative_slope, add_self_loop))."""
     n = rowptr.shape[0] - 1
@@ -99,6 +99,13 @@ def aggregate(aggr: int, rowptr: np.ndarray, colidx: np.ndarray, q: np.ndarray,
                                           C.c_int32(dim), _p(out), C.c_int64(2 * dim), _p(rows_a),
                                           C.c_int64(cnt))
         _check(rc, "oracle_aggregate_sage_mean")
+        return out
+    if aggr == SAGE_MAX:
+        out = np.zeros((cnt, 2 * dim), dtype=np.float32)
+        rc = L.oracle_aggregate_sage_max(C.c_int64(n), _p(rowptr), _p(colidx), _p(q), C.c_int64(q.shape[1]),
+                                         C.c_int32(dim), _p(out), C.c_int64(2 * dim), _p(rows_a),
+                                         C.c_int64(cnt))
+        _check(rc, "oracle_aggregate_sage_max")
         return out
     if aggr == GAT:
         heads, dh = int(gat["heads"]), int(gat["head_dim"])

@@ -124,6 +124,34 @@ int oracle_aggregate_sage_mean(int64_t n, const int64_t *rowptr, const int32_t *
     return failed ? ORACLE_NO_MEM : ORACLE_OK;
 }
 
+/* GraphSAGE with the max-pooling aggregator named in Section 2.2, COMBINE =
+ * concatenation: columns [0,dim) are the node's own row, column dim+j the
+ * largest q[u][j] over u in N(v) (v itself excluded); a node without
+ * neighbours gets zeros.  The pooling layer's own transform is not part of
+ * this function: q is taken as already transformed. */
+int oracle_aggregate_sage_max(int64_t n, const int64_t *rowptr, const int32_t *colidx,
+                              const float *q, int64_t ldq, int32_t dim,
+                              float *out, int64_t ldout,
+                              const int64_t *rows, int64_t n_rows)
+{
+    if (n < 0 || dim < 0 || ldq < dim || ldout < 2 * (int64_t)dim) return ORACLE_BAD_ARG;
+    int64_t cnt = rows ? n_rows : n;
+#pragma omp parallel for schedule(dynamic, 64)
+    for (int64_t i = 0; i < cnt; ++i) {
+        int64_t v = rows ? rows[i] : i;
+        for (int32_t j = 0; j < dim; ++j) {
+            float best = 0.0f;
+            for (int64_t e = rowptr[v]; e < rowptr[v + 1]; ++e) {
+                float x = q[(int64_t)colidx[e] * ldq + j];
+                if (e == rowptr[v] || x > best) best = x;
+            }
+            out[i * ldout + j] = q[v * ldq + j];
+            out[i * ldout + dim + j] = best;
+        }
+    }
+    return ORACLE_OK;
+}
+
 /* GAT (cited in Section 2.2; formula of the cited layer).  p holds the
  * already projected rows, heads*head_dim wide, head k in columns
  * [k*head_dim, (k+1)*head_dim).  For destination v and head k:

@@ -115,11 +115,51 @@ def test_sage_mean_of_constant_is_constant_and_star_closed_form():
     np.testing.assert_array_equal(got[1:, 2:], np.repeat(q[:1], 8, 0))  # leaf = centre
 
 
+@pytest.mark.parametrize("name,rowptr,colidx", GRAPHS, ids=[g[0] for g in GRAPHS])
+def test_sage_max_matches_dense_masked_maximum(name, rowptr, colidx):
+    """Max-pooling aggregator (Section 2.2): brute force over the dense
+    adjacency; all-negative features catch a maximum started at zero."""
+    n = rowptr.shape[0] - 1
+    rng = np.random.default_rng(8)
+    q = (rng.standard_normal((n, 5)) - 3.0).astype(np.float32)
+    a = dense_adj(rowptr, colidx) > 0
+    got = oracle.aggregate(oracle.SAGE_MAX, rowptr, colidx, q)
+    assert got.shape == (n, 10)
+    np.testing.assert_array_equal(got[:, :5], q)
+    for v in range(n):
+        want = q[a[v]].max(0) if a[v].any() else np.zeros(5, dtype=np.float32)
+        np.testing.assert_array_equal(got[v, 5:], want)
+
+
+def test_sage_max_star_ring_and_monotone_map():
+    rowptr, colidx = wl.star_graph(8)
+    q = np.random.default_rng(3).standard_normal((9, 4)).astype(np.float32)
+    got = oracle.aggregate(oracle.SAGE_MAX, rowptr, colidx, q)
+    np.testing.assert_array_equal(got[0, 4:], q[1:].max(0))            # centre = max over leaves
+    np.testing.assert_array_equal(got[1:, 4:], np.repeat(q[:1], 8, 0))  # leaf = centre's row
+    rowptr, colidx = wl.ring_graph(12)
+    q = np.random.default_rng(4).standard_normal((12, 3)).astype(np.float32)
+    got = oracle.aggregate(oracle.SAGE_MAX, rowptr, colidx, q)[:, 3:]
+    np.testing.assert_array_equal(got, np.maximum(np.roll(q, 1, 0), np.roll(q, -1, 0)))
+    # max commutes with an increasing map; min is max of the negation
+    rowptr, colidx = wl.random_small_graph(50, 45, seed=6)
+    q = np.random.default_rng(6).standard_normal((50, 4)).astype(np.float32)
+    deg = np.diff(rowptr)
+    base = oracle.aggregate(oracle.SAGE_MAX, rowptr, colidx, q)[:, 4:]
+    cubed = oracle.aggregate(oracle.SAGE_MAX, rowptr, colidx, q ** 3)[:, 4:]
+    np.testing.assert_array_equal(cubed[deg > 0], (base ** 3)[deg > 0])
+    mean = oracle.aggregate(oracle.SAGE_MEAN, rowptr, colidx, q)[:, 4:]
+    assert np.all(base[deg > 0] >= mean[deg > 0] - 1e-6)               # max >= mean
+    one = deg == 1
+    assert one.any()
+    np.testing.assert_allclose(base[one], mean[one], rtol=1e-6)          # single neighbour: both are its row
+
+
 def test_rows_subset_equals_full_result():
     rowptr, colidx = wl.random_small_graph(64, 300, seed=9)
     q = np.random.default_rng(9).standard_normal((64, 5)).astype(np.float32)
     rows = np.array([63, 0, 17, 17, 5])
-    for aggr in (oracle.GCN, oracle.SAGE_MEAN):
+    for aggr in (oracle.GCN, oracle.SAGE_MEAN, oracle.SAGE_MAX):
         full = oracle.aggregate(aggr, rowptr, colidx, q)
         np.testing.assert_array_equal(oracle.aggregate(aggr, rowptr, colidx, q, rows=rows), full[rows])
     gat = dict(heads=1, head_dim=5, a_src=np.ones((1, 5)), a_dst=np.ones((1, 5)))
