@@ -77,7 +77,7 @@ typedef struct retexo_csr {
 int retexo_validate_csr(const retexo_csr* g, int64_t* status_out, void* stream);
 
 /* ------------------------------------------------------------ aggregation */
-typedef enum retexo_aggr { RETEXO_GCN = 0, RETEXO_SAGE_MEAN = 1, RETEXO_GAT = 2 } retexo_aggr;
+typedef enum retexo_aggr { RETEXO_GCN = 0, RETEXO_SAGE_MEAN = 1, RETEXO_GAT = 2, RETEXO_SAGE_MAX = 3 } retexo_aggr;
 
 typedef struct retexo_gat_params {
     int32_t heads, head_dim;        /* dim must equal heads * head_dim; heads <= 8 */
@@ -100,6 +100,12 @@ size_t retexo_aggregate_workspace_size(int64_t n_nodes, int64_t n_edges, int32_t
  *                    q[v] in columns [0,dim) and the mean in [dim, 2 dim)
  *                    (COMBINE = concatenation); concat_self = 0: out is
  *                    [n x dim], the mean only.
+ *   RETEXO_SAGE_MAX  the max-pooling aggregator Section 2.2 names for
+ *                    GraphSAGE: max[v][j] = max_{u in N(v)} q[u][j], zeros
+ *                    if deg v = 0; the pooling layer's own transform is not
+ *                    applied here (q is taken as already transformed).  Same
+ *                    output layout and concat_self rule as RETEXO_SAGE_MEAN.
+ *                    Exact (no rounding) for finite q.
  *   RETEXO_GAT       q holds already projected rows, head k in columns
  *                    [k*head_dim, (k+1)*head_dim).  Per head:
  *                    e_uv = LeakyReLU(<a_src,q_u> + <a_dst,q_v>),

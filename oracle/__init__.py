@@ -239,6 +239,43 @@ def cross_partition(rowptr: np.ndarray, colidx: np.ndarray, part: np.ndarray, n_
                 dv_lazy_lt=2 * int(bt.value))
 
 
+# ---------------------------------------------------------------- analytical data volume
+def data_volume(H: Sequence[float], L: Sequence[float], n_workers: float, B: float, R: float) -> Dict:
+    """Network data volume of the analysis in Section 3.3 / Appendix A.1, in
+    elements.  H = [H_0 .. H_K] representation widths, L = [L_1 .. L_K] layer
+    sizes (their sum is the model size M), B boundary nodes per worker, R
+    training iterations.  Each of the four volumes is written out as its own
+    sum of messages; gamma is the ratio of the totals."""
+    K = len(L)
+    assert len(H) == K + 1 and K >= 1
+    n = n_workers
+    M = 0.0
+    for m in range(1, K + 1):
+        M += L[m - 1]
+    # lazy, local training: one exchange before each layer, widths H_0 .. H_{K-1}, both directions
+    lazy_lt = 0.0
+    for m in range(0, K):
+        lazy_lt += 2 * n * B * H[m]
+    # standard, local training: each iteration sends H_1 .. H_{K-1} forward and as many gradients back;
+    # the features are sent once and cached
+    std_lt = 2 * n * B * H[0]
+    for _ in range(int(R)):
+        for m in range(1, K):
+            std_lt += 2 * n * B * H[m]        # forward
+            std_lt += 2 * n * B * H[m]        # backward
+    # gradient aggregation: every iteration each worker sends and receives what it trains
+    std_red = 0.0
+    for _ in range(int(R)):
+        std_red += n * M + n * M
+    lazy_red = 0.0
+    for m in range(1, K + 1):
+        trained = L[m - 1] + (H[m] * H[K] if m < K else 0.0)      # the layer and its temporary classifier C_m
+        for _ in range(int(R)):
+            lazy_red += 2 * n * trained
+    return dict(lazy_lt=lazy_lt, standard_lt=std_lt, lazy_reduce=lazy_red, standard_reduce=std_red,
+                gamma=(std_lt + std_red) / (lazy_lt + lazy_red), model_size=M)
+
+
 # ---------------------------------------------------------------- the K-round loop
 def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
               rowptr, colidx, features, labels, train_idx, val_idx, test_idx,

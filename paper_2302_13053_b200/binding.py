@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libretexo.so")
 _lib = None
 
-GCN, SAGE_MEAN, GAT = 0, 1, 2
+GCN, SAGE_MEAN, GAT, SAGE_MAX = 0, 1, 2, 3
 SGD, ADAM = 0, 1
 
 
@@ -138,7 +138,7 @@ def retexo_aggregate(aggr: int, rowptr: torch.Tensor, colidx: torch.Tensor, q: t
     assert q.dtype == torch.float32 and q.stride(1) == 1
     n = rowptr.numel() - 1
     dim = int(q.shape[1] if dim is None else dim)
-    width = 2 * dim if (aggr == SAGE_MEAN and concat_self) else dim
+    width = 2 * dim if (aggr in (SAGE_MEAN, SAGE_MAX) and concat_self) else dim
     dev = q.device
     if want_f32 and out is None:
         out = torch.empty((n, width), dtype=torch.float32, device=dev)

@@ -72,6 +72,24 @@ __device__ __forceinline__ void vec_add(float4& a, const float4& x) { a.x += x.x
 __device__ __forceinline__ void vec_add(float2& a, const float2& x) { a.x += x.x; a.y += x.y; }
 __device__ __forceinline__ void vec_add(float& a, const float& x) { a += x; }
 
+__device__ __forceinline__ void vec_max(float4& a, const float4& x) {
+    a.x = fmaxf(a.x, x.x); a.y = fmaxf(a.y, x.y); a.z = fmaxf(a.z, x.z); a.w = fmaxf(a.w, x.w);
+}
+__device__ __forceinline__ void vec_max(float2& a, const float2& x) { a.x = fmaxf(a.x, x.x); a.y = fmaxf(a.y, x.y); }
+__device__ __forceinline__ void vec_max(float& a, const float& x) { a = fmaxf(a, x); }
+
+// What a row's accumulator does with a neighbour row: plain sum (SAGE mean),
+// sum weighted by coef[u] (GCN), or element-wise maximum (SAGE max-pooling).
+constexpr int kOpSum = 0, kOpGcn = 1, kOpMax = 2;
+
+template <int VEC, int OP>
+__device__ __forceinline__ void vec_init(typename VecT<VEC>::type& a) {
+    if constexpr (OP != kOpMax) vec_zero<VEC>(a);
+    else if constexpr (VEC == 4) a = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    else if constexpr (VEC == 2) a = make_float2(-INFINITY, -INFINITY);
+    else a = -INFINITY;
+}
+
 template <int VEC>
 __device__ __forceinline__ float vec_get(const typename VecT<VEC>::type& a, int i);
 template <> __device__ __forceinline__ float vec_get<4>(const float4& a, int i) {
@@ -103,7 +121,7 @@ struct AggArgs {
 
 // Adds the neighbour rows of CSR entries [beg, end) into acc, in order, for the
 // column vectors this lane owns in pass `pass`.  GCN weighs each row by coef[u].
-template <int VEC, int CH, bool GCN>
+template <int VEC, int CH, int OP>
 __device__ __forceinline__ void accumulate_range(const AggArgs& a, int64_t beg, int64_t end, int lane,
                                                  int vec0, int nvec,
                                                  typename VecT<VEC>::type (&acc)[CH]) {
@@ -116,7 +134,7 @@ __device__ __forceinline__ void accumulate_range(const AggArgs& a, int64_t beg, 
         float my_w = 0.f;
         if (lane < cnt) {
             my_u = __ldg(a.colidx + e0 + lane);
-            if (GCN) my_w = __ldg(a.coef + my_u);
+            if (OP == kOpGcn) my_w = __ldg(a.coef + my_u);
         }
         int j = 0;
         for (; j + kUnroll <= cnt; j += kUnroll) {
@@ -125,7 +143,7 @@ __device__ __forceinline__ void accumulate_range(const AggArgs& a, int64_t beg, 
 #pragma unroll
             for (int t = 0; t < kUnroll; ++t) {
                 const int u = __shfl_sync(0xffffffffu, my_u, j + t);
-                if (GCN) w[t] = __shfl_sync(0xffffffffu, my_w, j + t);
+                if (OP == kOpGcn) w[t] = __shfl_sync(0xffffffffu, my_w, j + t);
                 const V* row = qv + (int64_t)u * ldv;
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
@@ -138,21 +156,23 @@ __device__ __forceinline__ void accumulate_range(const AggArgs& a, int64_t beg, 
             for (int t = 0; t < kUnroll; ++t)
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
-                    if (GCN) vec_fma(acc[c], w[t], x[t][c]);
+                    if (OP == kOpGcn) vec_fma(acc[c], w[t], x[t][c]);
+                    else if (OP == kOpMax) vec_max(acc[c], x[t][c]);
                     else vec_add(acc[c], x[t][c]);
                 }
         }
         for (; j < cnt; ++j) {
             const int u = __shfl_sync(0xffffffffu, my_u, j);
             float w = 0.f;
-            if (GCN) w = __shfl_sync(0xffffffffu, my_w, j);
+            if (OP == kOpGcn) w = __shfl_sync(0xffffffffu, my_w, j);
             const V* row = qv + (int64_t)u * ldv;
 #pragma unroll
             for (int c = 0; c < CH; ++c) {
                 const int vi = vec0 + c * kWarp + lane;
                 if (vi < nvec) {
                     V x = __ldg(row + vi);
-                    if (GCN) vec_fma(acc[c], w, x);
+                    if (OP == kOpGcn) vec_fma(acc[c], w, x);
+                    else if (OP == kOpMax) vec_max(acc[c], x);
                     else vec_add(acc[c], x);
                 }
             }
@@ -167,7 +187,7 @@ __device__ __forceinline__ void store_elem(const AggArgs& a, int64_t v, int col,
 
 // Finishes row v for the column vectors of this lane: GCN adds the self term
 // and scales, SAGE divides by the degree and (optionally) copies the self row.
-template <int VEC, int CH, bool GCN>
+template <int VEC, int CH, int OP>
 __device__ __forceinline__ void finish_row(const AggArgs& a, int64_t v, int lane, int vec0, int nvec,
                                            typename VecT<VEC>::type (&acc)[CH]) {
     using V = typename VecT<VEC>::type;
@@ -185,10 +205,10 @@ __device__ __forceinline__ void finish_row(const AggArgs& a, int64_t v, int lane
             if (col >= a.dim) continue;
             const float sv = vec_get<VEC>(s, i);
             const float av = vec_get<VEC>(acc[c], i);
-            if (GCN) {
+            if (OP == kOpGcn) {
                 store_elem(a, v, col, cv * fmaf(cv, sv, av));
             } else {
-                const float mean = deg > 0 ? av / (float)deg : 0.0f;
+                const float mean = deg <= 0 ? 0.0f : OP == kOpMax ? av : av / (float)deg;
                 if (a.concat_self) {
                     store_elem(a, v, col, sv);
                     store_elem(a, v, a.dim + col, mean);
@@ -204,7 +224,7 @@ __device__ __forceinline__ void finish_row(const AggArgs& a, int64_t v, int lane
 // [0, n_seg) are segments of heavy rows (their raw sums go to scratch), items
 // [n_seg, n_seg + n) are whole rows (heavy ones are skipped: their segments
 // cover them).
-template <int VEC, int CH, bool GCN>
+template <int VEC, int CH, int OP>
 __global__ void __launch_bounds__(kAggThreads) agg_rows_kernel(AggArgs a) {
     using V = typename VecT<VEC>::type;
     const int lane = threadIdx.x & 31;
@@ -225,8 +245,8 @@ __global__ void __launch_bounds__(kAggThreads) agg_rows_kernel(AggArgs a) {
             for (int vec0 = 0; vec0 < nvec; vec0 += CH * kWarp) {
                 V acc[CH];
 #pragma unroll
-                for (int c = 0; c < CH; ++c) vec_zero<VEC>(acc[c]);
-                accumulate_range<VEC, CH, GCN>(a, beg, end, lane, vec0, nvec, acc);
+                for (int c = 0; c < CH; ++c) vec_init<VEC, OP>(acc[c]);
+                accumulate_range<VEC, CH, OP>(a, beg, end, lane, vec0, nvec, acc);
                 float* dst = a.seg_partial + item * a.ld_partial;
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
@@ -243,9 +263,9 @@ __global__ void __launch_bounds__(kAggThreads) agg_rows_kernel(AggArgs a) {
             for (int vec0 = 0; vec0 < nvec; vec0 += CH * kWarp) {
                 V acc[CH];
 #pragma unroll
-                for (int c = 0; c < CH; ++c) vec_zero<VEC>(acc[c]);
-                accumulate_range<VEC, CH, GCN>(a, beg, end, lane, vec0, nvec, acc);
-                finish_row<VEC, CH, GCN>(a, v, lane, vec0, nvec, acc);
+                for (int c = 0; c < CH; ++c) vec_init<VEC, OP>(acc[c]);
+                accumulate_range<VEC, CH, OP>(a, beg, end, lane, vec0, nvec, acc);
+                finish_row<VEC, CH, OP>(a, v, lane, vec0, nvec, acc);
             }
         }
     }
@@ -253,7 +273,7 @@ __global__ void __launch_bounds__(kAggThreads) agg_rows_kernel(AggArgs a) {
 
 // One warp per heavy row: adds the row's segment sums in segment order and
 // finishes the row.
-template <int VEC, int CH, bool GCN>
+template <int VEC, int CH, int OP>
 __global__ void __launch_bounds__(kAggThreads) agg_combine_kernel(AggArgs a) {
     using V = typename VecT<VEC>::type;
     const int lane = threadIdx.x & 31;
@@ -267,7 +287,7 @@ __global__ void __launch_bounds__(kAggThreads) agg_combine_kernel(AggArgs a) {
         for (int vec0 = 0; vec0 < nvec; vec0 += CH * kWarp) {
             V acc[CH];
 #pragma unroll
-            for (int c = 0; c < CH; ++c) vec_zero<VEC>(acc[c]);
+            for (int c = 0; c < CH; ++c) vec_init<VEC, OP>(acc[c]);
             for (int i = 0; i < nseg; ++i) {
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
@@ -280,37 +300,45 @@ __global__ void __launch_bounds__(kAggThreads) agg_combine_kernel(AggArgs a) {
                     if constexpr (VEC == 4) x = make_float4(t[0], t[1], t[2], t[3]);
                     else if constexpr (VEC == 2) x = make_float2(t[0], t[1]);
                     else x = t[0];
-                    vec_add(acc[c], x);
+                    if (OP == kOpMax) vec_max(acc[c], x);
+                    else vec_add(acc[c], x);
                 }
             }
-            finish_row<VEC, CH, GCN>(a, v, lane, vec0, nvec, acc);
+            finish_row<VEC, CH, OP>(a, v, lane, vec0, nvec, acc);
         }
     }
 }
 
-template <int VEC, int CH, bool GCN>
+template <int VEC, int CH, int OP>
 static int launch_agg(const AggArgs& a, int n_sm, cudaStream_t st) {
     int per_sm = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, agg_rows_kernel<VEC, CH, GCN>, kAggThreads, 0) !=
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, agg_rows_kernel<VEC, CH, OP>, kAggThreads, 0) !=
             cudaSuccess || per_sm < 1) {
         (void)cudaGetLastError();
         per_sm = 1;
     }
-    agg_rows_kernel<VEC, CH, GCN><<<n_sm * per_sm, kAggThreads, 0, st>>>(a);
-    agg_combine_kernel<VEC, CH, GCN><<<n_sm, kAggThreads, 0, st>>>(a);
+    agg_rows_kernel<VEC, CH, OP><<<n_sm * per_sm, kAggThreads, 0, st>>>(a);
+    agg_combine_kernel<VEC, CH, OP><<<n_sm, kAggThreads, 0, st>>>(a);
     return launch_status();
 }
 
-template <int VEC, bool GCN>
+template <int VEC, int OP>
 static int dispatch_ch(const AggArgs& a, int n_sm, cudaStream_t st) {
     const int nvec = (a.dim + VEC - 1) / VEC;
     const int need = (nvec + kWarp - 1) / kWarp;      // column chunks for one pass
-    if (need <= 1) return launch_agg<VEC, 1, GCN>(a, n_sm, st);
-    if (need <= 2) return launch_agg<VEC, 2, GCN>(a, n_sm, st);
-    if (need <= 3) return launch_agg<VEC, 3, GCN>(a, n_sm, st);
-    if (need <= 4) return launch_agg<VEC, 4, GCN>(a, n_sm, st);
-    if (need <= 5) return launch_agg<VEC, 5, GCN>(a, n_sm, st);
-    return launch_agg<VEC, 6, GCN>(a, n_sm, st);      // wider rows: several passes of 6 chunks
+    if (need <= 1) return launch_agg<VEC, 1, OP>(a, n_sm, st);
+    if (need <= 2) return launch_agg<VEC, 2, OP>(a, n_sm, st);
+    if (need <= 3) return launch_agg<VEC, 3, OP>(a, n_sm, st);
+    if (need <= 4) return launch_agg<VEC, 4, OP>(a, n_sm, st);
+    if (need <= 5) return launch_agg<VEC, 5, OP>(a, n_sm, st);
+    return launch_agg<VEC, 6, OP>(a, n_sm, st);      // wider rows: several passes of 6 chunks
+}
+
+template <int VEC>
+static int dispatch_op(int op, const AggArgs& a, int n_sm, cudaStream_t st) {
+    if (op == kOpGcn) return dispatch_ch<VEC, kOpGcn>(a, n_sm, st);
+    if (op == kOpMax) return dispatch_ch<VEC, kOpMax>(a, n_sm, st);
+    return dispatch_ch<VEC, kOpSum>(a, n_sm, st);
 }
 
 // ---------------------------------------------------------------- GAT
@@ -473,12 +501,14 @@ extern "C" int retexo_aggregate(const retexo_csr* g, int32_t type, const float* 
                                 int32_t concat_self, void* out_bf16, int64_t ldout_bf16,
                                 void* workspace, size_t workspace_bytes, void* stream) {
     if (!g || g->n_nodes < 0 || g->n_edges < 0 || g->n_nodes > INT32_MAX) return RETEXO_ERR_INVALID_ARG;
-    if (type != RETEXO_GCN && type != RETEXO_SAGE_MEAN && type != RETEXO_GAT) return RETEXO_ERR_INVALID_ARG;
+    if (type != RETEXO_GCN && type != RETEXO_SAGE_MEAN && type != RETEXO_GAT && type != RETEXO_SAGE_MAX)
+        return RETEXO_ERR_INVALID_ARG;
     if (dim <= 0 || ldq < dim) return RETEXO_ERR_INVALID_ARG;
     if (g->n_nodes == 0) return RETEXO_OK;                      // nothing to aggregate
     if (!out && !out_bf16) return RETEXO_ERR_INVALID_ARG;
     if (!g->rowptr || !q || (g->n_edges > 0 && !g->colidx)) return RETEXO_ERR_INVALID_ARG;
-    const int64_t width = (type == RETEXO_SAGE_MEAN && concat_self) ? 2 * (int64_t)dim : dim;
+    const bool sage = type == RETEXO_SAGE_MEAN || type == RETEXO_SAGE_MAX;
+    const int64_t width = (sage && concat_self) ? 2 * (int64_t)dim : dim;
     if (out && ldout < width) return RETEXO_ERR_INVALID_ARG;
     if (out_bf16 && ldout_bf16 < width) return RETEXO_ERR_INVALID_ARG;
     if (dim > 4096) return RETEXO_ERR_UNSUPPORTED;
@@ -534,10 +564,10 @@ extern "C" int retexo_aggregate(const retexo_csr* g, int32_t type, const float* 
     prep_rows_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(n, g->rowptr, type, coef, heavy_list,
                                                                   heavy_seg_base, seg_slot, counters);
 
-    const bool gcn = type == RETEXO_GCN;
+    const int op = type == RETEXO_GCN ? kOpGcn : type == RETEXO_SAGE_MAX ? kOpMax : kOpSum;
     const bool v4 = aligned_to(q, 16) && ldq % 4 == 0 && ldq >= (dim + 3) / 4 * 4;
     const bool v2 = aligned_to(q, 8) && ldq % 2 == 0 && ldq >= (dim + 1) / 2 * 2;
-    if (v4) return gcn ? dispatch_ch<4, true>(a, n_sm, st) : dispatch_ch<4, false>(a, n_sm, st);
-    if (v2) return gcn ? dispatch_ch<2, true>(a, n_sm, st) : dispatch_ch<2, false>(a, n_sm, st);
-    return gcn ? dispatch_ch<1, true>(a, n_sm, st) : dispatch_ch<1, false>(a, n_sm, st);
+    if (v4) return dispatch_op<4>(op, a, n_sm, st);
+    if (v2) return dispatch_op<2>(op, a, n_sm, st);
+    return dispatch_op<1>(op, a, n_sm, st);
 }

@@ -59,7 +59,7 @@ static RoundDims round_dims(const retexo_lmp_config& c, int m /*1-based*/) {
     RoundDims r;
     r.rep_dim = m == 1 ? c.d0 : c.hidden;
     if (c.aggr == RETEXO_GAT) { r.agg_dim = c.gat_heads * c.gat_head_dim; r.d_in = r.agg_dim; }
-    else if (c.aggr == RETEXO_SAGE_MEAN) { r.agg_dim = r.rep_dim; r.d_in = 2 * r.rep_dim; }
+    else if (c.aggr == RETEXO_SAGE_MEAN || c.aggr == RETEXO_SAGE_MAX) { r.agg_dim = r.rep_dim; r.d_in = 2 * r.rep_dim; }
     else { r.agg_dim = r.rep_dim; r.d_in = r.rep_dim; }
     r.hidden = m < c.K ? c.hidden : 0;
     return r;
@@ -175,7 +175,8 @@ static int check_cfg(const retexo_lmp_config* c) {
     if (!c) return RETEXO_ERR_INVALID_ARG;
     if (c->K < 1 || c->K > 8 || c->R < 1 || c->d0 <= 0 || c->n_classes <= 0) return RETEXO_ERR_INVALID_ARG;
     if (c->K > 1 && c->hidden <= 0) return RETEXO_ERR_INVALID_ARG;
-    if (c->aggr != RETEXO_GCN && c->aggr != RETEXO_SAGE_MEAN && c->aggr != RETEXO_GAT) return RETEXO_ERR_INVALID_ARG;
+    if (c->aggr != RETEXO_GCN && c->aggr != RETEXO_SAGE_MEAN && c->aggr != RETEXO_GAT && c->aggr != RETEXO_SAGE_MAX)
+        return RETEXO_ERR_INVALID_ARG;
     if (c->aggr == RETEXO_GAT && (c->gat_heads <= 0 || c->gat_head_dim <= 0)) return RETEXO_ERR_INVALID_ARG;
     if (c->eval_every < 1) return RETEXO_ERR_INVALID_ARG;
     if (c->n_classes > 64 || c->hidden > 512) return RETEXO_ERR_UNSUPPORTED;

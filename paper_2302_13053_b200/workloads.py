@@ -18,14 +18,14 @@ from typing import Dict, List, Optional
 
 import numpy as np
 
-GCN, SAGE_MEAN, GAT = 0, 1, 2
-AGGR_NAMES = {GCN: "gcn", SAGE_MEAN: "sage_mean", GAT: "gat"}
+GCN, SAGE_MEAN, GAT, SAGE_MAX = 0, 1, 2, 3
+AGGR_NAMES = {GCN: "gcn", SAGE_MEAN: "sage_mean", GAT: "gat", SAGE_MAX: "sage_max"}
 
 
 @dataclass
 class Workload:
     name: str
-    aggr: int                 # GCN / SAGE_MEAN / GAT
+    aggr: int                 # GCN / SAGE_MEAN / GAT / SAGE_MAX
     K: int                    # rounds = GNN layers
     R: int                    # training iterations per round
     hidden: int
@@ -65,7 +65,7 @@ class Workload:
             if self.aggr == GAT:
                 agg_in = self.heads * self.head_dim      # projected width
                 d_in = agg_in
-            elif self.aggr == SAGE_MEAN:
+            elif self.aggr in (SAGE_MEAN, SAGE_MAX):
                 agg_in = d_prev
                 d_in = 2 * d_prev
             else:

@@ -69,6 +69,33 @@ def test_empty_and_edgeless_graphs(aggr):
     assert out.shape[0] == 0
 
 
+@pytest.mark.parametrize("dim,ld", [(1, 1), (3, 3), (5, 8), (100, 100), (127, 128), (602, 608), (256, 256),
+                                    (1433, 1436), (769, 772)])
+def test_max_pooling_is_bit_exact_over_every_degree_bin(dim, ld):
+    """A maximum involves no rounding: every element must equal the checker's,
+    signed features included (heavy rows are cut into segments here too)."""
+    n, rowptr, colidx, _ = wl.degree_ladder_graph(LADDER, seed=dim)
+    q = (np.random.default_rng(dim).standard_normal((n, dim)) - 1.0).astype(np.float32)
+    ref = oracle.aggregate(oracle.SAGE_MAX, rowptr, colidx, q)
+    got, got16 = run_gpu(oracle.SAGE_MAX, rowptr, colidx, q, ld=ld)
+    np.testing.assert_array_equal(got, ref)
+    np.testing.assert_array_equal(got16[:, :got.shape[1]],
+                                  torch.from_numpy(got).to(torch.bfloat16).float().numpy())
+    only, _ = run_gpu(oracle.SAGE_MAX, rowptr, colidx, q, ld=ld, concat_self=False)
+    np.testing.assert_array_equal(only, ref[:, dim:])
+
+
+def test_max_pooling_on_a_power_law_graph_and_edgeless_rows():
+    w = wl.make_config(5, scale=0.01)
+    ref = oracle.aggregate(oracle.SAGE_MAX, w.rowptr, w.colidx, w.features)
+    got, _ = run_gpu(oracle.SAGE_MAX, w.rowptr, w.colidx, w.features)
+    np.testing.assert_array_equal(got, ref)
+    rowptr = np.zeros(6, dtype=np.int64)
+    q = np.random.default_rng(0).standard_normal((5, 7)).astype(np.float32)
+    got, _ = run_gpu(oracle.SAGE_MAX, rowptr, np.zeros(0, dtype=np.int32), q)
+    np.testing.assert_array_equal(got, np.concatenate([q, np.zeros_like(q)], 1))
+
+
 def test_sage_mean_only_without_concat():
     rowptr, colidx = wl.random_small_graph(200, 900, seed=2)
     q = np.random.default_rng(2).standard_normal((200, 36)).astype(np.float32)

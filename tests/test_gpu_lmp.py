@@ -47,6 +47,17 @@ def test_last_iterate_runs_track_the_checker_round_by_round(idx, scale, R):
         # overshoot (the loss rises before it falls) and the trajectory amplifies rounding-level
         # differences, so a short run is compared at a tenth of it.
         w.lr *= 0.1
+    check_last_iterate_run(w, R)
+
+
+def test_max_pooling_rounds_track_the_checker():
+    """The K-round loop with the max-pooling aggregator of Section 2.2 in place of the mean."""
+    w = wl.make_config(2)
+    w.aggr = wl.SAGE_MAX
+    check_last_iterate_run(w, 25)
+
+
+def check_last_iterate_run(w, R):
     ref, got = run_both(w, R, eval_every=R)
     check_counts(ref, got)
     n_val, n_test = len(w.val_idx), len(w.test_idx)
