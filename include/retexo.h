@@ -270,6 +270,27 @@ int retexo_cross_partition_bytes_static(const retexo_csr* g, const int32_t* part
                                         uint64_t* bytes_per_round, uint64_t* bytes_total,
                                         uint64_t* send_per_part, uint64_t* recv_per_part, void* stream);
 
+/* ------------------------------------------- analytical data volume */
+typedef struct retexo_data_volume_result {
+    double lazy_lt;             /* DV^{lazy}_{lt}:     one exchange of H_0..H_{K-1} per boundary row, both ways */
+    double standard_lt;         /* DV^{standard}_{lt}: 2 R exchanges of H_1..H_{K-1} + the cached features */
+    double lazy_reduce;         /* DV^{lazy}_{reduce}: 2 n R (M + sum of the temporary classifiers C_m) */
+    double standard_reduce;     /* DV^{standard}_{reduce}: 2 n R M */
+    double gamma;               /* Eq. 2: (standard_lt + standard_reduce) / (lazy_lt + lazy_reduce) */
+    double model_size;          /* M = sum of L */
+} retexo_data_volume_result;
+
+/* The closed-form network data volumes of Section 3.3 / Appendix A.1, in
+ * elements, and their ratio gamma (Eq. 2).  Host arithmetic only: no device
+ * is touched.  H (host) holds the K + 1 representation widths H_0..H_K, L
+ * (host) the K layer sizes L_1..L_K; n_workers > 0, B >= 0 boundary nodes per
+ * worker, R > 0 training iterations.  C_m = H_m x H_K for m < K.  With
+ * n_workers * B set to the boundary_pairs counted by
+ * retexo_cross_partition_bytes, lazy_lt equals that call's 2 x bytes_total at
+ * elem_bytes = 1.  Errors: INVALID_ARG. */
+int retexo_data_volume(int32_t K, const int64_t* H, const int64_t* L, double n_workers, double B, double R,
+                       retexo_data_volume_result* out);
+
 /* -------------------------------------------------- the K-round LMP loop */
 typedef struct retexo_lmp_config {
     int32_t aggr;                   /* retexo_aggr */

@@ -57,6 +57,11 @@ class _LmpInputs(C.Structure):
                 ("theta0", C.POINTER(C.c_void_p)), ("gat_w", C.POINTER(C.c_void_p))]
 
 
+class _DataVolume(C.Structure):
+    _fields_ = [("lazy_lt", C.c_double), ("standard_lt", C.c_double), ("lazy_reduce", C.c_double),
+                ("standard_reduce", C.c_double), ("gamma", C.c_double), ("model_size", C.c_double)]
+
+
 class _LmpOutputs(C.Structure):
     _fields_ = [("loss_history", C.c_void_p), ("val_correct", C.c_void_p), ("best_val_correct", C.c_void_p),
                 ("best_iter", C.c_void_p), ("test_correct", C.c_void_p), ("test_correct_last", C.c_void_p),
@@ -69,7 +74,7 @@ EXPORTS = ["retexo_status_string", "retexo_version", "retexo_validate_csr", "ret
            "retexo_mlp_train_step", "retexo_embed_workspace_size", "retexo_embed",
            "retexo_cross_partition_workspace_size", "retexo_cross_partition_bytes",
            "retexo_cross_partition_static_scratch_bytes", "retexo_cross_partition_bytes_static",
-           "retexo_lmp_workspace_size",
+           "retexo_data_volume", "retexo_lmp_workspace_size",
            "retexo_lmp_train"]
 
 
@@ -439,3 +444,16 @@ def retexo_lmp_train(problem: LmpProblem) -> None:
     rc = lib().retexo_lmp_train(C.byref(problem.cfg), C.byref(problem.inputs), C.byref(problem.outputs),
                                 _ptr(problem.workspace), C.c_size_t(problem.workspace.numel()), _stream())
     _check(rc, "retexo_lmp_train")
+
+
+def retexo_data_volume(H, L, n_workers: float, B: float, R: float) -> dict:
+    """Closed-form data volumes and gamma (Eq. 2); H = [H_0..H_K], L = [L_1..L_K].  Host only."""
+    K = len(L)
+    if len(H) != K + 1:
+        raise RetexoError("H must hold K + 1 widths")
+    h = (C.c_int64 * (K + 1))(*[int(x) for x in H])
+    l = (C.c_int64 * K)(*[int(x) for x in L])
+    out = _DataVolume()
+    _check(lib().retexo_data_volume(C.c_int32(K), h, l, C.c_double(n_workers), C.c_double(B), C.c_double(R),
+                                    C.byref(out)), "retexo_data_volume")
+    return {k: getattr(out, k) for k, _ in _DataVolume._fields_}

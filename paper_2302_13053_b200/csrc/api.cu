@@ -16,3 +16,28 @@ extern "C" const char* retexo_status_string(int status) {
 }
 
 extern "C" int retexo_version(void) { return 100; }
+
+// Closed forms of Section 3.3 / Appendix A.1 (host arithmetic).
+extern "C" int retexo_data_volume(int32_t K, const int64_t* H, const int64_t* L, double n_workers, double B, double R,
+                                  retexo_data_volume_result* out) {
+    if (K < 1 || !H || !L || !out || !(n_workers > 0.0) || !(B >= 0.0) || !(R > 0.0)) return RETEXO_ERR_INVALID_ARG;
+    double hidden_sum = 0.0, model = 0.0, classifiers = 0.0;
+    for (int32_t m = 0; m <= K; ++m) if (H[m] < 0) return RETEXO_ERR_INVALID_ARG;
+    for (int32_t m = 1; m < K; ++m) {
+        hidden_sum += (double)H[m];
+        classifiers += (double)H[m] * (double)H[K];
+    }
+    for (int32_t m = 0; m < K; ++m) {
+        if (L[m] < 0) return RETEXO_ERR_INVALID_ARG;
+        model += (double)L[m];
+    }
+    const double pairs = 2.0 * n_workers * B;                  // boundary rows sent plus received
+    out->lazy_lt = pairs * (hidden_sum + (double)H[0]);
+    out->standard_lt = pairs * (2.0 * R * hidden_sum + (double)H[0]);
+    out->standard_reduce = 2.0 * n_workers * R * model;
+    out->lazy_reduce = 2.0 * n_workers * R * (model + classifiers);
+    out->model_size = model;
+    const double den = out->lazy_lt + out->lazy_reduce;
+    out->gamma = den > 0.0 ? (out->standard_lt + out->standard_reduce) / den : 0.0;
+    return RETEXO_OK;
+}

@@ -70,3 +70,23 @@ def test_lazy_local_volume_matches_the_counted_boundary_rows():
     c = oracle.cross_partition(rowptr, colidx, part, 5, dims, elem_bytes=1)
     d = oracle.data_volume(dims + [4], [1, 1, 1], 5, c["boundary_pairs"] / 5.0, 10)
     assert d["lazy_lt"] == pytest.approx(c["dv_lazy_lt"], rel=1e-12)
+
+
+@pytest.mark.parametrize("H,L,n,B,R", CASES)
+def test_library_closed_forms_agree_with_the_written_out_sums(H, L, n, B, R):
+    """The C-ABI's host-side calculator (closed forms) against the checker's message-by-message sums."""
+    from paper_2302_13053_b200 import binding
+    got = binding.retexo_data_volume(H, L, n, B, R)
+    ref = oracle.data_volume(H, L, n, B, R)
+    for k in ref:
+        assert got[k] == pytest.approx(ref[k], rel=1e-12), k
+
+
+def test_library_rejects_bad_arguments():
+    from paper_2302_13053_b200 import binding
+    with pytest.raises(binding.RetexoError):
+        binding.retexo_data_volume([4, 4], [16], 0, 1.0, 10)
+    with pytest.raises(binding.RetexoError):
+        binding.retexo_data_volume([4, 4], [16], 2, 1.0, 0)
+    with pytest.raises(binding.RetexoError):
+        binding.retexo_data_volume([4, 4, 4], [16], 2, 1.0, 10)
