@@ -11,6 +11,7 @@
 
 #include "common.cuh"
 #include "gemm_tc.h"
+#include <string.h>
 
 namespace retexo {
 
@@ -52,6 +53,20 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+
+// Bulk tensor store of a [32 x 32] bf16 box from shared memory (64-byte swizzle) to global memory;
+// the part of the box outside the tensor is not written.  One bulk group per store.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int32_t x, int32_t y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(smem_src)) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Waits until all but the newest bulk group of this thread have finished reading shared memory.
+__device__ __forceinline__ void bulk_wait_read_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+// Waits until every bulk group of this thread is complete (the data is in global memory).
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Orders this thread's shared-memory writes before later asynchronous-proxy reads of them.
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128
 // bytes, 8-row groups 1024 bytes apart.
@@ -120,14 +135,31 @@ struct TcKernelArgs {
     int32_t* pred; unsigned long long* correct;
     int64_t n_train; const int32_t* y_eval;       // SOFTMAX_CE: rows >= n_train are evaluated, not trained on
     int32_t* status;
+    int tma_rows, tma_t;          // out_bf16 / out_bf16_t leave through bulk tensor stores (map_rows / map_t)
 };
 
 // Per-warp staging of one 32 x 32 bf16 block: 32 lines of 64 bytes.  A line is one output row
 // (row-major store) or one output column (transposed store).  The four 16-byte pieces of a line
 // are XOR-swizzled with the line index so that both the fill (one thread per row) and the drain
 // (eight lines of 64 contiguous bytes per instruction) are free of bank conflicts.
-constexpr int kStageBytesPerWarp = 32 * 64;
+// This is also the 64-byte swizzle of a tensor map (address bits 4-5 XOR bits 7-8), so a block staged in a
+// 1024-byte aligned buffer can leave as one bulk tensor store.  Every warp owns two such buffers and
+// alternates between them, so that a store may still be reading one while the next block is staged.
+constexpr int kStageBlockBytes = 32 * 64;
+constexpr int kStageBytesPerWarp = 2 * kStageBlockBytes;
 __device__ __forceinline__ int stage_piece(int line, int piece) { return piece ^ ((line >> 1) & 3); }
+
+struct WarpStage {
+    uint8_t* base;      // two blocks of kStageBlockBytes
+    int cur;
+};
+// The block staged two stores ago: its bulk store (if there was one) has finished reading it.
+__device__ __forceinline__ uint8_t* stage_acquire(WarpStage& ws, int lane) {
+    if (lane == 0) bulk_wait_read_but_one();
+    __syncwarp();
+    ws.cur ^= 1;
+    return ws.base + ws.cur * kStageBlockBytes;
+}
 
 // Drains the staged block: line L goes to dst + L * stride (elements), 64 contiguous bytes each.
 __device__ __forceinline__ void drain_stage(const uint8_t* stage, __nv_bfloat16* dst, int64_t stride, int64_t n_lines,
@@ -142,21 +174,29 @@ __device__ __forceinline__ void drain_stage(const uint8_t* stage, __nv_bfloat16*
 }
 
 // Writes a warp's 32 x 32 block (lane = row, v[j] = column col0 + j) into the transposed output
-// out_t[col][row].  Full, aligned blocks go through shared memory so that every column leaves
-// as one 64-byte run; ragged ones fall back to guarded element stores.
+// out_t[col][row].  With a tensor map the staged block leaves as one bulk store (clipped to rows
+// < M and columns < n_cols by the map's extents; the caller guarantees row0 < M, col0 < n_cols).
+// Otherwise full, aligned blocks are drained with 64-byte runs and ragged ones fall back to
+// guarded element stores.
 __device__ __forceinline__ void store_block_transposed(__nv_bfloat16* out_t, int64_t ld_t, int64_t col0, int64_t n_cols,
                                                        int64_t row0, int64_t M, const float (&v)[32], uint8_t* stage,
-                                                       int lane) {
-    const bool fast = row0 + 32 <= M && (ld_t & 7) == 0 && aligned16(out_t);
+                                                       int lane, const CUtensorMap* map) {
+    const bool fast = map || (row0 + 32 <= M && (ld_t & 7) == 0 && aligned16(out_t));
     if (fast) {
 #pragma unroll
         for (int j = 0; j < 32; ++j)      // line j = column col0 + j; this lane's row is element `lane` of the line
             *reinterpret_cast<__nv_bfloat16*>(stage + j * 64 + stage_piece(j, lane >> 3) * 16 + (lane & 7) * 2) =
                 __float2bfloat16_rn(v[j]);
-        __syncwarp();
-        const int64_t n_lines = n_cols - col0 < 32 ? n_cols - col0 : 32;
-        drain_stage(stage, out_t + col0 * ld_t + row0, ld_t, n_lines, lane);
-        __syncwarp();
+        if (map) {
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) tma_store_2d(map, stage, (int32_t)row0, (int32_t)col0);
+        } else {
+            __syncwarp();
+            const int64_t n_lines = n_cols - col0 < 32 ? n_cols - col0 : 32;
+            drain_stage(stage, out_t + col0 * ld_t + row0, ld_t, n_lines, lane);
+            __syncwarp();
+        }
     } else {
         const int64_t row = row0 + lane;
         if (row < M) {
@@ -167,10 +207,11 @@ __device__ __forceinline__ void store_block_transposed(__nv_bfloat16* out_t, int
     }
 }
 
-// Row-major counterpart: out[row][col0 .. col0+32).  The caller guarantees a full, aligned
-// block of columns; rows beyond M are dropped.
+// Row-major counterpart: out[row][col0 .. col0+32).  With a tensor map: one bulk store, clipped
+// to the map's extents (row0 < M, col0 < its columns guaranteed by the caller).  Without: the
+// caller guarantees a full, aligned block of columns; rows beyond M are dropped.
 __device__ __forceinline__ void store_block_rows(__nv_bfloat16* out, int64_t ld, int64_t col0, int64_t row0, int64_t M,
-                                                 const float (&v)[32], uint8_t* stage, int lane) {
+                                                 const float (&v)[32], uint8_t* stage, int lane, const CUtensorMap* map) {
 #pragma unroll
     for (int p = 0; p < 4; ++p) {         // line = this lane's row; four 16-byte pieces of 8 columns
         __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * p], v[8 * p + 1]), b = __floats2bfloat162_rn(v[8 * p + 2], v[8 * p + 3]);
@@ -180,15 +221,40 @@ __device__ __forceinline__ void store_block_rows(__nv_bfloat16* out, int64_t ld,
         pk.z = *reinterpret_cast<uint32_t*>(&c); pk.w = *reinterpret_cast<uint32_t*>(&d);
         *reinterpret_cast<uint4*>(stage + lane * 64 + stage_piece(lane, p) * 16) = pk;
     }
+    if (map) {
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) tma_store_2d(map, stage, (int32_t)col0, (int32_t)row0);
+    } else {
+        __syncwarp();
+        const int64_t n_lines = M - row0 < 32 ? M - row0 : 32;
+        drain_stage(stage, out + row0 * ld + col0, ld, n_lines, lane);
+        __syncwarp();
+    }
+}
+
+// Reads this lane's row of a [32 x 32] bf16 block (rows row0.., columns col0..; full and aligned,
+// guaranteed by the caller) through the staging block, so that global memory is read in 64-byte
+// runs: m[j] = block[lane][j].  Rows beyond M read as zero.
+__device__ __forceinline__ void load_block_rows(const __nv_bfloat16* src, int64_t ld, int64_t col0, int64_t row0, int64_t M,
+                                                uint4 (&m)[4], uint8_t* stage, int lane) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int line = (lane >> 2) + 8 * i, piece = lane & 3;
+        uint4 pk = make_uint4(0u, 0u, 0u, 0u);
+        if (row0 + line < M) pk = __ldg(reinterpret_cast<const uint4*>(src + (row0 + line) * ld + col0 + piece * 8));
+        *reinterpret_cast<uint4*>(stage + line * 64 + stage_piece(line, piece) * 16) = pk;
+    }
     __syncwarp();
-    const int64_t n_lines = M - row0 < 32 ? M - row0 : 32;
-    drain_stage(stage, out + row0 * ld + col0, ld, n_lines, lane);
+#pragma unroll
+    for (int p = 0; p < 4; ++p) m[p] = *reinterpret_cast<const uint4*>(stage + lane * 64 + stage_piece(lane, p) * 16);
     __syncwarp();
 }
 
 template <int BN, int STAGES>
 __global__ void __launch_bounds__(kTcThreads, 1)
-tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, TcKernelArgs g) {
+tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_rows, const __grid_constant__ CUtensorMap map_t, TcKernelArgs g) {
     // Persistent: the block walks over output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...  The
     // stage ring runs on across tiles and the accumulator is double-buffered in tensor memory, so
     // the loads and MMAs of the next tile overlap the epilogue of the current one.
@@ -202,9 +268,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     float* warp_loss = reinterpret_cast<float*>(tmem_slot + 2);                  // [4]
-    uint8_t* stage_base = reinterpret_cast<uint8_t*>(                           // kEpiWarps x kStageBytesPerWarp, 16-byte aligned
-        (reinterpret_cast<uintptr_t>(tmem_slot) + 64 + 15) & ~uintptr_t(15));
-
+    // staging blocks: kEpiWarps x kStageBytesPerWarp, 1024 bytes behind the barrier area (so 1024-byte aligned)
+    uint8_t* stage_base = tiles + STAGES * kStageBytes + 1024;
     float (*xch)[2][128] = reinterpret_cast<float (*)[2][128]>(stage_base + kEpiWarps * kStageBytesPerWarp);   // [4][2][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -290,7 +355,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         const int q = warp & 3;                           // tensor-memory lane quarter this warp may read
         const int half = (warp - 2) >> 2;                 // which half of the tile's columns this warp drains
-        uint8_t* stage = stage_base + (warp - 2) * kStageBytesPerWarp;
+        WarpStage ws{stage_base + (warp - 2) * kStageBytesPerWarp, 0};
+        const CUtensorMap* rows_map = g.tma_rows ? &map_rows : nullptr;
+        const CUtensorMap* t_map = g.tma_t ? &map_t : nullptr;
         const bool row_owner = BN == 64 && g.mode == TC_EPI_ARGMAX;
         int64_t lt = 0;
         for (int64_t t = blockIdx.x; t < n_tiles && !(row_owner && half == 1); t += gridDim.x, ++lt) {
@@ -359,7 +426,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const float scale = g.inv_rows / den;
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = cb + j < g.N ? (v[j] * scale - (cb + j == yi ? g.inv_rows : 0.f)) : 0.f;
-                if (live && g.out_bf16) {       // dL row-major: this thread's columns, 16 bytes at a time
+                if (rows_map) {                 // dL row-major: one bulk store per warp, clipped to the trained rows
+                    if (g.out_bf16 && row0 < g.n_train && cb < g.ld_bf16)
+                        store_block_rows(g.out_bf16, g.ld_bf16, cb, row0, g.n_train, v, stage_acquire(ws, lane), lane, rows_map);
+                } else if (live && g.out_bf16) {       // this thread's columns, 16 bytes at a time
                     __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16 + cb;
 #pragma unroll
                     for (int c = 0; c < 32; c += 8) {
@@ -372,8 +442,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         *reinterpret_cast<uint4*>(dst + c) = pk;
                     }
                 }
-                if (g.out_bf16_t && cb < g.N)
-                    store_block_transposed(g.out_bf16_t, g.ld_t, cb, g.N, row0, g.n_train, v, stage, lane);
+                if (g.out_bf16_t && cb < g.N && (!t_map || row0 < g.n_train))
+                    store_block_transposed(g.out_bf16_t, g.ld_t, cb, g.N, row0, g.n_train, v, stage_acquire(ws, lane), lane, t_map);
                 if (half == 0) {
                     float loss = live ? (mx + __logf(den)) - ly : 0.f;
                     loss = warp_sum(loss);
@@ -459,30 +529,33 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
                     } else if (g.mode == TC_EPI_MASK_T || g.mode == TC_EPI_MASK) {
                         float v[32];
-                        if (row < g.M) {
-                            const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
-                            if (col0 + 32 <= g.N && (g.ld_mask & 7) == 0 && aligned16(g.mask)) {
+                        uint8_t* stage = stage_acquire(ws, lane);
+                        if (col0 + 32 <= g.N && (g.ld_mask & 7) == 0 && aligned16(g.mask)) {
+                            uint4 mk[4];      // the gate block, read in 64-byte runs through the staging block
+                            load_block_rows(g.mask, g.ld_mask, col0, row0, g.M, mk, stage, lane);
 #pragma unroll
-                                for (int j = 0; j < 32; j += 8) {
-                                    const uint4 pk = *reinterpret_cast<const uint4*>(mrow + j);
-                                    const __nv_bfloat16* mv = reinterpret_cast<const __nv_bfloat16*>(&pk);
+                            for (int p = 0; p < 4; ++p) {
+                                const __nv_bfloat16* mv = reinterpret_cast<const __nv_bfloat16*>(&mk[p]);
 #pragma unroll
-                                    for (int k = 0; k < 8; ++k)
-                                        v[j + k] = __bfloat162float(mv[k]) > 0.f ? __uint_as_float(r[j + k]) : 0.f;
-                                }
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j)
-                                    v[j] = (col0 + j < g.N && __bfloat162float(mrow[j]) > 0.f) ? __uint_as_float(r[j]) : 0.f;
+                                for (int k = 0; k < 8; ++k)
+                                    v[8 * p + k] = __bfloat162float(mv[k]) > 0.f ? __uint_as_float(r[8 * p + k]) : 0.f;
                             }
+                        } else if (row < g.M) {
+                            const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                v[j] = (col0 + j < g.N && __bfloat162float(mrow[j]) > 0.f) ? __uint_as_float(r[j]) : 0.f;
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j) v[j] = 0.f;
                         }
                         if (g.mode == TC_EPI_MASK_T) {
-                            store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane);
+                            if (!t_map || row0 < g.M)
+                                store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane, t_map);
+                        } else if (rows_map) {
+                            if (row0 < g.M) store_block_rows(g.out_bf16, g.ld_bf16, col0, row0, g.M, v, stage, lane, rows_map);
                         } else if (col0 + 32 <= g.N && (g.ld_bf16 & 7) == 0 && aligned16(g.out_bf16)) {
-                            store_block_rows(g.out_bf16, g.ld_bf16, col0, row0, g.M, v, stage, lane);
+                            store_block_rows(g.out_bf16, g.ld_bf16, col0, row0, g.M, v, stage, lane, nullptr);
                         } else if (row < g.M) {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
@@ -500,11 +573,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             v[j] = x;
                         }
                         if (g.out_bf16_t) {
-                            store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane);
+                            if (!t_map || row0 < g.M)
+                                store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage_acquire(ws, lane), lane, t_map);
                             if (g.ones_row_t && col0 == 0 && row < g.M) g.out_bf16_t[g.N * g.ld_t + row] = __float2bfloat16_rn(1.0f);
                         }
-                        const bool rows_fast = g.out_bf16 && col0 + 32 <= g.N && (g.ld_bf16 & 7) == 0 && aligned16(g.out_bf16);
-                        if (rows_fast) store_block_rows(g.out_bf16, g.ld_bf16, col0, row0, g.M, v, stage, lane);
+                        const bool rows_fast = g.out_bf16 && (rows_map || (col0 + 32 <= g.N && (g.ld_bf16 & 7) == 0 && aligned16(g.out_bf16)));
+                        if (rows_fast && (!rows_map || row0 < g.M))
+                            store_block_rows(g.out_bf16, g.ld_bf16, col0, row0, g.M, v, stage_acquire(ws, lane), lane, rows_map);
                         if (row >= g.M) continue;
                         if (g.out_f32) {
                             float* dst = g.out_f32 + row * g.ld_f32 + col0;
@@ -530,6 +605,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(acc_empty + b)) : "memory");
         }
+        if (lane == 0) bulk_wait_all();       // this thread's bulk stores have reached global memory
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -569,9 +645,27 @@ static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t c
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of a bf16 output matrix [rows x cols] (row stride ld elements) for [32 x 32] stores with the
+// 64-byte swizzle of the staging blocks.  Returns false where the layout does not allow one.
+static bool make_store_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || !base || rows <= 0 || cols <= 0 || !aligned_to(base, 16) || ld % 8 != 0 || ld < cols) return false;
+    if (rows > INT32_MAX || cols > INT32_MAX) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int BN, int STAGES>
 static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
-    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 512 + kEpiWarps * kStageBytesPerWarp + 4 * 2 * 128 * 4;
+    // stage ring + alignment slack + barrier area + staging blocks (+ the soft-max exchange arrays)
+    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 1024 + kEpiWarps * kStageBytesPerWarp +
+                            (BN == 64 ? 4 * 2 * 128 * 4 : 0);
+    static_assert(smem <= 227 * 1024, "shared memory budget");
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
@@ -595,11 +689,20 @@ static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& 
     g.y = t.y; g.inv_rows = t.inv_rows; g.loss_partial = t.loss_partial; g.pred = t.pred; g.correct = t.correct;
     g.n_train = (t.mode == TC_EPI_SOFTMAX_CE && t.eval_from > 0 && t.eval_from < t.M) ? t.eval_from : t.M;
     g.y_eval = t.y_eval;
+    // bf16 outputs leave through bulk tensor stores where their layout allows it
+    CUtensorMap m_rows, m_t;
+    memset(&m_rows, 0, sizeof(m_rows));
+    memset(&m_t, 0, sizeof(m_t));
+    const bool ce = t.mode == TC_EPI_SOFTMAX_CE;
+    if (t.out_bf16 && (t.mode == TC_EPI_BIAS || t.mode == TC_EPI_MASK || ce))
+        g.tma_rows = make_store_map(&m_rows, t.out_bf16, ce ? g.n_train : t.M, ce ? t.ld_bf16 : t.N, t.ld_bf16) ? 1 : 0;
+    if (t.out_bf16_t && (t.mode == TC_EPI_BIAS || t.mode == TC_EPI_MASK_T || ce))
+        g.tma_t = make_store_map(&m_t, t.out_bf16_t, t.N, ce ? g.n_train : t.M, t.ld_t) ? 1 : 0;
     const int64_t n_tiles = ((t.M + kTcBM - 1) / kTcBM) * ((t.N + BN - 1) / BN) * splits;
     const int n_sm = sm_count();
     if (n_sm <= 0) return RETEXO_ERR_CUDA;
     const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);      // one persistent block per SM
-    tc_gemm_kernel<BN, STAGES><<<grid, kTcThreads, smem, st>>>(ma, mb, g);
+    tc_gemm_kernel<BN, STAGES><<<grid, kTcThreads, smem, st>>>(ma, mb, m_rows, m_t, g);
     return launch_status();
 }
 
@@ -624,7 +727,7 @@ int tc_gemm_launch(const TcGemm& t, cudaStream_t st) {
     if (!make_map(&mb, t.B, t.N, t.K, t.ldb, bn)) return RETEXO_ERR_CUDA;
     if (bn == 256) return launch_tc<256, 4>(t, ma, mb, st);
     if (bn == 128) return launch_tc<128, 6>(t, ma, mb, st);
-    return launch_tc<64, 8>(t, ma, mb, st);
+    return launch_tc<64, 7>(t, ma, mb, st);
 }
 
 }  // namespace retexo
