@@ -55,14 +55,15 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
 }
 
 // Bulk tensor store of a [32 x 32] bf16 box from shared memory (64-byte swizzle) to global memory;
-// the part of the box outside the tensor is not written.  One bulk group per store.
+// the part of the box outside the tensor is not written.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int32_t x, int32_t y) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
                  ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(smem_src)) : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
 }
-// Waits until all but the newest bulk group of this thread have finished reading shared memory.
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Wait until all (all but the newest) bulk groups of this thread have finished reading shared memory.
 __device__ __forceinline__ void bulk_wait_read_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 // Waits until every bulk group of this thread is complete (the data is in global memory).
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // Orders this thread's shared-memory writes before later asynchronous-proxy reads of them.
@@ -143,23 +144,11 @@ struct TcKernelArgs {
 // are XOR-swizzled with the line index so that both the fill (one thread per row) and the drain
 // (eight lines of 64 contiguous bytes per instruction) are free of bank conflicts.
 // This is also the 64-byte swizzle of a tensor map (address bits 4-5 XOR bits 7-8), so a block staged in a
-// 1024-byte aligned buffer can leave as one bulk tensor store.  Every warp owns two such buffers and
-// alternates between them, so that a store may still be reading one while the next block is staged.
+// 1024-byte aligned buffer can leave as one bulk tensor store.  Every warp owns two such blocks: the
+// first stages transposed output, the second row-major output.
 constexpr int kStageBlockBytes = 32 * 64;
 constexpr int kStageBytesPerWarp = 2 * kStageBlockBytes;
 __device__ __forceinline__ int stage_piece(int line, int piece) { return piece ^ ((line >> 1) & 3); }
-
-struct WarpStage {
-    uint8_t* base;      // two blocks of kStageBlockBytes
-    int cur;
-};
-// The block staged two stores ago: its bulk store (if there was one) has finished reading it.
-__device__ __forceinline__ uint8_t* stage_acquire(WarpStage& ws, int lane) {
-    if (lane == 0) bulk_wait_read_but_one();
-    __syncwarp();
-    ws.cur ^= 1;
-    return ws.base + ws.cur * kStageBlockBytes;
-}
 
 // Drains the staged block: line L goes to dst + L * stride (elements), 64 contiguous bytes each.
 __device__ __forceinline__ void drain_stage(const uint8_t* stage, __nv_bfloat16* dst, int64_t stride, int64_t n_lines,
@@ -173,30 +162,21 @@ __device__ __forceinline__ void drain_stage(const uint8_t* stage, __nv_bfloat16*
     }
 }
 
-// Writes a warp's 32 x 32 block (lane = row, v[j] = column col0 + j) into the transposed output
-// out_t[col][row].  With a tensor map the staged block leaves as one bulk store (clipped to rows
-// < M and columns < n_cols by the map's extents; the caller guarantees row0 < M, col0 < n_cols).
-// Otherwise full, aligned blocks are drained with 64-byte runs and ragged ones fall back to
-// guarded element stores.
+// Fallback stores (no tensor map).  Transposed: out_t[col][row]; full, aligned blocks are staged and drained
+// in 64-byte runs, ragged ones use guarded element stores.
 __device__ __forceinline__ void store_block_transposed(__nv_bfloat16* out_t, int64_t ld_t, int64_t col0, int64_t n_cols,
                                                        int64_t row0, int64_t M, const float (&v)[32], uint8_t* stage,
-                                                       int lane, const CUtensorMap* map) {
-    const bool fast = map || (row0 + 32 <= M && (ld_t & 7) == 0 && aligned16(out_t));
+                                                       int lane) {
+    const bool fast = row0 + 32 <= M && (ld_t & 7) == 0 && aligned16(out_t);
     if (fast) {
 #pragma unroll
         for (int j = 0; j < 32; ++j)      // line j = column col0 + j; this lane's row is element `lane` of the line
             *reinterpret_cast<__nv_bfloat16*>(stage + j * 64 + stage_piece(j, lane >> 3) * 16 + (lane & 7) * 2) =
                 __float2bfloat16_rn(v[j]);
-        if (map) {
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) tma_store_2d(map, stage, (int32_t)row0, (int32_t)col0);
-        } else {
-            __syncwarp();
-            const int64_t n_lines = n_cols - col0 < 32 ? n_cols - col0 : 32;
-            drain_stage(stage, out_t + col0 * ld_t + row0, ld_t, n_lines, lane);
-            __syncwarp();
-        }
+        __syncwarp();
+        const int64_t n_lines = n_cols - col0 < 32 ? n_cols - col0 : 32;
+        drain_stage(stage, out_t + col0 * ld_t + row0, ld_t, n_lines, lane);
+        __syncwarp();
     } else {
         const int64_t row = row0 + lane;
         if (row < M) {
@@ -207,51 +187,114 @@ __device__ __forceinline__ void store_block_transposed(__nv_bfloat16* out_t, int
     }
 }
 
-// Row-major counterpart: out[row][col0 .. col0+32).  With a tensor map: one bulk store, clipped
-// to the map's extents (row0 < M, col0 < its columns guaranteed by the caller).  Without: the
-// caller guarantees a full, aligned block of columns; rows beyond M are dropped.
-__device__ __forceinline__ void store_block_rows(__nv_bfloat16* out, int64_t ld, int64_t col0, int64_t row0, int64_t M,
-                                                 const float (&v)[32], uint8_t* stage, int lane, const CUtensorMap* map) {
+// Row-major fallback: out[row][col0 .. col0+32); a full, aligned block of columns goes through the staging
+// block, anything else through guarded element stores.  Rows beyond M are dropped.
+__device__ __forceinline__ void store_block_rows(__nv_bfloat16* out, int64_t ld, int64_t col0, int64_t n_cols, int64_t row0,
+                                                 int64_t M, const float (&v)[32], uint8_t* stage, int lane) {
+    if (col0 + 32 <= n_cols && (ld & 7) == 0 && aligned16(out)) {
 #pragma unroll
-    for (int p = 0; p < 4; ++p) {         // line = this lane's row; four 16-byte pieces of 8 columns
-        __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * p], v[8 * p + 1]), b = __floats2bfloat162_rn(v[8 * p + 2], v[8 * p + 3]);
-        __nv_bfloat162 c = __floats2bfloat162_rn(v[8 * p + 4], v[8 * p + 5]), d = __floats2bfloat162_rn(v[8 * p + 6], v[8 * p + 7]);
-        uint4 pk;
-        pk.x = *reinterpret_cast<uint32_t*>(&a); pk.y = *reinterpret_cast<uint32_t*>(&b);
-        pk.z = *reinterpret_cast<uint32_t*>(&c); pk.w = *reinterpret_cast<uint32_t*>(&d);
-        *reinterpret_cast<uint4*>(stage + lane * 64 + stage_piece(lane, p) * 16) = pk;
-    }
-    if (map) {
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) tma_store_2d(map, stage, (int32_t)col0, (int32_t)row0);
-    } else {
+        for (int p = 0; p < 4; ++p) {         // line = this lane's row; four 16-byte pieces of 8 columns
+            __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * p], v[8 * p + 1]), b = __floats2bfloat162_rn(v[8 * p + 2], v[8 * p + 3]);
+            __nv_bfloat162 c = __floats2bfloat162_rn(v[8 * p + 4], v[8 * p + 5]), d = __floats2bfloat162_rn(v[8 * p + 6], v[8 * p + 7]);
+            uint4 pk;
+            pk.x = *reinterpret_cast<uint32_t*>(&a); pk.y = *reinterpret_cast<uint32_t*>(&b);
+            pk.z = *reinterpret_cast<uint32_t*>(&c); pk.w = *reinterpret_cast<uint32_t*>(&d);
+            *reinterpret_cast<uint4*>(stage + lane * 64 + stage_piece(lane, p) * 16) = pk;
+        }
         __syncwarp();
         const int64_t n_lines = M - row0 < 32 ? M - row0 : 32;
         drain_stage(stage, out + row0 * ld + col0, ld, n_lines, lane);
         __syncwarp();
+    } else if (row0 + lane < M) {
+        __nv_bfloat16* dst = out + (row0 + lane) * ld + col0;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) if (col0 + j < n_cols) dst[j] = __float2bfloat16_rn(v[j]);
     }
 }
 
-// Reads this lane's row of a [32 x 32] bf16 block (rows row0.., columns col0..; full and aligned,
-// guaranteed by the caller) through the staging block, so that global memory is read in 64-byte
-// runs: m[j] = block[lane][j].  Rows beyond M read as zero.
-__device__ __forceinline__ void load_block_rows(const __nv_bfloat16* src, int64_t ld, int64_t col0, int64_t row0, int64_t M,
-                                                uint4 (&m)[4], uint8_t* stage, int lane) {
+// Bulk-store core: p[k] holds columns col0 + 2k (low half) and col0 + 2k + 1 (high half) of this lane's row as bf16.
+// The block is staged row-major (if rows_map) and / or transposed (if t_map) and leaves as bulk tensor
+// stores, clipped to the maps' extents (the caller guarantees row0 and col0 inside them); both stores
+// are issued behind one proxy fence.  ready_block (optional, for a single output): a staging block the
+// caller has already made sure no bulk store is reading; it is used instead of the output's own block
+// and nothing is waited for.  Warp-uniform arguments except p.
+__device__ __forceinline__ void store_block_packed(const uint32_t (&p)[16], uint8_t* stage, int lane, int64_t col0, int64_t row0,
+                                                   const CUtensorMap* rows_map, const CUtensorMap* t_map,
+                                                   uint8_t* ready_block = nullptr) {
+    uint8_t* t_block = stage;
+    uint8_t* rows_block = stage + kStageBlockBytes;
+    if (ready_block && (rows_map == nullptr) != (t_map == nullptr)) {
+        t_block = rows_block = ready_block;
+    } else {
+        if (lane == 0) bulk_wait_read_all();      // the previous block's stores have read the staging blocks
+        __syncwarp();
+    }
+    if (t_map) {
+        // 2 x 2 exchange with the neighbouring lane: even lanes end up with rows (lane, lane + 1) of column 2k,
+        // odd lanes with rows (lane - 1, lane) of column 2k + 1, one 32-bit word each; line = column
+        uint8_t* base = t_block + (lane & 1) * 64 + (lane >> 1 & 3) * 4;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            const uint32_t x = __shfl_xor_sync(0xffffffffu, p[k], 1);
+            const uint32_t w = (lane & 1) ? __byte_perm(x, p[k], 0x7632) : __byte_perm(p[k], x, 0x5410);
+            *reinterpret_cast<uint32_t*>(base + k * 128 + ((lane >> 3) ^ (k & 3)) * 16) = w;
+        }
+    }
+    if (rows_map) {
+        uint8_t* line = rows_block + lane * 64;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            *reinterpret_cast<uint4*>(line + stage_piece(lane, q) * 16) = make_uint4(p[4 * q], p[4 * q + 1], p[4 * q + 2], p[4 * q + 3]);
+    }
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        if (t_map) tma_store_2d(t_map, t_block, (int32_t)row0, (int32_t)col0);
+        if (rows_map) tma_store_2d(rows_map, rows_block, (int32_t)col0, (int32_t)row0);
+        bulk_commit();
+    }
+}
+
+// Stores a warp's 32 x 32 block (lane = row, v[j] = column col0 + j) as bf16: row-major into out
+// (if do_rows) and / or transposed into out_t (if do_t).  An output with a tensor map leaves through
+// store_block_packed, one without through the fallbacks above.  Warp-uniform arguments except v.
+__device__ __forceinline__ void store_block(const float (&v)[32], uint8_t* stage, int lane, int64_t col0, int64_t n_cols,
+                                            int64_t row0, int64_t M, bool do_rows, __nv_bfloat16* out, int64_t ld,
+                                            const CUtensorMap* rows_map, bool do_t, __nv_bfloat16* out_t, int64_t ld_t,
+                                            const CUtensorMap* t_map) {
+    const bool rows_tma = do_rows && rows_map, t_tma = do_t && t_map;
+    // (an output without a map never shares its staging block with a bulk store in flight)
+    if (do_t && !t_map) store_block_transposed(out_t, ld_t, col0, n_cols, row0, M, v, stage, lane);
+    if (do_rows && !rows_map) store_block_rows(out, ld, col0, n_cols, row0, M, v, stage + kStageBlockBytes, lane);
+    if (rows_tma || t_tma) {
+        uint32_t p[16];
+#pragma unroll
+        for (int k = 0; k < 16; ++k) {
+            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+            p[k] = *reinterpret_cast<uint32_t*>(&b2);
+        }
+        store_block_packed(p, stage, lane, col0, row0, rows_tma ? rows_map : nullptr, t_tma ? t_map : nullptr);
+    }
+}
+
+// Copies a [32 x 32] bf16 block (rows row0.., columns col0..; full and aligned columns, guaranteed by the
+// caller) into a staging block in 64-byte runs; rows beyond M are filled with zeros.  Afterwards lane L
+// finds piece q (columns 8q .. 8q+7) of row L at block + L * 64 + stage_piece(L, q) * 16.
+__device__ __forceinline__ void stage_block_from_global(const __nv_bfloat16* src, int64_t ld, int64_t col0, int64_t row0,
+                                                        int64_t M, uint8_t* block, int lane) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int line = (lane >> 2) + 8 * i, piece = lane & 3;
         uint4 pk = make_uint4(0u, 0u, 0u, 0u);
         if (row0 + line < M) pk = __ldg(reinterpret_cast<const uint4*>(src + (row0 + line) * ld + col0 + piece * 8));
-        *reinterpret_cast<uint4*>(stage + line * 64 + stage_piece(line, piece) * 16) = pk;
+        *reinterpret_cast<uint4*>(block + line * 64 + stage_piece(line, piece) * 16) = pk;
     }
-    __syncwarp();
-#pragma unroll
-    for (int p = 0; p < 4; ++p) m[p] = *reinterpret_cast<const uint4*>(stage + lane * 64 + stage_piece(lane, p) * 16);
     __syncwarp();
 }
 
-template <int BN, int STAGES>
+// MODE (a TcEpilogue value) is a template parameter so that every instantiation carries the registers of
+// its own epilogue only.
+template <int BN, int STAGES, int MODE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_rows, const __grid_constant__ CUtensorMap map_t, TcKernelArgs g) {
@@ -280,7 +323,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
         // the arg-max epilogue lets one thread own a whole row of logits: it uses four of the eight warps
-        const bool row_owner = BN == 64 && g.mode == TC_EPI_ARGMAX;
+        const bool row_owner = BN == 64 && MODE == TC_EPI_ARGMAX;
         for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, row_owner ? 4 : kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -355,10 +398,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         const int q = warp & 3;                           // tensor-memory lane quarter this warp may read
         const int half = (warp - 2) >> 2;                 // which half of the tile's columns this warp drains
-        WarpStage ws{stage_base + (warp - 2) * kStageBytesPerWarp, 0};
+        uint8_t* stage = stage_base + (warp - 2) * kStageBytesPerWarp;      // this warp's two staging blocks
+        int flip = 0;
         const CUtensorMap* rows_map = g.tma_rows ? &map_rows : nullptr;
         const CUtensorMap* t_map = g.tma_t ? &map_t : nullptr;
-        const bool row_owner = BN == 64 && g.mode == TC_EPI_ARGMAX;
+        const bool row_owner = BN == 64 && MODE == TC_EPI_ARGMAX;
         int64_t lt = 0;
         for (int64_t t = blockIdx.x; t < n_tiles && !(row_owner && half == 1); t += gridDim.x, ++lt) {
             const int64_t z = t / per_split, rem = t % per_split;
@@ -374,7 +418,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const bool ok = mbar_wait(acc_full + b, pb, g.status, abort_flag);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (!ok) break;
-            if (BN == 64 && g.mode == TC_EPI_SOFTMAX_CE) {
+            if constexpr (BN == 64 && MODE == TC_EPI_SOFTMAX_CE) {
                 // Two threads share a row of logits: warp q takes columns [0, 32), warp q + 4 columns
                 // [32, 64); row maximum, sum and the label's logit are exchanged through shared memory.
                 const int cb = half * 32;
@@ -426,10 +470,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const float scale = g.inv_rows / den;
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = cb + j < g.N ? (v[j] * scale - (cb + j == yi ? g.inv_rows : 0.f)) : 0.f;
-                if (rows_map) {                 // dL row-major: one bulk store per warp, clipped to the trained rows
-                    if (g.out_bf16 && row0 < g.n_train && cb < g.ld_bf16)
-                        store_block_rows(g.out_bf16, g.ld_bf16, cb, row0, g.n_train, v, stage_acquire(ws, lane), lane, rows_map);
-                } else if (live && g.out_bf16) {       // this thread's columns, 16 bytes at a time
+                {   // dL row-major (clipped to the trained rows, padding columns zero) and transposed
+                    const bool t_out = g.out_bf16_t && cb < g.N && (!t_map || row0 < g.n_train);
+                    const bool rows_out = rows_map && g.out_bf16 && row0 < g.n_train && cb < g.ld_bf16;
+                    store_block(v, stage, lane, cb, g.N, row0, g.n_train, rows_out, g.out_bf16, g.ld_bf16, rows_map, t_out,
+                                g.out_bf16_t, g.ld_t, t_map);
+                }
+                if (!rows_map && live && g.out_bf16) {       // this thread's columns, 16 bytes at a time
                     __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16 + cb;
 #pragma unroll
                     for (int c = 0; c < 32; c += 8) {
@@ -442,8 +489,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         *reinterpret_cast<uint4*>(dst + c) = pk;
                     }
                 }
-                if (g.out_bf16_t && cb < g.N && (!t_map || row0 < g.n_train))
-                    store_block_transposed(g.out_bf16_t, g.ld_t, cb, g.N, row0, g.n_train, v, stage_acquire(ws, lane), lane, t_map);
                 if (half == 0) {
                     float loss = live ? (mx + __logf(den)) - ly : 0.f;
                     loss = warp_sum(loss);
@@ -454,7 +499,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     g.loss_partial[mt] = ((warp_loss[0] + warp_loss[1]) + warp_loss[2]) + warp_loss[3];
                 // (the exchange arrays and warp_loss are next written after the following tile's first
                 //  barrier-protected phase: every warp passes two more barriers before reusing them)
-            } else if (BN == 64 && g.mode == TC_EPI_ARGMAX) {
+            } else if constexpr (BN == 64 && MODE == TC_EPI_ARGMAX) {
                 // one thread owns the whole row of logits (four of the eight warps take part)
                 float v[64];
                 if (ok) {
@@ -515,7 +560,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (n_kb > 0 && c0 + 32 < c_end) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)(c0 + 32), nxt);
                     const int64_t col0 = n0 + c0;
                     if (col0 >= g.N) continue;
-                    if (g.mode == TC_EPI_PARTIAL) {
+                    if constexpr (MODE == TC_EPI_PARTIAL) {
                         if (row >= g.M) continue;
                         float* dst = g.partial + ((int64_t)z * g.M + row) * g.N + col0;
                         if (col0 + 32 <= g.N && (g.N & 3) == 0 && aligned16(g.partial)) {
@@ -527,39 +572,47 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                             for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __uint_as_float(r[j]);
                         }
-                    } else if (g.mode == TC_EPI_MASK_T || g.mode == TC_EPI_MASK) {
-                        float v[32];
-                        uint8_t* stage = stage_acquire(ws, lane);
-                        if (col0 + 32 <= g.N && (g.ld_mask & 7) == 0 && aligned16(g.mask)) {
-                            uint4 mk[4];      // the gate block, read in 64-byte runs through the staging block
-                            load_block_rows(g.mask, g.ld_mask, col0, row0, g.M, mk, stage, lane);
+                    } else if constexpr (MODE == TC_EPI_MASK_T || MODE == TC_EPI_MASK) {
+                        const bool to_t = MODE == TC_EPI_MASK_T;
+                        const CUtensorMap* out_map = to_t ? t_map : rows_map;
+                        const bool gate_runs = col0 + 32 <= g.N && (g.ld_mask & 7) == 0 && aligned16(g.mask);
+                        if (gate_runs && out_map) {
+                            // the two staging blocks take turns: the bulk store issued two chunks ago has read this one
+                            flip ^= 1;
+                            uint8_t* blk = stage + flip * kStageBlockBytes;
+                            if (lane == 0) bulk_wait_read_but_one();
+                            __syncwarp();
+                            stage_block_from_global(g.mask, g.ld_mask, col0, row0, g.M, blk, lane);   // the gate, in 64-byte runs
+                            uint32_t p[16];
 #pragma unroll
-                            for (int p = 0; p < 4; ++p) {
-                                const __nv_bfloat16* mv = reinterpret_cast<const __nv_bfloat16*>(&mk[p]);
+                            for (int qd = 0; qd < 4; ++qd) {
+                                const uint4 mk = *reinterpret_cast<const uint4*>(blk + lane * 64 + stage_piece(lane, qd) * 16);
+                                const __nv_bfloat16* mv = reinterpret_cast<const __nv_bfloat16*>(&mk);
 #pragma unroll
-                                for (int k = 0; k < 8; ++k)
-                                    v[8 * p + k] = __bfloat162float(mv[k]) > 0.f ? __uint_as_float(r[8 * p + k]) : 0.f;
+                                for (int i = 0; i < 4; ++i) {
+                                    const float lo = __bfloat162float(mv[2 * i]) > 0.f ? __uint_as_float(r[8 * qd + 2 * i]) : 0.f;
+                                    const float hi = __bfloat162float(mv[2 * i + 1]) > 0.f ? __uint_as_float(r[8 * qd + 2 * i + 1]) : 0.f;
+                                    __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
+                                    p[4 * qd + i] = *reinterpret_cast<uint32_t*>(&b2);
+                                }
                             }
-                        } else if (row < g.M) {
-                            const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                v[j] = (col0 + j < g.N && __bfloat162float(mrow[j]) > 0.f) ? __uint_as_float(r[j]) : 0.f;
+                            __syncwarp();         // every lane has read its gate row: the block may take the output
+                            if (row0 < g.M)
+                                store_block_packed(p, stage, lane, col0, row0, to_t ? nullptr : rows_map, to_t ? t_map : nullptr, blk);
                         } else {
+                            float v[32];
+                            if (row < g.M) {
+                                const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) v[j] = 0.f;
-                        }
-                        if (g.mode == TC_EPI_MASK_T) {
-                            if (!t_map || row0 < g.M)
-                                store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage, lane, t_map);
-                        } else if (rows_map) {
-                            if (row0 < g.M) store_block_rows(g.out_bf16, g.ld_bf16, col0, row0, g.M, v, stage, lane, rows_map);
-                        } else if (col0 + 32 <= g.N && (g.ld_bf16 & 7) == 0 && aligned16(g.out_bf16)) {
-                            store_block_rows(g.out_bf16, g.ld_bf16, col0, row0, g.M, v, stage, lane, nullptr);
-                        } else if (row < g.M) {
+                                for (int j = 0; j < 32; ++j)
+                                    v[j] = (col0 + j < g.N && __bfloat162float(mrow[j]) > 0.f) ? __uint_as_float(r[j]) : 0.f;
+                            } else {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + j < g.N) g.out_bf16[row * g.ld_bf16 + col0 + j] = __float2bfloat16_rn(v[j]);
+                                for (int j = 0; j < 32; ++j) v[j] = 0.f;
+                            }
+                            if (row0 < g.M)
+                                store_block(v, stage, lane, col0, g.N, row0, g.M, !to_t, g.out_bf16, g.ld_bf16, rows_map, to_t,
+                                            g.out_bf16_t, g.ld_t, t_map);
                         }
                     } else {
                         float v[32];
@@ -572,16 +625,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             if (g.relu) x = fmaxf(x, 0.f);
                             v[j] = x;
                         }
-                        if (g.out_bf16_t) {
-                            if (!t_map || row0 < g.M)
-                                store_block_transposed(g.out_bf16_t, g.ld_t, col0, g.N, row0, g.M, v, stage_acquire(ws, lane), lane, t_map);
-                            if (g.ones_row_t && col0 == 0 && row < g.M) g.out_bf16_t[g.N * g.ld_t + row] = __float2bfloat16_rn(1.0f);
-                        }
-                        const bool rows_fast = g.out_bf16 && (rows_map || (col0 + 32 <= g.N && (g.ld_bf16 & 7) == 0 && aligned16(g.out_bf16)));
-                        if (rows_fast && (!rows_map || row0 < g.M))
-                            store_block_rows(g.out_bf16, g.ld_bf16, col0, row0, g.M, v, stage_acquire(ws, lane), lane, rows_map);
-                        if (row >= g.M) continue;
-                        if (g.out_f32) {
+                        if (g.out_f32 && row < g.M) {
                             float* dst = g.out_f32 + row * g.ld_f32 + col0;
                             if (col0 + 32 <= g.N && (g.ld_f32 & 3) == 0 && aligned16(g.out_f32)) {
 #pragma unroll
@@ -592,11 +636,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = v[j];
                             }
                         }
-                        if (g.out_bf16 && !rows_fast) {
-                            __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16 + col0;
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __float2bfloat16_rn(v[j]);
-                        }
+                        if (row0 < g.M && (g.out_bf16 || g.out_bf16_t))
+                            store_block(v, stage, lane, col0, g.N, row0, g.M, g.out_bf16 != nullptr, g.out_bf16, g.ld_bf16, rows_map,
+                                        g.out_bf16_t != nullptr, g.out_bf16_t, g.ld_t, t_map);
+                        if (g.out_bf16_t && g.ones_row_t && col0 == 0 && row < g.M)
+                            g.out_bf16_t[g.N * g.ld_t + row] = __float2bfloat16_rn(1.0f);
                     }
                 }
             }
@@ -660,15 +704,15 @@ static bool make_store_map(CUtensorMap* map, const void* base, int64_t rows, int
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int STAGES>
-static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
+template <int BN, int STAGES, int MODE>
+static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
     // stage ring + alignment slack + barrier area + staging blocks (+ the soft-max exchange arrays)
     constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 1024 + kEpiWarps * kStageBytesPerWarp +
                             (BN == 64 ? 4 * 2 * 128 * 4 : 0);
     static_assert(smem <= 227 * 1024, "shared memory budget");
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
             cudaSuccess) {
             (void)cudaGetLastError();
             return RETEXO_ERR_CUDA;
@@ -702,8 +746,26 @@ static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& 
     const int n_sm = sm_count();
     if (n_sm <= 0) return RETEXO_ERR_CUDA;
     const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);      // one persistent block per SM
-    tc_gemm_kernel<BN, STAGES><<<grid, kTcThreads, smem, st>>>(ma, mb, m_rows, m_t, g);
+    tc_gemm_kernel<BN, STAGES, MODE><<<grid, kTcThreads, smem, st>>>(ma, mb, m_rows, m_t, g);
     return launch_status();
+}
+
+template <int BN, int STAGES>
+static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
+    switch (t.mode) {
+        case TC_EPI_BIAS: return launch_tc_mode<BN, STAGES, TC_EPI_BIAS>(t, ma, mb, st);
+        case TC_EPI_PARTIAL: return launch_tc_mode<BN, STAGES, TC_EPI_PARTIAL>(t, ma, mb, st);
+        case TC_EPI_MASK_T: return launch_tc_mode<BN, STAGES, TC_EPI_MASK_T>(t, ma, mb, st);
+        case TC_EPI_MASK: return launch_tc_mode<BN, STAGES, TC_EPI_MASK>(t, ma, mb, st);
+        case TC_EPI_SOFTMAX_CE:
+            if constexpr (BN == 64) return launch_tc_mode<BN, STAGES, TC_EPI_SOFTMAX_CE>(t, ma, mb, st);
+            break;
+        case TC_EPI_ARGMAX:
+            if constexpr (BN == 64) return launch_tc_mode<BN, STAGES, TC_EPI_ARGMAX>(t, ma, mb, st);
+            break;
+        default: break;
+    }
+    return RETEXO_ERR_UNSUPPORTED;
 }
 
 bool tc_gemm_supported(const TcGemm& t) {
