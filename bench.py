@@ -189,7 +189,7 @@ def phase_breakdown(w, ws, R: int, peaks):
         else:
             q = torch.rand((n, ld), dtype=torch.float32, device=dev)
         width = rd["d_in"]
-        x16 = torch.empty((n, (width + 7) // 8 * 8), dtype=torch.bfloat16, device=dev)
+        x16 = torch.empty((n, (width + 63) // 64 * 64), dtype=torch.bfloat16, device=dev)
         if w.aggr == wl.GAT:
             hd = w.heads * w.head_dim
             p = torch.randn((n, (hd + 31) // 32 * 32), dtype=torch.float32, device=dev)

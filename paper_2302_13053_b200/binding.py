@@ -148,7 +148,7 @@ def retexo_aggregate(aggr: int, rowptr: torch.Tensor, colidx: torch.Tensor, q: t
     if want_f32 and out is None:
         out = torch.empty((n, width), dtype=torch.float32, device=dev)
     if want_bf16 and out_bf16 is None:
-        out_bf16 = torch.empty((n, (width + 7) // 8 * 8), dtype=torch.bfloat16, device=dev)
+        out_bf16 = torch.empty((n, (width + 63) // 64 * 64), dtype=torch.bfloat16, device=dev)
     g = _csr(rowptr, colidx)
     gp = None
     keep = []
@@ -175,19 +175,22 @@ def retexo_aggregate(aggr: int, rowptr: torch.Tensor, colidx: torch.Tensor, q: t
 
 
 def retexo_pack_rows(src: torch.Tensor, idx: Optional[torch.Tensor] = None, dim: Optional[int] = None,
-                     transpose: bool = False, ones_row: bool = False):
+                     transpose: bool = False, ones_row: bool = False, ld_multiple: int = 64):
     """bf16 batch of the rows src[idx] (all rows if idx is None).  Returns
-    (dst [n_rows, round_up(dim, 8)], dst_t [dim (+1 with ones_row), round_up(n_rows, 8)] or None)."""
+    (dst [n_rows, round_up(dim, ld_multiple)], dst_t [dim (+1 with ones_row), round_up(n_rows, ld_multiple)]
+    or None).  The library needs leading dimensions that are multiples of 8; multiples of 64 put
+    every row on a 128-byte line, which its bulk tensor loads prefer."""
+    assert ld_multiple % 8 == 0 and ld_multiple > 0
     assert src.dtype in (torch.float32, torch.bfloat16) and src.stride(1) == 1
     dim = int(src.shape[1] if dim is None else dim)
     n_rows = int(src.shape[0] if idx is None else idx.numel())
     dev = src.device
-    ld = (dim + 7) // 8 * 8
+    ld = (dim + ld_multiple - 1) // ld_multiple * ld_multiple
     dst = torch.empty((n_rows, ld), dtype=torch.bfloat16, device=dev)
     dst_t = None
     ld_t = 0
     if transpose:
-        ld_t = (n_rows + 7) // 8 * 8
+        ld_t = (n_rows + ld_multiple - 1) // ld_multiple * ld_multiple
         dst_t = torch.empty((dim + (1 if ones_row else 0), ld_t), dtype=torch.bfloat16, device=dev)
     if idx is not None:
         assert idx.dtype == torch.int32

@@ -107,7 +107,7 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
         s = retexo_aggregate_workspace_size(n, e, c.aggr, r.agg_dim, c.gat_heads);
         if (s > agg_b) agg_b = s;
     }
-    const int64_t ld16 = round_up(max_din, 8);
+    const int64_t ld16 = round_up(max_din, 64);      // bf16 rows start on 128-byte lines
     l.features = t.template take<float>((size_t)n * round_up(c.d0, 32));   // 128-byte-row copy of the features
     if (host) {
         l.rowptr = t.template take<int64_t>((size_t)n + 1);
@@ -124,7 +124,7 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
     l.x16 = t.template take<bf16>((size_t)n * ld16);
     if (c.aggr == RETEXO_GAT) {
         const int32_t hd = c.gat_heads * c.gat_head_dim;
-        l.q16 = t.template take<bf16>((size_t)n * round_up(max_rep, 8));
+        l.q16 = t.template take<bf16>((size_t)n * round_up(max_rep, 64));
         l.proj = t.template take<float>((size_t)n * round_up(hd, 32));
         l.watt16 = t.template take<bf16>((size_t)max_rep * hd);
         l.gat_vec = t.template take<float>((size_t)2 * hd);
@@ -132,7 +132,7 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
     }
     l.xtr16 = t.template take<bf16>((size_t)(n_tr + n_val) * ld16);     // training rows, then validation rows
     l.xval16 = nullptr;
-    l.xtr_t16 = t.template take<bf16>((size_t)(max_din + 1) * (size_t)round_up(n_tr, 8));
+    l.xtr_t16 = t.template take<bf16>((size_t)(max_din + 1) * (size_t)round_up(n_tr, 64));
     l.y_tr = t.template take<int32_t>((size_t)n_tr);
     l.y_val = t.template take<int32_t>((size_t)(n_val > 0 ? n_val : 1));
     l.y_test = t.template take<int32_t>((size_t)(n_te > 0 ? n_te : 1));
@@ -275,19 +275,19 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
     {   // padding columns of the bf16 inputs are never read as data, but keep them defined
         int32_t max_din = 0;
         for (int m = 1; m <= c.K; ++m) if (round_dims(c, m).d_in > max_din) max_din = round_dims(c, m).d_in;
-        RETEXO_CUDA_TRY(cudaMemsetAsync(b.x16, 0, sizeof(bf16) * (size_t)n * (size_t)round_up(max_din, 8), st));
+        RETEXO_CUDA_TRY(cudaMemsetAsync(b.x16, 0, sizeof(bf16) * (size_t)n * (size_t)round_up(max_din, 64), st));
     }
     const float* q = feat;
     int64_t ldq = ld_feat;
     for (int m = 1; m <= c.K; ++m) {
         const RoundDims r = round_dims(c, m);
-        const int64_t ld16 = round_up(r.d_in, 8);
+        const int64_t ld16 = round_up(r.d_in, 64);
         const int64_t nt = retexo_theta_size(r.d_in, r.hidden, c.n_classes);
 
         // ---- one message-passing round: X = COMBINE(Q, AGGR(Q)), emitted in bf16 for the model
         if (c.aggr == RETEXO_GAT) {
             const int32_t hd = r.agg_dim;
-            const int64_t ldq16 = round_up(r.rep_dim, 8), ldp = round_up(hd, 32);
+            const int64_t ldq16 = round_up(r.rep_dim, 64), ldp = round_up(hd, 32);
             const size_t wcount = (size_t)r.rep_dim * hd + 2 * (size_t)hd;
             RETEXO_CUDA_TRY(cudaMemcpyAsync(b.gat_stage, in->gat_w[m - 1], sizeof(float) * wcount,
                                             cudaMemcpyDefault, st));
@@ -308,7 +308,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         }
 
         // ---- the round's batches and model state
-        const int64_t ld_xt = round_up(n_tr, 8);
+        const int64_t ld_xt = round_up(n_tr, 64);
         RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld16, b.xtr_t16, ld_xt, 1, st));
         bf16* xval16 = b.xtr16 + (size_t)n_tr * ld16;
         if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, xval16, ld16, nullptr, 0, 0, st));

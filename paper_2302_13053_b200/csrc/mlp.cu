@@ -19,7 +19,9 @@ using namespace retexo;
 
 namespace retexo {
 
-static inline int64_t round_up8(int64_t x) { return (x + 7) / 8 * 8; }
+// Leading dimension of a bf16 matrix: rows start on 128-byte lines, so that no 128-byte row of a
+// tensor-map box straddles two lines.
+static inline int64_t pad_ld(int64_t x) { return (x + 63) / 64 * 64; }
 
 static int launch_gemm(const GemmArgs& g, cudaStream_t st) {
     if (g.M <= 0 || g.N <= 0) return RETEXO_OK;
@@ -58,10 +60,10 @@ MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_row
     p.d_in = d_in; p.hidden = hidden; p.n_classes = n_classes; p.n_rows = n_rows; p.n_eval = n_eval;
     p.out1 = hidden > 0 ? hidden : n_classes;
     p.nt = retexo_theta_size(d_in, hidden, n_classes);
-    p.ld_dl = round_up8(n_classes);
-    p.ld_h = round_up8(hidden > 0 ? hidden : 1);
-    p.ld_k = round_up8(d_in);
-    p.ld_n = round_up8(n_rows + n_eval);
+    p.ld_dl = pad_ld(n_classes);
+    p.ld_h = pad_ld(hidden > 0 ? hidden : 1);
+    p.ld_k = pad_ld(d_in);
+    p.ld_n = pad_ld(n_rows + n_eval);
     p.sm_blocks = (n_rows + n_eval + 127) / 128;          // one loss partial per 128-row tile of the head product
     p.split_w1 = tc_split((int64_t)d_in + 1, p.out1, n_rows);
     p.split_w2 = hidden > 0 ? tc_split((int64_t)hidden + 1, n_classes, n_rows) : 0;
@@ -259,7 +261,8 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     const double t = (double)(model->step + 1);
     u.corr1 = (float)(1.0 - pow((double)model->beta1, t));
     u.corr2 = (float)(1.0 - pow((double)model->beta2, t));
-    u.loss_partial = b.loss_partial; u.n_loss = p.sm_blocks; u.inv_rows = 1.0f / (float)n; u.loss_out = loss_out;
+    u.loss_partial = b.loss_partial; u.n_loss = (n_all + 127) / 128;      // the tiles this launch's head product wrote
+    u.inv_rows = 1.0f / (float)n; u.loss_out = loss_out;
     u.status = b.status;
     u.w1t16 = b.w1t16; u.ld_k = p.ld_k; u.w2t16 = H > 0 ? b.w2t16 : nullptr; u.ld_h = p.ld_h;
     u.w2p16 = H > 0 ? b.w2p16 : nullptr; u.ld_dl = p.ld_dl;
@@ -295,11 +298,11 @@ extern "C" size_t retexo_embed_workspace_size(int32_t d_in, int32_t hidden, int3
     if (d_in <= 0 || hidden < 0 || n_classes <= 0 || n_rows < 0) return 0;
     Sizer s;
     const size_t out1 = hidden > 0 ? hidden : n_classes;
-    s.take<bf16>(out1 * (size_t)round_up8(d_in));                                   // W1^T
-    s.take<bf16>(hidden > 0 ? (size_t)n_classes * round_up8(hidden) : 1);           // W2^T
-    s.take<bf16>(hidden > 0 ? (size_t)hidden * round_up8(n_classes) : 1);           // W2 padded (unused here)
+    s.take<bf16>(out1 * (size_t)pad_ld(d_in));                                   // W1^T
+    s.take<bf16>(hidden > 0 ? (size_t)n_classes * pad_ld(hidden) : 1);           // W2^T
+    s.take<bf16>(hidden > 0 ? (size_t)hidden * pad_ld(n_classes) : 1);           // W2 padded (unused here)
     s.take<bf16>((size_t)retexo_theta_size(d_in, hidden, n_classes));               // row-major bf16 theta
-    s.take<bf16>(hidden > 0 ? (size_t)n_rows * round_up8(hidden) : 1);              // Hd
+    s.take<bf16>(hidden > 0 ? (size_t)n_rows * pad_ld(hidden) : 1);              // Hd
     s.take<float>((size_t)n_rows * n_classes);                                      // logits
     s.take<int32_t>(64);
     return s.off + kAlign;

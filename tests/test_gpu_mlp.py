@@ -37,8 +37,10 @@ def test_pack_rows_gathers_rounds_and_transposes():
     src = rng.standard_normal((70, 37)).astype(np.float32)
     idx = rng.integers(0, 70, 45).astype(np.int32)
     want = torch.from_numpy(src[idx]).to(torch.bfloat16)
+    dst, dst_t = B().retexo_pack_rows(dev(src), dev(idx), transpose=True)
+    assert dst.shape == (45, 64) and dst_t.shape == (37, 64)          # default: rows on 128-byte lines
     for source in (dev(src), dev(src).to(torch.bfloat16)):
-        dst, dst_t = B().retexo_pack_rows(source, dev(idx), transpose=True)
+        dst, dst_t = B().retexo_pack_rows(source, dev(idx), transpose=True, ld_multiple=8)
         assert dst.shape == (45, 40) and dst_t.shape == (37, 48)
         ref = want if source.dtype == torch.float32 else want
         assert torch.equal(dst[:, :37].cpu(), ref)
@@ -47,7 +49,7 @@ def test_pack_rows_gathers_rounds_and_transposes():
     dst, _ = B().retexo_pack_rows(dev(src), None, dim=20)
     assert torch.equal(dst[:, :20].cpu(), torch.from_numpy(src[:, :20]).to(torch.bfloat16))
     # the row of ones that carries the bias gradient through the weight-gradient product
-    _, dst_t = B().retexo_pack_rows(dev(src), dev(idx), transpose=True, ones_row=True)
+    _, dst_t = B().retexo_pack_rows(dev(src), dev(idx), transpose=True, ones_row=True, ld_multiple=8)
     assert dst_t.shape == (38, 48)
     assert torch.equal(dst_t[:37, :45].cpu(), want.T)
     assert torch.equal(dst_t[37].float().cpu(), torch.cat([torch.ones(45), torch.zeros(3)]))
@@ -64,7 +66,7 @@ def test_train_steps_track_the_checker(d_in, hidden, n_classes, n, opt):
     # Adam's first steps move every weight by about lr whatever the gradient's size, so weights whose
     # gradient is at rounding level take a different step in fp32 and fp64: keep that step small.
     ref, gpu = make_pair(d_in, hidden, n_classes, 1, opt=opt, lr=0.02 if opt == oracle.SGD else 1e-3)
-    x16, x_t = B().retexo_pack_rows(dev(x), None, transpose=True, ones_row=True)
+    x16, x_t = B().retexo_pack_rows(dev(x), None, transpose=True, ones_row=True, ld_multiple=8 if n % 2 else 64)
     yd = dev(y)
     for it in range(4):
         # Every iteration starts from the GPU's own state, so that each step is compared on its
