@@ -403,6 +403,31 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const CUtensorMap* rows_map = g.tma_rows ? &map_rows : nullptr;
         const CUtensorMap* t_map = g.tma_t ? &map_t : nullptr;
         const bool row_owner = BN == 64 && MODE == TC_EPI_ARGMAX;
+        constexpr bool kGated = MODE == TC_EPI_MASK || MODE == TC_EPI_MASK_T;
+        // soft-max epilogue: this warp's 32 bias values never change (its columns are the same in every tile)
+        float ce_bias_lane = 0.f;
+        if constexpr (BN == 64 && MODE == TC_EPI_SOFTMAX_CE)
+            ce_bias_lane = (g.bias && half * 32 + lane < g.N) ? __ldg(g.bias + half * 32 + lane) : 0.f;
+        // gated epilogue: the gate block of the next chunk is fetched while the current chunk is processed
+        uint4 gate_next[4];
+        bool gate_have = false;
+        [[maybe_unused]] auto gate_prefetch = [&](int64_t tile, int c0) {
+            gate_have = false;
+            if (tile >= n_tiles) return;
+            const int64_t rem = tile % per_split;
+            const int64_t r0 = (rem % n_m) * kTcBM + q * 32, cc0 = (rem / n_m) * BN + c0;
+            const CUtensorMap* out_map = MODE == TC_EPI_MASK_T ? t_map : rows_map;
+            if (!out_map || r0 >= g.M || cc0 + 32 > g.N || (g.ld_mask & 7) != 0 || !aligned16(g.mask)) return;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int line = (lane >> 2) + 8 * i, piece = lane & 3;
+                gate_next[i] = make_uint4(0u, 0u, 0u, 0u);
+                if (r0 + line < g.M)
+                    gate_next[i] = __ldg(reinterpret_cast<const uint4*>(g.mask + (r0 + line) * g.ld_mask + cc0 + piece * 8));
+            }
+            gate_have = true;
+        };
+        if constexpr (kGated) gate_prefetch(blockIdx.x, half * (BN / 2));
         int64_t lt = 0;
         for (int64_t t = blockIdx.x; t < n_tiles && !(row_owner && half == 1); t += gridDim.x, ++lt) {
             const int64_t z = t / per_split, rem = t % per_split;
@@ -415,6 +440,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t acc_addr = tmem_acc + (uint32_t)(b * BN);
             const int64_t row0 = m0 + q * 32;
             const int64_t row = row0 + lane;
+            int32_t ce_label = -1;          // soft-max epilogue: fetched before the wait so that its latency is hidden
+            if constexpr (BN == 64 && MODE == TC_EPI_SOFTMAX_CE)
+                ce_label = (row < g.M && row < g.n_train && g.y) ? g.y[row] : -1;
             const bool ok = mbar_wait(acc_full + b, pb, g.status, abort_flag);
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             if (!ok) break;
@@ -431,14 +459,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                         for (int j = 0; j < 32; ++j) r[j] = 0u;
                     }
-                    const float bias_lane = (g.bias && cb + lane < g.N) ? __ldg(g.bias + cb + lane) : 0.f;
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        v[j] = cb + j < g.N ? __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j) : -INFINITY;
+                        v[j] = cb + j < g.N ? __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, ce_bias_lane, j) : -INFINITY;
                 }
                 const bool is_eval = row >= g.n_train;
                 const bool live = row < g.M && !is_eval;
-                const int32_t yi = (live && g.y) ? g.y[row] : -1;
+                const int32_t yi = live ? ce_label : -1;
                 float mx = v[0];
                 int best = 0;
 #pragma unroll
@@ -542,24 +569,39 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (lane == 0 && hits) atomicAdd(g.correct, (unsigned long long)__popc(hits));
                 }
             } else if (ok) {
-                // the load of chunk c + 1 is in flight while chunk c is processed
-                uint32_t nxt[32];
+                // the accumulator load of chunk c + 1 is in flight while chunk c is processed (gated modes
+                // spend those registers on the gate block of chunk c + 1 instead)
+                [[maybe_unused]] uint32_t nxt[32];
                 constexpr int kHalfCols = BN / 2;
                 const int c_begin = half * kHalfCols, c_end = c_begin + kHalfCols;
-                if (n_kb > 0) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)c_begin, nxt);
-                else {
+                if constexpr (!kGated) {
+                    if (n_kb > 0) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)c_begin, nxt);
+                    else {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) nxt[j] = 0u;
+                        for (int j = 0; j < 32; ++j) nxt[j] = 0u;
+                    }
                 }
 #pragma unroll 1
                 for (int c0 = c_begin; c0 < c_end; c0 += 32) {
                     uint32_t r[32];
-                    if (n_kb > 0) tmem_ld_wait(nxt);
+                    if constexpr (!kGated) {
+                        if (n_kb > 0) tmem_ld_wait(nxt);
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = nxt[j];
-                    if (n_kb > 0 && c0 + 32 < c_end) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)(c0 + 32), nxt);
+                        for (int j = 0; j < 32; ++j) r[j] = nxt[j];
+                        if (n_kb > 0 && c0 + 32 < c_end)
+                            tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)(c0 + 32), nxt);
+                    } else {
+                        if (n_kb > 0) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                        else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) r[j] = 0u;
+                        }
+                    }
                     const int64_t col0 = n0 + c0;
-                    if (col0 >= g.N) continue;
+                    if (col0 >= g.N) {
+                        if constexpr (kGated) { if (n_kb > 0) tmem_ld_wait(r); }
+                        continue;
+                    }
                     if constexpr (MODE == TC_EPI_PARTIAL) {
                         if (row >= g.M) continue;
                         float* dst = g.partial + ((int64_t)z * g.M + row) * g.N + col0;
@@ -576,13 +618,30 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const bool to_t = MODE == TC_EPI_MASK_T;
                         const CUtensorMap* out_map = to_t ? t_map : rows_map;
                         const bool gate_runs = col0 + 32 <= g.N && (g.ld_mask & 7) == 0 && aligned16(g.mask);
+                        // this chunk's gate block (if it was fetched ahead), then the fetch for the next chunk
+                        uint4 gate_cur[4];
+                        const bool have_gate = gate_have;
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) gate_cur[i] = gate_next[i];
+                        if (c0 + 32 < c_end) gate_prefetch(t, c0 + 32);
+                        else gate_prefetch(t + gridDim.x, c_begin);
                         if (gate_runs && out_map) {
                             // the two staging blocks take turns: the bulk store issued two chunks ago has read this one
                             flip ^= 1;
                             uint8_t* blk = stage + flip * kStageBlockBytes;
                             if (lane == 0) bulk_wait_read_but_one();
                             __syncwarp();
-                            stage_block_from_global(g.mask, g.ld_mask, col0, row0, g.M, blk, lane);   // the gate, in 64-byte runs
+                            if (have_gate) {      // 64-byte runs from global memory, one row per lane out of the block
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) {
+                                    const int line = (lane >> 2) + 8 * i, piece = lane & 3;
+                                    *reinterpret_cast<uint4*>(blk + line * 64 + stage_piece(line, piece) * 16) = gate_cur[i];
+                                }
+                                __syncwarp();
+                            } else {
+                                stage_block_from_global(g.mask, g.ld_mask, col0, row0, g.M, blk, lane);
+                            }
+                            if (n_kb > 0) tmem_ld_wait(r);
                             uint32_t p[16];
 #pragma unroll
                             for (int qd = 0; qd < 4; ++qd) {
@@ -600,6 +659,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             if (row0 < g.M)
                                 store_block_packed(p, stage, lane, col0, row0, to_t ? nullptr : rows_map, to_t ? t_map : nullptr, blk);
                         } else {
+                            if (n_kb > 0) tmem_ld_wait(r);
                             float v[32];
                             if (row < g.M) {
                                 const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
