@@ -172,3 +172,42 @@ def test_gat_config3_projected_input():
     ref = oracle.aggregate(oracle.GAT, w.rowptr, w.colidx, p, gat=gat)
     got, _ = gat_gpu(w.rowptr, w.colidx, p, gat)
     assert_rows_close(got, ref, what=w.name)
+
+
+def ladder_in_a_large_graph(n, seed):
+    """The degree ladder (hubs of every bin, isolated nodes) embedded in a graph of n nodes whose
+    other nodes have a few random neighbours; node ids shuffled."""
+    rng = np.random.default_rng(seed)
+    edges = []
+    nxt = len(LADDER)
+    for h, d in enumerate(LADDER):
+        edges.append(np.stack([np.full(d, h, dtype=np.int64), np.arange(nxt, nxt + d, dtype=np.int64)], axis=1))
+        nxt += d
+    assert nxt + 16 < n
+    rest = rng.integers(nxt + 8, n, size=(3 * n, 2))          # nodes nxt .. nxt+7 stay isolated
+    e = np.concatenate(edges + [rest])
+    perm = rng.permutation(n)
+    return wl.csr_from_edge_list(n, perm[e])
+
+
+@pytest.mark.parametrize("aggr,n,dim", [(oracle.SAGE_MEAN, 120000, 850), (oracle.GCN, 170000, 602),
+                                        (oracle.SAGE_MEAN, 300000, 340), (oracle.GCN, 300000, 342),
+                                        (oracle.SAGE_MAX, 170000, 600)])
+def test_matrices_beyond_the_cache_take_the_column_slab_variant(aggr, n, dim):
+    """A feature matrix of ~400 MB or more is aggregated slab of columns by slab of columns (32, 16
+    or 8 vectors per slab, by the number of rows): same tolerance, every degree bin, ragged last slab."""
+    rowptr, colidx = ladder_in_a_large_graph(n, seed=dim)
+    rng = np.random.default_rng(dim)
+    q = rng.standard_normal((n, dim)).astype(np.float32)
+    if aggr != oracle.SAGE_MAX:
+        q = np.abs(q) + 0.5
+    ld = (dim + 3) // 4 * 4
+    ref = oracle.aggregate(aggr, rowptr, colidx, q)
+    got, got16 = run_gpu(aggr, rowptr, colidx, q, ld=ld)
+    if aggr == oracle.SAGE_MAX:
+        np.testing.assert_array_equal(got, ref)
+    else:
+        assert_rows_close(got, ref, what="fp32 out")
+    np.testing.assert_array_equal(got16[:, :got.shape[1]], torch.from_numpy(got).to(torch.bfloat16).float().numpy())
+    again, _ = run_gpu(aggr, rowptr, colidx, q, ld=ld)
+    np.testing.assert_array_equal(again, got)                 # repeatable bit for bit
