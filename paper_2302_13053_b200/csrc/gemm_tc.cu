@@ -2,9 +2,9 @@
 //   C[M x N] = A[M x K] * B[N x K]^T,  A and B bf16 with K contiguous,
 //   fp32 accumulation in tensor memory (tcgen05.mma, cta_group::1, M = 128).
 // Operand tiles are brought in by TMA (128-byte swizzle) through a ring of
-// shared-memory stages guarded by mbarriers; one thread issues the MMAs; four
-// warps drain the accumulator with tcgen05.ld and apply the fused epilogue
-// (bias / ReLU / bf16 down-cast, or a raw split-K partial).
+// shared-memory stages guarded by mbarriers; one thread issues the MMAs; eight
+// or sixteen warps drain the accumulators with tcgen05.ld and apply the fused
+// epilogue (bias / ReLU / bf16 down-cast, soft-max loss, gate, split-K partial).
 // Every wait is bounded: a wait that runs out sets *status and the block
 // tears down in order (outstanding copies awaited, tensor memory freed).
 #include <cuda.h>
@@ -17,9 +17,23 @@ namespace retexo {
 
 constexpr int kTcBM = 128;
 constexpr int kTcBK = 64;                  // 64 bf16 = 128 bytes = one swizzle row
-constexpr int kTcThreads = 320;            // warp 0: TMA, warp 1: MMA + tensor-memory owner, warps 2..9: epilogue
-constexpr int kEpiWarps = 8;               // two per tensor-memory lane quarter, each taking half of the columns
+// Threads: warp 0 TMA, warp 1 MMA + tensor-memory owner, then EW epilogue warps (8 or 16).  The epilogues
+// are chains of dependent instructions, so their speed is set by how many warps share an SM's schedulers:
+// with 16 warps a tile's columns are cut four ways (BN >= 128), or (BN = 64, where a row of logits is
+// shared by two threads) two groups of 8 warps take alternate tiles out of four accumulators.
 constexpr uint32_t kSpinLimit = 1u << 26;
+#ifndef TC256_EW
+#define TC256_EW 8
+#define TC256_STAGES 4
+#endif
+#ifndef TC128_EW
+#define TC128_EW 16
+#define TC128_STAGES 4
+#endif
+#ifndef TC64_EW
+#define TC64_EW 16
+#define TC64_STAGES 5
+#endif
 
 __device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -294,26 +308,30 @@ __device__ __forceinline__ void stage_block_from_global(const __nv_bfloat16* src
 
 // MODE (a TcEpilogue value) is a template parameter so that every instantiation carries the registers of
 // its own epilogue only.
-template <int BN, int STAGES, int MODE>
-__global__ void __launch_bounds__(kTcThreads, 1)
+template <int BN, int STAGES, int MODE, int EW>
+__global__ void __launch_bounds__(64 + 32 * EW, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_rows, const __grid_constant__ CUtensorMap map_t, TcKernelArgs g) {
     // Persistent: the block walks over output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...  The
-    // stage ring runs on across tiles and the accumulator is double-buffered in tensor memory, so
-    // the loads and MMAs of the next tile overlap the epilogue of the current one.
+    // stage ring runs on across tiles and the accumulator is multi-buffered in tensor memory, so
+    // the loads and MMAs of the next tile(s) overlap the epilogue of the current one.
+    constexpr int TG = (BN == 64 && EW == 16) ? 2 : 1;      // groups of epilogue warps that take alternate tiles
+    constexpr int CP = EW / 4 / TG;                         // column parts a tile is cut into
+    constexpr int NACC = 2 * TG;                            // accumulators in tensor memory
+    static_assert(BN % (32 * CP) == 0 && NACC * BN <= 512, "tile split");
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t kABytes = kTcBM * kTcBK * 2, kBBytes = BN * kTcBK * 2, kStageBytes = kABytes + kBBytes;
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(tiles + STAGES * kStageBytes);
     uint64_t* empty = full + STAGES;
-    uint64_t* acc_full = empty + STAGES;          // [2] accumulator b holds a finished tile
-    uint64_t* acc_empty = acc_full + 2;           // [2] accumulator b has been drained
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+    uint64_t* acc_full = empty + STAGES;          // [NACC] accumulator b holds a finished tile
+    uint64_t* acc_empty = acc_full + NACC;        // [NACC] accumulator b has been drained
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + NACC);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    float* warp_loss = reinterpret_cast<float*>(tmem_slot + 2);                  // [4]
-    // staging blocks: kEpiWarps x kStageBytesPerWarp, 1024 bytes behind the barrier area (so 1024-byte aligned)
+    float* warp_loss_all = reinterpret_cast<float*>(tmem_slot + 2);              // [TG][4]
+    // staging blocks: EW x kStageBytesPerWarp, 1024 bytes behind the barrier area (so 1024-byte aligned)
     uint8_t* stage_base = tiles + STAGES * kStageBytes + 1024;
-    float (*xch)[2][128] = reinterpret_cast<float (*)[2][128]>(stage_base + kEpiWarps * kStageBytesPerWarp);   // [4][2][128]
+    float (*xch_all)[2][128] = reinterpret_cast<float (*)[2][128]>(stage_base + EW * kStageBytesPerWarp);   // [TG][4][2][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int64_t n_m = (g.M + kTcBM - 1) / kTcBM, n_n = (g.N + BN - 1) / BN;
@@ -324,12 +342,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int s = 0; s < STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
         // the arg-max epilogue lets one thread own a whole row of logits: it uses four of the eight warps
         const bool row_owner = BN == 64 && MODE == TC_EPI_ARGMAX;
-        for (int b = 0; b < 2; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, row_owner ? 4 : kEpiWarps); }
+        for (int b = 0; b < NACC; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, row_owner ? 4 : EW / TG); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {      // tensor memory: two accumulators of BN fp32 columns x 128 lanes
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(2 * BN));
+    if (warp == 1) {      // tensor memory: NACC accumulators of BN fp32 columns x 128 lanes
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(NACC * BN));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -373,8 +391,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const int64_t z = t / per_split;
                 const int32_t kb0 = (int32_t)z * g.k_blocks_per_split;
                 const int32_t kb1 = min(g.k_blocks_total, kb0 + g.k_blocks_per_split);
-                const int b = (int)(lt & 1);
-                const uint32_t pb = (uint32_t)(lt >> 1) & 1;
+                const int b = (int)(lt % NACC);
+                const uint32_t pb = (uint32_t)(lt / NACC) & 1;
                 ok = mbar_wait(acc_empty + b, pb ^ 1, g.status, abort_flag);      // drained by the epilogue
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -397,8 +415,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else {
         const int q = warp & 3;                           // tensor-memory lane quarter this warp may read
-        const int half = (warp - 2) >> 2;                 // which half of the tile's columns this warp drains
-        uint8_t* stage = stage_base + (warp - 2) * kStageBytesPerWarp;      // this warp's two staging blocks
+        const int ew = warp - 2;
+        const int gi = TG == 2 ? ew >> 3 : 0;             // tile group of this warp
+        const int half = (ew >> 2) % CP;                  // which part of the tile's columns this warp drains
+        constexpr int kPartCols = BN / CP;
+        float* warp_loss = warp_loss_all + gi * 4;
+        float (*xch)[2][128] = xch_all + gi * 4;
+        uint8_t* stage = stage_base + ew * kStageBytesPerWarp;      // this warp's two staging blocks
         int flip = 0;
         const CUtensorMap* rows_map = g.tma_rows ? &map_rows : nullptr;
         const CUtensorMap* t_map = g.tma_t ? &map_t : nullptr;
@@ -427,16 +450,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             gate_have = true;
         };
-        if constexpr (kGated) gate_prefetch(blockIdx.x, half * (BN / 2));
-        int64_t lt = 0;
-        for (int64_t t = blockIdx.x; t < n_tiles && !(row_owner && half == 1); t += gridDim.x, ++lt) {
+        if constexpr (kGated) gate_prefetch(blockIdx.x + (int64_t)gi * gridDim.x, half * kPartCols);
+        int64_t lt = gi;
+        for (int64_t t = blockIdx.x + (int64_t)gi * gridDim.x; t < n_tiles && !(row_owner && half == 1);
+             t += (int64_t)TG * gridDim.x, lt += TG) {
             const int64_t z = t / per_split, rem = t % per_split;
             const int64_t mt = rem % n_m;
             const int64_t m0 = mt * kTcBM, n0 = (rem / n_m) * BN;
             const int32_t kb0 = (int32_t)z * g.k_blocks_per_split;
             const int32_t n_kb = min(g.k_blocks_total, kb0 + g.k_blocks_per_split) - kb0;
-            const int b = (int)(lt & 1);
-            const uint32_t pb = (uint32_t)(lt >> 1) & 1;
+            const int b = (int)(lt % NACC);
+            const uint32_t pb = (uint32_t)(lt / NACC) & 1;
             const uint32_t acc_addr = tmem_acc + (uint32_t)(b * BN);
             const int64_t row0 = m0 + q * 32;
             const int64_t row = row0 + lane;
@@ -472,7 +496,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 for (int j = 1; j < 32; ++j) if (v[j] > mx) { mx = v[j]; best = j; }      // strict: lowest index on ties
                 xch[0][half][slot] = mx;
                 xch[1][half][slot] = __int_as_float(cb + best);
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+                asm volatile("bar.sync %0, 256;" ::"r"(1 + gi) : "memory");
                 const float m0v = xch[0][0][slot], m1v = xch[0][1][slot];
                 if (g.n_train < g.M && m0 + kTcBM > g.n_train && half == 0) {
                     // evaluation rows in this tile: arg-max over both halves (the lower half wins ties)
@@ -491,7 +515,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 }
                 xch[2][half][slot] = den;
                 xch[3][half][slot] = ly;
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+                asm volatile("bar.sync %0, 256;" ::"r"(1 + gi) : "memory");
                 den = xch[2][0][slot] + xch[2][1][slot];
                 ly = xch[3][0][slot] + xch[3][1][slot];
                 const float scale = g.inv_rows / den;
@@ -521,8 +545,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     loss = warp_sum(loss);
                     if (lane == 0) warp_loss[q] = loss;
                 }
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (warp == 2 && lane == 0 && g.loss_partial)
+                asm volatile("bar.sync %0, 256;" ::"r"(1 + gi) : "memory");
+                if ((ew & 7) == 0 && lane == 0 && g.loss_partial)
                     g.loss_partial[mt] = ((warp_loss[0] + warp_loss[1]) + warp_loss[2]) + warp_loss[3];
                 // (the exchange arrays and warp_loss are next written after the following tile's first
                 //  barrier-protected phase: every warp passes two more barriers before reusing them)
@@ -572,8 +596,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 // the accumulator load of chunk c + 1 is in flight while chunk c is processed (gated modes
                 // spend those registers on the gate block of chunk c + 1 instead)
                 [[maybe_unused]] uint32_t nxt[32];
-                constexpr int kHalfCols = BN / 2;
-                const int c_begin = half * kHalfCols, c_end = c_begin + kHalfCols;
+                const int c_begin = half * kPartCols, c_end = c_begin + kPartCols;
                 if constexpr (!kGated) {
                     if (n_kb > 0) tmem_ld_issue(acc_addr + ((uint32_t)(q * 32) << 16) + (uint32_t)c_begin, nxt);
                     else {
@@ -624,7 +647,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                         for (int i = 0; i < 4; ++i) gate_cur[i] = gate_next[i];
                         if (c0 + 32 < c_end) gate_prefetch(t, c0 + 32);
-                        else gate_prefetch(t + gridDim.x, c_begin);
+                        else gate_prefetch(t + (int64_t)TG * gridDim.x, c_begin);
                         if (gate_runs && out_map) {
                             // the two staging blocks take turns: the bulk store issued two chunks ago has read this one
                             flip ^= 1;
@@ -715,7 +738,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __syncthreads();
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(2 * BN));
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(NACC * BN));
     }
 }
 
@@ -764,15 +787,15 @@ static bool make_store_map(CUtensorMap* map, const void* base, int64_t rows, int
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int STAGES, int MODE>
+template <int BN, int STAGES, int MODE, int EW>
 static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
     // stage ring + alignment slack + barrier area + staging blocks (+ the soft-max exchange arrays)
-    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 1024 + kEpiWarps * kStageBytesPerWarp +
-                            (BN == 64 ? 4 * 2 * 128 * 4 : 0);
+    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 1024 + EW * kStageBytesPerWarp +
+                            (BN == 64 ? (EW / 8) * 4 * 2 * 128 * 4 : 0);
     static_assert(smem <= 227 * 1024, "shared memory budget");
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES, MODE, EW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
             cudaSuccess) {
             (void)cudaGetLastError();
             return RETEXO_ERR_CUDA;
@@ -806,22 +829,22 @@ static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensor
     const int n_sm = sm_count();
     if (n_sm <= 0) return RETEXO_ERR_CUDA;
     const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);      // one persistent block per SM
-    tc_gemm_kernel<BN, STAGES, MODE><<<grid, kTcThreads, smem, st>>>(ma, mb, m_rows, m_t, g);
+    tc_gemm_kernel<BN, STAGES, MODE, EW><<<grid, 64 + 32 * EW, smem, st>>>(ma, mb, m_rows, m_t, g);
     return launch_status();
 }
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, int EW>
 static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
     switch (t.mode) {
-        case TC_EPI_BIAS: return launch_tc_mode<BN, STAGES, TC_EPI_BIAS>(t, ma, mb, st);
-        case TC_EPI_PARTIAL: return launch_tc_mode<BN, STAGES, TC_EPI_PARTIAL>(t, ma, mb, st);
-        case TC_EPI_MASK_T: return launch_tc_mode<BN, STAGES, TC_EPI_MASK_T>(t, ma, mb, st);
-        case TC_EPI_MASK: return launch_tc_mode<BN, STAGES, TC_EPI_MASK>(t, ma, mb, st);
+        case TC_EPI_BIAS: return launch_tc_mode<BN, STAGES, TC_EPI_BIAS, EW>(t, ma, mb, st);
+        case TC_EPI_PARTIAL: return launch_tc_mode<BN, STAGES, TC_EPI_PARTIAL, EW>(t, ma, mb, st);
+        case TC_EPI_MASK_T: return launch_tc_mode<BN, STAGES, TC_EPI_MASK_T, EW>(t, ma, mb, st);
+        case TC_EPI_MASK: return launch_tc_mode<BN, STAGES, TC_EPI_MASK, EW>(t, ma, mb, st);
         case TC_EPI_SOFTMAX_CE:
-            if constexpr (BN == 64) return launch_tc_mode<BN, STAGES, TC_EPI_SOFTMAX_CE>(t, ma, mb, st);
+            if constexpr (BN == 64) return launch_tc_mode<BN, STAGES, TC_EPI_SOFTMAX_CE, EW>(t, ma, mb, st);
             break;
         case TC_EPI_ARGMAX:
-            if constexpr (BN == 64) return launch_tc_mode<BN, STAGES, TC_EPI_ARGMAX>(t, ma, mb, st);
+            if constexpr (BN == 64) return launch_tc_mode<BN, STAGES, TC_EPI_ARGMAX, EW>(t, ma, mb, st);
             break;
         default: break;
     }
@@ -847,9 +870,9 @@ int tc_gemm_launch(const TcGemm& t, cudaStream_t st) {
     CUtensorMap ma, mb;
     if (!make_map(&ma, t.A, t.M, t.K, t.lda, kTcBM)) return RETEXO_ERR_CUDA;
     if (!make_map(&mb, t.B, t.N, t.K, t.ldb, bn)) return RETEXO_ERR_CUDA;
-    if (bn == 256) return launch_tc<256, 4>(t, ma, mb, st);
-    if (bn == 128) return launch_tc<128, 6>(t, ma, mb, st);
-    return launch_tc<64, 7>(t, ma, mb, st);
+    if (bn == 256) return launch_tc<256, TC256_STAGES, TC256_EW>(t, ma, mb, st);
+    if (bn == 128) return launch_tc<128, TC128_STAGES, TC128_EW>(t, ma, mb, st);
+    return launch_tc<64, TC64_STAGES, TC64_EW>(t, ma, mb, st);
 }
 
 }  // namespace retexo
