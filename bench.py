@@ -34,11 +34,26 @@ import numpy as np
 METRIC = "edges aggregated/s"
 UNIT = "edges/s"
 
-# DRAM bytes (read + write) per launch of the aggregation kernel, from the one-pass ncu capture
-# summarised in profiles/agg_rows_kernel_cfg4.txt.  Valid for that kernel and workload only:
-# set an entry to None when agg_rows_kernel or the workload changes.
-AGG_DRAM_TRAFFIC = {("cfg4_sage_reddit_like", 1): 193.76e9, ("cfg4_sage_reddit_like", 2): 55.57e9,
-                    ("cfg4_sage_reddit_like", 3): 55.59e9}
+# DRAM bytes (read + write) per launch of the aggregation kernel, from the one-pass ncu captures
+# summarised in profiles/agg_kernels_cfg4.txt and profiles/agg_rows_kernel_cfg5.txt.  Valid for that
+# kernel and workload only: set an entry to None when the kernel or the workload changes.
+AGG_DRAM_TRAFFIC = {("cfg4_sage_reddit_like", 1): 14.68e9, ("cfg4_sage_reddit_like", 2): 6.24e9,
+                    ("cfg4_sage_reddit_like", 3): 5.99e9, ("cfg5_gcn_products_like", 1): 54.13e9}
+# DRAM bytes of one stand-alone training iteration (its five tc_gemm_kernel launches and
+# reduce_update_kernel), from the one-pass capture summarised in profiles/tc_gemm_kernel_cfg4.txt.
+STEP_DRAM_TRAFFIC = {("cfg4_sage_reddit_like", 1): 1.280e9}
+
+
+def min_time_roofline(flops: float, nbytes: float, ms: float, peaks) -> dict:
+    """Min-time roofline of a dense product (or a chain of them): the slower of flops / tensor peak
+    and bytes / HBM peak is the bound; `achieved` is quoted in that bound's unit."""
+    t_tensor = flops / (peaks["bf16_sustained"] * 1e12) * 1e3
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+    if t_hbm >= t_tensor:
+        return dict(bound="hbm", achieved=nbytes / ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s",
+                    algorithmic_bytes=nbytes, flops=flops, tflops=flops / ms / 1e9, min_ms=t_hbm)
+    return dict(bound="tensor", achieved=flops / ms / 1e9, peak=peaks["bf16_sustained"], unit="TFLOP/s",
+                algorithmic_bytes=nbytes, flops=flops, gbs=nbytes / ms / 1e6, min_ms=t_tensor)
 
 
 def load_peaks():
@@ -210,33 +225,46 @@ def phase_breakdown(w, ws, R: int, peaks):
         xva, _ = B.retexo_pack_rows(x16, va, dim=width)
         H, O = rd["hidden"], w.n_classes
         n_tr, n_va = tr.numel(), va.numel()
+        # algorithmic bytes: every product reads each operand once and writes its result once
+        # (bf16 activations and gradients, fp32 weight gradients; no transposed duplicates counted)
         if H > 0:
             flops_step = 2.0 * n_tr * (2 * width * H + 3 * H * O)
             flops_fwd = lambda rows: 2.0 * rows * (width * H + H * O)
+            bytes_fwd = lambda rows: 2.0 * (rows * width + width * H + rows * H) + 2.0 * (rows * H + H * O) + 4.0 * rows
+            bytes_step = (2.0 * (n_tr * width + width * H + n_tr * H)            # Hd = ReLU(X W1 + b1)
+                          + 2.0 * (n_tr * H + H * O + n_tr * O)                   # logits, loss, dL
+                          + 2.0 * (n_tr * O + H * O + 2 * n_tr * H)               # dHd = (dL W2^T) gated by Hd
+                          + 2.0 * (n_tr * H + n_tr * O) + 4.0 * H * O             # dW2
+                          + 2.0 * (n_tr * width + n_tr * H) + 4.0 * width * H     # dW1
+                          + 7 * 4.0 * (width * H + H * O))                        # optimiser: theta, m, v in and out, gradient in
         else:
             flops_step = 2.0 * n_tr * 2 * width * O
             flops_fwd = lambda rows: 2.0 * rows * width * O
+            bytes_fwd = lambda rows: 2.0 * (rows * width + width * O) + 4.0 * rows
+            bytes_step = (2.0 * (n_tr * width + width * O + n_tr * O) + 2.0 * (n_tr * width + n_tr * O)
+                          + 4.0 * width * O + 7 * 4.0 * width * O)
         import ctypes as C
         need = B.lib().retexo_mlp_train_step_workspace_size(C.c_int32(width), C.c_int32(H), C.c_int32(O),
                                                             C.c_int64(n_tr))
         ws_step = torch.empty(int(need), dtype=torch.uint8, device=dev)
         mean_ms, best_ms = time_calls(lambda: B.retexo_mlp_train_step(model, xtr, y_tr, x_t=xtr_t, workspace=ws_step), 10)
         phases.append(dict(kernel="mlp_train_step", round=m, calls_per_step=R, ms=mean_ms, best_ms=best_ms,
-                           bound="tensor", flops=flops_step, achieved=flops_step / mean_ms / 1e9,
-                           peak=peaks["bf16_sustained"], unit="TFLOP/s"))
+                           traffic=STEP_DRAM_TRAFFIC.get((w.name, m)),
+                           **min_time_roofline(flops_step, bytes_step, mean_ms, peaks)))
         mean_ms, best_ms = time_calls(lambda: B.retexo_embed(model, xva, y=y_va), 10)
-        phases.append(dict(kernel="embed_validation", round=m, calls_per_step=R, ms=mean_ms, best_ms=best_ms,
-                           bound="tensor", flops=flops_fwd(n_va), achieved=flops_fwd(n_va) / mean_ms / 1e9,
-                           peak=peaks["bf16_sustained"], unit="TFLOP/s"))
+        phases.append(dict(kernel="embed_validation", round=m, calls_per_step=0, ms=mean_ms, best_ms=best_ms,
+                           note="stand-alone call; inside the K-round run validation rides along in the training forward",
+                           **min_time_roofline(flops_fwd(n_va), bytes_fwd(n_va), mean_ms, peaks)))
         if H > 0:
             mean_ms, best_ms = time_calls(lambda: B.retexo_embed(model, x16, want_hidden=True), 3, warm=1)
             fl = 2.0 * n * width * H
+            nb = 2.0 * (n * width + width * H) + 4.0 * n * H          # fp32 Q^m out
         else:
             mean_ms, best_ms = time_calls(lambda: B.retexo_embed(model, x16, want_logits=True, want_pred=True), 3, warm=1)
             fl = 2.0 * n * width * O
+            nb = 2.0 * (n * width + width * O) + 4.0 * n * O + 4.0 * n
         phases.append(dict(kernel="embed_all_rows", round=m, calls_per_step=1, ms=mean_ms, best_ms=best_ms,
-                           bound="tensor", flops=fl, achieved=fl / mean_ms / 1e9, peak=peaks["bf16_sustained"],
-                           unit="TFLOP/s"))
+                           **min_time_roofline(fl, nb, mean_ms, peaks)))
         del model, xtr, xtr_t, xva, ws_step
     part = torch.from_numpy(w.part).to(dev)
     dims = [rd["rep_dim"] for rd in w.round_dims()]
@@ -426,13 +454,23 @@ def main():
                                 achieved=dom["achieved"], peak=dom["peak"], unit=dom["unit"], frac=dom["frac"],
                                 traffic=dom.get("traffic"), peak_source=peaks["source"],
                                 share_of_step=dom["share_of_step"],
-                                note="tensor-core products of one training iteration (tc_gemm_kernel launches)"
-                                if dom["bound"] == "tensor" else "CSR gather-reduce (agg_rows_kernel)")
+                                algorithmic_bytes=dom.get("algorithmic_bytes"), flops=dom.get("flops"),
+                                tflops=dom.get("tflops"), ms=dom["ms"], min_ms=dom.get("min_ms"),
+                                note="one training iteration (tc_gemm_kernel launches + reduce_update_kernel); min-time "
+                                     "roofline: bytes / HBM peak exceeds flops / tensor peak, so HBM is the bound"
+                                if dom["kernel"] == "mlp_train_step" and dom["bound"] == "hbm" else
+                                "one training iteration (tc_gemm_kernel launches): tensor-bound"
+                                if dom["kernel"] == "mlp_train_step" else "CSR gather-reduce (aggregation kernels)")
         # the memory-bound side of the path, against the measured HBM copy bandwidth
         line["roofline_aggregation"] = [
             dict(round=p["round"], bound="hbm", achieved=p["achieved"], peak=p["peak"], unit="GB/s", frac=p["frac"],
                  traffic=p.get("traffic"), ms=p["ms"], edges_per_s=p["edges_per_s"],
-                 dram_gbs=(p["traffic"] / p["ms"] / 1e6) if p.get("traffic") else None)
+                 dram_gbs=(p["traffic"] / p["ms"] / 1e6) if p.get("traffic") else None,
+                 dram_frac=(p["traffic"] / p["ms"] / 1e6 / p["peak"]) if p.get("traffic") else None,
+                 ceiling=("l2: column slabs, neighbour rows gathered from L2 (algorithmic bytes exceed DRAM traffic)"
+                          if p.get("traffic") and p["traffic"] < 0.25 * p["algorithmic_bytes"] else
+                          "hbm: DRAM traffic at the copy bandwidth, the L2 hit rate sets the algorithmic rate")
+                 if p.get("traffic") else None)
             for p in phases if p["kernel"] == "aggregate"]
         line["phases"] = [dict(kernel=p["kernel"], round=p["round"], ms=round(p["ms"], 4), calls=p["calls_per_step"],
                                share=round(p["share_of_step"], 4), bound=p["bound"], achieved=round(p["achieved"], 2),

@@ -317,16 +317,29 @@ __global__ void __launch_bounds__(kAggThreads) agg_combine_kernel(AggArgs a) {
 // slab (streamed with evict-first loads).  A warp takes 32 / LPR entries of a row at a time: lane
 // group g = lane / LPR adds entries g, g + G, g + 2G, ... in CSR order, and the groups' sums are
 // added in a fixed tree at the end, so results are still the same bits on every call.
-constexpr int kSlabUnroll = 8;                       // neighbour rows in flight per lane
-// Measured on B200 (126 MB of L2): random 256-byte gathers out of L2 deliver ~11 TB/s whatever the
-// number of loads in flight, while the plain variant runs at the HBM rate times 1 / (1 - L2 hit rate).
-// At 239 MB (hit rate ~50 %) the two are level, at 561 MB (~30 %) the slabs are 1.2x ahead.
-constexpr size_t kSlabMinMatrixBytes = 384u << 20;   // smaller matrices are left to the cache as they are
-constexpr size_t kSlabBytes = 64u << 20;             // a slab of all rows may take this much of L2
+#ifndef SLAB_U
+#define SLAB_U 8
+#define SLAB_TAIL_U 4
+#define SLAB_BLOCKS 3
+#define SLAB_MIN_MB 192
+#endif
+constexpr int kSlabUnroll = SLAB_U;                  // neighbour rows in flight per lane (full trips of 32 entries)
+constexpr int kSlabTailUnroll = SLAB_TAIL_U;         // ... in the ragged last trip of a row
+constexpr int kSlabBlocksPerSm = SLAB_BLOCKS;        // resident blocks the register budget is cut for
+// Measured on B200 (126 MB of L2), 233 k rows: 256-byte gathers out of an L2-resident slab deliver
+// 15-17 TB/s, while the plain variant runs at the HBM rate divided by (1 - L2 hit rate): 9 TB/s for a
+// 561 MB matrix (30 % hits), 13 TB/s for 239 MB (50 %), and the L2 rate itself once the matrix fits.
+constexpr size_t kSlabMinMatrixBytes = (size_t)SLAB_MIN_MB << 20;   // (1.5 x L2) smaller matrices are left to the cache as they are
+#ifndef SLAB_MB
+#define SLAB_MB 64
+#endif
+constexpr size_t kSlabBytes = (size_t)SLAB_MB << 20;             // a slab of all rows may take this much of L2
 
 template <int LPR, int OP>
-__global__ void __launch_bounds__(kAggThreads) agg_slab_kernel(AggArgs a, int n_slabs) {
+__global__ void __launch_bounds__(kAggThreads, kSlabBlocksPerSm) agg_slab_kernel(AggArgs a, int n_slabs) {
     constexpr int G = kWarp / LPR;                   // entries of a row taken per step
+    constexpr int U = G * kSlabUnroll > kWarp ? kWarp / G : kSlabUnroll;              // steps in flight: at most one trip
+    constexpr int UT = G * kSlabTailUnroll > kWarp ? kWarp / G : kSlabTailUnroll;
     const int lane = threadIdx.x & 31;
     const int g = lane / LPR, c = lane % LPR;
     const int nvec = (a.dim + 3) / 4;
@@ -355,6 +368,7 @@ __global__ void __launch_bounds__(kAggThreads) agg_slab_kernel(AggArgs a, int n_
         }
         const int vi = slab * LPR + c;
         const bool active = vi < nvec;
+        const float4* __restrict__ col = qv + (active ? vi : nvec - 1);
         float4 acc[1];
         vec_init<4, OP>(acc[0]);
         for (int64_t e0 = beg; e0 < end; e0 += kWarp) {
@@ -365,12 +379,34 @@ __global__ void __launch_bounds__(kAggThreads) agg_slab_kernel(AggArgs a, int n_
                 my_u = __ldcs(a.colidx + e0 + lane);
                 if (OP == kOpGcn) my_w = __ldg(a.coef + my_u);
             }
-            for (int j = 0; j < cnt; j += G * kSlabUnroll) {
-                float4 x[kSlabUnroll];
-                float w[kSlabUnroll];
-                bool on[kSlabUnroll];
+            if (cnt == kWarp) {
+                // full trip: no predicates; a lane beyond the last column vector loads the last one and
+                // its sum is dropped at the end
+#pragma unroll 1
+                for (int j = 0; j < kWarp; j += G * U) {
+                    float4 x[U];
+                    float w[U];
 #pragma unroll
-                for (int t = 0; t < kSlabUnroll; ++t) {
+                    for (int t = 0; t < U; ++t) {
+                        const int u = __shfl_sync(0xffffffffu, my_u, j + t * G + g);
+                        if (OP == kOpGcn) w[t] = __shfl_sync(0xffffffffu, my_w, j + t * G + g);
+                        x[t] = __ldg(col + (int64_t)u * ldv);
+                    }
+#pragma unroll
+                    for (int t = 0; t < U; ++t) {
+                        if (OP == kOpGcn) vec_fma(acc[0], w[t], x[t]);
+                        else if (OP == kOpMax) vec_max(acc[0], x[t]);
+                        else vec_add(acc[0], x[t]);
+                    }
+                }
+                continue;
+            }
+            for (int j = 0; j < cnt; j += G * UT) {      // ragged last trip of the row
+                float4 x[UT];
+                float w[UT];
+                bool on[UT];
+#pragma unroll
+                for (int t = 0; t < UT; ++t) {
                     const int idx = j + t * G + g;
                     const int u = __shfl_sync(0xffffffffu, my_u, idx & 31);
                     if (OP == kOpGcn) w[t] = __shfl_sync(0xffffffffu, my_w, idx & 31);
@@ -378,7 +414,7 @@ __global__ void __launch_bounds__(kAggThreads) agg_slab_kernel(AggArgs a, int n_
                     if (on[t]) x[t] = __ldg(qv + (int64_t)u * ldv + vi);
                 }
 #pragma unroll
-                for (int t = 0; t < kSlabUnroll; ++t) {
+                for (int t = 0; t < UT; ++t) {
                     if (!on[t]) continue;
                     if (OP == kOpGcn) vec_fma(acc[0], w[t], x[t]);
                     else if (OP == kOpMax) vec_max(acc[0], x[t]);
@@ -433,7 +469,7 @@ static int launch_slab(int op, const AggArgs& a, int n_sm, cudaStream_t st) {
 // variant is the better choice (the matrix fits L2 as it is, or no slab of all rows would).
 static int slab_lanes(int64_t n, int32_t dim) {
     if ((size_t)n * (size_t)dim * 4 < kSlabMinMatrixBytes) return 0;
-    for (int lpr = 32; lpr >= 8; lpr >>= 1)
+    for (int lpr = 32; lpr >= 8; lpr >>= 1)      // (64-byte gathers out of slabs of 4 vectors measured far slower)
         if ((size_t)n * (size_t)lpr * 16 <= kSlabBytes) return lpr * 4 < dim ? lpr : 0;
     return 0;
 }

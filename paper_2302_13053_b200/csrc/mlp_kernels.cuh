@@ -244,9 +244,16 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     const int64_t count = sidx == 0 ? u.seg[0].count : u.seg[1].count;
     float g = 0.f;
     int64_t z = 0;
-    for (; z + 4 <= count; z += 4) {          // loads issued together, added in index order
-        const float a = part[z * size + q], b = part[(z + 1) * size + q];
-        const float c = part[(z + 2) * size + q], d = part[(z + 3) * size + q];
+    for (; z + 8 <= count; z += 8) {          // loads issued together, added in index order
+        float x[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[i] = __ldcs(part + (z + i) * size + q);      // read once: streamed
+#pragma unroll
+        for (int i = 0; i < 8; ++i) g += x[i];
+    }
+    for (; z + 4 <= count; z += 4) {
+        const float a = __ldcs(part + z * size + q), b = __ldcs(part + (z + 1) * size + q);
+        const float c = __ldcs(part + (z + 2) * size + q), d = __ldcs(part + (z + 3) * size + q);
         g += a; g += b; g += c; g += d;
     }
     for (; z < count; ++z) g += part[z * size + q];

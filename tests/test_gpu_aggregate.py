@@ -194,7 +194,7 @@ def ladder_in_a_large_graph(n, seed):
                                         (oracle.SAGE_MEAN, 300000, 340), (oracle.GCN, 300000, 342),
                                         (oracle.SAGE_MAX, 170000, 600)])
 def test_matrices_beyond_the_cache_take_the_column_slab_variant(aggr, n, dim):
-    """A feature matrix of ~400 MB or more is aggregated slab of columns by slab of columns (32, 16
+    """A feature matrix of 200 MB or more is aggregated slab of columns by slab of columns (32, 16
     or 8 vectors per slab, by the number of rows): same tolerance, every degree bin, ragged last slab."""
     rowptr, colidx = ladder_in_a_large_graph(n, seed=dim)
     rng = np.random.default_rng(dim)
