@@ -34,7 +34,18 @@ struct CountArgs {
     uint32_t* big_bitmaps;                // kBigRowBlocks x words_per_bitmap, all zero between rows
     int64_t words_per_bitmap;
     unsigned long long* bad_part;         // set to 1 if a partition id is out of range
+    unsigned long long* next_row;         // work counter (zeroed before launch): rows are handed out in batches
+    int32_t row_batch;                    // rows per draw from the counter
 };
+
+// Rows are drawn from one counter, row_batch at a time, so that a power-law degree distribution
+// does not leave warps with a fixed share of hub rows behind the others.  Returns the first row
+// of this warp's next batch (>= n when the rows have run out).
+__device__ __forceinline__ int64_t next_rows(const CountArgs& a, int lane) {
+    unsigned long long u = 0;
+    if (lane == 0) u = atomicAdd(a.next_row, (unsigned long long)a.row_batch);
+    return (int64_t)__shfl_sync(0xffffffffu, u, 0);
+}
 
 // Partition id of node x; an id outside [0, n_parts) raises the flag and is
 // replaced by 0 so that every table access stays in bounds.
@@ -61,8 +72,8 @@ __global__ void __launch_bounds__(kCntThreads) count_bitmap_kernel(CountArgs a) 
     for (int i = lane; i < kBitmapWords; i += kWarp) bm[warp][i] = 0u;
     __syncwarp();
     unsigned long long my_cross = 0, my_pairs = 0;
-    const int64_t stride = (int64_t)gridDim.x * kCntWarps;
-    for (int64_t u = blockIdx.x * (int64_t)kCntWarps + warp; u < a.n; u += stride) {
+    for (int64_t u0 = next_rows(a, lane); u0 < a.n; u0 = next_rows(a, lane))
+    for (int64_t u = u0; u < min(a.n, u0 + a.row_batch); ++u) {
         const int64_t beg = a.rowptr[u], end = a.rowptr[u + 1];
         if (beg == end) continue;
         const int32_t pu = part_of(a, u);
@@ -133,8 +144,8 @@ __global__ void __launch_bounds__(kHashWarps * kWarp) count_general_kernel(Count
     for (int i = lane; i < kHashSlots; i += kWarp) tab[warp][i] = -1;
     __syncwarp();
     unsigned long long my_cross = 0, my_pairs = 0;
-    const int64_t stride = (int64_t)gridDim.x * kHashWarps;
-    for (int64_t u = blockIdx.x * (int64_t)kHashWarps + warp; u < a.n; u += stride) {
+    for (int64_t u0 = next_rows(a, lane); u0 < a.n; u0 = next_rows(a, lane))
+    for (int64_t u = u0; u < min(a.n, u0 + a.row_batch); ++u) {
         const int64_t beg = a.rowptr[u], end = a.rowptr[u + 1];
         if (beg == end) continue;
         const int32_t pu = part_of(a, u);
@@ -415,7 +426,8 @@ extern "C" int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* 
     int32_t* dims_dev = ws.take<int32_t>(64);
     CountArgs a;
     a.n = g->n_nodes; a.rowptr = g->rowptr; a.colidx = g->colidx; a.part = part; a.n_parts = n_parts;
-    a.cross_edges = acc; a.pairs = acc + 1; a.bad_part = acc + 2;
+    a.cross_edges = acc; a.pairs = acc + 1; a.bad_part = acc + 2; a.next_row = acc + 4;
+    a.row_batch = 1;
     a.send = reinterpret_cast<unsigned long long*>(send_per_part);
     a.recv = reinterpret_cast<unsigned long long*>(recv_per_part);
     a.big_list = nullptr; a.big_count = nullptr; a.big_bitmaps = nullptr; a.words_per_bitmap = 0;
@@ -429,6 +441,9 @@ extern "C" int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* 
         if (n_parts <= kBitmapParts) {
             const int64_t want = (a.n + kCntWarps - 1) / kCntWarps;
             const unsigned blocks = (unsigned)(want < (int64_t)n_sm * 8 ? want : (int64_t)n_sm * 8);
+            // ~16 draws per warp: fine enough to balance hub rows, coarse enough for the counter
+            const int64_t batch = a.n / ((int64_t)blocks * kCntWarps * 16);
+            a.row_batch = (int32_t)(batch < 1 ? 1 : batch > 64 ? 64 : batch);
             count_bitmap_kernel<<<blocks, kCntThreads, 0, st>>>(a);
         } else {
             a.big_list = ws.take<int32_t>((size_t)a.n);
@@ -440,6 +455,8 @@ extern "C" int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* 
                                             sizeof(uint32_t) * (size_t)kBigRowBlocks * (size_t)a.words_per_bitmap, st));
             const int64_t want = (a.n + kHashWarps - 1) / kHashWarps;
             const unsigned blocks = (unsigned)(want < (int64_t)n_sm * 32 ? want : (int64_t)n_sm * 32);
+            const int64_t batch = a.n / ((int64_t)blocks * kHashWarps * 16);
+            a.row_batch = (int32_t)(batch < 1 ? 1 : batch > 64 ? 64 : batch);
             count_general_kernel<<<blocks, kHashWarps * kWarp, 0, st>>>(a);
             count_big_rows_kernel<<<kBigRowBlocks, kCntThreads, 0, st>>>(a);
         }
