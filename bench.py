@@ -157,7 +157,8 @@ def launches_per_step(w, R: int) -> int:
             total += 3                               # prep, warp rows, block rows
         total += 2                                   # train / val batches
         step = 6 if h > 0 else 3                     # products, reduce + update (+ weight copies once)
-        total += R * (step + 1) + (2 if h > 0 else 1)     # + bookkeeping of the validation count that rides along
+        total += R * step + 1 + (2 if h > 0 else 1)       # (the update kernel's last block books the validation count
+                                                          #  that rides along; the last iterate's is booked by a kernel of its own)
         total += (2 if h > 0 else 1) + 1             # stand-alone validation of the last iterate + snapshot
         total += 2 * (4 if h > 0 else 3)             # test accuracy, kept and last iterate
         total += 3 if h > 0 else 2                   # emission of Q^m / final logits

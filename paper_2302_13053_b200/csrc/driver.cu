@@ -333,20 +333,24 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         MlpBuffers sb{};
         mlp_step_buffers(plan, b.ws_step, b.ws_step_bytes, &sb);
         bf16* val_hd = reinterpret_cast<bf16*>(b.ws_embed);      // [n_val x ld_h] scratch of a stand-alone validation forward
-        const EvalTail tail{b.y_val, b.cur_correct, b.best_correct, b.have_best, b.theta_best};
+        // cur_correct[0]: hits of the validation rows riding along; cur_correct[1]: the update kernel's
+        // count of finished blocks.  Both are cleared here once and left clear by the update kernel.
+        RETEXO_CUDA_TRY(cudaMemsetAsync(b.cur_correct, 0, 2 * sizeof(unsigned long long), st));
+        EvalTail tail{b.y_val, b.cur_correct, b.best_correct, b.have_best, b.theta_best};
+        tail.done = b.cur_correct + 1;
+        tail.best_iter = b.best_iter_cur;
         int pending_it = 0;       // iteration whose weights still await their validation count
         for (int it = 1; it <= c.R; ++it) {
             float* loss_slot = b.loss_history + (size_t)(m - 1) * c.R + (it - 1);
             // The weights of iteration it-1 are validated inside this iteration's forward pass (the
             // validation rows ride along; the update kernel keeps them if they are the best so far).
             // The update of iteration it-1 also left bf16 copies of the current weights behind.
+            // (its count is recorded as iteration pending_it's by the update kernel's last block)
+            tail.iter = pending_it;
+            tail.history_slot = b.val_history + (size_t)(m - 1) * c.R + (pending_it > 0 ? pending_it - 1 : 0);
             RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, loss_slot,
                                              nullptr, it > 1, pending_it ? &tail : nullptr, st));
             model.step += 1;
-            if (pending_it)
-                record_validation_kernel<<<1, 32, 0, st>>>(b.cur_correct, b.best_correct, b.have_best, pending_it,
-                                                           b.best_iter_cur,
-                                                           b.val_history + (size_t)(m - 1) * c.R + (pending_it - 1));
             const bool want = n_val && (it % c.eval_every == 0 || it == c.R);
             pending_it = (want && it < c.R) ? it : 0;
             if (want && it == c.R) {      // the last iterate has no next iteration to ride on

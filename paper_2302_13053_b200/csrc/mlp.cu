@@ -207,8 +207,11 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     const float* theta = model->theta;
     const float* b1 = theta + (int64_t)d_in * out1;
     const float* b2 = b1 + out1 + (int64_t)H * O;
-    RETEXO_CUDA_TRY(cudaMemsetAsync(b.status, 0, sizeof(int32_t), st));
-    if (!shadows_ready) RETEXO_TRY(build_weight_shadows(p, b, theta, st));
+    // (a caller that chains iterations clears the status word once: a give-up then marks every later loss)
+    if (!shadows_ready) {
+        RETEXO_CUDA_TRY(cudaMemsetAsync(b.status, 0, sizeof(int32_t), st));
+        RETEXO_TRY(build_weight_shadows(p, b, theta, st));
+    }
     if (!x_t) {      // no transposed batch from the caller: build [X^T ; 1] here (one more pass over X per call)
         RETEXO_TRY(retexo_pack_rows(x, 1, ldx, d_in, nullptr, n, nullptr, 0, b.xt16, p.ld_n, 1, st));
         x_t = b.xt16;
@@ -217,7 +220,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
 
     // ---- forward; the class-dimension product ends in the loss: softmax, cross-entropy and dL
     //      are computed in its epilogue, where one thread holds a whole row of logits
-    if (tail) RETEXO_CUDA_TRY(cudaMemsetAsync(tail->correct, 0, sizeof(unsigned long long), st));
+    if (tail && !tail->done) RETEXO_CUDA_TRY(cudaMemsetAsync(tail->correct, 0, sizeof(unsigned long long), st));
     TcGemm fwd = tc_base(x, ldx, b.w1t16, p.ld_k, n_all, out1, d_in, b.status);
     fwd.bias = b1;
     TcGemm head = fwd;
@@ -267,7 +270,10 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     u.w1t16 = b.w1t16; u.ld_k = p.ld_k; u.w2t16 = H > 0 ? b.w2t16 : nullptr; u.ld_h = p.ld_h;
     u.w2p16 = H > 0 ? b.w2p16 : nullptr; u.ld_dl = p.ld_dl;
     u.d_in = d_in; u.out1 = out1; u.hidden = H; u.n_classes = O;
-    if (tail) { u.snap_cur = tail->correct; u.snap_best = tail->best; u.snap_have = tail->have_best; u.theta_best = tail->theta_best; }
+    if (tail) {
+        u.snap_cur = tail->correct; u.snap_best = tail->best; u.snap_have = tail->have_best; u.theta_best = tail->theta_best;
+        u.done = tail->done; u.rec_iter = tail->iter; u.rec_best_iter = tail->best_iter; u.rec_history_slot = tail->history_slot;
+    }
     reduce_update_kernel<<<(unsigned)((p.nt + 255) / 256), 256, 0, st>>>(u);
     return launch_status();
 }

@@ -219,27 +219,14 @@ struct UpdateArgs {
     bf16* w2p16; int64_t ld_dl;      // W2   [hidden x ld_dl]
     int32_t d_in, out1, hidden, n_classes;
     // keep-the-best snapshot of theta as it is before this update (optional, see EvalTail)
-    const unsigned long long* snap_cur; const unsigned long long* snap_best; const int32_t* snap_have;
+    unsigned long long* snap_cur; unsigned long long* snap_best; int32_t* snap_have;
     float* theta_best;
+    // bookkeeping of the validation count by the last block to finish (optional, see EvalTail)
+    unsigned long long* done; int32_t rec_iter; int32_t* rec_best_iter; unsigned long long* rec_history_slot;
 };
 
-// Sums each parameter's split-K partials in index order, applies the optimiser, and refreshes
-// the bf16 weight copies.  Block 0 also reduces the loss (fixed order: per-lane strided sums,
-// then a shuffle tree).
-__global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
-    const int64_t p = blockIdx.x * 256ll + threadIdx.x;
-    if (blockIdx.x == 0 && threadIdx.x < 32 && u.loss_out) {
-        float s = 0.f;
-        for (int64_t i = threadIdx.x; i < u.n_loss; i += 32) s += u.loss_partial[i];
-        s = warp_sum(s);
-        if (threadIdx.x == 0) *u.loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
-    }
-    const int64_t size0 = u.seg[0].size;
-    const int sidx = p < size0 ? 0 : 1;
-    if (sidx >= u.n_seg) return;
-    const int64_t q = sidx == 0 ? p : p - size0;
-    const int64_t size = sidx == 0 ? size0 : u.seg[1].size;
-    if (q >= size) return;
+// One parameter: sum of its split-K partials in index order, optimiser step, bf16 copies.
+__device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p, int sidx, int64_t q, int64_t size) {
     const float* part = sidx == 0 ? u.seg[0].partial : u.seg[1].partial;
     const int64_t count = sidx == 0 ? u.seg[0].count : u.seg[1].count;
     float g = 0.f;
@@ -279,6 +266,45 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
         const int64_t jh = q / u.n_classes, c = q % u.n_classes;
         if (u.w2t16) u.w2t16[c * u.ld_h + jh] = f32_to_bf16(t);
         if (u.w2p16) u.w2p16[jh * u.ld_dl + c] = f32_to_bf16(t);
+    }
+}
+
+// Sums each parameter's split-K partials in index order, applies the optimiser, and refreshes
+// the bf16 weight copies.  Block 0 also reduces the loss (fixed order: per-lane strided sums,
+// then a shuffle tree).  With u.done set, the last block to finish does the validation bookkeeping.
+__global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
+    const int64_t p = blockIdx.x * 256ll + threadIdx.x;
+    if (blockIdx.x == 0 && threadIdx.x < 32 && u.loss_out) {
+        float s = 0.f;
+        for (int64_t i = threadIdx.x; i < u.n_loss; i += 32) s += u.loss_partial[i];
+        s = warp_sum(s);
+        if (threadIdx.x == 0) *u.loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
+    }
+    const int64_t size0 = u.seg[0].size;
+    const int sidx = p < size0 ? 0 : 1;
+    const int64_t q = sidx == 0 ? p : p - size0;
+    const int64_t size = sidx == 0 ? size0 : u.seg[1].size;
+    if (sidx < u.n_seg && q < size) update_parameter(u, p, sidx, q, size);
+    if (!u.done) return;
+    // every block has compared against the kept count by the time the last one records the new one
+    __shared__ bool is_last;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        is_last = atomicAdd(u.done, 1ull) == (unsigned long long)gridDim.x - 1ull;
+    }
+    __syncthreads();
+    if (is_last && threadIdx.x == 0) {
+        __threadfence();
+        const unsigned long long cur = *u.snap_cur;
+        if (u.rec_history_slot) *u.rec_history_slot = cur;
+        if (!*u.snap_have || cur > *u.snap_best) {
+            *u.snap_best = cur;
+            if (u.rec_best_iter) *u.rec_best_iter = u.rec_iter;
+            *u.snap_have = 1;
+        }
+        *u.snap_cur = 0ull;
+        *u.done = 0ull;
     }
 }
 

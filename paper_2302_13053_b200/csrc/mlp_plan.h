@@ -48,12 +48,21 @@ size_t mlp_step_workspace_size(const MlpPlan& p);
 // training rows; the forward pass covers them too, the loss epilogue counts their hits into
 // *correct (weights as they are before this iteration's update), and the update kernel first
 // copies theta to theta_best if that count beats *best (or nothing was kept yet).
+// With `done` set, the update kernel's last block also does the bookkeeping of that validation
+// count: history_slot receives it, best / have_best / best_iter are brought up to date for
+// iteration `iter`, and *correct is cleared for the next iteration (so the caller clears it once
+// per round, not once per iteration).  *done must be zero before the first launch; the kernel
+// leaves it zero.
 struct EvalTail {
     const int32_t* y_eval;
     unsigned long long* correct;
-    const unsigned long long* best;
-    const int32_t* have_best;
+    unsigned long long* best;
+    int32_t* have_best;
     float* theta_best;
+    unsigned long long* done = nullptr;
+    int32_t iter = 0;
+    int32_t* best_iter = nullptr;
+    unsigned long long* history_slot = nullptr;
 };
 
 // Lays the step's scratch buffers out over a workspace of retexo_mlp_train_step_workspace_size bytes.
