@@ -160,7 +160,7 @@ def launches_per_step(w, R: int) -> int:
         total += R * step + 1 + (2 if h > 0 else 1)       # (the update kernel's last block books the validation count
                                                           #  that rides along; the last iterate's is booked by a kernel of its own)
         total += (2 if h > 0 else 1) + 1             # stand-alone validation of the last iterate + snapshot
-        total += 2 * (4 if h > 0 else 3)             # test accuracy, kept and last iterate
+        total += 1 + 2 * (4 if h > 0 else 2)         # test rows gathered, then kept and last iterate (weight copies + products)
         total += 3 if h > 0 else 2                   # emission of Q^m / final logits
     return total
 

@@ -130,7 +130,8 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
         l.gat_vec = t.template take<float>((size_t)2 * hd);
         l.gat_stage = t.template take<float>((size_t)max_rep * hd + 2 * hd);
     }
-    l.xtr16 = t.template take<bf16>((size_t)(n_tr + n_val) * ld16);     // training rows, then validation rows
+    // training rows, then validation rows; after the round's last iteration the test rows take their place
+    l.xtr16 = t.template take<bf16>((size_t)(n_tr + n_val > n_te ? n_tr + n_val : n_te) * ld16);
     l.xval16 = nullptr;
     l.xtr_t16 = t.template take<bf16>((size_t)(max_din + 1) * (size_t)round_up(n_tr, 64));
     l.y_tr = t.template take<int32_t>((size_t)n_tr);
@@ -375,10 +376,14 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
 
         // ---- test accuracy of the kept and of the last iterate
         if (n_te) {
-            RETEXO_TRY(retexo_embed(&best, b.x16, ld16, test_idx, n_te, nullptr, 0, nullptr, 0, nullptr, 0, nullptr,
+            // the test rows are gathered once into a dense batch (the training batch is no longer needed),
+            // so both forward passes run on the tensor cores
+            bf16* xte16 = b.xtr16;
+            RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, test_idx, n_te, xte16, ld16, nullptr, 0, 0, st));
+            RETEXO_TRY(retexo_embed(&best, xte16, ld16, nullptr, n_te, nullptr, 0, nullptr, 0, nullptr, 0, nullptr,
                                     b.y_test, reinterpret_cast<uint64_t*>(b.test_best + (m - 1)), b.ws_embed,
                                     b.ws_embed_bytes, st));
-            RETEXO_TRY(retexo_embed(&model, b.x16, ld16, test_idx, n_te, nullptr, 0, nullptr, 0, nullptr, 0, nullptr,
+            RETEXO_TRY(retexo_embed(&model, xte16, ld16, nullptr, n_te, nullptr, 0, nullptr, 0, nullptr, 0, nullptr,
                                     b.y_test, reinterpret_cast<uint64_t*>(b.test_last + (m - 1)), b.ws_embed,
                                     b.ws_embed_bytes, st));
         } else {
