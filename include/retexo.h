@@ -349,7 +349,13 @@ size_t retexo_lmp_workspace_size(const retexo_lmp_config* cfg, int64_t n_nodes, 
  * draws, P = Q^{m-1} W_att is computed once, then aggregated.
  * With memory_is_host = 0 the call only enqueues work (outputs are device
  * memory); with 1 it copies inputs in, runs, copies outputs to the host
- * arrays and synchronises the stream before returning. */
+ * arrays and synchronises the stream before returning.
+ * Streams: the work is ordered after everything already enqueued on `stream`, and whatever is
+ * enqueued on `stream` after the call is ordered after the work.  In between it runs on a stream the
+ * call creates and releases itself, because the R iterations of a round (the same launches with the
+ * same arguments once the iteration number is kept on the device) are recorded once as a CUDA graph
+ * and replayed, which the legacy default stream does not allow.  If no stream or graph can be had
+ * the launches go to `stream` one by one.  Do not call it while `stream` is being captured. */
 int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_inputs* in,
                      const retexo_lmp_outputs* out,
                      void* workspace, size_t workspace_bytes, void* stream);

@@ -53,6 +53,53 @@ __global__ void pack_counts_kernel(const uint64_t* cross, const uint64_t* pairs,
     for (int m = 0; m < K; ++m) out[4 + m] = per_round[m];
 }
 
+// A stream of the library's own for the duration of one call, ordered after everything the caller
+// has enqueued and joined back into the caller's stream at the end: the iteration loop is recorded
+// as a CUDA graph, which the legacy default stream does not allow.  Falls back to the caller's stream.
+struct WorkStream {
+    cudaStream_t caller, s;
+    cudaEvent_t ev = nullptr;
+    bool own = false;
+    explicit WorkStream(cudaStream_t c) : caller(c), s(c) {
+        cudaStream_t ns = nullptr;
+        if (cudaStreamCreateWithFlags(&ns, cudaStreamNonBlocking) == cudaSuccess) {
+            if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess &&
+                cudaEventRecord(ev, caller) == cudaSuccess && cudaStreamWaitEvent(ns, ev, 0) == cudaSuccess) {
+                s = ns;
+                own = true;
+            } else {
+                if (ev) { (void)cudaEventDestroy(ev); ev = nullptr; }
+                (void)cudaStreamDestroy(ns);
+            }
+        }
+        (void)cudaGetLastError();
+    }
+    // Orders the caller's stream after the work enqueued here so far.
+    int join() {
+        if (!own) return RETEXO_OK;
+        if (cudaEventRecord(ev, s) != cudaSuccess || cudaStreamWaitEvent(caller, ev, 0) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return RETEXO_ERR_CUDA;
+        }
+        return RETEXO_OK;
+    }
+    ~WorkStream() {
+        if (!own) return;
+        (void)join();
+        (void)cudaEventDestroy(ev);
+        (void)cudaStreamDestroy(s);      // (work already enqueued still runs to completion)
+    }
+    WorkStream(const WorkStream&) = delete;
+    WorkStream& operator=(const WorkStream&) = delete;
+};
+
+// Owns the executable graph of one round's training iteration.
+struct IterationGraph {
+    cudaGraphExec_t exec = nullptr;
+    void reset() { if (exec) { (void)cudaGraphExecDestroy(exec); exec = nullptr; } }
+    ~IterationGraph() { reset(); }
+};
+
 struct RoundDims { int32_t rep_dim, agg_dim, d_in, hidden; };
 
 static RoundDims round_dims(const retexo_lmp_config& c, int m /*1-based*/) {
@@ -215,7 +262,9 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
     const int32_t n_parts = in->part ? in->n_parts : 0;
     const size_t need = retexo_lmp_workspace_size(cfg, n, e, in->n_train, in->n_val, in->n_test, n_parts);
     if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    WorkStream work(static_cast<cudaStream_t>(stream));
+    cudaStream_t st = work.s;
+    IterationGraph iteration;
     const bool host = c.memory_is_host != 0;
     const cudaMemcpyKind in_kind = host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
     const cudaMemcpyKind out_kind = host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice;
@@ -336,10 +385,17 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         bf16* val_hd = reinterpret_cast<bf16*>(b.ws_embed);      // [n_val x ld_h] scratch of a stand-alone validation forward
         // cur_correct[0]: hits of the validation rows riding along; cur_correct[1]: the update kernel's
         // count of finished blocks.  Both are cleared here once and left clear by the update kernel.
-        RETEXO_CUDA_TRY(cudaMemsetAsync(b.cur_correct, 0, 2 * sizeof(unsigned long long), st));
+        // cur_correct[2]: updates applied so far in this round (the iteration number lives on the device).
+        RETEXO_CUDA_TRY(cudaMemsetAsync(b.cur_correct, 0, 3 * sizeof(unsigned long long), st));
         EvalTail tail{b.y_val, b.cur_correct, b.best_correct, b.have_best, b.theta_best};
         tail.done = b.cur_correct + 1;
         tail.best_iter = b.best_iter_cur;
+        const DeviceIter dev{b.cur_correct + 2, b.cur_correct + 1, b.loss_history + (size_t)(m - 1) * c.R,
+                             b.val_history + (size_t)(m - 1) * c.R};
+        // With validation every iteration (or none) all iterations from the second on are the same six
+        // launches with the same arguments: the second one is recorded as a graph, the rest replay it.
+        const bool uniform = work.own && c.R > 3 && (n_val == 0 || c.eval_every == 1);
+        iteration.reset();
         int pending_it = 0;       // iteration whose weights still await their validation count
         for (int it = 1; it <= c.R; ++it) {
             float* loss_slot = b.loss_history + (size_t)(m - 1) * c.R + (it - 1);
@@ -349,8 +405,33 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
             // (its count is recorded as iteration pending_it's by the update kernel's last block)
             tail.iter = pending_it;
             tail.history_slot = b.val_history + (size_t)(m - 1) * c.R + (pending_it > 0 ? pending_it - 1 : 0);
-            RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, loss_slot,
-                                             nullptr, it > 1, pending_it ? &tail : nullptr, st));
+            const EvalTail* riding = pending_it ? &tail : nullptr;
+            if (iteration.exec) {
+                RETEXO_CUDA_TRY(cudaGraphLaunch(iteration.exec, st));
+            } else if (uniform && it == 2) {
+                bool recorded = false;
+                if (cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed) == cudaSuccess) {
+                    const int rc = mlp_train_step_launch(plan, sb, &model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, loss_slot,
+                                                         nullptr, true, riding, st, &dev);
+                    cudaGraph_t graph = nullptr;
+                    const cudaError_t ended = cudaStreamEndCapture(st, &graph);
+                    if (rc == RETEXO_OK && ended == cudaSuccess && graph &&
+                        cudaGraphInstantiate(&iteration.exec, graph, 0) == cudaSuccess)
+                        recorded = true;
+                    if (graph) (void)cudaGraphDestroy(graph);
+                }
+                (void)cudaGetLastError();
+                if (recorded) {
+                    RETEXO_CUDA_TRY(cudaGraphLaunch(iteration.exec, st));
+                } else {      // no graph on this stream: plain launches
+                    iteration.reset();
+                    RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, loss_slot,
+                                                     nullptr, true, riding, st, &dev));
+                }
+            } else {
+                RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, loss_slot,
+                                                 nullptr, it > 1, riding, st, &dev));
+            }
             model.step += 1;
             const bool want = n_val && (it % c.eval_every == 0 || it == c.R);
             pending_it = (want && it < c.R) ? it : 0;

@@ -200,7 +200,7 @@ namespace retexo {
 int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
                           const bf16* x, int64_t ldx, const bf16* x_t, int64_t ld_xt, const int32_t* y,
                           float* loss_out, float* grad_out, bool shadows_ready, const EvalTail* tail,
-                          cudaStream_t st) {
+                          cudaStream_t st, const DeviceIter* dev) {
     const int64_t n = p.n_rows;
     const int64_t n_all = n + (tail ? p.n_eval : 0);          // evaluation rows ride along in the forward pass
     const int32_t d_in = p.d_in, H = p.hidden, O = p.n_classes, out1 = p.out1;
@@ -273,6 +273,10 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     if (tail) {
         u.snap_cur = tail->correct; u.snap_best = tail->best; u.snap_have = tail->have_best; u.theta_best = tail->theta_best;
         u.done = tail->done; u.rec_iter = tail->iter; u.rec_best_iter = tail->best_iter; u.rec_history_slot = tail->history_slot;
+    }
+    if (dev) {
+        u.step_dev = dev->step; u.done = dev->done; u.loss_base = dev->loss_base; u.history_base = dev->history_base;
+        u.loss_out = nullptr;
     }
     reduce_update_kernel<<<(unsigned)((p.nt + 255) / 256), 256, 0, st>>>(u);
     return launch_status();

@@ -223,10 +223,15 @@ struct UpdateArgs {
     float* theta_best;
     // bookkeeping of the validation count by the last block to finish (optional, see EvalTail)
     unsigned long long* done; int32_t rec_iter; int32_t* rec_best_iter; unsigned long long* rec_history_slot;
+    // iteration state on the device (optional, see DeviceIter; needs `done`): with s = *step_dev updates applied
+    // so far, this launch applies update s + 1, writes its loss to loss_base[s], books the validation count
+    // as iteration s's into history_base[s - 1], and its last block leaves *step_dev = s + 1
+    unsigned long long* step_dev; float* loss_base; unsigned long long* history_base;
 };
 
 // One parameter: sum of its split-K partials in index order, optimiser step, bf16 copies.
-__device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p, int sidx, int64_t q, int64_t size) {
+__device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p, int sidx, int64_t q, int64_t size,
+                                                 float corr1, float corr2) {
     const float* part = sidx == 0 ? u.seg[0].partial : u.seg[1].partial;
     const int64_t count = sidx == 0 ? u.seg[0].count : u.seg[1].count;
     float g = 0.f;
@@ -254,7 +259,7 @@ __device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p,
         const float v = u.beta2 * u.v[p] + (1.f - u.beta2) * g * g;
         u.m[p] = m;
         u.v[p] = v;
-        t = u.theta[p] - u.lr * (m / u.corr1) / (sqrtf(v / u.corr2) + u.eps);
+        t = u.theta[p] - u.lr * (m / corr1) / (sqrtf(v / corr2) + u.eps);
     }
     u.theta[p] = t;
     if (sidx == 0) {
@@ -274,17 +279,31 @@ __device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p,
 // then a shuffle tree).  With u.done set, the last block to finish does the validation bookkeeping.
 __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     const int64_t p = blockIdx.x * 256ll + threadIdx.x;
-    if (blockIdx.x == 0 && threadIdx.x < 32 && u.loss_out) {
+    float corr1 = u.corr1, corr2 = u.corr2;
+    float* loss_out = u.loss_out;
+    unsigned long long step_now = 0;
+    if (u.step_dev) {      // the iteration number lives on the device: bias corrections and slots follow from it
+        __shared__ float corr_s[2];
+        step_now = *u.step_dev;
+        if (threadIdx.x == 0) {
+            corr_s[0] = (float)(1.0 - pow((double)u.beta1, (double)(step_now + 1)));
+            corr_s[1] = (float)(1.0 - pow((double)u.beta2, (double)(step_now + 1)));
+        }
+        __syncthreads();
+        corr1 = corr_s[0]; corr2 = corr_s[1];
+        loss_out = u.loss_base ? u.loss_base + step_now : nullptr;
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 32 && loss_out) {
         float s = 0.f;
         for (int64_t i = threadIdx.x; i < u.n_loss; i += 32) s += u.loss_partial[i];
         s = warp_sum(s);
-        if (threadIdx.x == 0) *u.loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
+        if (threadIdx.x == 0) *loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
     }
     const int64_t size0 = u.seg[0].size;
     const int sidx = p < size0 ? 0 : 1;
     const int64_t q = sidx == 0 ? p : p - size0;
     const int64_t size = sidx == 0 ? size0 : u.seg[1].size;
-    if (sidx < u.n_seg && q < size) update_parameter(u, p, sidx, q, size);
+    if (sidx < u.n_seg && q < size) update_parameter(u, p, sidx, q, size, corr1, corr2);
     if (!u.done) return;
     // every block has compared against the kept count by the time the last one records the new one
     __shared__ bool is_last;
@@ -296,14 +315,19 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     __syncthreads();
     if (is_last && threadIdx.x == 0) {
         __threadfence();
-        const unsigned long long cur = *u.snap_cur;
-        if (u.rec_history_slot) *u.rec_history_slot = cur;
-        if (!*u.snap_have || cur > *u.snap_best) {
-            *u.snap_best = cur;
-            if (u.rec_best_iter) *u.rec_best_iter = u.rec_iter;
-            *u.snap_have = 1;
+        if (u.snap_cur) {
+            const unsigned long long cur = *u.snap_cur;
+            unsigned long long* slot = u.step_dev ? (u.history_base && step_now > 0 ? u.history_base + (step_now - 1) : nullptr)
+                                                  : u.rec_history_slot;
+            if (slot) *slot = cur;
+            if (!*u.snap_have || cur > *u.snap_best) {
+                *u.snap_best = cur;
+                if (u.rec_best_iter) *u.rec_best_iter = u.step_dev ? (int32_t)step_now : u.rec_iter;
+                *u.snap_have = 1;
+            }
+            *u.snap_cur = 0ull;
         }
-        *u.snap_cur = 0ull;
+        if (u.step_dev) *u.step_dev = step_now + 1;
         *u.done = 0ull;
     }
 }

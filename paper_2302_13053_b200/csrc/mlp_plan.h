@@ -65,6 +65,19 @@ struct EvalTail {
     unsigned long long* history_slot = nullptr;
 };
 
+// Iteration state kept on the device, so that every iteration of a round is the same launch sequence
+// with the same arguments (which lets the K-round driver record it once as a CUDA graph and replay it).
+// With s = *step updates applied so far, a step launched with this state applies update s + 1 (Adam's bias
+// corrections follow from s), writes its loss to loss_base[s], books the validation count that rode along
+// as iteration s's (history_base[s - 1], best_iter) and leaves *step = s + 1.  *step and *done are cleared
+// by the caller once per round.
+struct DeviceIter {
+    unsigned long long* step;
+    unsigned long long* done;
+    float* loss_base;
+    unsigned long long* history_base;
+};
+
 // Lays the step's scratch buffers out over a workspace of retexo_mlp_train_step_workspace_size bytes.
 void mlp_step_buffers(const MlpPlan& p, void* workspace, size_t bytes, MlpBuffers* out);
 
@@ -74,7 +87,7 @@ void mlp_step_buffers(const MlpPlan& p, void* workspace, size_t bytes, MlpBuffer
 int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
                           const __nv_bfloat16* x, int64_t ldx, const __nv_bfloat16* x_t, int64_t ld_xt,
                           const int32_t* y, float* loss_out, float* grad_out, bool shadows_ready,
-                          const EvalTail* tail, cudaStream_t st);
+                          const EvalTail* tail, cudaStream_t st, const DeviceIter* dev = nullptr);
 
 // Forward + arg-max + hit count over a dense batch with the weight copies in `b` (which must
 // hold model->theta): what validation needs after every iteration.  hd_ws: bf16 [n_rows x p.ld_h].
