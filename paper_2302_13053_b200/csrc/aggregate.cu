@@ -615,7 +615,28 @@ __global__ void __launch_bounds__(kAggThreads) gat_rows_kernel(GatArgs a) {
             for (int h = 0; h < kGatMaxHeads; ++h) if (h == head_of[c]) sc = scale[h];
             acc[c] *= sc;
         }
-        for (int j = 0; j < cnt; ++j) {
+        // several neighbour rows in flight per lane (a hub's row is otherwise one dependent load after
+        // another); the products are still added in entry order
+        constexpr int U = NC <= 2 ? 8 : (NC <= 4 ? 4 : 2);
+        int j = 0;
+        for (; j + U <= cnt; j += U) {
+            float x[U][NC];
+#pragma unroll
+            for (int t = 0; t < U; ++t) {
+                const int u = __shfl_sync(0xffffffffu, my_u, j + t);
+                const float* row = a.p + (int64_t)u * a.ldp;
+#pragma unroll
+                for (int c = 0; c < NC; ++c) {
+                    const int col = c * kWarp + lane;
+                    x[t][c] = col < a.dim ? __ldg(row + col) : 0.f;
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < U; ++t)
+#pragma unroll
+                for (int c = 0; c < NC; ++c) acc[c] = fmaf(p_s[warp][j + t][head_of[c]], x[t][c], acc[c]);
+        }
+        for (; j < cnt; ++j) {
             const int u = __shfl_sync(0xffffffffu, my_u, j);
             const float* row = a.p + (int64_t)u * a.ldp;
 #pragma unroll
