@@ -126,6 +126,24 @@ def aggregate(aggr: int, rowptr: np.ndarray, colidx: np.ndarray, q: np.ndarray,
     raise ValueError("unknown aggregator")
 
 
+# ---------------------------------------------------------------- dropout generator
+def philox4x32_10(counter: Sequence[int], key: Sequence[int]) -> List[int]:
+    """One block of the Philox4x32-10 counter-based generator."""
+    c = (C.c_uint32 * 4)(*[int(v) & 0xffffffff for v in counter])
+    k = (C.c_uint32 * 2)(*[int(v) & 0xffffffff for v in key])
+    o = (C.c_uint32 * 4)()
+    lib().oracle_philox4x32_10(c, k, o)
+    return [int(v) for v in o]
+
+
+def dropout_mask(row: int, step: int, hidden: int, p: float, seed: int) -> np.ndarray:
+    """Keep factors (1/(1-p) or 0) of the hidden units of one batch row in update `step`."""
+    out = np.zeros(hidden, dtype=np.float64)
+    _check(lib().oracle_dropout_mask(C.c_int64(row), C.c_int64(step), C.c_int32(hidden), C.c_double(p),
+                                     C.c_uint64(seed), _p(out)), "oracle_dropout_mask")
+    return out
+
+
 # ---------------------------------------------------------------- per-node model
 class Mlp:
     """State of one round's per-node model in double precision."""
@@ -167,9 +185,11 @@ class Mlp:
         return d
 
     def train_step(self, x: np.ndarray, y: np.ndarray, row_idx: Optional[np.ndarray] = None,
-                   return_grad: bool = False):
+                   return_grad: bool = False, dropout: float = 0.0, dropout_seed: int = 0):
         """One full-batch step on rows x[row_idx] (all rows of x if None) with
-        labels y (one per batch row).  Returns the loss before the update."""
+        labels y (one per batch row).  Returns the loss before the update.
+        dropout > 0: hidden units are dropped with that probability (Philox
+        mask of (batch row, unit, update number), kept units scaled by 1/(1-p))."""
         x = _f32(x)
         y = np.ascontiguousarray(y, dtype=np.int32)
         ri = None if row_idx is None else np.ascontiguousarray(row_idx, dtype=np.int32)
@@ -178,12 +198,15 @@ class Mlp:
         loss = C.c_double(0.0)
         grad = np.zeros_like(self.theta) if return_grad else None
         self.step += 1
-        rc = lib().oracle_mlp_train_step(
-            C.c_int32(self.d_in), C.c_int32(self.hidden), C.c_int32(self.n_classes),
-            _p(self.theta), _p(self.m), _p(self.v), C.c_int32(self.optimizer),
-            C.c_double(self.lr), C.c_double(self.beta1), C.c_double(self.beta2), C.c_double(self.eps),
-            C.c_int64(self.step), C.c_int32(int(self.round_bf16)),
-            _p(x), C.c_int64(x.shape[1]), _p(ri), C.c_int64(n_rows), _p(y), C.byref(loss), _p(grad))
+        args = (C.c_int32(self.d_in), C.c_int32(self.hidden), C.c_int32(self.n_classes),
+                _p(self.theta), _p(self.m), _p(self.v), C.c_int32(self.optimizer),
+                C.c_double(self.lr), C.c_double(self.beta1), C.c_double(self.beta2), C.c_double(self.eps),
+                C.c_int64(self.step), C.c_int32(int(self.round_bf16)),
+                _p(x), C.c_int64(x.shape[1]), _p(ri), C.c_int64(n_rows), _p(y), C.byref(loss), _p(grad))
+        if dropout > 0.0:
+            rc = lib().oracle_mlp_train_step_dropout(*args, C.c_double(dropout), C.c_uint64(dropout_seed))
+        else:
+            rc = lib().oracle_mlp_train_step(*args)
         _check(rc, "oracle_mlp_train_step")
         return (loss.value, grad) if return_grad else loss.value
 

@@ -250,11 +250,59 @@ int64_t oracle_theta_size(int32_t d_in, int32_t hidden, int32_t n_classes)
     return (int64_t)d_in * n_classes + n_classes;
 }
 
+/* ------------------------------------------------------------------ */
+/* Dropout (Appendix B lists dropout rates among the hyper-parameters; */
+/* the configurations use none).  The random bits come from the        */
+/* counter-based generator Philox4x32-10 (Salmon, Moraes, Dror, Shaw:   */
+/* "Parallel random numbers: as easy as 1, 2, 3", SC'11), written out   */
+/* here from its definition: ten rounds of                              */
+/*   (c0,c1,c2,c3) <- (hi(M1 c2)^c1^k0, lo(M1 c2), hi(M0 c0)^c3^k1, lo(M0 c0)) */
+/* with the key raised by (W0, W1) between rounds.                      */
+/* ------------------------------------------------------------------ */
+void oracle_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = (uint64_t)M0 * c0, p1 = (uint64_t)M1 * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += W0; k1 += W1;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* Unit j of batch row i is kept in update number `step` iff word (j mod 4) of
+ * Philox(counter = (i, j / 4, step, 0), key = seed) is >= floor(p 2^32); a kept
+ * unit is scaled by 1 / (1 - p).  keep[j] receives that factor or 0. */
+static void dropout_row(int64_t i, int64_t step, int32_t hidden, double p, uint64_t seed, double *keep)
+{
+    const uint32_t thresh = (uint32_t)floor(p * 4294967296.0);
+    const double scale = 1.0 / (1.0 - p);
+    const uint32_t key[2] = {(uint32_t)(seed & 0xffffffffu), (uint32_t)(seed >> 32)};
+    for (int32_t j0 = 0; j0 < hidden; j0 += 4) {
+        const uint32_t ctr[4] = {(uint32_t)i, (uint32_t)(j0 >> 2), (uint32_t)step, 0u};
+        uint32_t w[4];
+        oracle_philox4x32_10(ctr, key, w);
+        for (int32_t t = 0; t < 4 && j0 + t < hidden; ++t) keep[j0 + t] = w[t] >= thresh ? scale : 0.0;
+    }
+}
+
+/* The keep factors of one row, for tests: keep_out[j] = 1/(1-p) or 0. */
+int oracle_dropout_mask(int64_t row, int64_t step, int32_t hidden, double p, uint64_t seed, double *keep_out)
+{
+    if (hidden <= 0 || p < 0.0 || p >= 1.0 || !keep_out) return ORACLE_BAD_ARG;
+    dropout_row(row, step, hidden, p, seed, keep_out);
+    return ORACLE_OK;
+}
+
 /* forward for one input row; a1 = pre-activation (hidden wide, may be NULL
- * when hidden == 0), logits = n_classes wide */
+ * when hidden == 0), logits = n_classes wide.  keep (optional, training with
+ * dropout only): factor applied to each hidden unit after the ReLU. */
 static void forward_row(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
                         int round_bf16, const float *xrow, const double *w1r, const double *w2r,
-                        double *a1, double *logits)
+                        double *a1, double *logits, const double *keep)
 {
     if (hidden > 0) {
         const double *b1 = theta + (int64_t)d_in * hidden;
@@ -270,6 +318,7 @@ static void forward_row(int32_t d_in, int32_t hidden, int32_t n_classes, const d
         for (int32_t c = 0; c < n_classes; ++c) logits[c] = 0.0;
         for (int32_t j = 0; j < hidden; ++j) {
             double h = a1[j] > 0.0 ? a1[j] : 0.0;
+            if (keep) h *= keep[j];
             h = opnd(h, round_bf16);
             if (h == 0.0) continue;
             const double *wrow = w2r + (int64_t)j * n_classes;
@@ -339,14 +388,17 @@ int oracle_apply_update(int64_t nt, double *theta, double *adam_m, double *adam_
  * optimizer: 0 = SGD (theta -= lr g), 1 = Adam (bias-corrected, eps outside
  * the root, no weight decay); `step` is the 1-based count of this update.
  * grad_out (optional) receives the gradient, laid out like theta. */
-int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
-                          double *theta, double *adam_m, double *adam_v,
-                          int32_t optimizer, double lr, double beta1, double beta2, double eps,
-                          int64_t step, int32_t round_bf16,
-                          const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
-                          const int32_t *y, double *loss_out, double *grad_out)
+static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
+                           double *theta, double *adam_m, double *adam_v,
+                           int32_t optimizer, double lr, double beta1, double beta2, double eps,
+                           int64_t step, int32_t round_bf16,
+                           const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                           const int32_t *y, double *loss_out, double *grad_out,
+                           double drop_p, uint64_t drop_seed)
 {
     if (d_in <= 0 || n_classes <= 0 || hidden < 0 || n_rows <= 0 || ldx < d_in) return ORACLE_BAD_ARG;
+    if (drop_p < 0.0 || drop_p >= 1.0) return ORACLE_BAD_ARG;
+    const int dropping = drop_p > 0.0 && hidden > 0;
     if (optimizer == 1 && (!adam_m || !adam_v || step < 1)) return ORACLE_BAD_ARG;
     int64_t nt = oracle_theta_size(d_in, hidden, n_classes);
     int32_t out1 = hidden > 0 ? hidden : n_classes;
@@ -369,10 +421,12 @@ int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
     {
         double *a1 = (double *)malloc(sizeof(double) * (size_t)(hidden > 0 ? hidden : 1));
         double *lg = (double *)malloc(sizeof(double) * (size_t)n_classes);
+        double *keep = dropping ? (double *)malloc(sizeof(double) * (size_t)hidden) : NULL;
 #pragma omp for schedule(static)
         for (int64_t i = 0; i < n_rows; ++i) {
             int64_t r = row_idx ? row_idx[i] : i;
-            forward_row(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg);
+            if (keep) dropout_row(i, step, hidden, drop_p, drop_seed, keep);
+            forward_row(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg, keep);
             int32_t yi = y[i];
             if (yi < 0 || yi >= n_classes) { bad_label = 1; yi = 0; }
             double mx = lg[0];
@@ -386,11 +440,13 @@ int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
             if (hidden > 0) {
                 for (int32_t j = 0; j < hidden; ++j) {
                     double h = a1[j] > 0.0 ? a1[j] : 0.0;
+                    if (keep) h *= keep[j];
                     hd[i * hidden + j] = h;
                     double acc = 0.0;
-                    if (a1[j] > 0.0) {
+                    if (a1[j] > 0.0 && (!keep || keep[j] != 0.0)) {
                         const double *wrow = w2r + (int64_t)j * n_classes;
                         for (int32_t c = 0; c < n_classes; ++c) acc += opnd(g[c], round_bf16) * wrow[c];
+                        if (keep) acc *= keep[j];
                     }
                     d1[i * hidden + j] = acc;
                 }
@@ -398,6 +454,7 @@ int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
         }
         free(a1);
         free(lg);
+        free(keep);
     }
 
     double loss = 0.0;
@@ -453,6 +510,32 @@ int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
     return bad_label ? ORACLE_BAD_ARG : ORACLE_OK;
 }
 
+int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
+                          double *theta, double *adam_m, double *adam_v,
+                          int32_t optimizer, double lr, double beta1, double beta2, double eps,
+                          int64_t step, int32_t round_bf16,
+                          const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                          const int32_t *y, double *loss_out, double *grad_out)
+{
+    return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0);
+}
+
+/* The same step with dropout on the hidden units: Hd = ReLU(X W1 + b1) .* keep,
+ * keep = 1/(1-p) with probability 1-p, else 0 (see dropout_row); the classifier,
+ * the loss and the backward pass see the masked, scaled Hd. */
+int oracle_mlp_train_step_dropout(int32_t d_in, int32_t hidden, int32_t n_classes,
+                                  double *theta, double *adam_m, double *adam_v,
+                                  int32_t optimizer, double lr, double beta1, double beta2, double eps,
+                                  int64_t step, int32_t round_bf16,
+                                  const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                                  const int32_t *y, double *loss_out, double *grad_out,
+                                  double drop_p, uint64_t drop_seed)
+{
+    return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, drop_p, drop_seed);
+}
+
 /* Forward of the trained per-node model over a set of rows.
  *   hidden > 0: hidden_out = ReLU(x W1 + b1)  — the representation Q^m that
  *               the next round aggregates, the classifier being dropped
@@ -479,7 +562,7 @@ int oracle_embed(int32_t d_in, int32_t hidden, int32_t n_classes, const double *
 #pragma omp for schedule(static)
         for (int64_t i = 0; i < n_rows; ++i) {
             int64_t r = row_idx ? row_idx[i] : i;
-            forward_row(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg);
+            forward_row(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg, NULL);
             if (hidden_out)
                 for (int32_t j = 0; j < hidden; ++j)
                     hidden_out[i * ld_hidden + j] = (float)(a1[j] > 0.0 ? a1[j] : 0.0);
