@@ -150,6 +150,13 @@ typedef struct retexo_mlp {
     int32_t optimizer;              /* retexo_optimizer */
     float lr, beta1, beta2, eps;    /* Adam: bias-corrected, eps outside the root, no weight decay */
     int64_t step;
+    /* Dropout on the hidden units while training (Appendix B lists dropout rates among the
+     * hyper-parameters): unit j of batch row i is dropped in update number s = step + 1 iff word (j mod 4)
+     * of Philox4x32-10(counter = (i, j / 4, s, 0), key = (low, high word of dropout_seed)) is below
+     * floor(dropout * 2^32); kept units are scaled by 1 / (1 - dropout).  0 <= dropout < 1; 0 = none.
+     * retexo_embed (evaluation) never drops.  retexo_lmp_train trains without dropout. */
+    float dropout;
+    uint64_t dropout_seed;
 } retexo_mlp;
 
 int64_t retexo_theta_size(int32_t d_in, int32_t hidden, int32_t n_classes);

@@ -40,7 +40,7 @@ class _Mlp(C.Structure):
     _fields_ = [("d_in", C.c_int32), ("hidden", C.c_int32), ("n_classes", C.c_int32),
                 ("theta", C.c_void_p), ("adam_m", C.c_void_p), ("adam_v", C.c_void_p),
                 ("optimizer", C.c_int32), ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
-                ("eps", C.c_float), ("step", C.c_int64)]
+                ("eps", C.c_float), ("step", C.c_int64), ("dropout", C.c_float), ("dropout_seed", C.c_uint64)]
 
 
 class _LmpConfig(C.Structure):
@@ -207,7 +207,7 @@ class Mlp:
 
     def __init__(self, d_in: int, hidden: int, n_classes: int, w1, b1, w2=None, b2=None, optimizer: int = ADAM,
                  lr: float = 0.003, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
-                 device: str = "cuda"):
+                 device: str = "cuda", dropout: float = 0.0, dropout_seed: int = 0):
         self.d_in, self.hidden, self.n_classes = int(d_in), int(hidden), int(n_classes)
         parts = [np.asarray(w1, dtype=np.float32).ravel(), np.asarray(b1, dtype=np.float32).ravel()]
         if hidden > 0:
@@ -218,7 +218,7 @@ class Mlp:
         self.m = torch.zeros_like(self.theta)
         self.v = torch.zeros_like(self.theta)
         self.c = _Mlp(self.d_in, self.hidden, self.n_classes, self.theta.data_ptr(), self.m.data_ptr(),
-                      self.v.data_ptr(), optimizer, lr, beta1, beta2, eps, 0)
+                      self.v.data_ptr(), optimizer, lr, beta1, beta2, eps, 0, dropout, dropout_seed)
 
     @property
     def step(self) -> int:

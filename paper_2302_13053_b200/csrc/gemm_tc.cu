@@ -134,6 +134,21 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
         :: "memory");
 }
 
+// One block of the counter-based generator Philox4x32-10 (Salmon et al., SC'11), from its definition:
+// ten rounds of (c0,c1,c2,c3) <- (hi(M1 c2)^c1^k0, lo(M1 c2), hi(M0 c0)^c3^k1, lo(M0 c0)), the key raised
+// by (W0, W1) between rounds.
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1,
+                                              uint32_t (&out)[4]) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        c0 = hi1 ^ c1 ^ k0; c1 = lo1; c2 = hi0 ^ c3 ^ k1; c3 = lo0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
 struct TcKernelArgs {
     int64_t M, N;
     int32_t k_blocks_total;       // ceil(K / 64)
@@ -145,6 +160,8 @@ struct TcKernelArgs {
     __nv_bfloat16* out_bf16; int64_t ld_bf16;
     __nv_bfloat16* out_bf16_t; int64_t ld_t; int ones_row_t;
     const __nv_bfloat16* mask; int64_t ld_mask;
+    float gate_scale;
+    uint32_t drop_thresh, drop_step, drop_key0, drop_key1; float drop_scale; int64_t drop_rows;
     float* partial;
     const int32_t* y; float inv_rows; float* loss_partial;
     int32_t* pred; unsigned long long* correct;
@@ -665,6 +682,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 stage_block_from_global(g.mask, g.ld_mask, col0, row0, g.M, blk, lane);
                             }
                             if (n_kb > 0) tmem_ld_wait(r);
+                            if (g.gate_scale != 1.f) {      // (dropout: the kept units' factor)
+#pragma unroll
+                                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * g.gate_scale);
+                            }
                             uint32_t p[16];
 #pragma unroll
                             for (int qd = 0; qd < 4; ++qd) {
@@ -688,7 +709,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 const __nv_bfloat16* mrow = g.mask + row * g.ld_mask + col0;
 #pragma unroll
                                 for (int j = 0; j < 32; ++j)
-                                    v[j] = (col0 + j < g.N && __bfloat162float(mrow[j]) > 0.f) ? __uint_as_float(r[j]) : 0.f;
+                                    v[j] = (col0 + j < g.N && __bfloat162float(mrow[j]) > 0.f) ? __uint_as_float(r[j]) * g.gate_scale : 0.f;
                             } else {
 #pragma unroll
                                 for (int j = 0; j < 32; ++j) v[j] = 0.f;
@@ -707,6 +728,19 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             float x = __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_lane, j);
                             if (g.relu) x = fmaxf(x, 0.f);
                             v[j] = x;
+                        }
+                        if constexpr (MODE == TC_EPI_BIAS_DROP) {
+                            if (row < g.drop_rows) {      // training rows only; col0 is a multiple of 32
+#pragma unroll
+                                for (int j4 = 0; j4 < 8; ++j4) {
+                                    uint32_t w[4];
+                                    philox4x32_10((uint32_t)row, (uint32_t)((col0 >> 2) + j4), g.drop_step, 0u, g.drop_key0,
+                                                  g.drop_key1, w);
+#pragma unroll
+                                    for (int t = 0; t < 4; ++t)
+                                        v[4 * j4 + t] = w[t] >= g.drop_thresh ? v[4 * j4 + t] * g.drop_scale : 0.f;
+                                }
+                            }
                         }
                         if (g.out_f32 && row < g.M) {
                             float* dst = g.out_f32 + row * g.ld_f32 + col0;
@@ -812,6 +846,9 @@ static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensor
     g.out_f32 = t.out_f32; g.ld_f32 = t.ld_f32; g.out_bf16 = t.out_bf16; g.ld_bf16 = t.ld_bf16;
     g.out_bf16_t = t.out_bf16_t; g.ld_t = t.ld_t; g.ones_row_t = t.ones_row_t;
     g.mask = t.mask; g.ld_mask = t.ld_mask;
+    g.gate_scale = t.gate_scale != 0.f ? t.gate_scale : 1.f;
+    g.drop_thresh = t.drop_thresh; g.drop_step = t.drop_step; g.drop_key0 = t.drop_key[0]; g.drop_key1 = t.drop_key[1];
+    g.drop_scale = t.drop_scale; g.drop_rows = t.drop_rows;
     g.partial = t.partial; g.status = t.status;
     g.y = t.y; g.inv_rows = t.inv_rows; g.loss_partial = t.loss_partial; g.pred = t.pred; g.correct = t.correct;
     g.n_train = (t.mode == TC_EPI_SOFTMAX_CE && t.eval_from > 0 && t.eval_from < t.M) ? t.eval_from : t.M;
@@ -821,9 +858,10 @@ static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensor
     memset(&m_rows, 0, sizeof(m_rows));
     memset(&m_t, 0, sizeof(m_t));
     const bool ce = t.mode == TC_EPI_SOFTMAX_CE;
-    if (t.out_bf16 && (t.mode == TC_EPI_BIAS || t.mode == TC_EPI_MASK || ce))
+    const bool bias_like = t.mode == TC_EPI_BIAS || t.mode == TC_EPI_BIAS_DROP;
+    if (t.out_bf16 && (bias_like || t.mode == TC_EPI_MASK || ce))
         g.tma_rows = make_store_map(&m_rows, t.out_bf16, ce ? g.n_train : t.M, ce ? t.ld_bf16 : t.N, t.ld_bf16) ? 1 : 0;
-    if (t.out_bf16_t && (t.mode == TC_EPI_BIAS || t.mode == TC_EPI_MASK_T || ce))
+    if (t.out_bf16_t && (bias_like || t.mode == TC_EPI_MASK_T || ce))
         g.tma_t = make_store_map(&m_t, t.out_bf16_t, t.N, ce ? g.n_train : t.M, t.ld_t) ? 1 : 0;
     const int64_t n_tiles = ((t.M + kTcBM - 1) / kTcBM) * ((t.N + BN - 1) / BN) * splits;
     const int n_sm = sm_count();
@@ -837,6 +875,7 @@ template <int BN, int STAGES, int EW>
 static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
     switch (t.mode) {
         case TC_EPI_BIAS: return launch_tc_mode<BN, STAGES, TC_EPI_BIAS, EW>(t, ma, mb, st);
+        case TC_EPI_BIAS_DROP: return launch_tc_mode<BN, STAGES, TC_EPI_BIAS_DROP, EW>(t, ma, mb, st);
         case TC_EPI_PARTIAL: return launch_tc_mode<BN, STAGES, TC_EPI_PARTIAL, EW>(t, ma, mb, st);
         case TC_EPI_MASK_T: return launch_tc_mode<BN, STAGES, TC_EPI_MASK_T, EW>(t, ma, mb, st);
         case TC_EPI_MASK: return launch_tc_mode<BN, STAGES, TC_EPI_MASK, EW>(t, ma, mb, st);

@@ -7,7 +7,7 @@
 namespace retexo {
 
 enum TcEpilogue { TC_EPI_BIAS = 0, TC_EPI_PARTIAL = 1, TC_EPI_MASK_T = 2, TC_EPI_SOFTMAX_CE = 3, TC_EPI_ARGMAX = 4,
-                  TC_EPI_MASK = 5 };
+                  TC_EPI_MASK = 5, TC_EPI_BIAS_DROP = 6 };
 
 // C[M x N] = A[M x K] * B[N x K]^T with A and B bf16, K contiguous (row strides
 // lda / ldb elements, multiples of 8; bases 16-byte aligned).
@@ -41,6 +41,11 @@ struct TcGemm {
     __nv_bfloat16* out_bf16; int64_t ld_bf16;
     __nv_bfloat16* out_bf16_t; int64_t ld_t; int ones_row_t;
     const __nv_bfloat16* mask; int64_t ld_mask;
+    float gate_scale;          // TC_EPI_MASK / TC_EPI_MASK_T: factor on the gated values (0 is read as 1)
+    // TC_EPI_BIAS_DROP: as TC_EPI_BIAS, then dropout on rows [0, drop_rows): element (m, n) is kept iff word
+    // (n mod 4) of Philox4x32-10(counter = (m, n / 4, drop_step, 0), key = drop_key) >= drop_thresh, and a
+    // kept element is multiplied by drop_scale; rows from drop_rows on (evaluation rows) are left as they are.
+    uint32_t drop_thresh, drop_step, drop_key[2]; float drop_scale; int64_t drop_rows;
     float* partial;
     const int32_t* y; float inv_rows; float* loss_partial;      // TC_EPI_SOFTMAX_CE / TC_EPI_ARGMAX
     // TC_EPI_SOFTMAX_CE only: rows [eval_from, M) are not trained on but only evaluated: their arg-max is

@@ -112,6 +112,7 @@ size_t mlp_step_workspace_size(const MlpPlan& p) {
 static int check_model(const retexo_mlp* m) {
     if (!m || m->d_in <= 0 || m->hidden < 0 || m->n_classes <= 0 || !m->theta) return RETEXO_ERR_INVALID_ARG;
     if (m->n_classes > 64 || m->hidden > 512) return RETEXO_ERR_UNSUPPORTED;
+    if (!(m->dropout >= 0.f && m->dropout < 1.f)) return RETEXO_ERR_INVALID_ARG;
     return RETEXO_OK;
 }
 
@@ -224,9 +225,21 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     TcGemm fwd = tc_base(x, ldx, b.w1t16, p.ld_k, n_all, out1, d_in, b.status);
     fwd.bias = b1;
     TcGemm head = fwd;
+    const bool dropping = H > 0 && model->dropout > 0.f;
+    if (dropping && dev) return RETEXO_ERR_UNSUPPORTED;      // (the update number would have to come from the device)
+    const float keep_scale = dropping ? (float)(1.0 / (1.0 - (double)model->dropout)) : 1.f;
     if (H > 0) {
         fwd.relu = 1; fwd.out_bf16 = b.hd16; fwd.ld_bf16 = p.ld_h;
         fwd.out_bf16_t = b.hdt16; fwd.ld_t = p.ld_n; fwd.ones_row_t = 1;
+        if (dropping) {
+            fwd.mode = TC_EPI_BIAS_DROP;
+            fwd.drop_thresh = (uint32_t)floor((double)model->dropout * 4294967296.0);
+            fwd.drop_step = (uint32_t)(model->step + 1);
+            fwd.drop_key[0] = (uint32_t)(model->dropout_seed & 0xffffffffu);
+            fwd.drop_key[1] = (uint32_t)(model->dropout_seed >> 32);
+            fwd.drop_scale = keep_scale;
+            fwd.drop_rows = n;
+        }
         RETEXO_TRY(tc_gemm_launch(fwd, st));
         head = tc_base(b.hd16, p.ld_h, b.w2t16, p.ld_h, n_all, O, H, b.status);
         head.bias = b2;
@@ -243,6 +256,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         // gradient reads, so mask and output are both row-major for the epilogue
         TcGemm bk = tc_base(b.w2p16, p.ld_dl, b.dl16, p.ld_dl, H, n, O, b.status);
         bk.mode = TC_EPI_MASK; bk.mask = b.hdt16; bk.ld_mask = p.ld_n; bk.out_bf16 = b.dhdt16; bk.ld_bf16 = p.ld_n;
+        bk.gate_scale = keep_scale;      // a dropped unit has Hd = 0, so the gate already holds the mask
         RETEXO_TRY(tc_gemm_launch(bk, st));
         TcGemm g2 = tc_base(b.hdt16, p.ld_n, b.dlt16, p.ld_n, (int64_t)H + 1, O, n, b.status);
         g2.mode = TC_EPI_PARTIAL; g2.splits = (int)p.split_w2; g2.partial = b.pw2;
