@@ -154,7 +154,7 @@ typedef struct retexo_mlp {
      * hyper-parameters): unit j of batch row i is dropped in update number s = step + 1 iff word (j mod 4)
      * of Philox4x32-10(counter = (i, j / 4, s, 0), key = (low, high word of dropout_seed)) is below
      * floor(dropout * 2^32); kept units are scaled by 1 / (1 - dropout).  0 <= dropout < 1; 0 = none.
-     * retexo_embed (evaluation) never drops.  retexo_lmp_train trains without dropout. */
+     * retexo_embed (evaluation) never drops. */
     float dropout;
     uint64_t dropout_seed;
 } retexo_mlp;
@@ -314,6 +314,8 @@ typedef struct retexo_lmp_config {
     int32_t memory_is_host;         /* 0: every input array below is on the device;
                                        1: every input array is in HOST memory and is copied to the
                                           device inside the call; results are also written to host */
+    float dropout;                  /* dropout rate of the hidden units while training (see retexo_mlp); 0 = none */
+    uint64_t dropout_seed;          /* round m = 1..K draws its masks with the key dropout_seed + (m - 1) */
 } retexo_lmp_config;
 
 typedef struct retexo_lmp_inputs {

@@ -304,7 +304,8 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
               rowptr, colidx, features, labels, train_idx, val_idx, test_idx,
               weights: List[Dict[str, np.ndarray]], gat: Optional[Dict] = None,
               optimizer: int = ADAM, round_bf16: bool = True, eval_every: int = 1,
-              part=None, n_parts: int = 0, forced_best_iter: Optional[Sequence[int]] = None) -> Dict:
+              part=None, n_parts: int = 0, forced_best_iter: Optional[Sequence[int]] = None,
+              dropout: float = 0.0, dropout_seed: int = 0) -> Dict:
     """Lazy message passing (Section 3.1): for each layer m = 1..K, one
     message-passing round builds the layer's inputs, the layer (with a
     temporary classifier unless it is the last) is trained alone for R
@@ -345,7 +346,9 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
         best, best_correct, best_iter = None, -1, -1
         losses, val_hist = [], []
         for r in range(1, R + 1):
-            losses.append(model.train_step(x, y_tr, row_idx=train_idx))
+            # (dropout: round m draws its masks with the key dropout_seed + (m - 1), update numbers from 1)
+            losses.append(model.train_step(x, y_tr, row_idx=train_idx, dropout=dropout,
+                                           dropout_seed=(dropout_seed + m - 1) & 0xffffffffffffffff))
             report["n_steps"] += 1
             if r % eval_every == 0 or r == R:
                 c = model.embed(x, row_idx=val_idx, y=y_va, want_logits=False)["correct"]

@@ -47,7 +47,8 @@ class _LmpConfig(C.Structure):
     _fields_ = [("aggr", C.c_int32), ("K", C.c_int32), ("R", C.c_int32), ("d0", C.c_int32), ("hidden", C.c_int32),
                 ("n_classes", C.c_int32), ("optimizer", C.c_int32), ("lr", C.c_float), ("beta1", C.c_float),
                 ("beta2", C.c_float), ("eps", C.c_float), ("eval_every", C.c_int32), ("gat_heads", C.c_int32),
-                ("gat_head_dim", C.c_int32), ("gat_negative_slope", C.c_float), ("memory_is_host", C.c_int32)]
+                ("gat_head_dim", C.c_int32), ("gat_negative_slope", C.c_float), ("memory_is_host", C.c_int32),
+                ("dropout", C.c_float), ("dropout_seed", C.c_uint64)]
 
 
 class _LmpInputs(C.Structure):
@@ -351,13 +352,14 @@ class LmpProblem:
                  weights: List[Dict[str, np.ndarray]], part: Optional[np.ndarray] = None, n_parts: int = 0,
                  heads: int = 0, head_dim: int = 0, negative_slope: float = 0.2, optimizer: int = ADAM,
                  beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, eval_every: int = 1,
-                 host: bool = False, want_logits: bool = True, device: str = "cuda"):
+                 host: bool = False, want_logits: bool = True, device: str = "cuda", dropout: float = 0.0,
+                 dropout_seed: int = 0):
         self.host = bool(host)
         self.device = torch.device(device)
         n, e = rowptr.shape[0] - 1, colidx.shape[0]
         self.n, self.e, self.K, self.R, self.n_classes = n, e, K, R, n_classes
         self.cfg = _LmpConfig(aggr, K, R, features.shape[1], hidden, n_classes, optimizer, lr, beta1, beta2, eps,
-                              eval_every, heads, head_dim, negative_slope, 1 if host else 0)
+                              eval_every, heads, head_dim, negative_slope, 1 if host else 0, dropout, dropout_seed)
 
         def put(a: np.ndarray) -> torch.Tensor:
             t = torch.from_numpy(np.ascontiguousarray(a))

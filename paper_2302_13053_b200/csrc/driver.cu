@@ -227,6 +227,7 @@ static int check_cfg(const retexo_lmp_config* c) {
         return RETEXO_ERR_INVALID_ARG;
     if (c->aggr == RETEXO_GAT && (c->gat_heads <= 0 || c->gat_head_dim <= 0)) return RETEXO_ERR_INVALID_ARG;
     if (c->eval_every < 1) return RETEXO_ERR_INVALID_ARG;
+    if (!(c->dropout >= 0.f && c->dropout < 1.f)) return RETEXO_ERR_INVALID_ARG;
     if (c->n_classes > 64 || c->hidden > 512) return RETEXO_ERR_UNSUPPORTED;
     return RETEXO_OK;
 }
@@ -375,6 +376,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         model.theta = b.theta; model.adam_m = b.adam_m; model.adam_v = b.adam_v;
         model.optimizer = c.optimizer; model.lr = c.lr; model.beta1 = c.beta1; model.beta2 = c.beta2;
         model.eps = c.eps; model.step = 0;
+        model.dropout = c.dropout; model.dropout_seed = c.dropout_seed + (uint64_t)(m - 1);
         retexo_mlp best = model;
         best.theta = b.theta_best;
 

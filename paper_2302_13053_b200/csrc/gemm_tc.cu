@@ -162,6 +162,7 @@ struct TcKernelArgs {
     const __nv_bfloat16* mask; int64_t ld_mask;
     float gate_scale;
     uint32_t drop_thresh, drop_step, drop_key0, drop_key1; float drop_scale; int64_t drop_rows;
+    const unsigned long long* drop_step_dev;
     float* partial;
     const int32_t* y; float inv_rows; float* loss_partial;
     int32_t* pred; unsigned long long* correct;
@@ -731,10 +732,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         }
                         if constexpr (MODE == TC_EPI_BIAS_DROP) {
                             if (row < g.drop_rows) {      // training rows only; col0 is a multiple of 32
+                                const uint32_t update = g.drop_step_dev ? (uint32_t)__ldg(g.drop_step_dev) + 1u : g.drop_step;
 #pragma unroll
                                 for (int j4 = 0; j4 < 8; ++j4) {
                                     uint32_t w[4];
-                                    philox4x32_10((uint32_t)row, (uint32_t)((col0 >> 2) + j4), g.drop_step, 0u, g.drop_key0,
+                                    philox4x32_10((uint32_t)row, (uint32_t)((col0 >> 2) + j4), update, 0u, g.drop_key0,
                                                   g.drop_key1, w);
 #pragma unroll
                                     for (int t = 0; t < 4; ++t)
@@ -848,7 +850,7 @@ static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensor
     g.mask = t.mask; g.ld_mask = t.ld_mask;
     g.gate_scale = t.gate_scale != 0.f ? t.gate_scale : 1.f;
     g.drop_thresh = t.drop_thresh; g.drop_step = t.drop_step; g.drop_key0 = t.drop_key[0]; g.drop_key1 = t.drop_key[1];
-    g.drop_scale = t.drop_scale; g.drop_rows = t.drop_rows;
+    g.drop_scale = t.drop_scale; g.drop_rows = t.drop_rows; g.drop_step_dev = t.drop_step_dev;
     g.partial = t.partial; g.status = t.status;
     g.y = t.y; g.inv_rows = t.inv_rows; g.loss_partial = t.loss_partial; g.pred = t.pred; g.correct = t.correct;
     g.n_train = (t.mode == TC_EPI_SOFTMAX_CE && t.eval_from > 0 && t.eval_from < t.M) ? t.eval_from : t.M;

@@ -45,7 +45,9 @@ struct TcGemm {
     // TC_EPI_BIAS_DROP: as TC_EPI_BIAS, then dropout on rows [0, drop_rows): element (m, n) is kept iff word
     // (n mod 4) of Philox4x32-10(counter = (m, n / 4, drop_step, 0), key = drop_key) >= drop_thresh, and a
     // kept element is multiplied by drop_scale; rows from drop_rows on (evaluation rows) are left as they are.
+    // drop_step_dev (optional): the update number is *drop_step_dev + 1 instead of drop_step.
     uint32_t drop_thresh, drop_step, drop_key[2]; float drop_scale; int64_t drop_rows;
+    const unsigned long long* drop_step_dev;
     float* partial;
     const int32_t* y; float inv_rows; float* loss_partial;      // TC_EPI_SOFTMAX_CE / TC_EPI_ARGMAX
     // TC_EPI_SOFTMAX_CE only: rows [eval_from, M) are not trained on but only evaluated: their arg-max is

@@ -226,7 +226,6 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     fwd.bias = b1;
     TcGemm head = fwd;
     const bool dropping = H > 0 && model->dropout > 0.f;
-    if (dropping && dev) return RETEXO_ERR_UNSUPPORTED;      // (the update number would have to come from the device)
     const float keep_scale = dropping ? (float)(1.0 / (1.0 - (double)model->dropout)) : 1.f;
     if (H > 0) {
         fwd.relu = 1; fwd.out_bf16 = b.hd16; fwd.ld_bf16 = p.ld_h;
@@ -235,6 +234,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
             fwd.mode = TC_EPI_BIAS_DROP;
             fwd.drop_thresh = (uint32_t)floor((double)model->dropout * 4294967296.0);
             fwd.drop_step = (uint32_t)(model->step + 1);
+            fwd.drop_step_dev = dev ? dev->step : nullptr;      // (iteration state on the device: read there)
             fwd.drop_key[0] = (uint32_t)(model->dropout_seed & 0xffffffffu);
             fwd.drop_key[1] = (uint32_t)(model->dropout_seed >> 32);
             fwd.drop_scale = keep_scale;
