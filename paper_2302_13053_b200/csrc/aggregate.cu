@@ -117,7 +117,29 @@ struct AggArgs {
     int32_t* counters;               // [0] heavy rows, [1] segments, [2] next work item
     float* seg_partial;              // [segments x round_up(dim, 4)] raw sums
     int64_t ld_partial;
+    float hub_coef;                  // GCN, matrix larger than L2: rows of nodes with coef <= hub_coef (hubs) are
+                                     // loaded "evict last", all others "evict first"; 0 = no hints
 };
+
+// L2 eviction priorities for the gathers of a matrix that does not fit the cache: a power-law graph
+// reads its hubs' rows again and again, every other row a few times; left to itself the cache keeps
+// neither.  The hints change nothing but which lines stay resident.
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ float4 ldg_hinted(const float4* ptr, uint64_t policy) {
+    float4 v;
+    asm volatile("ld.global.nc.L2::cache_hint.v4.f32 {%0, %1, %2, %3}, [%4], %5;"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(ptr), "l"(policy));
+    return v;
+}
 
 // Adds the neighbour rows of CSR entries [beg, end) into acc, in order, for the
 // column vectors this lane owns in pass `pass`.  GCN weighs each row by coef[u].
@@ -128,6 +150,12 @@ __device__ __forceinline__ void accumulate_range(const AggArgs& a, int64_t beg, 
     using V = typename VecT<VEC>::type;
     const int64_t ldv = a.ldq / VEC;
     const V* __restrict__ qv = reinterpret_cast<const V*>(a.q);
+    constexpr bool kCanHint = OP == kOpGcn && VEC == 4;
+    [[maybe_unused]] uint64_t keep = 0, pass = 0;
+    [[maybe_unused]] const bool hinting = kCanHint && a.hub_coef > 0.f;
+    if constexpr (kCanHint) {
+        if (hinting) { keep = l2_policy_evict_last(); pass = l2_policy_evict_first(); }
+    }
     for (int64_t e0 = beg; e0 < end; e0 += kWarp) {
         const int cnt = (int)min((int64_t)kWarp, end - e0);
         int my_u = 0;
@@ -148,8 +176,14 @@ __device__ __forceinline__ void accumulate_range(const AggArgs& a, int64_t beg, 
 #pragma unroll
                 for (int c = 0; c < CH; ++c) {
                     const int vi = vec0 + c * kWarp + lane;
-                    if (vi < nvec) x[t][c] = __ldg(row + vi);
-                    else vec_zero<VEC>(x[t][c]);
+                    if (vi < nvec) {
+                        if constexpr (kCanHint) {
+                            if (hinting) x[t][c] = ldg_hinted(row + vi, w[t] <= a.hub_coef ? keep : pass);
+                            else x[t][c] = __ldg(row + vi);
+                        } else {
+                            x[t][c] = __ldg(row + vi);
+                        }
+                    } else vec_zero<VEC>(x[t][c]);
                 }
             }
 #pragma unroll
@@ -742,6 +776,10 @@ extern "C" int retexo_aggregate(const retexo_csr* g, int32_t type, const float* 
     a.ld_partial = (dim + 3) / 4 * 4;
     a.seg_partial = ws.take<float>((size_t)max_segments(e) * (size_t)a.ld_partial);
     a.coef = coef; a.heavy_list = heavy_list; a.heavy_seg_base = heavy_seg_base; a.seg_slot = seg_slot;
+    // hubs = nodes of at least four times the mean degree; hinted only where the matrix is larger than L2
+    a.hub_coef = 0.f;
+    if (type == RETEXO_GCN && (size_t)n * (size_t)dim * 4 >= kSlabMinMatrixBytes && n > 0)
+        a.hub_coef = (float)(1.0 / sqrt(4.0 * (double)e / (double)n + 1.0));
     a.counters = counters;
     a.out = out; a.ldout = ldout;
     a.out16 = static_cast<__nv_bfloat16*>(out_bf16); a.ldout16 = ldout_bf16;
