@@ -38,8 +38,8 @@ UNIT = "edges/s"
 # summarised in profiles/agg_kernels_cfg4.txt and profiles/agg_rows_kernel_cfg5.txt.  Valid for that
 # kernel and workload only: set an entry to None when the kernel or the workload changes.
 AGG_DRAM_TRAFFIC = {("cfg4_sage_reddit_like", 1): 14.68e9, ("cfg4_sage_reddit_like", 2): 6.24e9,
-                    ("cfg4_sage_reddit_like", 3): 5.99e9, ("cfg5_gcn_products_like", 1): 52.61e9,
-                    ("cfg5_gcn_products_like", 2): 116.56e9, ("cfg5_gcn_products_like", 3): 116.55e9}
+                    ("cfg4_sage_reddit_like", 3): 5.99e9, ("cfg5_gcn_products_like", 1): 46.68e9,
+                    ("cfg5_gcn_products_like", 2): 102.92e9, ("cfg5_gcn_products_like", 3): 102.93e9}
 # DRAM bytes of one stand-alone training iteration (its five tc_gemm_kernel launches and
 # reduce_update_kernel), from the one-pass capture summarised in profiles/tc_gemm_kernel_cfg4.txt.
 STEP_DRAM_TRAFFIC = {("cfg4_sage_reddit_like", 1): 1.280e9}

@@ -231,7 +231,7 @@ struct UpdateArgs {
 
 // One parameter: sum of its split-K partials in index order, optimiser step, bf16 copies.
 __device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p, int sidx, int64_t q, int64_t size,
-                                                 float corr1, float corr2) {
+                                                 float corr1, float corr2, bool snapshot) {
     const float* part = sidx == 0 ? u.seg[0].partial : u.seg[1].partial;
     const int64_t count = sidx == 0 ? u.seg[0].count : u.seg[1].count;
     float g = 0.f;
@@ -250,7 +250,7 @@ __device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p,
     }
     for (; z < count; ++z) g += part[z * size + q];
     if (u.grad_out) u.grad_out[p] = g;
-    if (u.theta_best && (!*u.snap_have || *u.snap_cur > *u.snap_best)) u.theta_best[p] = u.theta[p];
+    if (snapshot) u.theta_best[p] = u.theta[p];
     float t;
     if (u.optimizer == RETEXO_SGD) {
         t = u.theta[p] - u.lr * g;
@@ -276,7 +276,7 @@ __device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p,
 
 // Sums each parameter's split-K partials in index order, applies the optimiser, and refreshes
 // the bf16 weight copies.  Block 0 also reduces the loss (fixed order: per-lane strided sums,
-// then a shuffle tree).  With u.done set, the last block to finish does the validation bookkeeping.
+// then a shuffle tree).  With u.done set, the last block to arrive does the validation bookkeeping.
 __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     const int64_t p = blockIdx.x * 256ll + threadIdx.x;
     float corr1 = u.corr1, corr2 = u.corr2;
@@ -299,37 +299,42 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
         s = warp_sum(s);
         if (threadIdx.x == 0) *loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
     }
+    // keep-the-best: are the weights as they stand (validated in this iteration's forward pass) the best so far?
+    const bool snapshot = u.theta_best && (!*u.snap_have || *u.snap_cur > *u.snap_best);
+    if (u.done) {
+        // Once every block has read the validation state and the iteration number (signalled here, before
+        // the block's own stores, so the fence has nothing to wait for), the last block to arrive books
+        // the count and moves the state on, while the others are already updating their parameters.
+        __shared__ bool is_last;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            __threadfence();
+            is_last = atomicAdd(u.done, 1ull) == (unsigned long long)gridDim.x - 1ull;
+        }
+        __syncthreads();
+        if (is_last && threadIdx.x == 0) {
+            __threadfence();
+            if (u.snap_cur) {
+                const unsigned long long cur = *u.snap_cur;
+                unsigned long long* slot = u.step_dev ? (u.history_base && step_now > 0 ? u.history_base + (step_now - 1) : nullptr)
+                                                      : u.rec_history_slot;
+                if (slot) *slot = cur;
+                if (!*u.snap_have || cur > *u.snap_best) {
+                    *u.snap_best = cur;
+                    if (u.rec_best_iter) *u.rec_best_iter = u.step_dev ? (int32_t)step_now : u.rec_iter;
+                    *u.snap_have = 1;
+                }
+                *u.snap_cur = 0ull;
+            }
+            if (u.step_dev) *u.step_dev = step_now + 1;
+            *u.done = 0ull;
+        }
+    }
     const int64_t size0 = u.seg[0].size;
     const int sidx = p < size0 ? 0 : 1;
     const int64_t q = sidx == 0 ? p : p - size0;
     const int64_t size = sidx == 0 ? size0 : u.seg[1].size;
-    if (sidx < u.n_seg && q < size) update_parameter(u, p, sidx, q, size, corr1, corr2);
-    if (!u.done) return;
-    // every block has compared against the kept count by the time the last one records the new one
-    __shared__ bool is_last;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        __threadfence();
-        is_last = atomicAdd(u.done, 1ull) == (unsigned long long)gridDim.x - 1ull;
-    }
-    __syncthreads();
-    if (is_last && threadIdx.x == 0) {
-        __threadfence();
-        if (u.snap_cur) {
-            const unsigned long long cur = *u.snap_cur;
-            unsigned long long* slot = u.step_dev ? (u.history_base && step_now > 0 ? u.history_base + (step_now - 1) : nullptr)
-                                                  : u.rec_history_slot;
-            if (slot) *slot = cur;
-            if (!*u.snap_have || cur > *u.snap_best) {
-                *u.snap_best = cur;
-                if (u.rec_best_iter) *u.rec_best_iter = u.step_dev ? (int32_t)step_now : u.rec_iter;
-                *u.snap_have = 1;
-            }
-            *u.snap_cur = 0ull;
-        }
-        if (u.step_dev) *u.step_dev = step_now + 1;
-        *u.done = 0ull;
-    }
+    if (sidx < u.n_seg && q < size) update_parameter(u, p, sidx, q, size, corr1, corr2, snapshot);
 }
 
 __global__ void __launch_bounds__(256) f32_to_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int64_t n) {
