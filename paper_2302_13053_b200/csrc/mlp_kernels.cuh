@@ -229,6 +229,18 @@ struct UpdateArgs {
     unsigned long long* step_dev; float* loss_base; unsigned long long* history_base;
 };
 
+// base^e for a whole exponent by repeated squaring (a handful of double multiplications: the library
+// power function costs microseconds on a part with few double-precision units).
+__device__ __forceinline__ double pow_whole(double base, unsigned long long e) {
+    double r = 1.0;
+    while (e) {
+        if (e & 1ull) r *= base;
+        base *= base;
+        e >>= 1;
+    }
+    return r;
+}
+
 // One parameter: sum of its split-K partials in index order, optimiser step, bf16 copies.
 __device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p, int sidx, int64_t q, int64_t size,
                                                  float corr1, float corr2, bool snapshot) {
@@ -286,8 +298,8 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
         __shared__ float corr_s[2];
         step_now = *u.step_dev;
         if (threadIdx.x == 0) {
-            corr_s[0] = (float)(1.0 - pow((double)u.beta1, (double)(step_now + 1)));
-            corr_s[1] = (float)(1.0 - pow((double)u.beta2, (double)(step_now + 1)));
+            corr_s[0] = (float)(1.0 - pow_whole((double)u.beta1, step_now + 1));
+            corr_s[1] = (float)(1.0 - pow_whole((double)u.beta2, step_now + 1));
         }
         __syncthreads();
         corr1 = corr_s[0]; corr2 = corr_s[1];
