@@ -68,8 +68,16 @@ __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v)
 // partitions already seen is a bitmap in shared memory.
 __global__ void __launch_bounds__(kCntThreads) count_bitmap_kernel(CountArgs a) {
     __shared__ uint32_t bm[kCntWarps][kBitmapWords];
+    // per-partition receive tally of this block (only when asked for: n_parts words of dynamic shared
+    // memory), added to the global one once at the end: one global atomic per message would serialise
+    // on the few hundred addresses
+    extern __shared__ uint32_t recv_block[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (int i = lane; i < kBitmapWords; i += kWarp) bm[warp][i] = 0u;
+    if (a.recv) {
+        for (int i = threadIdx.x; i < a.n_parts; i += kCntThreads) recv_block[i] = 0u;
+        __syncthreads();
+    }
     __syncwarp();
     unsigned long long my_cross = 0, my_pairs = 0;
     for (int64_t u0 = next_rows(a, lane); u0 < a.n; u0 = next_rows(a, lane))
@@ -97,7 +105,7 @@ __global__ void __launch_bounds__(kCntThreads) count_bitmap_kernel(CountArgs a) 
                     const uint32_t bit = 1u << (pv[t] & 31);
                     const uint32_t old = atomicOr(&bm[warp][pv[t] >> 5], bit);
                     is_new = !(old & bit);
-                    if (is_new && a.recv) atomicAdd(a.recv + pv[t], 1ull);
+                    if (is_new && a.recv) atomicAdd(&recv_block[pv[t]], 1u);
                 }
                 my_cross += cross ? 1ull : 0ull;
                 row_new += __popc(__ballot_sync(0xffffffffu, is_new));
@@ -123,6 +131,11 @@ __global__ void __launch_bounds__(kCntThreads) count_bitmap_kernel(CountArgs a) 
     if (lane == 0) {
         if (my_cross) atomicAdd(a.cross_edges, my_cross);
         if (my_pairs) atomicAdd(a.pairs, my_pairs);
+    }
+    if (a.recv) {
+        __syncthreads();
+        for (int i = threadIdx.x; i < a.n_parts; i += kCntThreads)
+            if (recv_block[i]) atomicAdd(a.recv + i, (unsigned long long)recv_block[i]);
     }
 }
 
@@ -444,7 +457,8 @@ extern "C" int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* 
             // ~16 draws per warp: fine enough to balance hub rows, coarse enough for the counter
             const int64_t batch = a.n / ((int64_t)blocks * kCntWarps * 16);
             a.row_batch = (int32_t)(batch < 1 ? 1 : batch > 64 ? 64 : batch);
-            count_bitmap_kernel<<<blocks, kCntThreads, 0, st>>>(a);
+            const size_t tally = a.recv ? sizeof(uint32_t) * (size_t)n_parts : 0;      // <= 32 KB
+            count_bitmap_kernel<<<blocks, kCntThreads, tally, st>>>(a);
         } else {
             a.big_list = ws.take<int32_t>((size_t)a.n);
             a.big_count = ws.take<int32_t>(64);
