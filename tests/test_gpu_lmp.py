@@ -124,3 +124,37 @@ def test_eval_every_skips_validation_and_marks_the_gaps():
     evaluated = [i for i in range(10) if v[i] != 2 ** 64 - 1]
     assert evaluated == [3, 7, 9]
     assert got["best_iter"][0] in (4, 8, 10)
+
+
+def test_a_callers_own_stream_gives_the_same_bits_and_orders_later_work():
+    """The run is ordered inside the stream it is given: launched on a stream of the caller's with
+    work queued before and after it, it gives the same bits as on the default stream (plain
+    launches and the replayed graph alike: validation every iteration, and every third one)."""
+    from paper_2302_13053_b200 import binding as B
+    w = wl.make_config(2, scale=0.3)
+    ws = wl.initial_weights(w)
+    for eval_every in (1, 3):
+        res = []
+        for own in (False, True):
+            prob = B.LmpProblem(w.aggr, w.K, 9, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
+                                w.train_idx, w.val_idx, w.test_idx, ws, part=w.part, n_parts=w.n_parts,
+                                eval_every=eval_every)
+            if own:
+                s = torch.cuda.Stream()
+                s.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(s):
+                    busy = torch.randn(4096, 4096, device="cuda") @ torch.randn(4096, 4096, device="cuda")   # queued first
+                    B.retexo_lmp_train(prob)
+                    after = prob.loss_history.clone()                          # queued behind the run, same stream
+                s.synchronize()
+                assert torch.isfinite(busy).all()
+                res.append((prob.results(), after.cpu().numpy()))
+            else:
+                B.retexo_lmp_train(prob)
+                torch.cuda.synchronize()
+                res.append((prob.results(), None))
+        a, (b, after) = res[0][0], res[1]
+        np.testing.assert_array_equal(a["loss_history"], b["loss_history"])
+        np.testing.assert_array_equal(a["val_correct"], b["val_correct"])
+        np.testing.assert_array_equal(a["final_logits"], b["final_logits"])
+        np.testing.assert_array_equal(after.reshape(b["loss_history"].shape), b["loss_history"])
