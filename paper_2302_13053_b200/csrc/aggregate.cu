@@ -560,7 +560,11 @@ struct GatArgs {
     int64_t ldout;
     __nv_bfloat16* out16;
     int64_t ldout16;
+    int32_t* hub_list;      // rows left to gat_hub_kernel (order arbitrary; no result depends on it)
+    int32_t* hub_count;
 };
+
+constexpr int kGatHubEntries = 512;     // rows with at least this many entries are taken by a whole block
 
 // s_u = <a_src, p_u>, t_u = <a_dst, p_u> per head; one warp per node.
 __global__ void __launch_bounds__(kAggThreads) gat_scores_kernel(GatArgs a) {
@@ -584,37 +588,18 @@ __global__ void __launch_bounds__(kAggThreads) gat_scores_kernel(GatArgs a) {
     }
 }
 
-// One warp per destination v.  Entries are taken 32 at a time: lane j scores
-// entry j for every head, the chunk maximum and the rescale of the running
-// softmax state are warp reductions (one exp per entry and head in total),
-// then all lanes add the weighted neighbour rows for the columns they own.
+// The running soft-max state and weighted sum of one warp over the entries [e0, e0 + 32) of row v, for
+// e0 = e_first, e_first + e_step, ...  (entry `deg`, if any, is the self loop).  Entries are taken 32 at
+// a time: lane j scores entry j for every head, the chunk maximum and the rescale of the running
+// soft-max state are warp reductions (one exp per entry and head in total), then all lanes add the
+// weighted neighbour rows for the columns they own.
 template <int NC>
-__global__ void __launch_bounds__(kAggThreads) gat_rows_kernel(GatArgs a) {
-    __shared__ float p_s[kAggWarps][kWarp][kGatMaxHeads];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t v = blockIdx.x * (int64_t)kAggWarps + warp;
-    if (v >= a.n) return;
-    const int64_t beg = a.rowptr[v];
-    const int64_t deg = a.rowptr[v + 1] - beg;
-    const int64_t total = deg + (a.self_loop ? 1 : 0);
-
-    float m[kGatMaxHeads], l[kGatMaxHeads], tv[kGatMaxHeads];
-#pragma unroll
-    for (int h = 0; h < kGatMaxHeads; ++h) {
-        m[h] = -INFINITY;
-        l[h] = 0.f;
-        tv[h] = h < a.heads ? a.t[v * a.heads + h] : 0.f;
-    }
-    float acc[NC];
-    int head_of[NC];
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-        acc[c] = 0.f;
-        const int col = c * kWarp + lane;
-        head_of[c] = col < a.dim ? col / a.head_dim : 0;
-    }
-
-    for (int64_t e0 = 0; e0 < total; e0 += kWarp) {
+__device__ __forceinline__ void gat_accumulate(const GatArgs& a, int64_t v, int64_t beg, int64_t deg, int64_t total,
+                                               int64_t e_first, int64_t e_step, int lane, int warp,
+                                               float (*p_s)[kWarp][kGatMaxHeads], const float (&tv)[kGatMaxHeads],
+                                               const int (&head_of)[NC], float (&m)[kGatMaxHeads],
+                                               float (&l)[kGatMaxHeads], float (&acc)[NC]) {
+    for (int64_t e0 = e_first; e0 < total; e0 += e_step) {
         const int cnt = (int)min((int64_t)kWarp, total - e0);
         int my_u = 0;
         float e[kGatMaxHeads];
@@ -681,6 +666,40 @@ __global__ void __launch_bounds__(kAggThreads) gat_rows_kernel(GatArgs a) {
         }
         __syncwarp();
     }
+}
+
+// One warp per destination v (rows of kGatHubEntries entries or more are left to gat_hub_kernel).
+template <int NC>
+__global__ void __launch_bounds__(kAggThreads) gat_rows_kernel(GatArgs a) {
+    __shared__ float p_s[kAggWarps][kWarp][kGatMaxHeads];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t v = blockIdx.x * (int64_t)kAggWarps + warp;
+    if (v >= a.n) return;
+    const int64_t beg = a.rowptr[v];
+    const int64_t deg = a.rowptr[v + 1] - beg;
+    const int64_t total = deg + (a.self_loop ? 1 : 0);
+    if (total >= kGatHubEntries && a.hub_list) {      // a whole block takes this row
+        if (lane == 0) a.hub_list[atomicAdd(a.hub_count, 1)] = (int32_t)v;
+        return;
+    }
+
+    float m[kGatMaxHeads], l[kGatMaxHeads], tv[kGatMaxHeads];
+#pragma unroll
+    for (int h = 0; h < kGatMaxHeads; ++h) {
+        m[h] = -INFINITY;
+        l[h] = 0.f;
+        tv[h] = h < a.heads ? a.t[v * a.heads + h] : 0.f;
+    }
+    float acc[NC];
+    int head_of[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        acc[c] = 0.f;
+        const int col = c * kWarp + lane;
+        head_of[c] = col < a.dim ? col / a.head_dim : 0;
+    }
+
+    gat_accumulate<NC>(a, v, beg, deg, total, 0, kWarp, lane, warp, p_s, tv, head_of, m, l, acc);
 #pragma unroll
     for (int c = 0; c < NC; ++c) {
         const int col = c * kWarp + lane;
@@ -691,6 +710,68 @@ __global__ void __launch_bounds__(kAggThreads) gat_rows_kernel(GatArgs a) {
         const float val = total > 0 ? acc[c] / den : 0.f;
         if (a.out) a.out[v * a.ldout + col] = val;
         if (a.out16) a.out16[v * a.ldout16 + col] = f32_to_bf16(val);
+    }
+}
+
+
+// One block per hub row (listed by gat_rows_kernel): warp w takes the chunks w, w + 8, ... of the row
+// with a soft-max state of its own; the eight states are then merged in warp order
+//   M = max m_w,  L = sum l_w e^(m_w - M),  Z = sum acc_w e^(m_w - M) / L,
+// so the result does not depend on scheduling (it differs from the one-warp order only in rounding).
+template <int NC>
+__global__ void __launch_bounds__(kAggThreads) gat_hub_kernel(GatArgs a) {
+    __shared__ float p_s[kAggWarps][kWarp][kGatMaxHeads];
+    __shared__ float sm_m[kAggWarps][kGatMaxHeads], sm_l[kAggWarps][kGatMaxHeads];
+    __shared__ float sm_acc[kAggWarps][NC * kWarp];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int n_hubs = *a.hub_count;
+    for (int hub = blockIdx.x; hub < n_hubs; hub += gridDim.x) {
+        const int64_t v = a.hub_list[hub];
+        const int64_t beg = a.rowptr[v];
+        const int64_t deg = a.rowptr[v + 1] - beg;
+        const int64_t total = deg + (a.self_loop ? 1 : 0);
+        float m[kGatMaxHeads], l[kGatMaxHeads], tv[kGatMaxHeads];
+#pragma unroll
+        for (int h = 0; h < kGatMaxHeads; ++h) {
+            m[h] = -INFINITY;
+            l[h] = 0.f;
+            tv[h] = h < a.heads ? a.t[v * a.heads + h] : 0.f;
+        }
+        float acc[NC];
+        int head_of[NC];
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            acc[c] = 0.f;
+            const int col = c * kWarp + lane;
+            head_of[c] = col < a.dim ? col / a.head_dim : 0;
+        }
+        gat_accumulate<NC>(a, v, beg, deg, total, (int64_t)warp * kWarp, (int64_t)kAggWarps * kWarp, lane, warp, p_s, tv,
+                           head_of, m, l, acc);
+        if (lane < kGatMaxHeads) {
+            float mm = -INFINITY, ll = 0.f;
+#pragma unroll
+            for (int h = 0; h < kGatMaxHeads; ++h) if (h == lane) { mm = m[h]; ll = l[h]; }
+            sm_m[warp][lane] = mm;
+            sm_l[warp][lane] = ll;
+        }
+#pragma unroll
+        for (int c = 0; c < NC; ++c) sm_acc[warp][c * kWarp + lane] = acc[c];
+        __syncthreads();
+        for (int col = threadIdx.x; col < a.dim; col += kAggThreads) {
+            const int h = col / a.head_dim;
+            float big = -INFINITY;
+            for (int w = 0; w < kAggWarps; ++w) big = fmaxf(big, sm_m[w][h]);
+            float den = 0.f, num = 0.f;
+            for (int w = 0; w < kAggWarps; ++w) {
+                const float f = sm_m[w][h] == -INFINITY ? 0.f : expf(sm_m[w][h] - big);     // (a warp without chunks)
+                den = fmaf(sm_l[w][h], f, den);
+                num = fmaf(sm_acc[w][col], f, num);
+            }
+            const float val = num / den;
+            if (a.out) a.out[v * a.ldout + col] = val;
+            if (a.out16) a.out16[v * a.ldout16 + col] = f32_to_bf16(val);
+        }
+        __syncthreads();
     }
 }
 
@@ -705,6 +786,8 @@ extern "C" size_t retexo_aggregate_workspace_size(int64_t n_nodes, int64_t n_edg
     if (type == RETEXO_GAT) {
         s.take<float>((size_t)n_nodes * (size_t)(heads > 0 ? heads : 1));
         s.take<float>((size_t)n_nodes * (size_t)(heads > 0 ? heads : 1));
+        s.take<int32_t>((size_t)n_nodes);                                 // hub rows
+        s.take<int32_t>(64);                                              // their count
     } else {
         s.take<float>((size_t)n_nodes);                                   // coef
         s.take<int32_t>((size_t)(n_edges / kHeavyDegree + 1));            // heavy rows
@@ -753,15 +836,19 @@ extern "C" int retexo_aggregate(const retexo_csr* g, int32_t type, const float* 
         a.self_loop = gat->add_self_loop ? 1 : 0;
         a.s = ws.take<float>((size_t)n * gat->heads);
         a.t = ws.take<float>((size_t)n * gat->heads);
+        a.hub_list = ws.take<int32_t>((size_t)n);
+        a.hub_count = ws.take<int32_t>(64);
+        RETEXO_CUDA_TRY(cudaMemsetAsync(a.hub_count, 0, sizeof(int32_t), st));
         a.out = out; a.ldout = ldout;
         a.out16 = static_cast<__nv_bfloat16*>(out_bf16); a.ldout16 = ldout_bf16;
         const unsigned blocks = (unsigned)((n + kAggWarps - 1) / kAggWarps);
         gat_scores_kernel<<<blocks, kAggThreads, 0, st>>>(a);
         const int nc = (dim + kWarp - 1) / kWarp;
-        if (nc <= 1) gat_rows_kernel<1><<<blocks, kAggThreads, 0, st>>>(a);
-        else if (nc <= 2) gat_rows_kernel<2><<<blocks, kAggThreads, 0, st>>>(a);
-        else if (nc <= 4) gat_rows_kernel<4><<<blocks, kAggThreads, 0, st>>>(a);
-        else gat_rows_kernel<8><<<blocks, kAggThreads, 0, st>>>(a);
+        const unsigned hub_blocks = (unsigned)(2 * n_sm);
+        if (nc <= 1) { gat_rows_kernel<1><<<blocks, kAggThreads, 0, st>>>(a); gat_hub_kernel<1><<<hub_blocks, kAggThreads, 0, st>>>(a); }
+        else if (nc <= 2) { gat_rows_kernel<2><<<blocks, kAggThreads, 0, st>>>(a); gat_hub_kernel<2><<<hub_blocks, kAggThreads, 0, st>>>(a); }
+        else if (nc <= 4) { gat_rows_kernel<4><<<blocks, kAggThreads, 0, st>>>(a); gat_hub_kernel<4><<<hub_blocks, kAggThreads, 0, st>>>(a); }
+        else { gat_rows_kernel<8><<<blocks, kAggThreads, 0, st>>>(a); gat_hub_kernel<8><<<hub_blocks, kAggThreads, 0, st>>>(a); }
         return launch_status();
     }
 

@@ -150,17 +150,24 @@ def test_gat_random_graphs(heads, dh, self_loop):
     assert_rows_close(got, ref, what="gat %dx%d" % (heads, dh))
 
 
-def test_gat_long_rows_isolated_nodes_and_large_scores():
-    n, rowptr, colidx, _ = wl.degree_ladder_graph([0, 1, 31, 32, 33, 700, 3000], seed=5)
+@pytest.mark.parametrize("heads,dh", [(4, 16), (8, 32), (1, 7)])
+def test_gat_long_rows_isolated_nodes_and_large_scores(heads, dh):
+    """Rows on both sides of the 512-entry mark, from which a whole block takes a row and merges the
+    soft-max states of its eight warps."""
+    n, rowptr, colidx, _ = wl.degree_ladder_graph([0, 1, 31, 32, 33, 510, 511, 512, 513, 700, 3000], seed=5)
     rng = np.random.default_rng(5)
-    p = (rng.standard_normal((n, 64)) * 3).astype(np.float32)
+    p = (rng.standard_normal((n, heads * dh)) * 3).astype(np.float32)
+    if heads * dh < 16:
+        p = np.abs(p) + 0.5
     for self_loop in (0, 1):
-        gat = dict(heads=4, head_dim=16, a_src=(rng.standard_normal((4, 16)) * 2).astype(np.float32),
-                   a_dst=(rng.standard_normal((4, 16)) * 2).astype(np.float32), negative_slope=0.2,
+        gat = dict(heads=heads, head_dim=dh, a_src=(rng.standard_normal((heads, dh)) * 2).astype(np.float32),
+                   a_dst=(rng.standard_normal((heads, dh)) * 2).astype(np.float32), negative_slope=0.2,
                    add_self_loop=self_loop)
         ref = oracle.aggregate(oracle.GAT, rowptr, colidx, p, gat=gat)
-        got, _ = gat_gpu(rowptr, colidx, p, gat, ld=96)
+        got, _ = gat_gpu(rowptr, colidx, p, gat, ld=(heads * dh + 31) // 32 * 32 + 32)
         assert_rows_close(got, ref, what="gat ladder self=%d" % self_loop)
+        again, _ = gat_gpu(rowptr, colidx, p, gat, ld=(heads * dh + 31) // 32 * 32 + 32)
+        np.testing.assert_array_equal(again, got)        # repeatable bit for bit
 
 
 def test_gat_config3_projected_input():
