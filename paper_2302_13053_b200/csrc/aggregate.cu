@@ -560,17 +560,20 @@ struct GatArgs {
     int64_t ldout;
     __nv_bfloat16* out16;
     int64_t ldout16;
-    int32_t* hub_list;      // rows left to gat_hub_kernel (order arbitrary; no result depends on it)
+    int32_t* hub_list;      // rows a whole block takes, listed by gat_scores_kernel (order arbitrary; no result depends on it)
     int32_t* hub_count;
 };
 
-constexpr int kGatHubEntries = 512;     // rows with at least this many entries are taken by a whole block
+constexpr int kGatHubEntries = 128;     // rows with at least this many entries are taken by a whole block
 
-// s_u = <a_src, p_u>, t_u = <a_dst, p_u> per head; one warp per node.
+// s_u = <a_src, p_u>, t_u = <a_dst, p_u> per head; one warp per node.  The warp also lists its node
+// if the node's row is long enough for a whole block.
 __global__ void __launch_bounds__(kAggThreads) gat_scores_kernel(GatArgs a) {
     const int lane = threadIdx.x & 31;
     const int64_t u = blockIdx.x * (int64_t)kAggWarps + (threadIdx.x >> 5);
     if (u >= a.n) return;
+    if (lane == 0 && a.rowptr[u + 1] - a.rowptr[u] + (a.self_loop ? 1 : 0) >= kGatHubEntries)
+        a.hub_list[atomicAdd(a.hub_count, 1)] = (int32_t)u;
     const float* row = a.p + u * a.ldp;
     for (int h = 0; h < a.heads; ++h) {
         float ss = 0.f, tt = 0.f;
@@ -668,83 +671,78 @@ __device__ __forceinline__ void gat_accumulate(const GatArgs& a, int64_t v, int6
     }
 }
 
-// One warp per destination v (rows of kGatHubEntries entries or more are left to gat_hub_kernel).
-template <int NC>
-__global__ void __launch_bounds__(kAggThreads) gat_rows_kernel(GatArgs a) {
-    __shared__ float p_s[kAggWarps][kWarp][kGatMaxHeads];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t v = blockIdx.x * (int64_t)kAggWarps + warp;
-    if (v >= a.n) return;
-    const int64_t beg = a.rowptr[v];
-    const int64_t deg = a.rowptr[v + 1] - beg;
-    const int64_t total = deg + (a.self_loop ? 1 : 0);
-    if (total >= kGatHubEntries && a.hub_list) {      // a whole block takes this row
-        if (lane == 0) a.hub_list[atomicAdd(a.hub_count, 1)] = (int32_t)v;
-        return;
-    }
-
-    float m[kGatMaxHeads], l[kGatMaxHeads], tv[kGatMaxHeads];
-#pragma unroll
-    for (int h = 0; h < kGatMaxHeads; ++h) {
-        m[h] = -INFINITY;
-        l[h] = 0.f;
-        tv[h] = h < a.heads ? a.t[v * a.heads + h] : 0.f;
-    }
-    float acc[NC];
-    int head_of[NC];
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-        acc[c] = 0.f;
-        const int col = c * kWarp + lane;
-        head_of[c] = col < a.dim ? col / a.head_dim : 0;
-    }
-
-    gat_accumulate<NC>(a, v, beg, deg, total, 0, kWarp, lane, warp, p_s, tv, head_of, m, l, acc);
-#pragma unroll
-    for (int c = 0; c < NC; ++c) {
-        const int col = c * kWarp + lane;
-        if (col >= a.dim) continue;
-        float den = 1.f;
-#pragma unroll
-        for (int h = 0; h < kGatMaxHeads; ++h) if (h == head_of[c]) den = l[h];
-        const float val = total > 0 ? acc[c] / den : 0.f;
-        if (a.out) a.out[v * a.ldout + col] = val;
-        if (a.out16) a.out16[v * a.ldout16 + col] = f32_to_bf16(val);
-    }
-}
-
-
-// One block per hub row (listed by gat_rows_kernel): warp w takes the chunks w, w + 8, ... of the row
-// with a soft-max state of its own; the eight states are then merged in warp order
+// Blocks [0, hub_blocks): one block per listed hub row at a time.  Warp w takes the trips w, w + 8, ...
+// of the row with a soft-max state of its own; the eight states are then merged in warp order
 //   M = max m_w,  L = sum l_w e^(m_w - M),  Z = sum acc_w e^(m_w - M) / L,
 // so the result does not depend on scheduling (it differs from the one-warp order only in rounding).
+// Blocks from hub_blocks on: one warp per destination v, rows of fewer than kGatHubEntries entries.
+// The hub blocks come first in launch order, so the longest rows start ahead of the short ones.
 template <int NC>
-__global__ void __launch_bounds__(kAggThreads) gat_hub_kernel(GatArgs a) {
+__global__ void __launch_bounds__(kAggThreads) gat_rows_kernel(GatArgs a, int hub_blocks) {
     __shared__ float p_s[kAggWarps][kWarp][kGatMaxHeads];
     __shared__ float sm_m[kAggWarps][kGatMaxHeads], sm_l[kAggWarps][kGatMaxHeads];
     __shared__ float sm_acc[kAggWarps][NC * kWarp];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int n_hubs = *a.hub_count;
-    for (int hub = blockIdx.x; hub < n_hubs; hub += gridDim.x) {
-        const int64_t v = a.hub_list[hub];
+    const bool hub_block = (int)blockIdx.x < hub_blocks;
+    const int n_hubs = hub_block ? *a.hub_count : 0;
+    int hub = blockIdx.x;
+    int64_t v = hub_block ? -1 : (int64_t)(blockIdx.x - hub_blocks) * kAggWarps + warp;
+    if (!hub_block && v >= a.n) return;
+
+    float m[kGatMaxHeads], l[kGatMaxHeads], tv[kGatMaxHeads];
+    float acc[NC];
+    int head_of[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int col = c * kWarp + lane;
+        head_of[c] = col < a.dim ? col / a.head_dim : 0;
+    }
+
+    if (!hub_block) {
         const int64_t beg = a.rowptr[v];
         const int64_t deg = a.rowptr[v + 1] - beg;
         const int64_t total = deg + (a.self_loop ? 1 : 0);
-        float m[kGatMaxHeads], l[kGatMaxHeads], tv[kGatMaxHeads];
+        if (total >= kGatHubEntries) return;                 // a hub block takes this row
 #pragma unroll
         for (int h = 0; h < kGatMaxHeads; ++h) {
             m[h] = -INFINITY;
             l[h] = 0.f;
             tv[h] = h < a.heads ? a.t[v * a.heads + h] : 0.f;
         }
-        float acc[NC];
-        int head_of[NC];
+#pragma unroll
+        for (int c = 0; c < NC; ++c) acc[c] = 0.f;
+        gat_accumulate<NC>(a, v, beg, deg, total, 0, kWarp, lane, warp, p_s, tv, head_of, m, l, acc);
 #pragma unroll
         for (int c = 0; c < NC; ++c) {
-            acc[c] = 0.f;
             const int col = c * kWarp + lane;
-            head_of[c] = col < a.dim ? col / a.head_dim : 0;
+            if (col < a.dim) {
+                float val = 0.f;
+                if (total > 0) {
+                    float lh = 1.f;
+#pragma unroll
+                    for (int h = 0; h < kGatMaxHeads; ++h) if (h == head_of[c]) lh = l[h];
+                    val = acc[c] / lh;
+                }
+                if (a.out) a.out[v * a.ldout + col] = val;
+                if (a.out16) a.out16[v * a.ldout16 + col] = f32_to_bf16(val);
+            }
         }
+        return;
+    }
+
+    for (; hub < n_hubs; hub += hub_blocks) {
+        v = a.hub_list[hub];
+        const int64_t beg = a.rowptr[v];
+        const int64_t deg = a.rowptr[v + 1] - beg;
+        const int64_t total = deg + (a.self_loop ? 1 : 0);
+#pragma unroll
+        for (int h = 0; h < kGatMaxHeads; ++h) {
+            m[h] = -INFINITY;
+            l[h] = 0.f;
+            tv[h] = h < a.heads ? a.t[v * a.heads + h] : 0.f;
+        }
+#pragma unroll
+        for (int c = 0; c < NC; ++c) acc[c] = 0.f;
         gat_accumulate<NC>(a, v, beg, deg, total, (int64_t)warp * kWarp, (int64_t)kAggWarps * kWarp, lane, warp, p_s, tv,
                            head_of, m, l, acc);
         if (lane < kGatMaxHeads) {
@@ -763,7 +761,7 @@ __global__ void __launch_bounds__(kAggThreads) gat_hub_kernel(GatArgs a) {
             for (int w = 0; w < kAggWarps; ++w) big = fmaxf(big, sm_m[w][h]);
             float den = 0.f, num = 0.f;
             for (int w = 0; w < kAggWarps; ++w) {
-                const float f = sm_m[w][h] == -INFINITY ? 0.f : expf(sm_m[w][h] - big);     // (a warp without chunks)
+                const float f = sm_m[w][h] == -INFINITY ? 0.f : expf(sm_m[w][h] - big);     // (a warp without trips)
                 den = fmaf(sm_l[w][h], f, den);
                 num = fmaf(sm_acc[w][col], f, num);
             }
@@ -844,11 +842,12 @@ extern "C" int retexo_aggregate(const retexo_csr* g, int32_t type, const float* 
         const unsigned blocks = (unsigned)((n + kAggWarps - 1) / kAggWarps);
         gat_scores_kernel<<<blocks, kAggThreads, 0, st>>>(a);
         const int nc = (dim + kWarp - 1) / kWarp;
-        const unsigned hub_blocks = (unsigned)(2 * n_sm);
-        if (nc <= 1) { gat_rows_kernel<1><<<blocks, kAggThreads, 0, st>>>(a); gat_hub_kernel<1><<<hub_blocks, kAggThreads, 0, st>>>(a); }
-        else if (nc <= 2) { gat_rows_kernel<2><<<blocks, kAggThreads, 0, st>>>(a); gat_hub_kernel<2><<<hub_blocks, kAggThreads, 0, st>>>(a); }
-        else if (nc <= 4) { gat_rows_kernel<4><<<blocks, kAggThreads, 0, st>>>(a); gat_hub_kernel<4><<<hub_blocks, kAggThreads, 0, st>>>(a); }
-        else { gat_rows_kernel<8><<<blocks, kAggThreads, 0, st>>>(a); gat_hub_kernel<8><<<hub_blocks, kAggThreads, 0, st>>>(a); }
+        const int hub_blocks = 3 * n_sm;       // as many as are resident at once; those without a row leave at once
+        const unsigned grid = blocks + (unsigned)hub_blocks;
+        if (nc <= 1) gat_rows_kernel<1><<<grid, kAggThreads, 0, st>>>(a, hub_blocks);
+        else if (nc <= 2) gat_rows_kernel<2><<<grid, kAggThreads, 0, st>>>(a, hub_blocks);
+        else if (nc <= 4) gat_rows_kernel<4><<<grid, kAggThreads, 0, st>>>(a, hub_blocks);
+        else gat_rows_kernel<8><<<grid, kAggThreads, 0, st>>>(a, hub_blocks);
         return launch_status();
     }
 

@@ -152,9 +152,10 @@ def test_gat_random_graphs(heads, dh, self_loop):
 
 @pytest.mark.parametrize("heads,dh", [(4, 16), (8, 32), (1, 7)])
 def test_gat_long_rows_isolated_nodes_and_large_scores(heads, dh):
-    """Rows on both sides of the 512-entry mark, from which a whole block takes a row and merges the
-    soft-max states of its eight warps."""
-    n, rowptr, colidx, _ = wl.degree_ladder_graph([0, 1, 31, 32, 33, 510, 511, 512, 513, 700, 3000], seed=5)
+    """Rows on both sides of the 128-entry mark, from which a whole block takes a row and merges the
+    soft-max states of its eight warps (some of them without a trip below 256 entries)."""
+    n, rowptr, colidx, _ = wl.degree_ladder_graph([0, 1, 31, 32, 33, 126, 127, 128, 129, 160, 255, 256, 257, 700, 3000],
+                                                  seed=5)
     rng = np.random.default_rng(5)
     p = (rng.standard_normal((n, heads * dh)) * 3).astype(np.float32)
     if heads * dh < 16:
