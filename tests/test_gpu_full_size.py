@@ -121,3 +121,29 @@ def test_whole_run_properties_on_the_products_shaped_graph():
     for m in range(w.K):
         v = a["val_correct"][m].astype(np.int64)
         assert a["best_iter"][m] == int(np.argmax(v)) + 1
+
+
+def test_gat_aggregation_on_the_products_shaped_graph():
+    """The fused GAT kernel far outside L2 (2.4 M rows of 64 columns, 124 M entries, tens of thousands
+    of rows long enough to be taken by whole blocks): sampled destination rows, the longest included,
+    against the checker; two runs give the same bits although the list of long rows is built with
+    atomics in arbitrary order."""
+    from paper_2302_13053_b200 import binding as B
+    w = config(5)
+    heads, dh = 4, 16
+    rng = np.random.default_rng(11)
+    p_host = rng.standard_normal((w.n_nodes, heads * dh), dtype=np.float32)
+    gat = dict(heads=heads, head_dim=dh, a_src=(rng.standard_normal((heads, dh)) * 0.5).astype(np.float32),
+               a_dst=(rng.standard_normal((heads, dh)) * 0.5).astype(np.float32), negative_slope=0.2, add_self_loop=1)
+    g = dict(gat)
+    g["a_src"], g["a_dst"] = torch.from_numpy(gat["a_src"]), torch.from_numpy(gat["a_dst"])
+    rp, ci, p = dev(w.rowptr), dev(w.colidx), dev(p_host)
+    out, _ = B.retexo_aggregate(oracle.GAT, rp, ci, p, dim=heads * dh, gat=g, want_f32=True)
+    again, _ = B.retexo_aggregate(oracle.GAT, rp, ci, p, dim=heads * dh, gat=g, want_f32=True)
+    torch.cuda.synchronize()
+    assert torch.equal(out, again)
+    rows = sampled_rows(w)
+    assert (np.diff(w.rowptr)[rows] >= 128).sum() >= 24 and (np.diff(w.rowptr)[rows] < 127).sum() >= 8
+    ref = oracle.aggregate(oracle.GAT, w.rowptr, w.colidx, p_host, rows=rows, gat=gat)
+    got = out[torch.from_numpy(rows).cuda()].cpu().numpy()
+    assert_rows_close(got, ref, what="gat on " + w.name)
