@@ -305,7 +305,8 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
               weights: List[Dict[str, np.ndarray]], gat: Optional[Dict] = None,
               optimizer: int = ADAM, round_bf16: bool = True, eval_every: int = 1,
               part=None, n_parts: int = 0, forced_best_iter: Optional[Sequence[int]] = None,
-              dropout: float = 0.0, dropout_seed: int = 0) -> Dict:
+              dropout: float = 0.0, dropout_seed: int = 0,
+              forced_theta: Optional[Sequence[np.ndarray]] = None) -> Dict:
     """Lazy message passing (Section 3.1): for each layer m = 1..K, one
     message-passing round builds the layer's inputs, the layer (with a
     temporary classifier unless it is the last) is trained alone for R
@@ -316,7 +317,18 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
     round instead of the checker's own choice.  The choice is an arg-max over
     floating-point results, so two correct implementations may pick different
     iterates on a flat validation curve; fixing it lets everything downstream
-    of the choice be compared."""
+    of the choice be compared.
+
+    forced_theta (a test hook): K flat parameter vectors; round m still trains
+    its own model from the given initial weights (losses, validation counts and
+    its own kept iterate are reported as usual), but the representations handed
+    to round m + 1, the final logits and `test_correct_best` come from
+    forced_theta[m - 1].  An optimiser turns rounding-level differences into
+    full-size steps on weights whose gradient is near zero, so after R
+    iterations two correct implementations hold slightly different weights and
+    every later round would start from different inputs; with the weights of the
+    implementation under test forced in, each round is compared from the same
+    starting point."""
     labels = np.ascontiguousarray(labels, dtype=np.int32)
     q = _f32(features)
     y_tr, y_va, y_te = labels[train_idx], labels[val_idx], labels[test_idx]
@@ -359,10 +371,15 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
                 elif c > best_correct:
                     best, best_correct, best_iter = model.copy(), c, r
         last_test = model.embed(x, row_idx=test_idx, y=y_te, want_logits=False)["correct"]
+        own_best = best
+        if forced_theta is not None:
+            best = model.copy()
+            best.theta = np.ascontiguousarray(forced_theta[m - 1], dtype=np.float64).copy()
+            assert best.theta.shape == model.theta.shape
         best_test = best.embed(x, row_idx=test_idx, y=y_te, want_logits=False)["correct"]
         rd = dict(round=m, losses=np.asarray(losses), val_correct=np.asarray(val_hist),
                   best_iter=best_iter, best_val_correct=best_correct,
-                  test_correct_best=best_test, test_correct_last=last_test, model=best, x=x)
+                  test_correct_best=best_test, test_correct_last=last_test, model=best, own_model=own_best, x=x)
         if m < K:
             q = best.embed(x, want_hidden=True, want_logits=False)["hidden"]
             rd["q_out"] = q

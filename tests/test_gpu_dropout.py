@@ -87,28 +87,27 @@ def lmp_both(w, R, p, seed, eval_every):
     return prob.results(), ws
 
 
-@pytest.mark.parametrize("idx,scale,R,eval_every", [(1, 1.0, 12, 1), (2, 1.0, 12, 12), (4, 0.01, 10, 1)])
+@pytest.mark.parametrize("idx,scale,R,eval_every", [(1, 1.0, 12, 1), (2, 1.0, 12, 12), (4, 0.05, 10, 1)])
 def test_k_round_run_with_dropout_tracks_the_checker(idx, scale, R, eval_every):
     """The whole loop with dropout 0.5: with validation every iteration the iterations are replayed
     from a recorded graph and the update number that keys the mask lives on the device, so the first
     iterations' losses (same weights up to rounding, same masks) pin that bookkeeping."""
     from paper_2302_13053_b200 import workloads as wl
     w = wl.make_config(idx, scale=scale)
-    if idx == 4:
-        w.lr *= 0.1
     p, seed = 0.5, 0xfeedfacecafebeef
     got, ws = lmp_both(w, R, p, seed, eval_every)
     ref = oracle.lmp_train(w.aggr, w.K, R, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
                            w.train_idx, w.val_idx, w.test_idx, ws, part=w.part, n_parts=w.n_parts,
                            eval_every=eval_every, forced_best_iter=list(got["best_iter"]), dropout=p,
-                           dropout_seed=seed)
+                           dropout_seed=seed, forced_theta=got["theta_best"])
     rl, gl = ref["rounds"][0]["losses"], got["loss_history"][0]
     assert abs(gl[0] - rl[0]) <= 1e-3 * max(1.0, rl[0]), (gl[0], rl[0])
     assert np.abs(gl[:4] - rl[:4]).max() <= 1e-2 * max(1.0, rl[:4].max()), (gl[:4], rl[:4])
     for m, rd in enumerate(ref["rounds"]):
         g = got["loss_history"][m]
         assert np.isfinite(g).all()
-        assert np.abs(g - rd["losses"]).max() <= 0.15 * max(1.0, rd["losses"].max()), (m, np.abs(g - rd["losses"]).max())
+        # (every round starts from the GPU's kept weights on both sides, at the configuration's own learning rate)
+        assert np.abs(g - rd["losses"]).max() <= 2e-2 * max(1.0, rd["losses"].max()), (m, np.abs(g - rd["losses"]).max())
     # the run without dropout is a different run, the same seed the same bits, another seed other masks
     plain, _ = lmp_both(w, R, 0.0, seed, eval_every)
     assert np.abs(plain["loss_history"][0] - gl).max() > 1e-3

@@ -96,6 +96,71 @@ def test_one_training_iteration_of_the_reddit_shaped_round_one():
     assert np.abs(gpu.theta.cpu().numpy() - given.theta).max() <= 2e-6 * max(1.0, np.abs(given.theta).max())
 
 
+def round_inputs(w, m):
+    """Model input of round m at full size in the benchmark's layout: round 1 aggregates the features,
+    later rounds a seeded stand-in for the previous round's output (non-negative, as a ReLU leaves it)."""
+    from paper_2302_13053_b200 import binding as B
+    rd = w.round_dims()[m - 1]
+    n, d = w.n_nodes, rd["rep_dim"]
+    ld = (d + 31) // 32 * 32
+    q = torch.zeros((n, ld), dtype=torch.float32, device="cuda")
+    if m == 1:
+        q[:, :d] = dev(w.features)
+    else:
+        g = torch.Generator(device="cuda")
+        g.manual_seed(100 * m + d)
+        q[:, :d] = torch.randn((n, d), generator=g, device="cuda").clamp_(min=0)
+    _, x16 = B.retexo_aggregate(w.aggr, dev(w.rowptr), dev(w.colidx), q, dim=d, want_f32=False, want_bf16=True)
+    return rd, x16
+
+
+@pytest.mark.parametrize("idx,m", [(4, 2), (4, 3), (5, 1), (5, 2), (5, 3)])
+def test_one_training_iteration_and_emission_at_full_size(idx, m):
+    """The shapes of the two large configurations that the first-round test above does not cover: one
+    whole training iteration on all train rows (loss, gradient, update) and the emission of sampled
+    rows, each against the checker on the very batch the GPU works on."""
+    from paper_2302_13053_b200 import binding as B
+    from gpu_util import assert_logits_close
+    w = config(idx)
+    rd, x16 = round_inputs(w, m)
+    d_in, H, O = rd["d_in"], rd["hidden"], w.n_classes
+    tr = dev(w.train_idx)
+    xtr, xtr_t = B.retexo_pack_rows(x16, tr, dim=d_in, transpose=True, ones_row=True)
+    y = w.labels[w.train_idx]
+    wt = wl.initial_weights(w)[m - 1]
+    gpu = B.Mlp(d_in, H, O, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
+    ref = oracle.Mlp(d_in, H, O, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr, round_bf16=True)
+    x_host = xtr[:, :d_in].float().cpu().numpy()
+    given = ref.copy()
+    rl, rg = ref.train_step(x_host, y, return_grad=True)
+    gl, gg = B.retexo_mlp_train_step(gpu, xtr, dev(y), x_t=xtr_t, return_grad=True)
+    assert abs(gl.item() - rl) <= 2e-4 * max(1.0, abs(rl)), (gl.item(), rl)
+    gg = gg.cpu().numpy().astype(np.float64)
+    err, scale = np.abs(gg - rg), np.abs(rg).max()
+    assert err.max() <= 5e-3 * scale + 1e-7, (err.max(), scale)
+    assert np.median(err) <= 2e-5 * scale
+    given.apply_update(gg)
+    assert np.abs(gpu.theta.cpu().numpy() - given.theta).max() <= 2e-6 * max(1.0, np.abs(given.theta).max())
+    del xtr, xtr_t, x_host
+    # emission over all rows with the updated weights, as the K-round run calls it; 4096 sampled rows checked
+    rows = np.sort(np.random.default_rng(m).choice(w.n_nodes, 4096, replace=False))
+    out = B.retexo_embed(gpu, x16, want_hidden=H > 0, want_logits=True, want_pred=True)
+    sel = torch.from_numpy(rows).cuda()
+    xs = x16[sel][:, :d_in].float().cpu().numpy()
+    ref.theta = gpu.theta.cpu().numpy().astype(np.float64)
+    r = ref.embed(xs, want_hidden=H > 0)
+    lg = out["logits"][sel].cpu().numpy()
+    assert_logits_close(lg, r["logits"], rel=5e-3, what="vs bf16-operand checker")
+    exact = ref.copy()
+    exact.round_bf16 = False
+    assert_logits_close(lg, exact.embed(xs)["logits"], rel=2e-2, what="vs unrounded checker")
+    if H > 0:
+        assert_logits_close(out["hidden"][sel].cpu().numpy(), r["hidden"], rel=1e-3, what="hidden")
+    srt = np.sort(r["logits"], axis=1)
+    clear = (srt[:, -1] - srt[:, -2]) > 1e-2 * np.abs(r["logits"]).max(axis=1)
+    np.testing.assert_array_equal(out["pred"][sel].cpu().numpy()[clear], r["pred"][clear])
+
+
 def test_whole_run_properties_on_the_products_shaped_graph():
     """At a size the checker cannot train on in reasonable time: the K-round run must be repeatable
     bit for bit, count every edge as a message, reduce the loss in every round, and beat chance."""

@@ -1,14 +1,20 @@
 """The K-round loop on the device (retexo_lmp_train) against the CPU checker's
-loop: counts exact, first-iteration losses tight, loss curves and accuracy
-within the stated bounds (test accuracy within 0.5 points)."""
+loop: counts exact; the emitted logits element by element against the checker's
+aggregate / embed chain on the kept weights; loss curves, validation and test
+counts round by round from the same start; test accuracy within 0.5 points."""
 import numpy as np
 import pytest
 import torch
 
 import oracle
 from paper_2302_13053_b200 import workloads as wl
+from gpu_util import assert_logits_close
 
 pytestmark = pytest.mark.gpu
+
+# Loss curves of a round that starts from the same weights and the same inputs on both sides: what is left
+# is fp32-versus-fp64 arithmetic carried through R optimiser steps.
+CURVE_TOL = 2e-2
 
 
 def run_both(w, R, host=False, eval_every=1, force=False):
@@ -37,46 +43,108 @@ def check_counts(ref, got):
     np.testing.assert_array_equal(got["counts"]["bytes_per_round"], ref["counts"]["bytes_per_round"])
 
 
-@pytest.mark.parametrize("idx,scale,R", [(1, 1.0, 30), (2, 1.0, 25), (3, 1.0, 30), (4, 0.01, 12), (5, 0.004, 12)])
-def test_last_iterate_runs_track_the_checker_round_by_round(idx, scale, R):
-    """With validation only at the last iteration both sides keep the same iterate, so every
-    round starts from comparable representations and the loss curves can be compared directly."""
+def oracle_chain(w, ws, thetas, round_bf16):
+    """What the K-round run emits, recomputed by the checker without any training: the raw features
+    go through aggregate -> per-node model with the given weights -> aggregate -> ... (Section 3.1:
+    the kept layer's output representations are the next round's inputs, the classifier dropped)."""
+    q = w.features
+    out = None
+    for m, (rd, wt) in enumerate(zip(w.round_dims(), ws)):
+        if w.aggr == wl.GAT:
+            hd = w.heads * w.head_dim
+            proj = oracle.Mlp(q.shape[1], 0, hd, wt["w_att"], np.zeros(hd), round_bf16=round_bf16)
+            g = dict(heads=w.heads, head_dim=w.head_dim, negative_slope=w.negative_slope, add_self_loop=1,
+                     a_src=wt["a_src"], a_dst=wt["a_dst"])
+            x = oracle.aggregate(oracle.GAT, w.rowptr, w.colidx, proj.embed(q)["logits"], gat=g)
+        else:
+            x = oracle.aggregate(w.aggr, w.rowptr, w.colidx, q)
+        model = oracle.Mlp(rd["d_in"], rd["hidden"], w.n_classes, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"),
+                           round_bf16=round_bf16)
+        model.theta = np.ascontiguousarray(thetas[m], dtype=np.float64)
+        if rd["hidden"] > 0:
+            q = model.embed(x, want_hidden=True, want_logits=False)["hidden"]
+        else:
+            out = model.embed(x, want_logits=True)
+    return out["logits"], out["pred"]
+
+
+@pytest.mark.parametrize("idx,scale,R", [(1, 1.0, 30), (2, 1.0, 25), (3, 1.0, 30), (4, 0.1, 10), (5, 0.05, 10)])
+def test_emitted_logits_match_the_checkers_chain_on_the_kept_weights(idx, scale, R):
+    """The weights the run kept in every round, pushed through the checker's own aggregate / embed
+    chain from the raw features, must reproduce the logits the run emits element by element at the
+    stated bf16 tolerance (no training happens on the checker's side, so nothing can drift)."""
+    from paper_2302_13053_b200 import binding as B
     w = wl.make_config(idx, scale=scale)
-    if idx == 4:
-        # At this configuration's lr = 0.01 the first dozen Adam steps on the unnormalised features
-        # overshoot (the loss rises before it falls) and the trajectory amplifies rounding-level
-        # differences, so a short run is compared at a tenth of it.
-        w.lr *= 0.1
-    check_last_iterate_run(w, R)
+    ws = wl.initial_weights(w)
+    prob = B.LmpProblem(w.aggr, w.K, R, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
+                        w.train_idx, w.val_idx, w.test_idx, ws, part=w.part, n_parts=w.n_parts, heads=w.heads,
+                        head_dim=w.head_dim, negative_slope=w.negative_slope)
+    B.retexo_lmp_train(prob)
+    torch.cuda.synchronize()
+    got = prob.results()
+    assert all(np.abs(t).max() > 0 for t in got["theta_best"])
+    lg = got["final_logits"]
+    np.testing.assert_array_equal(got["final_pred"], lg.argmax(1))
+    for round_bf16 in (True, False):
+        rl, rp = oracle_chain(w, ws, got["theta_best"], round_bf16)
+        # Against the checker under the same operand-rounding contract: the stated 2e-2.  Against the
+        # checker that rounds nothing, each of the K per-node models in the chain (and, for GAT, each
+        # projection) adds its own bf16 operand rounding on top of what it inherits, so the stated
+        # per-model 2e-2 is allowed once per round.
+        rel = 2e-2 if round_bf16 else 2e-2 * w.K
+        assert_logits_close(lg, rl, rel=rel, what="%s, checker %s operand rounding" % (
+            w.name, "with" if round_bf16 else "without"))
+        srt = np.sort(rl, axis=1)
+        rms = float(np.sqrt(np.mean(rl.astype(np.float64) ** 2)))
+        clear = (srt[:, -1] - srt[:, -2]) > 2 * rel * np.maximum(np.abs(rl).max(axis=1), rms)
+        np.testing.assert_array_equal(got["final_pred"][clear], rp[clear])
+        hits = int((rp[w.test_idx] == w.labels[w.test_idx]).sum())
+        unclear = int((~clear[w.test_idx]).sum())
+        assert abs(int(got["test_correct"][-1]) - hits) <= unclear
+
+
+@pytest.mark.parametrize("idx,scale,R", [(1, 1.0, 30), (2, 1.0, 25), (3, 1.0, 30), (4, 0.05, 20), (5, 0.01, 20)])
+def test_every_round_tracks_the_checker_from_the_same_start(idx, scale, R):
+    """Validation only at the last iteration, so both sides keep the last iterate; the checker hands
+    the GPU's kept weights to the next round (`forced_theta`), so every round trains on the same
+    inputs on both sides, each at the configuration's own learning rate, and loss curves, validation
+    and test counts can be compared round by round."""
+    check_rounds_from_the_same_start(wl.make_config(idx, scale=scale), R)
 
 
 def test_max_pooling_rounds_track_the_checker():
     """The K-round loop with the max-pooling aggregator of Section 2.2 in place of the mean."""
     w = wl.make_config(2)
     w.aggr = wl.SAGE_MAX
-    check_last_iterate_run(w, 25)
+    check_rounds_from_the_same_start(w, 25)
 
 
-def check_last_iterate_run(w, R):
-    ref, got = run_both(w, R, eval_every=R)
+def check_rounds_from_the_same_start(w, R):
+    from paper_2302_13053_b200 import binding as B
+    ws = wl.initial_weights(w)
+    gat = dict(heads=w.heads, head_dim=w.head_dim, negative_slope=w.negative_slope,
+               add_self_loop=1) if w.aggr == wl.GAT else None
+    prob = B.LmpProblem(w.aggr, w.K, R, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
+                        w.train_idx, w.val_idx, w.test_idx, ws, part=w.part, n_parts=w.n_parts, heads=w.heads,
+                        head_dim=w.head_dim, negative_slope=w.negative_slope, eval_every=R)
+    B.retexo_lmp_train(prob)
+    torch.cuda.synchronize()
+    got = prob.results()
+    ref = oracle.lmp_train(w.aggr, w.K, R, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
+                           w.train_idx, w.val_idx, w.test_idx, ws, gat=gat, part=w.part, n_parts=w.n_parts,
+                           eval_every=R, forced_theta=got["theta_best"])
     check_counts(ref, got)
     n_val, n_test = len(w.val_idx), len(w.test_idx)
     for m, rd in enumerate(ref["rounds"]):
         gl, rl = got["loss_history"][m], rd["losses"]
-        tol0 = 1e-3 if m == 0 else 2e-2          # round 1: same weights and inputs; later: after R fp32 vs fp64 steps
-        assert abs(gl[0] - rl[0]) <= tol0 * max(1.0, rl[0]), (m, gl[0], rl[0])
-        assert np.abs(gl - rl).max() <= 0.15 * max(1.0, rl.max()), (m, np.abs(gl - rl).max())
+        assert abs(gl[0] - rl[0]) <= 1e-3 * max(1.0, rl[0]), (m, gl[0], rl[0])     # same weights, same inputs
+        assert np.abs(gl - rl).max() <= CURVE_TOL * max(1.0, rl.max()), (m, np.abs(gl - rl).max(), rl.max())
         assert got["best_iter"][m] == R == rd["best_iter"]
-        assert abs(int(got["best_val_correct"][m]) - rd["best_val_correct"]) <= max(3, 0.03 * n_val)
-        assert abs(int(got["test_correct"][m]) - rd["test_correct_best"]) <= max(3, 0.02 * n_test)
+        assert abs(int(got["best_val_correct"][m]) - rd["best_val_correct"]) <= max(2, 0.01 * n_val)
+        # the checker's own last iterate and the GPU's, both on the test rows of the same inputs
+        assert abs(int(got["test_correct"][m]) - rd["test_correct_last"]) <= max(2, 0.01 * n_test)
         assert got["test_correct"][m] == got["test_correct_last"][m]
-    lg, rl = got["final_logits"], ref["rounds"][-1]["logits"]
-    srt = np.sort(rl, axis=1)
-    clear = (srt[:, -1] - srt[:, -2]) > 0.10 * np.abs(rl).max(axis=1)
-    if clear.sum() >= 50:               # (a short run on weak features may leave no row with a clear margin)
-        agree = (got["final_pred"][clear] == ref["rounds"][-1]["pred"][clear]).mean()
-        assert agree > 0.97, agree      # after K rounds of fp32-vs-fp64 training on every earlier layer
-    assert abs(got["test_acc"] - ref["test_acc"]) <= 0.005 + 2.0 / n_test, (got["test_acc"], ref["test_acc"])
+    assert abs(got["test_acc"] - ref["test_acc_last"]) <= 0.005 + 1.0 / n_test, (got["test_acc"], ref["test_acc_last"])
 
 
 @pytest.mark.parametrize("idx,scale,R", [(1, 1.0, 100), (2, 1.0, 100), (3, 1.0, 100)])

@@ -68,3 +68,20 @@ def test_forced_iterate_hook_keeps_the_named_iterate():
     other = run(w, 8, forced_best_iter=[8, 8, 8])
     assert [r["best_iter"] for r in other["rounds"]] == [8, 8, 8]
     assert other["rounds"][0]["test_correct_best"] == other["rounds"][0]["test_correct_last"]
+
+
+def test_forced_weights_hook_feeds_the_given_weights_forward_and_leaves_the_training_alone():
+    w = wl.make_config(2, scale=0.05)
+    free = run(w, 6, eval_every=6)
+    own = [r["model"].theta for r in free["rounds"]]
+    same = run(w, 6, eval_every=6, forced_theta=own)
+    np.testing.assert_array_equal(free["rounds"][-1]["logits"], same["rounds"][-1]["logits"])
+    # other weights in round 1: round 1's own training is untouched, everything downstream moves
+    bumped = [t.copy() for t in own]
+    bumped[0] = bumped[0] * 1.5
+    other = run(w, 6, eval_every=6, forced_theta=bumped)
+    np.testing.assert_array_equal(other["rounds"][0]["losses"], free["rounds"][0]["losses"])
+    np.testing.assert_array_equal(other["rounds"][0]["own_model"].theta, own[0])
+    np.testing.assert_array_equal(other["rounds"][0]["model"].theta, bumped[0])
+    assert np.abs(other["rounds"][1]["x"] - free["rounds"][1]["x"]).max() > 1e-3
+    assert abs(other["rounds"][1]["losses"][0] - free["rounds"][1]["losses"][0]) > 1e-6
