@@ -336,8 +336,12 @@ __global__ void __launch_bounds__(kCntThreads) count_big_rows_kernel(CountArgs a
     }
 }
 
+// The widths of the K rounds travel in the kernel's arguments (K <= 64), so the call makes no copy from the
+// caller's host array that could outlive it.
+struct RoundDimsArg { int32_t d[64]; };
+
 __global__ void count_finalize_kernel(const unsigned long long* cross_acc, const unsigned long long* pairs_acc,
-                                      const unsigned long long* bad_part, int32_t K, const int32_t* dims, int32_t elem_bytes,
+                                      const unsigned long long* bad_part, int32_t K, const RoundDimsArg dims, int32_t elem_bytes,
                                       uint64_t* cross_edges, uint64_t* boundary_pairs,
                                       uint64_t* bytes_per_round, uint64_t* bytes_total) {
     if (blockIdx.x != 0 || threadIdx.x != 0) return;
@@ -353,7 +357,7 @@ __global__ void count_finalize_kernel(const unsigned long long* cross_acc, const
     if (boundary_pairs) *boundary_pairs = bp;
     uint64_t tot = 0;
     for (int m = 0; m < K; ++m) {
-        const uint64_t b = bp * (uint64_t)dims[m] * (uint64_t)elem_bytes;
+        const uint64_t b = bp * (uint64_t)dims.d[m] * (uint64_t)elem_bytes;
         if (bytes_per_round) bytes_per_round[m] = b;
         tot += b;
     }
@@ -409,7 +413,6 @@ extern "C" size_t retexo_cross_partition_workspace_size(int64_t n_nodes, int64_t
     if (n_nodes < 0 || n_parts <= 0) return 0;
     Sizer s;
     s.take<unsigned long long>(32);                       // accumulators
-    s.take<int32_t>(64);                                  // dims copy
     if (n_parts > kBitmapParts) {
         s.take<int32_t>((size_t)n_nodes);                 // long-row list
         s.take<int32_t>(64);
@@ -436,7 +439,8 @@ extern "C" int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* 
 
     Arena ws(workspace, workspace_bytes);
     unsigned long long* acc = ws.take<unsigned long long>(32);
-    int32_t* dims_dev = ws.take<int32_t>(64);
+    RoundDimsArg dims_arg{};
+    for (int m = 0; m < K; ++m) dims_arg.d[m] = dims[m];
     CountArgs a;
     a.n = g->n_nodes; a.rowptr = g->rowptr; a.colidx = g->colidx; a.part = part; a.n_parts = n_parts;
     a.cross_edges = acc; a.pairs = acc + 1; a.bad_part = acc + 2; a.next_row = acc + 4;
@@ -446,7 +450,6 @@ extern "C" int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* 
     a.big_list = nullptr; a.big_count = nullptr; a.big_bitmaps = nullptr; a.words_per_bitmap = 0;
 
     RETEXO_CUDA_TRY(cudaMemsetAsync(acc, 0, 32 * sizeof(unsigned long long), st));
-    if (K > 0) RETEXO_CUDA_TRY(cudaMemcpyAsync(dims_dev, dims, sizeof(int32_t) * K, cudaMemcpyHostToDevice, st));
     if (send_per_part) RETEXO_CUDA_TRY(cudaMemsetAsync(send_per_part, 0, sizeof(uint64_t) * (size_t)n_parts, st));
     if (recv_per_part) RETEXO_CUDA_TRY(cudaMemsetAsync(recv_per_part, 0, sizeof(uint64_t) * (size_t)n_parts, st));
 
@@ -475,7 +478,7 @@ extern "C" int retexo_cross_partition_bytes(const retexo_csr* g, const int32_t* 
             count_big_rows_kernel<<<kBigRowBlocks, kCntThreads, 0, st>>>(a);
         }
     }
-    count_finalize_kernel<<<1, 32, 0, st>>>(acc, acc + 1, acc + 2, K, dims_dev, elem_bytes, cross_edges, boundary_pairs,
+    count_finalize_kernel<<<1, 32, 0, st>>>(acc, acc + 1, acc + 2, K, dims_arg, elem_bytes, cross_edges, boundary_pairs,
                                             bytes_per_round, bytes_total);
     return launch_status();
 }

@@ -829,14 +829,12 @@ static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensor
     constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + BN * kTcBK * 2) + 1024 + 1024 + EW * kStageBytesPerWarp +
                             (BN == 64 ? (EW / 8) * 4 * 2 * 128 * 4 : 0);
     static_assert(smem <= 227 * 1024, "shared memory budget");
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES, MODE, EW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-            cudaSuccess) {
-            (void)cudaGetLastError();
-            return RETEXO_ERR_CUDA;
-        }
-        configured = true;
+    // (the attribute belongs to the current device's copy of the kernel: set on every launch, which is cheap,
+    //  instead of remembered per process)
+    if (cudaFuncSetAttribute(tc_gemm_kernel<BN, STAGES, MODE, EW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess) {
+        (void)cudaGetLastError();
+        return RETEXO_ERR_CUDA;
     }
     TcKernelArgs g{};
     g.M = t.M; g.N = t.N;

@@ -37,6 +37,15 @@ def test_static_scratch_entry_point_matches_the_workspace_one_twice_in_a_row():
             assert int(got[1]) == ref["boundary_pairs"], call
             assert int(got[2]) == ref["bytes_total"], call
             np.testing.assert_array_equal(got[3:3 + len(dims)], ref["bytes_per_round"])
+        # what the entry point exists for: a further call takes no device memory, neither from the
+        # driver (free bytes of the device unchanged) nor through torch's allocator
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
+        held_before = torch.cuda.memory_allocated()
+        B.retexo_cross_partition_bytes_static(rp, ci, pt, n_parts, dims, out)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+        assert torch.cuda.memory_allocated() == held_before
 
 
 def test_static_scratch_entry_point_rejects_what_does_not_fit():
