@@ -223,7 +223,7 @@ def phase_breakdown(w, ws, R: int, peaks):
                            edges_per_s=e / mean_ms * 1e3, traffic=AGG_DRAM_TRAFFIC.get((w.name, m))))
         # the round's model at its training / validation / full shapes
         model = B.Mlp(rd["d_in"], rd["hidden"], w.n_classes, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
-        xtr, xtr_t = B.retexo_pack_rows(x16, tr, dim=width, transpose=True, ones_row=True)
+        xtr, _ = B.retexo_pack_rows(x16, tr, dim=width, ones=True)
         xva, _ = B.retexo_pack_rows(x16, va, dim=width)
         H, O = rd["hidden"], w.n_classes
         n_tr, n_va = tr.numel(), va.numel()
@@ -249,7 +249,7 @@ def phase_breakdown(w, ws, R: int, peaks):
         need = B.lib().retexo_mlp_train_step_workspace_size(C.c_int32(width), C.c_int32(H), C.c_int32(O),
                                                             C.c_int64(n_tr))
         ws_step = torch.empty(int(need), dtype=torch.uint8, device=dev)
-        mean_ms, best_ms = time_calls(lambda: B.retexo_mlp_train_step(model, xtr, y_tr, x_t=xtr_t, workspace=ws_step), 10)
+        mean_ms, best_ms = time_calls(lambda: B.retexo_mlp_train_step(model, xtr, y_tr, x_has_ones=True, workspace=ws_step), 10)
         phases.append(dict(kernel="mlp_train_step", round=m, calls_per_step=R, ms=mean_ms, best_ms=best_ms,
                            traffic=STEP_DRAM_TRAFFIC.get((w.name, m)),
                            **min_time_roofline(flops_step, bytes_step, mean_ms, peaks)))
@@ -267,7 +267,7 @@ def phase_breakdown(w, ws, R: int, peaks):
             nb = 2.0 * (n * width + width * O) + 4.0 * n * O + 4.0 * n
         phases.append(dict(kernel="embed_all_rows", round=m, calls_per_step=1, ms=mean_ms, best_ms=best_ms,
                            **min_time_roofline(fl, nb, mean_ms, peaks)))
-        del model, xtr, xtr_t, xva, ws_step
+        del model, xtr, xva, ws_step
     part = torch.from_numpy(w.part).to(dev)
     dims = [rd["rep_dim"] for rd in w.round_dims()]
     mean_ms, best_ms = time_calls(lambda: B.retexo_cross_partition_bytes(rp, ci, part, w.n_parts, dims, 4,

@@ -165,13 +165,15 @@ int64_t retexo_theta_size(int32_t d_in, int32_t hidden, int32_t n_classes);
  * src is fp32 (src_is_bf16 = 0) or bf16 (1), row stride ld_src elements;
  * dst is bf16 [n_rows x ld_dst], ld_dst >= dim; columns [dim, ld_dst) are
  * zero-filled.  dst_t (optional) receives the transpose, bf16 [dim x ld_t],
- * ld_t >= n_rows, columns [n_rows, ld_t) zero-filled; with ones_row = 1 it has
- * one more row (index dim) that holds 1 for every batch row: the form
- * retexo_mlp_train_step takes as x_t.  dst may be NULL if only the transpose
- * is wanted.  Needs no workspace. */
+ * ld_t >= n_rows, columns [n_rows, ld_t) zero-filled.  With ones = 1 the batch
+ * carries the all-ones vector as well: column `dim` of dst holds 1 in every row
+ * (ld_dst > dim required) and dst_t has one more row (index dim) that holds 1
+ * for every batch row; the form retexo_mlp_train_step takes with
+ * x_has_ones = 1.  dst may be NULL if only the transpose is wanted.
+ * Needs no workspace. */
 int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld_src, int32_t dim,
                      const int32_t* idx, int64_t n_rows,
-                     void* dst, int64_t ld_dst, void* dst_t, int64_t ld_t, int32_t ones_row, void* stream);
+                     void* dst, int64_t ld_dst, void* dst_t, int64_t ld_t, int32_t ones, void* stream);
 
 size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes,
                                             int64_t n_rows);
@@ -184,12 +186,12 @@ size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_
  *   then one SGD / Adam update of theta in place.
  * x     bf16 [n_rows x ldx]: the batch, one training node per row
  *       (retexo_pack_rows builds it once per round); ldx % 8 == 0 and x
- *       16-byte aligned.
- * x_t   optional bf16 [(d_in + 1) x ld_xt]: the transpose of x with one more
- *       row of ones (retexo_pack_rows with ones_row = 1; ld_xt % 8 == 0,
- *       16-byte aligned).  The weight-gradient product streams it along the
- *       batch; the row of ones makes the bias gradient one more output row.
- *       NULL is allowed: the call then builds it in the workspace, at the
+ *       16-byte aligned.  The weight-gradient products read it as it lies,
+ *       reducing over the rows.
+ * x_has_ones  1: column d_in of x holds 1 in every row (ldx > d_in;
+ *       retexo_pack_rows with ones = 1 writes it).  That column makes the bias
+ *       gradient one more output row of the weight-gradient product.  0: the
+ *       call first copies x into its workspace with that column added, at the
  *       price of one more pass over x per call.
  * y     int32 [n_rows] labels in [0, n_classes).
  * loss_out  device float, the loss before the update (may be NULL).
@@ -197,7 +199,7 @@ size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_
  * Increments model->step (host struct).  n_classes <= 64, hidden <= 512.
  * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED. */
 int retexo_mlp_train_step(retexo_mlp* model,
-                          const void* x, int64_t ldx, const void* x_t, int64_t ld_xt,
+                          const void* x, int64_t ldx, int32_t x_has_ones,
                           const int32_t* y, int64_t n_rows,
                           float* loss_out, float* grad_out,
                           void* workspace, size_t workspace_bytes, void* stream);

@@ -176,29 +176,30 @@ def retexo_aggregate(aggr: int, rowptr: torch.Tensor, colidx: torch.Tensor, q: t
 
 
 def retexo_pack_rows(src: torch.Tensor, idx: Optional[torch.Tensor] = None, dim: Optional[int] = None,
-                     transpose: bool = False, ones_row: bool = False, ld_multiple: int = 64):
+                     transpose: bool = False, ones: bool = False, ld_multiple: int = 64):
     """bf16 batch of the rows src[idx] (all rows if idx is None).  Returns
-    (dst [n_rows, round_up(dim, ld_multiple)], dst_t [dim (+1 with ones_row), round_up(n_rows, ld_multiple)]
-    or None).  The library needs leading dimensions that are multiples of 8; multiples of 64 put
-    every row on a 128-byte line, which its bulk tensor loads prefer."""
+    (dst [n_rows, round_up(dim (+1 with ones), ld_multiple)], dst_t [dim (+1 with ones), round_up(n_rows, ld_multiple)]
+    or None).  With `ones`, column `dim` of dst (and row `dim` of dst_t) holds 1: the form
+    retexo_mlp_train_step takes with x_has_ones.  The library needs leading dimensions that are
+    multiples of 8; multiples of 64 put every row on a 128-byte line, which its bulk tensor loads prefer."""
     assert ld_multiple % 8 == 0 and ld_multiple > 0
     assert src.dtype in (torch.float32, torch.bfloat16) and src.stride(1) == 1
     dim = int(src.shape[1] if dim is None else dim)
     n_rows = int(src.shape[0] if idx is None else idx.numel())
     dev = src.device
-    ld = (dim + ld_multiple - 1) // ld_multiple * ld_multiple
+    ld = (dim + (1 if ones else 0) + ld_multiple - 1) // ld_multiple * ld_multiple
     dst = torch.empty((n_rows, ld), dtype=torch.bfloat16, device=dev)
     dst_t = None
     ld_t = 0
     if transpose:
         ld_t = (n_rows + ld_multiple - 1) // ld_multiple * ld_multiple
-        dst_t = torch.empty((dim + (1 if ones_row else 0), ld_t), dtype=torch.bfloat16, device=dev)
+        dst_t = torch.empty((dim + (1 if ones else 0), ld_t), dtype=torch.bfloat16, device=dev)
     if idx is not None:
         assert idx.dtype == torch.int32
     rc = lib().retexo_pack_rows(_ptr(src), C.c_int32(1 if src.dtype == torch.bfloat16 else 0),
                                 C.c_int64(src.stride(0)), C.c_int32(dim), _ptr(idx), C.c_int64(n_rows),
                                 _ptr(dst), C.c_int64(ld), _ptr(dst_t), C.c_int64(ld_t),
-                                C.c_int32(1 if (ones_row and transpose) else 0), _stream())
+                                C.c_int32(1 if ones else 0), _stream())
     _check(rc, "retexo_pack_rows")
     return dst, dst_t
 
@@ -238,9 +239,10 @@ class Mlp:
         return d
 
 
-def retexo_mlp_train_step(model: Mlp, x: torch.Tensor, y: torch.Tensor, x_t: Optional[torch.Tensor] = None,
+def retexo_mlp_train_step(model: Mlp, x: torch.Tensor, y: torch.Tensor, x_has_ones: bool = False,
                           return_grad: bool = False, workspace: Optional[torch.Tensor] = None):
     """One full-batch iteration on the bf16 batch x [n_rows, ld] with labels y.
+    x_has_ones: column d_in of x holds 1 in every row (retexo_pack_rows(ones=True)).
     Returns the loss before the update as a 0-dim device tensor (and the
     gradient if asked)."""
     assert x.dtype == torch.bfloat16 and y.dtype == torch.int32 and x.stride(1) == 1
@@ -251,8 +253,8 @@ def retexo_mlp_train_step(model: Mlp, x: torch.Tensor, y: torch.Tensor, x_t: Opt
     need = lib().retexo_mlp_train_step_workspace_size(C.c_int32(model.d_in), C.c_int32(model.hidden),
                                                       C.c_int32(model.n_classes), C.c_int64(n_rows))
     ws = workspace if workspace is not None else _workspace(need, dev)
-    rc = lib().retexo_mlp_train_step(C.byref(model.c), _ptr(x), C.c_int64(x.stride(0)), _ptr(x_t),
-                                     C.c_int64(x_t.stride(0) if x_t is not None else 0), _ptr(y),
+    rc = lib().retexo_mlp_train_step(C.byref(model.c), _ptr(x), C.c_int64(x.stride(0)),
+                                     C.c_int32(1 if x_has_ones else 0), _ptr(y),
                                      C.c_int64(n_rows), _ptr(loss), _ptr(grad), _ptr(ws), C.c_size_t(ws.numel()),
                                      _stream())
     _check(rc, "retexo_mlp_train_step")

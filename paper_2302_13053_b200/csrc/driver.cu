@@ -119,7 +119,7 @@ struct LmpBuffers {
     // representations
     float* q[2];
     bf16* x16; bf16* q16; float* proj; bf16* watt16; float* gat_vec; float* gat_stage;
-    bf16 *xtr16, *xval16, *xtr_t16;
+    bf16 *xtr16, *xval16;
     int32_t *y_tr, *y_val, *y_test;
     float *theta, *adam_m, *adam_v, *theta_best;
     unsigned long long *cur_correct, *best_correct, *scratch_u64;
@@ -177,10 +177,10 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
         l.gat_vec = t.template take<float>((size_t)2 * hd);
         l.gat_stage = t.template take<float>((size_t)max_rep * hd + 2 * hd);
     }
-    // training rows, then validation rows; after the round's last iteration the test rows take their place
-    l.xtr16 = t.template take<bf16>((size_t)(n_tr + n_val > n_te ? n_tr + n_val : n_te) * ld16);
+    // training rows, then validation rows, each followed by a column of ones (it carries the bias gradient
+    // through the weight-gradient product); after the round's last iteration the test rows take their place
+    l.xtr16 = t.template take<bf16>((size_t)(n_tr + n_val > n_te ? n_tr + n_val : n_te) * (size_t)round_up(max_din + 1, 64));
     l.xval16 = nullptr;
-    l.xtr_t16 = t.template take<bf16>((size_t)(max_din + 1) * (size_t)round_up(n_tr, 64));
     l.y_tr = t.template take<int32_t>((size_t)n_tr);
     l.y_val = t.template take<int32_t>((size_t)(n_val > 0 ? n_val : 1));
     l.y_test = t.template take<int32_t>((size_t)(n_te > 0 ? n_te : 1));
@@ -359,10 +359,10 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         }
 
         // ---- the round's batches and model state
-        const int64_t ld_xt = round_up(n_tr, 64);
-        RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld16, b.xtr_t16, ld_xt, 1, st));
-        bf16* xval16 = b.xtr16 + (size_t)n_tr * ld16;
-        if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, xval16, ld16, nullptr, 0, 0, st));
+        const int64_t ld_tr = round_up(r.d_in + 1, 64);
+        RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld_tr, nullptr, 0, 1, st));
+        bf16* xval16 = b.xtr16 + (size_t)n_tr * ld_tr;
+        if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, xval16, ld_tr, nullptr, 0, 0, st));
         RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta, in->theta0[m - 1], sizeof(float) * (size_t)nt, cudaMemcpyDefault, st));
         RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta_best, b.theta, sizeof(float) * (size_t)nt, cudaMemcpyDeviceToDevice, st));
         RETEXO_CUDA_TRY(cudaMemsetAsync(b.adam_m, 0, sizeof(float) * (size_t)nt, st));
@@ -413,7 +413,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
             } else if (uniform && it == 2) {
                 bool recorded = false;
                 if (cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed) == cudaSuccess) {
-                    const int rc = mlp_train_step_launch(plan, sb, &model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, loss_slot,
+                    const int rc = mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot,
                                                          nullptr, true, riding, st, &dev);
                     cudaGraph_t graph = nullptr;
                     const cudaError_t ended = cudaStreamEndCapture(st, &graph);
@@ -427,18 +427,18 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
                     RETEXO_CUDA_TRY(cudaGraphLaunch(iteration.exec, st));
                 } else {      // no graph on this stream: plain launches
                     iteration.reset();
-                    RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, loss_slot,
+                    RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot,
                                                      nullptr, true, riding, st, &dev));
                 }
             } else {
-                RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld16, b.xtr_t16, ld_xt, b.y_tr, loss_slot,
+                RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot,
                                                  nullptr, it > 1, riding, st, &dev));
             }
             model.step += 1;
             const bool want = n_val && (it % c.eval_every == 0 || it == c.R);
             pending_it = (want && it < c.R) ? it : 0;
             if (want && it == c.R) {      // the last iterate has no next iteration to ride on
-                RETEXO_TRY(mlp_count_hits_launch(plan, sb, &model, xval16, ld16, n_val, val_hd, b.y_val,
+                RETEXO_TRY(mlp_count_hits_launch(plan, sb, &model, xval16, ld_tr, n_val, val_hd, b.y_val,
                                                  b.cur_correct, st));
                 snapshot_if_better_kernel<<<(unsigned)((nt + 255) / 256), 256, 0, st>>>(
                     b.cur_correct, b.best_correct, b.have_best, b.theta, b.theta_best, nt);

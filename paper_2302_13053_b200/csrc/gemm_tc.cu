@@ -1,5 +1,6 @@
 // Tensor-core GEMM for the dense products of the per-node model on sm_100a:
-//   C[M x N] = A[M x K] * B[N x K]^T,  A and B bf16 with K contiguous,
+//   C[M x N] = A[M x K] * B[N x K]^T,  A and B bf16 with K contiguous, or (the split-K weight-gradient
+//   products, whose reduction runs over the batch) C = A^T B with A [K x M] and B [K x N] row-major;
 //   fp32 accumulation in tensor memory (tcgen05.mma, cta_group::1, M = 128).
 // Operand tiles are brought in by TMA (128-byte swizzle) through a ring of
 // shared-memory stages guarded by mbarriers; one thread issues the MMAs; eight
@@ -7,21 +8,17 @@
 // epilogue (bias / ReLU / bf16 down-cast, soft-max loss, gate, split-K partial).
 // Every wait is bounded: a wait that runs out sets *status and the block
 // tears down in order (outstanding copies awaited, tensor memory freed).
-#include <cuda.h>
-
-#include "common.cuh"
-#include "gemm_tc.h"
 #include <string.h>
+
+#include "gemm_tc.h"
+#include "tc_common.cuh"
 
 namespace retexo {
 
-constexpr int kTcBM = 128;
-constexpr int kTcBK = 64;                  // 64 bf16 = 128 bytes = one swizzle row
 // Threads: warp 0 TMA, warp 1 MMA + tensor-memory owner, then EW epilogue warps (8 or 16).  The epilogues
 // are chains of dependent instructions, so their speed is set by how many warps share an SM's schedulers:
 // with 16 warps a tile's columns are cut four ways (BN >= 128), or (BN = 64, where a row of logits is
 // shared by two threads) two groups of 8 warps take alternate tiles out of four accumulators.
-constexpr uint32_t kSpinLimit = 1u << 26;
 #ifndef TC256_EW
 #define TC256_EW 8
 #define TC256_STAGES 4
@@ -34,105 +31,6 @@ constexpr uint32_t kSpinLimit = 1u << 26;
 #define TC64_EW 16
 #define TC64_STAGES 5
 #endif
-
-__device__ __forceinline__ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait; returns false (and raises *status) if the phase never completes.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, int32_t* status, volatile int* abort_flag) {
-    for (uint32_t i = 0; i < kSpinLimit; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 1023u) == 1023u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    if (status) atomicExch(status, RETEXO_ERR_TIMEOUT);
-    return false;
-}
-
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, int32_t x, int32_t y, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
-}
-
-// Bulk tensor store of a [32 x 32] bf16 box from shared memory (64-byte swizzle) to global memory;
-// the part of the box outside the tensor is not written.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int32_t x, int32_t y) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
-                 ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(smem_src)) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// Wait until all (all but the newest) bulk groups of this thread have finished reading shared memory.
-__device__ __forceinline__ void bulk_wait_read_but_one() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
-__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-// Waits until every bulk group of this thread is complete (the data is in global memory).
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-// Orders this thread's shared-memory writes before later asynchronous-proxy reads of them.
-__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-// Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128
-// bytes, 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((smem_addr & 0x3ffffu) >> 4);          // start address
-    d |= (uint64_t)1 << 16;                                // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)(1024 >> 4) << 32;                      // stride byte offset
-    d |= (uint64_t)1 << 46;                                // descriptor version
-    d |= (uint64_t)2 << 61;                                // 128-byte swizzle
-    return d;
-}
-
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = BN.
-__host__ __device__ constexpr uint32_t make_idesc(int bn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n"
-        " tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// Starts the load of 32 accumulator columns (this warp's 32 lanes) into r; the values may be
-// used only after tmem_ld_wait(r).
-__device__ __forceinline__ void tmem_ld_issue(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr));
-}
-// Waits for the loads in flight.  The registers are passed through as in/out operands so that
-// no use of them can be scheduled ahead of the wait.
-__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.wait::ld.sync.aligned;"
-        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-        :: "memory");
-}
 
 // One block of the counter-based generator Philox4x32-10 (Salmon et al., SC'11), from its definition:
 // ten rounds of (c0,c1,c2,c3) <- (hi(M1 c2)^c1^k0, lo(M1 c2), hi(M0 c0)^c3^k1, lo(M0 c0)), the key raised
@@ -158,7 +56,7 @@ struct TcKernelArgs {
     const float* bias;
     float* out_f32; int64_t ld_f32;
     __nv_bfloat16* out_bf16; int64_t ld_bf16;
-    __nv_bfloat16* out_bf16_t; int64_t ld_t; int ones_row_t;
+    int ones_col;
     const __nv_bfloat16* mask; int64_t ld_mask;
     float gate_scale;
     uint32_t drop_thresh, drop_step, drop_key0, drop_key1; float drop_scale; int64_t drop_rows;
@@ -168,16 +66,15 @@ struct TcKernelArgs {
     int32_t* pred; unsigned long long* correct;
     int64_t n_train; const int32_t* y_eval;       // SOFTMAX_CE: rows >= n_train are evaluated, not trained on
     int32_t* status;
-    int tma_rows, tma_t;          // out_bf16 / out_bf16_t leave through bulk tensor stores (map_rows / map_t)
+    int tma_rows;                 // out_bf16 leaves through bulk tensor stores (map_rows)
 };
 
-// Per-warp staging of one 32 x 32 bf16 block: 32 lines of 64 bytes.  A line is one output row
-// (row-major store) or one output column (transposed store).  The four 16-byte pieces of a line
-// are XOR-swizzled with the line index so that both the fill (one thread per row) and the drain
-// (eight lines of 64 contiguous bytes per instruction) are free of bank conflicts.
+// Per-warp staging of one 32 x 32 bf16 block: 32 lines of 64 bytes, a line being one output row.  The four
+// 16-byte pieces of a line are XOR-swizzled with the line index so that both the fill (one thread per row)
+// and the drain (eight lines of 64 contiguous bytes per instruction) are free of bank conflicts.
 // This is also the 64-byte swizzle of a tensor map (address bits 4-5 XOR bits 7-8), so a block staged in a
-// 1024-byte aligned buffer can leave as one bulk tensor store.  Every warp owns two such blocks: the
-// first stages transposed output, the second row-major output.
+// 1024-byte aligned buffer can leave as one bulk tensor store.  Every warp owns two such blocks (the gated
+// epilogue alternates between them, so that one can be filled while the other's store is in flight).
 constexpr int kStageBlockBytes = 32 * 64;
 constexpr int kStageBytesPerWarp = 2 * kStageBlockBytes;
 __device__ __forceinline__ int stage_piece(int line, int piece) { return piece ^ ((line >> 1) & 3); }
@@ -194,32 +91,7 @@ __device__ __forceinline__ void drain_stage(const uint8_t* stage, __nv_bfloat16*
     }
 }
 
-// Fallback stores (no tensor map).  Transposed: out_t[col][row]; full, aligned blocks are staged and drained
-// in 64-byte runs, ragged ones use guarded element stores.
-__device__ __forceinline__ void store_block_transposed(__nv_bfloat16* out_t, int64_t ld_t, int64_t col0, int64_t n_cols,
-                                                       int64_t row0, int64_t M, const float (&v)[32], uint8_t* stage,
-                                                       int lane) {
-    const bool fast = row0 + 32 <= M && (ld_t & 7) == 0 && aligned16(out_t);
-    if (fast) {
-#pragma unroll
-        for (int j = 0; j < 32; ++j)      // line j = column col0 + j; this lane's row is element `lane` of the line
-            *reinterpret_cast<__nv_bfloat16*>(stage + j * 64 + stage_piece(j, lane >> 3) * 16 + (lane & 7) * 2) =
-                __float2bfloat16_rn(v[j]);
-        __syncwarp();
-        const int64_t n_lines = n_cols - col0 < 32 ? n_cols - col0 : 32;
-        drain_stage(stage, out_t + col0 * ld_t + row0, ld_t, n_lines, lane);
-        __syncwarp();
-    } else {
-        const int64_t row = row0 + lane;
-        if (row < M) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (col0 + j < n_cols) out_t[(col0 + j) * ld_t + row] = __float2bfloat16_rn(v[j]);
-        }
-    }
-}
-
-// Row-major fallback: out[row][col0 .. col0+32); a full, aligned block of columns goes through the staging
+// Row-major store without a tensor map: out[row][col0 .. col0+32); a full, aligned block of columns goes through the staging
 // block, anything else through guarded element stores.  Rows beyond M are dropped.
 __device__ __forceinline__ void store_block_rows(__nv_bfloat16* out, int64_t ld, int64_t col0, int64_t n_cols, int64_t row0,
                                                  int64_t M, const float (&v)[32], uint8_t* stage, int lane) {
@@ -245,68 +117,48 @@ __device__ __forceinline__ void store_block_rows(__nv_bfloat16* out, int64_t ld,
 }
 
 // Bulk-store core: p[k] holds columns col0 + 2k (low half) and col0 + 2k + 1 (high half) of this lane's row as bf16.
-// The block is staged row-major (if rows_map) and / or transposed (if t_map) and leaves as bulk tensor
-// stores, clipped to the maps' extents (the caller guarantees row0 and col0 inside them); both stores
-// are issued behind one proxy fence.  ready_block (optional, for a single output): a staging block the
-// caller has already made sure no bulk store is reading; it is used instead of the output's own block
-// and nothing is waited for.  Warp-uniform arguments except p.
+// The block is staged row-major and leaves as one bulk tensor store, clipped to the map's extents (the caller
+// guarantees row0 and col0 inside them).  ready_block (optional): a staging block the caller has already made
+// sure no bulk store is reading; it is used instead of the warp's own block and nothing is waited for.
+// Warp-uniform arguments except p.
 __device__ __forceinline__ void store_block_packed(const uint32_t (&p)[16], uint8_t* stage, int lane, int64_t col0, int64_t row0,
-                                                   const CUtensorMap* rows_map, const CUtensorMap* t_map,
-                                                   uint8_t* ready_block = nullptr) {
-    uint8_t* t_block = stage;
+                                                   const CUtensorMap* rows_map, uint8_t* ready_block = nullptr) {
     uint8_t* rows_block = stage + kStageBlockBytes;
-    if (ready_block && (rows_map == nullptr) != (t_map == nullptr)) {
-        t_block = rows_block = ready_block;
+    if (ready_block) {
+        rows_block = ready_block;
     } else {
-        if (lane == 0) bulk_wait_read_all();      // the previous block's stores have read the staging blocks
+        if (lane == 0) bulk_wait_read_all();      // the previous block's store has read the staging block
         __syncwarp();
     }
-    if (t_map) {
-        // 2 x 2 exchange with the neighbouring lane: even lanes end up with rows (lane, lane + 1) of column 2k,
-        // odd lanes with rows (lane - 1, lane) of column 2k + 1, one 32-bit word each; line = column
-        uint8_t* base = t_block + (lane & 1) * 64 + (lane >> 1 & 3) * 4;
+    uint8_t* line = rows_block + lane * 64;
 #pragma unroll
-        for (int k = 0; k < 16; ++k) {
-            const uint32_t x = __shfl_xor_sync(0xffffffffu, p[k], 1);
-            const uint32_t w = (lane & 1) ? __byte_perm(x, p[k], 0x7632) : __byte_perm(p[k], x, 0x5410);
-            *reinterpret_cast<uint32_t*>(base + k * 128 + ((lane >> 3) ^ (k & 3)) * 16) = w;
-        }
-    }
-    if (rows_map) {
-        uint8_t* line = rows_block + lane * 64;
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-            *reinterpret_cast<uint4*>(line + stage_piece(lane, q) * 16) = make_uint4(p[4 * q], p[4 * q + 1], p[4 * q + 2], p[4 * q + 3]);
-    }
+    for (int q = 0; q < 4; ++q)
+        *reinterpret_cast<uint4*>(line + stage_piece(lane, q) * 16) = make_uint4(p[4 * q], p[4 * q + 1], p[4 * q + 2], p[4 * q + 3]);
     fence_proxy_async_smem();
     __syncwarp();
     if (lane == 0) {
-        if (t_map) tma_store_2d(t_map, t_block, (int32_t)row0, (int32_t)col0);
-        if (rows_map) tma_store_2d(rows_map, rows_block, (int32_t)col0, (int32_t)row0);
+        tma_store_2d(rows_map, rows_block, (int32_t)col0, (int32_t)row0);
         bulk_commit();
     }
 }
 
-// Stores a warp's 32 x 32 block (lane = row, v[j] = column col0 + j) as bf16: row-major into out
-// (if do_rows) and / or transposed into out_t (if do_t).  An output with a tensor map leaves through
-// store_block_packed, one without through the fallbacks above.  Warp-uniform arguments except v.
+// Stores a warp's 32 x 32 block (lane = row, v[j] = column col0 + j) as bf16, row-major, into out: through a
+// bulk tensor store where the output has a tensor map, else through store_block_rows.  Warp-uniform
+// arguments except v.
 __device__ __forceinline__ void store_block(const float (&v)[32], uint8_t* stage, int lane, int64_t col0, int64_t n_cols,
-                                            int64_t row0, int64_t M, bool do_rows, __nv_bfloat16* out, int64_t ld,
-                                            const CUtensorMap* rows_map, bool do_t, __nv_bfloat16* out_t, int64_t ld_t,
-                                            const CUtensorMap* t_map) {
-    const bool rows_tma = do_rows && rows_map, t_tma = do_t && t_map;
-    // (an output without a map never shares its staging block with a bulk store in flight)
-    if (do_t && !t_map) store_block_transposed(out_t, ld_t, col0, n_cols, row0, M, v, stage, lane);
-    if (do_rows && !rows_map) store_block_rows(out, ld, col0, n_cols, row0, M, v, stage + kStageBlockBytes, lane);
-    if (rows_tma || t_tma) {
-        uint32_t p[16];
-#pragma unroll
-        for (int k = 0; k < 16; ++k) {
-            __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
-            p[k] = *reinterpret_cast<uint32_t*>(&b2);
-        }
-        store_block_packed(p, stage, lane, col0, row0, rows_tma ? rows_map : nullptr, t_tma ? t_map : nullptr);
+                                            int64_t row0, int64_t M, __nv_bfloat16* out, int64_t ld,
+                                            const CUtensorMap* rows_map) {
+    if (!rows_map) {
+        store_block_rows(out, ld, col0, n_cols, row0, M, v, stage + kStageBlockBytes, lane);
+        return;
     }
+    uint32_t p[16];
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+        __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);
+        p[k] = *reinterpret_cast<uint32_t*>(&b2);
+    }
+    store_block_packed(p, stage, lane, col0, row0, rows_map);
 }
 
 // Copies a [32 x 32] bf16 block (rows row0.., columns col0..; full and aligned columns, guaranteed by the
@@ -329,7 +181,7 @@ __device__ __forceinline__ void stage_block_from_global(const __nv_bfloat16* src
 template <int BN, int STAGES, int MODE, int EW>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_rows, const __grid_constant__ CUtensorMap map_t, TcKernelArgs g) {
+               const __grid_constant__ CUtensorMap map_rows, TcKernelArgs g) {
     // Persistent: the block walks over output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...  The
     // stage ring runs on across tiles and the accumulator is multi-buffered in tensor memory, so
     // the loads and MMAs of the next tile(s) overlap the epilogue of the current one.
@@ -339,6 +191,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     static_assert(BN % (32 * CP) == 0 && NACC * BN <= 512, "tile split");
     extern __shared__ uint8_t smem_raw[];
     constexpr uint32_t kABytes = kTcBM * kTcBK * 2, kBBytes = BN * kTcBK * 2, kStageBytes = kABytes + kBBytes;
+    // The split-K products reduce over the batch, and their operands (activations and gradients, one batch row
+    // per line) are read as they lie in memory: M and N are the contiguous dimensions ("MN-major" operands).
+    constexpr bool kMnMajor = MODE == TC_EPI_PARTIAL;
+    constexpr uint32_t kMnBoxBytes = kTcBK * 64 * 2;      // one box: 64 reduction rows of 64 elements
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(tiles + STAGES * kStageBytes);
     uint64_t* empty = full + STAGES;
@@ -388,8 +244,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (!mbar_wait(empty + s, ph ^ 1, g.status, abort_flag)) { ok = false; break; }
                     mbar_expect_tx(full + s, kStageBytes);
                     uint8_t* a_dst = tiles + s * kStageBytes;
-                    tma_load_2d(a_dst, &map_a, kb * kTcBK, m0, full + s);
-                    tma_load_2d(a_dst + kABytes, &map_b, kb * kTcBK, n0, full + s);
+                    if constexpr (kMnMajor) {
+                        // operands stored [reduction index][M or N]: boxes of 64 reduction rows x 64 elements
+#pragma unroll
+                        for (int i = 0; i < kTcBM / 64; ++i)
+                            tma_load_2d(a_dst + i * kMnBoxBytes, &map_a, m0 + 64 * i, kb * kTcBK, full + s);
+#pragma unroll
+                        for (int i = 0; i < BN / 64; ++i)
+                            tma_load_2d(a_dst + kABytes + i * kMnBoxBytes, &map_b, n0 + 64 * i, kb * kTcBK, full + s);
+                    } else {
+                        tma_load_2d(a_dst, &map_a, kb * kTcBK, m0, full + s);
+                        tma_load_2d(a_dst + kABytes, &map_b, kb * kTcBK, n0, full + s);
+                    }
                 }
             }
             if (*abort_flag) {    // await (bounded) what was issued and not consumed, so nothing lands after exit
@@ -402,7 +268,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BN);
+            constexpr uint32_t idesc = make_idesc(BN, kMnMajor, kMnMajor);
             int64_t it = 0, lt = 0;               // k-blocks consumed, tiles done by this block
             bool ok = true;
             for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++lt) {
@@ -422,10 +288,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t a_addr = smem_u32(tiles + s * kStageBytes);
-                    const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(a_addr + kABytes);
+                    if constexpr (kMnMajor) {
+                        const uint64_t adesc = make_smem_desc_mn(a_addr, kMnBoxBytes);
+                        const uint64_t bdesc = make_smem_desc_mn(a_addr + kABytes, kMnBoxBytes);
 #pragma unroll
-                    for (int k = 0; k < kTcBK / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K: +2 in 16-byte units
-                        umma_bf16(acc_addr, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                        for (int k = 0; k < kTcBK / 16; ++k)      // 16 reduction rows = two 1024-byte atoms: +128 in 16-byte units
+                            umma_bf16(acc_addr, adesc + 128 * k, bdesc + 128 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                    } else {
+                        const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(a_addr + kABytes);
+#pragma unroll
+                        for (int k = 0; k < kTcBK / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K: +2 in 16-byte units
+                            umma_bf16(acc_addr, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                    }
                     umma_commit(empty + s);                   // frees the stage once these MMAs have read it
                 }
                 if (ok) umma_commit(acc_full + b);            // accumulator complete (at once for an empty K range)
@@ -442,9 +316,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint8_t* stage = stage_base + ew * kStageBytesPerWarp;      // this warp's two staging blocks
         int flip = 0;
         const CUtensorMap* rows_map = g.tma_rows ? &map_rows : nullptr;
-        const CUtensorMap* t_map = g.tma_t ? &map_t : nullptr;
         const bool row_owner = BN == 64 && MODE == TC_EPI_ARGMAX;
-        constexpr bool kGated = MODE == TC_EPI_MASK || MODE == TC_EPI_MASK_T;
+        constexpr bool kGated = MODE == TC_EPI_MASK;
         // soft-max epilogue: this warp's 32 bias values never change (its columns are the same in every tile)
         float ce_bias_lane = 0.f;
         if constexpr (BN == 64 && MODE == TC_EPI_SOFTMAX_CE)
@@ -457,8 +330,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (tile >= n_tiles) return;
             const int64_t rem = tile % per_split;
             const int64_t r0 = (rem % n_m) * kTcBM + q * 32, cc0 = (rem / n_m) * BN + c0;
-            const CUtensorMap* out_map = MODE == TC_EPI_MASK_T ? t_map : rows_map;
-            if (!out_map || r0 >= g.M || cc0 + 32 > g.N || (g.ld_mask & 7) != 0 || !aligned16(g.mask)) return;
+            if (!rows_map || r0 >= g.M || cc0 + 32 > g.N || (g.ld_mask & 7) != 0 || !aligned16(g.mask)) return;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int line = (lane >> 2) + 8 * i, piece = lane & 3;
@@ -539,12 +411,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const float scale = g.inv_rows / den;
 #pragma unroll
                 for (int j = 0; j < 32; ++j) v[j] = cb + j < g.N ? (v[j] * scale - (cb + j == yi ? g.inv_rows : 0.f)) : 0.f;
-                {   // dL row-major (clipped to the trained rows, padding columns zero) and transposed
-                    const bool t_out = g.out_bf16_t && cb < g.N && (!t_map || row0 < g.n_train);
-                    const bool rows_out = rows_map && g.out_bf16 && row0 < g.n_train && cb < g.ld_bf16;
-                    store_block(v, stage, lane, cb, g.N, row0, g.n_train, rows_out, g.out_bf16, g.ld_bf16, rows_map, t_out,
-                                g.out_bf16_t, g.ld_t, t_map);
-                }
+                // dL row-major (clipped to the trained rows, padding columns zero)
+                if (rows_map && g.out_bf16 && row0 < g.n_train && cb < g.ld_bf16)
+                    store_block(v, stage, lane, cb, g.N, row0, g.n_train, g.out_bf16, g.ld_bf16, rows_map);
                 if (!rows_map && live && g.out_bf16) {       // this thread's columns, 16 bytes at a time
                     __nv_bfloat16* dst = g.out_bf16 + row * g.ld_bf16 + cb;
 #pragma unroll
@@ -655,9 +524,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                             for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = __uint_as_float(r[j]);
                         }
-                    } else if constexpr (MODE == TC_EPI_MASK_T || MODE == TC_EPI_MASK) {
-                        const bool to_t = MODE == TC_EPI_MASK_T;
-                        const CUtensorMap* out_map = to_t ? t_map : rows_map;
+                    } else if constexpr (MODE == TC_EPI_MASK) {
+                        const CUtensorMap* out_map = rows_map;
                         const bool gate_runs = col0 + 32 <= g.N && (g.ld_mask & 7) == 0 && aligned16(g.mask);
                         // this chunk's gate block (if it was fetched ahead), then the fetch for the next chunk
                         uint4 gate_cur[4];
@@ -702,7 +570,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                             }
                             __syncwarp();         // every lane has read its gate row: the block may take the output
                             if (row0 < g.M)
-                                store_block_packed(p, stage, lane, col0, row0, to_t ? nullptr : rows_map, to_t ? t_map : nullptr, blk);
+                                store_block_packed(p, stage, lane, col0, row0, rows_map, blk);
                         } else {
                             if (n_kb > 0) tmem_ld_wait(r);
                             float v[32];
@@ -716,8 +584,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 for (int j = 0; j < 32; ++j) v[j] = 0.f;
                             }
                             if (row0 < g.M)
-                                store_block(v, stage, lane, col0, g.N, row0, g.M, !to_t, g.out_bf16, g.ld_bf16, rows_map, to_t,
-                                            g.out_bf16_t, g.ld_t, t_map);
+                                store_block(v, stage, lane, col0, g.N, row0, g.M, g.out_bf16, g.ld_bf16, rows_map);
                         }
                     } else {
                         float v[32];
@@ -755,11 +622,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 for (int j = 0; j < 32; ++j) if (col0 + j < g.N) dst[j] = v[j];
                             }
                         }
-                        if (row0 < g.M && (g.out_bf16 || g.out_bf16_t))
-                            store_block(v, stage, lane, col0, g.N, row0, g.M, g.out_bf16 != nullptr, g.out_bf16, g.ld_bf16, rows_map,
-                                        g.out_bf16_t != nullptr, g.out_bf16_t, g.ld_t, t_map);
-                        if (g.out_bf16_t && g.ones_row_t && col0 == 0 && row < g.M)
-                            g.out_bf16_t[g.N * g.ld_t + row] = __float2bfloat16_rn(1.0f);
+                        if (row0 < g.M && g.out_bf16)
+                            store_block(v, stage, lane, col0, g.N, row0, g.M, g.out_bf16, g.ld_bf16, rows_map);
+                        // the column of ones behind the last output column (it makes the bias gradient one more
+                        // row of the weight-gradient product that reads this matrix)
+                        if (g.out_bf16 && g.ones_col && col0 == 0 && row < g.M)
+                            g.out_bf16[row * g.ld_bf16 + g.N] = __float2bfloat16_rn(1.0f);
                     }
                 }
             }
@@ -795,32 +663,32 @@ static EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// 2-D bf16 tensor [rows x cols], cols contiguous, row stride ld elements; box = [box_rows x 64].
-static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+// Tensor map of a 2-D bf16 matrix [rows x cols], cols contiguous, row stride ld elements, for boxes of
+// [box_rows x box_cols] with the given swizzle width in bytes (128 or 64; box_cols * 2 must equal it).
+bool tc_make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows, int box_cols,
+                    int swizzle_bytes, bool l2_promote) {
     EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
+    if (!fn || !base || rows <= 0 || cols <= 0 || !aligned_to(base, 16) || ld % 8 != 0 || ld < cols) return false;
+    if (rows > INT32_MAX || cols > INT32_MAX || box_cols * 2 != swizzle_bytes || box_rows < 1 || box_rows > 256) return false;
     cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    cuuint32_t box[2] = {(cuuint32_t)kTcBK, (cuuint32_t)box_rows};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+              l2_promote ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B : CU_TENSOR_MAP_L2_PROMOTION_NONE,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Operand tile loads: box = [box_rows x 64], 128-byte swizzle.
+static bool make_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld, int box_rows) {
+    return tc_make_map_2d(map, base, rows, cols, ld, box_rows, kTcBK, 128, true);
 }
 
 // Tensor map of a bf16 output matrix [rows x cols] (row stride ld elements) for [32 x 32] stores with the
 // 64-byte swizzle of the staging blocks.  Returns false where the layout does not allow one.
 static bool make_store_map(CUtensorMap* map, const void* base, int64_t rows, int64_t cols, int64_t ld) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn || !base || rows <= 0 || cols <= 0 || !aligned_to(base, 16) || ld % 8 != 0 || ld < cols) return false;
-    if (rows > INT32_MAX || cols > INT32_MAX) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    cuuint32_t box[2] = {32, 32};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return tc_make_map_2d(map, base, rows, cols, ld, 32, 32, 64, false);
 }
 
 template <int BN, int STAGES, int MODE, int EW>
@@ -844,7 +712,7 @@ static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensor
     g.splits = splits;
     g.mode = t.mode; g.relu = t.relu; g.bias = t.bias;
     g.out_f32 = t.out_f32; g.ld_f32 = t.ld_f32; g.out_bf16 = t.out_bf16; g.ld_bf16 = t.ld_bf16;
-    g.out_bf16_t = t.out_bf16_t; g.ld_t = t.ld_t; g.ones_row_t = t.ones_row_t;
+    g.ones_col = (t.ones_col && t.out_bf16 && t.ld_bf16 > t.N) ? 1 : 0;
     g.mask = t.mask; g.ld_mask = t.ld_mask;
     g.gate_scale = t.gate_scale != 0.f ? t.gate_scale : 1.f;
     g.drop_thresh = t.drop_thresh; g.drop_step = t.drop_step; g.drop_key0 = t.drop_key[0]; g.drop_key1 = t.drop_key[1];
@@ -854,20 +722,19 @@ static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensor
     g.n_train = (t.mode == TC_EPI_SOFTMAX_CE && t.eval_from > 0 && t.eval_from < t.M) ? t.eval_from : t.M;
     g.y_eval = t.y_eval;
     // bf16 outputs leave through bulk tensor stores where their layout allows it
-    CUtensorMap m_rows, m_t;
+    CUtensorMap m_rows;
     memset(&m_rows, 0, sizeof(m_rows));
-    memset(&m_t, 0, sizeof(m_t));
     const bool ce = t.mode == TC_EPI_SOFTMAX_CE;
     const bool bias_like = t.mode == TC_EPI_BIAS || t.mode == TC_EPI_BIAS_DROP;
-    if (t.out_bf16 && (bias_like || t.mode == TC_EPI_MASK || ce))
+    // (with a column of ones behind an output whose width is not a whole number of 16-byte pieces, the store of
+    //  the last piece and the plain store of the ones would meet in one piece: such shapes take plain stores)
+    if (t.out_bf16 && (bias_like || t.mode == TC_EPI_MASK || ce) && !(g.ones_col && t.N % 8 != 0))
         g.tma_rows = make_store_map(&m_rows, t.out_bf16, ce ? g.n_train : t.M, ce ? t.ld_bf16 : t.N, t.ld_bf16) ? 1 : 0;
-    if (t.out_bf16_t && (bias_like || t.mode == TC_EPI_MASK_T || ce))
-        g.tma_t = make_store_map(&m_t, t.out_bf16_t, t.N, ce ? g.n_train : t.M, t.ld_t) ? 1 : 0;
     const int64_t n_tiles = ((t.M + kTcBM - 1) / kTcBM) * ((t.N + BN - 1) / BN) * splits;
     const int n_sm = sm_count();
     if (n_sm <= 0) return RETEXO_ERR_CUDA;
     const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);      // one persistent block per SM
-    tc_gemm_kernel<BN, STAGES, MODE, EW><<<grid, 64 + 32 * EW, smem, st>>>(ma, mb, m_rows, m_t, g);
+    tc_gemm_kernel<BN, STAGES, MODE, EW><<<grid, 64 + 32 * EW, smem, st>>>(ma, mb, m_rows, g);
     return launch_status();
 }
 
@@ -877,7 +744,6 @@ static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& 
         case TC_EPI_BIAS: return launch_tc_mode<BN, STAGES, TC_EPI_BIAS, EW>(t, ma, mb, st);
         case TC_EPI_BIAS_DROP: return launch_tc_mode<BN, STAGES, TC_EPI_BIAS_DROP, EW>(t, ma, mb, st);
         case TC_EPI_PARTIAL: return launch_tc_mode<BN, STAGES, TC_EPI_PARTIAL, EW>(t, ma, mb, st);
-        case TC_EPI_MASK_T: return launch_tc_mode<BN, STAGES, TC_EPI_MASK_T, EW>(t, ma, mb, st);
         case TC_EPI_MASK: return launch_tc_mode<BN, STAGES, TC_EPI_MASK, EW>(t, ma, mb, st);
         case TC_EPI_SOFTMAX_CE:
             if constexpr (BN == 64) return launch_tc_mode<BN, STAGES, TC_EPI_SOFTMAX_CE, EW>(t, ma, mb, st);
@@ -892,7 +758,6 @@ static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& 
 
 bool tc_gemm_supported(const TcGemm& t) {
     if (t.M <= 0 || t.N <= 0 || t.K <= 0) return false;
-    if (t.mode == TC_EPI_MASK_T && (!t.mask || !t.out_bf16_t)) return false;
     if (t.mode == TC_EPI_MASK && (!t.mask || !t.out_bf16)) return false;
     if (t.mode == TC_EPI_PARTIAL && !t.partial) return false;
     if ((t.mode == TC_EPI_SOFTMAX_CE || t.mode == TC_EPI_ARGMAX) && t.N > 64) return false;
@@ -909,10 +774,15 @@ int tc_gemm_launch(const TcGemm& t, cudaStream_t st) {
     // the gated products have a short reduction and a heavy epilogue: tiles of 128 columns put sixteen
     // epilogue warps on them (measured: the 256 x 153757 x 41 product itself is level with 256-column
     // tiles, the whole training iteration 1 % shorter)
-    if ((t.mode == TC_EPI_MASK || t.mode == TC_EPI_MASK_T) && bn == 256) bn = 128;
+    if (t.mode == TC_EPI_MASK && bn == 256) bn = 128;
     CUtensorMap ma, mb;
-    if (!make_map(&ma, t.A, t.M, t.K, t.lda, kTcBM)) return RETEXO_ERR_CUDA;
-    if (!make_map(&mb, t.B, t.N, t.K, t.ldb, bn)) return RETEXO_ERR_CUDA;
+    if (t.mode == TC_EPI_PARTIAL) {      // A [K x M], B [K x N] as they lie in memory: boxes of 64 reduction rows x 64 elements
+        if (!make_map(&ma, t.A, t.K, t.M, t.lda, kTcBK)) return RETEXO_ERR_CUDA;
+        if (!make_map(&mb, t.B, t.K, t.N, t.ldb, kTcBK)) return RETEXO_ERR_CUDA;
+    } else {
+        if (!make_map(&ma, t.A, t.M, t.K, t.lda, kTcBM)) return RETEXO_ERR_CUDA;
+        if (!make_map(&mb, t.B, t.N, t.K, t.ldb, bn)) return RETEXO_ERR_CUDA;
+    }
     if (bn == 256) return launch_tc<256, TC256_STAGES, TC256_EW>(t, ma, mb, st);
     if (bn == 128) return launch_tc<128, TC128_STAGES, TC128_EW>(t, ma, mb, st);
     return launch_tc<64, TC64_STAGES, TC64_EW>(t, ma, mb, st);

@@ -1,16 +1,18 @@
 // Host side of the per-node model calls: argument checks, workspace layout and
 // the launch sequence of one training iteration / one embedding pass.
 //
-// Every matrix product of an iteration runs on the tensor cores (gemm_tc.cu);
-// that kernel wants both operands with the reduction dimension contiguous,
-// hence the transposed copies kept next to the row-major ones:
-//   forward   Hd  = ReLU(X W1 + b1)           A = X        B = W1^T
-//             L   = Hd W2 + b2                A = Hd       B = W2^T
-//   backward  dHd^T = (W2 dL^T) .* [Hd^T > 0] A = W2 (rows padded)   B = dL
-//             [dW2 ; db2] = [Hd^T ; 1] dL     A = [Hd^T;1] B = dL^T               split over the batch
-//             [dW1 ; db1] = [X^T ; 1] dHd     A = [X^T;1]  B = dHd^T              split over the batch
-// The all-ones row turns each bias gradient into one more output row, so the
-// partial sums come out laid out exactly like theta = [W1 | b1 | W2 | b2].
+// Every matrix product of an iteration runs on the tensor cores.  Activations and
+// gradients are kept row-major only (one batch row per line): the forward products
+// read them with the reduction dimension contiguous, the weight-gradient products,
+// whose reduction runs over the batch, read the same arrays with M / N contiguous.
+//   forward   [Hd | 1] = ReLU(X W1 + b1)                 gemm_tc.cu, A = X, B = W1^T
+//   middle    L = Hd W2 + b2, loss, dL,                  mlp_fused.cu: one kernel, Hd read once,
+//             dHd = (dL W2^T) .* [Hd > 0]                the logits never leave the SM
+//   backward  [dW2 ; db2] = [Hd | 1]^T dL                gemm_tc.cu, split over the batch
+//             [dW1 ; db1] = [X | 1]^T dHd                gemm_tc.cu, split over the batch
+// (hidden > 256: the middle runs as two products of gemm_tc.cu instead.)
+// The column of ones behind X and Hd turns each bias gradient into one more output
+// row, so the partial sums come out laid out exactly like theta = [W1 | b1 | W2 | b2].
 #include "gemm_tc.h"
 #include "mlp_kernels.cuh"
 #include "mlp_plan.h"
@@ -60,11 +62,12 @@ MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_row
     p.d_in = d_in; p.hidden = hidden; p.n_classes = n_classes; p.n_rows = n_rows; p.n_eval = n_eval;
     p.out1 = hidden > 0 ? hidden : n_classes;
     p.nt = retexo_theta_size(d_in, hidden, n_classes);
-    p.ld_dl = pad_ld(n_classes);
+    p.ld_dl = pad_ld(n_classes);                           // 64: classes padded with zero columns
     p.ld_h = pad_ld(hidden > 0 ? hidden : 1);
+    p.ld_h1 = pad_ld(hidden > 0 ? hidden + 1 : 1);
     p.ld_k = pad_ld(d_in);
-    p.ld_n = pad_ld(n_rows + n_eval);
-    p.sm_blocks = (n_rows + n_eval + 127) / 128;          // one loss partial per 128-row tile of the head product
+    p.ld_x1 = pad_ld((int64_t)d_in + 1);
+    p.sm_blocks = 4 * ((n_rows + n_eval + 127) / 128);     // up to four loss partials per 128-row tile
     p.split_w1 = tc_split((int64_t)d_in + 1, p.out1, n_rows);
     p.split_w2 = hidden > 0 ? tc_split((int64_t)hidden + 1, n_classes, n_rows) : 0;
     return p;
@@ -79,13 +82,10 @@ static void layout(const MlpPlan& p, Taker& t, MlpBuffers* out) {
     b.w1t16 = t.template take<bf16>((size_t)p.out1 * p.ld_k);
     b.w2t16 = t.template take<bf16>(h ? (size_t)p.n_classes * p.ld_h : 1);
     b.w2p16 = t.template take<bf16>(h ? (size_t)p.hidden * p.ld_dl : 1);
-    b.xt16 = t.template take<bf16>((size_t)(p.d_in + 1) * p.ld_n);
-    b.hd16 = t.template take<bf16>(h ? n_all * p.ld_h : 1);
-    b.hdt16 = t.template take<bf16>(h ? (size_t)(p.hidden + 1) * p.ld_n : 1);
-    b.logits = t.template take<float>(n * p.n_classes);
+    b.x1 = t.template take<bf16>(n_all * p.ld_x1);
+    b.hd16 = t.template take<bf16>(h ? n_all * p.ld_h1 : 1);
     b.dl16 = t.template take<bf16>(n * p.ld_dl);
-    b.dlt16 = t.template take<bf16>((size_t)p.n_classes * p.ld_n);
-    b.dhdt16 = t.template take<bf16>(h ? (size_t)p.hidden * p.ld_n : 1);
+    b.dhd16 = t.template take<bf16>(h ? n * p.ld_h : 1);
     b.loss_partial = t.template take<float>((size_t)p.sm_blocks);
     b.pw1 = t.template take<float>((size_t)p.split_w1 * (p.d_in + 1) * p.out1);
     b.pw2 = t.template take<float>(h ? (size_t)p.split_w2 * (p.hidden + 1) * p.n_classes : 1);
@@ -144,11 +144,10 @@ extern "C" int64_t retexo_theta_size(int32_t d_in, int32_t hidden, int32_t n_cla
 
 extern "C" int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld_src, int32_t dim,
                                 const int32_t* idx, int64_t n_rows, void* dst, int64_t ld_dst,
-                                void* dst_t, int64_t ld_t, int32_t ones_row, void* stream) {
+                                void* dst_t, int64_t ld_t, int32_t ones, void* stream) {
     if (!src || dim <= 0 || ld_src < dim || n_rows < 0 || (!dst && !dst_t)) return RETEXO_ERR_INVALID_ARG;
-    if (dst && ld_dst < dim) return RETEXO_ERR_INVALID_ARG;
+    if (dst && ld_dst < dim + (ones ? 1 : 0)) return RETEXO_ERR_INVALID_ARG;
     if (dst_t && ld_t < n_rows) return RETEXO_ERR_INVALID_ARG;
-    if (ones_row && !dst_t) return RETEXO_ERR_INVALID_ARG;
     const int64_t rows_cover = dst_t ? (ld_t > n_rows ? ld_t : n_rows) : n_rows;
     const int64_t cols_cover = dst ? ld_dst : dim;
     if (rows_cover == 0) return RETEXO_OK;
@@ -157,10 +156,10 @@ extern "C" int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (src_is_bf16)
         pack_rows_kernel<true><<<grid, 256, 0, st>>>(src, ld_src, dim, idx, n_rows, static_cast<bf16*>(dst), ld_dst,
-                                                     static_cast<bf16*>(dst_t), ld_t, ones_row ? 1 : 0);
+                                                     static_cast<bf16*>(dst_t), ld_t, ones ? 1 : 0);
     else
         pack_rows_kernel<false><<<grid, 256, 0, st>>>(src, ld_src, dim, idx, n_rows, static_cast<bf16*>(dst), ld_dst,
-                                                      static_cast<bf16*>(dst_t), ld_t, ones_row ? 1 : 0);
+                                                      static_cast<bf16*>(dst_t), ld_t, ones ? 1 : 0);
     return launch_status();
 }
 
@@ -170,16 +169,15 @@ extern "C" size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hid
     return mlp_step_workspace_size(make_plan(d_in, hidden, n_classes, n_rows));
 }
 
-extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t ldx, const void* x_t, int64_t ld_xt,
+extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t ldx, int32_t x_has_ones,
                                      const int32_t* y, int64_t n_rows, float* loss_out, float* grad_out,
                                      void* workspace, size_t workspace_bytes, void* stream) {
     RETEXO_TRY(check_model(model));
     if (!x || !y || n_rows <= 0 || ldx < model->d_in) return RETEXO_ERR_INVALID_ARG;
     if (model->optimizer != RETEXO_SGD && model->optimizer != RETEXO_ADAM) return RETEXO_ERR_INVALID_ARG;
     if (model->optimizer == RETEXO_ADAM && (!model->adam_m || !model->adam_v)) return RETEXO_ERR_INVALID_ARG;
-    if (x_t && ld_xt < n_rows) return RETEXO_ERR_INVALID_ARG;
+    if (x_has_ones && ldx < (int64_t)model->d_in + 1) return RETEXO_ERR_INVALID_ARG;
     if (!aligned_to(x, 16) || ldx % 8 != 0) return RETEXO_ERR_ALIGNMENT;
-    if (x_t && (!aligned_to(x_t, 16) || ld_xt % 8 != 0)) return RETEXO_ERR_ALIGNMENT;
     const size_t need = retexo_mlp_train_step_workspace_size(model->d_in, model->hidden, model->n_classes, n_rows);
     if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -188,8 +186,8 @@ extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t l
     Arena ws(workspace, workspace_bytes);
     MlpBuffers b{};
     layout(p, ws, &b);
-    RETEXO_TRY(mlp_train_step_launch(p, b, model, static_cast<const bf16*>(x), ldx,
-                                     static_cast<const bf16*>(x_t), ld_xt, y, loss_out, grad_out, false, nullptr, st));
+    RETEXO_TRY(mlp_train_step_launch(p, b, model, static_cast<const bf16*>(x), ldx, x_has_ones != 0, y, loss_out, grad_out,
+                                     false, nullptr, st));
     model->step += 1;
     return RETEXO_OK;
 }
@@ -199,7 +197,7 @@ namespace retexo {
 // The launch sequence of one iteration; `model->step` is the count of updates
 // already applied.
 int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
-                          const bf16* x, int64_t ldx, const bf16* x_t, int64_t ld_xt, const int32_t* y,
+                          const bf16* x, int64_t ldx, bool x_has_ones, const int32_t* y,
                           float* loss_out, float* grad_out, bool shadows_ready, const EvalTail* tail,
                           cudaStream_t st, const DeviceIter* dev) {
     const int64_t n = p.n_rows;
@@ -213,23 +211,23 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         RETEXO_CUDA_TRY(cudaMemsetAsync(b.status, 0, sizeof(int32_t), st));
         RETEXO_TRY(build_weight_shadows(p, b, theta, st));
     }
-    if (!x_t) {      // no transposed batch from the caller: build [X^T ; 1] here (one more pass over X per call)
-        RETEXO_TRY(retexo_pack_rows(x, 1, ldx, d_in, nullptr, n, nullptr, 0, b.xt16, p.ld_n, 1, st));
-        x_t = b.xt16;
-        ld_xt = p.ld_n;
+    if (!x_has_ones) {      // no column of ones behind the caller's batch: copy it with one (one more pass over X per call)
+        RETEXO_TRY(retexo_pack_rows(x, 1, ldx, d_in, nullptr, n_all, b.x1, p.ld_x1, nullptr, 0, 1, st));
+        x = b.x1;
+        ldx = p.ld_x1;
     }
 
-    // ---- forward; the class-dimension product ends in the loss: softmax, cross-entropy and dL
-    //      are computed in its epilogue, where one thread holds a whole row of logits
+    // ---- forward
     if (tail && !tail->done) RETEXO_CUDA_TRY(cudaMemsetAsync(tail->correct, 0, sizeof(unsigned long long), st));
     TcGemm fwd = tc_base(x, ldx, b.w1t16, p.ld_k, n_all, out1, d_in, b.status);
     fwd.bias = b1;
-    TcGemm head = fwd;
     const bool dropping = H > 0 && model->dropout > 0.f;
     const float keep_scale = dropping ? (float)(1.0 / (1.0 - (double)model->dropout)) : 1.f;
+    const bf16* grad1 = b.dl16;      // gradient at the first layer's output, one batch row per line
+    int64_t ld_grad1 = p.ld_dl;
+    int64_t n_loss = (n_all + 127) / 128;
     if (H > 0) {
-        fwd.relu = 1; fwd.out_bf16 = b.hd16; fwd.ld_bf16 = p.ld_h;
-        fwd.out_bf16_t = b.hdt16; fwd.ld_t = p.ld_n; fwd.ones_row_t = 1;
+        fwd.relu = 1; fwd.out_bf16 = b.hd16; fwd.ld_bf16 = p.ld_h1; fwd.ones_col = 1;
         if (dropping) {
             fwd.mode = TC_EPI_BIAS_DROP;
             fwd.drop_thresh = (uint32_t)floor((double)model->dropout * 4294967296.0);
@@ -241,29 +239,44 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
             fwd.drop_rows = n;
         }
         RETEXO_TRY(tc_gemm_launch(fwd, st));
-        head = tc_base(b.hd16, p.ld_h, b.w2t16, p.ld_h, n_all, O, H, b.status);
-        head.bias = b2;
-    }
-    head.mode = TC_EPI_SOFTMAX_CE; head.y = y; head.inv_rows = 1.0f / (float)n; head.loss_partial = b.loss_partial;
-    head.out_bf16 = H > 0 ? b.dl16 : nullptr; head.ld_bf16 = p.ld_dl;
-    head.out_bf16_t = b.dlt16; head.ld_t = p.ld_n;
-    if (tail) { head.eval_from = n; head.y_eval = tail->y_eval; head.correct = tail->correct; }
-    RETEXO_TRY(tc_gemm_launch(head, st));
-    // ---- backward
-    const bf16* grad1_t = b.dlt16;      // gradient at the first layer's output, transposed
-    if (H > 0) {
-        // dHd^T = W2 dL^T, gated by Hd^T > 0: computed directly in the transposed orientation the weight
-        // gradient reads, so mask and output are both row-major for the epilogue
-        TcGemm bk = tc_base(b.w2p16, p.ld_dl, b.dl16, p.ld_dl, H, n, O, b.status);
-        bk.mode = TC_EPI_MASK; bk.mask = b.hdt16; bk.ld_mask = p.ld_n; bk.out_bf16 = b.dhdt16; bk.ld_bf16 = p.ld_n;
-        bk.gate_scale = keep_scale;      // a dropped unit has Hd = 0, so the gate already holds the mask
-        RETEXO_TRY(tc_gemm_launch(bk, st));
-        TcGemm g2 = tc_base(b.hdt16, p.ld_n, b.dlt16, p.ld_n, (int64_t)H + 1, O, n, b.status);
+        // ---- class product, loss and gated back-propagation
+        HeadBackward hb{};
+        hb.hd = b.hd16; hb.ld_hd = p.ld_h1; hb.w2t = b.w2t16; hb.ld_w2t = p.ld_h; hb.b2 = b2;
+        hb.hidden = H; hb.n_classes = O; hb.n_train = n; hb.n_all = n_all;
+        hb.y = y; hb.y_eval = tail ? tail->y_eval : nullptr;
+        hb.inv_rows = 1.0f / (float)n; hb.gate_scale = keep_scale;      // a dropped unit has Hd = 0: the gate holds the mask
+        hb.dl = b.dl16; hb.ld_dl = p.ld_dl; hb.dhd = b.dhd16; hb.ld_dhd = p.ld_h;
+        hb.loss_partial = b.loss_partial; hb.correct = tail ? tail->correct : nullptr; hb.status = b.status;
+        if (head_backward_supported(hb)) {
+            RETEXO_TRY(head_backward_launch(hb, st));
+            n_loss *= 4;
+        } else {      // wide hidden layers: the same three steps as two products
+            TcGemm head = tc_base(b.hd16, p.ld_h1, b.w2t16, p.ld_h, n_all, O, H, b.status);
+            head.bias = b2;
+            head.mode = TC_EPI_SOFTMAX_CE; head.y = y; head.inv_rows = 1.0f / (float)n; head.loss_partial = b.loss_partial;
+            head.out_bf16 = b.dl16; head.ld_bf16 = p.ld_dl;
+            if (tail) { head.eval_from = n; head.y_eval = tail->y_eval; head.correct = tail->correct; }
+            RETEXO_TRY(tc_gemm_launch(head, st));
+            TcGemm bk = tc_base(b.dl16, p.ld_dl, b.w2p16, p.ld_dl, n, H, O, b.status);
+            bk.mode = TC_EPI_MASK; bk.mask = b.hd16; bk.ld_mask = p.ld_h1; bk.out_bf16 = b.dhd16; bk.ld_bf16 = p.ld_h;
+            bk.gate_scale = keep_scale;
+            RETEXO_TRY(tc_gemm_launch(bk, st));
+        }
+        // ---- [dW2 ; db2] = [Hd | 1]^T dL
+        TcGemm g2 = tc_base(b.hd16, p.ld_h1, b.dl16, p.ld_dl, (int64_t)H + 1, O, n, b.status);
         g2.mode = TC_EPI_PARTIAL; g2.splits = (int)p.split_w2; g2.partial = b.pw2;
         RETEXO_TRY(tc_gemm_launch(g2, st));
-        grad1_t = b.dhdt16;
+        grad1 = b.dhd16;
+        ld_grad1 = p.ld_h;
+    } else {
+        // last round: the single linear layer ends in the loss
+        fwd.mode = TC_EPI_SOFTMAX_CE; fwd.y = y; fwd.inv_rows = 1.0f / (float)n; fwd.loss_partial = b.loss_partial;
+        fwd.out_bf16 = b.dl16; fwd.ld_bf16 = p.ld_dl;
+        if (tail) { fwd.eval_from = n; fwd.y_eval = tail->y_eval; fwd.correct = tail->correct; }
+        RETEXO_TRY(tc_gemm_launch(fwd, st));
     }
-    TcGemm g1 = tc_base(x_t, ld_xt, grad1_t, p.ld_n, (int64_t)d_in + 1, out1, n, b.status);
+    // ---- [dW1 ; db1] = [X | 1]^T grad1
+    TcGemm g1 = tc_base(x, ldx, grad1, ld_grad1, (int64_t)d_in + 1, out1, n, b.status);
     g1.mode = TC_EPI_PARTIAL; g1.splits = (int)p.split_w1; g1.partial = b.pw1;
     RETEXO_TRY(tc_gemm_launch(g1, st));
 
@@ -278,7 +291,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     const double t = (double)(model->step + 1);
     u.corr1 = (float)(1.0 - pow((double)model->beta1, t));
     u.corr2 = (float)(1.0 - pow((double)model->beta2, t));
-    u.loss_partial = b.loss_partial; u.n_loss = (n_all + 127) / 128;      // the tiles this launch's head product wrote
+    u.loss_partial = b.loss_partial; u.n_loss = n_loss;      // the partials this launch's loss kernel wrote
     u.inv_rows = 1.0f / (float)n; u.loss_out = loss_out;
     u.status = b.status;
     u.w1t16 = b.w1t16; u.ld_k = p.ld_k; u.w2t16 = H > 0 ? b.w2t16 : nullptr; u.ld_h = p.ld_h;

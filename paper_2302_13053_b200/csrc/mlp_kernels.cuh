@@ -12,14 +12,15 @@ typedef __nv_bfloat16 bf16;
 
 // ---------------------------------------------------------------- packing
 // dst[i][c] = bf16(src[idx ? idx[i] : i][c]); dst_t[c][i] likewise.  Padding
-// columns of both outputs are written as zero.  With ones_row, dst_t gets one
-// more row (index dim) holding 1 for every batch row: the all-ones row that
-// makes the bias gradient one more output row of the weight-gradient product.
+// columns of both outputs are written as zero.  With ones, dst gets one more
+// column (index dim) and dst_t one more row (index dim) holding 1 for every
+// batch row: the all-ones vector that makes the bias gradient one more output
+// row of the weight-gradient product.
 template <bool SRC_BF16>
 __global__ void __launch_bounds__(256) pack_rows_kernel(const void* __restrict__ src, int64_t ld_src, int32_t dim,
                                                         const int32_t* __restrict__ idx, int64_t n_rows,
                                                         bf16* __restrict__ dst, int64_t ld_dst,
-                                                        bf16* __restrict__ dst_t, int64_t ld_t, int ones_row) {
+                                                        bf16* __restrict__ dst_t, int64_t ld_t, int ones) {
     __shared__ float tile[32][33];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;     // 32 x 8
     const int64_t r0 = blockIdx.x * 32ll;
@@ -33,7 +34,7 @@ __global__ void __launch_bounds__(256) pack_rows_kernel(const void* __restrict__
                          : static_cast<const float*>(src)[sr * ld_src + c];
         }
         tile[i][tx] = v;
-        if (dst && r < n_rows && c < ld_dst) dst[r * ld_dst + c] = f32_to_bf16(v);
+        if (dst && r < n_rows && c < ld_dst) dst[r * ld_dst + c] = f32_to_bf16((ones && c == dim) ? 1.0f : v);
     }
     if (!dst_t) return;
     __syncthreads();
@@ -41,7 +42,7 @@ __global__ void __launch_bounds__(256) pack_rows_kernel(const void* __restrict__
         const int64_t c = c0 + i, r = r0 + tx;
         if (c < dim && r < ld_t) dst_t[c * ld_t + r] = f32_to_bf16(tile[tx][i]);
     }
-    if (ones_row && blockIdx.y == 0 && ty == 0) {
+    if (ones && blockIdx.y == 0 && ty == 0) {
         const int64_t r = r0 + tx;
         if (r < ld_t) dst_t[(int64_t)dim * ld_t + r] = f32_to_bf16(r < n_rows ? 1.0f : 0.0f);
     }

@@ -16,11 +16,12 @@ struct MlpPlan {
     int32_t d_in, hidden, n_classes, out1;  // out1 = width of the first linear layer's output
     int64_t n_rows, nt;                     // training rows; nt = parameters in theta
     int64_t n_eval;                         // rows after the training rows that are only evaluated (validation)
-    int64_t ld_dl;                          // row stride of bf16 dL and of the padded W2 (classes rounded up to 8)
-    int64_t ld_h;                           // row stride of bf16 Hd and of W2^T (hidden rounded up to 8)
-    int64_t ld_k;                           // row stride of W1^T (d_in rounded up to 8)
-    int64_t ld_n;                           // row stride of everything stored transposed (all rows, rounded up to 8)
-    int64_t sm_blocks;                      // softmax blocks = number of loss partials
+    int64_t ld_dl;                          // row stride of bf16 dL and of the padded W2 (classes rounded up to 64)
+    int64_t ld_h;                           // row stride of bf16 dHd and of W2^T (hidden rounded up to 64)
+    int64_t ld_h1;                          // row stride of [Hd | 1] (hidden + 1 rounded up to 64)
+    int64_t ld_k;                           // row stride of W1^T (d_in rounded up to 64)
+    int64_t ld_x1;                          // row stride of the workspace copy [X | 1] (d_in + 1 rounded up to 64)
+    int64_t sm_blocks;                      // loss partials the workspace has room for
     int64_t split_w1, split_w2;             // split-K factors of the two weight-gradient products
 };
 
@@ -28,13 +29,11 @@ struct MlpBuffers {
     __nv_bfloat16* w1t16;                   // W1^T            [out1 x ld_k]
     __nv_bfloat16* w2t16;                   // W2^T            [n_classes x ld_h]
     __nv_bfloat16* w2p16;                   // W2, padded rows [hidden x ld_dl]
-    __nv_bfloat16* xt16;                    // [X^T ; 1]       [(d_in+1) x ld_n]  (only when the caller gives no x_t)
-    __nv_bfloat16* hd16;                    // Hd              [n x ld_h]
-    __nv_bfloat16* hdt16;                   // [Hd^T ; 1]      [(hidden+1) x ld_n]
-    float* logits;                          //                 [n x n_classes]
+    __nv_bfloat16* x1;                      // [X | 1]         [n x ld_x1]  (only when the caller's batch has no column of ones)
+    __nv_bfloat16* hd16;                    // [Hd | 1]        [n x ld_h1]
+    float* logits;                          //                 [n x n_classes]  (retexo_embed only)
     __nv_bfloat16* dl16;                    // dL              [n x ld_dl]
-    __nv_bfloat16* dlt16;                   // dL^T            [n_classes x ld_n]
-    __nv_bfloat16* dhdt16;                  // dHd^T           [hidden x ld_n]
+    __nv_bfloat16* dhd16;                   // dHd             [n x ld_h]
     float* loss_partial;
     float* pw1;                             // [split_w1 x (d_in+1) x out1]   partials of [dW1 ; db1]
     float* pw2;                             // [split_w2 x (hidden+1) x n_classes]   partials of [dW2 ; db2]
@@ -84,8 +83,10 @@ void mlp_step_buffers(const MlpPlan& p, void* workspace, size_t bytes, MlpBuffer
 // One training iteration.  shadows_ready: the bf16 weight copies in `b` already hold the
 // current theta (the previous iteration's update refreshed them), so they are not rebuilt.
 // On return they hold the updated theta.
+// x_has_ones: column d_in of x holds 1 in every row (ldx > d_in); otherwise the batch is first copied into
+// the workspace with that column added.
 int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
-                          const __nv_bfloat16* x, int64_t ldx, const __nv_bfloat16* x_t, int64_t ld_xt,
+                          const __nv_bfloat16* x, int64_t ldx, bool x_has_ones,
                           const int32_t* y, float* loss_out, float* grad_out, bool shadows_ready,
                           const EvalTail* tail, cudaStream_t st, const DeviceIter* dev = nullptr);
 

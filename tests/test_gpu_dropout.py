@@ -36,14 +36,14 @@ def test_masked_steps_track_the_checker(d_in, hidden, n_classes, n, p):
     x = rng.standard_normal((n, d_in)).astype(np.float32)
     y = rng.integers(0, n_classes, n).astype(np.int32)
     ref, gpu = pair(d_in, hidden, n_classes, 1, p, drop_seed)
-    x16, x_t = B().retexo_pack_rows(dev(x), None, transpose=True, ones_row=True, ld_multiple=8 if n % 2 else 64)
+    x16, _ = B().retexo_pack_rows(dev(x), None, ones=True, ld_multiple=8 if n % 2 else 64)
     x_host = x16[:, :d_in].float().cpu().numpy()
     losses = []
     for it in range(3):
         # each iteration starts from the GPU's state (see test_gpu_mlp.py); update numbers stay in step
         ref.theta = gpu.theta.cpu().numpy().astype(np.float64)
         rl, rg = ref.train_step(x_host, y, return_grad=True, dropout=p, dropout_seed=drop_seed)
-        gl, gg = B().retexo_mlp_train_step(gpu, x16, dev(y), x_t=x_t, return_grad=True)
+        gl, gg = B().retexo_mlp_train_step(gpu, x16, dev(y), x_has_ones=True, return_grad=True)
         gg = gg.cpu().numpy().astype(np.float64)
         assert ref.step == gpu.step == it + 1
         assert abs(gl.item() - rl) <= 2e-4 * max(1.0, abs(rl)), (it, gl.item(), rl)
@@ -62,17 +62,17 @@ def test_rate_zero_is_bit_for_bit_the_plain_step_and_bad_rates_are_rejected():
     rng = np.random.default_rng(0)
     x = rng.standard_normal((200, 48)).astype(np.float32)
     y = rng.integers(0, 5, 200).astype(np.int32)
-    x16, x_t = B().retexo_pack_rows(dev(x), None, transpose=True, ones_row=True)
+    x16, _ = B().retexo_pack_rows(dev(x), None, ones=True)
     _, a = pair(48, 64, 5, 3, 0.0, 0)
     _, b = pair(48, 64, 5, 3, 0.0, 12345)
-    la = B().retexo_mlp_train_step(a, x16, dev(y), x_t=x_t)
-    lb = B().retexo_mlp_train_step(b, x16, dev(y), x_t=x_t)
+    la = B().retexo_mlp_train_step(a, x16, dev(y), x_has_ones=True)
+    lb = B().retexo_mlp_train_step(b, x16, dev(y), x_has_ones=True)
     assert la.item() == lb.item()
     assert (a.theta == b.theta).all()
     for bad in (1.0, -0.1, float("nan")):
         _, c = pair(48, 64, 5, 3, bad, 1)
         with pytest.raises(B().RetexoError):
-            B().retexo_mlp_train_step(c, x16, dev(y), x_t=x_t)
+            B().retexo_mlp_train_step(c, x16, dev(y), x_has_ones=True)
 
 
 def lmp_both(w, R, p, seed, eval_every):

@@ -78,7 +78,7 @@ def test_one_training_iteration_of_the_reddit_shaped_round_one():
     q[:, :d] = dev(w.features)
     _, x16 = B.retexo_aggregate(w.aggr, dev(w.rowptr), dev(w.colidx), q, dim=d, want_f32=False, want_bf16=True)
     tr = dev(w.train_idx)
-    xtr, xtr_t = B.retexo_pack_rows(x16, tr, dim=2 * d, transpose=True, ones_row=True)
+    xtr, _ = B.retexo_pack_rows(x16, tr, dim=2 * d, ones=True)
     y = w.labels[w.train_idx]
     wt = wl.initial_weights(w)[0]
     gpu = B.Mlp(2 * d, w.hidden, w.n_classes, wt["w1"], wt["b1"], wt["w2"], wt["b2"], lr=w.lr)
@@ -86,7 +86,7 @@ def test_one_training_iteration_of_the_reddit_shaped_round_one():
     x_host = xtr[:, :2 * d].float().cpu().numpy()           # the checker sees the very batch the GPU trains on
     given = ref.copy()
     rl, rg = ref.train_step(x_host, y, return_grad=True)
-    gl, gg = B.retexo_mlp_train_step(gpu, xtr, dev(y), x_t=xtr_t, return_grad=True)
+    gl, gg = B.retexo_mlp_train_step(gpu, xtr, dev(y), x_has_ones=True, return_grad=True)
     assert abs(gl.item() - rl) <= 2e-4 * max(1.0, abs(rl)), (gl.item(), rl)
     gg = gg.cpu().numpy().astype(np.float64)
     err, scale = np.abs(gg - rg), np.abs(rg).max()
@@ -125,7 +125,7 @@ def test_one_training_iteration_and_emission_at_full_size(idx, m):
     rd, x16 = round_inputs(w, m)
     d_in, H, O = rd["d_in"], rd["hidden"], w.n_classes
     tr = dev(w.train_idx)
-    xtr, xtr_t = B.retexo_pack_rows(x16, tr, dim=d_in, transpose=True, ones_row=True)
+    xtr, _ = B.retexo_pack_rows(x16, tr, dim=d_in, ones=True)
     y = w.labels[w.train_idx]
     wt = wl.initial_weights(w)[m - 1]
     gpu = B.Mlp(d_in, H, O, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
@@ -133,7 +133,7 @@ def test_one_training_iteration_and_emission_at_full_size(idx, m):
     x_host = xtr[:, :d_in].float().cpu().numpy()
     given = ref.copy()
     rl, rg = ref.train_step(x_host, y, return_grad=True)
-    gl, gg = B.retexo_mlp_train_step(gpu, xtr, dev(y), x_t=xtr_t, return_grad=True)
+    gl, gg = B.retexo_mlp_train_step(gpu, xtr, dev(y), x_has_ones=True, return_grad=True)
     assert abs(gl.item() - rl) <= 2e-4 * max(1.0, abs(rl)), (gl.item(), rl)
     gg = gg.cpu().numpy().astype(np.float64)
     err, scale = np.abs(gg - rg), np.abs(rg).max()
@@ -141,7 +141,7 @@ def test_one_training_iteration_and_emission_at_full_size(idx, m):
     assert np.median(err) <= 2e-5 * scale
     given.apply_update(gg)
     assert np.abs(gpu.theta.cpu().numpy() - given.theta).max() <= 2e-6 * max(1.0, np.abs(given.theta).max())
-    del xtr, xtr_t, x_host
+    del xtr, x_host
     # emission over all rows with the updated weights, as the K-round run calls it; 4096 sampled rows checked
     rows = np.sort(np.random.default_rng(m).choice(w.n_nodes, 4096, replace=False))
     out = B.retexo_embed(gpu, x16, want_hidden=H > 0, want_logits=True, want_pred=True)

@@ -48,11 +48,15 @@ def test_pack_rows_gathers_rounds_and_transposes():
         assert dst[:, 37:].abs().sum() == 0 and dst_t[:, 45:].abs().sum() == 0
     dst, _ = B().retexo_pack_rows(dev(src), None, dim=20)
     assert torch.equal(dst[:, :20].cpu(), torch.from_numpy(src[:, :20]).to(torch.bfloat16))
-    # the row of ones that carries the bias gradient through the weight-gradient product
-    _, dst_t = B().retexo_pack_rows(dev(src), dev(idx), transpose=True, ones_row=True, ld_multiple=8)
-    assert dst_t.shape == (38, 48)
-    assert torch.equal(dst_t[:37, :45].cpu(), want.T)
+    # the ones that carry the bias gradient through the weight-gradient product: a column behind the batch,
+    # a row under its transpose
+    dst, dst_t = B().retexo_pack_rows(dev(src), dev(idx), transpose=True, ones=True, ld_multiple=8)
+    assert dst.shape == (45, 40) and dst_t.shape == (38, 48)
+    assert torch.equal(dst[:, :37].cpu(), want) and torch.equal(dst_t[:37, :45].cpu(), want.T)
+    assert torch.equal(dst[:, 37].float().cpu(), torch.ones(45)) and dst[:, 38:].abs().sum() == 0
     assert torch.equal(dst_t[37].float().cpu(), torch.cat([torch.ones(45), torch.zeros(3)]))
+    dst, _ = B().retexo_pack_rows(dev(src)[:, :32].contiguous(), None, ones=True)      # a full last line: one more line
+    assert dst.shape == (70, 64) and torch.equal(dst[:, 32].float().cpu(), torch.ones(70)) and dst[:, 33:].abs().sum() == 0
 
 
 @pytest.mark.parametrize("d_in,hidden,n_classes,n", [(5, 0, 3, 17), (64, 64, 7, 140), (33, 20, 4, 65),
@@ -66,7 +70,7 @@ def test_train_steps_track_the_checker(d_in, hidden, n_classes, n, opt):
     # Adam's first steps move every weight by about lr whatever the gradient's size, so weights whose
     # gradient is at rounding level take a different step in fp32 and fp64: keep that step small.
     ref, gpu = make_pair(d_in, hidden, n_classes, 1, opt=opt, lr=0.02 if opt == oracle.SGD else 1e-3)
-    x16, x_t = B().retexo_pack_rows(dev(x), None, transpose=True, ones_row=True, ld_multiple=8 if n % 2 else 64)
+    x16, _ = B().retexo_pack_rows(dev(x), None, ones=True, ld_multiple=8 if n % 2 else 64)
     yd = dev(y)
     for it in range(4):
         # Every iteration starts from the GPU's own state, so that each step is compared on its
@@ -78,7 +82,7 @@ def test_train_steps_track_the_checker(d_in, hidden, n_classes, n, opt):
         ref.v = gpu.v.cpu().numpy().astype(np.float64)
         given = ref.copy()
         rl, rg = ref.train_step(x, y, return_grad=True)
-        gl, gg = B().retexo_mlp_train_step(gpu, x16, yd, x_t=x_t, return_grad=True)
+        gl, gg = B().retexo_mlp_train_step(gpu, x16, yd, x_has_ones=True, return_grad=True)
         assert abs(gl.item() - rl) <= 2e-4 * max(1.0, abs(rl)), (it, gl.item(), rl)
         gg = gg.cpu().numpy().astype(np.float64)
         scale = np.abs(rg).max()
@@ -98,7 +102,7 @@ def test_zero_weights_give_log_of_class_count():
     y = np.random.default_rng(4).integers(0, o, n).astype(np.int32)
     gpu = B().Mlp(d, h, o, np.zeros((d, h)), np.zeros(h), np.zeros((h, o)), np.zeros(o), optimizer=oracle.SGD, lr=0.1)
     x16, _ = B().retexo_pack_rows(dev(x))
-    loss = B().retexo_mlp_train_step(gpu, x16, dev(y))      # no x_t given: the call builds it itself
+    loss = B().retexo_mlp_train_step(gpu, x16, dev(y))      # no column of ones given: the call adds it itself
     assert abs(loss.item() - np.log(o)) < 1e-6
 
 
