@@ -34,15 +34,39 @@ import numpy as np
 METRIC = "edges aggregated/s"
 UNIT = "edges/s"
 
-# DRAM bytes (read + write) per launch of the aggregation kernel, from the one-pass ncu captures
-# summarised in profiles/agg_kernels_cfg4.txt and profiles/agg_rows_kernel_cfg5.txt.  Valid for that
-# kernel and workload only: set an entry to None when the kernel or the workload changes.
-AGG_DRAM_TRAFFIC = {("cfg4_sage_reddit_like", 1): 14.68e9, ("cfg4_sage_reddit_like", 2): 6.24e9,
-                    ("cfg4_sage_reddit_like", 3): 5.99e9, ("cfg5_gcn_products_like", 1): 46.68e9,
-                    ("cfg5_gcn_products_like", 2): 102.92e9, ("cfg5_gcn_products_like", 3): 102.93e9}
-# DRAM bytes of one stand-alone training iteration (its five tc_gemm_kernel launches and
-# reduce_update_kernel), from the one-pass capture summarised in profiles/tc_gemm_kernel_cfg4.txt.
-STEP_DRAM_TRAFFIC = {("cfg4_sage_reddit_like", 1): 1.280e9}
+import hashlib
+
+CSRC = os.path.join(ROOT, "paper_2302_13053_b200", "csrc")
+
+
+def source_fingerprint(names) -> str:
+    """First 12 hex digits of the SHA-256 of the named kernel sources: the counters below are only valid
+    for the kernels they were captured from."""
+    h = hashlib.sha256()
+    for name in names:
+        with open(os.path.join(CSRC, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:12]
+
+
+# DRAM bytes (read + write) per launch, from one-pass ncu captures summarised under profiles/.  Each table names
+# the sources of the kernels it was captured from and their fingerprint at capture time; where the sources
+# have changed since, `traffic` is reported as null.
+AGG_SOURCES = ("aggregate.cu",)
+AGG_DRAM_TRAFFIC = {
+    "fingerprint": "b169e13d7982",      # profiles/agg_kernels_cfg4.txt, profiles/agg_rows_kernel_cfg5.txt
+    "bytes": {("cfg4_sage_reddit_like", 1): 14.68e9, ("cfg4_sage_reddit_like", 2): 6.24e9,
+              ("cfg4_sage_reddit_like", 3): 5.99e9, ("cfg5_gcn_products_like", 1): 46.68e9,
+              ("cfg5_gcn_products_like", 2): 102.92e9, ("cfg5_gcn_products_like", 3): 102.93e9}}
+# one stand-alone training iteration (its tensor-core launches and reduce_update_kernel): profiles/mlp_iteration_cfg4.txt
+STEP_SOURCES = ("gemm_tc.cu", "mlp_fused.cu", "mlp.cu", "mlp_kernels.cuh", "tc_common.cuh")
+STEP_DRAM_TRAFFIC = {"fingerprint": None, "bytes": {}}
+
+
+def measured_traffic(table, sources, key):
+    if table["fingerprint"] is None or table["fingerprint"] != source_fingerprint(sources):
+        return None
+    return table["bytes"].get(key)
 
 
 def min_time_roofline(flops: float, nbytes: float, ms: float, peaks) -> dict:
@@ -220,7 +244,7 @@ def phase_breakdown(w, ws, R: int, peaks):
         mean_ms, best_ms = time_calls(fn, 5)
         phases.append(dict(kernel="aggregate", round=m, calls_per_step=1, ms=mean_ms, best_ms=best_ms, bound="hbm",
                            algorithmic_bytes=alg, achieved=alg / mean_ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s",
-                           edges_per_s=e / mean_ms * 1e3, traffic=AGG_DRAM_TRAFFIC.get((w.name, m))))
+                           edges_per_s=e / mean_ms * 1e3, traffic=measured_traffic(AGG_DRAM_TRAFFIC, AGG_SOURCES, (w.name, m))))
         # the round's model at its training / validation / full shapes
         model = B.Mlp(rd["d_in"], rd["hidden"], w.n_classes, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
         xtr, _ = B.retexo_pack_rows(x16, tr, dim=width, ones=True)
@@ -251,7 +275,7 @@ def phase_breakdown(w, ws, R: int, peaks):
         ws_step = torch.empty(int(need), dtype=torch.uint8, device=dev)
         mean_ms, best_ms = time_calls(lambda: B.retexo_mlp_train_step(model, xtr, y_tr, x_has_ones=True, workspace=ws_step), 10)
         phases.append(dict(kernel="mlp_train_step", round=m, calls_per_step=R, ms=mean_ms, best_ms=best_ms,
-                           traffic=STEP_DRAM_TRAFFIC.get((w.name, m)),
+                           traffic=measured_traffic(STEP_DRAM_TRAFFIC, STEP_SOURCES, (w.name, m)),
                            **min_time_roofline(flops_step, bytes_step, mean_ms, peaks)))
         mean_ms, best_ms = time_calls(lambda: B.retexo_embed(model, xva, y=y_va), 10)
         phases.append(dict(kernel="embed_validation", round=m, calls_per_step=0, ms=mean_ms, best_ms=best_ms,

@@ -57,6 +57,7 @@ struct TcKernelArgs {
     float* out_f32; int64_t ld_f32;
     __nv_bfloat16* out_bf16; int64_t ld_bf16;
     int ones_col;
+    uint32_t* relu_bits; int64_t ld_bits;
     const __nv_bfloat16* mask; int64_t ld_mask;
     float gate_scale;
     uint32_t drop_thresh, drop_step, drop_key0, drop_key1; float drop_scale; int64_t drop_rows;
@@ -611,6 +612,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                                 }
                             }
                         }
+                        if (g.relu_bits && row < g.M) {      // one bit per unit: is the value that goes out positive?
+                            uint32_t word = 0u;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) word |= (v[j] > 0.f ? 1u : 0u) << j;
+                            g.relu_bits[row * g.ld_bits + (col0 >> 5)] = word;
+                        }
                         if (g.out_f32 && row < g.M) {
                             float* dst = g.out_f32 + row * g.ld_f32 + col0;
                             if (col0 + 32 <= g.N && (g.ld_f32 & 3) == 0 && aligned16(g.out_f32)) {
@@ -713,6 +720,7 @@ static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensor
     g.mode = t.mode; g.relu = t.relu; g.bias = t.bias;
     g.out_f32 = t.out_f32; g.ld_f32 = t.ld_f32; g.out_bf16 = t.out_bf16; g.ld_bf16 = t.ld_bf16;
     g.ones_col = (t.ones_col && t.out_bf16 && t.ld_bf16 > t.N) ? 1 : 0;
+    g.relu_bits = t.relu_bits; g.ld_bits = t.ld_bits;
     g.mask = t.mask; g.ld_mask = t.ld_mask;
     g.gate_scale = t.gate_scale != 0.f ? t.gate_scale : 1.f;
     g.drop_thresh = t.drop_thresh; g.drop_step = t.drop_step; g.drop_key0 = t.drop_key[0]; g.drop_key1 = t.drop_key[1];

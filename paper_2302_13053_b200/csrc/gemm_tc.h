@@ -16,7 +16,8 @@ enum TcEpilogue { TC_EPI_BIAS = 0, TC_EPI_PARTIAL = 1, TC_EPI_SOFTMAX_CE = 3, TC
 //                   fp32 (out_f32, ld_f32) and/or bf16 (out_bf16, ld_bf16).  With ones_col
 //                   (needs ld_bf16 > N) column N of out_bf16 is set to 1 in every row: the
 //                   all-ones column that turns a bias gradient into one more output row of
-//                   the weight-gradient product that reads this matrix.
+//                   the weight-gradient product that reads this matrix.  relu_bits (optional)
+//                   receives one bit per element, set where the value written is positive.
 //   TC_EPI_PARTIAL: C = A^T B with the operands as they lie in memory, A [K x lda] holding M
 //                   columns and B [K x ldb] holding N columns (the reduction runs over the rows,
 //                   i.e. over the batch; no transposed copy is needed).  K is cut into `splits`
@@ -41,6 +42,8 @@ struct TcGemm {
     float* out_f32; int64_t ld_f32;
     __nv_bfloat16* out_bf16; int64_t ld_bf16;
     int ones_col;
+    // TC_EPI_BIAS / TC_EPI_BIAS_DROP (optional): one bit per output element, bit n & 31 of word [m][n / 32] = [out > 0]
+    uint32_t* relu_bits; int64_t ld_bits;
     const __nv_bfloat16* mask; int64_t ld_mask;
     float gate_scale;          // TC_EPI_MASK: factor on the gated values (0 is read as 1)
     // TC_EPI_BIAS_DROP: as TC_EPI_BIAS, then dropout on rows [0, drop_rows): element (m, n) is kept iff word
@@ -71,6 +74,7 @@ bool tc_make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int64_t co
 // one kernel (hidden <= 256, n_classes <= 64); see mlp_fused.cu.
 struct HeadBackward {
     const __nv_bfloat16* hd; int64_t ld_hd;         // Hd [n_all x ld_hd], hidden columns
+    const uint32_t* gate_bits; int64_t ld_bits;     // [n_train x ld_bits] words: bit j & 31 of word j / 32 = [Hd[row][j] > 0]
     const __nv_bfloat16* w2t; int64_t ld_w2t;       // W2^T [n_classes x ld_w2t]
     const float* b2;
     int32_t hidden, n_classes;

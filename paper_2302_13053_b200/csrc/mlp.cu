@@ -65,6 +65,7 @@ MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_row
     p.ld_dl = pad_ld(n_classes);                           // 64: classes padded with zero columns
     p.ld_h = pad_ld(hidden > 0 ? hidden : 1);
     p.ld_h1 = pad_ld(hidden > 0 ? hidden + 1 : 1);
+    p.ld_bits = hidden > 0 ? 2 * (((int64_t)hidden + 63) / 64) : 2;
     p.ld_k = pad_ld(d_in);
     p.ld_x1 = pad_ld((int64_t)d_in + 1);
     p.sm_blocks = 4 * ((n_rows + n_eval + 127) / 128);     // up to four loss partials per 128-row tile
@@ -86,6 +87,7 @@ static void layout(const MlpPlan& p, Taker& t, MlpBuffers* out) {
     b.hd16 = t.template take<bf16>(h ? n_all * p.ld_h1 : 1);
     b.dl16 = t.template take<bf16>(n * p.ld_dl);
     b.dhd16 = t.template take<bf16>(h ? n * p.ld_h : 1);
+    b.gate_bits = t.template take<uint32_t>(h ? n_all * (size_t)p.ld_bits : 1);
     b.loss_partial = t.template take<float>((size_t)p.sm_blocks);
     b.pw1 = t.template take<float>((size_t)p.split_w1 * (p.d_in + 1) * p.out1);
     b.pw2 = t.template take<float>(h ? (size_t)p.split_w2 * (p.hidden + 1) * p.n_classes : 1);
@@ -228,6 +230,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     int64_t n_loss = (n_all + 127) / 128;
     if (H > 0) {
         fwd.relu = 1; fwd.out_bf16 = b.hd16; fwd.ld_bf16 = p.ld_h1; fwd.ones_col = 1;
+        fwd.relu_bits = b.gate_bits; fwd.ld_bits = p.ld_bits;
         if (dropping) {
             fwd.mode = TC_EPI_BIAS_DROP;
             fwd.drop_thresh = (uint32_t)floor((double)model->dropout * 4294967296.0);
@@ -241,7 +244,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         RETEXO_TRY(tc_gemm_launch(fwd, st));
         // ---- class product, loss and gated back-propagation
         HeadBackward hb{};
-        hb.hd = b.hd16; hb.ld_hd = p.ld_h1; hb.w2t = b.w2t16; hb.ld_w2t = p.ld_h; hb.b2 = b2;
+        hb.hd = b.hd16; hb.ld_hd = p.ld_h1; hb.gate_bits = b.gate_bits; hb.ld_bits = p.ld_bits; hb.w2t = b.w2t16; hb.ld_w2t = p.ld_h; hb.b2 = b2;
         hb.hidden = H; hb.n_classes = O; hb.n_train = n; hb.n_all = n_all;
         hb.y = y; hb.y_eval = tail ? tail->y_eval : nullptr;
         hb.inv_rows = 1.0f / (float)n; hb.gate_scale = keep_scale;      // a dropped unit has Hd = 0: the gate holds the mask

@@ -19,6 +19,7 @@ struct MlpPlan {
     int64_t ld_dl;                          // row stride of bf16 dL and of the padded W2 (classes rounded up to 64)
     int64_t ld_h;                           // row stride of bf16 dHd and of W2^T (hidden rounded up to 64)
     int64_t ld_h1;                          // row stride of [Hd | 1] (hidden + 1 rounded up to 64)
+    int64_t ld_bits;                        // words per row of the ReLU bits (two per 64 hidden units)
     int64_t ld_k;                           // row stride of W1^T (d_in rounded up to 64)
     int64_t ld_x1;                          // row stride of the workspace copy [X | 1] (d_in + 1 rounded up to 64)
     int64_t sm_blocks;                      // loss partials the workspace has room for
@@ -34,6 +35,7 @@ struct MlpBuffers {
     float* logits;                          //                 [n x n_classes]  (retexo_embed only)
     __nv_bfloat16* dl16;                    // dL              [n x ld_dl]
     __nv_bfloat16* dhd16;                   // dHd             [n x ld_h]
+    uint32_t* gate_bits;                    // [Hd > 0], a bit per unit   [n x ld_bits]
     float* loss_partial;
     float* pw1;                             // [split_w1 x (d_in+1) x out1]   partials of [dW1 ; db1]
     float* pw2;                             // [split_w2 x (hidden+1) x n_classes]   partials of [dW2 ; db2]

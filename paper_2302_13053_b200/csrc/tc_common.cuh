@@ -44,8 +44,13 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* m
         ::"r"(smem_u32(smem_dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
 
-// Bulk tensor store of a [32 x 32] bf16 box from shared memory (64-byte swizzle) to global memory;
-// the part of the box outside the tensor is not written.
+// Asks the box at (x, y) of the mapped tensor into L2; nothing is written to shared memory and nothing is signalled.
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int32_t x, int32_t y) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y) : "memory");
+}
+
+// Bulk tensor store of one box of the map's shape from shared memory (laid out with the map's swizzle) to global
+// memory; the part of the box outside the tensor is not written.
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* smem_src, int32_t x, int32_t y) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
                  ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(smem_src)) : "memory");
