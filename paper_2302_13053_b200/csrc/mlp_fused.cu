@@ -317,6 +317,7 @@ head_backward_kernel(const __grid_constant__ CUtensorMap map_hd, const __grid_co
         // ---- gate role: dHd = accumulator where the unit's ReLU bit is set, staged per warp and sent out
         const int q = warp & 3, h = (warp - kHbGateWarp0) >> 2;
         uint8_t* stage = out_stage + (warp - kHbGateWarp0) * kHbSlabBytes;
+        const bool scaled = g.gate_scale != 1.f;      // (dropout: the kept units' factor)
         for (int64_t i = 0; i < nt; ++i) {
             const int64_t tile = blockIdx.x + i * gridDim.x;
             const int64_t row0 = tile * 128 + q * 32, row = row0 + lane;
@@ -337,25 +338,30 @@ head_backward_kernel(const __grid_constant__ CUtensorMap map_hd, const __grid_co
                     const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + kHbGradCol0 + (uint32_t)(64 * p);
                     tmem_ld_issue(taddr, ra);
                     tmem_ld_issue(taddr + 32u, rb);
-                    if (lane == 0) bulk_wait_read_all();      // the store of the previous panel has read the staging block
-                    __syncwarp();
                     tmem_ld_wait(ra);
                     tmem_ld_wait(rb);
+                    // A unit whose bit is clear gives zero: the accumulator's bits are ANDed with 0 - bit.  Everything
+                    // is packed in registers first, so that the wait for the staging block comes after the arithmetic.
+                    uint32_t o[32];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const uint32_t word = (j < 4 ? bits[k].x : bits[k].y) >> (8 * (j & 3));
-                        uint32_t o[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int c = 8 * (j & 3) + 2 * e;
-                            const float a0 = __uint_as_float(j < 4 ? ra[c] : rb[c]), a1 = __uint_as_float(j < 4 ? ra[c + 1] : rb[c + 1]);
-                            const float lo = (word >> (2 * e)) & 1u ? a0 * g.gate_scale : 0.f;
-                            const float hi = (word >> (2 * e + 1)) & 1u ? a1 * g.gate_scale : 0.f;
+                            const uint32_t x0 = (j < 4 ? ra[c] : rb[c]) & (0u - ((word >> (2 * e)) & 1u));
+                            const uint32_t x1 = (j < 4 ? ra[c + 1] : rb[c + 1]) & (0u - ((word >> (2 * e + 1)) & 1u));
+                            float lo = __uint_as_float(x0), hi = __uint_as_float(x1);
+                            if (scaled) { lo *= g.gate_scale; hi *= g.gate_scale; }
                             __nv_bfloat162 b2 = __floats2bfloat162_rn(lo, hi);
-                            o[e] = *reinterpret_cast<uint32_t*>(&b2);
+                            o[4 * j + e] = *reinterpret_cast<uint32_t*>(&b2);
                         }
-                        *reinterpret_cast<uint4*>(stage + lane * 128 + ((j ^ (lane & 7)) * 16)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
+                    if (lane == 0) bulk_wait_read_all();      // the store of the previous panel has read the staging block
+                    __syncwarp();
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        *reinterpret_cast<uint4*>(stage + lane * 128 + ((j ^ (lane & 7)) * 16)) = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
                 }
                 if (k == 1 || p + 2 >= np) {      // this warp's last read of the accumulator for this tile
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
