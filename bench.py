@@ -63,6 +63,12 @@ STEP_SOURCES = ("gemm_tc.cu", "mlp_fused.cu", "mlp.cu", "mlp_kernels.cuh", "tc_c
 STEP_DRAM_TRAFFIC = {"fingerprint": None, "bytes": {}}
 
 
+# Peak of the L2 -> SM path in GB/s, as the profiler normalises it: in the section capture of the slab gather
+# (profiles/agg_kernels_cfg4.txt) the kernel delivered 15.6 / 16.7 TB/s of neighbour rows, all of them out of L2
+# (L1 hit rate 2 %), at lts__throughput = 68.3 / 72.5 % of peak; both give 22.9 TB/s for 100 %.
+L2_PEAK_GBS = 22900.0
+
+
 def measured_traffic(table, sources, key):
     if table["fingerprint"] is None or table["fingerprint"] != source_fingerprint(sources):
         return None
@@ -180,7 +186,7 @@ def launches_per_step(w, R: int) -> int:
         else:
             total += 3                               # prep, warp rows, block rows
         total += 2                                   # train / val batches
-        step = 6 if h > 0 else 3                     # products, reduce + update (+ weight copies once)
+        step = 5 if h > 0 else 3                     # products, fused middle, reduce + update (+ weight copies once)
         total += R * step + 1 + (2 if h > 0 else 1)       # (the update kernel's last block books the validation count
                                                           #  that rides along; the last iterate's is booked by a kernel of its own)
         total += (2 if h > 0 else 1) + 1             # stand-alone validation of the last iterate + snapshot
@@ -204,25 +210,32 @@ def time_calls(fn, reps: int, warm: int = 3):
     return statistics.mean(ts), min(ts)
 
 
-def phase_breakdown(w, ws, R: int, peaks):
-    """Times each entry point alone, at the shapes and launch configuration the
-    K-round run uses, and derives the roofline figures per kernel."""
+def measure_l2_gather_peak(rp, ci, n: int, e: int) -> float:
+    """Ceiling of the L2 -> SM path for a CSR gather, measured with the library's own gather on a matrix
+    that fits L2 whole (64 fp32 columns: 256-byte rows, every neighbour row a hit): bytes delivered to
+    the SMs per second, in GB/s."""
+    import torch
+    from paper_2302_13053_b200 import binding as B
+    d = 64
+    q = torch.rand((n, d), dtype=torch.float32, device="cuda")
+    out = torch.empty((n, 64), dtype=torch.bfloat16, device="cuda")
+    fn = lambda: B.retexo_aggregate(B.SAGE_MEAN, rp, ci, q, dim=d, concat_self=False, want_f32=False, out_bf16=out)
+    _, best_ms = time_calls(fn, 5)
+    return (e * (4 * d + 4) + 8 * (n + 1) + n * d * 2) / best_ms / 1e6
+
+
+def aggregation_phases(w, ws, peaks, rp, ci, l2_peak):
+    """Times every round's aggregation alone, in the launch configuration of the K-round run, and says
+    which ceiling binds: the L2 -> SM path where the kernel gathers from L2-resident column slabs (its DRAM
+    traffic is a small fraction of the bytes it delivers), HBM otherwise."""
     import torch
     from paper_2302_13053_b200 import binding as B
     from paper_2302_13053_b200 import workloads as wl
     dev = "cuda"
-    rp = torch.from_numpy(w.rowptr).to(dev)
-    ci = torch.from_numpy(w.colidx).to(dev)
     n, e = w.n_nodes, w.n_edges
-    tr = torch.from_numpy(w.train_idx).to(dev)
-    va = torch.from_numpy(w.val_idx).to(dev)
-    y = torch.from_numpy(w.labels).to(dev)
-    y_tr, y_va = y[tr.long()].contiguous(), y[va.long()].contiguous()
-    phases = []
-    q = None
+    out = []
     for rd, wt in zip(w.round_dims(), ws):
-        m = rd["round"]
-        d = rd["agg_dim"]
+        m, d = rd["round"], rd["agg_dim"]
         ld = (rd["rep_dim"] + 31) // 32 * 32
         if m == 1:
             q = torch.zeros((n, ld), dtype=torch.float32, device=dev)
@@ -242,33 +255,86 @@ def phase_breakdown(w, ws, R: int, peaks):
             fn = lambda: B.retexo_aggregate(w.aggr, rp, ci, q, dim=d, want_f32=False, out_bf16=x16)
             alg = e * (4 * d + 4) + 8 * (n + 1) + n * width * 2
         mean_ms, best_ms = time_calls(fn, 5)
-        phases.append(dict(kernel="aggregate", round=m, calls_per_step=1, ms=mean_ms, best_ms=best_ms, bound="hbm",
-                           algorithmic_bytes=alg, achieved=alg / mean_ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s",
-                           edges_per_s=e / mean_ms * 1e3, traffic=measured_traffic(AGG_DRAM_TRAFFIC, AGG_SOURCES, (w.name, m))))
+        traffic = measured_traffic(AGG_DRAM_TRAFFIC, AGG_SOURCES, (w.name, m))
+        alg_gbs = alg / mean_ms / 1e6
+        ph = dict(kernel="aggregate", workload=w.name, round=m, calls_per_step=1, ms=mean_ms, best_ms=best_ms,
+                  algorithmic_bytes=alg, algorithmic_gbs=alg_gbs, edges_per_s=e / mean_ms * 1e3, traffic=traffic,
+                  dram_gbs=(traffic / mean_ms / 1e6) if traffic else None,
+                  dram_frac=(traffic / mean_ms / 1e6 / peaks["hbm_gbs"]) if traffic else None, x16=x16)
+        if traffic and traffic < 0.25 * alg:
+            ph.update(bound="l2", achieved=alg_gbs, peak=L2_PEAK_GBS, unit="GB/s",
+                      ceiling="L2 -> SM path: neighbour rows gathered from L2-resident column slabs (DRAM traffic is %.2f "
+                              "of the bytes delivered); peak = 100 %% of the profiler's lts__throughput, from the "
+                              "section capture of this kernel; the plain kernel on a 64-column matrix that fits L2 "
+                              "whole delivers %.1f TB/s in this run" % (traffic / alg, (l2_peak or 0.0) / 1e3))
+        elif traffic:
+            ph.update(bound="hbm", achieved=traffic / mean_ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s",
+                      ceiling="HBM: achieved = DRAM bytes (ncu) / time; L2 serves the rest of the %.1f TB/s delivered"
+                              % (alg_gbs / 1e3))
+        else:
+            # no DRAM counters for this workload / these sources: the bytes delivered are an upper bound of the
+            # DRAM bytes, so this fraction can exceed 1 where L2 serves part of the gather
+            ph.update(bound="hbm", achieved=alg_gbs, peak=peaks["hbm_gbs"], unit="GB/s",
+                      ceiling="HBM (no DRAM counters for this workload: achieved = bytes delivered / time)")
+        out.append(ph)
+    return out
+
+
+def phase_breakdown(w, ws, R: int, peaks, l2_peak=None):
+    """Times each entry point alone, at the shapes and launch configuration the
+    K-round run uses, and derives the roofline figures per kernel."""
+    import torch
+    from paper_2302_13053_b200 import binding as B
+    dev = "cuda"
+    rp = torch.from_numpy(w.rowptr).to(dev)
+    ci = torch.from_numpy(w.colidx).to(dev)
+    n, e = w.n_nodes, w.n_edges
+    tr = torch.from_numpy(w.train_idx).to(dev)
+    va = torch.from_numpy(w.val_idx).to(dev)
+    y = torch.from_numpy(w.labels).to(dev)
+    y_tr, y_va = y[tr.long()].contiguous(), y[va.long()].contiguous()
+    if l2_peak is None and n * 64 * 4 < 100e6:
+        l2_peak = measure_l2_gather_peak(rp, ci, n, e)
+    agg = aggregation_phases(w, ws, peaks, rp, ci, l2_peak)
+    phases = []
+    for rd, wt, ag in zip(w.round_dims(), ws, agg):
+        m = rd["round"]
+        width = rd["d_in"]
+        x16 = ag.pop("x16")
+        phases.append(ag)
         # the round's model at its training / validation / full shapes
         model = B.Mlp(rd["d_in"], rd["hidden"], w.n_classes, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
         xtr, _ = B.retexo_pack_rows(x16, tr, dim=width, ones=True)
         xva, _ = B.retexo_pack_rows(x16, va, dim=width)
         H, O = rd["hidden"], w.n_classes
         n_tr, n_va = tr.numel(), va.numel()
-        # algorithmic bytes: every product reads each operand once and writes its result once
-        # (bf16 activations and gradients, fp32 weight gradients; no transposed duplicates counted)
+        # Algorithmic bytes, counted per product: every product reads each operand once and writes its result
+        # once (bf16 activations and gradients, fp32 weight gradients).  chain_bytes counts the launch sequence
+        # as it is built instead: the class product, the loss and the gated back-propagation are one kernel
+        # (Hd read once, no logits), the ReLU bits replace the gate operand, and the weight-gradient products
+        # re-read X, Hd, dL and dHd.
         if H > 0:
             flops_step = 2.0 * n_tr * (2 * width * H + 3 * H * O)
             flops_fwd = lambda rows: 2.0 * rows * (width * H + H * O)
             bytes_fwd = lambda rows: 2.0 * (rows * width + width * H + rows * H) + 2.0 * (rows * H + H * O) + 4.0 * rows
+            opt = 7 * 4.0 * (width * H + H * O)                                  # theta, m, v in and out, gradient in
             bytes_step = (2.0 * (n_tr * width + width * H + n_tr * H)            # Hd = ReLU(X W1 + b1)
                           + 2.0 * (n_tr * H + H * O + n_tr * O)                   # logits, loss, dL
                           + 2.0 * (n_tr * O + H * O + 2 * n_tr * H)               # dHd = (dL W2^T) gated by Hd
                           + 2.0 * (n_tr * H + n_tr * O) + 4.0 * H * O             # dW2
                           + 2.0 * (n_tr * width + n_tr * H) + 4.0 * width * H     # dW1
-                          + 7 * 4.0 * (width * H + H * O))                        # optimiser: theta, m, v in and out, gradient in
+                          + opt)
+            chain_bytes = (2.0 * (n_tr * width + width * H + n_tr * H) + n_tr * H / 8.0      # forward: X, W1 in; Hd and its bits out
+                           + 2.0 * (n_tr * H + H * O) + n_tr * H / 8.0 + 2.0 * n_tr * 64 + 2.0 * n_tr * H   # fused middle
+                           + 2.0 * (n_tr * H + n_tr * 64) + 2.0 * (n_tr * width + n_tr * H)   # the two weight-gradient products
+                           + opt)
         else:
             flops_step = 2.0 * n_tr * 2 * width * O
             flops_fwd = lambda rows: 2.0 * rows * width * O
             bytes_fwd = lambda rows: 2.0 * (rows * width + width * O) + 4.0 * rows
             bytes_step = (2.0 * (n_tr * width + width * O + n_tr * O) + 2.0 * (n_tr * width + n_tr * O)
                           + 4.0 * width * O + 7 * 4.0 * width * O)
+            chain_bytes = bytes_step + 2.0 * n_tr * (64 - O) * 2
         import ctypes as C
         need = B.lib().retexo_mlp_train_step_workspace_size(C.c_int32(width), C.c_int32(H), C.c_int32(O),
                                                             C.c_int64(n_tr))
@@ -276,6 +342,8 @@ def phase_breakdown(w, ws, R: int, peaks):
         mean_ms, best_ms = time_calls(lambda: B.retexo_mlp_train_step(model, xtr, y_tr, x_has_ones=True, workspace=ws_step), 10)
         phases.append(dict(kernel="mlp_train_step", round=m, calls_per_step=R, ms=mean_ms, best_ms=best_ms,
                            traffic=measured_traffic(STEP_DRAM_TRAFFIC, STEP_SOURCES, (w.name, m)),
+                           chain_bytes=chain_bytes, chain_min_ms=chain_bytes / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                           tensor_min_ms=flops_step / (peaks["bf16_sustained"] * 1e12) * 1e3,
                            **min_time_roofline(flops_step, bytes_step, mean_ms, peaks)))
         mean_ms, best_ms = time_calls(lambda: B.retexo_embed(model, xva, y=y_va), 10)
         phases.append(dict(kernel="embed_validation", round=m, calls_per_step=0, ms=mean_ms, best_ms=best_ms,
@@ -291,7 +359,7 @@ def phase_breakdown(w, ws, R: int, peaks):
             nb = 2.0 * (n * width + width * O) + 4.0 * n * O + 4.0 * n
         phases.append(dict(kernel="embed_all_rows", round=m, calls_per_step=1, ms=mean_ms, best_ms=best_ms,
                            **min_time_roofline(fl, nb, mean_ms, peaks)))
-        del model, xtr, xva, ws_step
+        del model, xtr, xva, ws_step, x16
     part = torch.from_numpy(w.part).to(dev)
     dims = [rd["rep_dim"] for rd in w.round_dims()]
     mean_ms, best_ms = time_calls(lambda: B.retexo_cross_partition_bytes(rp, ci, part, w.n_parts, dims, 4,
@@ -302,32 +370,57 @@ def phase_breakdown(w, ws, R: int, peaks):
                        unit="GB/s"))
     for p in phases:
         p["frac"] = p["achieved"] / p["peak"]
-    return phases
+    return phases, l2_peak
 
 
-def oracle_sample(w, ws, R: int, budget_rows: int = 1536, budget_train: int = 2048):
-    """Times the CPU checker on a bounded sample of the workload and
-    extrapolates to one full step (K rounds)."""
+def second_large_graph_aggregation(peaks, l2_peak):
+    """The aggregation rounds of the other of the two largest graphs (the products-shaped GCN run), timed
+    alone like the rounds of the benchmarked workload, so that one run reports both."""
+    import torch
+    w5, ws5, gen_s = build_workload(5, 1.0)
+    rp = torch.from_numpy(w5.rowptr).to("cuda")
+    ci = torch.from_numpy(w5.colidx).to("cuda")
+    out = aggregation_phases(w5, ws5, peaks, rp, ci, l2_peak)
+    for p in out:
+        p.pop("x16", None)
+        p["frac"] = p["achieved"] / p["peak"]
+    return out
+
+
+def oracle_sample(w, ws, R: int, budget_s: float = 75.0, budget_train: int = 2048):
+    """Times the CPU checker on the workload within about budget_s seconds and scales to one full step
+    (K rounds).  Every round's aggregation and the cross-partition count run in full where a short probe
+    says they fit the budget (otherwise on sampled destination rows, scaled by edges); the training
+    iteration and the forward pass are always timed on budget_train rows and scaled by rows."""
     import oracle
     rng = np.random.default_rng(0)
     n, e = w.n_nodes, w.n_edges
     deg = np.diff(w.rowptr)
-    rows = np.sort(rng.choice(n, size=min(n, budget_rows), replace=False))
-    sample_edges = int(deg[rows].sum())
-    total = 0.0
-    detail = []
-    for rd, wt in zip(w.round_dims(), ws):
-        d = rd["rep_dim"]
-        q = w.features if rd["round"] == 1 else rng.standard_normal((n, d)).astype(np.float32)
+    gat_of = lambda wt: dict(heads=w.heads, head_dim=w.head_dim, a_src=wt["a_src"], a_dst=wt["a_dst"])
+
+    def aggregate(q, wt, rows):
         t = time.time()
         if w.aggr == 2:
-            hd = w.heads * w.head_dim
-            p = rng.standard_normal((n, hd)).astype(np.float32)
-            oracle.aggregate(2, w.rowptr, w.colidx, p, rows=rows,
-                             gat=dict(heads=w.heads, head_dim=w.head_dim, a_src=wt["a_src"], a_dst=wt["a_dst"]))
+            oracle.aggregate(2, w.rowptr, w.colidx, q, rows=rows, gat=gat_of(wt))
         else:
             oracle.aggregate(w.aggr, w.rowptr, w.colidx, q, rows=rows)
-        t_agg = (time.time() - t) * (e / max(1, sample_edges))
+        return time.time() - t
+
+    inputs = []
+    for rd in w.round_dims():
+        d = w.heads * w.head_dim if w.aggr == 2 else rd["rep_dim"]
+        inputs.append(w.features if (rd["round"] == 1 and w.aggr != 2) else rng.standard_normal((n, d)).astype(np.float32))
+    probe_rows = np.sort(rng.choice(n, size=min(n, 512), replace=False))
+    probe_edges = max(1, int(deg[probe_rows].sum()))
+    est = [aggregate(q, wt, probe_rows) * e / probe_edges for q, wt in zip(inputs, ws)]
+    est_count = e / 8e6                                           # the count walks every entry once on one core
+    full = sum(est) + est_count <= 0.75 * budget_s
+    rows = None if full else np.sort(rng.choice(n, size=min(n, 1536), replace=False))
+    sample_edges = e if full else int(deg[rows].sum())
+    total = 0.0
+    detail = []
+    for rd, wt, q in zip(w.round_dims(), ws, inputs):
+        t_agg = aggregate(q, wt, rows) * (e / max(1, sample_edges))
         n_tr = len(w.train_idx)
         sub = min(n_tr, budget_train)
         x = rng.standard_normal((sub, rd["d_in"])).astype(np.float32)
@@ -342,7 +435,22 @@ def oracle_sample(w, ws, R: int, budget_rows: int = 1536, budget_train: int = 20
         t_round = t_agg + R * (t_step + t_fwd_row * len(w.val_idx)) + t_fwd_row * (n + 2 * len(w.test_idx))
         detail.append(dict(round=rd["round"], aggregate_s=t_agg, train_step_s=t_step, round_s=t_round))
         total += t_round
-    return total, detail, "aggregation of %d sampled rows (%d edges) and one train step + forward on %d train rows per round, scaled to the full graph and R=%d" % (len(rows), sample_edges, min(len(w.train_idx), budget_train), R)
+    count_s = None
+    if full:
+        t = time.time()
+        oracle.cross_partition(w.rowptr, w.colidx, w.part, w.n_parts, [rd["rep_dim"] for rd in w.round_dims()], 4)
+        count_s = time.time() - t
+        total += count_s
+    else:
+        total += est_count
+    detail.append(dict(count_s=count_s if count_s is not None else est_count))
+    what = ("every round's aggregation and the cross-partition count in full" if full else
+            "aggregation of %d sampled rows (%d edges), scaled by edges; the count estimated" % (len(rows), sample_edges))
+    sample = "%s; one training iteration + forward on %d train rows per round, scaled by rows to %d rows and R=%d" % (
+        what, min(len(w.train_idx), budget_train), len(w.train_idx), R)
+    kind = ("oracle, aggregation and count in full, training step extrapolated from %d rows" % min(len(w.train_idx), budget_train)
+            if full else "oracle, aggregation and training step extrapolated from samples")
+    return total, detail, sample, kind
 
 
 def run_reference(args):
@@ -353,11 +461,13 @@ def run_reference(args):
     w, ws, _ = build_workload(args.config, args.scale)
     R = args.iters or w.R
     times = []
-    sample = ""
+    sample = kind = ""
+    # the whole run (warm-up and timed steps) is kept to a few minutes: each step gets its share of ~150 s
+    per_step = max(4.0, 150.0 / max(1, args.steps + args.warmup))
     for _ in range(args.warmup):
-        oracle_sample(w, ws, R, budget_rows=256, budget_train=256)
+        oracle_sample(w, ws, R, budget_s=min(per_step, 8.0), budget_train=256)
     for _ in range(args.steps):
-        t, detail, sample = oracle_sample(w, ws, R)
+        t, detail, sample, kind = oracle_sample(w, ws, R, budget_s=per_step)
         times.append(t)
     step_s = statistics.mean(times)
     value = w.K * w.n_edges / step_s
@@ -365,8 +475,8 @@ def run_reference(args):
                 warmup=args.warmup, ms_per_step=step_s * 1e3, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic",
                 config=dict(workload=w.name, n_nodes=w.n_nodes, n_edges=w.n_edges, K=w.K, R=R,
-                            note="CPU checker timed on a bounded sample per step and extrapolated"),
-                cpu_baseline=dict(value=value, unit=UNIT, cores=oracle.n_threads(), kind="oracle", sample=sample),
+                            note="CPU checker; each step is a bounded sample of the workload, scaled to the whole"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=oracle.n_threads(), kind=kind, sample=sample),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
                 gpu_launches=0)
     print(json.dumps(line))
@@ -384,6 +494,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
+    ap.add_argument("--no-second-graph", action="store_true",
+                    help="with the default workload, do not time the products-shaped graph's aggregation rounds as well")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
@@ -477,7 +589,7 @@ def main():
                             bytes_total=res["counts"]["bytes_total"]))
 
     if not args.no_breakdown:
-        phases = phase_breakdown(w, ws, R, peaks)
+        phases, l2_peak = phase_breakdown(w, ws, R, peaks)
         for p in phases:
             p["share_of_step"] = p["ms"] * p["calls_per_step"] / ms_per_step
         dom = max(phases, key=lambda p: p["share_of_step"])
@@ -487,22 +599,29 @@ def main():
                                 share_of_step=dom["share_of_step"],
                                 algorithmic_bytes=dom.get("algorithmic_bytes"), flops=dom.get("flops"),
                                 tflops=dom.get("tflops"), ms=dom["ms"], min_ms=dom.get("min_ms"),
-                                note="one training iteration (tc_gemm_kernel launches + reduce_update_kernel); min-time "
-                                     "roofline: bytes / HBM peak exceeds flops / tensor peak, so HBM is the bound"
+                                chain_bytes=dom.get("chain_bytes"), chain_min_ms=dom.get("chain_min_ms"),
+                                tensor_min_ms=dom.get("tensor_min_ms"),
+                                note="one training iteration (forward product, fused class product / loss / gated "
+                                     "back-propagation, two weight-gradient products, reduce + update); min-time roofline "
+                                     "counted per product: bytes / HBM peak exceeds flops / tensor peak, so HBM is the "
+                                     "bound; chain_* counts the bytes of the launch sequence as built"
                                 if dom["kernel"] == "mlp_train_step" and dom["bound"] == "hbm" else
-                                "one training iteration (tc_gemm_kernel launches): tensor-bound"
+                                "one training iteration: tensor-bound"
                                 if dom["kernel"] == "mlp_train_step" else "CSR gather-reduce (aggregation kernels)")
-        # the memory-bound side of the path, against the measured HBM copy bandwidth
+        # the memory-bound side of the path, each round against the ceiling that binds it; with the default
+        # workload the rounds of the other large graph follow
+        agg = [p for p in phases if p["kernel"] == "aggregate"]
+        if args.config == 4 and args.scale == 1.0 and world == 1 and not args.no_second_graph:
+            torch.cuda.empty_cache()
+            agg += second_large_graph_aggregation(peaks, l2_peak)
         line["roofline_aggregation"] = [
-            dict(round=p["round"], bound="hbm", achieved=p["achieved"], peak=p["peak"], unit="GB/s", frac=p["frac"],
-                 traffic=p.get("traffic"), ms=p["ms"], edges_per_s=p["edges_per_s"],
-                 dram_gbs=(p["traffic"] / p["ms"] / 1e6) if p.get("traffic") else None,
-                 dram_frac=(p["traffic"] / p["ms"] / 1e6 / p["peak"]) if p.get("traffic") else None,
-                 ceiling=("l2: column slabs, neighbour rows gathered from L2 (algorithmic bytes exceed DRAM traffic)"
-                          if p.get("traffic") and p["traffic"] < 0.25 * p["algorithmic_bytes"] else
-                          "hbm: DRAM traffic at the copy bandwidth, the L2 hit rate sets the algorithmic rate")
-                 if p.get("traffic") else None)
-            for p in phases if p["kernel"] == "aggregate"]
+            dict(workload=p.get("workload", w.name), round=p["round"], bound=p["bound"], achieved=p["achieved"],
+                 peak=p["peak"], unit="GB/s", frac=p["frac"], traffic=p.get("traffic"), ms=p["ms"],
+                 edges_per_s=p["edges_per_s"], algorithmic_gbs=p["algorithmic_gbs"], dram_gbs=p["dram_gbs"],
+                 dram_frac=p["dram_frac"], hbm_peak=peaks["hbm_gbs"], ceiling=p["ceiling"])
+            for p in agg]
+        line["l2"] = dict(peak_gbs=L2_PEAK_GBS, peak_source="ncu lts__throughput, profiles/agg_kernels_cfg4.txt",
+                          plain_gather_on_l2_resident_matrix_gbs=l2_peak)
         line["phases"] = [dict(kernel=p["kernel"], round=p["round"], ms=round(p["ms"], 4), calls=p["calls_per_step"],
                                share=round(p["share_of_step"], 4), bound=p["bound"], achieved=round(p["achieved"], 2),
                                unit=p["unit"], frac=round(p["frac"], 4),
@@ -510,9 +629,9 @@ def main():
                           for p in phases]
     if not args.no_cpu_baseline:
         import oracle
-        t, detail, sample = oracle_sample(w, ws, R)
-        line["cpu_baseline"] = dict(value=edges_per_step / t, unit=UNIT, cores=oracle.n_threads(), kind="oracle",
-                                    sample=sample, est_step_s=t)
+        t, detail, sample, kind = oracle_sample(w, ws, R)
+        line["cpu_baseline"] = dict(value=edges_per_step / t, unit=UNIT, cores=oracle.n_threads(), kind=kind,
+                                    sample=sample, est_step_s=t, detail=detail)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -359,10 +359,13 @@ def make_config(index: int, seed: int = 0, scale: float = 1.0) -> Workload:
         mean_deg = 2.0 * n_und / n
         w = _power_law_weights(n, 2.5, min(20000.0, n / 6) / mean_deg)
         rowptr, colidx = random_graph(s_graph, n, n_und, labels, w, 0.56, None)
-        feats = _gaussian_features(s_feat, labels, 602, 0.2)
+        feats = _gaussian_features(s_feat, labels, 602, 2.0)
         # Graph and features follow the block; the label a node is observed with is its block for 88 % of the
         # nodes and a uniform draw for the rest.  Without this the mean over ~490 neighbours identifies the
-        # block almost surely and test accuracy saturates above 99 %, where an accuracy comparison says little.
+        # block almost surely and test accuracy saturates above 99 %, where an accuracy comparison says little;
+        # with it accuracy levels off near 0.88, and a class-mean shift of 2 (two standard deviations along the
+        # class direction) keeps the validation curves flat around their maximum, so that which iterate is kept
+        # does not hinge on rounding.
         noisy = s_noise.random(n) < 0.12
         labels = np.where(noisy, s_noise.integers(0, 41, size=n), labels).astype(np.int32)
         tr, va, te = _split_fraction(s_split, n, 0.66, 0.10)

@@ -49,5 +49,5 @@ def test_launch_count_formula_matches_the_round_structure():
     w = wl.make_config(1, scale=0.2)
     a, b = bench.launches_per_step(w, 10), bench.launches_per_step(w, 20)
     per_iter = (b - a) / 10
-    assert per_iter == (6 + 6 + 3)          # two rounds with a hidden layer, one without; validation rides along
+    assert per_iter == (5 + 5 + 3)          # two rounds with a hidden layer, one without; validation rides along
                                             # and is booked by the update kernel's last block
