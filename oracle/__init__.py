@@ -70,6 +70,18 @@ def bf16_round(a: np.ndarray) -> np.ndarray:
     return np.array([f(float(v)) for v in a.ravel()], dtype=np.float32).reshape(a.shape)
 
 
+def bf16_round_array(a: np.ndarray) -> np.ndarray:
+    """bf16_round for whole arrays (round to nearest, ties to even, on the top 16 bits of the binary32
+    pattern; NaN stays NaN), in numpy integer arithmetic; returned as fp32."""
+    a = _f32(a)
+    u = a.view(np.uint32).astype(np.uint64)
+    special = (u & 0x7f800000) == 0x7f800000
+    r = (u + 0x7fff + ((u >> 16) & 1)) & 0xffff0000
+    nan = special & ((u & 0x007fffff) != 0)
+    r = np.where(special, np.where(nan, (u | 0x00400000) & 0xffff0000, u & 0xffff0000), r)
+    return r.astype(np.uint32).view(np.float32).reshape(a.shape)
+
+
 # ---------------------------------------------------------------- aggregation
 def aggregate(aggr: int, rowptr: np.ndarray, colidx: np.ndarray, q: np.ndarray,
               rows: Optional[np.ndarray] = None, gat: Optional[Dict] = None,
@@ -124,6 +136,28 @@ def aggregate(aggr: int, rowptr: np.ndarray, colidx: np.ndarray, q: np.ndarray,
         _check(rc, "oracle_aggregate_gat")
         return (out, ae, aself) if return_alpha else out
     raise ValueError("unknown aggregator")
+
+
+def gat_backward(rowptr: np.ndarray, colidx: np.ndarray, p: np.ndarray, gat: Dict, dz: np.ndarray):
+    """Backward of the GAT aggregation: given dz = dLoss/dZ [n, heads*dh] (zero rows outside the loss),
+    returns (dp [n, heads*dh], da_src [heads, dh], da_dst [heads, dh]) in double."""
+    n = rowptr.shape[0] - 1
+    rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+    colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+    p = _f32(p)
+    heads, dh = int(gat["heads"]), int(gat["head_dim"])
+    assert p.shape[1] == heads * dh
+    a_src, a_dst = _f32(gat["a_src"]), _f32(gat["a_dst"])
+    dz = np.ascontiguousarray(dz, dtype=np.float64)
+    assert dz.shape == (n, heads * dh)
+    dp = np.zeros((n, heads * dh), dtype=np.float64)
+    da_src = np.zeros((heads, dh), dtype=np.float64)
+    da_dst = np.zeros((heads, dh), dtype=np.float64)
+    rc = lib().oracle_gat_backward(C.c_int64(n), _p(rowptr), _p(colidx), _p(p), C.c_int64(p.shape[1]), C.c_int32(heads),
+                                   C.c_int32(dh), _p(a_src), _p(a_dst), C.c_double(float(gat.get("negative_slope", 0.2))),
+                                   C.c_int32(int(gat.get("add_self_loop", 1))), _p(dz), _p(dp), _p(da_src), _p(da_dst))
+    _check(rc, "oracle_gat_backward")
+    return dp, da_src, da_dst
 
 
 # ---------------------------------------------------------------- dropout generator
@@ -184,6 +218,25 @@ class Mlp:
             d["b2"] = t[o:o + self.n_classes]
         return d
 
+    def train_step_dx(self, x: np.ndarray, y: np.ndarray, row_idx: Optional[np.ndarray] = None):
+        """One full-batch step that also returns the gradients: (loss, grad laid out like theta,
+        dX [n_rows, d_in] = gradient with respect to the batch rows), all before the update."""
+        x = _f32(x)
+        y = np.ascontiguousarray(y, dtype=np.int32)
+        ri = None if row_idx is None else np.ascontiguousarray(row_idx, dtype=np.int32)
+        n_rows = x.shape[0] if ri is None else ri.shape[0]
+        loss = C.c_double(0.0)
+        grad = np.zeros_like(self.theta)
+        dx = np.zeros((n_rows, self.d_in), dtype=np.float64)
+        self.step += 1
+        rc = lib().oracle_mlp_train_step_dx(
+            C.c_int32(self.d_in), C.c_int32(self.hidden), C.c_int32(self.n_classes), _p(self.theta), _p(self.m),
+            _p(self.v), C.c_int32(self.optimizer), C.c_double(self.lr), C.c_double(self.beta1), C.c_double(self.beta2),
+            C.c_double(self.eps), C.c_int64(self.step), C.c_int32(int(self.round_bf16)), _p(x), C.c_int64(x.shape[1]),
+            _p(ri), C.c_int64(n_rows), _p(y), C.byref(loss), _p(grad), _p(dx))
+        _check(rc, "oracle_mlp_train_step_dx")
+        return loss.value, grad, dx
+
     def train_step(self, x: np.ndarray, y: np.ndarray, row_idx: Optional[np.ndarray] = None,
                    return_grad: bool = False, dropout: float = 0.0, dropout_seed: int = 0):
         """One full-batch step on rows x[row_idx] (all rows of x if None) with
@@ -238,6 +291,79 @@ class Mlp:
             C.byref(correct))
         _check(rc, "oracle_embed")
         return dict(hidden=hid, logits=lg, pred=pred, correct=int(correct.value))
+
+
+class GatLayer:
+    """One RetexoGAT layer with its aggregator trained (Section 2.2: AGGR may have trainable parameters;
+    Section 3.1: a round trains the whole layer): projection W_att [d x heads*dh], attention vectors
+    a_src, a_dst [heads x dh], and the per-node model (f_theta, C_theta) on the aggregated rows.
+    The cross-worker exchange of a round fixes q = Q^{m-1}; the aggregation itself is local and is
+    redone with the current parameters in every iteration."""
+
+    def __init__(self, rowptr, colidx, gat: Dict, w_att, a_src, a_dst, mlp: Mlp):
+        self.rowptr = np.ascontiguousarray(rowptr, dtype=np.int64)
+        self.colidx = np.ascontiguousarray(colidx, dtype=np.int32)
+        self.heads, self.dh = int(gat["heads"]), int(gat["head_dim"])
+        self.slope = float(gat.get("negative_slope", 0.2))
+        self.d = int(np.asarray(w_att).shape[0])
+        self.hd = self.heads * self.dh
+        self.att = np.ascontiguousarray(np.concatenate([np.asarray(w_att, dtype=np.float64).ravel(),
+                                                        np.asarray(a_src, dtype=np.float64).ravel(),
+                                                        np.asarray(a_dst, dtype=np.float64).ravel()]))
+        self.att_m, self.att_v = np.zeros_like(self.att), np.zeros_like(self.att)
+        self.mlp = mlp
+
+    def copy(self) -> "GatLayer":
+        o = GatLayer.__new__(GatLayer)
+        o.__dict__.update(self.__dict__)
+        o.att, o.att_m, o.att_v = self.att.copy(), self.att_m.copy(), self.att_v.copy()
+        o.mlp = self.mlp.copy()
+        return o
+
+    def parts(self):
+        nw = self.d * self.hd
+        return (self.att[:nw].reshape(self.d, self.hd), self.att[nw:nw + self.hd].reshape(self.heads, self.dh),
+                self.att[nw + self.hd:].reshape(self.heads, self.dh))
+
+    def _gat(self) -> Dict:
+        _, a_src, a_dst = self.parts()
+        return dict(heads=self.heads, head_dim=self.dh, negative_slope=self.slope, add_self_loop=1,
+                    a_src=a_src.astype(np.float32), a_dst=a_dst.astype(np.float32))
+
+    def project(self, q: np.ndarray) -> np.ndarray:
+        """P = Q W_att, a bias-free product under the operand-rounding contract; fp32 result."""
+        w_att, _, _ = self.parts()
+        proj = Mlp(self.d, 0, self.hd, w_att, np.zeros(self.hd), round_bf16=self.mlp.round_bf16)
+        return proj.embed(q)["logits"]
+
+    def aggregate(self, q: np.ndarray, rows: Optional[np.ndarray] = None) -> np.ndarray:
+        return aggregate(GAT, self.rowptr, self.colidx, self.project(q), rows=rows, gat=self._gat())
+
+    def train_step(self, q: np.ndarray, y: np.ndarray, train_idx: np.ndarray, return_grad: bool = False):
+        """One full-batch iteration of the whole layer on the rows train_idx: forward through projection,
+        attention and the per-node model, loss, backward to every parameter, one optimiser update of all of
+        them.  Returns the loss before the update (and the gradients [att | theta] if asked)."""
+        q = _f32(q)
+        n = q.shape[0]
+        rnd = self.mlp.round_bf16
+        p = self.project(q)
+        gat = self._gat()
+        rows = np.ascontiguousarray(train_idx, dtype=np.int64)
+        x = aggregate(GAT, self.rowptr, self.colidx, p, rows=rows, gat=gat)
+        loss, grad_mlp, dx = self.mlp.train_step_dx(x, y)            # (updates the per-node model)
+        dz = np.zeros((n, self.hd), dtype=np.float64)
+        dz[rows] = dx
+        dp, da_src, da_dst = gat_backward(self.rowptr, self.colidx, p, gat, dz)
+        # dW_att = Q^T dP: one more product, operands rounded like the others
+        qq = bf16_round_array(q).astype(np.float64) if rnd else q.astype(np.float64)
+        dd = bf16_round_array(dp.astype(np.float32)).astype(np.float64) if rnd else dp
+        grad_att = np.concatenate([(qq.T @ dd).ravel(), da_src.ravel(), da_dst.ravel()])
+        m = self.mlp
+        rc = lib().oracle_apply_update(C.c_int64(self.att.shape[0]), _p(self.att), _p(self.att_m), _p(self.att_v),
+                                       _p(np.ascontiguousarray(grad_att)), C.c_int32(m.optimizer), C.c_double(m.lr),
+                                       C.c_double(m.beta1), C.c_double(m.beta2), C.c_double(m.eps), C.c_int64(m.step))
+        _check(rc, "oracle_apply_update")
+        return (loss, np.concatenate([grad_att, grad_mlp])) if return_grad else loss
 
 
 # ---------------------------------------------------------------- counting
@@ -306,7 +432,8 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
               optimizer: int = ADAM, round_bf16: bool = True, eval_every: int = 1,
               part=None, n_parts: int = 0, forced_best_iter: Optional[Sequence[int]] = None,
               dropout: float = 0.0, dropout_seed: int = 0,
-              forced_theta: Optional[Sequence[np.ndarray]] = None) -> Dict:
+              forced_theta: Optional[Sequence[np.ndarray]] = None, train_attention: bool = False,
+              forced_att: Optional[Sequence[np.ndarray]] = None) -> Dict:
     """Lazy message passing (Section 3.1): for each layer m = 1..K, one
     message-passing round builds the layer's inputs, the layer (with a
     temporary classifier unless it is the last) is trained alone for R
@@ -328,7 +455,12 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
     iterations two correct implementations hold slightly different weights and
     every later round would start from different inputs; with the weights of the
     implementation under test forced in, each round is compared from the same
-    starting point."""
+    starting point.
+
+    train_attention (GAT only): the round trains the whole layer, i.e. the projection and the
+    attention vectors together with the per-node model, re-aggregating locally in every iteration
+    (GatLayer); without it they stay at their given draws and the aggregation runs once per round.
+    forced_att: like forced_theta, for the kept [W_att | a_src | a_dst] of each round."""
     labels = np.ascontiguousarray(labels, dtype=np.int32)
     q = _f32(features)
     y_tr, y_va, y_te = labels[train_idx], labels[val_idx], labels[test_idx]
@@ -342,6 +474,49 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
         report["counts"] = cross_partition(rowptr, colidx, part, n_parts, dims, 4)
     for m in range(1, K + 1):
         w = weights[m - 1]
+        if aggr == GAT and train_attention:
+            hid = hidden if m < K else 0
+            hd = w["w_att"].shape[1]
+            layer = GatLayer(rowptr, colidx, gat, w["w_att"], w["a_src"], w["a_dst"],
+                             Mlp(hd, hid, n_classes, w["w1"], w["b1"], w.get("w2"), w.get("b2"), optimizer=optimizer,
+                                 lr=lr, round_bf16=round_bf16))
+            best, best_correct, best_iter = None, -1, -1
+            losses, val_hist = [], []
+            for r in range(1, R + 1):
+                losses.append(layer.train_step(q, y_tr, train_idx))
+                report["n_steps"] += 1
+                report["n_aggregations"] += 1
+                if r % eval_every == 0 or r == R:
+                    c = layer.mlp.embed(layer.aggregate(q, rows=np.asarray(val_idx, dtype=np.int64)), y=y_va,
+                                        want_logits=False)["correct"]
+                    val_hist.append(c)
+                    if forced_best_iter is not None:
+                        if r == forced_best_iter[m - 1]:
+                            best, best_correct, best_iter = layer.copy(), c, r
+                    elif c > best_correct:
+                        best, best_correct, best_iter = layer.copy(), c, r
+            te = np.asarray(test_idx, dtype=np.int64)
+            last_test = layer.mlp.embed(layer.aggregate(q, rows=te), y=y_te, want_logits=False)["correct"]
+            own_best = best
+            if forced_theta is not None or forced_att is not None:
+                best = best.copy()
+                if forced_theta is not None:
+                    best.mlp.theta = np.ascontiguousarray(forced_theta[m - 1], dtype=np.float64).copy()
+                if forced_att is not None:
+                    best.att = np.ascontiguousarray(forced_att[m - 1], dtype=np.float64).copy()
+            best_test = best.mlp.embed(best.aggregate(q, rows=te), y=y_te, want_logits=False)["correct"]
+            x = best.aggregate(q)
+            rd = dict(round=m, losses=np.asarray(losses), val_correct=np.asarray(val_hist), best_iter=best_iter,
+                      best_val_correct=best_correct, test_correct_best=best_test, test_correct_last=last_test,
+                      model=best.mlp, own_model=own_best.mlp, layer=best, own_layer=own_best, x=x)
+            if m < K:
+                q = best.mlp.embed(x, want_hidden=True, want_logits=False)["hidden"]
+                rd["q_out"] = q
+            else:
+                fin = best.mlp.embed(x, want_logits=True)
+                rd["logits"], rd["pred"] = fin["logits"], fin["pred"]
+            report["rounds"].append(rd)
+            continue
         if aggr == GAT:
             proj = Mlp(q.shape[1], 0, w["w_att"].shape[1], w["w_att"], np.zeros(w["w_att"].shape[1]),
                        round_bf16=round_bf16)

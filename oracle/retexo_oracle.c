@@ -228,6 +228,96 @@ int oracle_aggregate_gat(int64_t n, const int64_t *rowptr, const int32_t *colidx
     return failed ? ORACLE_NO_MEM : ORACLE_OK;
 }
 
+/* Backward of the GAT aggregation above (Section 2.2: "AGGR may have
+ * trainable parameters"; Section 3.1: the whole layer, AGGR included, is what a
+ * round trains).  dz [n x heads*head_dim] is the gradient of the loss with
+ * respect to the aggregation's output Z (zero rows for nodes outside the loss).
+ * With e_uv = LeakyReLU(z_uv), z_uv = s_u + t_v, alpha = softmax_u(e_uv),
+ * Z_v = sum_u alpha_uv p_u, the chain rule gives, per head,
+ *   dalpha_uv = <dz_v, p_u>
+ *   de_uv     = alpha_uv (dalpha_uv - sum_w alpha_wv dalpha_wv)
+ *   dz_uv     = de_uv * (z_uv > 0 ? 1 : slope)
+ *   ds_u = sum_v dz_uv,  dt_v = sum_u dz_uv
+ *   dp_u = sum_v alpha_uv dz_v + ds_u a_src + dt_u a_dst
+ *   da_src = sum_u ds_u p_u,  da_dst = sum_v dt_v p_v
+ * (the sums over v run over the destinations that attend over u, u itself
+ * included with the self loop).  Everything is carried in double; dp
+ * [n x heads*head_dim], da_src and da_dst [heads x head_dim] are outputs. */
+int oracle_gat_backward(int64_t n, const int64_t *rowptr, const int32_t *colidx,
+                        const float *p, int64_t ldp, int32_t heads, int32_t head_dim,
+                        const float *a_src, const float *a_dst, double slope, int32_t add_self_loop,
+                        const double *dz, double *dp, double *da_src, double *da_dst)
+{
+    int32_t dim = heads * head_dim;
+    if (n < 0 || heads <= 0 || head_dim <= 0 || ldp < dim || !dz || !dp || !da_src || !da_dst) return ORACLE_BAD_ARG;
+    size_t nh = (size_t)(n > 0 ? n : 1) * heads;
+    double *s = (double *)malloc(sizeof(double) * nh), *t = (double *)malloc(sizeof(double) * nh);
+    double *ds = (double *)calloc(nh, sizeof(double)), *dt = (double *)calloc(nh, sizeof(double));
+    if (!s || !t || !ds || !dt) { free(s); free(t); free(ds); free(dt); return ORACLE_NO_MEM; }
+    for (int64_t u = 0; u < n; ++u)
+        for (int32_t k = 0; k < heads; ++k) {
+            double ss = 0.0, tt = 0.0;
+            for (int32_t j = 0; j < head_dim; ++j) {
+                double x = (double)p[u * ldp + k * head_dim + j];
+                ss += (double)a_src[k * head_dim + j] * x;
+                tt += (double)a_dst[k * head_dim + j] * x;
+            }
+            s[u * heads + k] = ss;
+            t[u * heads + k] = tt;
+        }
+    for (int64_t i = 0; i < n * (int64_t)dim; ++i) dp[i] = 0.0;
+    for (int32_t i = 0; i < dim; ++i) { da_src[i] = 0.0; da_dst[i] = 0.0; }
+    int failed = 0;
+    for (int64_t v = 0; v < n && !failed; ++v) {
+        int64_t deg = rowptr[v + 1] - rowptr[v];
+        int64_t m = deg + (add_self_loop ? 1 : 0);
+        if (m == 0) continue;
+        double *alpha = (double *)malloc(sizeof(double) * (size_t)m);
+        double *dalpha = (double *)malloc(sizeof(double) * (size_t)m);
+        if (!alpha || !dalpha) { free(alpha); free(dalpha); failed = 1; break; }
+        for (int32_t k = 0; k < heads; ++k) {
+            const double *g = dz + v * dim + k * head_dim;
+            double mx = -INFINITY, den = 0.0, c = 0.0;
+            for (int64_t a = 0; a < m; ++a) {
+                int64_t u = a < deg ? (int64_t)colidx[rowptr[v] + a] : v;
+                double z = s[u * heads + k] + t[v * heads + k];
+                alpha[a] = z > 0.0 ? z : slope * z;
+                if (alpha[a] > mx) mx = alpha[a];
+            }
+            for (int64_t a = 0; a < m; ++a) { alpha[a] = exp(alpha[a] - mx); den += alpha[a]; }
+            for (int64_t a = 0; a < m; ++a) {
+                int64_t u = a < deg ? (int64_t)colidx[rowptr[v] + a] : v;
+                alpha[a] /= den;
+                double d = 0.0;
+                for (int32_t j = 0; j < head_dim; ++j) d += g[j] * (double)p[u * ldp + k * head_dim + j];
+                dalpha[a] = d;
+                c += alpha[a] * d;
+            }
+            for (int64_t a = 0; a < m; ++a) {
+                int64_t u = a < deg ? (int64_t)colidx[rowptr[v] + a] : v;
+                double z = s[u * heads + k] + t[v * heads + k];
+                double dzz = alpha[a] * (dalpha[a] - c) * (z > 0.0 ? 1.0 : slope);
+                ds[u * heads + k] += dzz;
+                dt[v * heads + k] += dzz;
+                for (int32_t j = 0; j < head_dim; ++j) dp[u * dim + k * head_dim + j] += alpha[a] * g[j];
+            }
+        }
+        free(alpha);
+        free(dalpha);
+    }
+    for (int64_t x = 0; x < n && !failed; ++x)
+        for (int32_t k = 0; k < heads; ++k)
+            for (int32_t j = 0; j < head_dim; ++j) {
+                double px = (double)p[x * ldp + k * head_dim + j];
+                dp[x * dim + k * head_dim + j] += ds[x * heads + k] * (double)a_src[k * head_dim + j] +
+                                                  dt[x * heads + k] * (double)a_dst[k * head_dim + j];
+                da_src[k * head_dim + j] += ds[x * heads + k] * px;
+                da_dst[k * head_dim + j] += dt[x * heads + k] * px;
+            }
+    free(s); free(t); free(ds); free(dt);
+    return failed ? ORACLE_NO_MEM : ORACLE_OK;
+}
+
 /* ================================================================== */
 /* Per-node model of one round (Section 3.1): f_theta = Linear+ReLU,   */
 /* temporary classifier C_theta = Linear; last round: one Linear.      */
@@ -394,7 +484,7 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
                            int64_t step, int32_t round_bf16,
                            const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
                            const int32_t *y, double *loss_out, double *grad_out,
-                           double drop_p, uint64_t drop_seed)
+                           double drop_p, uint64_t drop_seed, double *dx_out)
 {
     if (d_in <= 0 || n_classes <= 0 || hidden < 0 || n_rows <= 0 || ldx < d_in) return ORACLE_BAD_ARG;
     if (drop_p < 0.0 || drop_p >= 1.0) return ORACLE_BAD_ARG;
@@ -461,6 +551,19 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
     for (int64_t i = 0; i < n_rows; ++i) loss += row_loss[i];
     loss /= (double)n_rows;
 
+    /* gradient with respect to the batch itself, dX = d1 W1^T (needed when what produces X is trained too,
+     * e.g. an aggregator with parameters): one more matrix product, operands d1 and W1 rounded like the others */
+    if (dx_out) {
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < n_rows; ++i)
+            for (int32_t k = 0; k < d_in; ++k) {
+                double acc = 0.0;
+                const double *wrow = w1r + (int64_t)k * out1;
+                for (int32_t j = 0; j < out1; ++j) acc += opnd(d1[i * out1 + j], round_bf16) * wrow[j];
+                dx_out[i * d_in + k] = acc;
+            }
+    }
+
     /* weight gradients: sums over batch rows, taken in fixed chunks of rows
      * that are then added in chunk order */
     double *part = (double *)calloc((size_t)GRAD_CHUNKS * (size_t)nt, sizeof(double));
@@ -518,7 +621,20 @@ int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
                           const int32_t *y, double *loss_out, double *grad_out)
 {
     return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
-                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0);
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, NULL);
+}
+
+/* The same step, also returning dX [n_rows x d_in], the gradient of the loss with respect to the batch
+ * rows (taken with the weights as they are before the update). */
+int oracle_mlp_train_step_dx(int32_t d_in, int32_t hidden, int32_t n_classes,
+                             double *theta, double *adam_m, double *adam_v,
+                             int32_t optimizer, double lr, double beta1, double beta2, double eps,
+                             int64_t step, int32_t round_bf16,
+                             const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                             const int32_t *y, double *loss_out, double *grad_out, double *dx_out)
+{
+    return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, dx_out);
 }
 
 /* The same step with dropout on the hidden units: Hd = ReLU(X W1 + b1) .* keep,
@@ -533,7 +649,7 @@ int oracle_mlp_train_step_dropout(int32_t d_in, int32_t hidden, int32_t n_classe
                                   double drop_p, uint64_t drop_seed)
 {
     return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
-                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, drop_p, drop_seed);
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, drop_p, drop_seed, NULL);
 }
 
 /* Forward of the trained per-node model over a set of rows.

@@ -85,3 +85,28 @@ def test_forced_weights_hook_feeds_the_given_weights_forward_and_leaves_the_trai
     np.testing.assert_array_equal(other["rounds"][0]["model"].theta, bumped[0])
     assert np.abs(other["rounds"][1]["x"] - free["rounds"][1]["x"]).max() > 1e-3
     assert abs(other["rounds"][1]["losses"][0] - free["rounds"][1]["losses"][0]) > 1e-6
+
+
+def test_trainable_attention_loop_retrains_the_aggregator_every_iteration():
+    """RetexoGAT with its aggregator trained (Section 2.2 / 3.1): K x R local aggregations instead of K, the
+    attention parameters move, and the first iteration's loss equals the frozen-attention run's (same
+    initial parameters, same forward)."""
+    w = wl.make_config(3, scale=0.03)
+    gat = dict(heads=w.heads, head_dim=w.head_dim, negative_slope=w.negative_slope, add_self_loop=1)
+    ws = wl.initial_weights(w)
+    args = (w.aggr, w.K, 5, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels, w.train_idx,
+            w.val_idx, w.test_idx, ws)
+    frozen = oracle.lmp_train(*args, gat=gat)
+    trained = oracle.lmp_train(*args, gat=gat, train_attention=True)
+    assert frozen["n_aggregations"] == w.K and trained["n_aggregations"] == w.K * 5
+    assert abs(trained["rounds"][0]["losses"][0] - frozen["rounds"][0]["losses"][0]) < 1e-9
+    assert abs(trained["rounds"][0]["losses"][-1] - frozen["rounds"][0]["losses"][-1]) > 1e-7
+    layer = trained["rounds"][0]["layer"]
+    w_att, a_src, a_dst = layer.parts()
+    assert np.abs(w_att - ws[0]["w_att"]).max() > 1e-4 and np.abs(a_src - ws[0]["a_src"]).max() > 1e-4
+    assert trained["rounds"][-1]["logits"].shape == (w.n_nodes, w.n_classes)
+    # the forcing hooks hand the given attention parameters on
+    same = oracle.lmp_train(*args, gat=gat, train_attention=True,
+                            forced_att=[r["layer"].att for r in trained["rounds"]],
+                            forced_theta=[r["model"].theta for r in trained["rounds"]])
+    np.testing.assert_array_equal(same["rounds"][-1]["logits"], trained["rounds"][-1]["logits"])
