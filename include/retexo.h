@@ -128,6 +128,23 @@ int retexo_aggregate(const retexo_csr* g, int32_t type,
                      void* out_bf16, int64_t ldout_bf16,
                      void* workspace, size_t workspace_bytes, void* stream);
 
+size_t retexo_gat_backward_workspace_size(int64_t n_nodes, int32_t heads, int32_t dim);
+
+/* Backward of RETEXO_GAT, for rounds that train the aggregator as well (Section 2.2: "AGGR may have
+ * trainable parameters"; Section 3.1: a round trains the whole layer): given dz = dLoss / dOut
+ * (fp32 [n x lddz]; rows of nodes outside the loss are zero) and the same p and parameters the forward
+ * pass took, computes
+ *   dp      fp32 [n x lddp] and / or bf16 [n x lddp_bf16] (either may be NULL, not both): dLoss / dp,
+ *           through the weighted sum and through both score terms;
+ *   da_src, da_dst  fp32 [heads x head_dim]: gradients of the attention vectors.
+ * Scores, soft-max and every sum are fp32; sums run in CSR order per row, the parameter gradients are
+ * summed per thread block and then in block order (deterministic).  The graph must be symmetric (the rows
+ * that attend over u are read off u's own row).  heads <= 8, heads * head_dim <= 256.
+ * Errors: INVALID_ARG, WORKSPACE, UNSUPPORTED. */
+int retexo_gat_backward(const retexo_csr* g, const float* p, int64_t ldp, const retexo_gat_params* gat,
+                        const float* dz, int64_t lddz, float* dp, int64_t lddp, void* dp_bf16, int64_t lddp_bf16,
+                        float* da_src, float* da_dst, void* workspace, size_t workspace_bytes, void* stream);
+
 /* --------------------------------------------------------- per-node model */
 typedef enum retexo_optimizer { RETEXO_SGD = 0, RETEXO_ADAM = 1 } retexo_optimizer;
 

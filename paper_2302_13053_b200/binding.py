@@ -71,7 +71,7 @@ class _LmpOutputs(C.Structure):
 
 
 EXPORTS = ["retexo_status_string", "retexo_version", "retexo_validate_csr", "retexo_aggregate_workspace_size",
-           "retexo_aggregate", "retexo_theta_size", "retexo_pack_rows", "retexo_mlp_train_step_workspace_size",
+           "retexo_aggregate", "retexo_gat_backward_workspace_size", "retexo_gat_backward", "retexo_theta_size", "retexo_pack_rows", "retexo_mlp_train_step_workspace_size",
            "retexo_mlp_train_step", "retexo_embed_workspace_size", "retexo_embed",
            "retexo_cross_partition_workspace_size", "retexo_cross_partition_bytes",
            "retexo_cross_partition_static_scratch_bytes", "retexo_cross_partition_bytes_static",
@@ -89,7 +89,8 @@ def lib():
         L = C.CDLL(LIB_PATH)
         L.retexo_status_string.restype = C.c_char_p
         L.retexo_status_string.argtypes = [C.c_int]
-        for name in ("retexo_aggregate_workspace_size", "retexo_mlp_train_step_workspace_size",
+        for name in ("retexo_aggregate_workspace_size", "retexo_gat_backward_workspace_size",
+                     "retexo_mlp_train_step_workspace_size",
                      "retexo_embed_workspace_size", "retexo_cross_partition_workspace_size",
                      "retexo_lmp_workspace_size", "retexo_cross_partition_static_scratch_bytes"):
             getattr(L, name).restype = C.c_size_t
@@ -173,6 +174,33 @@ def retexo_aggregate(aggr: int, rowptr: torch.Tensor, colidx: torch.Tensor, q: t
                                 _ptr(ws), C.c_size_t(ws.numel()), _stream())
     _check(rc, "retexo_aggregate")
     return out, out_bf16
+
+
+def retexo_gat_backward(rowptr: torch.Tensor, colidx: torch.Tensor, p: torch.Tensor, gat: Dict, dz: torch.Tensor,
+                        want_f32: bool = True, want_bf16: bool = False):
+    """Backward of the GAT aggregation: returns (dp fp32 or None, dp bf16 or None, da_src, da_dst)."""
+    assert p.dtype == torch.float32 and dz.dtype == torch.float32 and p.stride(1) == 1 and dz.stride(1) == 1
+    n = rowptr.numel() - 1
+    dev = p.device
+    heads, dh = int(gat["heads"]), int(gat["head_dim"])
+    dim = heads * dh
+    a_src = gat["a_src"].to(device=dev, dtype=torch.float32).contiguous()
+    a_dst = gat["a_dst"].to(device=dev, dtype=torch.float32).contiguous()
+    gp = _GatParams(heads, dh, a_src.data_ptr(), a_dst.data_ptr(), float(gat.get("negative_slope", 0.2)),
+                    int(gat.get("add_self_loop", 1)))
+    dp = torch.empty((n, dim), dtype=torch.float32, device=dev) if want_f32 else None
+    dp16 = torch.empty((n, (dim + 63) // 64 * 64), dtype=torch.bfloat16, device=dev) if want_bf16 else None
+    da_src = torch.empty((heads, dh), dtype=torch.float32, device=dev)
+    da_dst = torch.empty((heads, dh), dtype=torch.float32, device=dev)
+    g = _csr(rowptr, colidx)
+    need = lib().retexo_gat_backward_workspace_size(C.c_int64(n), C.c_int32(heads), C.c_int32(dim))
+    ws = _workspace(need, dev)
+    rc = lib().retexo_gat_backward(C.byref(g), _ptr(p), C.c_int64(p.stride(0) if n > 0 else dim), C.byref(gp), _ptr(dz),
+                                   C.c_int64(dz.stride(0) if n > 0 else dim), _ptr(dp), C.c_int64(dim), _ptr(dp16),
+                                   C.c_int64(dp16.stride(0) if dp16 is not None else 0), _ptr(da_src), _ptr(da_dst),
+                                   _ptr(ws), C.c_size_t(ws.numel()), _stream())
+    _check(rc, "retexo_gat_backward")
+    return dp, dp16, da_src, da_dst
 
 
 def retexo_pack_rows(src: torch.Tensor, idx: Optional[torch.Tensor] = None, dim: Optional[int] = None,

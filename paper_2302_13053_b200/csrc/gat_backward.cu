@@ -1,0 +1,295 @@
+// Backward of the GAT aggregation (Section 2.2: AGGR may have trainable parameters; Section 3.1: a round
+// trains the whole layer).  With z_uv = s_u + t_v, e = LeakyReLU(z), alpha = softmax over u in N(v) (+ v),
+// Z_v = sum_u alpha_uv p_u and dz = dLoss/dZ:
+//   dalpha_uv = <dz_v, p_u>             de_uv = alpha_uv (dalpha_uv - c_v),  c_v = sum_w alpha_wv dalpha_wv
+//   dzz_uv    = de_uv (z_uv > 0 ? 1 : slope)
+//   dt_v = sum_u dzz_uv                 ds_u = sum_v dzz_uv
+//   dp_u = sum_v alpha_uv dz_v + ds_u a_src + dt_u a_dst
+//   da_src = sum_u ds_u p_u             da_dst = sum_v dt_v p_v
+// Two passes over the same CSR (the graph is symmetric, so the rows that attend over u are u's own row):
+// one warp per destination v computes the soft-max statistics, c_v and dt_v; one warp per source u then walks
+// the destinations v that attend over it and accumulates ds_u and dp_u in CSR order.  No floating-point
+// atomics: the parameter gradients are summed per block and the block sums in block order.
+#include "common.cuh"
+
+namespace retexo {
+
+constexpr int kGbThreads = 256, kGbWarps = kGbThreads / kWarp, kGbMaxHeads = 8;
+
+struct GatBwdArgs {
+    int64_t n;
+    const int64_t* rowptr;
+    const int32_t* colidx;
+    const float* p; int64_t ldp;
+    int32_t heads, head_dim, dim;
+    const float* a_src; const float* a_dst;
+    float slope; int32_t self_loop;
+    const float* dz; int64_t lddz;
+    float* s; float* t;              // [n x heads]
+    float4* stats;                   // [n x heads]: (row maximum, 1 / soft-max sum (0 = dz_v is zero), c_v, dt_v)
+    float* dp; int64_t lddp;
+    __nv_bfloat16* dp16; int64_t lddp16;
+    float* partial;                  // [blocks x 2 x dim]: per-block sums of ds_u p_u and dt_u p_u
+};
+
+__global__ void __launch_bounds__(kGbThreads) gat_bwd_scores_kernel(GatBwdArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int64_t u = blockIdx.x * (int64_t)kGbWarps + (threadIdx.x >> 5);
+    if (u >= a.n) return;
+    const float* row = a.p + u * a.ldp;
+    for (int h = 0; h < a.heads; ++h) {
+        float ss = 0.f, tt = 0.f;
+        for (int j = lane; j < a.head_dim; j += kWarp) {
+            const float x = row[h * a.head_dim + j];
+            ss = fmaf(a.a_src[h * a.head_dim + j], x, ss);
+            tt = fmaf(a.a_dst[h * a.head_dim + j], x, tt);
+        }
+        ss = warp_sum(ss);
+        tt = warp_sum(tt);
+        if (lane == 0) { a.s[u * a.heads + h] = ss; a.t[u * a.heads + h] = tt; }
+    }
+}
+
+// <x, y> restricted to each head's columns, summed over the warp: every lane ends up with all heads' values.
+template <int NC>
+__device__ __forceinline__ void head_dots(const float (&x)[NC], const float (&y)[NC], const int (&head_of)[NC], int heads,
+                                          float (&out)[kGbMaxHeads]) {
+#pragma unroll
+    for (int h = 0; h < kGbMaxHeads; ++h) {
+        out[h] = 0.f;
+        if (h < heads) {
+            float part = 0.f;
+#pragma unroll
+            for (int c = 0; c < NC; ++c) part = head_of[c] == h ? fmaf(x[c], y[c], part) : part;
+            out[h] = warp_sum(part);
+        }
+    }
+}
+
+// Pass over destinations: one warp per v.  Lane L owns the columns L, L + 32, ...
+template <int NC>
+__global__ void __launch_bounds__(kGbThreads) gat_bwd_dst_kernel(GatBwdArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int64_t v = blockIdx.x * (int64_t)kGbWarps + (threadIdx.x >> 5);
+    if (v >= a.n) return;
+    int head_of[NC];
+    float g[NC];
+    bool any = false;
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int col = c * kWarp + lane;
+        head_of[c] = col < a.dim ? col / a.head_dim : -1;
+        g[c] = col < a.dim ? a.dz[v * a.lddz + col] : 0.f;
+        any = any || g[c] != 0.f;
+    }
+    const int64_t beg = a.rowptr[v];
+    const int64_t deg = a.rowptr[v + 1] - beg;
+    const int64_t total = deg + (a.self_loop ? 1 : 0);
+    if (!__any_sync(0xffffffffu, any) || total == 0) {       // outside the loss: nothing flows back through this row
+        if (lane < a.heads) a.stats[v * a.heads + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
+    float tv[kGbMaxHeads], m[kGbMaxHeads], den[kGbMaxHeads];
+#pragma unroll
+    for (int h = 0; h < kGbMaxHeads; ++h) {
+        tv[h] = h < a.heads ? a.t[v * a.heads + h] : 0.f;
+        m[h] = -INFINITY;
+        den[h] = 0.f;
+    }
+    // sweep 1: row maximum and soft-max sum per head, 32 entries at a time (lane j scores entry j)
+    for (int64_t e0 = 0; e0 < total; e0 += kWarp) {
+        const bool valid = e0 + lane < total;
+        const int64_t u = !valid ? v : (e0 + lane < deg ? (int64_t)__ldg(a.colidx + beg + e0 + lane) : v);
+#pragma unroll
+        for (int h = 0; h < kGbMaxHeads; ++h) {
+            if (h < a.heads) {
+                const float z = a.s[u * a.heads + h] + tv[h];
+                const float e = valid ? (z > 0.f ? z : a.slope * z) : -INFINITY;
+                const float mn = fmaxf(m[h], warp_max(e));
+                den[h] = den[h] * expf(m[h] - mn) + warp_sum(valid ? expf(e - mn) : 0.f);
+                m[h] = mn;
+            }
+        }
+    }
+    // sweep 2: c_v = sum alpha dalpha, and the two sums that give dt_v = sum alpha (dalpha - c_v) g'
+    float csum[kGbMaxHeads], a1[kGbMaxHeads], a2[kGbMaxHeads];
+#pragma unroll
+    for (int h = 0; h < kGbMaxHeads; ++h) { csum[h] = 0.f; a1[h] = 0.f; a2[h] = 0.f; }
+    for (int64_t e = 0; e < total; ++e) {
+        const int64_t u = e < deg ? (int64_t)__ldg(a.colidx + beg + e) : v;
+        float x[NC], dalpha[kGbMaxHeads];
+#pragma unroll
+        for (int c = 0; c < NC; ++c) {
+            const int col = c * kWarp + lane;
+            x[c] = col < a.dim ? __ldg(a.p + u * a.ldp + col) : 0.f;
+        }
+        head_dots<NC>(g, x, head_of, a.heads, dalpha);
+#pragma unroll
+        for (int h = 0; h < kGbMaxHeads; ++h) {
+            if (h < a.heads) {
+                const float z = a.s[u * a.heads + h] + tv[h];
+                const float alpha = expf((z > 0.f ? z : a.slope * z) - m[h]) / den[h];
+                const float gp = z > 0.f ? 1.f : a.slope;
+                csum[h] = fmaf(alpha, dalpha[h], csum[h]);
+                a1[h] = fmaf(alpha * gp, dalpha[h], a1[h]);
+                a2[h] = fmaf(alpha, gp, a2[h]);
+            }
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < kGbMaxHeads; ++h)
+        if (h < a.heads && lane == h) a.stats[v * a.heads + h] = make_float4(m[h], 1.f / den[h], csum[h], a1[h] - csum[h] * a2[h]);
+}
+
+// Pass over sources: one warp per u walks the destinations that attend over u (its own row, and itself).
+template <int NC>
+__global__ void __launch_bounds__(kGbThreads) gat_bwd_src_kernel(GatBwdArgs a) {
+    __shared__ float sm_part[kGbWarps][2][NC * kWarp];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t u = blockIdx.x * (int64_t)kGbWarps + warp;
+    int head_of[NC];
+    float px[NC], acc[NC];
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int col = c * kWarp + lane;
+        head_of[c] = col < a.dim ? col / a.head_dim : -1;
+        px[c] = (u < a.n && col < a.dim) ? a.p[u * a.ldp + col] : 0.f;
+        acc[c] = 0.f;
+    }
+    float ds[kGbMaxHeads], dtu[kGbMaxHeads], su[kGbMaxHeads];
+#pragma unroll
+    for (int h = 0; h < kGbMaxHeads; ++h) { ds[h] = 0.f; dtu[h] = 0.f; su[h] = 0.f; }
+    if (u < a.n) {
+#pragma unroll
+        for (int h = 0; h < kGbMaxHeads; ++h) {
+            if (h < a.heads) {
+                su[h] = a.s[u * a.heads + h];
+                dtu[h] = a.stats[u * a.heads + h].w;
+            }
+        }
+        const int64_t beg = a.rowptr[u];
+        const int64_t deg = a.rowptr[u + 1] - beg;
+        const int64_t total = deg + (a.self_loop ? 1 : 0);
+        for (int64_t e = 0; e < total; ++e) {
+            const int64_t v = e < deg ? (int64_t)__ldg(a.colidx + beg + e) : u;
+            if (a.stats[v * a.heads].y == 0.f) continue;      // dz_v is zero (the same for every lane)
+            float g[NC], dalpha[kGbMaxHeads], alpha[kGbMaxHeads];
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                const int col = c * kWarp + lane;
+                g[c] = col < a.dim ? __ldg(a.dz + v * a.lddz + col) : 0.f;
+            }
+            head_dots<NC>(g, px, head_of, a.heads, dalpha);
+#pragma unroll
+            for (int h = 0; h < kGbMaxHeads; ++h) {
+                alpha[h] = 0.f;
+                if (h < a.heads) {
+                    const float4 st = a.stats[v * a.heads + h];
+                    const float z = su[h] + a.t[v * a.heads + h];
+                    alpha[h] = expf((z > 0.f ? z : a.slope * z) - st.x) * st.y;
+                    ds[h] = fmaf(alpha[h] * (z > 0.f ? 1.f : a.slope), dalpha[h] - st.z, ds[h]);
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < NC; ++c) {
+                float al = 0.f;
+#pragma unroll
+                for (int h = 0; h < kGbMaxHeads; ++h) al = head_of[c] == h ? alpha[h] : al;
+                acc[c] = fmaf(al, g[c], acc[c]);
+            }
+        }
+    }
+#pragma unroll
+    for (int c = 0; c < NC; ++c) {
+        const int col = c * kWarp + lane;
+        float dsc = 0.f, dtc = 0.f;
+#pragma unroll
+        for (int h = 0; h < kGbMaxHeads; ++h) { dsc = head_of[c] == h ? ds[h] : dsc; dtc = head_of[c] == h ? dtu[h] : dtc; }
+        if (u < a.n && col < a.dim) {
+            const float val = acc[c] + dsc * a.a_src[col] + dtc * a.a_dst[col];
+            if (a.dp) a.dp[u * a.lddp + col] = val;
+            if (a.dp16) a.dp16[u * a.lddp16 + col] = f32_to_bf16(val);
+        }
+        sm_part[warp][0][c * kWarp + lane] = dsc * px[c];       // (zero beyond the last node / column)
+        sm_part[warp][1][c * kWarp + lane] = dtc * px[c];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2 * a.dim; i += kGbThreads) {
+        const int which = i / a.dim, col = i % a.dim;
+        float sum = 0.f;
+        for (int w = 0; w < kGbWarps; ++w) sum += sm_part[w][which][col];
+        a.partial[((int64_t)blockIdx.x * 2 + which) * a.dim + col] = sum;
+    }
+}
+
+__global__ void __launch_bounds__(256) gat_bwd_reduce_kernel(const float* partial, int64_t n_blocks, int32_t dim,
+                                                             float* da_src, float* da_dst) {
+    const int i = blockIdx.x * 256 + threadIdx.x;
+    if (i >= 2 * dim) return;
+    const int which = i / dim, col = i % dim;
+    float sum = 0.f;
+    for (int64_t b = 0; b < n_blocks; ++b) sum += partial[(b * 2 + which) * dim + col];
+    (which ? da_dst : da_src)[col] = sum;
+}
+
+template <int NC>
+static int launch_bwd(const GatBwdArgs& a, unsigned blocks, float* da_src, float* da_dst, cudaStream_t st) {
+    gat_bwd_dst_kernel<NC><<<blocks, kGbThreads, 0, st>>>(a);
+    gat_bwd_src_kernel<NC><<<blocks, kGbThreads, 0, st>>>(a);
+    gat_bwd_reduce_kernel<<<(unsigned)((2 * a.dim + 255) / 256), 256, 0, st>>>(a.partial, blocks, a.dim, da_src, da_dst);
+    return launch_status();
+}
+
+}  // namespace retexo
+
+using namespace retexo;
+
+extern "C" size_t retexo_gat_backward_workspace_size(int64_t n_nodes, int32_t heads, int32_t dim) {
+    if (n_nodes < 0 || heads <= 0 || dim <= 0) return 0;
+    Sizer s;
+    s.take<float>((size_t)n_nodes * heads);
+    s.take<float>((size_t)n_nodes * heads);
+    s.take<float4>((size_t)n_nodes * heads);
+    s.take<float>((size_t)((n_nodes + kGbWarps - 1) / kGbWarps + 1) * 2 * (size_t)dim);
+    return s.off + kAlign;
+}
+
+extern "C" int retexo_gat_backward(const retexo_csr* g, const float* p, int64_t ldp, const retexo_gat_params* gat,
+                                   const float* dz, int64_t lddz, float* dp, int64_t lddp, void* dp_bf16,
+                                   int64_t lddp_bf16, float* da_src, float* da_dst, void* workspace,
+                                   size_t workspace_bytes, void* stream) {
+    if (!g || g->n_nodes < 0 || g->n_edges < 0 || g->n_nodes > INT32_MAX) return RETEXO_ERR_INVALID_ARG;
+    if (!gat || gat->heads <= 0 || gat->head_dim <= 0 || !gat->a_src || !gat->a_dst) return RETEXO_ERR_INVALID_ARG;
+    const int32_t dim = gat->heads * gat->head_dim;
+    if (gat->heads > kGbMaxHeads || dim > 256) return RETEXO_ERR_UNSUPPORTED;
+    if (!da_src || !da_dst || (!dp && !dp_bf16)) return RETEXO_ERR_INVALID_ARG;
+    if (ldp < dim || lddz < dim || (dp && lddp < dim) || (dp_bf16 && lddp_bf16 < dim)) return RETEXO_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (g->n_nodes == 0) {
+        RETEXO_CUDA_TRY(cudaMemsetAsync(da_src, 0, sizeof(float) * dim, st));
+        RETEXO_CUDA_TRY(cudaMemsetAsync(da_dst, 0, sizeof(float) * dim, st));
+        return RETEXO_OK;
+    }
+    if (!g->rowptr || !p || !dz || (g->n_edges > 0 && !g->colidx)) return RETEXO_ERR_INVALID_ARG;
+    const size_t need = retexo_gat_backward_workspace_size(g->n_nodes, gat->heads, dim);
+    if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
+    const int64_t n = g->n_nodes;
+    Arena ws(workspace, workspace_bytes);
+    GatBwdArgs a;
+    a.n = n; a.rowptr = g->rowptr; a.colidx = g->colidx; a.p = p; a.ldp = ldp;
+    a.heads = gat->heads; a.head_dim = gat->head_dim; a.dim = dim;
+    a.a_src = gat->a_src; a.a_dst = gat->a_dst; a.slope = gat->negative_slope; a.self_loop = gat->add_self_loop ? 1 : 0;
+    a.dz = dz; a.lddz = lddz;
+    a.s = ws.take<float>((size_t)n * gat->heads);
+    a.t = ws.take<float>((size_t)n * gat->heads);
+    a.stats = ws.take<float4>((size_t)n * gat->heads);
+    const unsigned blocks = (unsigned)((n + kGbWarps - 1) / kGbWarps);
+    a.partial = ws.take<float>((size_t)(blocks + 1) * 2 * (size_t)dim);
+    a.dp = dp; a.lddp = lddp; a.dp16 = static_cast<__nv_bfloat16*>(dp_bf16); a.lddp16 = lddp_bf16;
+    gat_bwd_scores_kernel<<<blocks, kGbThreads, 0, st>>>(a);
+    const int nc = (dim + kWarp - 1) / kWarp;
+    if (nc <= 1) return launch_bwd<1>(a, blocks, da_src, da_dst, st);
+    if (nc <= 2) return launch_bwd<2>(a, blocks, da_src, da_dst, st);
+    if (nc <= 4) return launch_bwd<4>(a, blocks, da_src, da_dst, st);
+    return launch_bwd<8>(a, blocks, da_src, da_dst, st);
+}
