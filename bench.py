@@ -181,12 +181,18 @@ def launches_per_step(w, R: int) -> int:
     total += (2 if n_parts <= 8192 else 3) + 1       # count kernels + finalize + pack
     for rd in w.round_dims():
         h = rd["hidden"]
+        gat_forward = 1 + 1 + 2                      # W_att^T copy, projection, scores + rows
         if w.aggr == wl.GAT:
-            total += 1 + 1 + 1 + 2                   # weight convert, pack, projection, scores + rows
+            total += 1                               # the round's input as a bf16 operand
+            total += 3 * gat_forward                 # last and kept iterate for the test rows, kept iterate for the emission
         else:
-            total += 3                               # prep, warp rows, block rows
-        total += 2                                   # train / val batches
+            total += 3 + 2                           # prep, warp rows, block rows; train / val batches
         step = 5 if h > 0 else 3                     # products, fused middle, reduce + update (+ weight copies once)
+        if w.aggr == wl.GAT:
+            # the aggregator is trained with the model: per iteration projection + aggregation + batches before
+            # the step, input gradient inside it, kept copy + scatter + backward (4) + dW_att + update after it
+            step += gat_forward + 2 + 1 + 8
+            total += gat_forward + 2                 # the last iterate's own validation pass
         total += R * step + 1 + (2 if h > 0 else 1)       # (the update kernel's last block books the validation count
                                                           #  that rides along; the last iterate's is booked by a kernel of its own)
         total += (2 if h > 0 else 1) + 1             # stand-alone validation of the last iterate + snapshot

@@ -213,12 +213,15 @@ size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_
  * y     int32 [n_rows] labels in [0, n_classes).
  * loss_out  device float, the loss before the update (may be NULL).
  * grad_out  optional device fp32 array shaped like theta: the gradient.
+ * dx_out    optional device fp32 [n_rows x ld_dx], ld_dx >= d_in: dLoss / dx, the gradient with respect
+ *           to the batch rows themselves (one more product, dHd W1^T).  A round whose aggregator has
+ *           parameters (Section 2.2) passes it on to retexo_gat_backward.
  * Increments model->step (host struct).  n_classes <= 64, hidden <= 512.
  * Errors: INVALID_ARG, ALIGNMENT, WORKSPACE, UNSUPPORTED. */
 int retexo_mlp_train_step(retexo_mlp* model,
                           const void* x, int64_t ldx, int32_t x_has_ones,
                           const int32_t* y, int64_t n_rows,
-                          float* loss_out, float* grad_out,
+                          float* loss_out, float* grad_out, float* dx_out, int64_t ld_dx,
                           void* workspace, size_t workspace_bytes, void* stream);
 
 size_t retexo_embed_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows);
@@ -335,6 +338,11 @@ typedef struct retexo_lmp_config {
                                           device inside the call; results are also written to host */
     float dropout;                  /* dropout rate of the hidden units while training (see retexo_mlp); 0 = none */
     uint64_t dropout_seed;          /* round m = 1..K draws its masks with the key dropout_seed + (m - 1) */
+    int32_t gat_freeze_attention;   /* RETEXO_GAT only.  0 (default): the round trains the whole layer, i.e. the
+                                       projection W_att and the attention vectors together with the per-node model
+                                       (Section 2.2: AGGR may have trainable parameters; Section 3.1), re-aggregating
+                                       locally in every iteration.  1: they stay at the values given in gat_w and the
+                                       aggregation runs once per round */
 } retexo_lmp_config;
 
 typedef struct retexo_lmp_inputs {
@@ -348,7 +356,8 @@ typedef struct retexo_lmp_inputs {
     const float* const* theta0;    /* HOST array of K pointers to the initial theta of each round
                                       (pointees: device or host memory, like the other inputs) */
     const float* const* gat_w;     /* GAT only: HOST array of K pointers, each to
-                                      [rep_dim x heads*head_dim | a_src | a_dst] fp32 (frozen) */
+                                      [W_att (rep_dim x heads*head_dim) | a_src | a_dst] fp32: the initial
+                                      (gat_freeze_attention = 1: the fixed) parameters of each round's aggregator */
 } retexo_lmp_inputs;
 
 typedef struct retexo_lmp_outputs {
@@ -363,6 +372,8 @@ typedef struct retexo_lmp_outputs {
     float* final_logits; int64_t ld_logits;   /* [n x ld] logits of the last round's kept model; may be NULL */
     int32_t* final_pred;            /* [n]; may be NULL */
     float* const* theta_best;       /* HOST array of K pointers receiving each round's kept theta; may be NULL */
+    float* const* gat_best;         /* GAT only: HOST array of K pointers receiving each round's kept
+                                       [W_att | a_src | a_dst]; may be NULL */
 } retexo_lmp_outputs;
 
 size_t retexo_lmp_workspace_size(const retexo_lmp_config* cfg, int64_t n_nodes, int64_t n_edges,
@@ -373,8 +384,13 @@ size_t retexo_lmp_workspace_size(const retexo_lmp_config* cfg, int64_t n_nodes, 
  *   from theta0[m]; every eval_every iterations measure validation accuracy
  *   and keep the iterate with the most hits (earliest on ties); emit Q^m from
  *   the kept model (last round: logits, predictions, test accuracy) }.
- * GAT: the round's projection and attention vectors (gat_w[m]) are fixed
- * draws, P = Q^{m-1} W_att is computed once, then aggregated.
+ * GAT: P = Q^{m-1} W_att, then scores, soft-max and weighted sum.  By default the
+ * aggregator's parameters are trained with the per-node model: every iteration
+ * recomputes P and the aggregation with the current parameters (all local once the
+ * round's exchange has delivered Q^{m-1}), back-propagates through the attention
+ * (retexo_gat_backward) and updates [W_att | a_src | a_dst] with the same optimiser;
+ * the iterate kept on validation keeps its aggregator parameters with it.  With
+ * gat_freeze_attention = 1 they stay fixed and the aggregation runs once.
  * With memory_is_host = 0 the call only enqueues work (outputs are device
  * memory); with 1 it copies inputs in, runs, copies outputs to the host
  * arrays and synchronises the stream before returning.

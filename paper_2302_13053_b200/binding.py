@@ -48,7 +48,7 @@ class _LmpConfig(C.Structure):
                 ("n_classes", C.c_int32), ("optimizer", C.c_int32), ("lr", C.c_float), ("beta1", C.c_float),
                 ("beta2", C.c_float), ("eps", C.c_float), ("eval_every", C.c_int32), ("gat_heads", C.c_int32),
                 ("gat_head_dim", C.c_int32), ("gat_negative_slope", C.c_float), ("memory_is_host", C.c_int32),
-                ("dropout", C.c_float), ("dropout_seed", C.c_uint64)]
+                ("dropout", C.c_float), ("dropout_seed", C.c_uint64), ("gat_freeze_attention", C.c_int32)]
 
 
 class _LmpInputs(C.Structure):
@@ -67,7 +67,7 @@ class _LmpOutputs(C.Structure):
     _fields_ = [("loss_history", C.c_void_p), ("val_correct", C.c_void_p), ("best_val_correct", C.c_void_p),
                 ("best_iter", C.c_void_p), ("test_correct", C.c_void_p), ("test_correct_last", C.c_void_p),
                 ("counts", C.c_void_p), ("final_logits", C.c_void_p), ("ld_logits", C.c_int64),
-                ("final_pred", C.c_void_p), ("theta_best", C.POINTER(C.c_void_p))]
+                ("final_pred", C.c_void_p), ("theta_best", C.POINTER(C.c_void_p)), ("gat_best", C.POINTER(C.c_void_p))]
 
 
 EXPORTS = ["retexo_status_string", "retexo_version", "retexo_validate_csr", "retexo_aggregate_workspace_size",
@@ -268,24 +268,27 @@ class Mlp:
 
 
 def retexo_mlp_train_step(model: Mlp, x: torch.Tensor, y: torch.Tensor, x_has_ones: bool = False,
-                          return_grad: bool = False, workspace: Optional[torch.Tensor] = None):
+                          return_grad: bool = False, workspace: Optional[torch.Tensor] = None, return_dx: bool = False):
     """One full-batch iteration on the bf16 batch x [n_rows, ld] with labels y.
     x_has_ones: column d_in of x holds 1 in every row (retexo_pack_rows(ones=True)).
     Returns the loss before the update as a 0-dim device tensor (and the
-    gradient if asked)."""
+    gradient, and dLoss/dx [n_rows, d_in], if asked: (loss, grad, dx) with None for what was not)."""
     assert x.dtype == torch.bfloat16 and y.dtype == torch.int32 and x.stride(1) == 1
     n_rows = x.shape[0]
     dev = x.device
     loss = torch.zeros((), dtype=torch.float32, device=dev)
     grad = torch.zeros_like(model.theta) if return_grad else None
+    dx = torch.empty((n_rows, model.d_in), dtype=torch.float32, device=dev) if return_dx else None
     need = lib().retexo_mlp_train_step_workspace_size(C.c_int32(model.d_in), C.c_int32(model.hidden),
                                                       C.c_int32(model.n_classes), C.c_int64(n_rows))
     ws = workspace if workspace is not None else _workspace(need, dev)
     rc = lib().retexo_mlp_train_step(C.byref(model.c), _ptr(x), C.c_int64(x.stride(0)),
                                      C.c_int32(1 if x_has_ones else 0), _ptr(y),
-                                     C.c_int64(n_rows), _ptr(loss), _ptr(grad), _ptr(ws), C.c_size_t(ws.numel()),
-                                     _stream())
+                                     C.c_int64(n_rows), _ptr(loss), _ptr(grad), _ptr(dx), C.c_int64(model.d_in),
+                                     _ptr(ws), C.c_size_t(ws.numel()), _stream())
     _check(rc, "retexo_mlp_train_step")
+    if return_dx:
+        return loss, grad, dx
     return (loss, grad) if return_grad else loss
 
 
@@ -383,13 +386,14 @@ class LmpProblem:
                  heads: int = 0, head_dim: int = 0, negative_slope: float = 0.2, optimizer: int = ADAM,
                  beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, eval_every: int = 1,
                  host: bool = False, want_logits: bool = True, device: str = "cuda", dropout: float = 0.0,
-                 dropout_seed: int = 0):
+                 dropout_seed: int = 0, freeze_attention: bool = False):
         self.host = bool(host)
         self.device = torch.device(device)
         n, e = rowptr.shape[0] - 1, colidx.shape[0]
         self.n, self.e, self.K, self.R, self.n_classes = n, e, K, R, n_classes
         self.cfg = _LmpConfig(aggr, K, R, features.shape[1], hidden, n_classes, optimizer, lr, beta1, beta2, eps,
-                              eval_every, heads, head_dim, negative_slope, 1 if host else 0, dropout, dropout_seed)
+                              eval_every, heads, head_dim, negative_slope, 1 if host else 0, dropout, dropout_seed,
+                              1 if freeze_attention else 0)
 
         def put(a: np.ndarray) -> torch.Tensor:
             t = torch.from_numpy(np.ascontiguousarray(a))
@@ -421,14 +425,16 @@ class LmpProblem:
         self.final_logits = out((n, n_classes), torch.float32) if want_logits else None
         self.final_pred = out((n,), torch.int32) if want_logits else None
         self.theta_best = [out(t.shape, torch.float32) for t in self.theta0]
+        self.gat_best = [out(t.shape, torch.float32) for t in self.gat_w] if self.gat_w else None
         self.d2h_bytes = sum(t.numel() * t.element_size() for t in
                              [self.loss_history, self.val_correct, self.best_val, self.best_iter, self.test_correct,
-                              self.test_last, self.counts] + self.theta_best +
+                              self.test_last, self.counts] + self.theta_best + (self.gat_best or []) +
                              ([self.final_logits, self.final_pred] if want_logits else []))
 
         self._theta0_arr = (C.c_void_p * K)(*[t.data_ptr() for t in self.theta0])
         self._gat_arr = (C.c_void_p * K)(*[t.data_ptr() for t in self.gat_w]) if self.gat_w else None
         self._best_arr = (C.c_void_p * K)(*[t.data_ptr() for t in self.theta_best])
+        self._gat_best_arr = (C.c_void_p * K)(*[t.data_ptr() for t in self.gat_best]) if self.gat_best else None
         g = _Csr(n, e, self.rowptr.data_ptr(), self.colidx.data_ptr())
         self.inputs = _LmpInputs(g, self.features.data_ptr(), features.shape[1], self.labels.data_ptr(),
                                  self.train_idx.data_ptr(), self.train_idx.numel(),
@@ -442,7 +448,8 @@ class LmpProblem:
                                    self.test_correct.data_ptr(), self.test_last.data_ptr(), self.counts.data_ptr(),
                                    self.final_logits.data_ptr() if want_logits else None, n_classes,
                                    self.final_pred.data_ptr() if want_logits else None,
-                                   C.cast(self._best_arr, C.POINTER(C.c_void_p)))
+                                   C.cast(self._best_arr, C.POINTER(C.c_void_p)),
+                                   C.cast(self._gat_best_arr, C.POINTER(C.c_void_p)) if self._gat_best_arr else None)
         need = lib().retexo_lmp_workspace_size(C.byref(self.cfg), C.c_int64(n), C.c_int64(e),
                                                C.c_int64(self.train_idx.numel()), C.c_int64(self.val_idx.numel()),
                                                C.c_int64(self.test_idx.numel()),
@@ -469,7 +476,8 @@ class LmpProblem:
                                 bytes_per_round=counts[4:4 + K].copy()),
                     final_logits=None if self.final_logits is None else cpu(self.final_logits),
                     final_pred=None if self.final_pred is None else cpu(self.final_pred),
-                    theta_best=[cpu(t) for t in self.theta_best])
+                    theta_best=[cpu(t) for t in self.theta_best],
+                    gat_best=[cpu(t) for t in self.gat_best] if self.gat_best else None)
 
 
 def retexo_lmp_train(problem: LmpProblem) -> None:

@@ -5,6 +5,7 @@
 #include <vector>
 
 #include "common.cuh"
+#include "gemm_tc.h"
 #include "mlp_plan.h"
 
 using namespace retexo;
@@ -40,6 +41,52 @@ __global__ void record_validation_kernel(const unsigned long long* cur, unsigned
         *best_iter = iter;
         *have_best = 1;
     }
+}
+// dz[idx[i]][0 .. dim) = dx[i][0 .. dim): the batch-ordered input gradient goes back to node order.
+__global__ void scatter_rows_kernel(const float* __restrict__ dx, int64_t ld_dx, const int32_t* __restrict__ idx,
+                                    int64_t n_rows, int32_t dim, float* __restrict__ dz, int64_t ld_dz) {
+    const int64_t t = blockIdx.x * 256ll + threadIdx.x;
+    const int64_t i = t / dim;
+    const int32_t c = (int32_t)(t % dim);
+    if (i < n_rows) dz[(int64_t)idx[i] * ld_dz + c] = dx[i * ld_dx + c];
+}
+// dst = src if *decision is set (the trained aggregator's parameters follow theta into the kept copy).
+__global__ void copy_if_kernel(const int32_t* decision, const float* src, float* dst, int64_t n) {
+    if (!*decision) return;
+    const int64_t p = blockIdx.x * 256ll + threadIdx.x;
+    if (p < n) dst[p] = src[p];
+}
+// One optimiser update of the aggregator's parameters [W_att | a_src | a_dst]: the gradient of W_att is the
+// sum of split-K partials (added in index order), those of the attention vectors come ready-made.
+// `step` is the 1-based number of this update, read on the device.
+__device__ __forceinline__ double whole_power(double base, unsigned long long e) {      // base^e by repeated squaring
+    double r = 1.0;
+    for (; e; e >>= 1, base *= base) if (e & 1ull) r *= base;
+    return r;
+}
+struct AttUpdateArgs {
+    float *att, *m, *v;
+    const float* partial; int64_t n_w, splits;
+    const float* da; int64_t n_att;
+    int optimizer; float lr, beta1, beta2, eps;
+    const unsigned long long* step;
+    float* grad_out;      // optional
+};
+__global__ void att_update_kernel(AttUpdateArgs a) {
+    const int64_t p = blockIdx.x * 256ll + threadIdx.x;
+    if (p >= a.n_att) return;
+    float g = 0.f;
+    if (p < a.n_w) for (int64_t z = 0; z < a.splits; ++z) g += a.partial[z * a.n_w + p];
+    else g = a.da[p - a.n_w];
+    if (a.grad_out) a.grad_out[p] = g;
+    if (a.optimizer == RETEXO_SGD) { a.att[p] -= a.lr * g; return; }
+    const unsigned long long t = *a.step;
+    const float c1 = (float)(1.0 - whole_power((double)a.beta1, t)), c2 = (float)(1.0 - whole_power((double)a.beta2, t));
+    const float m = a.beta1 * a.m[p] + (1.f - a.beta1) * g;
+    const float v = a.beta2 * a.v[p] + (1.f - a.beta2) * g * g;
+    a.m[p] = m;
+    a.v[p] = v;
+    a.att[p] -= a.lr * (m / c1) / (sqrtf(v / c2) + a.eps);
 }
 __global__ void fill_u64_kernel(unsigned long long* p, int64_t n, unsigned long long v) {
     const int64_t i = blockIdx.x * 256ll + threadIdx.x;
@@ -118,7 +165,9 @@ struct LmpBuffers {
     int32_t *train_idx, *val_idx, *test_idx, *part;
     // representations
     float* q[2];
-    bf16* x16; bf16* q16; float* proj; bf16* watt16; float* gat_vec; float* gat_stage;
+    bf16* x16; bf16* q16; float* proj; bf16* watt_t16;
+    float *att, *att_m, *att_v, *att_best, *att_partial, *da, *dx, *dz; bf16* dp16; int32_t* decision; int32_t* status;
+    int64_t att_splits; void* ws_gatbwd; size_t ws_gatbwd_bytes;
     bf16 *xtr16, *xval16;
     int32_t *y_tr, *y_val, *y_test;
     float *theta, *adam_m, *adam_v, *theta_best;
@@ -171,11 +220,24 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
     l.x16 = t.template take<bf16>((size_t)n * ld16);
     if (c.aggr == RETEXO_GAT) {
         const int32_t hd = c.gat_heads * c.gat_head_dim;
+        const size_t n_att = (size_t)max_rep * hd + 2 * (size_t)hd;
         l.q16 = t.template take<bf16>((size_t)n * round_up(max_rep, 64));
         l.proj = t.template take<float>((size_t)n * round_up(hd, 32));
-        l.watt16 = t.template take<bf16>((size_t)max_rep * hd);
-        l.gat_vec = t.template take<float>((size_t)2 * hd);
-        l.gat_stage = t.template take<float>((size_t)max_rep * hd + 2 * hd);
+        l.watt_t16 = t.template take<bf16>((size_t)hd * round_up(max_rep, 64));
+        l.att = t.template take<float>(n_att);
+        l.att_m = t.template take<float>(n_att);
+        l.att_v = t.template take<float>(n_att);
+        l.att_best = t.template take<float>(n_att);
+        l.att_splits = gemm_split((int64_t)max_rep, hd, n);
+        l.att_partial = t.template take<float>((size_t)l.att_splits * (size_t)max_rep * hd);
+        l.da = t.template take<float>((size_t)2 * hd);
+        l.dx = t.template take<float>((size_t)n_tr * round_up(hd, 32));
+        l.dz = t.template take<float>((size_t)n * round_up(hd, 32));
+        l.dp16 = t.template take<bf16>((size_t)n * round_up(hd, 64));
+        l.decision = t.template take<int32_t>(64);
+        l.status = t.template take<int32_t>(64);
+        l.ws_gatbwd_bytes = retexo_gat_backward_workspace_size(n, c.gat_heads, hd);
+        l.ws_gatbwd = t.template take<char>(l.ws_gatbwd_bytes);
     }
     // training rows, then validation rows, each followed by a column of ones (it carries the bias gradient
     // through the weight-gradient product); after the round's last iteration the test rows take their place
@@ -336,23 +398,38 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         const int64_t nt = retexo_theta_size(r.d_in, r.hidden, c.n_classes);
 
         // ---- one message-passing round: X = COMBINE(Q, AGGR(Q)), emitted in bf16 for the model
-        if (c.aggr == RETEXO_GAT) {
-            const int32_t hd = r.agg_dim;
-            const int64_t ldq16 = round_up(r.rep_dim, 64), ldp = round_up(hd, 32);
-            const size_t wcount = (size_t)r.rep_dim * hd + 2 * (size_t)hd;
-            RETEXO_CUDA_TRY(cudaMemcpyAsync(b.gat_stage, in->gat_w[m - 1], sizeof(float) * wcount,
-                                            cudaMemcpyDefault, st));
-            RETEXO_TRY(convert_f32_to_bf16_launch(b.gat_stage, b.watt16, (int64_t)r.rep_dim * hd, st));
-            RETEXO_CUDA_TRY(cudaMemcpyAsync(b.gat_vec, b.gat_stage + (size_t)r.rep_dim * hd, sizeof(float) * 2 * hd,
-                                            cudaMemcpyDeviceToDevice, st));
-            RETEXO_TRY(retexo_pack_rows(q, 0, ldq, r.rep_dim, nullptr, n, b.q16, ldq16, nullptr, 0, 0, st));
-            // P = Q W_att: the projection as a bias-free single linear layer
-            RETEXO_TRY(project_rows_launch(b.q16, ldq16, b.watt16, hd, n, hd, r.rep_dim, b.proj, ldp, st));
+        const bool gat = c.aggr == RETEXO_GAT;
+        const bool gat_train = gat && !c.gat_freeze_attention;      // the round trains the aggregator too
+        const int32_t hd = gat ? r.agg_dim : 0;
+        const int64_t ldq16 = round_up(r.rep_dim, 64), ldp = round_up(hd > 0 ? hd : 1, 32);
+        const int64_t n_att = (int64_t)r.rep_dim * hd + 2 * (int64_t)hd;
+        // GAT: P = Q W_att on the tensor cores (a bias-free product), then scores, soft-max and weighted sum in
+        // one pass, with the projection and attention vectors at `att` = [W_att | a_src | a_dst]
+        auto gat_forward = [&](const float* att) -> int {
+            RETEXO_TRY(retexo_pack_rows(att, 0, hd, hd, nullptr, r.rep_dim, nullptr, 0, b.watt_t16, ldq16, 0, st));
+            TcGemm pr{};
+            pr.A = b.q16; pr.lda = ldq16; pr.B = b.watt_t16; pr.ldb = ldq16; pr.M = n; pr.N = hd; pr.K = r.rep_dim;
+            pr.mode = TC_EPI_BIAS; pr.out_f32 = b.proj; pr.ld_f32 = ldp; pr.status = b.status;
+            RETEXO_TRY(tc_gemm_launch(pr, st));
             retexo_gat_params gp;
-            gp.heads = c.gat_heads; gp.head_dim = c.gat_head_dim; gp.a_src = b.gat_vec; gp.a_dst = b.gat_vec + hd;
-            gp.negative_slope = c.gat_negative_slope; gp.add_self_loop = 1;
-            RETEXO_TRY(retexo_aggregate(&g, RETEXO_GAT, b.proj, ldp, hd, &gp, nullptr, 0, 0, b.x16, ld16, b.ws_agg,
-                                        b.ws_agg_bytes, st));
+            gp.heads = c.gat_heads; gp.head_dim = c.gat_head_dim; gp.a_src = att + (int64_t)r.rep_dim * hd;
+            gp.a_dst = gp.a_src + hd; gp.negative_slope = c.gat_negative_slope; gp.add_self_loop = 1;
+            return retexo_aggregate(&g, RETEXO_GAT, b.proj, ldp, hd, &gp, nullptr, 0, 0, b.x16, ld16, b.ws_agg,
+                                    b.ws_agg_bytes, st);
+        };
+        if (gat) {
+            RETEXO_CUDA_TRY(cudaMemcpyAsync(b.att, in->gat_w[m - 1], sizeof(float) * (size_t)n_att, cudaMemcpyDefault, st));
+            RETEXO_CUDA_TRY(cudaMemcpyAsync(b.att_best, b.att, sizeof(float) * (size_t)n_att, cudaMemcpyDeviceToDevice, st));
+            RETEXO_CUDA_TRY(cudaMemsetAsync(b.status, 0, sizeof(int32_t), st));
+            RETEXO_TRY(retexo_pack_rows(q, 0, ldq, r.rep_dim, nullptr, n, b.q16, ldq16, nullptr, 0, 0, st));
+            if (gat_train) {
+                RETEXO_CUDA_TRY(cudaMemsetAsync(b.att_m, 0, sizeof(float) * (size_t)n_att, st));
+                RETEXO_CUDA_TRY(cudaMemsetAsync(b.att_v, 0, sizeof(float) * (size_t)n_att, st));
+                RETEXO_CUDA_TRY(cudaMemsetAsync(b.dz, 0, sizeof(float) * (size_t)n * (size_t)ldp, st));
+                RETEXO_CUDA_TRY(cudaMemsetAsync(b.decision, 0, sizeof(int32_t), st));
+            } else {
+                RETEXO_TRY(gat_forward(b.att));
+            }
         } else {
             RETEXO_TRY(retexo_aggregate(&g, c.aggr, q, ldq, r.agg_dim, nullptr, nullptr, 0, 1, b.x16, ld16, b.ws_agg,
                                         b.ws_agg_bytes, st));
@@ -360,9 +437,15 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
 
         // ---- the round's batches and model state
         const int64_t ld_tr = round_up(r.d_in + 1, 64);
-        RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld_tr, nullptr, 0, 1, st));
         bf16* xval16 = b.xtr16 + (size_t)n_tr * ld_tr;
-        if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, xval16, ld_tr, nullptr, 0, 0, st));
+        // the training rows (followed by their column of ones), then the validation rows; a round that trains
+        // its aggregator packs them anew after every local aggregation
+        auto pack_batches = [&]() -> int {
+            RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, train_idx, n_tr, b.xtr16, ld_tr, nullptr, 0, 1, st));
+            if (n_val) RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, val_idx, n_val, xval16, ld_tr, nullptr, 0, 0, st));
+            return RETEXO_OK;
+        };
+        if (!gat_train) RETEXO_TRY(pack_batches());
         RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta, in->theta0[m - 1], sizeof(float) * (size_t)nt, cudaMemcpyDefault, st));
         RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta_best, b.theta, sizeof(float) * (size_t)nt, cudaMemcpyDeviceToDevice, st));
         RETEXO_CUDA_TRY(cudaMemsetAsync(b.adam_m, 0, sizeof(float) * (size_t)nt, st));
@@ -396,7 +479,33 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
                              b.val_history + (size_t)(m - 1) * c.R};
         // With validation every iteration (or none) all iterations from the second on are the same six
         // launches with the same arguments: the second one is recorded as a graph, the rest replay it.
-        const bool uniform = work.own && c.R > 3 && (n_val == 0 || c.eval_every == 1);
+        const bool uniform = work.own && c.R > 3 && (n_val == 0 || c.eval_every == 1) && !gat_train;
+        tail.decision = gat_train ? b.decision : nullptr;
+        const int64_t ld_dx = ldp;
+        // What a round that trains its aggregator adds to an iteration (Section 3.1: after the round's exchange
+        // everything an iteration needs is local, so the aggregation is redone with the current parameters):
+        // before the step, projection + aggregation + batches; after it, the kept copy follows theta's, the
+        // input gradient goes back through the attention, and [W_att | a_src | a_dst] take their update.
+        auto gat_backward_and_update = [&]() -> int {
+            copy_if_kernel<<<(unsigned)((n_att + 255) / 256), 256, 0, st>>>(b.decision, b.att, b.att_best, n_att);
+            scatter_rows_kernel<<<(unsigned)((n_tr * hd + 255) / 256), 256, 0, st>>>(b.dx, ld_dx, train_idx, n_tr, hd, b.dz, ldp);
+            retexo_gat_params gp;
+            gp.heads = c.gat_heads; gp.head_dim = c.gat_head_dim; gp.a_src = b.att + (int64_t)r.rep_dim * hd;
+            gp.a_dst = gp.a_src + hd; gp.negative_slope = c.gat_negative_slope; gp.add_self_loop = 1;
+            RETEXO_TRY(retexo_gat_backward(&g, b.proj, ldp, &gp, b.dz, ldp, nullptr, 0, b.dp16, round_up(hd, 64), b.da,
+                                           b.da + hd, b.ws_gatbwd, b.ws_gatbwd_bytes, st));
+            TcGemm gw{};      // dW_att = Q^T dP, reduced over the nodes
+            gw.A = b.q16; gw.lda = ldq16; gw.B = b.dp16; gw.ldb = round_up(hd, 64); gw.M = r.rep_dim; gw.N = hd; gw.K = n;
+            gw.mode = TC_EPI_PARTIAL; gw.splits = (int)gemm_split(r.rep_dim, hd, n); gw.partial = b.att_partial;
+            gw.status = b.status;
+            RETEXO_TRY(tc_gemm_launch(gw, st));
+            AttUpdateArgs au{};
+            au.att = b.att; au.m = b.att_m; au.v = b.att_v; au.partial = b.att_partial; au.n_w = (int64_t)r.rep_dim * hd;
+            au.splits = gw.splits; au.da = b.da; au.n_att = n_att; au.optimizer = c.optimizer; au.lr = c.lr;
+            au.beta1 = c.beta1; au.beta2 = c.beta2; au.eps = c.eps; au.step = b.cur_correct + 2;      // (already advanced)
+            att_update_kernel<<<(unsigned)((n_att + 255) / 256), 256, 0, st>>>(au);
+            return launch_status();
+        };
         iteration.reset();
         int pending_it = 0;       // iteration whose weights still await their validation count
         for (int it = 1; it <= c.R; ++it) {
@@ -408,7 +517,14 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
             tail.iter = pending_it;
             tail.history_slot = b.val_history + (size_t)(m - 1) * c.R + (pending_it > 0 ? pending_it - 1 : 0);
             const EvalTail* riding = pending_it ? &tail : nullptr;
-            if (iteration.exec) {
+            if (gat_train) {
+                RETEXO_TRY(gat_forward(b.att));
+                RETEXO_TRY(pack_batches());
+                if (!riding) RETEXO_CUDA_TRY(cudaMemsetAsync(b.decision, 0, sizeof(int32_t), st));
+                RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot, nullptr, it > 1,
+                                                 riding, st, &dev, b.dx, ld_dx));
+                RETEXO_TRY(gat_backward_and_update());
+            } else if (iteration.exec) {
                 RETEXO_CUDA_TRY(cudaGraphLaunch(iteration.exec, st));
             } else if (uniform && it == 2) {
                 bool recorded = false;
@@ -438,16 +554,25 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
             const bool want = n_val && (it % c.eval_every == 0 || it == c.R);
             pending_it = (want && it < c.R) ? it : 0;
             if (want && it == c.R) {      // the last iterate has no next iteration to ride on
+                if (gat_train) {
+                    RETEXO_TRY(gat_forward(b.att));
+                    RETEXO_TRY(pack_batches());
+                }
                 RETEXO_TRY(mlp_count_hits_launch(plan, sb, &model, xval16, ld_tr, n_val, val_hd, b.y_val,
                                                  b.cur_correct, st));
                 snapshot_if_better_kernel<<<(unsigned)((nt + 255) / 256), 256, 0, st>>>(
                     b.cur_correct, b.best_correct, b.have_best, b.theta, b.theta_best, nt);
+                if (gat_train)
+                    snapshot_if_better_kernel<<<(unsigned)((n_att + 255) / 256), 256, 0, st>>>(
+                        b.cur_correct, b.best_correct, b.have_best, b.att, b.att_best, n_att);
                 record_validation_kernel<<<1, 32, 0, st>>>(b.cur_correct, b.best_correct, b.have_best, it,
                                                            b.best_iter_cur,
                                                            b.val_history + (size_t)(m - 1) * c.R + (it - 1));
             }
         }
         if (!n_val) {   // nothing to select on: keep the last iterate
+            if (gat_train)
+                RETEXO_CUDA_TRY(cudaMemcpyAsync(b.att_best, b.att, sizeof(float) * (size_t)n_att, cudaMemcpyDeviceToDevice, st));
             RETEXO_CUDA_TRY(cudaMemcpyAsync(b.theta_best, b.theta, sizeof(float) * (size_t)nt, cudaMemcpyDeviceToDevice, st));
             const int32_t last = c.R;
             RETEXO_CUDA_TRY(cudaMemcpyAsync(b.best_iter_cur, &last, sizeof(int32_t), cudaMemcpyHostToDevice, st));
@@ -462,17 +587,26 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
             // the test rows are gathered once into a dense batch (the training batch is no longer needed),
             // so both forward passes run on the tensor cores
             bf16* xte16 = b.xtr16;
+            if (gat_train) RETEXO_TRY(gat_forward(b.att));           // the last iterate's own aggregation
             RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, test_idx, n_te, xte16, ld16, nullptr, 0, 0, st));
-            RETEXO_TRY(retexo_embed(&best, xte16, ld16, nullptr, n_te, nullptr, 0, nullptr, 0, nullptr, 0, nullptr,
-                                    b.y_test, reinterpret_cast<uint64_t*>(b.test_best + (m - 1)), b.ws_embed,
-                                    b.ws_embed_bytes, st));
             RETEXO_TRY(retexo_embed(&model, xte16, ld16, nullptr, n_te, nullptr, 0, nullptr, 0, nullptr, 0, nullptr,
                                     b.y_test, reinterpret_cast<uint64_t*>(b.test_last + (m - 1)), b.ws_embed,
+                                    b.ws_embed_bytes, st));
+            if (gat_train) {                                          // the kept iterate's: x16 then stays for the emission
+                RETEXO_TRY(gat_forward(b.att_best));
+                RETEXO_TRY(retexo_pack_rows(b.x16, 1, ld16, r.d_in, test_idx, n_te, xte16, ld16, nullptr, 0, 0, st));
+            }
+            RETEXO_TRY(retexo_embed(&best, xte16, ld16, nullptr, n_te, nullptr, 0, nullptr, 0, nullptr, 0, nullptr,
+                                    b.y_test, reinterpret_cast<uint64_t*>(b.test_best + (m - 1)), b.ws_embed,
                                     b.ws_embed_bytes, st));
         } else {
             RETEXO_CUDA_TRY(cudaMemsetAsync(b.test_best + (m - 1), 0, sizeof(unsigned long long), st));
             RETEXO_CUDA_TRY(cudaMemsetAsync(b.test_last + (m - 1), 0, sizeof(unsigned long long), st));
+            if (gat_train) RETEXO_TRY(gat_forward(b.att_best));
         }
+        if (gat && out->gat_best && out->gat_best[m - 1])
+            RETEXO_CUDA_TRY(cudaMemcpyAsync(out->gat_best[m - 1], b.att_best, sizeof(float) * (size_t)n_att,
+                                            cudaMemcpyDefault, st));
         if (out->theta_best && out->theta_best[m - 1])
             RETEXO_CUDA_TRY(cudaMemcpyAsync(out->theta_best[m - 1], b.theta_best, sizeof(float) * (size_t)nt,
                                             cudaMemcpyDefault, st));

@@ -222,21 +222,209 @@ __global__ void __launch_bounds__(kGbThreads) gat_bwd_src_kernel(GatBwdArgs a) {
     }
 }
 
+// da_src / da_dst: one block per column sums the per-block partials, each thread its share in index order,
+// then the 256 shares in thread order.
 __global__ void __launch_bounds__(256) gat_bwd_reduce_kernel(const float* partial, int64_t n_blocks, int32_t dim,
                                                              float* da_src, float* da_dst) {
-    const int i = blockIdx.x * 256 + threadIdx.x;
-    if (i >= 2 * dim) return;
-    const int which = i / dim, col = i % dim;
+    __shared__ float share[256];
+    const int which = blockIdx.x / dim, col = blockIdx.x % dim;
     float sum = 0.f;
-    for (int64_t b = 0; b < n_blocks; ++b) sum += partial[(b * 2 + which) * dim + col];
-    (which ? da_dst : da_src)[col] = sum;
+    for (int64_t b = threadIdx.x; b < n_blocks; b += 256) sum += partial[(b * 2 + which) * dim + col];
+    share[threadIdx.x] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float total = 0.f;
+        for (int t = 0; t < 256; ++t) total += share[t];
+        (which ? da_dst : da_src)[col] = total;
+    }
+}
+
+// ---- rows of up to 64 columns, head width a power of two (the shapes of the paper's RetexoGAT): one lane per
+// entry.  A lane fetches its entry's whole row (16-byte loads, all independent) and takes the per-head dot
+// products by itself against the warp's own row, which sits in shared memory; nothing is exchanged between
+// lanes until the row is done, so a row of several hundred entries is a few dozen trips of 32.
+constexpr int kGb64Warps = 4, kGb64Threads = kGb64Warps * kWarp;
+
+template <int HD>
+__global__ void __launch_bounds__(kGb64Threads) gat_bwd_dst64_kernel(GatBwdArgs a) {
+    __shared__ __align__(16) float g_s[kGb64Warps][64];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t v = blockIdx.x * (int64_t)kGb64Warps + warp;
+    if (v >= a.n) return;
+    const int nv = a.dim >> 2;                      // float4 pieces per row
+    bool any = false;
+    for (int c = lane; c < 64; c += kWarp) {
+        const float x = c < a.dim ? a.dz[v * a.lddz + c] : 0.f;
+        g_s[warp][c] = x;
+        any = any || x != 0.f;
+    }
+    const int64_t beg = a.rowptr[v];
+    const int64_t deg = a.rowptr[v + 1] - beg;
+    const int64_t total = deg + (a.self_loop ? 1 : 0);
+    if (!__any_sync(0xffffffffu, any) || total == 0) {
+        if (lane < a.heads) a.stats[v * a.heads + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
+    __syncwarp();
+    constexpr int NH = 64 / HD;                     // heads at most
+    float tv[NH], m[NH], den[NH], csum[NH], a1[NH], a2[NH];
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+        tv[h] = h < a.heads ? a.t[v * a.heads + h] : 0.f;
+        m[h] = -INFINITY; den[h] = 0.f; csum[h] = 0.f; a1[h] = 0.f; a2[h] = 0.f;
+    }
+    for (int64_t e0 = 0; e0 < total; e0 += kWarp) {
+        const bool valid = e0 + lane < total;
+        const int64_t u = !valid ? v : (e0 + lane < deg ? (int64_t)__ldg(a.colidx + beg + e0 + lane) : v);
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+            if (h < a.heads) {
+                const float z = a.s[u * a.heads + h] + tv[h];
+                const float e = valid ? (z > 0.f ? z : a.slope * z) : -INFINITY;
+                const float mn = fmaxf(m[h], warp_max(e));
+                den[h] = den[h] * expf(m[h] - mn) + warp_sum(valid ? expf(e - mn) : 0.f);
+                m[h] = mn;
+            }
+        }
+    }
+    for (int64_t e0 = 0; e0 < total; e0 += kWarp) {
+        const bool valid = e0 + lane < total;
+        const int64_t u = !valid ? v : (e0 + lane < deg ? (int64_t)__ldg(a.colidx + beg + e0 + lane) : v);
+        float dalpha[NH];
+#pragma unroll
+        for (int h = 0; h < NH; ++h) dalpha[h] = 0.f;
+        const float4* row = reinterpret_cast<const float4*>(a.p + u * a.ldp);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            if (i < nv) {
+                const float4 x = valid ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float4 gg = *reinterpret_cast<const float4*>(&g_s[warp][4 * i]);
+                dalpha[(4 * i) / HD] += (x.x * gg.x + x.y * gg.y) + (x.z * gg.z + x.w * gg.w);
+            }
+        }
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+            if (h < a.heads && valid) {
+                const float z = a.s[u * a.heads + h] + tv[h];
+                const float alpha = expf((z > 0.f ? z : a.slope * z) - m[h]) / den[h];
+                const float gp = z > 0.f ? 1.f : a.slope;
+                csum[h] = fmaf(alpha, dalpha[h], csum[h]);
+                a1[h] = fmaf(alpha * gp, dalpha[h], a1[h]);
+                a2[h] = fmaf(alpha, gp, a2[h]);
+            }
+        }
+    }
+#pragma unroll
+    for (int h = 0; h < NH; ++h) {
+        if (h < a.heads) {
+            const float c = warp_sum(csum[h]), s1 = warp_sum(a1[h]), s2 = warp_sum(a2[h]);
+            if (lane == 0) a.stats[v * a.heads + h] = make_float4(m[h], 1.f / den[h], c, s1 - c * s2);
+        }
+    }
+}
+
+template <int HD>
+__global__ void __launch_bounds__(kGb64Threads) gat_bwd_src64_kernel(GatBwdArgs a) {
+    __shared__ __align__(16) float p_s[kGb64Warps][64];
+    __shared__ float red[kGb64Warps][kWarp][65];
+    __shared__ float sm_part[kGb64Warps][2][64];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t u = blockIdx.x * (int64_t)kGb64Warps + warp;
+    const int nv = a.dim >> 2;
+    constexpr int NH = 64 / HD;
+    float acc[64], ds[NH], su[NH];
+#pragma unroll
+    for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+#pragma unroll
+    for (int h = 0; h < NH; ++h) { ds[h] = 0.f; su[h] = 0.f; }
+    for (int c = lane; c < 64; c += kWarp) p_s[warp][c] = (u < a.n && c < a.dim) ? a.p[u * a.ldp + c] : 0.f;
+    __syncwarp();
+    if (u < a.n) {
+#pragma unroll
+        for (int h = 0; h < NH; ++h) if (h < a.heads) su[h] = a.s[u * a.heads + h];
+        const int64_t beg = a.rowptr[u];
+        const int64_t deg = a.rowptr[u + 1] - beg;
+        const int64_t total = deg + (a.self_loop ? 1 : 0);
+        for (int64_t e0 = 0; e0 < total; e0 += kWarp) {
+            const bool valid = e0 + lane < total;
+            const int64_t v = !valid ? u : (e0 + lane < deg ? (int64_t)__ldg(a.colidx + beg + e0 + lane) : u);
+            const bool live = valid && a.stats[v * a.heads].y != 0.f;      // dz_v is zero otherwise
+            float4 g[16];
+            float dalpha[NH], alpha[NH];
+#pragma unroll
+            for (int h = 0; h < NH; ++h) { dalpha[h] = 0.f; alpha[h] = 0.f; }
+            const float4* row = reinterpret_cast<const float4*>(a.dz + v * a.lddz);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                g[i] = (live && i < nv) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float4 pp = *reinterpret_cast<const float4*>(&p_s[warp][4 * i]);
+                dalpha[(4 * i) / HD] += (g[i].x * pp.x + g[i].y * pp.y) + (g[i].z * pp.z + g[i].w * pp.w);
+            }
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+                if (h < a.heads && live) {
+                    const float4 st = a.stats[v * a.heads + h];
+                    const float z = su[h] + a.t[v * a.heads + h];
+                    alpha[h] = expf((z > 0.f ? z : a.slope * z) - st.x) * st.y;
+                    ds[h] = fmaf(alpha[h] * (z > 0.f ? 1.f : a.slope), dalpha[h] - st.z, ds[h]);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float al = alpha[(4 * i) / HD];
+                acc[4 * i] = fmaf(al, g[i].x, acc[4 * i]);
+                acc[4 * i + 1] = fmaf(al, g[i].y, acc[4 * i + 1]);
+                acc[4 * i + 2] = fmaf(al, g[i].z, acc[4 * i + 2]);
+                acc[4 * i + 3] = fmaf(al, g[i].w, acc[4 * i + 3]);
+            }
+        }
+    }
+    // the lanes' partial rows are added in lane order; the lanes' ds in a shuffle tree
+#pragma unroll
+    for (int c = 0; c < 64; ++c) red[warp][lane][c] = acc[c];
+#pragma unroll
+    for (int h = 0; h < NH; ++h) ds[h] = warp_sum(ds[h]);
+    __syncwarp();
+    for (int c = lane; c < 64; c += kWarp) {
+        float sum = 0.f;
+        for (int l = 0; l < kWarp; ++l) sum += red[warp][l][c];
+        float dsc = 0.f, dtc = 0.f;
+#pragma unroll
+        for (int h = 0; h < NH; ++h) if (h == c / HD) dsc = ds[h];
+        if (u < a.n && c < a.dim) {
+            dtc = a.stats[u * a.heads + c / HD].w;
+            const float val = sum + dsc * a.a_src[c] + dtc * a.a_dst[c];
+            if (a.dp) a.dp[u * a.lddp + c] = val;
+            if (a.dp16) a.dp16[u * a.lddp16 + c] = f32_to_bf16(val);
+        } else {
+            dsc = 0.f;
+        }
+        sm_part[warp][0][c] = dsc * p_s[warp][c];
+        sm_part[warp][1][c] = dtc * p_s[warp][c];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2 * a.dim; i += kGb64Threads) {
+        const int which = i / a.dim, col = i % a.dim;
+        float sum = 0.f;
+        for (int w = 0; w < kGb64Warps; ++w) sum += sm_part[w][which][col];
+        a.partial[((int64_t)blockIdx.x * 2 + which) * a.dim + col] = sum;
+    }
+}
+
+template <int HD>
+static int launch_bwd64(const GatBwdArgs& a, float* da_src, float* da_dst, cudaStream_t st) {
+    const unsigned blocks = (unsigned)((a.n + kGb64Warps - 1) / kGb64Warps);
+    gat_bwd_dst64_kernel<HD><<<blocks, kGb64Threads, 0, st>>>(a);
+    gat_bwd_src64_kernel<HD><<<blocks, kGb64Threads, 0, st>>>(a);
+    gat_bwd_reduce_kernel<<<(unsigned)(2 * a.dim), 256, 0, st>>>(a.partial, blocks, a.dim, da_src, da_dst);
+    return launch_status();
 }
 
 template <int NC>
 static int launch_bwd(const GatBwdArgs& a, unsigned blocks, float* da_src, float* da_dst, cudaStream_t st) {
     gat_bwd_dst_kernel<NC><<<blocks, kGbThreads, 0, st>>>(a);
     gat_bwd_src_kernel<NC><<<blocks, kGbThreads, 0, st>>>(a);
-    gat_bwd_reduce_kernel<<<(unsigned)((2 * a.dim + 255) / 256), 256, 0, st>>>(a.partial, blocks, a.dim, da_src, da_dst);
+    gat_bwd_reduce_kernel<<<(unsigned)(2 * a.dim), 256, 0, st>>>(a.partial, blocks, a.dim, da_src, da_dst);
     return launch_status();
 }
 
@@ -250,7 +438,7 @@ extern "C" size_t retexo_gat_backward_workspace_size(int64_t n_nodes, int32_t he
     s.take<float>((size_t)n_nodes * heads);
     s.take<float>((size_t)n_nodes * heads);
     s.take<float4>((size_t)n_nodes * heads);
-    s.take<float>((size_t)((n_nodes + kGbWarps - 1) / kGbWarps + 1) * 2 * (size_t)dim);
+    s.take<float>((size_t)((n_nodes + kGb64Warps - 1) / kGb64Warps + 1) * 2 * (size_t)dim);
     return s.off + kAlign;
 }
 
@@ -284,9 +472,18 @@ extern "C" int retexo_gat_backward(const retexo_csr* g, const float* p, int64_t 
     a.t = ws.take<float>((size_t)n * gat->heads);
     a.stats = ws.take<float4>((size_t)n * gat->heads);
     const unsigned blocks = (unsigned)((n + kGbWarps - 1) / kGbWarps);
-    a.partial = ws.take<float>((size_t)(blocks + 1) * 2 * (size_t)dim);
+    a.partial = ws.take<float>((size_t)((n + kGb64Warps - 1) / kGb64Warps + 1) * 2 * (size_t)dim);
     a.dp = dp; a.lddp = lddp; a.dp16 = static_cast<__nv_bfloat16*>(dp_bf16); a.lddp16 = lddp_bf16;
     gat_bwd_scores_kernel<<<blocks, kGbThreads, 0, st>>>(a);
+    // rows of up to 64 columns in whole 16-byte pieces, head width 8 / 16 / 32 / 64: one lane per entry
+    const int hdw = gat->head_dim;
+    if (dim <= 64 && dim % 4 == 0 && ldp % 4 == 0 && lddz % 4 == 0 && aligned_to(p, 16) && aligned_to(dz, 16) &&
+        (hdw == 8 || hdw == 16 || hdw == 32 || hdw == 64)) {
+        if (hdw == 8) return launch_bwd64<8>(a, da_src, da_dst, st);
+        if (hdw == 16) return launch_bwd64<16>(a, da_src, da_dst, st);
+        if (hdw == 32) return launch_bwd64<32>(a, da_src, da_dst, st);
+        return launch_bwd64<64>(a, da_src, da_dst, st);
+    }
     const int nc = (dim + kWarp - 1) / kWarp;
     if (nc <= 1) return launch_bwd<1>(a, blocks, da_src, da_dst, st);
     if (nc <= 2) return launch_bwd<2>(a, blocks, da_src, da_dst, st);

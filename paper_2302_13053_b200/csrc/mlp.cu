@@ -32,14 +32,6 @@ static int launch_gemm(const GemmArgs& g, cudaStream_t st) {
     return launch_status();
 }
 
-int project_rows_launch(const bf16* A, int64_t lda, const bf16* B, int64_t ldb, int64_t M, int64_t N, int64_t K,
-                        float* out, int64_t ld_out, cudaStream_t st) {
-    GemmArgs g{};
-    g.M = M; g.N = N; g.K = K; g.A = A; g.lda = lda; g.B = B; g.ldb = ldb;
-    g.out_f32 = out; g.ld_f32 = ld_out;
-    return launch_gemm(g, st);
-}
-
 int convert_f32_to_bf16_launch(const float* src, bf16* dst, int64_t n, cudaStream_t st) {
     if (n > 0) f32_to_bf16_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(src, dst, n);
     return launch_status();
@@ -57,6 +49,8 @@ static int64_t tc_split(int64_t M, int64_t N, int64_t K) {
     return s;
 }
 
+int64_t gemm_split(int64_t M, int64_t N, int64_t K) { return tc_split(M, N, K); }
+
 MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval) {
     MlpPlan p{};
     p.d_in = d_in; p.hidden = hidden; p.n_classes = n_classes; p.n_rows = n_rows; p.n_eval = n_eval;
@@ -67,6 +61,7 @@ MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_row
     p.ld_h1 = pad_ld(hidden > 0 ? hidden + 1 : 1);
     p.ld_bits = hidden > 0 ? 2 * (((int64_t)hidden + 63) / 64) : 2;
     p.ld_k = pad_ld(d_in);
+    p.ld_o1 = pad_ld(p.out1);
     p.ld_x1 = pad_ld((int64_t)d_in + 1);
     p.sm_blocks = 4 * ((n_rows + n_eval + 127) / 128);     // up to four loss partials per 128-row tile
     p.split_w1 = tc_split((int64_t)d_in + 1, p.out1, n_rows);
@@ -81,6 +76,7 @@ static void layout(const MlpPlan& p, Taker& t, MlpBuffers* out) {
     const size_t n_all = (size_t)(p.n_rows + p.n_eval);
     const bool h = p.hidden > 0;
     b.w1t16 = t.template take<bf16>((size_t)p.out1 * p.ld_k);
+    b.w1r16 = t.template take<bf16>((size_t)p.d_in * p.ld_o1);
     b.w2t16 = t.template take<bf16>(h ? (size_t)p.n_classes * p.ld_h : 1);
     b.w2p16 = t.template take<bf16>(h ? (size_t)p.hidden * p.ld_dl : 1);
     b.x1 = t.template take<bf16>(n_all * p.ld_x1);
@@ -121,7 +117,7 @@ static int check_model(const retexo_mlp* m) {
 // bf16 shadows of the weights in the orientations the products need.
 static int build_weight_shadows(const MlpPlan& p, const MlpBuffers& b, const float* theta, cudaStream_t st) {
     const int32_t d_in = p.d_in, H = p.hidden, O = p.n_classes, out1 = p.out1;
-    RETEXO_TRY(retexo_pack_rows(theta, 0, out1, out1, nullptr, d_in, nullptr, 0, b.w1t16, p.ld_k, 0, st));
+    RETEXO_TRY(retexo_pack_rows(theta, 0, out1, out1, nullptr, d_in, b.w1r16, b.w1r16 ? p.ld_o1 : 0, b.w1t16, p.ld_k, 0, st));
     if (H > 0) {
         const float* w2 = theta + (int64_t)d_in * out1 + out1;
         RETEXO_TRY(retexo_pack_rows(w2, 0, O, O, nullptr, H, b.w2p16, p.ld_dl, b.w2t16, p.ld_h, 0, st));
@@ -173,12 +169,14 @@ extern "C" size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hid
 
 extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t ldx, int32_t x_has_ones,
                                      const int32_t* y, int64_t n_rows, float* loss_out, float* grad_out,
+                                     float* dx_out, int64_t ld_dx,
                                      void* workspace, size_t workspace_bytes, void* stream) {
     RETEXO_TRY(check_model(model));
     if (!x || !y || n_rows <= 0 || ldx < model->d_in) return RETEXO_ERR_INVALID_ARG;
     if (model->optimizer != RETEXO_SGD && model->optimizer != RETEXO_ADAM) return RETEXO_ERR_INVALID_ARG;
     if (model->optimizer == RETEXO_ADAM && (!model->adam_m || !model->adam_v)) return RETEXO_ERR_INVALID_ARG;
     if (x_has_ones && ldx < (int64_t)model->d_in + 1) return RETEXO_ERR_INVALID_ARG;
+    if (dx_out && ld_dx < model->d_in) return RETEXO_ERR_INVALID_ARG;
     if (!aligned_to(x, 16) || ldx % 8 != 0) return RETEXO_ERR_ALIGNMENT;
     const size_t need = retexo_mlp_train_step_workspace_size(model->d_in, model->hidden, model->n_classes, n_rows);
     if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
@@ -189,7 +187,7 @@ extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t l
     MlpBuffers b{};
     layout(p, ws, &b);
     RETEXO_TRY(mlp_train_step_launch(p, b, model, static_cast<const bf16*>(x), ldx, x_has_ones != 0, y, loss_out, grad_out,
-                                     false, nullptr, st));
+                                     false, nullptr, st, nullptr, dx_out, ld_dx));
     model->step += 1;
     return RETEXO_OK;
 }
@@ -201,7 +199,7 @@ namespace retexo {
 int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
                           const bf16* x, int64_t ldx, bool x_has_ones, const int32_t* y,
                           float* loss_out, float* grad_out, bool shadows_ready, const EvalTail* tail,
-                          cudaStream_t st, const DeviceIter* dev) {
+                          cudaStream_t st, const DeviceIter* dev, float* dx_out, int64_t ld_dx) {
     const int64_t n = p.n_rows;
     const int64_t n_all = n + (tail ? p.n_eval : 0);          // evaluation rows ride along in the forward pass
     const int32_t d_in = p.d_in, H = p.hidden, O = p.n_classes, out1 = p.out1;
@@ -278,6 +276,12 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         if (tail) { fwd.eval_from = n; fwd.y_eval = tail->y_eval; fwd.correct = tail->correct; }
         RETEXO_TRY(tc_gemm_launch(fwd, st));
     }
+    // ---- dX = grad1 W1^T, for a caller that trains what produced X (an aggregator with parameters)
+    if (dx_out) {
+        TcGemm dxg = tc_base(grad1, ld_grad1, b.w1r16, p.ld_o1, n, d_in, out1, b.status);
+        dxg.out_f32 = dx_out; dxg.ld_f32 = ld_dx;
+        RETEXO_TRY(tc_gemm_launch(dxg, st));
+    }
     // ---- [dW1 ; db1] = [X | 1]^T grad1
     TcGemm g1 = tc_base(x, ldx, grad1, ld_grad1, (int64_t)d_in + 1, out1, n, b.status);
     g1.mode = TC_EPI_PARTIAL; g1.splits = (int)p.split_w1; g1.partial = b.pw1;
@@ -297,10 +301,11 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     u.loss_partial = b.loss_partial; u.n_loss = n_loss;      // the partials this launch's loss kernel wrote
     u.inv_rows = 1.0f / (float)n; u.loss_out = loss_out;
     u.status = b.status;
-    u.w1t16 = b.w1t16; u.ld_k = p.ld_k; u.w2t16 = H > 0 ? b.w2t16 : nullptr; u.ld_h = p.ld_h;
+    u.w1t16 = b.w1t16; u.ld_k = p.ld_k; u.w1r16 = b.w1r16; u.ld_o1 = p.ld_o1; u.w2t16 = H > 0 ? b.w2t16 : nullptr; u.ld_h = p.ld_h;
     u.w2p16 = H > 0 ? b.w2p16 : nullptr; u.ld_dl = p.ld_dl;
     u.d_in = d_in; u.out1 = out1; u.hidden = H; u.n_classes = O;
     if (tail) {
+        u.snap_decision = tail->decision;
         u.snap_cur = tail->correct; u.snap_best = tail->best; u.snap_have = tail->have_best; u.theta_best = tail->theta_best;
         u.done = tail->done; u.rec_iter = tail->iter; u.rec_best_iter = tail->best_iter; u.rec_history_slot = tail->history_slot;
     }

@@ -216,12 +216,14 @@ struct UpdateArgs {
     const int32_t* status;     // non-zero: a kernel of this step gave up on a bounded wait -> loss = NaN
     // bf16 copies of the updated weights in the orientations the next products read (optional)
     bf16* w1t16; int64_t ld_k;       // W1^T [out1 x ld_k]
+    bf16* w1r16; int64_t ld_o1;      // W1   [d_in x ld_o1]
     bf16* w2t16; int64_t ld_h;       // W2^T [n_classes x ld_h]
     bf16* w2p16; int64_t ld_dl;      // W2   [hidden x ld_dl]
     int32_t d_in, out1, hidden, n_classes;
     // keep-the-best snapshot of theta as it is before this update (optional, see EvalTail)
     unsigned long long* snap_cur; unsigned long long* snap_best; int32_t* snap_have;
     float* theta_best;
+    int32_t* snap_decision;          // (optional) receives whether this launch copied theta to theta_best
     // bookkeeping of the validation count by the last block to finish (optional, see EvalTail)
     unsigned long long* done; int32_t rec_iter; int32_t* rec_best_iter; unsigned long long* rec_history_slot;
     // iteration state on the device (optional, see DeviceIter; needs `done`): with s = *step_dev updates applied
@@ -232,7 +234,7 @@ struct UpdateArgs {
 
 // base^e for a whole exponent by repeated squaring (a handful of double multiplications: the library
 // power function costs microseconds on a part with few double-precision units).
-__device__ __forceinline__ double pow_whole(double base, unsigned long long e) {
+__host__ __device__ __forceinline__ double pow_whole(double base, unsigned long long e) {
     double r = 1.0;
     while (e) {
         if (e & 1ull) r *= base;
@@ -279,6 +281,7 @@ __device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p,
         if (u.w1t16 && q < (int64_t)u.d_in * u.out1) {
             const int64_t k = q / u.out1, j = q % u.out1;
             u.w1t16[j * u.ld_k + k] = f32_to_bf16(t);
+            if (u.w1r16) u.w1r16[k * u.ld_o1 + j] = f32_to_bf16(t);
         }
     } else if (q < (int64_t)u.hidden * u.n_classes) {
         const int64_t jh = q / u.n_classes, c = q % u.n_classes;
@@ -327,6 +330,7 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
         __syncthreads();
         if (is_last && threadIdx.x == 0) {
             __threadfence();
+            if (u.snap_decision) *u.snap_decision = snapshot ? 1 : 0;
             if (u.snap_cur) {
                 const unsigned long long cur = *u.snap_cur;
                 unsigned long long* slot = u.step_dev ? (u.history_base && step_now > 0 ? u.history_base + (step_now - 1) : nullptr)

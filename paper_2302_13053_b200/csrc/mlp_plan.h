@@ -21,6 +21,7 @@ struct MlpPlan {
     int64_t ld_h1;                          // row stride of [Hd | 1] (hidden + 1 rounded up to 64)
     int64_t ld_bits;                        // words per row of the ReLU bits (two per 64 hidden units)
     int64_t ld_k;                           // row stride of W1^T (d_in rounded up to 64)
+    int64_t ld_o1;                          // row stride of the bf16 copy of W1 (out1 rounded up to 64)
     int64_t ld_x1;                          // row stride of the workspace copy [X | 1] (d_in + 1 rounded up to 64)
     int64_t sm_blocks;                      // loss partials the workspace has room for
     int64_t split_w1, split_w2;             // split-K factors of the two weight-gradient products
@@ -28,6 +29,7 @@ struct MlpPlan {
 
 struct MlpBuffers {
     __nv_bfloat16* w1t16;                   // W1^T            [out1 x ld_k]
+    __nv_bfloat16* w1r16;                   // W1              [d_in x ld_o1]  (may be null: retexo_embed does not need it)
     __nv_bfloat16* w2t16;                   // W2^T            [n_classes x ld_h]
     __nv_bfloat16* w2p16;                   // W2, padded rows [hidden x ld_dl]
     __nv_bfloat16* x1;                      // [X | 1]         [n x ld_x1]  (only when the caller's batch has no column of ones)
@@ -41,6 +43,9 @@ struct MlpBuffers {
     float* pw2;                             // [split_w2 x (hidden+1) x n_classes]   partials of [dW2 ; db2]
     int32_t* status;                        // raised by a tensor-core kernel whose bounded wait gave up
 };
+
+// Split-K factor the library uses for a weight-gradient product C[M x N] = A^T B reduced over K rows.
+int64_t gemm_split(int64_t M, int64_t N, int64_t K);
 
 MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval = 0);
 size_t mlp_step_workspace_size(const MlpPlan& p);
@@ -64,6 +69,9 @@ struct EvalTail {
     int32_t iter = 0;
     int32_t* best_iter = nullptr;
     unsigned long long* history_slot = nullptr;
+    // (optional, with `done`) receives 1 if this launch copied theta to theta_best, else 0: a caller that keeps
+    // further parameters next to theta (a trained aggregator) takes the same decision from it
+    int32_t* decision = nullptr;
 };
 
 // Iteration state kept on the device, so that every iteration of a round is the same launch sequence
@@ -90,7 +98,8 @@ void mlp_step_buffers(const MlpPlan& p, void* workspace, size_t bytes, MlpBuffer
 int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
                           const __nv_bfloat16* x, int64_t ldx, bool x_has_ones,
                           const int32_t* y, float* loss_out, float* grad_out, bool shadows_ready,
-                          const EvalTail* tail, cudaStream_t st, const DeviceIter* dev = nullptr);
+                          const EvalTail* tail, cudaStream_t st, const DeviceIter* dev = nullptr,
+                          float* dx_out = nullptr, int64_t ld_dx = 0);      // dx_out: fp32 [n_rows x ld_dx], dLoss / dX
 
 // Forward + arg-max + hit count over a dense batch with the weight copies in `b` (which must
 // hold model->theta): what validation needs after every iteration.  hd_ws: bf16 [n_rows x p.ld_h].
@@ -98,9 +107,6 @@ int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
                           const __nv_bfloat16* x, int64_t ldx, int64_t n_rows, __nv_bfloat16* hd_ws,
                           const int32_t* y, unsigned long long* correct, cudaStream_t st);
 
-// out[M x N] (fp32, row stride ld_out) = A[M x K] (bf16) * B[K x N] (bf16), no bias.
-int project_rows_launch(const __nv_bfloat16* A, int64_t lda, const __nv_bfloat16* B, int64_t ldb, int64_t M, int64_t N,
-                        int64_t K, float* out, int64_t ld_out, cudaStream_t st);
 int convert_f32_to_bf16_launch(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st);
 
 }  // namespace retexo

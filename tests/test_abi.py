@@ -71,16 +71,16 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
                                             None, None, None, C.c_size_t(0), None) == INVALID
     m = _Mlp(0, 4, 3, 256, None, None, 1, 0.1, 0.9, 0.999, 1e-8, 0)
     assert lib.retexo_mlp_train_step(C.byref(m), C.c_void_p(256), C.c_int64(8), C.c_int32(0),
-                                     C.c_void_p(256), C.c_int64(4), None, None, None, C.c_size_t(0), None) == INVALID
+                                     C.c_void_p(256), C.c_int64(4), None, None, None, C.c_int64(0), None, C.c_size_t(0), None) == INVALID
     m = _Mlp(8, 4, 3, 256, None, None, 1, 0.1, 0.9, 0.999, 1e-8, 0)      # Adam without moments
     assert lib.retexo_mlp_train_step(C.byref(m), C.c_void_p(256), C.c_int64(8), C.c_int32(0),
-                                     C.c_void_p(256), C.c_int64(4), None, None, None, C.c_size_t(0), None) == INVALID
+                                     C.c_void_p(256), C.c_int64(4), None, None, None, C.c_int64(0), None, C.c_size_t(0), None) == INVALID
     m = _Mlp(8, 4, 3, 256, None, None, 0, 0.1, 0.9, 0.999, 1e-8, 0)
     ALIGNMENT = 3
     assert lib.retexo_mlp_train_step(C.byref(m), C.c_void_p(256), C.c_int64(9), C.c_int32(0),
-                                     C.c_void_p(256), C.c_int64(4), None, None, None, C.c_size_t(0), None) == ALIGNMENT
+                                     C.c_void_p(256), C.c_int64(4), None, None, None, C.c_int64(0), None, C.c_size_t(0), None) == ALIGNMENT
     # a column of ones is claimed, but the rows have no room for it
     assert lib.retexo_mlp_train_step(C.byref(m), C.c_void_p(256), C.c_int64(8), C.c_int32(1),
-                                     C.c_void_p(256), C.c_int64(4), None, None, None, C.c_size_t(0), None) == INVALID
+                                     C.c_void_p(256), C.c_int64(4), None, None, None, C.c_int64(0), None, C.c_size_t(0), None) == INVALID
     assert lib.retexo_embed(C.byref(m), C.c_void_p(256), C.c_int64(8), None, C.c_int64(4), None, C.c_int64(0), None,
                             C.c_int64(0), None, C.c_int64(0), None, None, None, None, C.c_size_t(0), None) == WORKSPACE

@@ -147,3 +147,25 @@ def test_argmax_tie_rule_lowest_index():
     x16, _ = B().retexo_pack_rows(dev(np.ones((5, 8), dtype=np.float32)))
     out = B().retexo_embed(gpu, x16, want_pred=True)
     assert out["pred"].cpu().tolist() == [1] * 5
+
+
+@pytest.mark.parametrize("d_in,hidden,n_classes,n", [(64, 64, 4, 300), (64, 0, 4, 300), (33, 20, 5, 129), (128, 256, 41, 513)])
+def test_input_gradient_matches_the_checker(d_in, hidden, n_classes, n):
+    """dLoss / dx, the extra output a round with a trained aggregator needs."""
+    rng = np.random.default_rng(n + hidden)
+    x = rng.standard_normal((n, d_in)).astype(np.float32)
+    y = rng.integers(0, n_classes, n).astype(np.int32)
+    ref, gpu = make_pair(d_in, hidden, n_classes, 3, opt=oracle.SGD, lr=0.01)
+    x16, _ = B().retexo_pack_rows(dev(x), None, ones=True)
+    x_host = x16[:, :d_in].float().cpu().numpy()
+    rl, rg, rdx = ref.train_step_dx(x_host, y)
+    gl, gg, gdx = B().retexo_mlp_train_step(gpu, x16, dev(y), x_has_ones=True, return_grad=True, return_dx=True)
+    assert abs(gl.item() - rl) <= 2e-4 * max(1.0, abs(rl))
+    gdx = gdx.cpu().numpy().astype(np.float64)
+    err, scale = np.abs(gdx - rdx), np.abs(rdx).max()
+    assert err.max() <= 5e-3 * scale + 1e-9, (err.max(), scale)
+    assert np.median(err) <= 1e-4 * scale
+    # asking for it changes nothing else
+    _, gpu2 = make_pair(d_in, hidden, n_classes, 3, opt=oracle.SGD, lr=0.01)
+    gl2, gg2 = B().retexo_mlp_train_step(gpu2, x16, dev(y), x_has_ones=True, return_grad=True)
+    assert gl2.item() == gl.item() and torch.equal(gg, gg2) and torch.equal(gpu.theta, gpu2.theta)
