@@ -174,6 +174,11 @@ typedef struct retexo_mlp {
      * retexo_embed (evaluation) never drops. */
     float dropout;
     uint64_t dropout_seed;
+    /* Optional device int32.  Every device-side wait of the tensor-core kernels is bounded; one that runs out
+     * (it never should) makes its block give up in order and raises a status word.  After the kernels of a
+     * retexo_mlp_train_step / retexo_embed call the word is copied here: RETEXO_OK, or RETEXO_ERR_TIMEOUT
+     * (the loss of that step is then NaN and its outputs are not to be used).  Read it after synchronising. */
+    int32_t* status_out;
 } retexo_mlp;
 
 int64_t retexo_theta_size(int32_t d_in, int32_t hidden, int32_t n_classes);
@@ -374,6 +379,9 @@ typedef struct retexo_lmp_outputs {
     float* const* theta_best;       /* HOST array of K pointers receiving each round's kept theta; may be NULL */
     float* const* gat_best;         /* GAT only: HOST array of K pointers receiving each round's kept
                                        [W_att | a_src | a_dst]; may be NULL */
+    int32_t* status;                /* optional, one int32 (device, or host with memory_is_host): RETEXO_OK, or
+                                       RETEXO_ERR_TIMEOUT if a bounded device-side wait ran out in any round
+                                       (the results are then not to be used) */
 } retexo_lmp_outputs;
 
 size_t retexo_lmp_workspace_size(const retexo_lmp_config* cfg, int64_t n_nodes, int64_t n_edges,

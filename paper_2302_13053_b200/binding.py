@@ -40,7 +40,8 @@ class _Mlp(C.Structure):
     _fields_ = [("d_in", C.c_int32), ("hidden", C.c_int32), ("n_classes", C.c_int32),
                 ("theta", C.c_void_p), ("adam_m", C.c_void_p), ("adam_v", C.c_void_p),
                 ("optimizer", C.c_int32), ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
-                ("eps", C.c_float), ("step", C.c_int64), ("dropout", C.c_float), ("dropout_seed", C.c_uint64)]
+                ("eps", C.c_float), ("step", C.c_int64), ("dropout", C.c_float), ("dropout_seed", C.c_uint64),
+                ("status_out", C.c_void_p)]
 
 
 class _LmpConfig(C.Structure):
@@ -67,7 +68,8 @@ class _LmpOutputs(C.Structure):
     _fields_ = [("loss_history", C.c_void_p), ("val_correct", C.c_void_p), ("best_val_correct", C.c_void_p),
                 ("best_iter", C.c_void_p), ("test_correct", C.c_void_p), ("test_correct_last", C.c_void_p),
                 ("counts", C.c_void_p), ("final_logits", C.c_void_p), ("ld_logits", C.c_int64),
-                ("final_pred", C.c_void_p), ("theta_best", C.POINTER(C.c_void_p)), ("gat_best", C.POINTER(C.c_void_p))]
+                ("final_pred", C.c_void_p), ("theta_best", C.POINTER(C.c_void_p)), ("gat_best", C.POINTER(C.c_void_p)),
+                ("status", C.c_void_p)]
 
 
 EXPORTS = ["retexo_status_string", "retexo_version", "retexo_validate_csr", "retexo_aggregate_workspace_size",
@@ -247,8 +249,10 @@ class Mlp:
         self.theta = torch.from_numpy(theta).to(device)
         self.m = torch.zeros_like(self.theta)
         self.v = torch.zeros_like(self.theta)
+        self.status = torch.full((1,), -1, dtype=torch.int32, device=device)      # written by every step / embed call
         self.c = _Mlp(self.d_in, self.hidden, self.n_classes, self.theta.data_ptr(), self.m.data_ptr(),
-                      self.v.data_ptr(), optimizer, lr, beta1, beta2, eps, 0, dropout, dropout_seed)
+                      self.v.data_ptr(), optimizer, lr, beta1, beta2, eps, 0, dropout, dropout_seed,
+                      self.status.data_ptr())
 
     @property
     def step(self) -> int:
@@ -426,6 +430,8 @@ class LmpProblem:
         self.final_pred = out((n,), torch.int32) if want_logits else None
         self.theta_best = [out(t.shape, torch.float32) for t in self.theta0]
         self.gat_best = [out(t.shape, torch.float32) for t in self.gat_w] if self.gat_w else None
+        self.status = out((1,), torch.int32)
+        self.status.fill_(-1)
         self.d2h_bytes = sum(t.numel() * t.element_size() for t in
                              [self.loss_history, self.val_correct, self.best_val, self.best_iter, self.test_correct,
                               self.test_last, self.counts] + self.theta_best + (self.gat_best or []) +
@@ -449,7 +455,8 @@ class LmpProblem:
                                    self.final_logits.data_ptr() if want_logits else None, n_classes,
                                    self.final_pred.data_ptr() if want_logits else None,
                                    C.cast(self._best_arr, C.POINTER(C.c_void_p)),
-                                   C.cast(self._gat_best_arr, C.POINTER(C.c_void_p)) if self._gat_best_arr else None)
+                                   C.cast(self._gat_best_arr, C.POINTER(C.c_void_p)) if self._gat_best_arr else None,
+                                   self.status.data_ptr())
         need = lib().retexo_lmp_workspace_size(C.byref(self.cfg), C.c_int64(n), C.c_int64(e),
                                                C.c_int64(self.train_idx.numel()), C.c_int64(self.val_idx.numel()),
                                                C.c_int64(self.test_idx.numel()),
@@ -477,7 +484,8 @@ class LmpProblem:
                     final_logits=None if self.final_logits is None else cpu(self.final_logits),
                     final_pred=None if self.final_pred is None else cpu(self.final_pred),
                     theta_best=[cpu(t) for t in self.theta_best],
-                    gat_best=[cpu(t) for t in self.gat_best] if self.gat_best else None)
+                    gat_best=[cpu(t) for t in self.gat_best] if self.gat_best else None,
+                    status=int(cpu(self.status)[0]))
 
 
 def retexo_lmp_train(problem: LmpProblem) -> None:

@@ -88,6 +88,12 @@ __global__ void att_update_kernel(AttUpdateArgs a) {
     a.v[p] = v;
     a.att[p] -= a.lr * (m / c1) / (sqrtf(v / c2) + a.eps);
 }
+// Keeps the first non-zero status of the run.
+__global__ void merge_status_kernel(int32_t* run, const int32_t* a, const int32_t* b) {
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    if (*run == 0 && a && *a != 0) *run = *a;
+    if (*run == 0 && b && *b != 0) *run = *b;
+}
 __global__ void fill_u64_kernel(unsigned long long* p, int64_t n, unsigned long long v) {
     const int64_t i = blockIdx.x * 256ll + threadIdx.x;
     if (i < n) p[i] = v;
@@ -172,7 +178,7 @@ struct LmpBuffers {
     int32_t *y_tr, *y_val, *y_test;
     float *theta, *adam_m, *adam_v, *theta_best;
     unsigned long long *cur_correct, *best_correct, *scratch_u64;
-    int32_t *have_best, *best_iter_cur;
+    int32_t *have_best, *best_iter_cur, *run_status;
     // device copies of the outputs
     float* loss_history; unsigned long long* val_history;
     unsigned long long *best_val, *test_best, *test_last; int32_t* best_iter;
@@ -255,6 +261,7 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
     l.scratch_u64 = t.template take<unsigned long long>(4);
     l.have_best = t.template take<int32_t>(4);
     l.best_iter_cur = t.template take<int32_t>(4);
+    l.run_status = t.template take<int32_t>(4);
     l.loss_history = t.template take<float>((size_t)c.K * c.R);
     l.val_history = t.template take<unsigned long long>((size_t)c.K * c.R);
     l.best_val = t.template take<unsigned long long>((size_t)c.K);
@@ -373,6 +380,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
     if (n_te) gather_i32_kernel<<<(unsigned)((n_te + 255) / 256), 256, 0, st>>>(labels, test_idx, n_te, b.y_test);
     fill_u64_kernel<<<(unsigned)(((int64_t)c.K * c.R + 255) / 256), 256, 0, st>>>(b.val_history, (int64_t)c.K * c.R,
                                                                                   ~0ull);
+    RETEXO_CUDA_TRY(cudaMemsetAsync(b.run_status, 0, sizeof(int32_t), st));
 
     // ---- messages and bytes across the partition, all rounds
     if (part) {
@@ -460,6 +468,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         model.optimizer = c.optimizer; model.lr = c.lr; model.beta1 = c.beta1; model.beta2 = c.beta2;
         model.eps = c.eps; model.step = 0;
         model.dropout = c.dropout; model.dropout_seed = c.dropout_seed + (uint64_t)(m - 1);
+        model.status_out = nullptr;
         retexo_mlp best = model;
         best.theta = b.theta_best;
 
@@ -611,6 +620,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
             RETEXO_CUDA_TRY(cudaMemcpyAsync(out->theta_best[m - 1], b.theta_best, sizeof(float) * (size_t)nt,
                                             cudaMemcpyDefault, st));
 
+        merge_status_kernel<<<1, 32, 0, st>>>(b.run_status, sb.status, c.aggr == RETEXO_GAT ? b.status : nullptr);
         // ---- emit Q^m (classifier dropped) or the final logits
         if (m < c.K) {
             float* qn = b.q[(m - 1) & 1];
@@ -637,6 +647,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
     if (out->best_iter) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->best_iter, b.best_iter, sizeof(int32_t) * c.K, out_kind, st));
     if (out->test_correct) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->test_correct, b.test_best, sizeof(uint64_t) * c.K, out_kind, st));
     if (out->test_correct_last) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->test_correct_last, b.test_last, sizeof(uint64_t) * c.K, out_kind, st));
+    if (out->status) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->status, b.run_status, sizeof(int32_t), out_kind, st));
     if (out->counts && part) RETEXO_CUDA_TRY(cudaMemcpyAsync(out->counts, b.counts, sizeof(uint64_t) * (4 + c.K), out_kind, st));
     if (host) {
         if (out->final_logits)

@@ -314,6 +314,8 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         u.loss_out = nullptr;
     }
     reduce_update_kernel<<<(unsigned)((p.nt + 255) / 256), 256, 0, st>>>(u);
+    if (model->status_out)
+        RETEXO_CUDA_TRY(cudaMemcpyAsync(model->status_out, b.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
     return launch_status();
 }
 
@@ -444,9 +446,13 @@ extern "C" int retexo_embed(const retexo_mlp* model, const void* x, int64_t ldx,
             fwd.pred = pred_out; fwd.y = y; fwd.correct = correct;
             RETEXO_TRY(tc_gemm_launch(fwd, st));
         }
+        if (model->status_out)
+            RETEXO_CUDA_TRY(cudaMemcpyAsync(model->status_out, b.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
         return launch_status();
     }
     if (pred_out || correct)
         argmax_kernel<<<(unsigned)((n_rows + 255) / 256), 256, 0, st>>>(lg, ld_lg, n_rows, O, pred_out, y, correct);
+    if (model->status_out)
+        RETEXO_CUDA_TRY(cudaMemcpyAsync(model->status_out, b.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
     return launch_status();
 }

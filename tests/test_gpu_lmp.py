@@ -155,6 +155,7 @@ def check_rounds_from_the_same_start(w, R, freeze=False):
                            eval_every=R, forced_theta=got["theta_best"], train_attention=trained,
                            forced_att=got["gat_best"] if trained else None)
     check_counts(ref, got)
+    assert got["status"] == 0                       # written by the run: no bounded device-side wait ran out
     n_val, n_test = len(w.val_idx), len(w.test_idx)
     for m, rd in enumerate(ref["rounds"]):
         gl, rl = got["loss_history"][m], rd["losses"]

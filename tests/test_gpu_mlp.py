@@ -94,6 +94,7 @@ def test_train_steps_track_the_checker(d_in, hidden, n_classes, n, opt):
         given.apply_update(gg)
         gt = gpu.theta.cpu().numpy().astype(np.float64)
         assert np.abs(gt - given.theta).max() <= 2e-6 * max(1.0, np.abs(given.theta).max()), it
+        assert int(gpu.status.item()) == 0          # the status word reaches the caller: no bounded wait ran out
 
 
 def test_zero_weights_give_log_of_class_count():
