@@ -179,7 +179,7 @@ __device__ __forceinline__ void stage_block_from_global(const __nv_bfloat16* src
 
 // MODE (a TcEpilogue value) is a template parameter so that every instantiation carries the registers of
 // its own epilogue only.
-template <int BN, int STAGES, int MODE, int EW>
+template <int BN, int STAGES, int MODE, int EW, bool PAIR = false>
 __global__ void __launch_bounds__(64 + 32 * EW, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_rows, TcKernelArgs g) {
@@ -191,7 +191,15 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     constexpr int NACC = 2 * TG;                            // accumulators in tensor memory
     static_assert(BN % (32 * CP) == 0 && NACC * BN <= 512, "tile split");
     extern __shared__ uint8_t smem_raw[];
-    constexpr uint32_t kABytes = kTcBM * kTcBK * 2, kBBytes = BN * kTcBK * 2, kStageBytes = kABytes + kBBytes;
+    // PAIR: the block is one of a pair (cluster of two) that shares 256-row tiles: it holds its own 128 rows of A
+    // and its own half of the B tile (BN / 2 rows), so a stage is a third smaller and every B tile crosses the
+    // L2 -> SM path once per 256 rows instead of once per 128.
+    constexpr uint32_t kABytes = kTcBM * kTcBK * 2, kBBytes = (PAIR ? BN / 2 : BN) * kTcBK * 2, kStageBytes = kABytes + kBBytes;
+    constexpr int kTileRows = PAIR ? 2 * kTcBM : kTcBM;
+    static_assert(!PAIR || (MODE != TC_EPI_PARTIAL && BN == 256 && TG == 1), "pairs: K-major 256-column tiles");
+    const uint32_t pair_rank = PAIR ? cluster_rank() : 0u;
+    const int64_t tile_first = PAIR ? (int64_t)(blockIdx.x >> 1) : (int64_t)blockIdx.x;
+    const int64_t tile_stride = PAIR ? (int64_t)(gridDim.x >> 1) : (int64_t)gridDim.x;
     // The split-K products reduce over the batch, and their operands (activations and gradients, one batch row
     // per line) are read as they lie in memory: M and N are the contiguous dimensions ("MN-major" operands).
     constexpr bool kMnMajor = MODE == TC_EPI_PARTIAL;
@@ -209,7 +217,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     float (*xch_all)[2][128] = reinterpret_cast<float (*)[2][128]>(stage_base + EW * kStageBytesPerWarp);   // [TG][4][2][128]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t n_m = (g.M + kTcBM - 1) / kTcBM, n_n = (g.N + BN - 1) / BN;
+    const int64_t n_m = (g.M + kTileRows - 1) / kTileRows, n_n = (g.N + BN - 1) / BN;
     const int64_t per_split = n_m * n_n;
     const int64_t n_tiles = per_split * g.splits;
 
@@ -217,16 +225,23 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         for (int s = 0; s < STAGES; ++s) { mbar_init(full + s, 1); mbar_init(empty + s, 1); }
         // the arg-max epilogue lets one thread own a whole row of logits: it uses four of the eight warps
         const bool row_owner = BN == 64 && MODE == TC_EPI_ARGMAX;
-        for (int b = 0; b < NACC; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, row_owner ? 4 : EW / TG); }
+        // (pairs: the even block's "accumulator drained" barrier collects the epilogue warps of both blocks)
+        for (int b = 0; b < NACC; ++b) { mbar_init(acc_full + b, 1); mbar_init(acc_empty + b, row_owner ? 4 : (PAIR ? 2 : 1) * EW / TG); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {      // tensor memory: NACC accumulators of BN fp32 columns x 128 lanes
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(NACC * BN));
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+        if constexpr (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(NACC * BN));
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(NACC * BN));
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+        }
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();      // both blocks' barriers exist before either signals the other's
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_acc = *tmem_slot;
 
@@ -234,17 +249,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (lane == 0) {
             int64_t it = 0;                       // k-blocks issued so far, over all tiles
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+            for (int64_t t = tile_first; t < n_tiles && ok; t += tile_stride) {
                 const int64_t z = t / per_split, rem = t % per_split;
-                const int32_t m0 = (int32_t)((rem % n_m) * kTcBM), n0 = (int32_t)((rem / n_m) * BN);
+                const int32_t m0 = (int32_t)((rem % n_m) * kTileRows + pair_rank * kTcBM), n0 = (int32_t)((rem / n_m) * BN);
                 const int32_t kb0 = (int32_t)z * g.k_blocks_per_split;
                 const int32_t kb1 = min(g.k_blocks_total, kb0 + g.k_blocks_per_split);
                 for (int32_t kb = kb0; kb < kb1; ++kb, ++it) {
                     const int s = (int)(it % STAGES);
                     const uint32_t ph = (uint32_t)(it / STAGES) & 1;
                     if (!mbar_wait(empty + s, ph ^ 1, g.status, abort_flag)) { ok = false; break; }
-                    mbar_expect_tx(full + s, kStageBytes);
                     uint8_t* a_dst = tiles + s * kStageBytes;
+                    if constexpr (PAIR) {
+                        // the even block's barrier counts the bytes of both blocks' loads
+                        if (pair_rank == 0) mbar_expect_tx(full + s, 2 * kStageBytes);
+                        tma_load_2d_pair(a_dst, &map_a, kb * kTcBK, m0, full + s);
+                        tma_load_2d_pair(a_dst + kABytes, &map_b, kb * kTcBK, n0 + (int32_t)pair_rank * (BN / 2), full + s);
+                        continue;
+                    }
+                    mbar_expect_tx(full + s, kStageBytes);
                     if constexpr (kMnMajor) {
                         // operands stored [reduction index][M or N]: boxes of 64 reduction rows x 64 elements
 #pragma unroll
@@ -259,7 +281,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     }
                 }
             }
-            if (*abort_flag) {    // await (bounded) what was issued and not consumed, so nothing lands after exit
+            if (*abort_flag && !(PAIR && pair_rank != 0)) {    // await (bounded) what was issued and not consumed, so nothing lands after exit
                 for (int64_t i = it > STAGES ? it - STAGES : 0; i < it; ++i) {
                     const int s = (int)(i % STAGES);
                     const uint32_t ph = (uint32_t)(i / STAGES) & 1;
@@ -268,11 +290,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BN, kMnMajor, kMnMajor);
+        if (lane == 0 && pair_rank == 0) {        // (of a pair, the even block issues the MMAs for both)
+            constexpr uint32_t idesc = make_idesc(BN, kMnMajor, kMnMajor, kTileRows);
             int64_t it = 0, lt = 0;               // k-blocks consumed, tiles done by this block
             bool ok = true;
-            for (int64_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++lt) {
+            for (int64_t t = tile_first; t < n_tiles && ok; t += tile_stride, ++lt) {
                 const int64_t z = t / per_split;
                 const int32_t kb0 = (int32_t)z * g.k_blocks_per_split;
                 const int32_t kb1 = min(g.k_blocks_total, kb0 + g.k_blocks_per_split);
@@ -295,15 +317,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                         for (int k = 0; k < kTcBK / 16; ++k)      // 16 reduction rows = two 1024-byte atoms: +128 in 16-byte units
                             umma_bf16(acc_addr, adesc + 128 * k, bdesc + 128 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+                    } else if constexpr (PAIR) {
+                        // one MMA over both blocks' shared memory (same offsets in either) and tensor memory
+                        const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(a_addr + kABytes);
+#pragma unroll
+                        for (int k = 0; k < kTcBK / 16; ++k)
+                            umma_bf16_pair(acc_addr, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
                     } else {
                         const uint64_t adesc = make_smem_desc(a_addr), bdesc = make_smem_desc(a_addr + kABytes);
 #pragma unroll
                         for (int k = 0; k < kTcBK / 16; ++k)      // 16 bf16 = 32 bytes per MMA along K: +2 in 16-byte units
                             umma_bf16(acc_addr, adesc + 2 * k, bdesc + 2 * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
                     }
-                    umma_commit(empty + s);                   // frees the stage once these MMAs have read it
+                    if constexpr (PAIR) umma_commit_pair(empty + s);      // frees the stage in both blocks
+                    else umma_commit(empty + s);              // frees the stage once these MMAs have read it
                 }
-                if (ok) umma_commit(acc_full + b);            // accumulator complete (at once for an empty K range)
+                if (ok) {                                     // accumulator complete (at once for an empty K range)
+                    if constexpr (PAIR) umma_commit_pair(acc_full + b);
+                    else umma_commit(acc_full + b);
+                }
             }
         }
     } else {
@@ -341,13 +373,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             gate_have = true;
         };
-        if constexpr (kGated) gate_prefetch(blockIdx.x + (int64_t)gi * gridDim.x, half * kPartCols);
+        if constexpr (kGated) gate_prefetch(tile_first + (int64_t)gi * tile_stride, half * kPartCols);
         int64_t lt = gi;
-        for (int64_t t = blockIdx.x + (int64_t)gi * gridDim.x; t < n_tiles && !(row_owner && half == 1);
-             t += (int64_t)TG * gridDim.x, lt += TG) {
+        for (int64_t t = tile_first + (int64_t)gi * tile_stride; t < n_tiles && !(row_owner && half == 1);
+             t += (int64_t)TG * tile_stride, lt += TG) {
             const int64_t z = t / per_split, rem = t % per_split;
             const int64_t mt = rem % n_m;
-            const int64_t m0 = mt * kTcBM, n0 = (rem / n_m) * BN;
+            const int64_t m0 = mt * kTileRows + (int64_t)pair_rank * kTcBM, n0 = (rem / n_m) * BN;
             const int32_t kb0 = (int32_t)z * g.k_blocks_per_split;
             const int32_t n_kb = min(g.k_blocks_total, kb0 + g.k_blocks_per_split) - kb0;
             const int b = (int)(lt % NACC);
@@ -534,7 +566,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
                         for (int i = 0; i < 4; ++i) gate_cur[i] = gate_next[i];
                         if (c0 + 32 < c_end) gate_prefetch(t, c0 + 32);
-                        else gate_prefetch(t + (int64_t)TG * gridDim.x, c_begin);
+                        else gate_prefetch(t + (int64_t)TG * tile_stride, c_begin);
                         if (gate_runs && out_map) {
                             // the two staging blocks take turns: the bulk store issued two chunks ago has read this one
                             flip ^= 1;
@@ -641,15 +673,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             // hand the accumulator back to the MMA thread
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
-            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(acc_empty + b)) : "memory");
+            if (lane == 0) {
+                if constexpr (PAIR) mbar_arrive_even_block(acc_empty + b);      // the MMA thread lives in the even block
+                else asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(acc_empty + b)) : "memory");
+            }
         }
         if (lane == 0) bulk_wait_all();       // this thread's bulk stores have reached global memory
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();   // neither block leaves while the other may still signal it or use its tensor memory
     if (warp == 1) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(NACC * BN));
+        if constexpr (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(NACC * BN));
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(NACC * BN));
     }
 }
 
@@ -746,6 +783,67 @@ static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensor
     return launch_status();
 }
 
+// The forward products in pairs of thread blocks (clusters of two): 256-row tiles, each block loading its own
+// rows of A and half of the B tile.  `t`'s epilogue arguments are those of launch_tc_mode.
+template <int MODE>
+static int launch_tc_pair(const TcGemm& t, cudaStream_t st) {
+    constexpr int BN = 256, EW = 8, STAGES = 6;
+    constexpr size_t smem = (size_t)STAGES * (kTcBM * kTcBK * 2 + (BN / 2) * kTcBK * 2) + 1024 + 1024 + EW * kStageBytesPerWarp;
+    static_assert(smem <= 227 * 1024, "shared memory budget");
+    auto kernel = tc_gemm_kernel<BN, STAGES, MODE, EW, true>;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return RETEXO_ERR_CUDA;
+    }
+    CUtensorMap ma, mb, m_rows;
+    memset(&m_rows, 0, sizeof(m_rows));
+    if (!make_map(&ma, t.A, t.M, t.K, t.lda, kTcBM)) return RETEXO_ERR_CUDA;
+    if (!make_map(&mb, t.B, t.N, t.K, t.ldb, BN / 2)) return RETEXO_ERR_CUDA;
+    TcKernelArgs g{};
+    g.M = t.M; g.N = t.N;
+    g.k_blocks_total = (int32_t)((t.K + kTcBK - 1) / kTcBK);
+    g.k_blocks_per_split = g.k_blocks_total;
+    g.splits = 1;
+    g.mode = t.mode; g.relu = t.relu; g.bias = t.bias;
+    g.out_f32 = t.out_f32; g.ld_f32 = t.ld_f32; g.out_bf16 = t.out_bf16; g.ld_bf16 = t.ld_bf16;
+    g.ones_col = (t.ones_col && t.out_bf16 && t.ld_bf16 > t.N) ? 1 : 0;
+    g.relu_bits = t.relu_bits; g.ld_bits = t.ld_bits;
+    g.drop_thresh = t.drop_thresh; g.drop_step = t.drop_step; g.drop_key0 = t.drop_key[0]; g.drop_key1 = t.drop_key[1];
+    g.drop_scale = t.drop_scale; g.drop_rows = t.drop_rows; g.drop_step_dev = t.drop_step_dev;
+    g.status = t.status; g.n_train = t.M;
+    if (t.out_bf16 && !(g.ones_col && t.N % 8 != 0)) g.tma_rows = make_store_map(&m_rows, t.out_bf16, t.M, t.N, t.ld_bf16) ? 1 : 0;
+    const int64_t n_tiles = ((t.M + 2 * kTcBM - 1) / (2 * kTcBM)) * ((t.N + BN - 1) / BN);
+    cudaLaunchConfig_t cfg{};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(64 + 32 * EW, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    // as many pairs as can be resident at once (persistent blocks), found once per device
+    static int max_pairs[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return RETEXO_ERR_CUDA;
+    if (max_pairs[dev] == 0) {
+        cfg.gridDim = dim3(2 * (unsigned)sm_count(), 1, 1);
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            return RETEXO_ERR_UNSUPPORTED;
+        }
+        max_pairs[dev] = n;
+    }
+    const int64_t pairs = n_tiles < max_pairs[dev] ? n_tiles : max_pairs[dev];
+    cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+    if (cudaLaunchKernelEx(&cfg, kernel, ma, mb, m_rows, g) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return RETEXO_ERR_CUDA;
+    }
+    return launch_status();
+}
+
 template <int BN, int STAGES, int EW>
 static int launch_tc(const TcGemm& t, const CUtensorMap& ma, const CUtensorMap& mb, cudaStream_t st) {
     switch (t.mode) {
@@ -783,6 +881,12 @@ int tc_gemm_launch(const TcGemm& t, cudaStream_t st) {
     // epilogue warps on them (measured: the 256 x 153757 x 41 product itself is level with 256-column
     // tiles, the whole training iteration 1 % shorter)
     if (t.mode == TC_EPI_MASK && bn == 256) bn = 128;
+    // wide forward products over many rows go to pairs of thread blocks: the B tile (the weights) is then
+    // fetched once per 256 rows, which is what bounds these products on the L2 -> SM path
+    if (bn == 256 && t.M >= 4096 && (t.mode == TC_EPI_BIAS || t.mode == TC_EPI_BIAS_DROP)) {
+        const int rc = t.mode == TC_EPI_BIAS ? launch_tc_pair<TC_EPI_BIAS>(t, st) : launch_tc_pair<TC_EPI_BIAS_DROP>(t, st);
+        if (rc != RETEXO_ERR_UNSUPPORTED) return rc;
+    }
     CUtensorMap ma, mb;
     if (t.mode == TC_EPI_PARTIAL) {      // A [K x M], B [K x N] as they lie in memory: boxes of 64 reduction rows x 64 elements
         if (!make_map(&ma, t.A, t.K, t.M, t.lda, kTcBK)) return RETEXO_ERR_CUDA;

@@ -170,3 +170,26 @@ def test_input_gradient_matches_the_checker(d_in, hidden, n_classes, n):
     _, gpu2 = make_pair(d_in, hidden, n_classes, 3, opt=oracle.SGD, lr=0.01)
     gl2, gg2 = B().retexo_mlp_train_step(gpu2, x16, dev(y), x_has_ones=True, return_grad=True)
     assert gl2.item() == gl.item() and torch.equal(gg, gg2) and torch.equal(gpu.theta, gpu2.theta)
+
+
+@pytest.mark.parametrize("d_in,hidden,n_classes,n", [(200, 256, 10, 5000), (72, 192, 5, 4224), (1204, 256, 41, 9000)])
+def test_wide_forward_over_many_rows_runs_in_block_pairs_and_matches_the_checker(d_in, hidden, n_classes, n):
+    """Forward products with more than 128 output columns and at least 4096 rows run on pairs of thread
+    blocks (256-row tiles, odd tails included): hidden representation, logits and one training step."""
+    rng = np.random.default_rng(n)
+    x = rng.standard_normal((n, d_in)).astype(np.float32)
+    y = rng.integers(0, n_classes, n).astype(np.int32)
+    ref, gpu = make_pair(d_in, hidden, n_classes, 5, opt=oracle.SGD, lr=0.01)
+    x16, _ = B().retexo_pack_rows(dev(x), None, ones=True)
+    x_host = x16[:, :d_in].float().cpu().numpy()
+    out = B().retexo_embed(gpu, x16, want_hidden=True, want_hidden_bf16=True, want_logits=True)
+    r = ref.embed(x_host, want_hidden=True)
+    assert_logits_close(out["hidden"].cpu().numpy(), r["hidden"], rel=1e-3, what="hidden")
+    assert torch.equal(out["hidden_bf16"][:, :hidden].cpu(), out["hidden"].to(torch.bfloat16).cpu())
+    assert_logits_close(out["logits"].cpu().numpy(), r["logits"], rel=5e-3, what="logits")
+    rl, rg = ref.train_step(x_host, y, return_grad=True)
+    gl, gg = B().retexo_mlp_train_step(gpu, x16, dev(y), x_has_ones=True, return_grad=True)
+    assert abs(gl.item() - rl) <= 2e-4 * max(1.0, abs(rl))
+    err, scale = np.abs(gg.cpu().numpy().astype(np.float64) - rg), np.abs(rg).max()
+    assert err.max() <= 5e-3 * scale + 1e-7 and np.median(err) <= 2e-5 * scale
+    assert int(gpu.status.item()) == 0
