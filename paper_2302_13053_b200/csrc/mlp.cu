@@ -313,7 +313,8 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         u.step_dev = dev->step; u.done = dev->done; u.loss_base = dev->loss_base; u.history_base = dev->history_base;
         u.loss_out = nullptr;
     }
-    reduce_update_kernel<<<(unsigned)((p.nt + 255) / 256), 256, 0, st>>>(u);
+    const int64_t tiles = (((int64_t)d_in + 16) / 16) * ((out1 + 15) / 16) + (H > 0 ? (((int64_t)H + 16) / 16) * ((O + 15) / 16) : 0);
+    reduce_update_kernel<<<(unsigned)tiles, 256, 0, st>>>(u);
     if (model->status_out)
         RETEXO_CUDA_TRY(cudaMemcpyAsync(model->status_out, b.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
     return launch_status();

@@ -244,114 +244,134 @@ __host__ __device__ __forceinline__ double pow_whole(double base, unsigned long 
     return r;
 }
 
-// One parameter: sum of its split-K partials in index order, optimiser step, bf16 copies.
-__device__ __forceinline__ void update_parameter(const UpdateArgs& u, int64_t p, int sidx, int64_t q, int64_t size,
-                                                 float corr1, float corr2, bool snapshot) {
-    const float* part = sidx == 0 ? u.seg[0].partial : u.seg[1].partial;
-    const int64_t count = sidx == 0 ? u.seg[0].count : u.seg[1].count;
+// Sum of one parameter's split-K partials in index order.  Up to 32 loads are in flight before the
+// first addition waits for one (warps issue in order, so a loop of small batches would pay the
+// memory latency once per batch).
+__device__ __forceinline__ float sum_partials(const float* __restrict__ src, int64_t count, int64_t stride) {
     float g = 0.f;
-    int64_t z = 0;
-    for (; z + 8 <= count; z += 8) {          // loads issued together, added in index order
-        float x[8];
+    for (int64_t z = 0; z < count; z += 32) {
+        float x[32];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) x[i] = __ldcs(part + (z + i) * size + q);      // read once: streamed
+        for (int i = 0; i < 32; ++i) x[i] = z + i < count ? __ldcs(src + (z + i) * stride) : 0.f;   // read once: streamed
 #pragma unroll
-        for (int i = 0; i < 8; ++i) g += x[i];
+        for (int i = 0; i < 32; ++i) g += x[i];
     }
-    for (; z + 4 <= count; z += 4) {
-        const float a = __ldcs(part + z * size + q), b = __ldcs(part + (z + 1) * size + q);
-        const float c = __ldcs(part + (z + 2) * size + q), d = __ldcs(part + (z + 3) * size + q);
-        g += a; g += b; g += c; g += d;
-    }
-    for (; z < count; ++z) g += part[z * size + q];
-    if (u.grad_out) u.grad_out[p] = g;
-    if (snapshot) u.theta_best[p] = u.theta[p];
-    float t;
-    if (u.optimizer == RETEXO_SGD) {
-        t = u.theta[p] - u.lr * g;
-    } else {
-        const float m = u.beta1 * u.m[p] + (1.f - u.beta1) * g;
-        const float v = u.beta2 * u.v[p] + (1.f - u.beta2) * g * g;
-        u.m[p] = m;
-        u.v[p] = v;
-        t = u.theta[p] - u.lr * (m / corr1) / (sqrtf(v / corr2) + u.eps);
-    }
-    u.theta[p] = t;
-    if (sidx == 0) {
-        if (u.w1t16 && q < (int64_t)u.d_in * u.out1) {
-            const int64_t k = q / u.out1, j = q % u.out1;
-            u.w1t16[j * u.ld_k + k] = f32_to_bf16(t);
-            if (u.w1r16) u.w1r16[k * u.ld_o1 + j] = f32_to_bf16(t);
-        }
-    } else if (q < (int64_t)u.hidden * u.n_classes) {
-        const int64_t jh = q / u.n_classes, c = q % u.n_classes;
-        if (u.w2t16) u.w2t16[c * u.ld_h + jh] = f32_to_bf16(t);
-        if (u.w2p16) u.w2p16[jh * u.ld_dl + c] = f32_to_bf16(t);
-    }
+    return g;
 }
 
 // Sums each parameter's split-K partials in index order, applies the optimiser, and refreshes
 // the bf16 weight copies.  Block 0 also reduces the loss (fixed order: per-lane strided sums,
 // then a shuffle tree).  With u.done set, the last block to arrive does the validation bookkeeping.
+// The kernel sits between two products on the critical path of an iteration and moves little
+// data, so it is laid out for latency: every load that depends on nothing (the iteration state,
+// the partials, the parameter and its moments) is issued before anything waits.
 __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
-    const int64_t p = blockIdx.x * 256ll + threadIdx.x;
+    // A block owns a 16 x 16 tile of one segment's (inputs + 1) x outputs matrix (the last row is the
+    // bias): 64-byte runs of each partial on the way in, and whole 32-byte sectors of the transposed
+    // bf16 copy on the way out (a 2-byte store per parameter into a row of its own has every store
+    // read-modify-write a sector that fifteen other blocks are writing too).
+    const int32_t rows0 = u.d_in + 1, cols0 = u.out1;
+    const int32_t tc0 = (cols0 + 15) >> 4, tiles0 = ((rows0 + 15) >> 4) * tc0;
+    const int sidx = (int32_t)blockIdx.x < tiles0 ? 0 : 1;
+    const int32_t rows = sidx == 0 ? rows0 : u.hidden + 1, cols = sidx == 0 ? cols0 : u.n_classes;
+    const int32_t tcs = (cols + 15) >> 4, tile = sidx == 0 ? (int32_t)blockIdx.x : (int32_t)blockIdx.x - tiles0;
+    const int32_t row0 = (tile / tcs) << 4, col0 = (tile % tcs) << 4;
+    const int32_t row = row0 + ((int32_t)threadIdx.x >> 4), col = col0 + ((int32_t)threadIdx.x & 15);
+    const int64_t size = (int64_t)rows * cols;
+    const int64_t q = (int64_t)row * cols + col;
+    const int64_t p = sidx == 0 ? q : q + u.seg[0].size;
+    const bool live = row < rows && col < cols;
+    const bool adam = u.optimizer != RETEXO_SGD;
+
+    // ---- loads with no dependence
+    unsigned long long step_now = 0, snap_cur = 0, snap_best = 0;
+    int32_t snap_have = 1;
+    if (u.step_dev) step_now = *u.step_dev;
+    if (u.snap_cur) { snap_have = *u.snap_have; snap_cur = *u.snap_cur; snap_best = *u.snap_best; }
+    float theta = 0.f, m = 0.f, v = 0.f, g = 0.f;
+    if (live) {
+        theta = u.theta[p];
+        if (adam) { m = u.m[p]; v = u.v[p]; }
+        g = sum_partials((sidx == 0 ? u.seg[0].partial : u.seg[1].partial) + q,
+                         sidx == 0 ? u.seg[0].count : u.seg[1].count, size);
+    }
+
     float corr1 = u.corr1, corr2 = u.corr2;
     float* loss_out = u.loss_out;
-    unsigned long long step_now = 0;
     if (u.step_dev) {      // the iteration number lives on the device: bias corrections and slots follow from it
         __shared__ float corr_s[2];
-        step_now = *u.step_dev;
-        if (threadIdx.x == 0) {
-            corr_s[0] = (float)(1.0 - pow_whole((double)u.beta1, step_now + 1));
-            corr_s[1] = (float)(1.0 - pow_whole((double)u.beta2, step_now + 1));
-        }
+        if (threadIdx.x == 0) corr_s[0] = (float)(1.0 - pow_whole((double)u.beta1, step_now + 1));
+        if (threadIdx.x == 32) corr_s[1] = (float)(1.0 - pow_whole((double)u.beta2, step_now + 1));
         __syncthreads();
         corr1 = corr_s[0]; corr2 = corr_s[1];
         loss_out = u.loss_base ? u.loss_base + step_now : nullptr;
     }
-    if (blockIdx.x == 0 && threadIdx.x < 32 && loss_out) {
-        float s = 0.f;
-        for (int64_t i = threadIdx.x; i < u.n_loss; i += 32) s += u.loss_partial[i];
-        s = warp_sum(s);
-        if (threadIdx.x == 0) *loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
-    }
     // keep-the-best: are the weights as they stand (validated in this iteration's forward pass) the best so far?
-    const bool snapshot = u.theta_best && (!*u.snap_have || *u.snap_cur > *u.snap_best);
+    const bool snapshot = u.theta_best && (!snap_have || snap_cur > snap_best);
     if (u.done) {
         // Once every block has read the validation state and the iteration number (signalled here, before
         // the block's own stores, so the fence has nothing to wait for), the last block to arrive books
         // the count and moves the state on, while the others are already updating their parameters.
-        __shared__ bool is_last;
         __syncthreads();
         if (threadIdx.x == 0) {
             __threadfence();
-            is_last = atomicAdd(u.done, 1ull) == (unsigned long long)gridDim.x - 1ull;
-        }
-        __syncthreads();
-        if (is_last && threadIdx.x == 0) {
-            __threadfence();
-            if (u.snap_decision) *u.snap_decision = snapshot ? 1 : 0;
-            if (u.snap_cur) {
-                const unsigned long long cur = *u.snap_cur;
-                unsigned long long* slot = u.step_dev ? (u.history_base && step_now > 0 ? u.history_base + (step_now - 1) : nullptr)
-                                                      : u.rec_history_slot;
-                if (slot) *slot = cur;
-                if (!*u.snap_have || cur > *u.snap_best) {
-                    *u.snap_best = cur;
-                    if (u.rec_best_iter) *u.rec_best_iter = u.step_dev ? (int32_t)step_now : u.rec_iter;
-                    *u.snap_have = 1;
+            if (atomicAdd(u.done, 1ull) == (unsigned long long)gridDim.x - 1ull) {
+                __threadfence();
+                if (u.snap_decision) *u.snap_decision = snapshot ? 1 : 0;
+                if (u.snap_cur) {
+                    unsigned long long* slot = u.step_dev ? (u.history_base && step_now > 0 ? u.history_base + (step_now - 1) : nullptr)
+                                                          : u.rec_history_slot;
+                    if (slot) *slot = snap_cur;
+                    if (!snap_have || snap_cur > snap_best) {
+                        *u.snap_best = snap_cur;
+                        if (u.rec_best_iter) *u.rec_best_iter = u.step_dev ? (int32_t)step_now : u.rec_iter;
+                        *u.snap_have = 1;
+                    }
+                    *u.snap_cur = 0ull;
                 }
-                *u.snap_cur = 0ull;
+                if (u.step_dev) *u.step_dev = step_now + 1;
+                *u.done = 0ull;
             }
-            if (u.step_dev) *u.step_dev = step_now + 1;
-            *u.done = 0ull;
         }
     }
-    const int64_t size0 = u.seg[0].size;
-    const int sidx = p < size0 ? 0 : 1;
-    const int64_t q = sidx == 0 ? p : p - size0;
-    const int64_t size = sidx == 0 ? size0 : u.seg[1].size;
-    if (sidx < u.n_seg && q < size) update_parameter(u, p, sidx, q, size, corr1, corr2, snapshot);
+    if (blockIdx.x == 0 && threadIdx.x >= 224 && loss_out) {      // the block's last warp: not the one that signals
+        const int lane = threadIdx.x - 224;
+        float s = 0.f;
+        for (int64_t i = lane; i < u.n_loss; i += 32) s += u.loss_partial[i];
+        s = warp_sum(s);
+        if (lane == 0) *loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
+    }
+
+    bf16 t16 = f32_to_bf16(0.f);
+    if (live) {
+        if (u.grad_out) u.grad_out[p] = g;
+        if (snapshot) u.theta_best[p] = theta;
+        float t;
+        if (!adam) {
+            t = theta - u.lr * g;
+        } else {
+            m = u.beta1 * m + (1.f - u.beta1) * g;
+            v = u.beta2 * v + (1.f - u.beta2) * g * g;
+            u.m[p] = m;
+            u.v[p] = v;
+            t = theta - u.lr * (m / corr1) / (sqrtf(v / corr2) + u.eps);
+        }
+        u.theta[p] = t;
+        t16 = f32_to_bf16(t);
+        if (row < rows - 1) {                   // the weights (not the bias row), as the products read them
+            if (sidx == 0) { if (u.w1r16) u.w1r16[(int64_t)row * u.ld_o1 + col] = t16; }
+            else if (u.w2p16) u.w2p16[(int64_t)row * u.ld_dl + col] = t16;
+        }
+    }
+    bf16* wt = sidx == 0 ? u.w1t16 : u.w2t16;
+    if (wt) {                                   // uniform over the block
+        __shared__ bf16 tile16[16][18];
+        tile16[threadIdx.x >> 4][threadIdx.x & 15] = t16;
+        __syncthreads();
+        const int32_t trow = row0 + ((int32_t)threadIdx.x & 15), tcol = col0 + ((int32_t)threadIdx.x >> 4);
+        if (trow < rows - 1 && tcol < cols)
+            wt[(int64_t)tcol * (sidx == 0 ? u.ld_k : u.ld_h) + trow] = tile16[threadIdx.x & 15][threadIdx.x >> 4];
+    }
 }
 
 __global__ void __launch_bounds__(256) f32_to_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int64_t n) {
