@@ -146,7 +146,9 @@ struct WorkStream {
     WorkStream& operator=(const WorkStream&) = delete;
 };
 
-// Owns the executable graph of one round's training iteration.
+constexpr int kGraphIterations = 8;      // iterations replayed by one launch of the chunk graph
+
+// Owns an executable graph of one round's training iterations.
 struct IterationGraph {
     cudaGraphExec_t exec = nullptr;
     void reset() { if (exec) { (void)cudaGraphExecDestroy(exec); exec = nullptr; } }
@@ -334,7 +336,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
     if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
     WorkStream work(static_cast<cudaStream_t>(stream));
     cudaStream_t st = work.s;
-    IterationGraph iteration;
+    IterationGraph iteration, chunk;
     const bool host = c.memory_is_host != 0;
     const cudaMemcpyKind in_kind = host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
     const cudaMemcpyKind out_kind = host ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice;
@@ -516,8 +518,11 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
             return launch_status();
         };
         iteration.reset();
+        chunk.reset();
+        bool graphs_ok = true;
         int pending_it = 0;       // iteration whose weights still await their validation count
         for (int it = 1; it <= c.R; ++it) {
+            int done_now = 1;     // iterations this pass of the loop enqueues
             float* loss_slot = b.loss_history + (size_t)(m - 1) * c.R + (it - 1);
             // The weights of iteration it-1 are validated inside this iteration's forward pass (the
             // validation rows ride along; the update kernel keeps them if they are the best so far).
@@ -533,25 +538,37 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
                 RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot, nullptr, it > 1,
                                                  riding, st, &dev, b.dx, ld_dx));
                 RETEXO_TRY(gat_backward_and_update());
-            } else if (iteration.exec) {
-                RETEXO_CUDA_TRY(cudaGraphLaunch(iteration.exec, st));
-            } else if (uniform && it == 2) {
-                bool recorded = false;
-                if (cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed) == cudaSuccess) {
-                    const int rc = mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot,
-                                                         nullptr, true, riding, st, &dev);
-                    cudaGraph_t graph = nullptr;
-                    const cudaError_t ended = cudaStreamEndCapture(st, &graph);
-                    if (rc == RETEXO_OK && ended == cudaSuccess && graph &&
-                        cudaGraphInstantiate(&iteration.exec, graph, 0) == cudaSuccess)
-                        recorded = true;
-                    if (graph) (void)cudaGraphDestroy(graph);
-                }
-                (void)cudaGetLastError();
-                if (recorded) {
+            } else if (uniform && it >= 2) {
+                // Iterations 2..R are the same launches (their iteration-dependent state lives on the device), so
+                // they are replayed from graphs: a chunk of kGraphIterations while that many remain (inside a
+                // graph consecutive kernels overlap their set-up with the predecessor's tail, across graph
+                // launches they do not), a single iteration for the rest.
+                auto record = [&](IterationGraph& gr, int count) -> bool {
+                    bool recorded = false;
+                    if (cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed) == cudaSuccess) {
+                        int rc = RETEXO_OK;
+                        for (int i = 0; i < count && rc == RETEXO_OK; ++i)
+                            rc = mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot, nullptr,
+                                                       true, riding, st, &dev);
+                        cudaGraph_t graph = nullptr;
+                        const cudaError_t ended = cudaStreamEndCapture(st, &graph);
+                        if (rc == RETEXO_OK && ended == cudaSuccess && graph &&
+                            cudaGraphInstantiate(&gr.exec, graph, 0) == cudaSuccess)
+                            recorded = true;
+                        if (graph) (void)cudaGraphDestroy(graph);
+                    }
+                    (void)cudaGetLastError();
+                    if (!recorded) gr.reset();
+                    return recorded;
+                };
+                const int remaining = c.R - it + 1;
+                if (graphs_ok && remaining >= kGraphIterations && (chunk.exec || record(chunk, kGraphIterations))) {
+                    RETEXO_CUDA_TRY(cudaGraphLaunch(chunk.exec, st));
+                    done_now = kGraphIterations;
+                } else if (graphs_ok && (iteration.exec || record(iteration, 1))) {
                     RETEXO_CUDA_TRY(cudaGraphLaunch(iteration.exec, st));
                 } else {      // no graph on this stream: plain launches
-                    iteration.reset();
+                    graphs_ok = false;
                     RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot,
                                                      nullptr, true, riding, st, &dev));
                 }
@@ -559,6 +576,8 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
                 RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot,
                                                  nullptr, it > 1, riding, st, &dev));
             }
+            it += done_now - 1;
+            model.step += done_now - 1;
             model.step += 1;
             const bool want = n_val && (it % c.eval_every == 0 || it == c.R);
             pending_it = (want && it < c.R) ? it : 0;

@@ -239,6 +239,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
         }
     }
+    grid_dependency_wait();          // everything from here on may read what the previous kernel wrote
+    grid_dependency_release();
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if constexpr (PAIR) cluster_sync_all();      // both blocks' barriers exist before either signals the other's
@@ -779,7 +781,11 @@ static int launch_tc_mode(const TcGemm& t, const CUtensorMap& ma, const CUtensor
     const int n_sm = sm_count();
     if (n_sm <= 0) return RETEXO_ERR_CUDA;
     const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);      // one persistent block per SM
-    tc_gemm_kernel<BN, STAGES, MODE, EW><<<grid, 64 + 32 * EW, smem, st>>>(ma, mb, m_rows, g);
+    OverlapLaunch ol(dim3(grid), dim3(64 + 32 * EW), smem, st);
+    if (cudaLaunchKernelEx(&ol.cfg, tc_gemm_kernel<BN, STAGES, MODE, EW>, ma, mb, m_rows, g) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return RETEXO_ERR_CUDA;
+    }
     return launch_status();
 }
 
@@ -813,15 +819,8 @@ static int launch_tc_pair(const TcGemm& t, cudaStream_t st) {
     g.status = t.status; g.n_train = t.M;
     if (t.out_bf16 && !(g.ones_col && t.N % 8 != 0)) g.tma_rows = make_store_map(&m_rows, t.out_bf16, t.M, t.N, t.ld_bf16) ? 1 : 0;
     const int64_t n_tiles = ((t.M + 2 * kTcBM - 1) / (2 * kTcBM)) * ((t.N + BN - 1) / BN);
-    cudaLaunchConfig_t cfg{};
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.blockDim = dim3(64 + 32 * EW, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    OverlapLaunch ol(dim3(2), dim3(64 + 32 * EW), smem, st, 2);
+    cudaLaunchConfig_t& cfg = ol.cfg;
     // as many pairs as can be resident at once (persistent blocks), found once per device
     static int max_pairs[64] = {};
     int dev = 0;

@@ -314,9 +314,12 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         u.loss_out = nullptr;
     }
     const int64_t tiles = (((int64_t)d_in + 16) / 16) * ((out1 + 15) / 16) + (H > 0 ? (((int64_t)H + 16) / 16) * ((O + 15) / 16) : 0);
-    reduce_update_kernel<<<(unsigned)tiles, 256, 0, st>>>(u);
-    if (model->status_out)
-        RETEXO_CUDA_TRY(cudaMemcpyAsync(model->status_out, b.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
+    u.status_out = model->status_out;
+    OverlapLaunch ol(dim3((unsigned)tiles), dim3(256), 0, st);
+    if (cudaLaunchKernelEx(&ol.cfg, reduce_update_kernel, u) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return RETEXO_ERR_CUDA;
+    }
     return launch_status();
 }
 

@@ -85,13 +85,15 @@ head_backward_kernel(const __grid_constant__ CUtensorMap map_hd, const __grid_co
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (threadIdx.x >= 64 && threadIdx.x < 128) {
-        const int c = threadIdx.x - 64;
-        bias_s[c] = (g.b2 && c < g.O) ? g.b2[c] : 0.f;
-    }
     if (warp == 1) {      // all of tensor memory: two logit accumulators of 64 columns, one gradient accumulator of 256
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;");
+    }
+    grid_dependency_wait();          // everything from here on may read what the previous kernel wrote
+    grid_dependency_release();
+    if (threadIdx.x >= 64 && threadIdx.x < 128) {
+        const int c = threadIdx.x - 64;
+        bias_s[c] = (g.b2 && c < g.O) ? g.b2[c] : 0.f;
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -421,7 +423,11 @@ int head_backward_launch(const HeadBackward& h, cudaStream_t st) {
     const int n_sm = sm_count();
     if (n_sm <= 0) return RETEXO_ERR_CUDA;
     const unsigned grid = (unsigned)(n_tiles < n_sm ? n_tiles : n_sm);
-    head_backward_kernel<<<grid, kHbThreads, smem, st>>>(m_hd, m_w2, m_dl, m_dhd, g);
+    OverlapLaunch ol(dim3(grid), dim3(kHbThreads), smem, st);
+    if (cudaLaunchKernelEx(&ol.cfg, head_backward_kernel, m_hd, m_w2, m_dl, m_dhd, g) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return RETEXO_ERR_CUDA;
+    }
     return launch_status();
 }
 

@@ -5,6 +5,7 @@
 // gradient-reduce + optimiser update.
 #pragma once
 #include "common.cuh"
+#include "launch_overlap.cuh"
 
 namespace retexo {
 
@@ -214,6 +215,7 @@ struct UpdateArgs {
     float lr, beta1, beta2, eps, corr1, corr2;     // corr = 1 - beta^step
     const float* loss_partial; int64_t n_loss; float inv_rows; float* loss_out;
     const int32_t* status;     // non-zero: a kernel of this step gave up on a bounded wait -> loss = NaN
+    int32_t* status_out;       // (optional) receives *status
     // bf16 copies of the updated weights in the orientations the next products read (optional)
     bf16* w1t16; int64_t ld_k;       // W1^T [out1 x ld_k]
     bf16* w1r16; int64_t ld_o1;      // W1   [d_in x ld_o1]
@@ -283,6 +285,8 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     const bool live = row < rows && col < cols;
     const bool adam = u.optimizer != RETEXO_SGD;
 
+    grid_dependency_wait();
+    grid_dependency_release();
     // ---- loads with no dependence
     unsigned long long step_now = 0, snap_cur = 0, snap_best = 0;
     int32_t snap_have = 1;
@@ -341,6 +345,7 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
         s = warp_sum(s);
         if (lane == 0) *loss_out = (u.status && *u.status) ? __int_as_float(0x7fc00000) : s * u.inv_rows;
     }
+    if (blockIdx.x == 0 && threadIdx.x == 64 && u.status_out && u.status) *u.status_out = *u.status;
 
     bf16 t16 = f32_to_bf16(0.f);
     if (live) {

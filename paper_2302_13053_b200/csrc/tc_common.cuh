@@ -4,6 +4,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "launch_overlap.cuh"
 
 namespace retexo {
 
