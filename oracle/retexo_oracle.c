@@ -340,6 +340,19 @@ int64_t oracle_theta_size(int32_t d_in, int32_t hidden, int32_t n_classes)
     return (int64_t)d_in * n_classes + n_classes;
 }
 
+/* Layer normalisation inside f_theta (Section 2.2 lists normalisation layers among its parts; the
+ * configurations use none).  Reading taken here: it sits between the fully-connected layer and the ReLU,
+ *   z = x W1 + b1,  zhat = (z - mean(z)) / sqrt(var(z) + ln_eps)  (mean and biased variance over the
+ *   hidden units of the row),  Hd = ReLU(gamma .* zhat + beta),
+ * with trainable gamma and beta appended to theta: [ W1 | b1 | W2 | b2 | gamma (hidden) | beta (hidden) ].
+ * In rounded mode the normalisation is computed wide, forward and backward; the gated gradient that enters
+ * its backward pass is rounded to bf16 first (it is handed on in the format the products read), and the
+ * gradient that leaves it is an operand of the weight-gradient products and rounded there like any other. */
+int64_t oracle_theta_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes, int32_t layer_norm)
+{
+    return oracle_theta_size(d_in, hidden, n_classes) + ((layer_norm && hidden > 0) ? 2 * (int64_t)hidden : 0);
+}
+
 /* ------------------------------------------------------------------ */
 /* Dropout (Appendix B lists dropout rates among the hyper-parameters; */
 /* the configurations use none).  The random bits come from the        */
@@ -390,9 +403,28 @@ int oracle_dropout_mask(int64_t row, int64_t step, int32_t hidden, double p, uin
 /* forward for one input row; a1 = pre-activation (hidden wide, may be NULL
  * when hidden == 0), logits = n_classes wide.  keep (optional, training with
  * dropout only): factor applied to each hidden unit after the ReLU. */
+static void forward_row_ln(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
+                           int round_bf16, const float *xrow, const double *w1r, const double *w2r,
+                           double *a1, double *logits, const double *keep,
+                           const double *ln_gamma, const double *ln_beta, double ln_eps,
+                           double *zhat_out, double *rstd_out);
+
 static void forward_row(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
                         int round_bf16, const float *xrow, const double *w1r, const double *w2r,
                         double *a1, double *logits, const double *keep)
+{
+    forward_row_ln(d_in, hidden, n_classes, theta, round_bf16, xrow, w1r, w2r, a1, logits, keep,
+                   NULL, NULL, 0.0, NULL, NULL);
+}
+
+/* ln_gamma != NULL: layer normalisation between the first linear layer and the ReLU; a1 then holds the
+ * normalised, scaled and shifted pre-activation, zhat_out (hidden wide) the normalised values and *rstd_out
+ * 1 / sqrt(var + eps) of the row. */
+static void forward_row_ln(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
+                           int round_bf16, const float *xrow, const double *w1r, const double *w2r,
+                           double *a1, double *logits, const double *keep,
+                           const double *ln_gamma, const double *ln_beta, double ln_eps,
+                           double *zhat_out, double *rstd_out)
 {
     if (hidden > 0) {
         const double *b1 = theta + (int64_t)d_in * hidden;
@@ -405,6 +437,20 @@ static void forward_row(int32_t d_in, int32_t hidden, int32_t n_classes, const d
             for (int32_t j = 0; j < hidden; ++j) a1[j] += xv * wrow[j];
         }
         for (int32_t j = 0; j < hidden; ++j) a1[j] += b1[j];
+        if (ln_gamma) {
+            double mean = 0.0, var = 0.0;
+            for (int32_t j = 0; j < hidden; ++j) mean += a1[j];
+            mean /= (double)hidden;
+            for (int32_t j = 0; j < hidden; ++j) var += (a1[j] - mean) * (a1[j] - mean);
+            var /= (double)hidden;
+            double rstd = 1.0 / sqrt(var + ln_eps);
+            for (int32_t j = 0; j < hidden; ++j) {
+                double zh = (a1[j] - mean) * rstd;
+                if (zhat_out) zhat_out[j] = zh;
+                a1[j] = ln_gamma[j] * zh + ln_beta[j];
+            }
+            if (rstd_out) *rstd_out = rstd;
+        }
         for (int32_t c = 0; c < n_classes; ++c) logits[c] = 0.0;
         for (int32_t j = 0; j < hidden; ++j) {
             double h = a1[j] > 0.0 ? a1[j] : 0.0;
@@ -484,16 +530,25 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
                            int64_t step, int32_t round_bf16,
                            const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
                            const int32_t *y, double *loss_out, double *grad_out,
-                           double drop_p, uint64_t drop_seed, double *dx_out)
+                           double drop_p, uint64_t drop_seed, double *dx_out,
+                           int32_t layer_norm, double ln_eps)
 {
     if (d_in <= 0 || n_classes <= 0 || hidden < 0 || n_rows <= 0 || ldx < d_in) return ORACLE_BAD_ARG;
     if (drop_p < 0.0 || drop_p >= 1.0) return ORACLE_BAD_ARG;
+    if (layer_norm && (hidden <= 0 || ln_eps <= 0.0)) return ORACLE_BAD_ARG;
     const int dropping = drop_p > 0.0 && hidden > 0;
     if (optimizer == 1 && (!adam_m || !adam_v || step < 1)) return ORACLE_BAD_ARG;
-    int64_t nt = oracle_theta_size(d_in, hidden, n_classes);
+    int64_t nt = oracle_theta_size_ln(d_in, hidden, n_classes, layer_norm);
     int32_t out1 = hidden > 0 ? hidden : n_classes;
+    /* layer normalisation: gamma and beta sit behind [W1 | b1 | W2 | b2] */
+    const double *ln_gamma = layer_norm ? theta + oracle_theta_size(d_in, hidden, n_classes) : NULL;
+    const double *ln_beta = layer_norm ? ln_gamma + hidden : NULL;
+    /* per row: the normalised values and the (bf16-rounded, in rounded mode) gated gradient, for d gamma / d beta */
+    double *zh_all = layer_norm ? (double *)malloc(sizeof(double) * (size_t)n_rows * hidden) : NULL;
+    double *dy_all = layer_norm ? (double *)malloc(sizeof(double) * (size_t)n_rows * hidden) : NULL;
+    if (layer_norm && (!zh_all || !dy_all)) { free(zh_all); free(dy_all); return ORACLE_NO_MEM; }
     double *w1r, *w2r;
-    if (rounded_weights(d_in, hidden, n_classes, theta, round_bf16, &w1r, &w2r)) return ORACLE_NO_MEM;
+    if (rounded_weights(d_in, hidden, n_classes, theta, round_bf16, &w1r, &w2r)) { free(zh_all); free(dy_all); return ORACLE_NO_MEM; }
 
     /* per-row results of the forward/backward through the row-local part */
     double *d1 = (double *)malloc(sizeof(double) * (size_t)n_rows * out1);       /* grad wrt first linear output */
@@ -503,7 +558,7 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
     double *grad = (double *)calloc((size_t)nt, sizeof(double));
     int bad_label = 0;
     if (!d1 || (hidden > 0 && (!hd || !dl)) || !row_loss || !grad) {
-        free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad);
+        free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad); free(zh_all); free(dy_all);
         return ORACLE_NO_MEM;
     }
 
@@ -516,7 +571,9 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
         for (int64_t i = 0; i < n_rows; ++i) {
             int64_t r = row_idx ? row_idx[i] : i;
             if (keep) dropout_row(i, step, hidden, drop_p, drop_seed, keep);
-            forward_row(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg, keep);
+            double rstd = 0.0;
+            forward_row_ln(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg, keep,
+                           ln_gamma, ln_beta, ln_eps, layer_norm ? zh_all + i * hidden : NULL, &rstd);
             int32_t yi = y[i];
             if (yi < 0 || yi >= n_classes) { bad_label = 1; yi = 0; }
             double mx = lg[0];
@@ -539,6 +596,23 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
                         if (keep) acc *= keep[j];
                     }
                     d1[i * hidden + j] = acc;
+                }
+                if (layer_norm) {
+                    /* backward through the normalisation: with dy the gated gradient at its output,
+                     *   dzhat = dy .* gamma,  dz = rstd (dzhat - mean(dzhat) - zhat mean(dzhat .* zhat)) */
+                    const double *zh = zh_all + i * hidden;
+                    double *dy = dy_all + i * hidden;
+                    double m1 = 0.0, m2 = 0.0;
+                    for (int32_t j = 0; j < hidden; ++j) {
+                        dy[j] = opnd(d1[i * hidden + j], round_bf16);
+                        double dzh = dy[j] * ln_gamma[j];
+                        m1 += dzh;
+                        m2 += dzh * zh[j];
+                    }
+                    m1 /= (double)hidden;
+                    m2 /= (double)hidden;
+                    for (int32_t j = 0; j < hidden; ++j)
+                        d1[i * hidden + j] = rstd * (dy[j] * ln_gamma[j] - m1 - zh[j] * m2);
                 }
             }
         }
@@ -568,7 +642,7 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
      * that are then added in chunk order */
     double *part = (double *)calloc((size_t)GRAD_CHUNKS * (size_t)nt, sizeof(double));
     if (!part) {
-        free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad);
+        free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad); free(zh_all); free(dy_all);
         return ORACLE_NO_MEM;
     }
 #pragma omp parallel for schedule(dynamic, 1)
@@ -600,6 +674,14 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
                 }
                 for (int32_t c = 0; c < n_classes; ++c) gb2[c] += opnd(dlrow[c], round_bf16);
             }
+            if (layer_norm) {
+                /* d gamma = sum_rows dy .* zhat,  d beta = sum_rows dy */
+                double *gg = gb2 + n_classes, *gbt = gg + hidden;
+                for (int32_t j = 0; j < hidden; ++j) {
+                    gg[j] += dy_all[i * hidden + j] * zh_all[i * hidden + j];
+                    gbt[j] += dy_all[i * hidden + j];
+                }
+            }
         }
     }
     for (int ch = 0; ch < GRAD_CHUNKS; ++ch)
@@ -609,7 +691,7 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
     oracle_apply_update(nt, theta, adam_m, adam_v, grad, optimizer, lr, beta1, beta2, eps, step);
     if (loss_out) *loss_out = loss;
     if (grad_out) memcpy(grad_out, grad, sizeof(double) * (size_t)nt);
-    free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad);
+    free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad); free(zh_all); free(dy_all);
     return bad_label ? ORACLE_BAD_ARG : ORACLE_OK;
 }
 
@@ -621,7 +703,7 @@ int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
                           const int32_t *y, double *loss_out, double *grad_out)
 {
     return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
-                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, NULL);
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, NULL, 0, 0.0);
 }
 
 /* The same step, also returning dX [n_rows x d_in], the gradient of the loss with respect to the batch
@@ -634,7 +716,7 @@ int oracle_mlp_train_step_dx(int32_t d_in, int32_t hidden, int32_t n_classes,
                              const int32_t *y, double *loss_out, double *grad_out, double *dx_out)
 {
     return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
-                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, dx_out);
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, dx_out, 0, 0.0);
 }
 
 /* The same step with dropout on the hidden units: Hd = ReLU(X W1 + b1) .* keep,
@@ -649,7 +731,20 @@ int oracle_mlp_train_step_dropout(int32_t d_in, int32_t hidden, int32_t n_classe
                                   double drop_p, uint64_t drop_seed)
 {
     return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
-                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, drop_p, drop_seed, NULL);
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, drop_p, drop_seed, NULL, 0, 0.0);
+}
+
+/* The same step with layer normalisation inside f_theta (see oracle_theta_size_ln for the reading and the
+ * layout of theta, adam_m, adam_v and grad_out); dx_out optional. */
+int oracle_mlp_train_step_ln(int32_t d_in, int32_t hidden, int32_t n_classes,
+                             double *theta, double *adam_m, double *adam_v,
+                             int32_t optimizer, double lr, double beta1, double beta2, double eps,
+                             int64_t step, int32_t round_bf16,
+                             const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                             const int32_t *y, double *loss_out, double *grad_out, double *dx_out, double ln_eps)
+{
+    return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, dx_out, 1, ln_eps);
 }
 
 /* Forward of the trained per-node model over a set of rows.
@@ -659,15 +754,19 @@ int oracle_mlp_train_step_dropout(int32_t d_in, int32_t hidden, int32_t n_classe
  *   hidden == 0: logits = x W1 + b1 (hidden_out must be NULL).
  * pred = argmax of the fp32-rounded logits, lowest index on ties;
  * correct = number of rows with pred == y[i] (y optional). */
-int oracle_embed(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
-                 int32_t round_bf16,
-                 const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
-                 float *hidden_out, int64_t ld_hidden,
-                 float *logits_out, int64_t ld_logits,
-                 int32_t *pred_out, const int32_t *y, uint64_t *correct_out)
+static int embed_impl(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
+                      int32_t round_bf16,
+                      const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                      float *hidden_out, int64_t ld_hidden,
+                      float *logits_out, int64_t ld_logits,
+                      int32_t *pred_out, const int32_t *y, uint64_t *correct_out,
+                      int32_t layer_norm, double ln_eps)
 {
     if (d_in <= 0 || n_classes <= 0 || hidden < 0 || n_rows < 0 || ldx < d_in) return ORACLE_BAD_ARG;
     if (hidden == 0 && hidden_out) return ORACLE_BAD_ARG;
+    if (layer_norm && (hidden <= 0 || ln_eps <= 0.0)) return ORACLE_BAD_ARG;
+    const double *ln_gamma = layer_norm ? theta + oracle_theta_size(d_in, hidden, n_classes) : NULL;
+    const double *ln_beta = layer_norm ? ln_gamma + hidden : NULL;
     double *w1r, *w2r;
     if (rounded_weights(d_in, hidden, n_classes, theta, round_bf16, &w1r, &w2r)) return ORACLE_NO_MEM;
     uint64_t correct = 0;
@@ -678,7 +777,8 @@ int oracle_embed(int32_t d_in, int32_t hidden, int32_t n_classes, const double *
 #pragma omp for schedule(static)
         for (int64_t i = 0; i < n_rows; ++i) {
             int64_t r = row_idx ? row_idx[i] : i;
-            forward_row(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg, NULL);
+            forward_row_ln(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg, NULL,
+                           ln_gamma, ln_beta, ln_eps, NULL, NULL);
             if (hidden_out)
                 for (int32_t j = 0; j < hidden; ++j)
                     hidden_out[i * ld_hidden + j] = (float)(a1[j] > 0.0 ? a1[j] : 0.0);
@@ -697,6 +797,30 @@ int oracle_embed(int32_t d_in, int32_t hidden, int32_t n_classes, const double *
     free(w1r);
     free(w2r);
     return ORACLE_OK;
+}
+
+int oracle_embed(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
+                 int32_t round_bf16,
+                 const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                 float *hidden_out, int64_t ld_hidden,
+                 float *logits_out, int64_t ld_logits,
+                 int32_t *pred_out, const int32_t *y, uint64_t *correct_out)
+{
+    return embed_impl(d_in, hidden, n_classes, theta, round_bf16, x, ldx, row_idx, n_rows, hidden_out, ld_hidden,
+                      logits_out, ld_logits, pred_out, y, correct_out, 0, 0.0);
+}
+
+/* The same with layer normalisation inside f_theta: hidden_out = ReLU(gamma .* zhat + beta), theta laid out as
+ * oracle_theta_size_ln says. */
+int oracle_embed_ln(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
+                    int32_t round_bf16,
+                    const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                    float *hidden_out, int64_t ld_hidden,
+                    float *logits_out, int64_t ld_logits,
+                    int32_t *pred_out, const int32_t *y, uint64_t *correct_out, double ln_eps)
+{
+    return embed_impl(d_in, hidden, n_classes, theta, round_bf16, x, ldx, row_idx, n_rows, hidden_out, ld_hidden,
+                      logits_out, ld_logits, pred_out, y, correct_out, 1, ln_eps);
 }
 
 /* ================================================================== */
