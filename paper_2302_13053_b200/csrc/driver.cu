@@ -202,11 +202,11 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
         const RoundDims r = round_dims(c, m);
         if (r.d_in > max_din) max_din = r.d_in;
         if (r.rep_dim > max_rep) max_rep = r.rep_dim;
-        const int64_t nt = retexo_theta_size(r.d_in, r.hidden, c.n_classes);
+        const int64_t nt = retexo_theta_size_ln(r.d_in, r.hidden, c.n_classes, c.layer_norm);
         if (nt > max_nt) max_nt = nt;
-        size_t s = mlp_step_workspace_size(make_plan(r.d_in, r.hidden, c.n_classes, n_tr, n_val));
+        size_t s = mlp_step_workspace_size(make_plan(r.d_in, r.hidden, c.n_classes, n_tr, n_val, c.layer_norm != 0));
         if (s > step_b) step_b = s;
-        s = retexo_embed_workspace_size(r.d_in, r.hidden, c.n_classes, n);
+        s = retexo_embed_workspace_size_ln(r.d_in, r.hidden, c.n_classes, n, c.layer_norm);
         if (s > embed_b) embed_b = s;
         s = retexo_aggregate_workspace_size(n, e, c.aggr, r.agg_dim, c.gat_heads);
         if (s > agg_b) agg_b = s;
@@ -300,6 +300,8 @@ static int check_cfg(const retexo_lmp_config* c) {
     if (c->eval_every < 1) return RETEXO_ERR_INVALID_ARG;
     if (!(c->dropout >= 0.f && c->dropout < 1.f)) return RETEXO_ERR_INVALID_ARG;
     if (c->n_classes > 64 || c->hidden > 512) return RETEXO_ERR_UNSUPPORTED;
+    if (c->layer_norm && !(c->ln_eps > 0.f)) return RETEXO_ERR_INVALID_ARG;
+    if (c->layer_norm && c->dropout > 0.f) return RETEXO_ERR_UNSUPPORTED;
     return RETEXO_OK;
 }
 
@@ -405,7 +407,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
     for (int m = 1; m <= c.K; ++m) {
         const RoundDims r = round_dims(c, m);
         const int64_t ld16 = round_up(r.d_in, 64);
-        const int64_t nt = retexo_theta_size(r.d_in, r.hidden, c.n_classes);
+        const int64_t nt = retexo_theta_size_ln(r.d_in, r.hidden, c.n_classes, c.layer_norm);
 
         // ---- one message-passing round: X = COMBINE(Q, AGGR(Q)), emitted in bf16 for the model
         const bool gat = c.aggr == RETEXO_GAT;
@@ -471,14 +473,19 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         model.eps = c.eps; model.step = 0;
         model.dropout = c.dropout; model.dropout_seed = c.dropout_seed + (uint64_t)(m - 1);
         model.status_out = nullptr;
+        model.layer_norm = c.layer_norm; model.ln_eps = c.ln_eps;
         retexo_mlp best = model;
         best.theta = b.theta_best;
 
         // ---- R training iterations; validation and best-iterate tracking stay on the device
-        const MlpPlan plan = make_plan(r.d_in, r.hidden, c.n_classes, n_tr, n_val);
+        const MlpPlan plan = make_plan(r.d_in, r.hidden, c.n_classes, n_tr, n_val, c.layer_norm != 0);
         MlpBuffers sb{};
         mlp_step_buffers(plan, b.ws_step, b.ws_step_bytes, &sb);
         bf16* val_hd = reinterpret_cast<bf16*>(b.ws_embed);      // [n_val x ld_h] scratch of a stand-alone validation forward
+        // (layer norm: its fp32 pre-normalisation rows [n_val x hidden] sit behind it; the embedding workspace
+        //  is sized for all n >= n_val rows of both)
+        float* val_z = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(b.ws_embed) +
+                                                round_up((int64_t)sizeof(bf16) * n_val * plan.ld_h, 256));
         // cur_correct[0]: hits of the validation rows riding along; cur_correct[1]: the update kernel's
         // count of finished blocks.  Both are cleared here once and left clear by the update kernel.
         // cur_correct[2]: updates applied so far in this round (the iteration number lives on the device).
@@ -587,7 +594,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
                     RETEXO_TRY(pack_batches());
                 }
                 RETEXO_TRY(mlp_count_hits_launch(plan, sb, &model, xval16, ld_tr, n_val, val_hd, b.y_val,
-                                                 b.cur_correct, st));
+                                                 b.cur_correct, st, val_z));
                 snapshot_if_better_kernel<<<(unsigned)((nt + 255) / 256), 256, 0, st>>>(
                     b.cur_correct, b.best_correct, b.have_best, b.theta, b.theta_best, nt);
                 if (gat_train)

@@ -14,6 +14,7 @@
 // The column of ones behind X and Hd turns each bias gradient into one more output
 // row, so the partial sums come out laid out exactly like theta = [W1 | b1 | W2 | b2].
 #include "gemm_tc.h"
+#include "layer_norm.h"
 #include "mlp_kernels.cuh"
 #include "mlp_plan.h"
 
@@ -51,11 +52,13 @@ static int64_t tc_split(int64_t M, int64_t N, int64_t K) {
 
 int64_t gemm_split(int64_t M, int64_t N, int64_t K) { return tc_split(M, N, K); }
 
-MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval) {
+MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval, bool layer_norm) {
     MlpPlan p{};
     p.d_in = d_in; p.hidden = hidden; p.n_classes = n_classes; p.n_rows = n_rows; p.n_eval = n_eval;
     p.out1 = hidden > 0 ? hidden : n_classes;
-    p.nt = retexo_theta_size(d_in, hidden, n_classes);
+    p.layer_norm = (layer_norm && hidden > 0) ? 1 : 0;
+    p.ln_blocks = p.layer_norm ? ln_backward_blocks(n_rows) : 0;
+    p.nt = retexo_theta_size_ln(d_in, hidden, n_classes, p.layer_norm);
     p.ld_dl = pad_ld(n_classes);                           // 64: classes padded with zero columns
     p.ld_h = pad_ld(hidden > 0 ? hidden : 1);
     p.ld_h1 = pad_ld(hidden > 0 ? hidden + 1 : 1);
@@ -88,6 +91,11 @@ static void layout(const MlpPlan& p, Taker& t, MlpBuffers* out) {
     b.pw1 = t.template take<float>((size_t)p.split_w1 * (p.d_in + 1) * p.out1);
     b.pw2 = t.template take<float>(h ? (size_t)p.split_w2 * (p.hidden + 1) * p.n_classes : 1);
     b.status = t.template take<int32_t>(64);
+    if (p.layer_norm) {
+        b.z1 = t.template take<float>(n_all * (size_t)p.hidden);
+        b.ln_stats = t.template take<float2>(n_all);
+        b.pln = t.template take<float>((size_t)p.ln_blocks * 2 * p.hidden);
+    }
     if (out) *out = b;
 }
 
@@ -111,8 +119,14 @@ static int check_model(const retexo_mlp* m) {
     if (!m || m->d_in <= 0 || m->hidden < 0 || m->n_classes <= 0 || !m->theta) return RETEXO_ERR_INVALID_ARG;
     if (m->n_classes > 64 || m->hidden > 512) return RETEXO_ERR_UNSUPPORTED;
     if (!(m->dropout >= 0.f && m->dropout < 1.f)) return RETEXO_ERR_INVALID_ARG;
+    if (m->layer_norm && m->hidden > 0) {
+        if (!(m->ln_eps > 0.f)) return RETEXO_ERR_INVALID_ARG;
+        if (m->hidden > kLnMaxHidden || m->dropout > 0.f) return RETEXO_ERR_UNSUPPORTED;
+    }
     return RETEXO_OK;
 }
+
+static bool uses_layer_norm(const retexo_mlp* m) { return m->layer_norm && m->hidden > 0; }
 
 // bf16 shadows of the weights in the orientations the products need.
 static int build_weight_shadows(const MlpPlan& p, const MlpBuffers& b, const float* theta, cudaStream_t st) {
@@ -140,6 +154,10 @@ extern "C" int64_t retexo_theta_size(int32_t d_in, int32_t hidden, int32_t n_cla
     return (int64_t)d_in * n_classes + n_classes;
 }
 
+extern "C" int64_t retexo_theta_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes, int32_t layer_norm) {
+    return retexo_theta_size(d_in, hidden, n_classes) + ((layer_norm && hidden > 0) ? 2 * (int64_t)hidden : 0);
+}
+
 extern "C" int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld_src, int32_t dim,
                                 const int32_t* idx, int64_t n_rows, void* dst, int64_t ld_dst,
                                 void* dst_t, int64_t ld_t, int32_t ones, void* stream) {
@@ -161,10 +179,15 @@ extern "C" int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld
     return launch_status();
 }
 
+extern "C" size_t retexo_mlp_train_step_workspace_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes,
+                                                          int64_t n_rows, int32_t layer_norm) {
+    if (d_in <= 0 || hidden < 0 || n_classes <= 0 || n_rows <= 0) return 0;
+    return mlp_step_workspace_size(make_plan(d_in, hidden, n_classes, n_rows, 0, layer_norm != 0));
+}
+
 extern "C" size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes,
                                                        int64_t n_rows) {
-    if (d_in <= 0 || hidden < 0 || n_classes <= 0 || n_rows <= 0) return 0;
-    return mlp_step_workspace_size(make_plan(d_in, hidden, n_classes, n_rows));
+    return retexo_mlp_train_step_workspace_size_ln(d_in, hidden, n_classes, n_rows, 0);
 }
 
 extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t ldx, int32_t x_has_ones,
@@ -178,11 +201,12 @@ extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t l
     if (x_has_ones && ldx < (int64_t)model->d_in + 1) return RETEXO_ERR_INVALID_ARG;
     if (dx_out && ld_dx < model->d_in) return RETEXO_ERR_INVALID_ARG;
     if (!aligned_to(x, 16) || ldx % 8 != 0) return RETEXO_ERR_ALIGNMENT;
-    const size_t need = retexo_mlp_train_step_workspace_size(model->d_in, model->hidden, model->n_classes, n_rows);
+    const size_t need = retexo_mlp_train_step_workspace_size_ln(model->d_in, model->hidden, model->n_classes, n_rows,
+                                                                uses_layer_norm(model));
     if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    const MlpPlan p = make_plan(model->d_in, model->hidden, model->n_classes, n_rows);
+    const MlpPlan p = make_plan(model->d_in, model->hidden, model->n_classes, n_rows, 0, uses_layer_norm(model));
     Arena ws(workspace, workspace_bytes);
     MlpBuffers b{};
     layout(p, ws, &b);
@@ -226,9 +250,17 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     const bf16* grad1 = b.dl16;      // gradient at the first layer's output, one batch row per line
     int64_t ld_grad1 = p.ld_dl;
     int64_t n_loss = (n_all + 127) / 128;
+    const bool ln = p.layer_norm != 0;
+    const float* ln_gamma = theta + retexo_theta_size(d_in, H, O);      // (layer norm) [gamma | beta] end theta
     if (H > 0) {
-        fwd.relu = 1; fwd.out_bf16 = b.hd16; fwd.ld_bf16 = p.ld_h1; fwd.ones_col = 1;
-        fwd.relu_bits = b.gate_bits; fwd.ld_bits = p.ld_bits;
+        if (ln) {
+            // the product leaves z = X W1 + b1 in fp32; the row-local kernel normalises, applies the ReLU and
+            // writes [Hd | 1] and the gate bits as the plain forward epilogue would
+            fwd.out_f32 = b.z1; fwd.ld_f32 = H;
+        } else {
+            fwd.relu = 1; fwd.out_bf16 = b.hd16; fwd.ld_bf16 = p.ld_h1; fwd.ones_col = 1;
+            fwd.relu_bits = b.gate_bits; fwd.ld_bits = p.ld_bits;
+        }
         if (dropping) {
             fwd.mode = TC_EPI_BIAS_DROP;
             fwd.drop_thresh = (uint32_t)floor((double)model->dropout * 4294967296.0);
@@ -240,6 +272,13 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
             fwd.drop_rows = n;
         }
         RETEXO_TRY(tc_gemm_launch(fwd, st));
+        if (ln) {
+            LnForward lf{};
+            lf.z = b.z1; lf.ld_z = H; lf.gamma = ln_gamma; lf.beta = ln_gamma + H; lf.eps = model->ln_eps; lf.H = H;
+            lf.n_rows = n_all; lf.out_bf16 = b.hd16; lf.ld_bf16 = p.ld_h1; lf.ones = 1;
+            lf.bits = b.gate_bits; lf.ld_bits = p.ld_bits; lf.stats = b.ln_stats;
+            RETEXO_TRY(ln_forward_launch(lf, st));
+        }
         // ---- class product, loss and gated back-propagation
         HeadBackward hb{};
         hb.hd = b.hd16; hb.ld_hd = p.ld_h1; hb.gate_bits = b.gate_bits; hb.ld_bits = p.ld_bits; hb.w2t = b.w2t16; hb.ld_w2t = p.ld_h; hb.b2 = b2;
@@ -267,6 +306,12 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         TcGemm g2 = tc_base(b.hd16, p.ld_h1, b.dl16, p.ld_dl, (int64_t)H + 1, O, n, b.status);
         g2.mode = TC_EPI_PARTIAL; g2.splits = (int)p.split_w2; g2.partial = b.pw2;
         RETEXO_TRY(tc_gemm_launch(g2, st));
+        if (ln) {      // through the normalisation: dHd (in place) becomes the gradient at z; partials of d gamma, d beta
+            LnBackward lb{};
+            lb.z = b.z1; lb.ld_z = H; lb.stats = b.ln_stats; lb.gamma = ln_gamma; lb.H = H; lb.n_rows = n;
+            lb.dy = b.dhd16; lb.ld_dy = p.ld_h; lb.partial = b.pln;
+            RETEXO_TRY(ln_backward_launch(lb, st));
+        }
         grad1 = b.dhd16;
         ld_grad1 = p.ld_h;
     } else {
@@ -292,6 +337,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     u.n_seg = H > 0 ? 2 : 1;
     u.seg[0] = {((int64_t)d_in + 1) * out1, b.pw1, p.split_w1};
     if (H > 0) u.seg[1] = {((int64_t)H + 1) * O, b.pw2, p.split_w2};
+    if (ln) { u.n_seg = 3; u.seg[2] = {2 * (int64_t)H, b.pln, p.ln_blocks}; }
     u.theta = model->theta; u.m = model->adam_m; u.v = model->adam_v; u.grad_out = grad_out;
     u.optimizer = model->optimizer; u.lr = model->lr; u.beta1 = model->beta1; u.beta2 = model->beta2;
     u.eps = model->eps;
@@ -313,7 +359,8 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         u.step_dev = dev->step; u.done = dev->done; u.loss_base = dev->loss_base; u.history_base = dev->history_base;
         u.loss_out = nullptr;
     }
-    const int64_t tiles = (((int64_t)d_in + 16) / 16) * ((out1 + 15) / 16) + (H > 0 ? (((int64_t)H + 16) / 16) * ((O + 15) / 16) : 0);
+    const int64_t tiles = (((int64_t)d_in + 16) / 16) * ((out1 + 15) / 16) + (H > 0 ? (((int64_t)H + 16) / 16) * ((O + 15) / 16) : 0) +
+                          (ln ? ((int64_t)H + 15) / 16 : 0);      // (layer norm: [gamma ; beta] is a 2 x hidden segment)
     u.status_out = model->status_out;
     OverlapLaunch ol(dim3((unsigned)tiles), dim3(256), 0, st);
     if (cudaLaunchKernelEx(&ol.cfg, reduce_update_kernel, u) != cudaSuccess) {
@@ -323,8 +370,20 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     return launch_status();
 }
 
+// Hd = ReLU(LayerNorm(z)) for rows whose z = x W1 + b1 the forward product has left in fp32.
+static int normalise_rows(const retexo_mlp* model, const float* z, int64_t n_rows, bf16* hd16, int64_t ld16,
+                          float* hidden_out, int64_t ld_hidden, cudaStream_t st) {
+    const int32_t H = model->hidden;
+    const float* gamma = model->theta + retexo_theta_size(model->d_in, H, model->n_classes);
+    LnForward lf{};
+    lf.z = z; lf.ld_z = H; lf.gamma = gamma; lf.beta = gamma + H; lf.eps = model->ln_eps; lf.H = H; lf.n_rows = n_rows;
+    lf.out_bf16 = hd16; lf.ld_bf16 = ld16; lf.out_f32 = hidden_out; lf.ld_f32 = ld_hidden;
+    return ln_forward_launch(lf, st);
+}
+
 int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model, const bf16* x, int64_t ldx,
-                          int64_t n_rows, bf16* hd_ws, const int32_t* y, unsigned long long* correct, cudaStream_t st) {
+                          int64_t n_rows, bf16* hd_ws, const int32_t* y, unsigned long long* correct, cudaStream_t st,
+                          float* z_ws) {
     const int32_t d_in = p.d_in, H = p.hidden, O = p.n_classes, out1 = p.out1;
     const float* b1 = model->theta + (int64_t)d_in * out1;
     const float* b2 = b1 + out1 + (int64_t)H * O;
@@ -333,8 +392,15 @@ int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     TcGemm fwd = tc_base(x, ldx, b.w1t16, p.ld_k, n_rows, out1, d_in, b.status);
     fwd.bias = b1;
     if (H > 0) {
-        fwd.relu = 1; fwd.out_bf16 = hd_ws; fwd.ld_bf16 = p.ld_h;
-        RETEXO_TRY(tc_gemm_launch(fwd, st));
+        if (p.layer_norm) {
+            if (!z_ws) return RETEXO_ERR_WORKSPACE;
+            fwd.out_f32 = z_ws; fwd.ld_f32 = H;
+            RETEXO_TRY(tc_gemm_launch(fwd, st));
+            RETEXO_TRY(normalise_rows(model, z_ws, n_rows, hd_ws, p.ld_h, nullptr, 0, st));
+        } else {
+            fwd.relu = 1; fwd.out_bf16 = hd_ws; fwd.ld_bf16 = p.ld_h;
+            RETEXO_TRY(tc_gemm_launch(fwd, st));
+        }
         TcGemm l2 = tc_base(hd_ws, p.ld_h, b.w2t16, p.ld_h, n_rows, O, H, b.status);
         l2.bias = b2; l2.mode = TC_EPI_ARGMAX; l2.y = y; l2.correct = correct;
         return tc_gemm_launch(l2, st);
@@ -346,6 +412,11 @@ int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
 }  // namespace retexo
 
 extern "C" size_t retexo_embed_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows) {
+    return retexo_embed_workspace_size_ln(d_in, hidden, n_classes, n_rows, 0);
+}
+
+extern "C" size_t retexo_embed_workspace_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows,
+                                                 int32_t layer_norm) {
     if (d_in <= 0 || hidden < 0 || n_classes <= 0 || n_rows < 0) return 0;
     Sizer s;
     const size_t out1 = hidden > 0 ? hidden : n_classes;
@@ -356,6 +427,7 @@ extern "C" size_t retexo_embed_workspace_size(int32_t d_in, int32_t hidden, int3
     s.take<bf16>(hidden > 0 ? (size_t)n_rows * pad_ld(hidden) : 1);              // Hd
     s.take<float>((size_t)n_rows * n_classes);                                      // logits
     s.take<int32_t>(64);
+    if (layer_norm && hidden > 0) s.take<float>((size_t)n_rows * hidden);           // z = x W1 + b1 before the normalisation
     return s.off + kAlign;
 }
 
@@ -374,7 +446,8 @@ extern "C" int retexo_embed(const retexo_mlp* model, const void* x, int64_t ldx,
     if (logits_out && ld_logits < O) return RETEXO_ERR_INVALID_ARG;
     if (correct_out && !y) return RETEXO_ERR_INVALID_ARG;
     if (!aligned_to(x, 16) || ldx % 8 != 0) return RETEXO_ERR_ALIGNMENT;
-    const size_t need = retexo_embed_workspace_size(d_in, H, O, n_rows);
+    const bool ln = uses_layer_norm(model);
+    const size_t need = retexo_embed_workspace_size_ln(d_in, H, O, n_rows, ln);
     if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     Arena ws(workspace, workspace_bytes);
@@ -387,6 +460,7 @@ extern "C" int retexo_embed(const retexo_mlp* model, const void* x, int64_t ldx,
     b.hd16 = ws.take<bf16>(H > 0 ? (size_t)n_rows * p.ld_h : 1);
     b.logits = ws.take<float>((size_t)n_rows * O);
     b.status = ws.take<int32_t>(64);
+    float* z_ws = ln ? ws.take<float>((size_t)n_rows * H) : nullptr;
     unsigned long long* correct = reinterpret_cast<unsigned long long*>(correct_out);
 
     if (correct) RETEXO_CUDA_TRY(cudaMemsetAsync(correct, 0, sizeof(unsigned long long), st));
@@ -409,10 +483,18 @@ extern "C" int retexo_embed(const retexo_mlp* model, const void* x, int64_t ldx,
         if (H > 0) {
             bf16* h16 = hidden_out_bf16 ? static_cast<bf16*>(hidden_out_bf16) : b.hd16;
             const int64_t ld16 = hidden_out_bf16 ? ld_hidden_bf16 : p.ld_h;
-            g.N = H; g.B = w1; g.ldb = H; g.relu = 1; g.bias = b1;
-            g.out_f32 = hidden_out; g.ld_f32 = ld_hidden;
-            g.out_bf16 = (want_logits || hidden_out_bf16) ? h16 : nullptr; g.ld_bf16 = ld16;
-            RETEXO_TRY(launch_gemm(g, st));
+            g.N = H; g.B = w1; g.ldb = H; g.bias = b1;
+            if (ln) {
+                g.out_f32 = z_ws; g.ld_f32 = H;
+                RETEXO_TRY(launch_gemm(g, st));
+                RETEXO_TRY(normalise_rows(model, z_ws, n_rows, (want_logits || hidden_out_bf16) ? h16 : nullptr, ld16,
+                                          hidden_out, ld_hidden, st));
+            } else {
+                g.relu = 1;
+                g.out_f32 = hidden_out; g.ld_f32 = ld_hidden;
+                g.out_bf16 = (want_logits || hidden_out_bf16) ? h16 : nullptr; g.ld_bf16 = ld16;
+                RETEXO_TRY(launch_gemm(g, st));
+            }
             if (want_logits) {
                 GemmArgs g2{};
                 g2.M = n_rows; g2.N = O; g2.K = H; g2.A = h16; g2.lda = ld16; g2.B = w2; g2.ldb = O;
@@ -428,13 +510,20 @@ extern "C" int retexo_embed(const retexo_mlp* model, const void* x, int64_t ldx,
         TcGemm fwd = tc_base(static_cast<const bf16*>(x), ldx, b.w1t16, p.ld_k, n_rows, out1, d_in, b.status);
         fwd.bias = b1;
         if (H > 0) {
-            fwd.relu = 1; fwd.out_f32 = hidden_out; fwd.ld_f32 = ld_hidden;
             // the logits product reads Hd through TMA, so it wants an aligned copy with a stride of 8 elements
             const bool user16_ok = hidden_out_bf16 && aligned_to(hidden_out_bf16, 16) && ld_hidden_bf16 % 8 == 0;
             bf16* h16 = user16_ok ? static_cast<bf16*>(hidden_out_bf16) : b.hd16;
             const int64_t ld16 = user16_ok ? ld_hidden_bf16 : p.ld_h;
-            fwd.out_bf16 = (want_logits || user16_ok) ? h16 : nullptr; fwd.ld_bf16 = ld16;
-            RETEXO_TRY(tc_gemm_launch(fwd, st));
+            if (ln) {
+                fwd.out_f32 = z_ws; fwd.ld_f32 = H;
+                RETEXO_TRY(tc_gemm_launch(fwd, st));
+                RETEXO_TRY(normalise_rows(model, z_ws, n_rows, (want_logits || user16_ok) ? h16 : nullptr, ld16, hidden_out,
+                                          ld_hidden, st));
+            } else {
+                fwd.relu = 1; fwd.out_f32 = hidden_out; fwd.ld_f32 = ld_hidden;
+                fwd.out_bf16 = (want_logits || user16_ok) ? h16 : nullptr; fwd.ld_bf16 = ld16;
+                RETEXO_TRY(tc_gemm_launch(fwd, st));
+            }
             if (hidden_out_bf16 && !user16_ok)      // odd layout asked for: a second, plain copy
                 RETEXO_TRY(retexo_pack_rows(hidden_out ? (const void*)hidden_out : (const void*)b.hd16,
                                             hidden_out ? 0 : 1, hidden_out ? ld_hidden : p.ld_h, H, nullptr, n_rows,

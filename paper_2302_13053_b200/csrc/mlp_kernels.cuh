@@ -205,7 +205,7 @@ struct GradSeg {
     int64_t count;
 };
 struct UpdateArgs {
-    GradSeg seg[2];            // [W1 | b1] and (hidden > 0) [W2 | b2], each laid out like theta
+    GradSeg seg[3];            // [W1 | b1], (hidden > 0) [W2 | b2] and (layer norm) [gamma | beta], each laid out like theta
     int n_seg;
     float* theta;
     float* m;
@@ -274,14 +274,17 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     // read-modify-write a sector that fifteen other blocks are writing too).
     const int32_t rows0 = u.d_in + 1, cols0 = u.out1;
     const int32_t tc0 = (cols0 + 15) >> 4, tiles0 = ((rows0 + 15) >> 4) * tc0;
-    const int sidx = (int32_t)blockIdx.x < tiles0 ? 0 : 1;
-    const int32_t rows = sidx == 0 ? rows0 : u.hidden + 1, cols = sidx == 0 ? cols0 : u.n_classes;
-    const int32_t tcs = (cols + 15) >> 4, tile = sidx == 0 ? (int32_t)blockIdx.x : (int32_t)blockIdx.x - tiles0;
+    const int32_t tiles1 = u.n_seg > 1 ? ((u.hidden + 1 + 15) >> 4) * ((u.n_classes + 15) >> 4) : 0;
+    // (the third segment, a layer norm's [gamma ; beta], is a 2 x hidden matrix: one row of tiles)
+    const int sidx = (int32_t)blockIdx.x < tiles0 ? 0 : ((int32_t)blockIdx.x < tiles0 + tiles1 ? 1 : 2);
+    const int32_t rows = sidx == 0 ? rows0 : (sidx == 1 ? u.hidden + 1 : 2), cols = sidx == 0 ? cols0 : (sidx == 1 ? u.n_classes : u.hidden);
+    const int32_t tcs = (cols + 15) >> 4;
+    const int32_t tile = (int32_t)blockIdx.x - (sidx == 0 ? 0 : (sidx == 1 ? tiles0 : tiles0 + tiles1));
     const int32_t row0 = (tile / tcs) << 4, col0 = (tile % tcs) << 4;
     const int32_t row = row0 + ((int32_t)threadIdx.x >> 4), col = col0 + ((int32_t)threadIdx.x & 15);
     const int64_t size = (int64_t)rows * cols;
     const int64_t q = (int64_t)row * cols + col;
-    const int64_t p = sidx == 0 ? q : q + u.seg[0].size;
+    const int64_t p = q + (sidx == 0 ? 0 : (sidx == 1 ? u.seg[0].size : u.seg[0].size + u.seg[1].size));
     const bool live = row < rows && col < cols;
     const bool adam = u.optimizer != RETEXO_SGD;
 
@@ -296,8 +299,7 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     if (live) {
         theta = u.theta[p];
         if (adam) { m = u.m[p]; v = u.v[p]; }
-        g = sum_partials((sidx == 0 ? u.seg[0].partial : u.seg[1].partial) + q,
-                         sidx == 0 ? u.seg[0].count : u.seg[1].count, size);
+        g = sum_partials(u.seg[sidx].partial + q, u.seg[sidx].count, size);
     }
 
     float corr1 = u.corr1, corr2 = u.corr2;
@@ -365,10 +367,10 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
         t16 = f32_to_bf16(t);
         if (row < rows - 1) {                   // the weights (not the bias row), as the products read them
             if (sidx == 0) { if (u.w1r16) u.w1r16[(int64_t)row * u.ld_o1 + col] = t16; }
-            else if (u.w2p16) u.w2p16[(int64_t)row * u.ld_dl + col] = t16;
+            else if (sidx == 1 && u.w2p16) u.w2p16[(int64_t)row * u.ld_dl + col] = t16;
         }
     }
-    bf16* wt = sidx == 0 ? u.w1t16 : u.w2t16;
+    bf16* wt = sidx == 0 ? u.w1t16 : (sidx == 1 ? u.w2t16 : nullptr);
     if (wt) {                                   // uniform over the block
         __shared__ bf16 tile16[16][18];
         tile16[threadIdx.x >> 4][threadIdx.x & 15] = t16;

@@ -25,6 +25,8 @@ struct MlpPlan {
     int64_t ld_x1;                          // row stride of the workspace copy [X | 1] (d_in + 1 rounded up to 64)
     int64_t sm_blocks;                      // loss partials the workspace has room for
     int64_t split_w1, split_w2;             // split-K factors of the two weight-gradient products
+    int32_t layer_norm;                     // f_theta = Linear -> LayerNorm -> ReLU; theta ends in [gamma | beta]
+    int64_t ln_blocks;                      // partial sums of [d gamma | d beta] the backward kernel leaves
 };
 
 struct MlpBuffers {
@@ -42,12 +44,16 @@ struct MlpBuffers {
     float* pw1;                             // [split_w1 x (d_in+1) x out1]   partials of [dW1 ; db1]
     float* pw2;                             // [split_w2 x (hidden+1) x n_classes]   partials of [dW2 ; db2]
     int32_t* status;                        // raised by a tensor-core kernel whose bounded wait gave up
+    float* z1;                              // layer norm: x W1 + b1 in fp32   [n x hidden]
+    float2* ln_stats;                       // layer norm: (mean, 1 / sqrt(var + eps)) per row   [n]
+    float* pln;                             // layer norm: [ln_blocks x 2 hidden] partials of [d gamma | d beta]
 };
 
 // Split-K factor the library uses for a weight-gradient product C[M x N] = A^T B reduced over K rows.
 int64_t gemm_split(int64_t M, int64_t N, int64_t K);
 
-MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval = 0);
+MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval = 0,
+                  bool layer_norm = false);
 size_t mlp_step_workspace_size(const MlpPlan& p);
 
 // Validation folded into a training iteration: the batch holds p.n_eval more rows after the
@@ -102,10 +108,11 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
                           float* dx_out = nullptr, int64_t ld_dx = 0);      // dx_out: fp32 [n_rows x ld_dx], dLoss / dX
 
 // Forward + arg-max + hit count over a dense batch with the weight copies in `b` (which must
-// hold model->theta): what validation needs after every iteration.  hd_ws: bf16 [n_rows x p.ld_h].
+// hold model->theta): what validation needs after every iteration.  hd_ws: bf16 [n_rows x p.ld_h];
+// z_ws: fp32 [n_rows x hidden], needed with layer normalisation only.
 int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
                           const __nv_bfloat16* x, int64_t ldx, int64_t n_rows, __nv_bfloat16* hd_ws,
-                          const int32_t* y, unsigned long long* correct, cudaStream_t st);
+                          const int32_t* y, unsigned long long* correct, cudaStream_t st, float* z_ws = nullptr);
 
 int convert_f32_to_bf16_launch(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st);
 
