@@ -59,7 +59,7 @@ AGG_DRAM_TRAFFIC = {
               ("cfg4_sage_reddit_like", 3): 5.99e9, ("cfg5_gcn_products_like", 1): 46.68e9,
               ("cfg5_gcn_products_like", 2): 102.92e9, ("cfg5_gcn_products_like", 3): 102.93e9}}
 # one stand-alone training iteration (its tensor-core launches and reduce_update_kernel): profiles/mlp_iteration_cfg4.txt
-STEP_SOURCES = ("gemm_tc.cu", "mlp_fused.cu", "mlp.cu", "mlp_kernels.cuh", "tc_common.cuh")
+STEP_SOURCES = ("gemm_tc.cu", "mlp_fused.cu", "mlp.cu", "mlp_kernels.cuh", "tc_common.cuh", "launch_overlap.cuh")
 STEP_DRAM_TRAFFIC = {"fingerprint": None, "bytes": {}}
 
 
@@ -379,6 +379,28 @@ def phase_breakdown(w, ws, R: int, peaks, l2_peak=None):
     return phases, l2_peak
 
 
+def iteration_only(w, ws, m: int, calls: int = 12):
+    """Runs `calls` stand-alone training iterations of round m's model at the shapes phase_breakdown times
+    (training rows only, column of ones in the batch) and nothing else after the round's input is built:
+    what a profiler capture of the iteration wants (`--iteration-only M`).  The batch holds synthetic
+    values of the aggregated rows' shape: the kernels' work does not depend on them."""
+    import torch
+    from paper_2302_13053_b200 import binding as B
+    rd, wt = w.round_dims()[m - 1], ws[m - 1]
+    tr = torch.from_numpy(w.train_idx).to("cuda")
+    y_tr = torch.from_numpy(w.labels).to("cuda")[tr.long()].contiguous()
+    g = torch.Generator(device="cuda").manual_seed(m)
+    x = torch.randn((tr.numel(), rd["d_in"]), generator=g, device="cuda", dtype=torch.float32)
+    xtr, _ = B.retexo_pack_rows(x, None, ones=True)
+    del x
+    model = B.Mlp(rd["d_in"], rd["hidden"], w.n_classes, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
+    for _ in range(calls):
+        B.retexo_mlp_train_step(model, xtr, y_tr, x_has_ones=True)
+    torch.cuda.synchronize()
+    print(json.dumps(dict(iteration_only=m, calls=calls, rows=int(tr.numel()), d_in=rd["d_in"], hidden=rd["hidden"],
+                          status=int(model.status.item()))))
+
+
 def second_large_graph_aggregation(peaks, l2_peak):
     """The aggregation rounds of the other of the two largest graphs (the products-shaped GCN run), timed
     alone like the rounds of the benchmarked workload, so that one run reports both."""
@@ -500,6 +522,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
+    ap.add_argument("--iteration-only", type=int, default=0, metavar="M",
+                    help="run a dozen stand-alone training iterations of round M's model and exit (profiler captures)")
     ap.add_argument("--no-second-graph", action="store_true",
                     help="with the default workload, do not time the products-shaped graph's aggregation rounds as well")
     args = ap.parse_args()
@@ -522,6 +546,9 @@ def main():
     peaks = load_peaks()
 
     w, ws, gen_s = build_workload(args.config, args.scale)
+    if args.iteration_only:
+        iteration_only(w, ws, args.iteration_only)
+        return
     R = args.iters or w.R
     prob = make_problem(w, ws, host=False, R=R)
     torch.cuda.synchronize()

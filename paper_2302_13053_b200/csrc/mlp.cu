@@ -363,7 +363,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
                           (ln ? ((int64_t)H + 15) / 16 : 0);      // (layer norm: [gamma ; beta] is a 2 x hidden segment)
     u.status_out = model->status_out;
     OverlapLaunch ol(dim3((unsigned)tiles), dim3(256), 0, st);
-    if (cudaLaunchKernelEx(&ol.cfg, reduce_update_kernel, u) != cudaSuccess) {
+    if (cudaLaunchKernelEx(&ol.cfg, p.split_w1 <= 16 ? reduce_update_kernel<16> : reduce_update_kernel<32>, u) != cudaSuccess) {
         (void)cudaGetLastError();
         return RETEXO_ERR_CUDA;
     }

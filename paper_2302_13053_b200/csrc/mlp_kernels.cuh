@@ -246,17 +246,24 @@ __host__ __device__ __forceinline__ double pow_whole(double base, unsigned long 
     return r;
 }
 
-// Sum of one parameter's split-K partials in index order.  Up to 32 loads are in flight before the
-// first addition waits for one (warps issue in order, so a loop of small batches would pay the
-// memory latency once per batch).
-__device__ __forceinline__ float sum_partials(const float* __restrict__ src, int64_t count, int64_t stride) {
+// Sum of one parameter's split-K partials in index order.  BATCH loads are in flight before the first addition
+// waits for one (warps issue in order, so a loop of small batches would pay the memory latency once per batch;
+// a larger batch costs registers, and with them the blocks an SM holds at once: the launcher picks 16 where
+// that covers the largest layer's partials in one go, else 32).
+template <int BATCH>
+__device__ __forceinline__ float sum_partials(const float* __restrict__ src, int32_t count, int64_t stride) {
     float g = 0.f;
-    for (int64_t z = 0; z < count; z += 32) {
-        float x[32];
+    for (int32_t z = 0; z < count; z += BATCH) {
+        float x[BATCH];
+        const float* s = src;
 #pragma unroll
-        for (int i = 0; i < 32; ++i) x[i] = z + i < count ? __ldcs(src + (z + i) * stride) : 0.f;   // read once: streamed
+        for (int i = 0; i < BATCH; ++i) {
+            x[i] = z + i < count ? __ldcs(s) : 0.f;      // read once: streamed
+            s += stride;
+        }
 #pragma unroll
-        for (int i = 0; i < 32; ++i) g += x[i];
+        for (int i = 0; i < BATCH; ++i) g += x[i];
+        src = s;
     }
     return g;
 }
@@ -267,7 +274,8 @@ __device__ __forceinline__ float sum_partials(const float* __restrict__ src, int
 // The kernel sits between two products on the critical path of an iteration and moves little
 // data, so it is laid out for latency: every load that depends on nothing (the iteration state,
 // the partials, the parameter and its moments) is issued before anything waits.
-__global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
+template <int BATCH>
+__global__ void __launch_bounds__(256, BATCH == 16 ? 4 : 2) reduce_update_kernel(UpdateArgs u) {
     // A block owns a 16 x 16 tile of one segment's (inputs + 1) x outputs matrix (the last row is the
     // bias): 64-byte runs of each partial on the way in, and whole 32-byte sectors of the transposed
     // bf16 copy on the way out (a 2-byte store per parameter into a row of its own has every store
@@ -299,7 +307,7 @@ __global__ void __launch_bounds__(256) reduce_update_kernel(UpdateArgs u) {
     if (live) {
         theta = u.theta[p];
         if (adam) { m = u.m[p]; v = u.v[p]; }
-        g = sum_partials(u.seg[sidx].partial + q, u.seg[sidx].count, size);
+        g = sum_partials<BATCH>(u.seg[sidx].partial + q, (int32_t)u.seg[sidx].count, size);
     }
 
     float corr1 = u.corr1, corr2 = u.corr2;
