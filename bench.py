@@ -169,11 +169,15 @@ def build_workload(index: int, scale: float):
     return w, ws, time.time() - t
 
 
+FREEZE_ATTENTION = False      # --freeze-attention: GAT with its aggregator's parameters fixed (one aggregation per round)
+
+
 def make_problem(w, ws, host: bool, R: int):
     from paper_2302_13053_b200 import binding as B
     return B.LmpProblem(w.aggr, w.K, R, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
                         w.train_idx, w.val_idx, w.test_idx, ws, part=w.part, n_parts=w.n_parts, heads=w.heads,
-                        head_dim=w.head_dim, negative_slope=w.negative_slope, host=host)
+                        head_dim=w.head_dim, negative_slope=w.negative_slope, host=host,
+                        freeze_attention=FREEZE_ATTENTION)
 
 
 def launches_per_step(w, R: int) -> int:
@@ -185,13 +189,16 @@ def launches_per_step(w, R: int) -> int:
     for rd in w.round_dims():
         h = rd["hidden"]
         gat_forward = 1 + 1 + 2                      # W_att^T copy, projection, scores + rows
-        if w.aggr == wl.GAT:
+        trained_gat = w.aggr == wl.GAT and not FREEZE_ATTENTION
+        if trained_gat:
             total += 1                               # the round's input as a bf16 operand
             total += 3 * gat_forward                 # last and kept iterate for the test rows, kept iterate for the emission
+        elif w.aggr == wl.GAT:
+            total += 1 + gat_forward + 2             # input operand, one aggregation; train / val batches
         else:
             total += 3 + 2                           # prep, warp rows, block rows; train / val batches
         step = 5 if h > 0 else 3                     # products, fused middle, reduce + update (+ weight copies once)
-        if w.aggr == wl.GAT:
+        if trained_gat:
             # the aggregator is trained with the model: per iteration projection + aggregation + batches before
             # the step, input gradient inside it, kept copy + scatter + backward (4) + dW_att + update after it
             step += gat_forward + 2 + 1 + 8
@@ -525,11 +532,15 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-breakdown", action="store_true")
+    ap.add_argument("--freeze-attention", action="store_true",
+                    help="GAT workloads: keep the aggregator's parameters fixed (the round aggregates once)")
     ap.add_argument("--iteration-only", type=int, default=0, metavar="M",
                     help="run a dozen stand-alone training iterations of round M's model and exit (profiler captures)")
     ap.add_argument("--no-second-graph", action="store_true",
                     help="with the default workload, do not time the products-shaped graph's aggregation rounds as well")
     args = ap.parse_args()
+    global FREEZE_ATTENTION
+    FREEZE_ATTENTION = bool(args.freeze_attention)
     if args.impl == "reference":
         run_reference(args)
         return

@@ -42,6 +42,7 @@ def lib():
         _lib = C.CDLL(build())
         _lib.oracle_theta_size.restype = C.c_int64
         _lib.oracle_theta_size_ln.restype = C.c_int64
+        _lib.oracle_theta_size_norm.restype = C.c_int64
         _lib.oracle_bf16_round.restype = C.c_float
         _lib.oracle_bf16_round.argtypes = [C.c_float]
     return _lib
@@ -186,20 +187,29 @@ class Mlp:
     def __init__(self, d_in: int, hidden: int, n_classes: int, w1, b1, w2=None, b2=None,
                  optimizer: int = ADAM, lr: float = 0.003, beta1: float = 0.9, beta2: float = 0.999,
                  eps: float = 1e-8, round_bf16: bool = True, layer_norm: bool = False, ln_eps: float = 1e-5,
-                 ln_gamma=None, ln_beta=None):
+                 ln_gamma=None, ln_beta=None, batch_norm: bool = False, bn_momentum: float = 0.1,
+                 bn_mean=None, bn_var=None):
         """layer_norm: f_theta = Linear -> LayerNorm -> ReLU (Section 2.2 lists normalisation layers among the
-        parts of f_theta); gamma (default ones) and beta (default zeros) are trained and sit at the end of theta."""
+        parts of f_theta); gamma (default ones) and beta (default zeros) are trained and sit at the end of theta.
+        batch_norm: Linear -> BatchNorm -> ReLU instead: batch statistics while training, running statistics
+        (init 0 / 1, behind gamma and beta in theta, moved by bn_momentum per step) in embed(); eps = ln_eps."""
         self.d_in, self.hidden, self.n_classes = int(d_in), int(hidden), int(n_classes)
+        assert not (layer_norm and batch_norm)
         self.layer_norm, self.ln_eps = bool(layer_norm) and hidden > 0, float(ln_eps)
+        self.batch_norm, self.bn_momentum = bool(batch_norm) and hidden > 0, float(bn_momentum)
         parts = [np.asarray(w1, dtype=np.float64).ravel(), np.asarray(b1, dtype=np.float64).ravel()]
         if hidden > 0:
             parts += [np.asarray(w2, dtype=np.float64).ravel(), np.asarray(b2, dtype=np.float64).ravel()]
-        if self.layer_norm:
+        if self.layer_norm or self.batch_norm:
             parts += [np.ones(hidden) if ln_gamma is None else np.asarray(ln_gamma, dtype=np.float64).ravel(),
                       np.zeros(hidden) if ln_beta is None else np.asarray(ln_beta, dtype=np.float64).ravel()]
+        if self.batch_norm:
+            parts += [np.zeros(hidden) if bn_mean is None else np.asarray(bn_mean, dtype=np.float64).ravel(),
+                      np.ones(hidden) if bn_var is None else np.asarray(bn_var, dtype=np.float64).ravel()]
         self.theta = np.ascontiguousarray(np.concatenate(parts))
-        assert self.theta.shape[0] == lib().oracle_theta_size_ln(C.c_int32(d_in), C.c_int32(hidden),
-                                                                 C.c_int32(n_classes), C.c_int32(int(self.layer_norm)))
+        self.norm = 1 if self.layer_norm else (2 if self.batch_norm else 0)
+        assert self.theta.shape[0] == lib().oracle_theta_size_norm(C.c_int32(d_in), C.c_int32(hidden),
+                                                                   C.c_int32(n_classes), C.c_int32(self.norm))
         self.m = np.zeros_like(self.theta)
         self.v = np.zeros_like(self.theta)
         self.optimizer, self.lr, self.beta1, self.beta2, self.eps = optimizer, lr, beta1, beta2, eps
@@ -225,9 +235,12 @@ class Mlp:
             o += self.hidden * self.n_classes
             d["b2"] = t[o:o + self.n_classes]
             o += self.n_classes
-        if self.layer_norm:
+        if self.layer_norm or self.batch_norm:
             d["ln_gamma"] = t[o:o + self.hidden]
             d["ln_beta"] = t[o + self.hidden:o + 2 * self.hidden]
+        if self.batch_norm:
+            d["bn_mean"] = t[o + 2 * self.hidden:o + 3 * self.hidden]
+            d["bn_var"] = t[o + 3 * self.hidden:o + 4 * self.hidden]
         return d
 
     def train_step_dx(self, x: np.ndarray, y: np.ndarray, row_idx: Optional[np.ndarray] = None):
@@ -247,6 +260,8 @@ class Mlp:
                 _p(ri), C.c_int64(n_rows), _p(y), C.byref(loss), _p(grad), _p(dx))
         if self.layer_norm:
             rc = lib().oracle_mlp_train_step_ln(*args, C.c_double(self.ln_eps))
+        elif self.batch_norm:
+            rc = lib().oracle_mlp_train_step_bn(*args, C.c_double(self.ln_eps), C.c_double(self.bn_momentum))
         else:
             rc = lib().oracle_mlp_train_step_dx(*args)
         _check(rc, "oracle_mlp_train_step_dx")
@@ -274,6 +289,9 @@ class Mlp:
         if self.layer_norm:
             assert dropout == 0.0, "layer normalisation and dropout are not combined here"
             rc = lib().oracle_mlp_train_step_ln(*args, None, C.c_double(self.ln_eps))
+        elif self.batch_norm:
+            assert dropout == 0.0, "batch normalisation and dropout are not combined here"
+            rc = lib().oracle_mlp_train_step_bn(*args, None, C.c_double(self.ln_eps), C.c_double(self.bn_momentum))
         elif dropout > 0.0:
             rc = lib().oracle_mlp_train_step_dropout(*args, C.c_double(dropout), C.c_uint64(dropout_seed))
         else:
@@ -306,7 +324,12 @@ class Mlp:
                 C.c_int32(int(self.round_bf16)), _p(x), C.c_int64(x.shape[1]), _p(ri), C.c_int64(n_rows),
                 _p(hid), C.c_int64(self.hidden), _p(lg), C.c_int64(self.n_classes), _p(pred), _p(yy),
                 C.byref(correct))
-        rc = lib().oracle_embed_ln(*args, C.c_double(self.ln_eps)) if self.layer_norm else lib().oracle_embed(*args)
+        if self.layer_norm:
+            rc = lib().oracle_embed_ln(*args, C.c_double(self.ln_eps))
+        elif self.batch_norm:
+            rc = lib().oracle_embed_bn(*args, C.c_double(self.ln_eps))
+        else:
+            rc = lib().oracle_embed(*args)
         _check(rc, "oracle_embed")
         return dict(hidden=hid, logits=lg, pred=pred, correct=int(correct.value))
 
@@ -452,7 +475,7 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
               dropout: float = 0.0, dropout_seed: int = 0,
               forced_theta: Optional[Sequence[np.ndarray]] = None, train_attention: bool = False,
               forced_att: Optional[Sequence[np.ndarray]] = None, layer_norm: bool = False,
-              ln_eps: float = 1e-5) -> Dict:
+              ln_eps: float = 1e-5, batch_norm: bool = False, bn_momentum: float = 0.1) -> Dict:
     """Lazy message passing (Section 3.1): for each layer m = 1..K, one
     message-passing round builds the layer's inputs, the layer (with a
     temporary classifier unless it is the last) is trained alone for R
@@ -498,7 +521,8 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
             hd = w["w_att"].shape[1]
             layer = GatLayer(rowptr, colidx, gat, w["w_att"], w["a_src"], w["a_dst"],
                              Mlp(hd, hid, n_classes, w["w1"], w["b1"], w.get("w2"), w.get("b2"), optimizer=optimizer,
-                                 lr=lr, round_bf16=round_bf16, layer_norm=layer_norm, ln_eps=ln_eps))
+                                 lr=lr, round_bf16=round_bf16, layer_norm=layer_norm, ln_eps=ln_eps, batch_norm=batch_norm,
+                                 bn_momentum=bn_momentum))
             best, best_correct, best_iter = None, -1, -1
             losses, val_hist = [], []
             for r in range(1, R + 1):
@@ -548,7 +572,8 @@ def lmp_train(aggr: int, K: int, R: int, hidden: int, n_classes: int, lr: float,
         report["n_aggregations"] += 1
         hid = hidden if m < K else 0
         model = Mlp(x.shape[1], hid, n_classes, w["w1"], w["b1"], w.get("w2"), w.get("b2"),
-                    optimizer=optimizer, lr=lr, round_bf16=round_bf16, layer_norm=layer_norm, ln_eps=ln_eps)
+                    optimizer=optimizer, lr=lr, round_bf16=round_bf16, layer_norm=layer_norm, ln_eps=ln_eps,
+                    batch_norm=batch_norm, bn_momentum=bn_momentum)
         best, best_correct, best_iter = None, -1, -1
         losses, val_hist = [], []
         for r in range(1, R + 1):

@@ -353,6 +353,23 @@ int64_t oracle_theta_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes, in
     return oracle_theta_size(d_in, hidden, n_classes) + ((layer_norm && hidden > 0) ? 2 * (int64_t)hidden : 0);
 }
 
+/* Batch normalisation inside f_theta (the other normalisation Section 2.2 names).  Reading taken here, the
+ * usual one of the framework the paper's code is written in: between the fully-connected layer and the ReLU,
+ *   training:   zhat = (z - mean_b) / sqrt(var_b + eps), mean_b and the biased variance var_b taken per hidden
+ *               unit over the rows of the (full) training batch;  Hd = ReLU(gamma .* zhat + beta);
+ *               running statistics  r_mean <- (1 - mom) r_mean + mom mean_b,
+ *                                   r_var  <- (1 - mom) r_var  + mom var_b n / (n - 1)   (unbiased);
+ *   evaluation: zhat = (z - r_mean) / sqrt(r_var + eps)  (validation, test, emission of Q^m);
+ * theta = [ W1 | b1 | W2 | b2 | gamma | beta | r_mean | r_var ]: gamma, beta trained, the running statistics
+ * state that the optimiser does not touch (their gradient entries are 0).  `norm`: 0 none, 1 layer
+ * normalisation, 2 batch normalisation.  Rounded mode: as for layer normalisation (wide inside, the gated
+ * gradient enters the backward pass rounded to bf16). */
+int64_t oracle_theta_size_norm(int32_t d_in, int32_t hidden, int32_t n_classes, int32_t norm)
+{
+    int64_t extra = (hidden > 0 && norm == 1) ? 2 * (int64_t)hidden : ((hidden > 0 && norm == 2) ? 4 * (int64_t)hidden : 0);
+    return oracle_theta_size(d_in, hidden, n_classes) + extra;
+}
+
 /* ------------------------------------------------------------------ */
 /* Dropout (Appendix B lists dropout rates among the hyper-parameters; */
 /* the configurations use none).  The random bits come from the        */
@@ -407,14 +424,14 @@ static void forward_row_ln(int32_t d_in, int32_t hidden, int32_t n_classes, cons
                            int round_bf16, const float *xrow, const double *w1r, const double *w2r,
                            double *a1, double *logits, const double *keep,
                            const double *ln_gamma, const double *ln_beta, double ln_eps,
-                           double *zhat_out, double *rstd_out);
+                           double *zhat_out, double *rstd_out, const double *bn_mean, const double *bn_rstd);
 
 static void forward_row(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
                         int round_bf16, const float *xrow, const double *w1r, const double *w2r,
                         double *a1, double *logits, const double *keep)
 {
     forward_row_ln(d_in, hidden, n_classes, theta, round_bf16, xrow, w1r, w2r, a1, logits, keep,
-                   NULL, NULL, 0.0, NULL, NULL);
+                   NULL, NULL, 0.0, NULL, NULL, NULL, NULL);
 }
 
 /* ln_gamma != NULL: layer normalisation between the first linear layer and the ReLU; a1 then holds the
@@ -424,8 +441,10 @@ static void forward_row_ln(int32_t d_in, int32_t hidden, int32_t n_classes, cons
                            int round_bf16, const float *xrow, const double *w1r, const double *w2r,
                            double *a1, double *logits, const double *keep,
                            const double *ln_gamma, const double *ln_beta, double ln_eps,
-                           double *zhat_out, double *rstd_out)
+                           double *zhat_out, double *rstd_out, const double *bn_mean, const double *bn_rstd)
 {
+    /* bn_mean != NULL (with ln_gamma, ln_beta): batch normalisation with the given per-unit mean and
+     * 1 / sqrt(var + eps) instead of the row's own statistics */
     if (hidden > 0) {
         const double *b1 = theta + (int64_t)d_in * hidden;
         const double *b2 = b1 + hidden + (int64_t)hidden * n_classes;
@@ -437,7 +456,13 @@ static void forward_row_ln(int32_t d_in, int32_t hidden, int32_t n_classes, cons
             for (int32_t j = 0; j < hidden; ++j) a1[j] += xv * wrow[j];
         }
         for (int32_t j = 0; j < hidden; ++j) a1[j] += b1[j];
-        if (ln_gamma) {
+        if (ln_gamma && bn_mean) {
+            for (int32_t j = 0; j < hidden; ++j) {
+                double zh = (a1[j] - bn_mean[j]) * bn_rstd[j];
+                if (zhat_out) zhat_out[j] = zh;
+                a1[j] = ln_gamma[j] * zh + ln_beta[j];
+            }
+        } else if (ln_gamma) {
             double mean = 0.0, var = 0.0;
             for (int32_t j = 0; j < hidden; ++j) mean += a1[j];
             mean /= (double)hidden;
@@ -531,14 +556,17 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
                            const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
                            const int32_t *y, double *loss_out, double *grad_out,
                            double drop_p, uint64_t drop_seed, double *dx_out,
-                           int32_t layer_norm, double ln_eps)
+                           int32_t layer_norm /* 0 none, 1 layer, 2 batch normalisation */, double ln_eps,
+                           double bn_momentum)
 {
     if (d_in <= 0 || n_classes <= 0 || hidden < 0 || n_rows <= 0 || ldx < d_in) return ORACLE_BAD_ARG;
     if (drop_p < 0.0 || drop_p >= 1.0) return ORACLE_BAD_ARG;
     if (layer_norm && (hidden <= 0 || ln_eps <= 0.0)) return ORACLE_BAD_ARG;
+    const int batch_norm = layer_norm == 2;
+    if (batch_norm && (n_rows < 2 || bn_momentum < 0.0 || bn_momentum > 1.0)) return ORACLE_BAD_ARG;
     const int dropping = drop_p > 0.0 && hidden > 0;
     if (optimizer == 1 && (!adam_m || !adam_v || step < 1)) return ORACLE_BAD_ARG;
-    int64_t nt = oracle_theta_size_ln(d_in, hidden, n_classes, layer_norm);
+    int64_t nt = oracle_theta_size_norm(d_in, hidden, n_classes, layer_norm);
     int32_t out1 = hidden > 0 ? hidden : n_classes;
     /* layer normalisation: gamma and beta sit behind [W1 | b1 | W2 | b2] */
     const double *ln_gamma = layer_norm ? theta + oracle_theta_size(d_in, hidden, n_classes) : NULL;
@@ -549,6 +577,41 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
     if (layer_norm && (!zh_all || !dy_all)) { free(zh_all); free(dy_all); return ORACLE_NO_MEM; }
     double *w1r, *w2r;
     if (rounded_weights(d_in, hidden, n_classes, theta, round_bf16, &w1r, &w2r)) { free(zh_all); free(dy_all); return ORACLE_NO_MEM; }
+    /* batch normalisation: the statistics of z = x W1 + b1 over the whole batch come first */
+    double *bn_mean = NULL, *bn_var = NULL, *bn_rstd = NULL;
+    if (batch_norm) {
+        bn_mean = (double *)calloc((size_t)hidden, sizeof(double));
+        bn_var = (double *)calloc((size_t)hidden, sizeof(double));
+        bn_rstd = (double *)calloc((size_t)hidden, sizeof(double));
+        double *z_all = (double *)malloc(sizeof(double) * (size_t)n_rows * hidden);
+        if (!bn_mean || !bn_var || !bn_rstd || !z_all) {
+            free(bn_mean); free(bn_var); free(bn_rstd); free(z_all); free(w1r); free(w2r); free(zh_all); free(dy_all);
+            return ORACLE_NO_MEM;
+        }
+#pragma omp parallel
+        {
+            double *lg0 = (double *)malloc(sizeof(double) * (size_t)n_classes);
+#pragma omp for schedule(static)
+            for (int64_t i = 0; i < n_rows; ++i) {
+                int64_t r = row_idx ? row_idx[i] : i;
+                forward_row(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, z_all + i * hidden, lg0, NULL);
+            }
+            free(lg0);
+        }
+        for (int64_t i = 0; i < n_rows; ++i)
+            for (int32_t j = 0; j < hidden; ++j) bn_mean[j] += z_all[i * hidden + j];
+        for (int32_t j = 0; j < hidden; ++j) bn_mean[j] /= (double)n_rows;
+        for (int64_t i = 0; i < n_rows; ++i)
+            for (int32_t j = 0; j < hidden; ++j) {
+                double d = z_all[i * hidden + j] - bn_mean[j];
+                bn_var[j] += d * d;
+            }
+        for (int32_t j = 0; j < hidden; ++j) {
+            bn_var[j] /= (double)n_rows;
+            bn_rstd[j] = 1.0 / sqrt(bn_var[j] + ln_eps);
+        }
+        free(z_all);
+    }
 
     /* per-row results of the forward/backward through the row-local part */
     double *d1 = (double *)malloc(sizeof(double) * (size_t)n_rows * out1);       /* grad wrt first linear output */
@@ -573,7 +636,7 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
             if (keep) dropout_row(i, step, hidden, drop_p, drop_seed, keep);
             double rstd = 0.0;
             forward_row_ln(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg, keep,
-                           ln_gamma, ln_beta, ln_eps, layer_norm ? zh_all + i * hidden : NULL, &rstd);
+                           ln_gamma, ln_beta, ln_eps, layer_norm ? zh_all + i * hidden : NULL, &rstd, bn_mean, bn_rstd);
             int32_t yi = y[i];
             if (yi < 0 || yi >= n_classes) { bad_label = 1; yi = 0; }
             double mx = lg[0];
@@ -597,7 +660,10 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
                     }
                     d1[i * hidden + j] = acc;
                 }
-                if (layer_norm) {
+                if (batch_norm) {
+                    /* the column sums its backward pass needs span the batch: keep the (rounded) gated gradient */
+                    for (int32_t j = 0; j < hidden; ++j) dy_all[i * hidden + j] = opnd(d1[i * hidden + j], round_bf16);
+                } else if (layer_norm) {
                     /* backward through the normalisation: with dy the gated gradient at its output,
                      *   dzhat = dy .* gamma,  dz = rstd (dzhat - mean(dzhat) - zhat mean(dzhat .* zhat)) */
                     const double *zh = zh_all + i * hidden;
@@ -624,6 +690,26 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
     double loss = 0.0;
     for (int64_t i = 0; i < n_rows; ++i) loss += row_loss[i];
     loss /= (double)n_rows;
+
+    if (batch_norm) {
+        /* backward through the batch normalisation: with dy the gated gradient at its output, per unit j
+         *   s1 = sum_rows dy,  s2 = sum_rows dy zhat,
+         *   dz = gamma rstd (dy - s1 / n - zhat s2 / n)                                   */
+        double *s1 = (double *)calloc((size_t)hidden, sizeof(double));
+        double *s2 = (double *)calloc((size_t)hidden, sizeof(double));
+        if (s1 && s2) {
+            for (int64_t i = 0; i < n_rows; ++i)
+                for (int32_t j = 0; j < hidden; ++j) {
+                    s1[j] += dy_all[i * hidden + j];
+                    s2[j] += dy_all[i * hidden + j] * zh_all[i * hidden + j];
+                }
+            for (int64_t i = 0; i < n_rows; ++i)
+                for (int32_t j = 0; j < hidden; ++j)
+                    d1[i * hidden + j] = ln_gamma[j] * bn_rstd[j] *
+                                         (dy_all[i * hidden + j] - s1[j] / (double)n_rows - zh_all[i * hidden + j] * s2[j] / (double)n_rows);
+        }
+        free(s1); free(s2);
+    }
 
     /* gradient with respect to the batch itself, dX = d1 W1^T (needed when what produces X is trained too,
      * e.g. an aggregator with parameters): one more matrix product, operands d1 and W1 rounded like the others */
@@ -689,6 +775,14 @@ static int train_step_impl(int32_t d_in, int32_t hidden, int32_t n_classes,
     free(part);
 
     oracle_apply_update(nt, theta, adam_m, adam_v, grad, optimizer, lr, beta1, beta2, eps, step);
+    if (batch_norm) {      /* running statistics: state, moved towards this batch's (gradient entries are 0) */
+        double *r_mean = theta + oracle_theta_size(d_in, hidden, n_classes) + 2 * (int64_t)hidden, *r_var = r_mean + hidden;
+        for (int32_t j = 0; j < hidden; ++j) {
+            r_mean[j] = (1.0 - bn_momentum) * r_mean[j] + bn_momentum * bn_mean[j];
+            r_var[j] = (1.0 - bn_momentum) * r_var[j] + bn_momentum * bn_var[j] * (double)n_rows / (double)(n_rows - 1);
+        }
+    }
+    free(bn_mean); free(bn_var); free(bn_rstd);
     if (loss_out) *loss_out = loss;
     if (grad_out) memcpy(grad_out, grad, sizeof(double) * (size_t)nt);
     free(w1r); free(w2r); free(d1); free(hd); free(dl); free(row_loss); free(grad); free(zh_all); free(dy_all);
@@ -703,7 +797,7 @@ int oracle_mlp_train_step(int32_t d_in, int32_t hidden, int32_t n_classes,
                           const int32_t *y, double *loss_out, double *grad_out)
 {
     return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
-                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, NULL, 0, 0.0);
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, NULL, 0, 0.0, 0.0);
 }
 
 /* The same step, also returning dX [n_rows x d_in], the gradient of the loss with respect to the batch
@@ -716,7 +810,7 @@ int oracle_mlp_train_step_dx(int32_t d_in, int32_t hidden, int32_t n_classes,
                              const int32_t *y, double *loss_out, double *grad_out, double *dx_out)
 {
     return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
-                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, dx_out, 0, 0.0);
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, dx_out, 0, 0.0, 0.0);
 }
 
 /* The same step with dropout on the hidden units: Hd = ReLU(X W1 + b1) .* keep,
@@ -731,7 +825,7 @@ int oracle_mlp_train_step_dropout(int32_t d_in, int32_t hidden, int32_t n_classe
                                   double drop_p, uint64_t drop_seed)
 {
     return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
-                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, drop_p, drop_seed, NULL, 0, 0.0);
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, drop_p, drop_seed, NULL, 0, 0.0, 0.0);
 }
 
 /* The same step with layer normalisation inside f_theta (see oracle_theta_size_ln for the reading and the
@@ -744,7 +838,22 @@ int oracle_mlp_train_step_ln(int32_t d_in, int32_t hidden, int32_t n_classes,
                              const int32_t *y, double *loss_out, double *grad_out, double *dx_out, double ln_eps)
 {
     return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
-                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, dx_out, 1, ln_eps);
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, dx_out, 1, ln_eps, 0.0);
+}
+
+/* The same step with batch normalisation inside f_theta (see oracle_theta_size_norm for the reading and the
+ * layout of theta, adam_m, adam_v and grad_out); dx_out optional. */
+int oracle_mlp_train_step_bn(int32_t d_in, int32_t hidden, int32_t n_classes,
+                             double *theta, double *adam_m, double *adam_v,
+                             int32_t optimizer, double lr, double beta1, double beta2, double eps,
+                             int64_t step, int32_t round_bf16,
+                             const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                             const int32_t *y, double *loss_out, double *grad_out, double *dx_out, double bn_eps,
+                             double bn_momentum)
+{
+    return train_step_impl(d_in, hidden, n_classes, theta, adam_m, adam_v, optimizer, lr, beta1, beta2, eps, step,
+                           round_bf16, x, ldx, row_idx, n_rows, y, loss_out, grad_out, 0.0, 0, dx_out, 2, bn_eps,
+                           bn_momentum);
 }
 
 /* Forward of the trained per-node model over a set of rows.
@@ -767,8 +876,16 @@ static int embed_impl(int32_t d_in, int32_t hidden, int32_t n_classes, const dou
     if (layer_norm && (hidden <= 0 || ln_eps <= 0.0)) return ORACLE_BAD_ARG;
     const double *ln_gamma = layer_norm ? theta + oracle_theta_size(d_in, hidden, n_classes) : NULL;
     const double *ln_beta = layer_norm ? ln_gamma + hidden : NULL;
+    /* batch normalisation (2): evaluation uses the running statistics kept in theta */
+    const double *bn_mean = layer_norm == 2 ? ln_beta + hidden : NULL;
+    double *bn_rstd = NULL;
+    if (layer_norm == 2) {
+        bn_rstd = (double *)malloc(sizeof(double) * (size_t)hidden);
+        if (!bn_rstd) return ORACLE_NO_MEM;
+        for (int32_t j = 0; j < hidden; ++j) bn_rstd[j] = 1.0 / sqrt(bn_mean[hidden + j] + ln_eps);
+    }
     double *w1r, *w2r;
-    if (rounded_weights(d_in, hidden, n_classes, theta, round_bf16, &w1r, &w2r)) return ORACLE_NO_MEM;
+    if (rounded_weights(d_in, hidden, n_classes, theta, round_bf16, &w1r, &w2r)) { free(bn_rstd); return ORACLE_NO_MEM; }
     uint64_t correct = 0;
 #pragma omp parallel reduction(+ : correct)
     {
@@ -778,7 +895,7 @@ static int embed_impl(int32_t d_in, int32_t hidden, int32_t n_classes, const dou
         for (int64_t i = 0; i < n_rows; ++i) {
             int64_t r = row_idx ? row_idx[i] : i;
             forward_row_ln(d_in, hidden, n_classes, theta, round_bf16, x + r * ldx, w1r, w2r, a1, lg, NULL,
-                           ln_gamma, ln_beta, ln_eps, NULL, NULL);
+                           ln_gamma, ln_beta, ln_eps, NULL, NULL, bn_mean, bn_rstd);
             if (hidden_out)
                 for (int32_t j = 0; j < hidden; ++j)
                     hidden_out[i * ld_hidden + j] = (float)(a1[j] > 0.0 ? a1[j] : 0.0);
@@ -796,6 +913,7 @@ static int embed_impl(int32_t d_in, int32_t hidden, int32_t n_classes, const dou
     if (correct_out) *correct_out = correct;
     free(w1r);
     free(w2r);
+    free(bn_rstd);
     return ORACLE_OK;
 }
 
@@ -808,6 +926,18 @@ int oracle_embed(int32_t d_in, int32_t hidden, int32_t n_classes, const double *
 {
     return embed_impl(d_in, hidden, n_classes, theta, round_bf16, x, ldx, row_idx, n_rows, hidden_out, ld_hidden,
                       logits_out, ld_logits, pred_out, y, correct_out, 0, 0.0);
+}
+
+/* The same with batch normalisation in evaluation mode (running statistics; theta as oracle_theta_size_norm says). */
+int oracle_embed_bn(int32_t d_in, int32_t hidden, int32_t n_classes, const double *theta,
+                    int32_t round_bf16,
+                    const float *x, int64_t ldx, const int32_t *row_idx, int64_t n_rows,
+                    float *hidden_out, int64_t ld_hidden,
+                    float *logits_out, int64_t ld_logits,
+                    int32_t *pred_out, const int32_t *y, uint64_t *correct_out, double bn_eps)
+{
+    return embed_impl(d_in, hidden, n_classes, theta, round_bf16, x, ldx, row_idx, n_rows, hidden_out, ld_hidden,
+                      logits_out, ld_logits, pred_out, y, correct_out, 2, bn_eps);
 }
 
 /* The same with layer normalisation inside f_theta: hidden_out = ReLU(gamma .* zhat + beta), theta laid out as

@@ -114,8 +114,9 @@ def round_inputs(w, m):
     return rd, x16
 
 
-@pytest.mark.parametrize("idx,m", [(4, 2), (4, 3), (5, 1), (5, 2), (5, 3)])
-def test_one_training_iteration_and_emission_at_full_size(idx, m):
+@pytest.mark.parametrize("idx,m,ln", [(4, 2, False), (4, 3, False), (5, 1, False), (5, 2, False), (5, 3, False),
+                                      (4, 1, True), (5, 2, True)])
+def test_one_training_iteration_and_emission_at_full_size(idx, m, ln):
     """The shapes of the two large configurations that the first-round test above does not cover: one
     whole training iteration on all train rows (loss, gradient, update) and the emission of sampled
     rows, each against the checker on the very batch the GPU works on."""
@@ -128,8 +129,10 @@ def test_one_training_iteration_and_emission_at_full_size(idx, m):
     xtr, _ = B.retexo_pack_rows(x16, tr, dim=d_in, ones=True)
     y = w.labels[w.train_idx]
     wt = wl.initial_weights(w)[m - 1]
-    gpu = B.Mlp(d_in, H, O, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr)
-    ref = oracle.Mlp(d_in, H, O, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr, round_bf16=True)
+    # (ln: the same with layer normalisation inside f_theta, gamma = 1 and beta = 0 to start with)
+    gpu = B.Mlp(d_in, H, O, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr, layer_norm=ln)
+    ref = oracle.Mlp(d_in, H, O, wt["w1"], wt["b1"], wt.get("w2"), wt.get("b2"), lr=w.lr, round_bf16=True,
+                     layer_norm=ln)
     x_host = xtr[:, :d_in].float().cpu().numpy()
     given = ref.copy()
     rl, rg = ref.train_step(x_host, y, return_grad=True)
