@@ -159,6 +159,8 @@ typedef enum retexo_optimizer { RETEXO_SGD = 0, RETEXO_ADAM = 1 } retexo_optimiz
  * vector with the layer's output gradient and follows the same rule); biases,
  * softmax, loss and the optimiser are fp32.  A device-side wait that runs out
  * (it never should) makes the reported loss NaN. */
+typedef enum retexo_norm { RETEXO_NORM_NONE = 0, RETEXO_NORM_LAYER = 1, RETEXO_NORM_BATCH = 2 } retexo_norm;
+
 typedef struct retexo_mlp {
     int32_t d_in, hidden, n_classes;
     float* theta;
@@ -179,20 +181,27 @@ typedef struct retexo_mlp {
      * retexo_mlp_train_step / retexo_embed call the word is copied here: RETEXO_OK, or RETEXO_ERR_TIMEOUT
      * (the loss of that step is then NaN and its outputs are not to be used).  Read it after synchronising. */
     int32_t* status_out;
-    /* Layer normalisation inside f_theta (Section 2.2 lists normalisation layers among its parts; the paper's
-     * configurations use none).  layer_norm != 0 and hidden > 0:
-     *   z = X W1 + b1,  zhat = (z - mean z) / sqrt(var z + ln_eps)  (over the hidden units of a row, biased
-     *   variance),  Hd = ReLU(gamma .* zhat + beta),
-     * gamma and beta trained, stored behind the other parameters: theta = [W1 | b1 | W2 | b2 | gamma | beta]
-     * (retexo_theta_size_ln entries; adam_m, adam_v and grad_out likewise).  The normalisation is computed in
-     * fp32, forward and backward; hidden <= 512; not combined with dropout (UNSUPPORTED).  Ignored when
-     * hidden == 0.  Workspaces: the *_workspace_size_ln functions with layer_norm = 1. */
-    int32_t layer_norm;
-    float ln_eps;
+    /* Normalisation inside f_theta (Section 2.2 names batch and layer normalisation among its parts; the
+     * paper's configurations use none).  With norm != RETEXO_NORM_NONE and hidden > 0 (ignored when hidden == 0):
+     *   z = X W1 + b1,  Hd = ReLU(gamma .* zhat + beta),  gamma and beta trained;
+     * RETEXO_NORM_LAYER: zhat = (z - mean z) / sqrt(var z + norm_eps) over the hidden units of a row (biased
+     *   variance); theta = [W1 | b1 | W2 | b2 | gamma | beta].
+     * RETEXO_NORM_BATCH: per hidden unit over the rows of the batch.  retexo_mlp_train_step uses the batch's own
+     *   mean and biased variance and then moves the running statistics kept in theta,
+     *   r_mean <- (1 - bn_momentum) r_mean + bn_momentum mean,  r_var likewise with the unbiased variance
+     *   (n_rows >= 2); retexo_embed (evaluation, emission) normalises with the running statistics;
+     *   theta = [W1 | b1 | W2 | b2 | gamma | beta | r_mean | r_var]; the running statistics are state: the
+     *   optimiser does not touch them and their entries of grad_out are 0.
+     * theta, adam_m, adam_v, grad_out hold retexo_theta_size_norm entries.  The normalisation is computed in fp32,
+     * forward and backward; hidden <= 512; not combined with dropout (UNSUPPORTED).  Workspaces: the
+     * *_workspace_size_norm functions. */
+    int32_t norm;                   /* retexo_norm */
+    float norm_eps;
+    float bn_momentum;
 } retexo_mlp;
 
 int64_t retexo_theta_size(int32_t d_in, int32_t hidden, int32_t n_classes);
-int64_t retexo_theta_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes, int32_t layer_norm);
+int64_t retexo_theta_size_norm(int32_t d_in, int32_t hidden, int32_t n_classes, int32_t norm);
 
 /* Gathers rows of a matrix into a dense bf16 batch: dst[i] = bf16(src[idx ? idx[i] : i]).
  * src is fp32 (src_is_bf16 = 0) or bf16 (1), row stride ld_src elements;
@@ -210,8 +219,8 @@ int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld_src, int32
 
 size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes,
                                             int64_t n_rows);
-size_t retexo_mlp_train_step_workspace_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes,
-                                               int64_t n_rows, int32_t layer_norm);
+size_t retexo_mlp_train_step_workspace_size_norm(int32_t d_in, int32_t hidden, int32_t n_classes,
+                                               int64_t n_rows, int32_t norm);
 
 /* One full-batch training iteration (Section 2.3: forward, loss, backward,
  * update; with a single worker the gradient average is the identity):
@@ -243,8 +252,8 @@ int retexo_mlp_train_step(retexo_mlp* model,
                           void* workspace, size_t workspace_bytes, void* stream);
 
 size_t retexo_embed_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows);
-size_t retexo_embed_workspace_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows,
-                                      int32_t layer_norm);
+size_t retexo_embed_workspace_size_norm(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows,
+                                      int32_t norm);
 
 /* Forward of the per-node model over rows x[row_idx ? row_idx[i] : i]
  * (x bf16, row stride ldx, 16-byte aligned, ldx % 8 == 0):
@@ -363,9 +372,12 @@ typedef struct retexo_lmp_config {
                                        (Section 2.2: AGGR may have trainable parameters; Section 3.1), re-aggregating
                                        locally in every iteration.  1: they stay at the values given in gat_w and the
                                        aggregation runs once per round */
-    int32_t layer_norm;             /* layer normalisation inside f_theta in the rounds that have a hidden layer (see
-                                       retexo_mlp): theta0[m], theta_best[m] then hold retexo_theta_size_ln entries */
-    float ln_eps;
+    int32_t norm;                   /* retexo_norm: normalisation inside f_theta in the rounds that have a hidden layer
+                                       (see retexo_mlp): theta0[m], theta_best[m] then hold retexo_theta_size_norm
+                                       entries (batch normalisation: theta0 carries the initial running statistics,
+                                       theta_best those of the kept iterate) */
+    float norm_eps;
+    float bn_momentum;
 } retexo_lmp_config;
 
 typedef struct retexo_lmp_inputs {

@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libretexo.so")
 _lib = None
 
 GCN, SAGE_MEAN, GAT, SAGE_MAX = 0, 1, 2, 3
+NORM_NONE, NORM_LAYER, NORM_BATCH = 0, 1, 2
 SGD, ADAM = 0, 1
 
 
@@ -41,7 +42,7 @@ class _Mlp(C.Structure):
                 ("theta", C.c_void_p), ("adam_m", C.c_void_p), ("adam_v", C.c_void_p),
                 ("optimizer", C.c_int32), ("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float),
                 ("eps", C.c_float), ("step", C.c_int64), ("dropout", C.c_float), ("dropout_seed", C.c_uint64),
-                ("status_out", C.c_void_p), ("layer_norm", C.c_int32), ("ln_eps", C.c_float)]
+                ("status_out", C.c_void_p), ("norm", C.c_int32), ("norm_eps", C.c_float), ("bn_momentum", C.c_float)]
 
 
 class _LmpConfig(C.Structure):
@@ -50,7 +51,7 @@ class _LmpConfig(C.Structure):
                 ("beta2", C.c_float), ("eps", C.c_float), ("eval_every", C.c_int32), ("gat_heads", C.c_int32),
                 ("gat_head_dim", C.c_int32), ("gat_negative_slope", C.c_float), ("memory_is_host", C.c_int32),
                 ("dropout", C.c_float), ("dropout_seed", C.c_uint64), ("gat_freeze_attention", C.c_int32),
-                ("layer_norm", C.c_int32), ("ln_eps", C.c_float)]
+                ("norm", C.c_int32), ("norm_eps", C.c_float), ("bn_momentum", C.c_float)]
 
 
 class _LmpInputs(C.Structure):
@@ -74,9 +75,9 @@ class _LmpOutputs(C.Structure):
 
 
 EXPORTS = ["retexo_status_string", "retexo_version", "retexo_validate_csr", "retexo_aggregate_workspace_size",
-           "retexo_aggregate", "retexo_gat_backward_workspace_size", "retexo_gat_backward", "retexo_theta_size", "retexo_theta_size_ln", "retexo_pack_rows",
-           "retexo_mlp_train_step_workspace_size", "retexo_mlp_train_step_workspace_size_ln",
-           "retexo_mlp_train_step", "retexo_embed_workspace_size", "retexo_embed_workspace_size_ln", "retexo_embed",
+           "retexo_aggregate", "retexo_gat_backward_workspace_size", "retexo_gat_backward", "retexo_theta_size", "retexo_theta_size_norm", "retexo_pack_rows",
+           "retexo_mlp_train_step_workspace_size", "retexo_mlp_train_step_workspace_size_norm",
+           "retexo_mlp_train_step", "retexo_embed_workspace_size", "retexo_embed_workspace_size_norm", "retexo_embed",
            "retexo_cross_partition_workspace_size", "retexo_cross_partition_bytes",
            "retexo_cross_partition_static_scratch_bytes", "retexo_cross_partition_bytes_static",
            "retexo_data_volume", "retexo_lmp_workspace_size",
@@ -94,12 +95,12 @@ def lib():
         L.retexo_status_string.restype = C.c_char_p
         L.retexo_status_string.argtypes = [C.c_int]
         for name in ("retexo_aggregate_workspace_size", "retexo_gat_backward_workspace_size",
-                     "retexo_mlp_train_step_workspace_size", "retexo_mlp_train_step_workspace_size_ln",
-                     "retexo_embed_workspace_size", "retexo_embed_workspace_size_ln", "retexo_cross_partition_workspace_size",
+                     "retexo_mlp_train_step_workspace_size", "retexo_mlp_train_step_workspace_size_norm",
+                     "retexo_embed_workspace_size", "retexo_embed_workspace_size_norm", "retexo_cross_partition_workspace_size",
                      "retexo_lmp_workspace_size", "retexo_cross_partition_static_scratch_bytes"):
             getattr(L, name).restype = C.c_size_t
         L.retexo_theta_size.restype = C.c_int64
-        L.retexo_theta_size_ln.restype = C.c_int64
+        L.retexo_theta_size_norm.restype = C.c_int64
         _lib = L
     return _lib
 
@@ -243,27 +244,35 @@ class Mlp:
     def __init__(self, d_in: int, hidden: int, n_classes: int, w1, b1, w2=None, b2=None, optimizer: int = ADAM,
                  lr: float = 0.003, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
                  device: str = "cuda", dropout: float = 0.0, dropout_seed: int = 0, layer_norm: bool = False,
-                 ln_eps: float = 1e-5, ln_gamma=None, ln_beta=None):
+                 ln_eps: float = 1e-5, ln_gamma=None, ln_beta=None, batch_norm: bool = False, bn_momentum: float = 0.1,
+                 bn_mean=None, bn_var=None):
         """layer_norm: f_theta = Linear -> LayerNorm -> ReLU, gamma (default ones) and beta (default zeros) trained
-        and stored at the end of theta."""
+        and stored at the end of theta.  batch_norm: Linear -> BatchNorm -> ReLU instead (eps = ln_eps); the running
+        mean (default zeros) and variance (default ones) follow gamma and beta in theta."""
         self.d_in, self.hidden, self.n_classes = int(d_in), int(hidden), int(n_classes)
+        assert not (layer_norm and batch_norm)
         self.layer_norm = bool(layer_norm) and hidden > 0
+        self.batch_norm = bool(batch_norm) and hidden > 0
+        self.norm = NORM_LAYER if self.layer_norm else (NORM_BATCH if self.batch_norm else NORM_NONE)
         parts = [np.asarray(w1, dtype=np.float32).ravel(), np.asarray(b1, dtype=np.float32).ravel()]
         if hidden > 0:
             parts += [np.asarray(w2, dtype=np.float32).ravel(), np.asarray(b2, dtype=np.float32).ravel()]
-        if self.layer_norm:
+        if self.norm:
             parts += [np.ones(hidden, np.float32) if ln_gamma is None else np.asarray(ln_gamma, dtype=np.float32).ravel(),
                       np.zeros(hidden, np.float32) if ln_beta is None else np.asarray(ln_beta, dtype=np.float32).ravel()]
+        if self.batch_norm:
+            parts += [np.zeros(hidden, np.float32) if bn_mean is None else np.asarray(bn_mean, dtype=np.float32).ravel(),
+                      np.ones(hidden, np.float32) if bn_var is None else np.asarray(bn_var, dtype=np.float32).ravel()]
         theta = np.concatenate(parts)
-        assert theta.shape[0] == lib().retexo_theta_size_ln(C.c_int32(d_in), C.c_int32(hidden), C.c_int32(n_classes),
-                                                            C.c_int32(int(self.layer_norm)))
+        assert theta.shape[0] == lib().retexo_theta_size_norm(C.c_int32(d_in), C.c_int32(hidden), C.c_int32(n_classes),
+                                                              C.c_int32(self.norm))
         self.theta = torch.from_numpy(theta).to(device)
         self.m = torch.zeros_like(self.theta)
         self.v = torch.zeros_like(self.theta)
         self.status = torch.full((1,), -1, dtype=torch.int32, device=device)      # written by every step / embed call
         self.c = _Mlp(self.d_in, self.hidden, self.n_classes, self.theta.data_ptr(), self.m.data_ptr(),
                       self.v.data_ptr(), optimizer, lr, beta1, beta2, eps, 0, dropout, dropout_seed,
-                      self.status.data_ptr(), int(self.layer_norm), ln_eps)
+                      self.status.data_ptr(), self.norm, ln_eps, bn_momentum)
 
     @property
     def step(self) -> int:
@@ -280,8 +289,10 @@ class Mlp:
             o += self.hidden * self.n_classes
             d["b2"] = t[o:o + self.n_classes]
             o += self.n_classes
-        if self.layer_norm:
+        if self.norm:
             d["ln_gamma"], d["ln_beta"] = t[o:o + self.hidden], t[o + self.hidden:o + 2 * self.hidden]
+        if self.batch_norm:
+            d["bn_mean"], d["bn_var"] = t[o + 2 * self.hidden:o + 3 * self.hidden], t[o + 3 * self.hidden:o + 4 * self.hidden]
         return d
 
 
@@ -297,9 +308,9 @@ def retexo_mlp_train_step(model: Mlp, x: torch.Tensor, y: torch.Tensor, x_has_on
     loss = torch.zeros((), dtype=torch.float32, device=dev)
     grad = torch.zeros_like(model.theta) if return_grad else None
     dx = torch.empty((n_rows, model.d_in), dtype=torch.float32, device=dev) if return_dx else None
-    need = lib().retexo_mlp_train_step_workspace_size_ln(C.c_int32(model.d_in), C.c_int32(model.hidden),
+    need = lib().retexo_mlp_train_step_workspace_size_norm(C.c_int32(model.d_in), C.c_int32(model.hidden),
                                                          C.c_int32(model.n_classes), C.c_int64(n_rows),
-                                                         C.c_int32(int(model.layer_norm)))
+                                                         C.c_int32(model.norm))
     ws = workspace if workspace is not None else _workspace(need, dev)
     rc = lib().retexo_mlp_train_step(C.byref(model.c), _ptr(x), C.c_int64(x.stride(0)),
                                      C.c_int32(1 if x_has_ones else 0), _ptr(y),
@@ -325,8 +336,8 @@ def retexo_embed(model: Mlp, x: torch.Tensor, row_idx: Optional[torch.Tensor] = 
     lg = torch.empty((n_rows, O), dtype=torch.float32, device=dev) if want_logits else None
     pred = torch.empty(n_rows, dtype=torch.int32, device=dev) if want_pred else None
     correct = torch.zeros(1, dtype=torch.int64, device=dev) if y is not None else None
-    need = lib().retexo_embed_workspace_size_ln(C.c_int32(model.d_in), C.c_int32(H), C.c_int32(O), C.c_int64(n_rows),
-                                                C.c_int32(int(model.layer_norm)))
+    need = lib().retexo_embed_workspace_size_norm(C.c_int32(model.d_in), C.c_int32(H), C.c_int32(O), C.c_int64(n_rows),
+                                                C.c_int32(model.norm))
     ws = workspace if workspace is not None else _workspace(need, dev)
     rc = lib().retexo_embed(C.byref(model.c), _ptr(x), C.c_int64(x.stride(0)), _ptr(row_idx), C.c_int64(n_rows),
                             _ptr(hid), C.c_int64(H), _ptr(hid16), C.c_int64(hid16.stride(0) if hid16 is not None else 0),
@@ -381,16 +392,20 @@ def retexo_cross_partition_bytes_static(rowptr: torch.Tensor, colidx: torch.Tens
     _check(rc, "retexo_cross_partition_bytes_static")
 
 
-def pack_theta(w: Dict[str, np.ndarray], layer_norm: bool = False) -> np.ndarray:
-    """theta of one round as the library lays it out; with layer_norm (and a hidden layer) it ends in
-    [gamma | beta], taken from w["ln_gamma"], w["ln_beta"] or, if absent, ones and zeros."""
+def pack_theta(w: Dict[str, np.ndarray], layer_norm: bool = False, batch_norm: bool = False) -> np.ndarray:
+    """theta of one round as the library lays it out; with layer_norm or batch_norm (and a hidden layer) it ends in
+    [gamma | beta], taken from w["ln_gamma"], w["ln_beta"] or, if absent, ones and zeros; with batch_norm the running
+    statistics follow (w["bn_mean"], w["bn_var"], else zeros and ones)."""
     parts = [np.asarray(w["w1"], dtype=np.float32).ravel(), np.asarray(w["b1"], dtype=np.float32).ravel()]
     if "w2" in w:
         parts += [np.asarray(w["w2"], dtype=np.float32).ravel(), np.asarray(w["b2"], dtype=np.float32).ravel()]
-        if layer_norm:
-            h = np.asarray(w["b1"]).shape[0]
+        h = np.asarray(w["b1"]).shape[0]
+        if layer_norm or batch_norm:
             parts += [np.asarray(w.get("ln_gamma", np.ones(h)), dtype=np.float32).ravel(),
                       np.asarray(w.get("ln_beta", np.zeros(h)), dtype=np.float32).ravel()]
+        if batch_norm:
+            parts += [np.asarray(w.get("bn_mean", np.zeros(h)), dtype=np.float32).ravel(),
+                      np.asarray(w.get("bn_var", np.ones(h)), dtype=np.float32).ravel()]
     return np.ascontiguousarray(np.concatenate(parts))
 
 
@@ -413,14 +428,15 @@ class LmpProblem:
                  beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, eval_every: int = 1,
                  host: bool = False, want_logits: bool = True, device: str = "cuda", dropout: float = 0.0,
                  dropout_seed: int = 0, freeze_attention: bool = False, layer_norm: bool = False,
-                 ln_eps: float = 1e-5):
+                 ln_eps: float = 1e-5, batch_norm: bool = False, bn_momentum: float = 0.1):
         self.host = bool(host)
         self.device = torch.device(device)
         n, e = rowptr.shape[0] - 1, colidx.shape[0]
         self.n, self.e, self.K, self.R, self.n_classes = n, e, K, R, n_classes
         self.cfg = _LmpConfig(aggr, K, R, features.shape[1], hidden, n_classes, optimizer, lr, beta1, beta2, eps,
                               eval_every, heads, head_dim, negative_slope, 1 if host else 0, dropout, dropout_seed,
-                              1 if freeze_attention else 0, 1 if layer_norm else 0, ln_eps)
+                              1 if freeze_attention else 0,
+                              NORM_LAYER if layer_norm else (NORM_BATCH if batch_norm else NORM_NONE), ln_eps, bn_momentum)
 
         def put(a: np.ndarray) -> torch.Tensor:
             t = torch.from_numpy(np.ascontiguousarray(a))
@@ -431,7 +447,7 @@ class LmpProblem:
         self.labels = put(labels.astype(np.int32))
         self.train_idx, self.val_idx, self.test_idx = (put(a.astype(np.int32)) for a in (train_idx, val_idx, test_idx))
         self.part = put(part.astype(np.int32)) if part is not None else None
-        self.theta0 = [put(pack_theta(w, layer_norm)) for w in weights]
+        self.theta0 = [put(pack_theta(w, layer_norm, batch_norm)) for w in weights]
         self.gat_w = [put(pack_gat(w)) for w in weights] if aggr == GAT else None
         self.h2d_bytes = sum(t.numel() * t.element_size() for t in
                              [self.rowptr, self.colidx, self.features, self.labels, self.train_idx, self.val_idx,

@@ -202,11 +202,11 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
         const RoundDims r = round_dims(c, m);
         if (r.d_in > max_din) max_din = r.d_in;
         if (r.rep_dim > max_rep) max_rep = r.rep_dim;
-        const int64_t nt = retexo_theta_size_ln(r.d_in, r.hidden, c.n_classes, c.layer_norm);
+        const int64_t nt = retexo_theta_size_norm(r.d_in, r.hidden, c.n_classes, c.norm);
         if (nt > max_nt) max_nt = nt;
-        size_t s = mlp_step_workspace_size(make_plan(r.d_in, r.hidden, c.n_classes, n_tr, n_val, c.layer_norm != 0));
+        size_t s = mlp_step_workspace_size(make_plan(r.d_in, r.hidden, c.n_classes, n_tr, n_val, c.norm));
         if (s > step_b) step_b = s;
-        s = retexo_embed_workspace_size_ln(r.d_in, r.hidden, c.n_classes, n, c.layer_norm);
+        s = retexo_embed_workspace_size_norm(r.d_in, r.hidden, c.n_classes, n, c.norm);
         if (s > embed_b) embed_b = s;
         s = retexo_aggregate_workspace_size(n, e, c.aggr, r.agg_dim, c.gat_heads);
         if (s > agg_b) agg_b = s;
@@ -300,8 +300,10 @@ static int check_cfg(const retexo_lmp_config* c) {
     if (c->eval_every < 1) return RETEXO_ERR_INVALID_ARG;
     if (!(c->dropout >= 0.f && c->dropout < 1.f)) return RETEXO_ERR_INVALID_ARG;
     if (c->n_classes > 64 || c->hidden > 512) return RETEXO_ERR_UNSUPPORTED;
-    if (c->layer_norm && !(c->ln_eps > 0.f)) return RETEXO_ERR_INVALID_ARG;
-    if (c->layer_norm && c->dropout > 0.f) return RETEXO_ERR_UNSUPPORTED;
+    if (c->norm != RETEXO_NORM_NONE && c->norm != RETEXO_NORM_LAYER && c->norm != RETEXO_NORM_BATCH) return RETEXO_ERR_INVALID_ARG;
+    if (c->norm && !(c->norm_eps > 0.f)) return RETEXO_ERR_INVALID_ARG;
+    if (c->norm == RETEXO_NORM_BATCH && !(c->bn_momentum >= 0.f && c->bn_momentum <= 1.f)) return RETEXO_ERR_INVALID_ARG;
+    if (c->norm && c->dropout > 0.f) return RETEXO_ERR_UNSUPPORTED;
     return RETEXO_OK;
 }
 
@@ -407,7 +409,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
     for (int m = 1; m <= c.K; ++m) {
         const RoundDims r = round_dims(c, m);
         const int64_t ld16 = round_up(r.d_in, 64);
-        const int64_t nt = retexo_theta_size_ln(r.d_in, r.hidden, c.n_classes, c.layer_norm);
+        const int64_t nt = retexo_theta_size_norm(r.d_in, r.hidden, c.n_classes, c.norm);
 
         // ---- one message-passing round: X = COMBINE(Q, AGGR(Q)), emitted in bf16 for the model
         const bool gat = c.aggr == RETEXO_GAT;
@@ -473,16 +475,16 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
         model.eps = c.eps; model.step = 0;
         model.dropout = c.dropout; model.dropout_seed = c.dropout_seed + (uint64_t)(m - 1);
         model.status_out = nullptr;
-        model.layer_norm = c.layer_norm; model.ln_eps = c.ln_eps;
+        model.norm = c.norm; model.norm_eps = c.norm_eps; model.bn_momentum = c.bn_momentum;
         retexo_mlp best = model;
         best.theta = b.theta_best;
 
         // ---- R training iterations; validation and best-iterate tracking stay on the device
-        const MlpPlan plan = make_plan(r.d_in, r.hidden, c.n_classes, n_tr, n_val, c.layer_norm != 0);
+        const MlpPlan plan = make_plan(r.d_in, r.hidden, c.n_classes, n_tr, n_val, c.norm);
         MlpBuffers sb{};
         mlp_step_buffers(plan, b.ws_step, b.ws_step_bytes, &sb);
         bf16* val_hd = reinterpret_cast<bf16*>(b.ws_embed);      // [n_val x ld_h] scratch of a stand-alone validation forward
-        // (layer norm: its fp32 pre-normalisation rows [n_val x hidden] sit behind it; the embedding workspace
+        // (normalisation: its fp32 pre-normalisation rows [n_val x hidden] sit behind it; the embedding workspace
         //  is sized for all n >= n_val rows of both)
         float* val_z = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(b.ws_embed) +
                                                 round_up((int64_t)sizeof(bf16) * n_val * plan.ld_h, 256));

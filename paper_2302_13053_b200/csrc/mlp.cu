@@ -14,6 +14,7 @@
 // The column of ones behind X and Hd turns each bias gradient into one more output
 // row, so the partial sums come out laid out exactly like theta = [W1 | b1 | W2 | b2].
 #include "gemm_tc.h"
+#include "batch_norm.h"
 #include "layer_norm.h"
 #include "mlp_kernels.cuh"
 #include "mlp_plan.h"
@@ -52,13 +53,14 @@ static int64_t tc_split(int64_t M, int64_t N, int64_t K) {
 
 int64_t gemm_split(int64_t M, int64_t N, int64_t K) { return tc_split(M, N, K); }
 
-MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval, bool layer_norm) {
+MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval, int32_t norm) {
     MlpPlan p{};
     p.d_in = d_in; p.hidden = hidden; p.n_classes = n_classes; p.n_rows = n_rows; p.n_eval = n_eval;
     p.out1 = hidden > 0 ? hidden : n_classes;
-    p.layer_norm = (layer_norm && hidden > 0) ? 1 : 0;
-    p.ln_blocks = p.layer_norm ? ln_backward_blocks(n_rows) : 0;
-    p.nt = retexo_theta_size_ln(d_in, hidden, n_classes, p.layer_norm);
+    p.norm = hidden > 0 ? norm : RETEXO_NORM_NONE;
+    p.ln_blocks = p.norm == RETEXO_NORM_LAYER ? ln_backward_blocks(n_rows) : 0;
+    p.bn_blocks = p.norm == RETEXO_NORM_BATCH ? bn_blocks(n_rows) : 0;
+    p.nt = retexo_theta_size_norm(d_in, hidden, n_classes, p.norm);
     p.ld_dl = pad_ld(n_classes);                           // 64: classes padded with zero columns
     p.ld_h = pad_ld(hidden > 0 ? hidden : 1);
     p.ld_h1 = pad_ld(hidden > 0 ? hidden + 1 : 1);
@@ -91,10 +93,16 @@ static void layout(const MlpPlan& p, Taker& t, MlpBuffers* out) {
     b.pw1 = t.template take<float>((size_t)p.split_w1 * (p.d_in + 1) * p.out1);
     b.pw2 = t.template take<float>(h ? (size_t)p.split_w2 * (p.hidden + 1) * p.n_classes : 1);
     b.status = t.template take<int32_t>(64);
-    if (p.layer_norm) {
+    if (p.norm) {
         b.z1 = t.template take<float>(n_all * (size_t)p.hidden);
-        b.ln_stats = t.template take<float2>(n_all);
-        b.pln = t.template take<float>((size_t)p.ln_blocks * 2 * p.hidden);
+        if (p.norm == RETEXO_NORM_LAYER) {
+            b.ln_stats = t.template take<float2>(n_all);
+            b.pln = t.template take<float>((size_t)p.ln_blocks * 2 * p.hidden);
+        } else {
+            b.bn_partial = t.template take<float>((size_t)p.bn_blocks * 2 * p.hidden);
+            b.bn_batch = t.template take<float>(3 * (size_t)p.hidden);
+            b.bn_sums = t.template take<float>(2 * (size_t)p.hidden);
+        }
     }
     if (out) *out = b;
 }
@@ -119,14 +127,16 @@ static int check_model(const retexo_mlp* m) {
     if (!m || m->d_in <= 0 || m->hidden < 0 || m->n_classes <= 0 || !m->theta) return RETEXO_ERR_INVALID_ARG;
     if (m->n_classes > 64 || m->hidden > 512) return RETEXO_ERR_UNSUPPORTED;
     if (!(m->dropout >= 0.f && m->dropout < 1.f)) return RETEXO_ERR_INVALID_ARG;
-    if (m->layer_norm && m->hidden > 0) {
-        if (!(m->ln_eps > 0.f)) return RETEXO_ERR_INVALID_ARG;
+    if (m->norm != RETEXO_NORM_NONE && m->norm != RETEXO_NORM_LAYER && m->norm != RETEXO_NORM_BATCH) return RETEXO_ERR_INVALID_ARG;
+    if (m->norm && m->hidden > 0) {
+        if (!(m->norm_eps > 0.f)) return RETEXO_ERR_INVALID_ARG;
+        if (m->norm == RETEXO_NORM_BATCH && !(m->bn_momentum >= 0.f && m->bn_momentum <= 1.f)) return RETEXO_ERR_INVALID_ARG;
         if (m->hidden > kLnMaxHidden || m->dropout > 0.f) return RETEXO_ERR_UNSUPPORTED;
     }
     return RETEXO_OK;
 }
 
-static bool uses_layer_norm(const retexo_mlp* m) { return m->layer_norm && m->hidden > 0; }
+static int32_t norm_of(const retexo_mlp* m) { return m->hidden > 0 ? m->norm : RETEXO_NORM_NONE; }
 
 // bf16 shadows of the weights in the orientations the products need.
 static int build_weight_shadows(const MlpPlan& p, const MlpBuffers& b, const float* theta, cudaStream_t st) {
@@ -154,8 +164,9 @@ extern "C" int64_t retexo_theta_size(int32_t d_in, int32_t hidden, int32_t n_cla
     return (int64_t)d_in * n_classes + n_classes;
 }
 
-extern "C" int64_t retexo_theta_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes, int32_t layer_norm) {
-    return retexo_theta_size(d_in, hidden, n_classes) + ((layer_norm && hidden > 0) ? 2 * (int64_t)hidden : 0);
+extern "C" int64_t retexo_theta_size_norm(int32_t d_in, int32_t hidden, int32_t n_classes, int32_t norm) {
+    if (hidden <= 0 || norm == RETEXO_NORM_NONE) return retexo_theta_size(d_in, hidden, n_classes);
+    return retexo_theta_size(d_in, hidden, n_classes) + (norm == RETEXO_NORM_BATCH ? 4 : 2) * (int64_t)hidden;
 }
 
 extern "C" int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld_src, int32_t dim,
@@ -179,15 +190,15 @@ extern "C" int retexo_pack_rows(const void* src, int32_t src_is_bf16, int64_t ld
     return launch_status();
 }
 
-extern "C" size_t retexo_mlp_train_step_workspace_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes,
-                                                          int64_t n_rows, int32_t layer_norm) {
+extern "C" size_t retexo_mlp_train_step_workspace_size_norm(int32_t d_in, int32_t hidden, int32_t n_classes,
+                                                          int64_t n_rows, int32_t norm) {
     if (d_in <= 0 || hidden < 0 || n_classes <= 0 || n_rows <= 0) return 0;
-    return mlp_step_workspace_size(make_plan(d_in, hidden, n_classes, n_rows, 0, layer_norm != 0));
+    return mlp_step_workspace_size(make_plan(d_in, hidden, n_classes, n_rows, 0, norm));
 }
 
 extern "C" size_t retexo_mlp_train_step_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes,
                                                        int64_t n_rows) {
-    return retexo_mlp_train_step_workspace_size_ln(d_in, hidden, n_classes, n_rows, 0);
+    return retexo_mlp_train_step_workspace_size_norm(d_in, hidden, n_classes, n_rows, 0);
 }
 
 extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t ldx, int32_t x_has_ones,
@@ -201,12 +212,12 @@ extern "C" int retexo_mlp_train_step(retexo_mlp* model, const void* x, int64_t l
     if (x_has_ones && ldx < (int64_t)model->d_in + 1) return RETEXO_ERR_INVALID_ARG;
     if (dx_out && ld_dx < model->d_in) return RETEXO_ERR_INVALID_ARG;
     if (!aligned_to(x, 16) || ldx % 8 != 0) return RETEXO_ERR_ALIGNMENT;
-    const size_t need = retexo_mlp_train_step_workspace_size_ln(model->d_in, model->hidden, model->n_classes, n_rows,
-                                                                uses_layer_norm(model));
+    const size_t need = retexo_mlp_train_step_workspace_size_norm(model->d_in, model->hidden, model->n_classes, n_rows,
+                                                                  norm_of(model));
     if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    const MlpPlan p = make_plan(model->d_in, model->hidden, model->n_classes, n_rows, 0, uses_layer_norm(model));
+    const MlpPlan p = make_plan(model->d_in, model->hidden, model->n_classes, n_rows, 0, norm_of(model));
     Arena ws(workspace, workspace_bytes);
     MlpBuffers b{};
     layout(p, ws, &b);
@@ -250,11 +261,13 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     const bf16* grad1 = b.dl16;      // gradient at the first layer's output, one batch row per line
     int64_t ld_grad1 = p.ld_dl;
     int64_t n_loss = (n_all + 127) / 128;
-    const bool ln = p.layer_norm != 0;
-    const float* ln_gamma = theta + retexo_theta_size(d_in, H, O);      // (layer norm) [gamma | beta] end theta
+    const bool ln = p.norm == RETEXO_NORM_LAYER, bn = p.norm == RETEXO_NORM_BATCH;
+    const float* ln_gamma = theta + retexo_theta_size(d_in, H, O);      // (normalisation) [gamma | beta (| r_mean | r_var)] end theta
+    const BnScratch bns{b.bn_partial, b.bn_batch, b.bn_sums};
+    if (bn && n < 2) return RETEXO_ERR_INVALID_ARG;                     // (the unbiased variance of the running statistics)
     if (H > 0) {
-        if (ln) {
-            // the product leaves z = X W1 + b1 in fp32; the row-local kernel normalises, applies the ReLU and
+        if (ln || bn) {
+            // the product leaves z = X W1 + b1 in fp32; the normalisation's kernel applies the ReLU and
             // writes [Hd | 1] and the gate bits as the plain forward epilogue would
             fwd.out_f32 = b.z1; fwd.ld_f32 = H;
         } else {
@@ -274,10 +287,18 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         RETEXO_TRY(tc_gemm_launch(fwd, st));
         if (ln) {
             LnForward lf{};
-            lf.z = b.z1; lf.ld_z = H; lf.gamma = ln_gamma; lf.beta = ln_gamma + H; lf.eps = model->ln_eps; lf.H = H;
+            lf.z = b.z1; lf.ld_z = H; lf.gamma = ln_gamma; lf.beta = ln_gamma + H; lf.eps = model->norm_eps; lf.H = H;
             lf.n_rows = n_all; lf.out_bf16 = b.hd16; lf.ld_bf16 = p.ld_h1; lf.ones = 1;
             lf.bits = b.gate_bits; lf.ld_bits = p.ld_bits; lf.stats = b.ln_stats;
             RETEXO_TRY(ln_forward_launch(lf, st));
+        }
+        if (bn) {      // training rows: the batch's own statistics; rows riding along for validation: the running ones
+            RETEXO_TRY(bn_batch_stats_launch(b.z1, H, n, H, model->norm_eps, bns, st));
+            BnForward bf{};
+            bf.z = b.z1; bf.ld_z = H; bf.gamma = ln_gamma; bf.beta = ln_gamma + H; bf.H = H; bf.n_rows = n_all; bf.n_batch = n;
+            bf.batch = b.bn_batch; bf.r_mean = ln_gamma + 2 * H; bf.r_var = ln_gamma + 3 * H; bf.eps = model->norm_eps;
+            bf.out_bf16 = b.hd16; bf.ld_bf16 = p.ld_h1; bf.ones = 1; bf.bits = b.gate_bits; bf.ld_bits = p.ld_bits;
+            RETEXO_TRY(bn_forward_launch(bf, st));
         }
         // ---- class product, loss and gated back-propagation
         HeadBackward hb{};
@@ -312,6 +333,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
             lb.dy = b.dhd16; lb.ld_dy = p.ld_h; lb.partial = b.pln;
             RETEXO_TRY(ln_backward_launch(lb, st));
         }
+        if (bn) RETEXO_TRY(bn_backward_launch(b.z1, H, n, H, ln_gamma, b.dhd16, p.ld_h, bns, st));
         grad1 = b.dhd16;
         ld_grad1 = p.ld_h;
     } else {
@@ -338,6 +360,10 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     u.seg[0] = {((int64_t)d_in + 1) * out1, b.pw1, p.split_w1};
     if (H > 0) u.seg[1] = {((int64_t)H + 1) * O, b.pw2, p.split_w2};
     if (ln) { u.n_seg = 3; u.seg[2] = {2 * (int64_t)H, b.pln, p.ln_blocks}; }
+    if (bn) {      // [d gamma | d beta] arrive summed; the running statistics behind them move towards the batch's
+        u.n_seg = 3; u.seg[2] = {2 * (int64_t)H, b.bn_sums, 1};
+        u.bn_batch = b.bn_batch; u.bn_momentum = model->bn_momentum; u.bn_unbias = (float)((double)n / (double)(n - 1));
+    }
     u.theta = model->theta; u.m = model->adam_m; u.v = model->adam_v; u.grad_out = grad_out;
     u.optimizer = model->optimizer; u.lr = model->lr; u.beta1 = model->beta1; u.beta2 = model->beta2;
     u.eps = model->eps;
@@ -360,7 +386,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
         u.loss_out = nullptr;
     }
     const int64_t tiles = (((int64_t)d_in + 16) / 16) * ((out1 + 15) / 16) + (H > 0 ? (((int64_t)H + 16) / 16) * ((O + 15) / 16) : 0) +
-                          (ln ? ((int64_t)H + 15) / 16 : 0);      // (layer norm: [gamma ; beta] is a 2 x hidden segment)
+                          ((ln || bn) ? ((int64_t)H + 15) / 16 : 0);      // (a normalisation's segment has 2 or 4 rows of hidden entries)
     u.status_out = model->status_out;
     OverlapLaunch ol(dim3((unsigned)tiles), dim3(256), 0, st);
     if (cudaLaunchKernelEx(&ol.cfg, p.split_w1 <= 16 ? reduce_update_kernel<16> : reduce_update_kernel<32>, u) != cudaSuccess) {
@@ -370,13 +396,21 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     return launch_status();
 }
 
-// Hd = ReLU(LayerNorm(z)) for rows whose z = x W1 + b1 the forward product has left in fp32.
+// Hd = ReLU(norm(z)) for rows whose z = x W1 + b1 the forward product has left in fp32 (evaluation: batch
+// normalisation uses its running statistics).
 static int normalise_rows(const retexo_mlp* model, const float* z, int64_t n_rows, bf16* hd16, int64_t ld16,
                           float* hidden_out, int64_t ld_hidden, cudaStream_t st) {
     const int32_t H = model->hidden;
     const float* gamma = model->theta + retexo_theta_size(model->d_in, H, model->n_classes);
+    if (model->norm == RETEXO_NORM_BATCH) {
+        BnForward bf{};
+        bf.z = z; bf.ld_z = H; bf.gamma = gamma; bf.beta = gamma + H; bf.H = H; bf.n_rows = n_rows; bf.n_batch = 0;
+        bf.r_mean = gamma + 2 * H; bf.r_var = gamma + 3 * H; bf.eps = model->norm_eps;
+        bf.out_bf16 = hd16; bf.ld_bf16 = ld16; bf.out_f32 = hidden_out; bf.ld_f32 = ld_hidden;
+        return bn_forward_launch(bf, st);
+    }
     LnForward lf{};
-    lf.z = z; lf.ld_z = H; lf.gamma = gamma; lf.beta = gamma + H; lf.eps = model->ln_eps; lf.H = H; lf.n_rows = n_rows;
+    lf.z = z; lf.ld_z = H; lf.gamma = gamma; lf.beta = gamma + H; lf.eps = model->norm_eps; lf.H = H; lf.n_rows = n_rows;
     lf.out_bf16 = hd16; lf.ld_bf16 = ld16; lf.out_f32 = hidden_out; lf.ld_f32 = ld_hidden;
     return ln_forward_launch(lf, st);
 }
@@ -392,7 +426,7 @@ int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     TcGemm fwd = tc_base(x, ldx, b.w1t16, p.ld_k, n_rows, out1, d_in, b.status);
     fwd.bias = b1;
     if (H > 0) {
-        if (p.layer_norm) {
+        if (p.norm) {
             if (!z_ws) return RETEXO_ERR_WORKSPACE;
             fwd.out_f32 = z_ws; fwd.ld_f32 = H;
             RETEXO_TRY(tc_gemm_launch(fwd, st));
@@ -412,11 +446,11 @@ int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
 }  // namespace retexo
 
 extern "C" size_t retexo_embed_workspace_size(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows) {
-    return retexo_embed_workspace_size_ln(d_in, hidden, n_classes, n_rows, 0);
+    return retexo_embed_workspace_size_norm(d_in, hidden, n_classes, n_rows, 0);
 }
 
-extern "C" size_t retexo_embed_workspace_size_ln(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows,
-                                                 int32_t layer_norm) {
+extern "C" size_t retexo_embed_workspace_size_norm(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows,
+                                                 int32_t norm) {
     if (d_in <= 0 || hidden < 0 || n_classes <= 0 || n_rows < 0) return 0;
     Sizer s;
     const size_t out1 = hidden > 0 ? hidden : n_classes;
@@ -427,7 +461,7 @@ extern "C" size_t retexo_embed_workspace_size_ln(int32_t d_in, int32_t hidden, i
     s.take<bf16>(hidden > 0 ? (size_t)n_rows * pad_ld(hidden) : 1);              // Hd
     s.take<float>((size_t)n_rows * n_classes);                                      // logits
     s.take<int32_t>(64);
-    if (layer_norm && hidden > 0) s.take<float>((size_t)n_rows * hidden);           // z = x W1 + b1 before the normalisation
+    if (norm && hidden > 0) s.take<float>((size_t)n_rows * hidden);           // z = x W1 + b1 before the normalisation
     return s.off + kAlign;
 }
 
@@ -446,8 +480,8 @@ extern "C" int retexo_embed(const retexo_mlp* model, const void* x, int64_t ldx,
     if (logits_out && ld_logits < O) return RETEXO_ERR_INVALID_ARG;
     if (correct_out && !y) return RETEXO_ERR_INVALID_ARG;
     if (!aligned_to(x, 16) || ldx % 8 != 0) return RETEXO_ERR_ALIGNMENT;
-    const bool ln = uses_layer_norm(model);
-    const size_t need = retexo_embed_workspace_size_ln(d_in, H, O, n_rows, ln);
+    const bool ln = norm_of(model) != RETEXO_NORM_NONE;
+    const size_t need = retexo_embed_workspace_size_norm(d_in, H, O, n_rows, norm_of(model));
     if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     Arena ws(workspace, workspace_bytes);

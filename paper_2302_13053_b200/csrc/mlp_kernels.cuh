@@ -205,7 +205,11 @@ struct GradSeg {
     int64_t count;
 };
 struct UpdateArgs {
-    GradSeg seg[3];            // [W1 | b1], (hidden > 0) [W2 | b2] and (layer norm) [gamma | beta], each laid out like theta
+    GradSeg seg[3];            // [W1 | b1], (hidden > 0) [W2 | b2] and (normalisation) [gamma | beta], each laid out like theta
+    // batch normalisation (optional): [r_mean | r_var] behind [gamma | beta] in theta are state, not parameters:
+    // r <- (1 - bn_momentum) r + bn_momentum s with s the batch's mean / its variance x bn_unbias (bn_batch holds
+    // mean | biased variance); their gradient entries are 0 and the optimiser's moments stay untouched
+    const float* bn_batch; float bn_momentum, bn_unbias;
     int n_seg;
     float* theta;
     float* m;
@@ -285,7 +289,7 @@ __global__ void __launch_bounds__(256, BATCH == 16 ? 4 : 2) reduce_update_kernel
     const int32_t tiles1 = u.n_seg > 1 ? ((u.hidden + 1 + 15) >> 4) * ((u.n_classes + 15) >> 4) : 0;
     // (the third segment, a layer norm's [gamma ; beta], is a 2 x hidden matrix: one row of tiles)
     const int sidx = (int32_t)blockIdx.x < tiles0 ? 0 : ((int32_t)blockIdx.x < tiles0 + tiles1 ? 1 : 2);
-    const int32_t rows = sidx == 0 ? rows0 : (sidx == 1 ? u.hidden + 1 : 2), cols = sidx == 0 ? cols0 : (sidx == 1 ? u.n_classes : u.hidden);
+    const int32_t rows = sidx == 0 ? rows0 : (sidx == 1 ? u.hidden + 1 : (u.bn_batch ? 4 : 2)), cols = sidx == 0 ? cols0 : (sidx == 1 ? u.n_classes : u.hidden);
     const int32_t tcs = (cols + 15) >> 4;
     const int32_t tile = (int32_t)blockIdx.x - (sidx == 0 ? 0 : (sidx == 1 ? tiles0 : tiles0 + tiles1));
     const int32_t row0 = (tile / tcs) << 4, col0 = (tile % tcs) << 4;
@@ -295,6 +299,7 @@ __global__ void __launch_bounds__(256, BATCH == 16 ? 4 : 2) reduce_update_kernel
     const int64_t p = q + (sidx == 0 ? 0 : (sidx == 1 ? u.seg[0].size : u.seg[0].size + u.seg[1].size));
     const bool live = row < rows && col < cols;
     const bool adam = u.optimizer != RETEXO_SGD;
+    const bool state = sidx == 2 && row >= 2;      // a running statistic of batch normalisation
 
     grid_dependency_wait();
     grid_dependency_release();
@@ -306,8 +311,12 @@ __global__ void __launch_bounds__(256, BATCH == 16 ? 4 : 2) reduce_update_kernel
     float theta = 0.f, m = 0.f, v = 0.f, g = 0.f;
     if (live) {
         theta = u.theta[p];
-        if (adam) { m = u.m[p]; v = u.v[p]; }
-        g = sum_partials<BATCH>(u.seg[sidx].partial + q, (int32_t)u.seg[sidx].count, size);
+        if (state) {
+            g = u.bn_batch[q - 2 * (int64_t)cols] * (row == 3 ? u.bn_unbias : 1.f);      // the statistic it moves towards
+        } else {
+            if (adam) { m = u.m[p]; v = u.v[p]; }
+            g = sum_partials<BATCH>(u.seg[sidx].partial + q, (int32_t)u.seg[sidx].count, sidx == 2 ? 2 * (int64_t)cols : size);      // (a partial of the third segment holds its two trained rows)
+        }
     }
 
     float corr1 = u.corr1, corr2 = u.corr2;
@@ -359,10 +368,12 @@ __global__ void __launch_bounds__(256, BATCH == 16 ? 4 : 2) reduce_update_kernel
 
     bf16 t16 = f32_to_bf16(0.f);
     if (live) {
-        if (u.grad_out) u.grad_out[p] = g;
+        if (u.grad_out) u.grad_out[p] = state ? 0.f : g;
         if (snapshot) u.theta_best[p] = theta;
         float t;
-        if (!adam) {
+        if (state) {
+            t = (1.f - u.bn_momentum) * theta + u.bn_momentum * g;
+        } else if (!adam) {
             t = theta - u.lr * g;
         } else {
             m = u.beta1 * m + (1.f - u.beta1) * g;

@@ -25,8 +25,10 @@ struct MlpPlan {
     int64_t ld_x1;                          // row stride of the workspace copy [X | 1] (d_in + 1 rounded up to 64)
     int64_t sm_blocks;                      // loss partials the workspace has room for
     int64_t split_w1, split_w2;             // split-K factors of the two weight-gradient products
-    int32_t layer_norm;                     // f_theta = Linear -> LayerNorm -> ReLU; theta ends in [gamma | beta]
-    int64_t ln_blocks;                      // partial sums of [d gamma | d beta] the backward kernel leaves
+    int32_t norm;                           // retexo_norm (0 where hidden == 0): f_theta = Linear -> norm -> ReLU; theta ends in
+                                            //   [gamma | beta] (layer) or [gamma | beta | r_mean | r_var] (batch)
+    int64_t ln_blocks;                      // layer norm: partial sums of [d gamma | d beta] the backward kernel leaves
+    int64_t bn_blocks;                      // batch norm: per-block column sums of its column-sum kernels
 };
 
 struct MlpBuffers {
@@ -44,16 +46,19 @@ struct MlpBuffers {
     float* pw1;                             // [split_w1 x (d_in+1) x out1]   partials of [dW1 ; db1]
     float* pw2;                             // [split_w2 x (hidden+1) x n_classes]   partials of [dW2 ; db2]
     int32_t* status;                        // raised by a tensor-core kernel whose bounded wait gave up
-    float* z1;                              // layer norm: x W1 + b1 in fp32   [n x hidden]
+    float* z1;                              // layer / batch norm: x W1 + b1 in fp32   [n x hidden]
     float2* ln_stats;                       // layer norm: (mean, 1 / sqrt(var + eps)) per row   [n]
     float* pln;                             // layer norm: [ln_blocks x 2 hidden] partials of [d gamma | d beta]
+    float* bn_partial;                      // batch norm: [bn_blocks x 2 hidden] per-block column sums
+    float* bn_batch;                        // batch norm: [3 hidden] mean | biased variance | 1 / sqrt(var + eps) of the batch
+    float* bn_sums;                         // batch norm: [2 hidden] d gamma | d beta
 };
 
 // Split-K factor the library uses for a weight-gradient product C[M x N] = A^T B reduced over K rows.
 int64_t gemm_split(int64_t M, int64_t N, int64_t K);
 
 MlpPlan make_plan(int32_t d_in, int32_t hidden, int32_t n_classes, int64_t n_rows, int64_t n_eval = 0,
-                  bool layer_norm = false);
+                  int32_t norm = RETEXO_NORM_NONE);
 size_t mlp_step_workspace_size(const MlpPlan& p);
 
 // Validation folded into a training iteration: the batch holds p.n_eval more rows after the
@@ -109,7 +114,7 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
 
 // Forward + arg-max + hit count over a dense batch with the weight copies in `b` (which must
 // hold model->theta): what validation needs after every iteration.  hd_ws: bf16 [n_rows x p.ld_h];
-// z_ws: fp32 [n_rows x hidden], needed with layer normalisation only.
+// z_ws: fp32 [n_rows x hidden], needed with a normalisation only.
 int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_mlp* model,
                           const __nv_bfloat16* x, int64_t ldx, int64_t n_rows, __nv_bfloat16* hd_ws,
                           const int32_t* y, unsigned long long* correct, cudaStream_t st, float* z_ws = nullptr);
