@@ -442,6 +442,51 @@ int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_inputs* in,
                      const retexo_lmp_outputs* out,
                      void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------- standard (end-to-end) training */
+/* The scheme lazy message passing is compared with (Section 2.3): one model of K layers,
+ *   H^0 = F,  X^m = COMBINE(H^{m-1}, AGGR(H^{m-1}))  (Eq. 1),  H^m = ReLU(X^m W_m + b_m) for m < K,
+ *   logits = X^K W_K + b_K,
+ * trained jointly: every iteration runs the aggregations forward and carries the gradient back through them
+ * (the transposed aggregation; on the symmetric graphs this library takes, GCN's is the aggregation itself and
+ * SAGE-mean's is dH[u] = g_self[u] + sum_{v in N(u)} g_mean[v] / deg v).  X^1 = AGGR(F) does not change and is
+ * computed once, so an iteration runs K - 1 forward and K - 1 transposed aggregations: the exchanges of
+ * H^1 .. H^{K-1} and of as many gradients that Appendix A.1 counts for standard training.
+ * aggr: RETEXO_GCN or RETEXO_SAGE_MEAN (others: UNSUPPORTED).  Layer m has theta_m = [W_m | b_m],
+ * W_m [d_m x out_m] row-major, d_m the width of X^m (d0 or hidden; twice that for SAGE), out_m = hidden for
+ * m < K and n_classes for m = K; hidden <= 512, n_classes <= 64.  Loss: mean soft-max cross-entropy over the
+ * train rows, full batch.  Validation after every iteration, the iterate with the most hits kept (earliest on
+ * ties).  Operand precision as in retexo_mlp (both operands of every product rounded to bf16, sums fp32). */
+typedef struct retexo_standard_config {
+    int32_t aggr, K, R, d0, hidden, n_classes, optimizer;
+    float lr, beta1, beta2, eps;
+} retexo_standard_config;
+
+typedef struct retexo_standard_outputs {
+    float* loss_history;            /* [R] loss of every iteration (before its update) */
+    uint64_t* val_correct;          /* [R] validation hits after every iteration */
+    uint64_t* best_val_correct;     /* [1] */
+    int32_t* best_iter;             /* [1] 1-based iteration whose weights were kept */
+    uint64_t* test_correct;         /* [1] test hits of the kept weights */
+    uint64_t* test_correct_last;    /* [1] test hits of the last iterate */
+    float* final_logits; int64_t ld_logits;   /* [n x ld] logits of the kept weights over all nodes; may be NULL */
+    int32_t* final_pred;            /* [n]; may be NULL */
+    float* const* theta_best;       /* HOST array of K device pointers receiving the kept theta_m; may be NULL */
+    float* const* grad_last;        /* HOST array of K device pointers receiving the gradients [dW_m | db_m] of the
+                                       last iteration run; may be NULL */
+    int32_t* status;                /* optional, one int32: RETEXO_OK, or RETEXO_ERR_TIMEOUT if a bounded device-side
+                                       wait ran out (the results are then not to be used) */
+} retexo_standard_outputs;
+
+size_t retexo_standard_workspace_size(const retexo_standard_config* cfg, int64_t n_nodes, int64_t n_edges,
+                                      int64_t n_train, int64_t n_val, int64_t n_test);
+
+/* Runs R iterations from in->theta0[m] (K device arrays; in->part, in->gat_w are ignored; all of `in` and `out`
+ * is device memory except the two pointer arrays).  Only enqueues work on `stream`; nothing synchronises.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA. */
+int retexo_standard_train(const retexo_standard_config* cfg, const retexo_lmp_inputs* in,
+                          const retexo_standard_outputs* out,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

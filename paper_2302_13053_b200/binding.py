@@ -61,6 +61,19 @@ class _LmpInputs(C.Structure):
                 ("theta0", C.POINTER(C.c_void_p)), ("gat_w", C.POINTER(C.c_void_p))]
 
 
+class _StandardConfig(C.Structure):
+    _fields_ = [("aggr", C.c_int32), ("K", C.c_int32), ("R", C.c_int32), ("d0", C.c_int32), ("hidden", C.c_int32),
+                ("n_classes", C.c_int32), ("optimizer", C.c_int32), ("lr", C.c_float), ("beta1", C.c_float),
+                ("beta2", C.c_float), ("eps", C.c_float)]
+
+
+class _StandardOutputs(C.Structure):
+    _fields_ = [("loss_history", C.c_void_p), ("val_correct", C.c_void_p), ("best_val_correct", C.c_void_p),
+                ("best_iter", C.c_void_p), ("test_correct", C.c_void_p), ("test_correct_last", C.c_void_p),
+                ("final_logits", C.c_void_p), ("ld_logits", C.c_int64), ("final_pred", C.c_void_p),
+                ("theta_best", C.POINTER(C.c_void_p)), ("grad_last", C.POINTER(C.c_void_p)), ("status", C.c_void_p)]
+
+
 class _DataVolume(C.Structure):
     _fields_ = [("lazy_lt", C.c_double), ("standard_lt", C.c_double), ("lazy_reduce", C.c_double),
                 ("standard_reduce", C.c_double), ("gamma", C.c_double), ("model_size", C.c_double)]
@@ -80,7 +93,7 @@ EXPORTS = ["retexo_status_string", "retexo_version", "retexo_validate_csr", "ret
            "retexo_mlp_train_step", "retexo_embed_workspace_size", "retexo_embed_workspace_size_norm", "retexo_embed",
            "retexo_cross_partition_workspace_size", "retexo_cross_partition_bytes",
            "retexo_cross_partition_static_scratch_bytes", "retexo_cross_partition_bytes_static",
-           "retexo_data_volume", "retexo_lmp_workspace_size",
+           "retexo_data_volume", "retexo_lmp_workspace_size", "retexo_standard_workspace_size", "retexo_standard_train",
            "retexo_lmp_train"]
 
 
@@ -97,7 +110,8 @@ def lib():
         for name in ("retexo_aggregate_workspace_size", "retexo_gat_backward_workspace_size",
                      "retexo_mlp_train_step_workspace_size", "retexo_mlp_train_step_workspace_size_norm",
                      "retexo_embed_workspace_size", "retexo_embed_workspace_size_norm", "retexo_cross_partition_workspace_size",
-                     "retexo_lmp_workspace_size", "retexo_cross_partition_static_scratch_bytes"):
+                     "retexo_lmp_workspace_size", "retexo_cross_partition_static_scratch_bytes",
+                     "retexo_standard_workspace_size"):
             getattr(L, name).restype = C.c_size_t
         L.retexo_theta_size.restype = C.c_int64
         L.retexo_theta_size_norm.restype = C.c_int64
@@ -534,6 +548,78 @@ def retexo_lmp_train(problem: LmpProblem) -> None:
     rc = lib().retexo_lmp_train(C.byref(problem.cfg), C.byref(problem.inputs), C.byref(problem.outputs),
                                 _ptr(problem.workspace), C.c_size_t(problem.workspace.numel()), _stream())
     _check(rc, "retexo_lmp_train")
+
+
+class StandardProblem:
+    """Inputs, workspace and outputs of a standard (end-to-end) training run of the K-layer GNN, all on the device.
+    weights[m] holds "w1" [d_m, out_m] and "b1" of layer m (other keys are ignored)."""
+
+    def __init__(self, aggr: int, R: int, hidden: int, n_classes: int, lr: float, rowptr: np.ndarray,
+                 colidx: np.ndarray, features: np.ndarray, labels: np.ndarray, train_idx: np.ndarray,
+                 val_idx: np.ndarray, test_idx: np.ndarray, weights: List[Dict[str, np.ndarray]], optimizer: int = ADAM,
+                 beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8, want_logits: bool = True,
+                 want_grad: bool = False, device: str = "cuda"):
+        dev = torch.device(device)
+        K = len(weights)
+        n, e = rowptr.shape[0] - 1, colidx.shape[0]
+        self.K, self.R, self.n = K, R, n
+        self.cfg = _StandardConfig(aggr, K, R, features.shape[1], hidden, n_classes, optimizer, lr, beta1, beta2, eps)
+        put = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+        self.rowptr, self.colidx = put(rowptr.astype(np.int64)), put(colidx.astype(np.int32))
+        self.features, self.labels = put(features.astype(np.float32)), put(labels.astype(np.int32))
+        self.train_idx, self.val_idx, self.test_idx = (put(a.astype(np.int32)) for a in (train_idx, val_idx, test_idx))
+        self.theta0 = [put(np.concatenate([np.asarray(w["w1"], dtype=np.float32).ravel(),
+                                           np.asarray(w["b1"], dtype=np.float32).ravel()])) for w in weights]
+        zeros = lambda shape, dtype: torch.zeros(shape, dtype=dtype, device=dev)
+        self.loss_history, self.val_correct = zeros((R,), torch.float32), zeros((R,), torch.int64)
+        self.best_val, self.best_iter = zeros((1,), torch.int64), zeros((1,), torch.int32)
+        self.test_correct, self.test_last = zeros((1,), torch.int64), zeros((1,), torch.int64)
+        self.final_logits = zeros((n, n_classes), torch.float32) if want_logits else None
+        self.final_pred = zeros((n,), torch.int32) if want_logits else None
+        self.theta_best = [torch.zeros_like(t) for t in self.theta0]
+        self.grad_last = [torch.zeros_like(t) for t in self.theta0] if want_grad else None
+        self.status = torch.full((1,), -1, dtype=torch.int32, device=dev)
+        arr = lambda ts: (C.c_void_p * K)(*[t.data_ptr() for t in ts])
+        self._theta0_arr, self._best_arr = arr(self.theta0), arr(self.theta_best)
+        self._grad_arr = arr(self.grad_last) if want_grad else None
+        g = _Csr(n, e, self.rowptr.data_ptr(), self.colidx.data_ptr())
+        ptr = lambda t: t.data_ptr() if t is not None and t.numel() else None
+        self.inputs = _LmpInputs(g, self.features.data_ptr(), features.shape[1], self.labels.data_ptr(),
+                                 self.train_idx.data_ptr(), self.train_idx.numel(), ptr(self.val_idx), self.val_idx.numel(),
+                                 ptr(self.test_idx), self.test_idx.numel(), None, 0,
+                                 C.cast(self._theta0_arr, C.POINTER(C.c_void_p)), None)
+        self.outputs = _StandardOutputs(self.loss_history.data_ptr(), self.val_correct.data_ptr(), self.best_val.data_ptr(),
+                                        self.best_iter.data_ptr(), self.test_correct.data_ptr(), self.test_last.data_ptr(),
+                                        ptr(self.final_logits), n_classes, ptr(self.final_pred),
+                                        C.cast(self._best_arr, C.POINTER(C.c_void_p)),
+                                        C.cast(self._grad_arr, C.POINTER(C.c_void_p)) if want_grad else None,
+                                        self.status.data_ptr())
+        need = lib().retexo_standard_workspace_size(C.byref(self.cfg), C.c_int64(n), C.c_int64(e),
+                                                    C.c_int64(self.train_idx.numel()), C.c_int64(self.val_idx.numel()),
+                                                    C.c_int64(self.test_idx.numel()))
+        if need == 0:
+            raise RetexoError("retexo_standard_workspace_size: configuration not supported")
+        self.workspace = _workspace(need, dev)
+
+    def results(self) -> Dict:
+        cpu = lambda t: t.cpu().numpy()
+        n_test = max(1, self.test_idx.numel())
+        return dict(loss_history=cpu(self.loss_history), val_correct=cpu(self.val_correct).view(np.uint64),
+                    best_val_correct=int(cpu(self.best_val)[0]), best_iter=int(cpu(self.best_iter)[0]),
+                    test_correct=int(cpu(self.test_correct)[0]), test_correct_last=int(cpu(self.test_last)[0]),
+                    test_acc=float(cpu(self.test_correct)[0]) / n_test,
+                    final_logits=None if self.final_logits is None else cpu(self.final_logits),
+                    final_pred=None if self.final_pred is None else cpu(self.final_pred),
+                    theta_best=[cpu(t) for t in self.theta_best],
+                    grad_last=[cpu(t) for t in self.grad_last] if self.grad_last else None,
+                    status=int(cpu(self.status)[0]))
+
+
+def retexo_standard_train(problem: StandardProblem) -> None:
+    """Enqueues R iterations of standard training on the current stream."""
+    rc = lib().retexo_standard_train(C.byref(problem.cfg), C.byref(problem.inputs), C.byref(problem.outputs),
+                                     _ptr(problem.workspace), C.c_size_t(problem.workspace.numel()), _stream())
+    _check(rc, "retexo_standard_train")
 
 
 def retexo_data_volume(H, L, n_workers: float, B: float, R: float) -> dict:

@@ -396,6 +396,33 @@ int mlp_train_step_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
     return launch_status();
 }
 
+// Update of one linear layer theta = [W | b] (W [d_in x out]) from the split-K partials of [X | 1]^T dZ; see mlp_plan.h.
+int linear_update_launch(int32_t d_in, int32_t out, float* theta, float* adam_m, float* adam_v, const float* partial,
+                         int64_t splits, int optimizer, float lr, float beta1, float beta2, float eps, int64_t step,
+                         bf16* wt16, int64_t ld_k, bf16* wr16, int64_t ld_o1, float* grad_out, cudaStream_t st) {
+    UpdateArgs u{};
+    u.n_seg = 1;
+    u.seg[0] = {((int64_t)d_in + 1) * out, partial, splits};
+    u.theta = theta; u.m = adam_m; u.v = adam_v; u.grad_out = grad_out;
+    u.optimizer = optimizer; u.lr = lr; u.beta1 = beta1; u.beta2 = beta2; u.eps = eps;
+    u.corr1 = (float)(1.0 - pow((double)beta1, (double)step));
+    u.corr2 = (float)(1.0 - pow((double)beta2, (double)step));
+    u.w1t16 = wt16; u.ld_k = ld_k; u.w1r16 = wr16; u.ld_o1 = ld_o1;
+    u.d_in = d_in; u.out1 = out; u.hidden = 0; u.n_classes = out;
+    const int64_t tiles = (((int64_t)d_in + 16) / 16) * ((out + 15) / 16);
+    OverlapLaunch ol(dim3((unsigned)tiles), dim3(256), 0, st);
+    if (cudaLaunchKernelEx(&ol.cfg, splits <= 16 ? reduce_update_kernel<16> : reduce_update_kernel<32>, u) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return RETEXO_ERR_CUDA;
+    }
+    return launch_status();
+}
+
+int linear_shadows_launch(int32_t d_in, int32_t out, const float* theta, bf16* wt16, int64_t ld_k, bf16* wr16, int64_t ld_o1,
+                          cudaStream_t st) {
+    return retexo_pack_rows(theta, 0, out, out, nullptr, d_in, wr16, wr16 ? ld_o1 : 0, wt16, ld_k, 0, st);
+}
+
 // Hd = ReLU(norm(z)) for rows whose z = x W1 + b1 the forward product has left in fp32 (evaluation: batch
 // normalisation uses its running statistics).
 static int normalise_rows(const retexo_mlp* model, const float* z, int64_t n_rows, bf16* hd16, int64_t ld16,

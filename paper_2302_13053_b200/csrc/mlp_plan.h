@@ -119,6 +119,17 @@ int mlp_count_hits_launch(const MlpPlan& p, const MlpBuffers& b, const retexo_ml
                           const __nv_bfloat16* x, int64_t ldx, int64_t n_rows, __nv_bfloat16* hd_ws,
                           const int32_t* y, unsigned long long* correct, cudaStream_t st, float* z_ws = nullptr);
 
+// One linear layer theta = [W | b] (W [d_in x out], row-major) of a jointly trained model: sums the `splits`
+// partials of [dW ; db] = [X | 1]^T dZ (each (d_in + 1) x out, fp32) in index order, applies update number `step`
+// of the optimiser, writes the gradient to grad_out (optional) and refreshes the bf16 copies W^T [out x ld_k] and
+// W [d_in x ld_o1] (either may be null).  linear_shadows_launch builds those copies from theta.
+int linear_update_launch(int32_t d_in, int32_t out, float* theta, float* adam_m, float* adam_v, const float* partial,
+                         int64_t splits, int optimizer, float lr, float beta1, float beta2, float eps, int64_t step,
+                         __nv_bfloat16* wt16, int64_t ld_k, __nv_bfloat16* wr16, int64_t ld_o1, float* grad_out,
+                         cudaStream_t st);
+int linear_shadows_launch(int32_t d_in, int32_t out, const float* theta, __nv_bfloat16* wt16, int64_t ld_k,
+                          __nv_bfloat16* wr16, int64_t ld_o1, cudaStream_t st);
+
 int convert_f32_to_bf16_launch(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st);
 
 }  // namespace retexo

@@ -1,0 +1,113 @@
+"""Standard (end-to-end) training of the K-layer GNN on the GPU (paper Section 2.3: the scheme lazy message
+passing is compared with) against the CPU checker: one iteration from the same weights (loss, the gradient of
+every layer, through the transposed aggregations), a short run (loss curve, what the kept weights emit), and
+the bookkeeping of the keep-the-best rule.
+
+Tolerances are those of the per-node model: loss 2e-4 for one iteration, gradients 5e-3 of a layer's largest entry,
+logits 2e-2 per rounded stage against the checker that rounds the same operands.  The median gradient error, 2e-5 of
+the largest entry for a layer that sits directly under the loss, is allowed once per layer between the loss and the
+layer judged: the gradient that reaches layer m has been rounded to bf16 as an operand K - m times on the way, and
+wherever the fp32 and the double value of an element straddle a rounding boundary the two sides carry different
+operands into everything below.  One more effect has no counterpart in the per-node model, whose two sides are handed
+the same batch: here each side aggregates its own X^m (fp32 sums in CSR order against double), so a few elements of
+X^m round to different bf16 neighbours, their rows' pre-activations move by ~1e-3, and a hidden unit that sits that
+close to zero passes the ReLU on one side only.  Such a unit (v, j) adds X^m[v][:] dH[v][j] to column j of one side's
+weight gradient: a few whole columns may therefore miss the 5e-3 bound (at most one in 32, and by no more than ten
+times), all others must meet it."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import standard
+from gpu_util import assert_logits_close
+
+pytestmark = pytest.mark.gpu
+
+
+def B():
+    from paper_2302_13053_b200 import binding
+    return binding
+
+
+def _workload(cfg, scale):
+    from paper_2302_13053_b200 import workloads as wl
+    w = wl.make_config(cfg, scale=scale)
+    return w, wl.initial_weights(w)
+
+
+def _problem(w, ws, R, **kw):
+    return B().StandardProblem(w.aggr, R, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
+                               w.train_idx, w.val_idx, w.test_idx, ws, **kw)
+
+
+@pytest.mark.parametrize("cfg,scale", [(1, 0.5), (2, 0.1), (4, 0.01), (5, 0.002)])
+def test_one_iteration_matches_the_checker(cfg, scale):
+    w, ws = _workload(cfg, scale)
+    prob = _problem(w, ws, 1, want_grad=True)
+    B().retexo_standard_train(prob)
+    torch.cuda.synchronize()
+    got = prob.results()
+    assert got["status"] == 0
+    model = standard.StandardGnn(w.aggr, w.rowptr, w.colidx, ws, lr=w.lr)
+    loss, grads = model.train_step(w.features, w.labels, w.train_idx, return_grad=True)
+    assert abs(got["loss_history"][0] - loss) <= 2e-4 * max(1.0, abs(loss)), (got["loss_history"][0], loss)
+    for m in range(w.K):
+        gg, rg = got["grad_last"][m].astype(np.float64), grads[m]
+        assert gg.shape == rg.shape
+        scale_m = np.abs(rg).max()
+        err = np.abs(gg - rg)
+        assert scale_m > 0
+        col_err = err.reshape(-1, ws[m]["w1"].shape[1]).max(axis=0)      # ([dW ; db] is (d + 1) x out)
+        off = col_err > 5e-3 * scale_m + 1e-7
+        assert off.sum() <= (len(col_err) // 32 if m < w.K - 1 else 0), (m, int(off.sum()), col_err.max(), scale_m)
+        assert col_err.max() <= 5e-2 * scale_m, (m, col_err.max(), scale_m, int(err.argmax()))
+        assert np.median(err) <= 2e-5 * (w.K - m) * scale_m, (m, np.median(err), scale_m)
+
+
+@pytest.mark.parametrize("cfg,scale", [(1, 0.5), (4, 0.01)])
+def test_short_run_tracks_the_checker_and_emits_what_its_kept_weights_give(cfg, scale):
+    w, ws = _workload(cfg, scale)
+    R = 8
+    prob = _problem(w, ws, R)
+    B().retexo_standard_train(prob)
+    torch.cuda.synchronize()
+    got = prob.results()
+    assert got["status"] == 0
+    ref = standard.standard_train(w.aggr, R, w.rowptr, w.colidx, w.features, w.labels, w.train_idx, w.val_idx, w.test_idx,
+                                  ws, lr=w.lr)
+    gl = got["loss_history"]
+    assert abs(gl[0] - ref["losses"][0]) <= 2e-4 * max(1.0, ref["losses"][0])
+    assert np.abs(gl - ref["losses"]).max() <= 2e-2 * max(1.0, np.abs(ref["losses"]).max())
+    assert gl[-1] < gl[0]
+    # the keep-the-best rule against the run's own validation curve
+    val = got["val_correct"].astype(np.int64)
+    assert got["best_val_correct"] == val.max() and got["best_iter"] == int(val.argmax()) + 1
+    assert np.abs(val - ref["val_correct"]).max() <= max(2, 0.02 * len(w.val_idx))
+    # what the run emits: the kept weights pushed through the checker's own forward pass
+    kept = standard.StandardGnn(w.aggr, w.rowptr, w.colidx, ws, lr=w.lr)
+    for m in range(w.K):
+        kept.layers[m].theta = got["theta_best"][m].astype(np.float64)
+    logits = kept.forward(w.features)[2]
+    assert_logits_close(got["final_logits"], logits, 2e-2 * w.K)
+    lg = np.sort(logits, axis=1)
+    clear = (lg[:, -1] - lg[:, -2]) > 2 * 2e-2 * w.K * np.abs(lg).max(axis=1)
+    assert np.array_equal(got["final_pred"][clear], np.argmax(logits, axis=1)[clear])
+    te = w.test_idx
+    want_hits = int((np.argmax(logits[te], axis=1) == w.labels[te]).sum())
+    assert abs(got["test_correct"] - want_hits) <= int((~clear[te]).sum())
+
+
+def test_a_second_run_gives_the_same_bits_and_other_aggregators_are_refused():
+    w, ws = _workload(4, 0.01)
+    outs = []
+    for _ in range(2):
+        prob = _problem(w, ws, 3)
+        B().retexo_standard_train(prob)
+        torch.cuda.synchronize()
+        outs.append(prob.results())
+    assert np.array_equal(outs[0]["loss_history"], outs[1]["loss_history"])
+    assert all(np.array_equal(a, b) for a, b in zip(outs[0]["theta_best"], outs[1]["theta_best"]))
+    with pytest.raises(B().RetexoError):
+        B().StandardProblem(B().GAT, 1, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
+                            w.train_idx, w.val_idx, w.test_idx, ws)
