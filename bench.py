@@ -425,6 +425,44 @@ def second_large_graph_aggregation(peaks, l2_peak):
     return out
 
 
+def standard_training(w, ws, R: int, lazy_ms_per_step: float, counts: dict):
+    """Standard (end-to-end) training of the same K-layer model on the same kernels (Section 2.3), timed beside
+    the lazy run: the time of one iteration is the difference between a run of 12 and a run of 4 iterations
+    (set-up, X^1 = AGGR(F) and the closing evaluation passes cancel), and the bytes a partitioned run would
+    exchange follow from the cross-partition count: per iteration K - 1 forward and K - 1 gradient exchanges of
+    the boundary rows at the hidden width, against one exchange per layer in all for the lazy run."""
+    import torch
+    from paper_2302_13053_b200 import binding as B
+
+    def run(iters):
+        prob = B.StandardProblem(w.aggr, iters, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features, w.labels,
+                                 w.train_idx, w.val_idx, w.test_idx, ws, want_logits=False)
+        B.retexo_standard_train(prob)                 # warm-up
+        torch.cuda.synchronize()
+        ms, _ = time_calls(lambda: B.retexo_standard_train(prob), 2, warm=0)
+        res = prob.results()
+        del prob
+        torch.cuda.empty_cache()
+        return ms, res
+    short, _ = run(4)
+    long, res = run(12)
+    per_iter = (long - short) / 8.0
+    fixed = max(short - 4 * per_iter, 0.0)
+    pairs = int(counts["boundary_pairs"])
+    lazy_bytes = int(counts["bytes_total"])
+    std_bytes = pairs * 4 * (w.d0 + R * 2 * (w.K - 1) * w.hidden)
+    est = fixed + R * per_iter
+    return dict(ms_per_iteration=per_iter, fixed_ms=fixed, est_ms_for_R_iterations=est, R=R,
+                aggregations_per_iteration=2 * (w.K - 1), lazy_ms_per_step=lazy_ms_per_step,
+                time_ratio_standard_over_lazy=est / lazy_ms_per_step,
+                exchanged_bytes_standard=std_bytes, exchanged_bytes_lazy=lazy_bytes,
+                gamma_messages=std_bytes / lazy_bytes if lazy_bytes else None, status=res["status"],
+                loss_first_last=[float(res["loss_history"][0]), float(res["loss_history"][-1])],
+                note="one GPU, no exchange: the time ratio compares computation only; gamma_messages counts the "
+                     "boundary rows a partitioned run of either scheme would send (one direction, features included "
+                     "once), without the gradient all-reduce")
+
+
 def oracle_sample(w, ws, R: int, budget_s: float = 75.0, budget_train: int = 2048):
     """Times the CPU checker on the workload within about budget_s seconds and scales to one full step
     (K rounds).  Every round's aggregation and the cross-partition count run in full where a short probe
@@ -536,6 +574,8 @@ def main():
                     help="GAT workloads: keep the aggregator's parameters fixed (the round aggregates once)")
     ap.add_argument("--iteration-only", type=int, default=0, metavar="M",
                     help="run a dozen stand-alone training iterations of round M's model and exit (profiler captures)")
+    ap.add_argument("--no-standard", action="store_true",
+                    help="skip the standard-training comparison (same model trained end to end on the same kernels)")
     ap.add_argument("--no-second-graph", action="store_true",
                     help="with the default workload, do not time the products-shaped graph's aggregation rounds as well")
     args = ap.parse_args()
@@ -674,6 +714,9 @@ def main():
                                unit=p["unit"], frac=round(p["frac"], 4),
                                **({"edges_per_s": p["edges_per_s"]} if "edges_per_s" in p else {}))
                           for p in phases]
+    if not args.no_standard and world == 1 and w.aggr in (B.GCN, B.SAGE_MEAN):
+        torch.cuda.empty_cache()
+        line["standard_training"] = standard_training(w, ws, R, ms_per_step, res["counts"])
     if not args.no_cpu_baseline:
         import oracle
         t, detail, sample, kind = oracle_sample(w, ws, R)
