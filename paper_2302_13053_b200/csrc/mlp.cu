@@ -27,17 +27,9 @@ namespace retexo {
 // tensor-map box straddles two lines.
 static inline int64_t pad_ld(int64_t x) { return (x + 63) / 64 * 64; }
 
-static int launch_gemm(const GemmArgs& g, cudaStream_t st) {
-    if (g.M <= 0 || g.N <= 0) return RETEXO_OK;
-    dim3 grid((unsigned)((g.N + kBN - 1) / kBN), (unsigned)((g.M + kBM - 1) / kBM), 1);
-    gemm_bf16_kernel<<<grid, kGemmThreads, 0, st>>>(g);
-    return launch_status();
-}
+// rows of a gathered batch that retexo_embed packs and multiplies at a time (bounds the scratch it needs for them)
+constexpr int64_t kEmbedGatherRows = 32768;
 
-int convert_f32_to_bf16_launch(const float* src, bf16* dst, int64_t n, cudaStream_t st) {
-    if (n > 0) f32_to_bf16_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(src, dst, n);
-    return launch_status();
-}
 
 // Split-K factor of a tensor-core weight-gradient product: one block per SM.
 static int64_t tc_split(int64_t M, int64_t N, int64_t K) {
@@ -484,7 +476,7 @@ extern "C" size_t retexo_embed_workspace_size_norm(int32_t d_in, int32_t hidden,
     s.take<bf16>(out1 * (size_t)pad_ld(d_in));                                   // W1^T
     s.take<bf16>(hidden > 0 ? (size_t)n_classes * pad_ld(hidden) : 1);           // W2^T
     s.take<bf16>(hidden > 0 ? (size_t)hidden * pad_ld(n_classes) : 1);           // W2 padded (unused here)
-    s.take<bf16>((size_t)retexo_theta_size(d_in, hidden, n_classes));               // row-major bf16 theta
+    s.take<bf16>((size_t)(n_rows < kEmbedGatherRows ? n_rows : kEmbedGatherRows) * pad_ld(d_in));   // gathered rows, a chunk
     s.take<bf16>(hidden > 0 ? (size_t)n_rows * pad_ld(hidden) : 1);              // Hd
     s.take<float>((size_t)n_rows * n_classes);                                      // logits
     s.take<int32_t>(64);
@@ -517,7 +509,7 @@ extern "C" int retexo_embed(const retexo_mlp* model, const void* x, int64_t ldx,
     b.w1t16 = ws.take<bf16>((size_t)out1 * p.ld_k);
     b.w2t16 = ws.take<bf16>(H > 0 ? (size_t)O * p.ld_h : 1);
     b.w2p16 = ws.take<bf16>(H > 0 ? (size_t)H * p.ld_dl : 1);
-    bf16* theta16 = ws.take<bf16>((size_t)p.nt);
+    bf16* xg = ws.take<bf16>((size_t)(n_rows < kEmbedGatherRows ? n_rows : kEmbedGatherRows) * p.ld_k);      // gathered rows, a chunk
     b.hd16 = ws.take<bf16>(H > 0 ? (size_t)n_rows * p.ld_h : 1);
     b.logits = ws.take<float>((size_t)n_rows * O);
     b.status = ws.take<int32_t>(64);
@@ -531,81 +523,58 @@ extern "C" int retexo_embed(const retexo_mlp* model, const void* x, int64_t ldx,
     const float* b1 = theta + (int64_t)d_in * out1;
     const float* b2 = b1 + out1 + (int64_t)H * O;
     const bool want_logits = logits_out || pred_out || correct;
-    float* lg = logits_out ? logits_out : b.logits;
-    const int64_t ld_lg = logits_out ? ld_logits : O;
 
-    if (row_idx) {
-        // gathered rows: CUDA-core products straight from the caller's matrix
-        RETEXO_TRY(convert_f32_to_bf16_launch(theta, theta16, p.nt, st));
-        const bf16* w1 = theta16;
-        const bf16* w2 = theta16 + (int64_t)d_in * out1 + out1;
-        GemmArgs g{};
-        g.M = n_rows; g.K = d_in; g.A = static_cast<const bf16*>(x); g.lda = ldx; g.a_row_idx = row_idx;
-        if (H > 0) {
-            bf16* h16 = hidden_out_bf16 ? static_cast<bf16*>(hidden_out_bf16) : b.hd16;
-            const int64_t ld16 = hidden_out_bf16 ? ld_hidden_bf16 : p.ld_h;
-            g.N = H; g.B = w1; g.ldb = H; g.bias = b1;
-            if (ln) {
-                g.out_f32 = z_ws; g.ld_f32 = H;
-                RETEXO_TRY(launch_gemm(g, st));
-                RETEXO_TRY(normalise_rows(model, z_ws, n_rows, (want_logits || hidden_out_bf16) ? h16 : nullptr, ld16,
-                                          hidden_out, ld_hidden, st));
-            } else {
-                g.relu = 1;
-                g.out_f32 = hidden_out; g.ld_f32 = ld_hidden;
-                g.out_bf16 = (want_logits || hidden_out_bf16) ? h16 : nullptr; g.ld_bf16 = ld16;
-                RETEXO_TRY(launch_gemm(g, st));
-            }
-            if (want_logits) {
-                GemmArgs g2{};
-                g2.M = n_rows; g2.N = O; g2.K = H; g2.A = h16; g2.lda = ld16; g2.B = w2; g2.ldb = O;
-                g2.bias = b2; g2.out_f32 = lg; g2.ld_f32 = ld_lg;
-                RETEXO_TRY(launch_gemm(g2, st));
-            }
-        } else if (want_logits) {
-            g.N = O; g.B = w1; g.ldb = O; g.bias = b1; g.out_f32 = lg; g.ld_f32 = ld_lg;
-            RETEXO_TRY(launch_gemm(g, st));
-        }
-    } else {
-        RETEXO_TRY(build_weight_shadows(p, b, theta, st));
-        TcGemm fwd = tc_base(static_cast<const bf16*>(x), ldx, b.w1t16, p.ld_k, n_rows, out1, d_in, b.status);
+    RETEXO_TRY(build_weight_shadows(p, b, theta, st));
+    // One pass of the tensor-core path over `rows` dense rows xd; `off` is their position in the outputs.
+    auto dense = [&](const bf16* xd, int64_t ldxd, int64_t rows, int64_t off) -> int {
+        float* hid = hidden_out ? hidden_out + off * ld_hidden : nullptr;
+        bf16* hid16 = hidden_out_bf16 ? static_cast<bf16*>(hidden_out_bf16) + off * ld_hidden_bf16 : nullptr;
+        float* lgo = logits_out ? logits_out + off * ld_logits : nullptr;
+        int32_t* pred = pred_out ? pred_out + off : nullptr;
+        const int32_t* yy = y ? y + off : nullptr;
+        TcGemm fwd = tc_base(xd, ldxd, b.w1t16, p.ld_k, rows, out1, d_in, b.status);
         fwd.bias = b1;
         if (H > 0) {
             // the logits product reads Hd through TMA, so it wants an aligned copy with a stride of 8 elements
-            const bool user16_ok = hidden_out_bf16 && aligned_to(hidden_out_bf16, 16) && ld_hidden_bf16 % 8 == 0;
-            bf16* h16 = user16_ok ? static_cast<bf16*>(hidden_out_bf16) : b.hd16;
+            const bool user16_ok = hid16 && aligned_to(hid16, 16) && ld_hidden_bf16 % 8 == 0;
+            bf16* h16 = user16_ok ? hid16 : b.hd16 + off * p.ld_h;
             const int64_t ld16 = user16_ok ? ld_hidden_bf16 : p.ld_h;
             if (ln) {
-                fwd.out_f32 = z_ws; fwd.ld_f32 = H;
+                float* z = z_ws + off * H;
+                fwd.out_f32 = z; fwd.ld_f32 = H;
                 RETEXO_TRY(tc_gemm_launch(fwd, st));
-                RETEXO_TRY(normalise_rows(model, z_ws, n_rows, (want_logits || user16_ok) ? h16 : nullptr, ld16, hidden_out,
-                                          ld_hidden, st));
+                RETEXO_TRY(normalise_rows(model, z, rows, (want_logits || hid16) ? h16 : nullptr, ld16, hid, ld_hidden, st));
             } else {
-                fwd.relu = 1; fwd.out_f32 = hidden_out; fwd.ld_f32 = ld_hidden;
-                fwd.out_bf16 = (want_logits || user16_ok) ? h16 : nullptr; fwd.ld_bf16 = ld16;
+                fwd.relu = 1; fwd.out_f32 = hid; fwd.ld_f32 = ld_hidden;
+                fwd.out_bf16 = (want_logits || hid16) ? h16 : nullptr; fwd.ld_bf16 = ld16;
                 RETEXO_TRY(tc_gemm_launch(fwd, st));
             }
-            if (hidden_out_bf16 && !user16_ok)      // odd layout asked for: a second, plain copy
-                RETEXO_TRY(retexo_pack_rows(hidden_out ? (const void*)hidden_out : (const void*)b.hd16,
-                                            hidden_out ? 0 : 1, hidden_out ? ld_hidden : p.ld_h, H, nullptr, n_rows,
-                                            hidden_out_bf16, ld_hidden_bf16, nullptr, 0, 0, st));
+            if (hid16 && !user16_ok)      // odd layout asked for: a second, plain copy
+                RETEXO_TRY(retexo_pack_rows(hid ? (const void*)hid : (const void*)h16, hid ? 0 : 1, hid ? ld_hidden : p.ld_h, H,
+                                            nullptr, rows, hid16, ld_hidden_bf16, nullptr, 0, 0, st));
             if (want_logits) {
-                TcGemm l2 = tc_base(h16, ld16, b.w2t16, p.ld_h, n_rows, O, H, b.status);
-                l2.bias = b2; l2.mode = TC_EPI_ARGMAX; l2.out_f32 = logits_out; l2.ld_f32 = ld_logits;
-                l2.pred = pred_out; l2.y = y; l2.correct = correct;
+                TcGemm l2 = tc_base(h16, ld16, b.w2t16, p.ld_h, rows, O, H, b.status);
+                l2.bias = b2; l2.mode = TC_EPI_ARGMAX; l2.out_f32 = lgo; l2.ld_f32 = ld_logits;
+                l2.pred = pred; l2.y = yy; l2.correct = correct;
                 RETEXO_TRY(tc_gemm_launch(l2, st));
             }
         } else if (want_logits) {
-            fwd.mode = TC_EPI_ARGMAX; fwd.out_f32 = logits_out; fwd.ld_f32 = ld_logits;
-            fwd.pred = pred_out; fwd.y = y; fwd.correct = correct;
+            fwd.mode = TC_EPI_ARGMAX; fwd.out_f32 = lgo; fwd.ld_f32 = ld_logits;
+            fwd.pred = pred; fwd.y = yy; fwd.correct = correct;
             RETEXO_TRY(tc_gemm_launch(fwd, st));
         }
-        if (model->status_out)
-            RETEXO_CUDA_TRY(cudaMemcpyAsync(model->status_out, b.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
-        return launch_status();
+        return RETEXO_OK;
+    };
+    if (row_idx) {
+        // gathered rows: packed into a dense batch a chunk at a time, so that these products run on the tensor cores too
+        for (int64_t off = 0; off < n_rows; off += kEmbedGatherRows) {
+            const int64_t rows = n_rows - off < kEmbedGatherRows ? n_rows - off : kEmbedGatherRows;
+            RETEXO_TRY(retexo_pack_rows(x, 1, ldx, d_in, row_idx + off, rows, xg, p.ld_k, nullptr, 0, 0, st));
+            RETEXO_TRY(dense(xg, p.ld_k, rows, off));
+        }
+    } else {
+        RETEXO_TRY(dense(static_cast<const bf16*>(x), ldx, n_rows, 0));
     }
-    if (pred_out || correct)
-        argmax_kernel<<<(unsigned)((n_rows + 255) / 256), 256, 0, st>>>(lg, ld_lg, n_rows, O, pred_out, y, correct);
     if (model->status_out)
         RETEXO_CUDA_TRY(cudaMemcpyAsync(model->status_out, b.status, sizeof(int32_t), cudaMemcpyDeviceToDevice, st));
     return launch_status();

@@ -1,7 +1,4 @@
-// Kernels of the per-node model (Section 3.1): batch packing, a general
-// CUDA-core bf16 GEMM with fused epilogues (used for the skinny products and
-// as the path for shapes the tensor-core kernel does not take), softmax
-// cross-entropy with its gradient, arg-max/accuracy, and the fused
+// Kernels of the per-node model (Section 3.1) beside its tensor-core products: batch packing and the fused
 // gradient-reduce + optimiser update.
 #pragma once
 #include "common.cuh"
@@ -46,155 +43,6 @@ __global__ void __launch_bounds__(256) pack_rows_kernel(const void* __restrict__
     if (ones && blockIdx.y == 0 && ty == 0) {
         const int64_t r = r0 + tx;
         if (r < ld_t) dst_t[(int64_t)dim * ld_t + r] = f32_to_bf16(r < n_rows ? 1.0f : 0.0f);
-    }
-}
-
-// ---------------------------------------------------------------- GEMM
-constexpr int kBM = 64, kBN = 64, kBK = 32, kGemmThreads = 256;
-
-struct GemmArgs {
-    int64_t M, N, K;
-    const bf16* A; int64_t lda;            // [M x K], row-major
-    const int32_t* a_row_idx;              // optional row gather for A
-    const bf16* B; int64_t ldb;            // [K x N], row-major
-    int relu;
-    const float* bias;                     // [N] (may be null)
-    float* out_f32; int64_t ld_f32;        // (may be null)
-    bf16* out_bf16; int64_t ld_bf16;       // (may be null)
-};
-
-// out = A B (+ bias) (ReLU), bf16 operands, fp32 accumulation on the CUDA cores.
-// Takes what the tensor-core kernel cannot: gathered rows and operands that
-// break the TMA alignment rules.
-__global__ void __launch_bounds__(kGemmThreads) gemm_bf16_kernel(GemmArgs g) {
-    __shared__ __align__(16) float As[kBK][kBM + 4];
-    __shared__ __align__(16) float Bs[kBK][kBN + 4];
-    const int t = threadIdx.x, tx = t & 15, ty = t >> 4;
-    const int64_t m0 = blockIdx.y * (int64_t)kBM, n0 = blockIdx.x * (int64_t)kBN;
-    float acc[4][4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i)
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-
-    for (int64_t k0 = 0; k0 < g.K; k0 += kBK) {
-#pragma unroll
-        for (int i = 0; i < (kBM * kBK) / kGemmThreads; ++i) {
-            const int e = t + i * kGemmThreads;
-            const int m = e / kBK, k = e % kBK;
-            const int64_t gm = m0 + m, gk = k0 + k;
-            float v = 0.f;
-            if (gm < g.M && gk < g.K) {
-                const int64_t r = g.a_row_idx ? g.a_row_idx[gm] : gm;
-                v = bf16_to_f32(g.A[r * g.lda + gk]);
-            }
-            As[k][m] = v;
-        }
-#pragma unroll
-        for (int i = 0; i < (kBN * kBK) / kGemmThreads; ++i) {
-            const int e = t + i * kGemmThreads;
-            const int k = e / kBN, n = e % kBN;
-            const int64_t gn = n0 + n, gk = k0 + k;
-            float v = 0.f;
-            if (gn < g.N && gk < g.K) v = bf16_to_f32(g.B[gk * g.ldb + gn]);
-            Bs[k][n] = v;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < kBK; ++k) {
-            const float4 a = *reinterpret_cast<const float4*>(&As[k][ty * 4]);
-            const float4 b = *reinterpret_cast<const float4*>(&Bs[k][tx * 4]);
-            const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int64_t m = m0 + ty * 4 + i;
-        if (m >= g.M) continue;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int64_t n = n0 + tx * 4 + j;
-            if (n >= g.N) continue;
-            float v = acc[i][j] + (g.bias ? g.bias[n] : 0.f);
-            if (g.relu) v = fmaxf(v, 0.f);
-            if (g.out_f32) g.out_f32[m * g.ld_f32 + n] = v;
-            if (g.out_bf16) g.out_bf16[m * g.ld_bf16 + n] = f32_to_bf16(v);
-        }
-    }
-}
-
-// ---------------------------------------------------------------- softmax CE
-// One warp per row (n_classes <= 64).  Writes dL = (softmax - onehot)/n_rows as
-// bf16, row-major (row stride ld_dl, padding columns zero) and transposed
-// (dl_t [n_classes x ld_t]), and per-block partial sums of the loss.
-constexpr int kSmThreads = 256;
-__global__ void __launch_bounds__(kSmThreads) softmax_ce_kernel(const float* __restrict__ logits, int64_t ld_logits,
-                                                                const int32_t* __restrict__ y, int64_t n_rows,
-                                                                int32_t n_classes, bf16* __restrict__ dl, int64_t ld_dl,
-                                                                bf16* __restrict__ dl_t, int64_t ld_t,
-                                                                float* __restrict__ loss_partial) {
-    __shared__ float s_loss[kSmThreads / kWarp];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float inv_n = 1.0f / (float)n_rows;
-    float my_loss = 0.f;
-    const int64_t stride = (int64_t)gridDim.x * (kSmThreads / kWarp);
-    for (int64_t r = blockIdx.x * (int64_t)(kSmThreads / kWarp) + warp; r < n_rows; r += stride) {
-        const float* row = logits + r * ld_logits;
-        const float l0 = lane < n_classes ? row[lane] : -INFINITY;
-        const float l1 = lane + 32 < n_classes ? row[lane + 32] : -INFINITY;
-        const float mx = warp_max(fmaxf(l0, l1));
-        const float e0 = lane < n_classes ? expf(l0 - mx) : 0.f;
-        const float e1 = lane + 32 < n_classes ? expf(l1 - mx) : 0.f;
-        const float den = warp_sum(e0 + e1);
-        const int32_t yi = y[r];
-        const float ly = __shfl_sync(0xffffffffu, (yi & 32) ? l1 : l0, yi & 31);
-        my_loss += (mx + logf(den)) - ly;
-        const float g0 = (e0 / den - (lane == yi ? 1.f : 0.f)) * inv_n;
-        const float g1 = (e1 / den - (lane + 32 == yi ? 1.f : 0.f)) * inv_n;
-        if (dl) {
-            if (lane < ld_dl) dl[r * ld_dl + lane] = f32_to_bf16(lane < n_classes ? g0 : 0.f);
-            if (lane + 32 < ld_dl) dl[r * ld_dl + lane + 32] = f32_to_bf16(lane + 32 < n_classes ? g1 : 0.f);
-        }
-        if (dl_t) {
-            if (lane < n_classes) dl_t[(int64_t)lane * ld_t + r] = f32_to_bf16(g0);
-            if (lane + 32 < n_classes) dl_t[(int64_t)(lane + 32) * ld_t + r] = f32_to_bf16(g1);
-        }
-    }
-    if (lane == 0) s_loss[warp] = my_loss;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        float s = 0.f;
-        for (int w = 0; w < kSmThreads / kWarp; ++w) s += s_loss[w];
-        loss_partial[blockIdx.x] = s;
-    }
-}
-
-// ---------------------------------------------------------------- arg-max / accuracy
-__global__ void __launch_bounds__(256) argmax_kernel(const float* __restrict__ logits, int64_t ld, int64_t n_rows,
-                                                     int32_t n_classes, int32_t* __restrict__ pred,
-                                                     const int32_t* __restrict__ y,
-                                                     unsigned long long* __restrict__ correct) {
-    const int64_t r = blockIdx.x * 256ll + threadIdx.x;
-    int hit = 0;
-    if (r < n_rows) {
-        const float* row = logits + r * ld;
-        int best = 0;
-        float bv = row[0];
-        for (int c = 1; c < n_classes; ++c) {
-            const float v = row[c];
-            if (v > bv) { bv = v; best = c; }       // strict: lowest index wins ties
-        }
-        if (pred) pred[r] = best;
-        if (y && best == y[r]) hit = 1;
-    }
-    if (correct) {
-        const unsigned b = __ballot_sync(0xffffffffu, hit);
-        if ((threadIdx.x & 31) == 0 && b) atomicAdd(correct, (unsigned long long)__popc(b));
     }
 }
 
@@ -398,11 +246,6 @@ __global__ void __launch_bounds__(256, BATCH == 16 ? 4 : 2) reduce_update_kernel
         if (trow < rows - 1 && tcol < cols)
             wt[(int64_t)tcol * (sidx == 0 ? u.ld_k : u.ld_h) + trow] = tile16[threadIdx.x & 15][threadIdx.x >> 4];
     }
-}
-
-__global__ void __launch_bounds__(256) f32_to_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int64_t n) {
-    const int64_t i = blockIdx.x * 256ll + threadIdx.x;
-    if (i < n) dst[i] = f32_to_bf16(src[i]);
 }
 
 }  // namespace retexo

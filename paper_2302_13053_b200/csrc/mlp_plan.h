@@ -130,6 +130,5 @@ int linear_update_launch(int32_t d_in, int32_t out, float* theta, float* adam_m,
 int linear_shadows_launch(int32_t d_in, int32_t out, const float* theta, __nv_bfloat16* wt16, int64_t ld_k,
                           __nv_bfloat16* wr16, int64_t ld_o1, cudaStream_t st);
 
-int convert_f32_to_bf16_launch(const float* src, __nv_bfloat16* dst, int64_t n, cudaStream_t st);
 
 }  // namespace retexo
