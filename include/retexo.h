@@ -128,7 +128,7 @@ int retexo_aggregate(const retexo_csr* g, int32_t type,
                      void* out_bf16, int64_t ldout_bf16,
                      void* workspace, size_t workspace_bytes, void* stream);
 
-size_t retexo_gat_backward_workspace_size(int64_t n_nodes, int32_t heads, int32_t dim);
+size_t retexo_gat_backward_workspace_size(int64_t n_nodes, int64_t n_edges, int32_t heads, int32_t dim);
 
 /* Backward of RETEXO_GAT, for rounds that train the aggregator as well (Section 2.2: "AGGR may have
  * trainable parameters"; Section 3.1: a round trains the whole layer): given dz = dLoss / dOut

@@ -213,7 +213,7 @@ def retexo_gat_backward(rowptr: torch.Tensor, colidx: torch.Tensor, p: torch.Ten
     da_src = torch.empty((heads, dh), dtype=torch.float32, device=dev)
     da_dst = torch.empty((heads, dh), dtype=torch.float32, device=dev)
     g = _csr(rowptr, colidx)
-    need = lib().retexo_gat_backward_workspace_size(C.c_int64(n), C.c_int32(heads), C.c_int32(dim))
+    need = lib().retexo_gat_backward_workspace_size(C.c_int64(n), C.c_int64(colidx.numel()), C.c_int32(heads), C.c_int32(dim))
     ws = _workspace(need, dev)
     rc = lib().retexo_gat_backward(C.byref(g), _ptr(p), C.c_int64(p.stride(0) if n > 0 else dim), C.byref(gp), _ptr(dz),
                                    C.c_int64(dz.stride(0) if n > 0 else dim), _ptr(dp), C.c_int64(dim), _ptr(dp16),

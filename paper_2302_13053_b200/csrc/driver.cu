@@ -244,7 +244,7 @@ static void lmp_layout(const retexo_lmp_config& c, int64_t n, int64_t e, int64_t
         l.dp16 = t.template take<bf16>((size_t)n * round_up(hd, 64));
         l.decision = t.template take<int32_t>(64);
         l.status = t.template take<int32_t>(64);
-        l.ws_gatbwd_bytes = retexo_gat_backward_workspace_size(n, c.gat_heads, hd);
+        l.ws_gatbwd_bytes = retexo_gat_backward_workspace_size(n, e, c.gat_heads, hd);
         l.ws_gatbwd = t.template take<char>(l.ws_gatbwd_bytes);
     }
     // training rows, then validation rows, each followed by a column of ones (it carries the bias gradient

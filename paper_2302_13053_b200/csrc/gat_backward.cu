@@ -30,7 +30,14 @@ struct GatBwdArgs {
     float* dp; int64_t lddp;
     __nv_bfloat16* dp16; int64_t lddp16;
     float* partial;                  // [blocks x 2 x dim]: per-block sums of ds_u p_u and dt_u p_u
+    // rows of kGbHubEntries entries or more ("hub rows") are listed by the score kernel and taken by whole blocks
+    int32_t* hub_count; int32_t* hub_list;      // how many, which (in the order the score kernel met them)
+    int32_t* hub_pos;                           // [n]: position in the list, -1 for every other row
+    float* hub_sum;                             // [hubs x 72]: per hub row the 64 column sums of its source pass, then ds per head
 };
+
+constexpr int kGbHubEntries = 128;   // a warp takes 32 entries per trip: rows this long keep one warp busy while the grid drains
+constexpr int kGbHubBlocks = 296;    // blocks of the hub kernels (they loop over the list)
 
 __global__ void __launch_bounds__(kGbThreads) gat_bwd_scores_kernel(GatBwdArgs a) {
     const int lane = threadIdx.x & 31;
@@ -47,6 +54,15 @@ __global__ void __launch_bounds__(kGbThreads) gat_bwd_scores_kernel(GatBwdArgs a
         ss = warp_sum(ss);
         tt = warp_sum(tt);
         if (lane == 0) { a.s[u * a.heads + h] = ss; a.t[u * a.heads + h] = tt; }
+    }
+    if (a.hub_pos && lane == 0) {
+        const int64_t total = a.rowptr[u + 1] - a.rowptr[u] + (a.self_loop ? 1 : 0);
+        int32_t pos = -1;
+        if (total >= kGbHubEntries) {      // (the list's order varies from run to run; no result depends on it)
+            pos = atomicAdd(a.hub_count, 1);
+            a.hub_list[pos] = (int32_t)u;
+        }
+        a.hub_pos[u] = pos;
     }
 }
 
@@ -261,6 +277,7 @@ __global__ void __launch_bounds__(kGb64Threads) gat_bwd_dst64_kernel(GatBwdArgs 
     const int64_t beg = a.rowptr[v];
     const int64_t deg = a.rowptr[v + 1] - beg;
     const int64_t total = deg + (a.self_loop ? 1 : 0);
+    if (total >= kGbHubEntries) return;             // a hub row: gat_bwd_dst64_hub_kernel's
     if (!__any_sync(0xffffffffu, any) || total == 0) {
         if (lane < a.heads) a.stats[v * a.heads + lane] = make_float4(0.f, 0.f, 0.f, 0.f);
         return;
@@ -344,7 +361,17 @@ __global__ void __launch_bounds__(kGb64Threads) gat_bwd_src64_kernel(GatBwdArgs 
         for (int h = 0; h < NH; ++h) if (h < a.heads) su[h] = a.s[u * a.heads + h];
         const int64_t beg = a.rowptr[u];
         const int64_t deg = a.rowptr[u + 1] - beg;
-        const int64_t total = deg + (a.self_loop ? 1 : 0);
+        int64_t total = deg + (a.self_loop ? 1 : 0);
+        if (total >= kGbHubEntries) {               // a hub row: its sums come from gat_bwd_src64_hub_kernel
+            const float* hs = a.hub_sum + (int64_t)a.hub_pos[u] * 72;
+            if (lane == 0) {
+#pragma unroll
+                for (int c = 0; c < 64; ++c) acc[c] = hs[c];
+#pragma unroll
+                for (int h = 0; h < NH; ++h) ds[h] = hs[64 + h];
+            }
+            total = 0;
+        }
         for (int64_t e0 = 0; e0 < total; e0 += kWarp) {
             const bool valid = e0 + lane < total;
             const int64_t v = !valid ? u : (e0 + lane < deg ? (int64_t)__ldg(a.colidx + beg + e0 + lane) : u);
@@ -411,10 +438,204 @@ __global__ void __launch_bounds__(kGb64Threads) gat_bwd_src64_kernel(GatBwdArgs 
     }
 }
 
+// ---- hub rows: one block per listed row, its warps taking the trips w, w + W, ...; per-warp results are merged in
+// warp order, so the bits depend neither on timing nor on the list's order.
+constexpr int kGbHubWarps = 8, kGbHubThreads = kGbHubWarps * kWarp;
+
+template <int HD>
+__global__ void __launch_bounds__(kGbHubThreads) gat_bwd_dst64_hub_kernel(GatBwdArgs a) {
+    constexpr int NH = 64 / HD;
+    __shared__ __align__(16) float g_s[64];
+    __shared__ float st_m[kGbHubWarps][NH], st_den[kGbHubWarps][NH], part[kGbHubWarps][NH][3];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nv = a.dim >> 2;
+    const int32_t count = *a.hub_count;
+    for (int32_t item = blockIdx.x; item < count; item += gridDim.x) {
+        const int64_t v = a.hub_list[item];
+        __syncthreads();                                 // the previous row's shared values are done with
+        bool any = false;
+        if (threadIdx.x < 64) {
+            const float x = (int)threadIdx.x < a.dim ? a.dz[v * a.lddz + threadIdx.x] : 0.f;
+            g_s[threadIdx.x] = x;
+            any = x != 0.f;
+        }
+        if (!__syncthreads_or(any)) {
+            if ((int)threadIdx.x < a.heads) a.stats[v * a.heads + threadIdx.x] = make_float4(0.f, 0.f, 0.f, 0.f);
+            continue;
+        }
+        const int64_t beg = a.rowptr[v];
+        const int64_t deg = a.rowptr[v + 1] - beg;
+        const int64_t total = deg + (a.self_loop ? 1 : 0);
+        float tv[NH], m[NH], den[NH], csum[NH], a1[NH], a2[NH];
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+            tv[h] = h < a.heads ? a.t[v * a.heads + h] : 0.f;
+            m[h] = -INFINITY; den[h] = 0.f; csum[h] = 0.f; a1[h] = 0.f; a2[h] = 0.f;
+        }
+        for (int64_t e0 = (int64_t)warp * kWarp; e0 < total; e0 += kGbHubThreads) {
+            const bool valid = e0 + lane < total;
+            const int64_t u = !valid ? v : (e0 + lane < deg ? (int64_t)__ldg(a.colidx + beg + e0 + lane) : v);
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+                if (h < a.heads) {
+                    const float z = a.s[u * a.heads + h] + tv[h];
+                    const float e = valid ? (z > 0.f ? z : a.slope * z) : -INFINITY;
+                    const float mn = fmaxf(m[h], warp_max(e));
+                    den[h] = den[h] * expf(m[h] - mn) + warp_sum(valid ? expf(e - mn) : 0.f);
+                    m[h] = mn;
+                }
+            }
+        }
+        if (lane == 0) {
+#pragma unroll
+            for (int h = 0; h < NH; ++h) { st_m[warp][h] = m[h]; st_den[warp][h] = den[h]; }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {                   // every thread merges the warps' states in warp order
+            float mm = -INFINITY, dd = 0.f;
+            for (int w = 0; w < kGbHubWarps; ++w) mm = fmaxf(mm, st_m[w][h]);
+            for (int w = 0; w < kGbHubWarps; ++w)
+                if (st_den[w][h] > 0.f) dd += st_den[w][h] * expf(st_m[w][h] - mm);
+            m[h] = mm; den[h] = dd;
+        }
+        for (int64_t e0 = (int64_t)warp * kWarp; e0 < total; e0 += kGbHubThreads) {
+            const bool valid = e0 + lane < total;
+            const int64_t u = !valid ? v : (e0 + lane < deg ? (int64_t)__ldg(a.colidx + beg + e0 + lane) : v);
+            float dalpha[NH];
+#pragma unroll
+            for (int h = 0; h < NH; ++h) dalpha[h] = 0.f;
+            const float4* row = reinterpret_cast<const float4*>(a.p + u * a.ldp);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                if (i < nv) {
+                    const float4 x = valid ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                    const float4 gg = *reinterpret_cast<const float4*>(&g_s[4 * i]);
+                    dalpha[(4 * i) / HD] += (x.x * gg.x + x.y * gg.y) + (x.z * gg.z + x.w * gg.w);
+                }
+            }
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+                if (h < a.heads && valid) {
+                    const float z = a.s[u * a.heads + h] + tv[h];
+                    const float alpha = expf((z > 0.f ? z : a.slope * z) - m[h]) / den[h];
+                    const float gp = z > 0.f ? 1.f : a.slope;
+                    csum[h] = fmaf(alpha, dalpha[h], csum[h]);
+                    a1[h] = fmaf(alpha * gp, dalpha[h], a1[h]);
+                    a2[h] = fmaf(alpha, gp, a2[h]);
+                }
+            }
+        }
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+            const float c = warp_sum(csum[h]), s1 = warp_sum(a1[h]), s2 = warp_sum(a2[h]);
+            if (lane == 0) { part[warp][h][0] = c; part[warp][h][1] = s1; part[warp][h][2] = s2; }
+        }
+        __syncthreads();
+        if ((int)threadIdx.x < a.heads && (int)threadIdx.x < NH) {
+            const int h = threadIdx.x;
+            float c = 0.f, s1 = 0.f, s2 = 0.f, mm = -INFINITY, dd = 0.f;
+            for (int w = 0; w < kGbHubWarps; ++w) { c += part[w][h][0]; s1 += part[w][h][1]; s2 += part[w][h][2]; }
+            for (int w = 0; w < kGbHubWarps; ++w) mm = fmaxf(mm, st_m[w][h]);
+            for (int w = 0; w < kGbHubWarps; ++w)
+                if (st_den[w][h] > 0.f) dd += st_den[w][h] * expf(st_m[w][h] - mm);
+            a.stats[v * a.heads + h] = make_float4(mm, 1.f / dd, c, s1 - c * s2);
+        }
+    }
+}
+
+// The source pass of a hub row u: the entry sums only (sum_v alpha_uv dz_v per column and ds_u per head); the row's
+// own epilogue (dp_u, the parameter-gradient partials) stays with gat_bwd_src64_kernel, which picks the sums up.
+template <int HD>
+__global__ void __launch_bounds__(kGb64Threads) gat_bwd_src64_hub_kernel(GatBwdArgs a) {
+    constexpr int NH = 64 / HD;
+    __shared__ __align__(16) float p_s[64];
+    __shared__ float red[kGb64Warps][kWarp][65];
+    __shared__ float rows[kGb64Warps][64], dsw[kGb64Warps][NH];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nv = a.dim >> 2;
+    const int32_t count = *a.hub_count;
+    for (int32_t item = blockIdx.x; item < count; item += gridDim.x) {
+        const int64_t u = a.hub_list[item];
+        __syncthreads();
+        if (threadIdx.x < 64) p_s[threadIdx.x] = (int)threadIdx.x < a.dim ? a.p[u * a.ldp + threadIdx.x] : 0.f;
+        __syncthreads();
+        float acc[64], ds[NH], su[NH];
+#pragma unroll
+        for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+#pragma unroll
+        for (int h = 0; h < NH; ++h) { ds[h] = 0.f; su[h] = h < a.heads ? a.s[u * a.heads + h] : 0.f; }
+        const int64_t beg = a.rowptr[u];
+        const int64_t deg = a.rowptr[u + 1] - beg;
+        const int64_t total = deg + (a.self_loop ? 1 : 0);
+        for (int64_t e0 = (int64_t)warp * kWarp; e0 < total; e0 += kGb64Threads) {
+            const bool valid = e0 + lane < total;
+            const int64_t v = !valid ? u : (e0 + lane < deg ? (int64_t)__ldg(a.colidx + beg + e0 + lane) : u);
+            const bool live = valid && a.stats[v * a.heads].y != 0.f;      // dz_v is zero otherwise
+            float4 g[16];
+            float dalpha[NH], alpha[NH];
+#pragma unroll
+            for (int h = 0; h < NH; ++h) { dalpha[h] = 0.f; alpha[h] = 0.f; }
+            const float4* row = reinterpret_cast<const float4*>(a.dz + v * a.lddz);
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                g[i] = (live && i < nv) ? __ldg(row + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+                const float4 pp = *reinterpret_cast<const float4*>(&p_s[4 * i]);
+                dalpha[(4 * i) / HD] += (g[i].x * pp.x + g[i].y * pp.y) + (g[i].z * pp.z + g[i].w * pp.w);
+            }
+#pragma unroll
+            for (int h = 0; h < NH; ++h) {
+                if (h < a.heads && live) {
+                    const float4 st = a.stats[v * a.heads + h];
+                    const float z = su[h] + a.t[v * a.heads + h];
+                    alpha[h] = expf((z > 0.f ? z : a.slope * z) - st.x) * st.y;
+                    ds[h] = fmaf(alpha[h] * (z > 0.f ? 1.f : a.slope), dalpha[h] - st.z, ds[h]);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const float al = alpha[(4 * i) / HD];
+                acc[4 * i] = fmaf(al, g[i].x, acc[4 * i]);
+                acc[4 * i + 1] = fmaf(al, g[i].y, acc[4 * i + 1]);
+                acc[4 * i + 2] = fmaf(al, g[i].z, acc[4 * i + 2]);
+                acc[4 * i + 3] = fmaf(al, g[i].w, acc[4 * i + 3]);
+            }
+        }
+        // lanes in lane order, then warps in warp order
+#pragma unroll
+        for (int c = 0; c < 64; ++c) red[warp][lane][c] = acc[c];
+#pragma unroll
+        for (int h = 0; h < NH; ++h) {
+            const float d = warp_sum(ds[h]);
+            if (lane == 0) dsw[warp][h] = d;
+        }
+        __syncwarp();
+        for (int c = lane; c < 64; c += kWarp) {
+            float sum = 0.f;
+            for (int l = 0; l < kWarp; ++l) sum += red[warp][l][c];
+            rows[warp][c] = sum;
+        }
+        __syncthreads();
+        float* hs = a.hub_sum + (int64_t)item * 72;
+        if (threadIdx.x < 64) {
+            float sum = 0.f;
+            for (int w = 0; w < kGb64Warps; ++w) sum += rows[w][threadIdx.x];
+            hs[threadIdx.x] = sum;
+        } else if ((int)threadIdx.x - 64 < NH) {
+            const int h = threadIdx.x - 64;
+            float sum = 0.f;
+            for (int w = 0; w < kGb64Warps; ++w) sum += dsw[w][h];
+            hs[64 + h] = sum;
+        }
+    }
+}
+
 template <int HD>
 static int launch_bwd64(const GatBwdArgs& a, float* da_src, float* da_dst, cudaStream_t st) {
     const unsigned blocks = (unsigned)((a.n + kGb64Warps - 1) / kGb64Warps);
     gat_bwd_dst64_kernel<HD><<<blocks, kGb64Threads, 0, st>>>(a);
+    gat_bwd_dst64_hub_kernel<HD><<<kGbHubBlocks, kGbHubThreads, 0, st>>>(a);
+    gat_bwd_src64_hub_kernel<HD><<<kGbHubBlocks, kGb64Threads, 0, st>>>(a);
     gat_bwd_src64_kernel<HD><<<blocks, kGb64Threads, 0, st>>>(a);
     gat_bwd_reduce_kernel<<<(unsigned)(2 * a.dim), 256, 0, st>>>(a.partial, blocks, a.dim, da_src, da_dst);
     return launch_status();
@@ -432,13 +653,20 @@ static int launch_bwd(const GatBwdArgs& a, unsigned blocks, float* da_src, float
 
 using namespace retexo;
 
-extern "C" size_t retexo_gat_backward_workspace_size(int64_t n_nodes, int32_t heads, int32_t dim) {
-    if (n_nodes < 0 || heads <= 0 || dim <= 0) return 0;
+// rows of kGbHubEntries entries or more a graph can hold at most (with the self loop counted as an entry)
+static inline int64_t max_hub_rows(int64_t n_nodes, int64_t n_edges) { return (n_edges + n_nodes) / kGbHubEntries + 1; }
+
+extern "C" size_t retexo_gat_backward_workspace_size(int64_t n_nodes, int64_t n_edges, int32_t heads, int32_t dim) {
+    if (n_nodes < 0 || n_edges < 0 || heads <= 0 || dim <= 0) return 0;
     Sizer s;
     s.take<float>((size_t)n_nodes * heads);
     s.take<float>((size_t)n_nodes * heads);
     s.take<float4>((size_t)n_nodes * heads);
     s.take<float>((size_t)((n_nodes + kGb64Warps - 1) / kGb64Warps + 1) * 2 * (size_t)dim);
+    s.take<int32_t>(64);
+    s.take<int32_t>((size_t)max_hub_rows(n_nodes, n_edges));
+    s.take<int32_t>((size_t)n_nodes);
+    s.take<float>((size_t)max_hub_rows(n_nodes, n_edges) * 72);
     return s.off + kAlign;
 }
 
@@ -459,7 +687,7 @@ extern "C" int retexo_gat_backward(const retexo_csr* g, const float* p, int64_t 
         return RETEXO_OK;
     }
     if (!g->rowptr || !p || !dz || (g->n_edges > 0 && !g->colidx)) return RETEXO_ERR_INVALID_ARG;
-    const size_t need = retexo_gat_backward_workspace_size(g->n_nodes, gat->heads, dim);
+    const size_t need = retexo_gat_backward_workspace_size(g->n_nodes, g->n_edges, gat->heads, dim);
     if (!workspace || !aligned_to(workspace, kAlign) || workspace_bytes < need) return RETEXO_ERR_WORKSPACE;
     const int64_t n = g->n_nodes;
     Arena ws(workspace, workspace_bytes);
@@ -474,11 +702,21 @@ extern "C" int retexo_gat_backward(const retexo_csr* g, const float* p, int64_t 
     const unsigned blocks = (unsigned)((n + kGbWarps - 1) / kGbWarps);
     a.partial = ws.take<float>((size_t)((n + kGb64Warps - 1) / kGb64Warps + 1) * 2 * (size_t)dim);
     a.dp = dp; a.lddp = lddp; a.dp16 = static_cast<__nv_bfloat16*>(dp_bf16); a.lddp16 = lddp_bf16;
-    gat_bwd_scores_kernel<<<blocks, kGbThreads, 0, st>>>(a);
-    // rows of up to 64 columns in whole 16-byte pieces, head width 8 / 16 / 32 / 64: one lane per entry
+    int32_t* hub_count = ws.take<int32_t>(64);
+    int32_t* hub_list = ws.take<int32_t>((size_t)max_hub_rows(n, g->n_edges));
+    int32_t* hub_pos = ws.take<int32_t>((size_t)n);
+    float* hub_sum = ws.take<float>((size_t)max_hub_rows(n, g->n_edges) * 72);
+    // rows of up to 64 columns in whole 16-byte pieces, head width 8 / 16 / 32 / 64: one lane per entry, hub rows by blocks
     const int hdw = gat->head_dim;
-    if (dim <= 64 && dim % 4 == 0 && ldp % 4 == 0 && lddz % 4 == 0 && aligned_to(p, 16) && aligned_to(dz, 16) &&
-        (hdw == 8 || hdw == 16 || hdw == 32 || hdw == 64)) {
+    const bool lane_per_entry = dim <= 64 && dim % 4 == 0 && ldp % 4 == 0 && lddz % 4 == 0 && aligned_to(p, 16) && aligned_to(dz, 16) &&
+                                (hdw == 8 || hdw == 16 || hdw == 32 || hdw == 64);
+    a.hub_count = nullptr; a.hub_list = nullptr; a.hub_pos = nullptr; a.hub_sum = nullptr;
+    if (lane_per_entry) {
+        a.hub_count = hub_count; a.hub_list = hub_list; a.hub_pos = hub_pos; a.hub_sum = hub_sum;
+        RETEXO_CUDA_TRY(cudaMemsetAsync(hub_count, 0, sizeof(int32_t), st));
+    }
+    gat_bwd_scores_kernel<<<blocks, kGbThreads, 0, st>>>(a);
+    if (lane_per_entry) {
         if (hdw == 8) return launch_bwd64<8>(a, da_src, da_dst, st);
         if (hdw == 16) return launch_bwd64<16>(a, da_src, da_dst, st);
         if (hdw == 32) return launch_bwd64<32>(a, da_src, da_dst, st);
