@@ -574,6 +574,8 @@ def main():
                     help="GAT workloads: keep the aggregator's parameters fixed (the round aggregates once)")
     ap.add_argument("--iteration-only", type=int, default=0, metavar="M",
                     help="run a dozen stand-alone training iterations of round M's model and exit (profiler captures)")
+    ap.add_argument("--standard-only", type=int, default=0, metavar="ITERS",
+                    help="run ITERS iterations of standard training twice and nothing else (profiler captures)")
     ap.add_argument("--no-standard", action="store_true",
                     help="skip the standard-training comparison (same model trained end to end on the same kernels)")
     ap.add_argument("--no-second-graph", action="store_true",
@@ -602,6 +604,15 @@ def main():
     w, ws, gen_s = build_workload(args.config, args.scale)
     if args.iteration_only:
         iteration_only(w, ws, args.iteration_only)
+        return
+    if args.standard_only:
+        sp = B.StandardProblem(w.aggr, args.standard_only, w.hidden, w.n_classes, w.lr, w.rowptr, w.colidx, w.features,
+                               w.labels, w.train_idx, w.val_idx, w.test_idx, ws, want_logits=False)
+        for _ in range(2):
+            B.retexo_standard_train(sp)
+        torch.cuda.synchronize()
+        r = sp.results()
+        print(json.dumps(dict(standard_only=args.standard_only, status=r["status"], loss=[float(x) for x in r["loss_history"]])))
         return
     R = args.iters or w.R
     prob = make_problem(w, ws, host=False, R=R)
