@@ -341,7 +341,7 @@ __global__ void __launch_bounds__(kGb64Threads) gat_bwd_dst64_kernel(GatBwdArgs 
 }
 
 template <int HD>
-__global__ void __launch_bounds__(kGb64Threads) gat_bwd_src64_kernel(GatBwdArgs a) {
+__global__ void __launch_bounds__(kGb64Threads, 5) gat_bwd_src64_kernel(GatBwdArgs a) {
     __shared__ __align__(16) float p_s[kGb64Warps][64];
     __shared__ float red[kGb64Warps][kWarp][65];
     __shared__ float sm_part[kGb64Warps][2][64];
@@ -349,13 +349,15 @@ __global__ void __launch_bounds__(kGb64Threads) gat_bwd_src64_kernel(GatBwdArgs 
     const int64_t u = blockIdx.x * (int64_t)kGb64Warps + warp;
     const int nv = a.dim >> 2;
     constexpr int NH = 64 / HD;
-    float acc[64], ds[NH], su[NH];
-#pragma unroll
-    for (int c = 0; c < 64; ++c) acc[c] = 0.f;
+    // A lane's 64 column sums live in its own row of `red` (stride 65: no two lanes of a warp meet in a bank), not
+    // in registers: the registers go to the sixteen loads in flight, and more warps fit on an SM.
+    float* mine = red[warp][lane];
+    float ds[NH], su[NH];
 #pragma unroll
     for (int h = 0; h < NH; ++h) { ds[h] = 0.f; su[h] = 0.f; }
     for (int c = lane; c < 64; c += kWarp) p_s[warp][c] = (u < a.n && c < a.dim) ? a.p[u * a.ldp + c] : 0.f;
     __syncwarp();
+    bool first = true;                              // nothing stored in `mine` yet
     if (u < a.n) {
 #pragma unroll
         for (int h = 0; h < NH; ++h) if (h < a.heads) su[h] = a.s[u * a.heads + h];
@@ -364,12 +366,13 @@ __global__ void __launch_bounds__(kGb64Threads) gat_bwd_src64_kernel(GatBwdArgs 
         int64_t total = deg + (a.self_loop ? 1 : 0);
         if (total >= kGbHubEntries) {               // a hub row: its sums come from gat_bwd_src64_hub_kernel
             const float* hs = a.hub_sum + (int64_t)a.hub_pos[u] * 72;
+#pragma unroll 8
+            for (int c = 0; c < 64; ++c) mine[c] = lane == 0 ? hs[c] : 0.f;
             if (lane == 0) {
-#pragma unroll
-                for (int c = 0; c < 64; ++c) acc[c] = hs[c];
 #pragma unroll
                 for (int h = 0; h < NH; ++h) ds[h] = hs[64 + h];
             }
+            first = false;
             total = 0;
         }
         for (int64_t e0 = 0; e0 < total; e0 += kWarp) {
@@ -396,19 +399,29 @@ __global__ void __launch_bounds__(kGb64Threads) gat_bwd_src64_kernel(GatBwdArgs 
                     ds[h] = fmaf(alpha[h] * (z > 0.f ? 1.f : a.slope), dalpha[h] - st.z, ds[h]);
                 }
             }
+            if (first) {
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const float al = alpha[(4 * i) / HD];
-                acc[4 * i] = fmaf(al, g[i].x, acc[4 * i]);
-                acc[4 * i + 1] = fmaf(al, g[i].y, acc[4 * i + 1]);
-                acc[4 * i + 2] = fmaf(al, g[i].z, acc[4 * i + 2]);
-                acc[4 * i + 3] = fmaf(al, g[i].w, acc[4 * i + 3]);
+                for (int i = 0; i < 16; ++i) {
+                    const float al = alpha[(4 * i) / HD];
+                    mine[4 * i] = al * g[i].x; mine[4 * i + 1] = al * g[i].y;
+                    mine[4 * i + 2] = al * g[i].z; mine[4 * i + 3] = al * g[i].w;
+                }
+                first = false;
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float al = alpha[(4 * i) / HD];
+                    mine[4 * i] = fmaf(al, g[i].x, mine[4 * i]); mine[4 * i + 1] = fmaf(al, g[i].y, mine[4 * i + 1]);
+                    mine[4 * i + 2] = fmaf(al, g[i].z, mine[4 * i + 2]); mine[4 * i + 3] = fmaf(al, g[i].w, mine[4 * i + 3]);
+                }
             }
         }
     }
+    if (first) {
+#pragma unroll 8
+        for (int c = 0; c < 64; ++c) mine[c] = 0.f;
+    }
     // the lanes' partial rows are added in lane order; the lanes' ds in a shuffle tree
-#pragma unroll
-    for (int c = 0; c < 64; ++c) red[warp][lane][c] = acc[c];
 #pragma unroll
     for (int h = 0; h < NH; ++h) ds[h] = warp_sum(ds[h]);
     __syncwarp();

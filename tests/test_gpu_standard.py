@@ -41,7 +41,7 @@ def _problem(w, ws, R, **kw):
                                w.train_idx, w.val_idx, w.test_idx, ws, **kw)
 
 
-@pytest.mark.parametrize("cfg,scale", [(1, 0.5), (2, 0.1), (4, 0.01), (5, 0.002)])
+@pytest.mark.parametrize("cfg,scale", [(1, 0.5), (2, 0.1), (4, 0.01), (5, 0.002), (1, 1.0), (4, 0.05), (5, 0.02)])
 def test_one_iteration_matches_the_checker(cfg, scale):
     w, ws = _workload(cfg, scale)
     prob = _problem(w, ws, 1, want_grad=True)
