@@ -499,7 +499,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
                              b.val_history + (size_t)(m - 1) * c.R};
         // With validation every iteration (or none) all iterations from the second on are the same six
         // launches with the same arguments: the second one is recorded as a graph, the rest replay it.
-        const bool uniform = work.own && c.R > 3 && (n_val == 0 || c.eval_every == 1) && !gat_train;
+        const bool uniform = work.own && c.R > 3 && (n_val == 0 || c.eval_every == 1);
         tail.decision = gat_train ? b.decision : nullptr;
         const int64_t ld_dx = ldp;
         // What a round that trains its aggregator adds to an iteration (Section 3.1: after the round's exchange
@@ -540,14 +540,20 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
             tail.iter = pending_it;
             tail.history_slot = b.val_history + (size_t)(m - 1) * c.R + (pending_it > 0 ? pending_it - 1 : 0);
             const EvalTail* riding = pending_it ? &tail : nullptr;
-            if (gat_train) {
+            // one iteration's launches (with a trained aggregator: projection, aggregation and batches before the
+            // per-node model's step, the attention's backward pass and update after it)
+            auto enqueue = [&](bool shadows_ready) -> int {
+                if (!gat_train)
+                    return mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot, nullptr,
+                                                 shadows_ready, riding, st, &dev);
                 RETEXO_TRY(gat_forward(b.att));
                 RETEXO_TRY(pack_batches());
                 if (!riding) RETEXO_CUDA_TRY(cudaMemsetAsync(b.decision, 0, sizeof(int32_t), st));
-                RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot, nullptr, it > 1,
-                                                 riding, st, &dev, b.dx, ld_dx));
-                RETEXO_TRY(gat_backward_and_update());
-            } else if (uniform && it >= 2) {
+                RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot, nullptr,
+                                                 shadows_ready, riding, st, &dev, b.dx, ld_dx));
+                return gat_backward_and_update();
+            };
+            if (uniform && it >= 2) {
                 // Iterations 2..R are the same launches (their iteration-dependent state lives on the device), so
                 // they are replayed from graphs: a chunk of kGraphIterations while that many remain (inside a
                 // graph consecutive kernels overlap their set-up with the predecessor's tail, across graph
@@ -556,9 +562,7 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
                     bool recorded = false;
                     if (cudaStreamBeginCapture(st, cudaStreamCaptureModeRelaxed) == cudaSuccess) {
                         int rc = RETEXO_OK;
-                        for (int i = 0; i < count && rc == RETEXO_OK; ++i)
-                            rc = mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot, nullptr,
-                                                       true, riding, st, &dev);
+                        for (int i = 0; i < count && rc == RETEXO_OK; ++i) rc = enqueue(true);
                         cudaGraph_t graph = nullptr;
                         const cudaError_t ended = cudaStreamEndCapture(st, &graph);
                         if (rc == RETEXO_OK && ended == cudaSuccess && graph &&
@@ -578,12 +582,10 @@ extern "C" int retexo_lmp_train(const retexo_lmp_config* cfg, const retexo_lmp_i
                     RETEXO_CUDA_TRY(cudaGraphLaunch(iteration.exec, st));
                 } else {      // no graph on this stream: plain launches
                     graphs_ok = false;
-                    RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot,
-                                                     nullptr, true, riding, st, &dev));
+                    RETEXO_TRY(enqueue(true));
                 }
             } else {
-                RETEXO_TRY(mlp_train_step_launch(plan, sb, &model, b.xtr16, ld_tr, true, b.y_tr, loss_slot,
-                                                 nullptr, it > 1, riding, st, &dev));
+                RETEXO_TRY(enqueue(it > 1));
             }
             it += done_now - 1;
             model.step += done_now - 1;
