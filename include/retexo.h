@@ -274,6 +274,14 @@ int retexo_embed(const retexo_mlp* model,
                  int32_t* pred_out, const int32_t* y, uint64_t* correct_out,
                  void* workspace, size_t workspace_bytes, void* stream);
 
+/* Packs rows of a fp32 matrix for the one exchange of a round (Section 3.4, sync_embeddings): dst[i] = src[idx[i]],
+ * dim columns each (idx: device, row indices into src; ld_src, ld_dst >= dim).  A worker of a sharded run calls it
+ * once per peer with the list of its owned rows that peer aggregates over, hands the packed rows to the transport
+ * (an all-to-all with per-peer counts), and aggregates over [owned rows | received rows] with retexo_aggregate on
+ * its local CSR.  Needs no workspace.  Errors: INVALID_ARG, CUDA. */
+int retexo_gather_rows(const float* src, int64_t ld_src, int32_t dim, const int32_t* idx, int64_t n_rows,
+                       float* dst, int64_t ld_dst, void* stream);
+
 /* ------------------------------------------------ cross-partition traffic */
 size_t retexo_cross_partition_workspace_size(int64_t n_nodes, int64_t n_edges, int32_t n_parts);
 

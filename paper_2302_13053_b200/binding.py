@@ -94,6 +94,7 @@ EXPORTS = ["retexo_status_string", "retexo_version", "retexo_validate_csr", "ret
            "retexo_cross_partition_workspace_size", "retexo_cross_partition_bytes",
            "retexo_cross_partition_static_scratch_bytes", "retexo_cross_partition_bytes_static",
            "retexo_data_volume", "retexo_lmp_workspace_size", "retexo_standard_workspace_size", "retexo_standard_train",
+           "retexo_gather_rows",
            "retexo_lmp_train"]
 
 
@@ -404,6 +405,19 @@ def retexo_cross_partition_bytes_static(rowptr: torch.Tensor, colidx: torch.Tens
                                                    C.c_void_p(base + 24), C.c_void_p(base + 16), None, None,
                                                    _stream())
     _check(rc, "retexo_cross_partition_bytes_static")
+
+
+def retexo_gather_rows(src: torch.Tensor, idx: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """out[i] = src[idx[i]] for a fp32 matrix src (rows contiguous) and int32 row indices idx, on the device."""
+    assert src.dtype == torch.float32 and idx.dtype == torch.int32 and src.stride(1) == 1
+    n, dim = idx.numel(), src.shape[1]
+    if out is None:
+        out = torch.empty((n, dim), dtype=torch.float32, device=src.device)
+    assert out.shape[0] >= n and out.shape[1] == dim and out.stride(1) == 1
+    rc = lib().retexo_gather_rows(_ptr(src), C.c_int64(src.stride(0)), C.c_int32(dim), _ptr(idx), C.c_int64(n), _ptr(out),
+                                  C.c_int64(out.stride(0)), _stream())
+    _check(rc, "retexo_gather_rows")
+    return out
 
 
 def pack_theta(w: Dict[str, np.ndarray], layer_norm: bool = False, batch_norm: bool = False) -> np.ndarray:

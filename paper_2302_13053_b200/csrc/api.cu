@@ -41,3 +41,31 @@ extern "C" int retexo_data_volume(int32_t K, const int64_t* H, const int64_t* L,
     out->gamma = den > 0.0 ? (out->standard_lt + out->standard_reduce) / den : 0.0;
     return RETEXO_OK;
 }
+
+// dst[i][0 .. dim) = src[idx[i]][0 .. dim): the owned rows a peer needs, packed for the round's one exchange.
+// A warp moves a row; 16-byte pieces where both sides allow.
+__global__ void __launch_bounds__(256) gather_rows_f32_kernel(const float* __restrict__ src, int64_t ld_src, int32_t dim,
+                                                              const int32_t* __restrict__ idx, int64_t n_rows,
+                                                              float* __restrict__ dst, int64_t ld_dst, int vec) {
+    const int lane = threadIdx.x & 31;
+    const int64_t i = blockIdx.x * 8ll + (threadIdx.x >> 5);
+    if (i >= n_rows) return;
+    const float* s = src + (int64_t)idx[i] * ld_src;
+    float* d = dst + i * ld_dst;
+    if (vec) {
+        for (int c = lane; c < dim / 4; c += 32) reinterpret_cast<float4*>(d)[c] = __ldg(reinterpret_cast<const float4*>(s) + c);
+    } else {
+        for (int c = lane; c < dim; c += 32) d[c] = s[c];
+    }
+}
+
+extern "C" int retexo_gather_rows(const float* src, int64_t ld_src, int32_t dim, const int32_t* idx, int64_t n_rows,
+                                  float* dst, int64_t ld_dst, void* stream) {
+    if (n_rows < 0 || dim <= 0 || ld_src < dim || ld_dst < dim) return RETEXO_ERR_INVALID_ARG;
+    if (n_rows == 0) return RETEXO_OK;
+    if (!src || !idx || !dst) return RETEXO_ERR_INVALID_ARG;
+    const int vec = dim % 4 == 0 && ld_src % 4 == 0 && ld_dst % 4 == 0 && retexo::aligned_to(src, 16) && retexo::aligned_to(dst, 16);
+    gather_rows_f32_kernel<<<(unsigned)((n_rows + 7) / 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(src, ld_src, dim, idx, n_rows,
+                                                                                                      dst, ld_dst, vec);
+    return retexo::launch_status();
+}

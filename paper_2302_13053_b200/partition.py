@@ -116,3 +116,58 @@ def exchange_rows(plan: RankPlan, q_owned: np.ndarray, dist) -> np.ndarray:
 def exchanged_bytes(plan: RankPlan, dim: int, elem_bytes: int = 4) -> int:
     """Bytes this rank receives in one round of width `dim` (summed over ranks: boundary_pairs x dim x elem_bytes)."""
     return plan.n_halo * dim * elem_bytes
+
+
+# ---------------------------------------------------------------- device data plane
+class DeviceRound:
+    """What a rank keeps on its GPU to run the aggregation of a sharded round: the local CSR over
+    [owned rows | received rows], the local indices of the owned rows each peer needs, and a buffer for
+    [owned | received] rows.  The exchange writes into this GPU's own memory; the aggregation kernel then reads
+    local memory only (no kernel reads a peer's memory)."""
+
+    def __init__(self, plan: RankPlan, device="cuda"):
+        import torch
+        self.plan = plan
+        self.device = torch.device(device)
+        self.rowptr = torch.from_numpy(plan.rowptr.astype(np.int64)).to(self.device)
+        self.colidx = torch.from_numpy(plan.colidx.astype(np.int32)).to(self.device)
+        send = np.concatenate([ids - plan.lo for ids in plan.send_ids]) if plan.world > 1 else np.zeros(0, np.int64)
+        self.send_local = torch.from_numpy(send.astype(np.int32)).to(self.device)      # peer by peer
+        self.n_send = int(send.shape[0])
+
+    def exchange(self, q_owned, dist=None):
+        """The round's one exchange on device tensors.  q_owned: fp32 [n_owned x d] on this GPU.  Returns fp32
+        [n_owned + n_halo, d]: the owned rows, then the received rows peer by peer.  With the `nccl` backend the
+        all-to-all moves device memory directly; with any other backend (`gloo`: tests on one GPU) the packed rows
+        are staged through host memory."""
+        import torch
+        from . import binding as B
+        p = self.plan
+        d = q_owned.shape[1]
+        q_local = torch.empty((p.n_owned + p.n_halo, d), dtype=torch.float32, device=self.device)
+        q_local[:p.n_owned].copy_(q_owned)
+        if p.world == 1:
+            return q_local
+        send = B.retexo_gather_rows(q_owned, self.send_local) if self.n_send else \
+            torch.empty((0, d), dtype=torch.float32, device=self.device)
+        recv = q_local[p.n_owned:]
+        if dist.get_backend() == "nccl":
+            dist.all_to_all_single(recv, send, output_split_sizes=p.recv_counts(), input_split_sizes=p.send_counts())
+        else:
+            recv_h = torch.empty((p.n_halo, d), dtype=torch.float32)
+            dist.all_to_all_single(recv_h, send.cpu(), output_split_sizes=p.recv_counts(), input_split_sizes=p.send_counts())
+            recv.copy_(recv_h)
+        return q_local
+
+    def aggregate(self, aggr: int, q_local, gat=None, want_bf16: bool = False):
+        """AGGR (+ COMBINE) over [owned | received] rows with the library's kernel; returns the owned rows' part
+        (fp32 [n_owned x width], and the bf16 copy if asked)."""
+        from . import binding as B
+        out, out16 = B.retexo_aggregate(aggr, self.rowptr, self.colidx, q_local, gat=gat, want_bf16=want_bf16)
+        n = self.plan.n_owned
+        return (out[:n], out16[:n]) if want_bf16 else out[:n]
+
+
+def sharded_aggregate(round_: DeviceRound, aggr: int, q_owned, dist=None, gat=None):
+    """One message-passing round of a sharded run on this rank: exchange, then local aggregation."""
+    return round_.aggregate(aggr, round_.exchange(q_owned, dist), gat=gat)
